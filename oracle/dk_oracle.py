@@ -1,0 +1,349 @@
+"""fp64 CPU oracle for DarKnight's masked linear-algebra path.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+path computes, written from the paper; it shares no code with the CUDA
+library and must never be imported by it.  Only the tests, the smoke check
+and the benchmark's CPU-baseline leg call it.
+
+Every function works on float64 NumPy arrays in the paper's logical shapes
+(samples first, then channels, then rows, columns) and follows the paper's
+steps in order, without blocking or fusion:
+
+* ``encode``            Eq. 1, plus the redundant encoding of Section 4.4
+* ``linear``            the bilinear operation <W, x> (matrix product or
+                        cross-correlation with zero padding), Section 4.1
+* ``decode``            Eq. 2: Y = Y_bar . A^{-1}; the W.r column is returned
+                        separately and dropped by the caller
+* ``verify``            Section 4.4: the (K+2)-th equation is re-predicted from
+                        the decoded unknowns and compared with what came back
+* ``derive_B``          the unique B that satisfies Eq. 5 for given A, Gamma
+* ``wgrad_masked``      Eq. 4 and Eq. 6, summed over virtual batches
+* ``linear_plain`` / ``wgrad_plain``   the unmasked definitions (Eq. 3) that
+                        the method must reproduce exactly in exact arithmetic
+
+Coefficient convention: ``C[g, i, k]`` = coefficient of source k (k < K the
+private inputs, k = K the noise) in encoding i; rows 0..K are the decodable
+square part C_sq (the transpose of the paper's A), row K+1 is the redundant
+row.
+
+Pins (see the ``-m "not gpu"`` tests): brute-force loops on tiny inputs, a
+library float64 convolution and its autograd, the decode/encode round trip
+against the plain definition, closed forms for K = 1, the exact residual
+change n[i]*Delta under a single injected fault, and the Eq. 5 residual.
+Parity unpinned: the numerical threshold ``tau`` of ``verify`` and its
+noise-scale normaliser are constants of this implementation, not the paper's
+(the paper compares exactly in a finite field); nothing outside this file
+fixes them.
+"""
+from __future__ import annotations
+
+from typing import Dict, Optional, Tuple
+
+import numpy as np
+
+F64 = np.float64
+
+
+# ---------------------------------------------------------------------------
+# small dense linear algebra, written out (no library inverse)
+# ---------------------------------------------------------------------------
+def invert(M: np.ndarray) -> np.ndarray:
+    """Gauss-Jordan inverse with partial pivoting of a small square matrix."""
+    n = M.shape[0]
+    a = np.array(M, dtype=F64)
+    inv = np.eye(n, dtype=F64)
+    for col in range(n):
+        piv = col + int(np.argmax(np.abs(a[col:, col])))
+        if a[piv, col] == 0.0:
+            raise ZeroDivisionError("singular coefficient matrix")
+        if piv != col:
+            a[[col, piv]] = a[[piv, col]]
+            inv[[col, piv]] = inv[[piv, col]]
+        p = a[col, col]
+        a[col] /= p
+        inv[col] /= p
+        for row in range(n):
+            if row != col and a[row, col] != 0.0:
+                f = a[row, col]
+                a[row] -= f * a[col]
+                inv[row] -= f * inv[col]
+    return inv
+
+
+def null_vector(Cg: np.ndarray) -> np.ndarray:
+    """n with n^T C = 0 and n[K+1] = 1 for a (K+2)x(K+1) block (Section 4.4).
+
+    Any consistency check between two (K+1)-subsets of the K+2 equations is a
+    multiple of n . y_bar, because the left null space of C has dimension one.
+    """
+    K1 = Cg.shape[1]
+    c = np.asarray(Cg, dtype=F64)
+    n = np.empty(K1 + 1, dtype=F64)
+    n[:K1] = -(c[K1] @ invert(c[:K1]))
+    n[K1] = 1.0
+    return n
+
+
+# ---------------------------------------------------------------------------
+# Eq. 1 / Section 4.4: encoding
+# ---------------------------------------------------------------------------
+def encode(x: np.ndarray, r: np.ndarray, C: np.ndarray) -> np.ndarray:
+    """x_bar[g*(K+2)+i] = sum_k C[g,i,k] x[g*K+k] + C[g,i,K] r[g]  (Eq. 1)."""
+    G, E, K1 = C.shape
+    K = K1 - 1
+    x = np.asarray(x, dtype=F64)
+    r = np.asarray(r, dtype=F64)
+    c = np.asarray(C, dtype=F64)
+    out = np.zeros((G * E,) + x.shape[1:], dtype=F64)
+    for g in range(G):
+        for i in range(E):
+            acc = c[g, i, K] * r[g]
+            for k in range(K):
+                acc = acc + c[g, i, k] * x[g * K + k]
+            out[g * E + i] = acc
+    return out
+
+
+# ---------------------------------------------------------------------------
+# the bilinear operation <W, x>
+# ---------------------------------------------------------------------------
+def _pad(x: np.ndarray, pad: int) -> np.ndarray:
+    if pad == 0:
+        return x
+    return np.pad(x, ((0, 0), (0, 0), (pad, pad), (pad, pad)))
+
+
+def linear(W: np.ndarray, x: np.ndarray, stride: int = 1, pad: int = 0) -> np.ndarray:
+    """<W, x> per sample: x @ W^T for 2-D x, else zero-padded cross-correlation
+    y[n,o,p,q] = sum_{c,u,v} W[o,c,u,v] x[n,c,p*stride+u-pad,q*stride+v-pad]."""
+    W = np.asarray(W, dtype=F64)
+    x = np.asarray(x, dtype=F64)
+    if x.ndim == 2:
+        return x @ W.T
+    n, cin, h, w = x.shape
+    cout, _, kh, kw = W.shape
+    ho = (h + 2 * pad - kh) // stride + 1
+    wo = (w + 2 * pad - kw) // stride + 1
+    xp = _pad(x, pad)
+    y = np.zeros((n, cout, ho, wo), dtype=F64)
+    for u in range(kh):
+        for v in range(kw):
+            win = xp[:, :, u:u + (ho - 1) * stride + 1:stride, v:v + (wo - 1) * stride + 1:stride]
+            # sum over channels c: y[n,o,p,q] += W[o,c,u,v] * win[n,c,p,q]
+            y += np.tensordot(win, W[:, :, u, v], axes=([1], [1])).transpose(0, 3, 1, 2)
+    return y
+
+
+def linear_at(W: np.ndarray, x_one: np.ndarray, co: int, oh: int, ow: int,
+              stride: int = 1, pad: int = 0) -> float:
+    """One output element of ``linear`` for one sample (x_one has no batch axis)."""
+    W = np.asarray(W, dtype=F64)
+    x_one = np.asarray(x_one, dtype=F64)
+    if x_one.ndim == 1:
+        return float(W[co] @ x_one)
+    cin, h, w = x_one.shape
+    _, _, kh, kw = W.shape
+    acc = 0.0
+    for u in range(kh):
+        ih = oh * stride + u - pad
+        if ih < 0 or ih >= h:
+            continue
+        for v in range(kw):
+            iw = ow * stride + v - pad
+            if iw < 0 or iw >= w:
+                continue
+            acc += float(W[co, :, u, v] @ x_one[:, ih, iw])
+    return acc
+
+
+def linear_plain(W, x, stride=1, pad=0):
+    """The result the method must reproduce: y^(k) = <W, x^(k)> (Section 4.1)."""
+    return linear(W, x, stride, pad)
+
+
+# ---------------------------------------------------------------------------
+# Eq. 2: decoding
+# ---------------------------------------------------------------------------
+def decode(ybar: np.ndarray, C: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Solve C_sq . [y^(1..K); z] = y_bar^(1..K+1) per group and element.
+
+    Because y_bar^(i) = sum_k C[i,k] <W,x^(k)> + C[i,K] <W,r>, stacking the
+    first K+1 encodings gives Y_bar = C_sq . Y (the transpose of Eq. 2), hence
+    Y = C_sq^{-1} . Y_bar.  Returns (y [G*K,...], z [G,...]) with z = <W, r>.
+    """
+    G, E, K1 = C.shape
+    K = K1 - 1
+    ybar = np.asarray(ybar, dtype=F64)
+    y = np.zeros((G * K,) + ybar.shape[1:], dtype=F64)
+    z = np.zeros((G,) + ybar.shape[1:], dtype=F64)
+    for g in range(G):
+        cinv = invert(np.asarray(C[g, :K1], dtype=F64))
+        for k in range(K1):
+            acc = 0.0
+            for i in range(K1):
+                acc = acc + cinv[k, i] * ybar[g * E + i]
+            if k < K:
+                y[g * K + k] = acc
+            else:
+                z[g] = acc
+    return y, z
+
+
+# ---------------------------------------------------------------------------
+# Section 4.4: integrity
+# ---------------------------------------------------------------------------
+def verify(ybar: np.ndarray, C: np.ndarray, y: np.ndarray, z: np.ndarray,
+           tau: float = 1e-4) -> Dict[str, np.ndarray]:
+    """Re-predict the redundant equation from the decoded unknowns.
+
+    rho[g] = y_bar^(K+2) - sum_k C[K+1,k] y^(k) - C[K+1,K] z.  An element is
+    flagged iff |rho| > tau * sum_i |n_i| |y_bar^(i)| where n is the null
+    vector of the group's C.  The final comparison is taken in float32 (the
+    precision in which the GPU takes it).  Returns per-element arrays
+    ``rho``, ``scale``, ``ratio`` = |rho|/scale and boolean ``flags`` of shape
+    [G, ...].
+    """
+    G, E, K1 = C.shape
+    K = K1 - 1
+    ybar = np.asarray(ybar, dtype=F64)
+    rho = np.zeros((G,) + ybar.shape[1:], dtype=F64)
+    scale = np.zeros_like(rho)
+    for g in range(G):
+        c = np.asarray(C[g], dtype=F64)
+        pred = c[K + 1, K] * z[g]
+        for k in range(K):
+            pred = pred + c[K + 1, k] * y[g * K + k]
+        rho[g] = ybar[g * E + K + 1] - pred
+        n = null_vector(c)
+        s = 0.0
+        for i in range(E):
+            s = s + abs(n[i]) * np.abs(ybar[g * E + i])
+        scale[g] = s
+    with np.errstate(divide="ignore", invalid="ignore"):
+        ratio = np.where(scale > 0, np.abs(rho) / scale, 0.0)
+    flags = np.abs(rho).astype(np.float32) > np.float32(tau) * scale.astype(np.float32)
+    return {"rho": rho, "scale": scale, "ratio": ratio, "flags": flags}
+
+
+def verdict(flags: np.ndarray, ratio: np.ndarray) -> Dict[str, float]:
+    """Summary of a verify pass over arrays given in the memory order of the
+    output tensor: ok, n_flagged, first flagged flat index (-1 if none) and
+    the largest ratio."""
+    flat = np.flatnonzero(np.asarray(flags).reshape(-1))
+    return {"ok": int(flat.size == 0), "n_flagged": int(flat.size),
+            "first_index": int(flat[0]) if flat.size else -1,
+            "max_ratio": float(np.max(ratio)) if ratio.size else 0.0}
+
+
+# ---------------------------------------------------------------------------
+# Eq. 4-6: weight gradient on encoded activations
+# ---------------------------------------------------------------------------
+def derive_B(Cg: np.ndarray, gamma_g: np.ndarray) -> np.ndarray:
+    """B in R^{(K+1) x K} with B^T . Gamma . A^T = [I_K | 0]  (Eq. 5).
+
+    With A square and invertible the solution is unique:
+    B = Gamma^{-1} . A^{-1} . [I_K; 0].  Since C_sq = A^T this reads
+    B[j,i] = (C_sq^{-1})[i,j] / gamma[j].
+    """
+    K1 = Cg.shape[1]
+    K = K1 - 1
+    cinv = invert(np.asarray(Cg[:K1], dtype=F64))
+    B = np.zeros((K1, K), dtype=F64)
+    for j in range(K1):
+        for i in range(K):
+            B[j, i] = cinv[i, j] / float(gamma_g[j])
+    return B
+
+
+def bilinear_wgrad(delta_one: np.ndarray, x_one: np.ndarray, kh: int = 1, kw: int = 1,
+                   stride: int = 1, pad: int = 0) -> np.ndarray:
+    """<delta, x> for one sample: the outer product for vectors, else
+    dW[o,c,u,v] = sum_{p,q} delta[o,p,q] x[c,p*stride+u-pad,q*stride+v-pad]."""
+    d = np.asarray(delta_one, dtype=F64)
+    x = np.asarray(x_one, dtype=F64)
+    if x.ndim == 1:
+        return np.outer(d, x)
+    cout, ho, wo = d.shape
+    cin = x.shape[0]
+    xp = _pad(x[None], pad)[0]
+    dW = np.zeros((cout, cin, kh, kw), dtype=F64)
+    for u in range(kh):
+        for v in range(kw):
+            win = xp[:, u:u + (ho - 1) * stride + 1:stride, v:v + (wo - 1) * stride + 1:stride]
+            dW[:, :, u, v] = np.tensordot(d, win, axes=([1, 2], [1, 2]))
+    return dW
+
+
+def wgrad_masked(delta: np.ndarray, xbar: np.ndarray, C: np.ndarray, gamma: np.ndarray,
+                 scale: float, kh: int = 1, kw: int = 1, stride: int = 1, pad: int = 0,
+                 xbar_rows_per_group: Optional[int] = None) -> np.ndarray:
+    """grad W = scale * sum_g sum_{j<=K} gamma[g,j] * Eq_j,
+    Eq_j = < sum_i B[j,i] delta^(i) , x_bar^(j) >   (Eq. 4, Eq. 6).
+
+    ``xbar`` holds ``xbar_rows_per_group`` encodings per group (K+2 as
+    produced by ``encode``, or K+1); only the first K+1 are used.
+    """
+    G, E, K1 = C.shape
+    K = K1 - 1
+    rows = E if xbar_rows_per_group is None else xbar_rows_per_group
+    delta = np.asarray(delta, dtype=F64)
+    xbar = np.asarray(xbar, dtype=F64)
+    total = None
+    for g in range(G):
+        B = derive_B(C[g], gamma[g])
+        for j in range(K1):
+            dbar = 0.0
+            for i in range(K):
+                dbar = dbar + B[j, i] * delta[g * K + i]
+            eq_j = bilinear_wgrad(dbar, xbar[g * rows + j], kh, kw, stride, pad)
+            term = float(gamma[g, j]) * eq_j
+            total = term if total is None else total + term
+    return scale * total
+
+
+def wgrad_plain(delta: np.ndarray, x: np.ndarray, scale: float, kh: int = 1, kw: int = 1,
+                stride: int = 1, pad: int = 0) -> np.ndarray:
+    """grad W = scale * sum_b <delta^(b), x^(b)>  (Eq. 3)."""
+    total = None
+    for b in range(x.shape[0]):
+        t = bilinear_wgrad(delta[b], x[b], kh, kw, stride, pad)
+        total = t if total is None else total + t
+    return scale * total
+
+
+def wgrad_plain_at(delta: np.ndarray, x: np.ndarray, scale: float, co: int, ci: int,
+                   u: int = 0, v: int = 0, stride: int = 1, pad: int = 0) -> float:
+    """One element of ``wgrad_plain``."""
+    d = np.asarray(delta, dtype=F64)
+    x = np.asarray(x, dtype=F64)
+    if x.ndim == 2:
+        return scale * float(d[:, co] @ x[:, ci])
+    _, _, ho, wo = d.shape
+    xp = _pad(x[:, ci:ci + 1], pad)[:, 0]
+    win = xp[:, u:u + (ho - 1) * stride + 1:stride, v:v + (wo - 1) * stride + 1:stride]
+    return scale * float(np.sum(d[:, co] * win))
+
+
+# ---------------------------------------------------------------------------
+# the whole masked forward, step by step
+# ---------------------------------------------------------------------------
+def masked_forward(W, x, r, C, stride=1, pad=0, tau=1e-4, fault=None, bias=None):
+    """encode -> linear on K+2 encodings -> (optional fault) -> decode -> verify.
+
+    ``fault`` = (row of y_bar, index tuple within that row, Delta) models an
+    accelerator that returns one wrong value (threat model, Section 3).
+    Returns dict with xbar, ybar, y, z and the verify arrays.
+    """
+    xbar = encode(x, r, C)
+    ybar = linear(W, xbar, stride, pad)
+    if fault is not None:
+        row, idx, dlt = fault
+        ybar[(row,) + tuple(idx)] += dlt
+    y, z = decode(ybar, C)
+    chk = verify(ybar, C, y, z, tau)
+    if bias is not None:
+        b = np.asarray(bias, dtype=F64)
+        y = y + (b if y.ndim == 2 else b[None, :, None, None])
+    out = {"xbar": xbar, "ybar": ybar, "y": y, "z": z}
+    out.update(chk)
+    return out
