@@ -1,0 +1,176 @@
+/*
+ * dk.h - C ABI of libdk: DarKnight's masked linear-algebra path on one GPU.
+ *
+ * A virtual batch of K private inputs plus one noise tensor is mixed by a
+ * small coefficient matrix (Eq. 1), the dense linear layer runs on the
+ * encoded inputs, the outputs are decoded with the inverse coefficients
+ * (Eq. 2) and checked against one redundant equation (Section 4.4); the
+ * weight gradient is computed on the stored encodings and decoded with the
+ * (B, Gamma) coefficients of Eq. 4-6.
+ *
+ * General conventions
+ *  - Every entry point returns a dk_status and never throws or exits.
+ *  - All tensors are fp32, contiguous, 16-byte aligned DEVICE pointers owned
+ *    by the caller.  Coefficient arrays (C, gamma) are small HOST pointers,
+ *    read before the call returns.
+ *  - Calls are asynchronous on the CUDA stream passed as `stream`
+ *    (a cudaStream_t cast to void*, NULL = default stream).  Outputs and the
+ *    dk_verdict are valid after that stream is synchronised.
+ *  - A batch holds G virtual batches ("groups") of K consecutive samples.
+ *    Sample tensors are stored row by row: x[G*K][n_in], r[G][n_in],
+ *    xbar[G*(K+2)][n_in], ybar[G*(K+2)][n_out], y[G*K][n_out].
+ *    For DK_CONV2D one row is an image; with layout DK_NHWC it is stored
+ *    [h][w][channels] and weights are [cout][kh][kw][cin]; with DK_NCHW it
+ *    is [channels][h][w] and weights are [cout][cin][kh][kw].  For DK_FC a
+ *    row is a vector of cin values and W is [cout][cin].
+ *  - Coefficients: C[g][i][k], g < G, i < K+2, k < K+1, is the weight of
+ *    source k (k < K: private input k of the group, k = K: the noise) in
+ *    encoding i.  Rows 0..K are the square, invertible part used for
+ *    decoding (the transpose of the paper's A in X_bar = X.A); row K+1 is
+ *    the redundant encoding used only by the integrity check.
+ *  - An integrity violation is a RESULT (dk_verdict.ok = 0), not an error:
+ *    the call still returns DK_OK.
+ *  - The library allocates only small per-context buffers in dk_create.
+ *    Large scratch memory is provided by the caller through
+ *    dk_set_workspace (size from dk_workspace_bytes).
+ *  - A context is not thread-safe, and calls that share a context but run
+ *    on different streams race on its scratch buffers.
+ */
+#ifndef DK_H_
+#define DK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DK_API __attribute__((visibility("default")))
+#else
+#define DK_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DK_OK = 0,
+  DK_ERR_INVALID_ARG = 1,  /* NULL pointer, misaligned pointer, bad enum          */
+  DK_ERR_SHAPE = 2,        /* geometry out of the supported range                 */
+  DK_ERR_SINGULAR = 3,     /* a group's square coefficient block is not invertible */
+  DK_ERR_WORKSPACE = 4,    /* workspace missing or too small                      */
+  DK_ERR_CUDA = 5,         /* a CUDA runtime/driver call failed                   */
+  DK_ERR_TIMEOUT = 6,      /* a bounded device-side wait expired                  */
+  DK_ERR_UNSUPPORTED = 7   /* valid request that this build cannot serve          */
+} dk_status;
+
+enum { DK_FC = 0, DK_CONV2D = 1 };
+enum { DK_NHWC = 0, DK_NCHW = 1 };
+/* Arithmetic of the dense contraction.  DK_TF32X3 (default) runs on the
+ * tensor cores with each fp32 operand split into two TF32 terms and three
+ * products kept (error ~2^-22 per product); DK_FP32_SIMT uses plain fp32 FMAs
+ * and accepts every geometry.  A request the tensor-core path cannot serve
+ * (see dk_linear_fwd) is executed by the SIMT path. */
+enum { DK_PREC_DEFAULT = 0, DK_TF32X3 = 1, DK_FP32_SIMT = 2 };
+
+#define DK_MAX_K 8
+
+typedef struct {
+  int32_t kind;       /* DK_FC | DK_CONV2D                                        */
+  int32_t layout;     /* DK_NHWC | DK_NCHW (ignored for DK_FC)                    */
+  int32_t cin, cout;  /* FC: input / output features                              */
+  int32_t h, w;       /* conv input height / width (FC: 1, 1)                     */
+  int32_t kh, kw;     /* filter size (FC: 1, 1)                                   */
+  int32_t stride, pad;/* same in both directions (FC: 1, 0)                       */
+  int32_t K, G;       /* virtual batch size (1..DK_MAX_K), number of groups       */
+  int32_t precision;  /* DK_PREC_DEFAULT | DK_TF32X3 | DK_FP32_SIMT               */
+  float tol;          /* integrity threshold tau; <= 0 selects 1e-4               */
+} dk_problem;
+
+/* Result of the integrity check, written to caller-provided device memory. */
+typedef struct {
+  int32_t ok;           /* 1 = every element consistent, 0 = at least one flagged */
+  uint32_t n_flagged;   /* number of flagged (group, output element) pairs        */
+  int64_t first_index;  /* smallest flagged g*n_out + e (e in memory order), or -1 */
+  float max_ratio;      /* max |rho| / sum_i |n_i||ybar_i| over all elements      */
+  int32_t status;       /* dk_status raised on the device (0 = none)              */
+} dk_verdict;
+
+/* Test hook modelling an accelerator that returns one wrong value (threat
+ * model, Section 3): delta is added to ybar[group*(K+2)+enc][out_index]
+ * before decoding. */
+typedef struct {
+  int32_t group, enc;
+  int64_t out_index;
+  float delta;
+} dk_fault;
+
+typedef struct dk_ctx dk_ctx;
+
+/* Create / destroy a context bound to CUDA device `device`.  The context owns
+ * a few MB of device and pinned host memory for coefficient upload. */
+DK_API dk_status dk_create(dk_ctx** ctx, int device);
+DK_API dk_status dk_destroy(dk_ctx* ctx);
+
+/* Human-readable name of a status code (static storage). */
+DK_API const char* dk_status_string(dk_status s);
+
+/* Scratch bytes the calls below may need for problem `p` (the maximum over
+ * all entry points), and registration of a caller-owned device buffer of at
+ * least that size (256-byte aligned).  The buffer must stay valid until it is
+ * replaced or the context is destroyed. */
+DK_API dk_status dk_workspace_bytes(const dk_problem* p, size_t* bytes);
+DK_API dk_status dk_set_workspace(dk_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* Eq. 1 and the redundant encoding of Section 4.4:
+ *   xbar[g*(K+2)+i][e] = sum_{k<K} C[g][i][k]*x[g*K+k][e] + C[g][i][K]*r[g][e]
+ * x: [G*K][n_in], r: [G][n_in]  ->  xbar: [G*(K+2)][n_in].  HBM-bound. */
+DK_API dk_status dk_encode(dk_ctx* ctx, const dk_problem* p, const float* x, const float* r,
+                           const float* C_host, float* xbar, void* stream);
+
+/* The bilinear operation <W, xbar> of Section 4.1 on all G*(K+2) encoded
+ * samples (the untrusted accelerator's role; knows nothing about C):
+ *   FC:   ybar[n][o] = sum_c W[o][c]*xbar[n][c]
+ *   conv: ybar[n][o][p][q] = sum_{c,u,v} W[o][c][u][v]*xbar[n][c][p*s+u-pad][q*s+v-pad]
+ * (cross-correlation, zero padding).  The tensor-core path serves DK_FC and
+ * DK_CONV2D/DK_NHWC with stride 1 and cin % 4 == 0 and needs the workspace;
+ * everything else runs on the SIMT path. */
+DK_API dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W,
+                               const float* xbar, float* ybar, void* stream);
+
+/* Eq. 2 and Section 4.4.  Per group and output element e:
+ *   [y_0..y_{K-1}, z] = C_sq^{-1} . [ybar_0..ybar_K]      (z = <W,r> is dropped)
+ *   rho = sum_i n[i]*ybar_i with n^T C = 0, n[K+1] = 1     (redundant equation)
+ *   flagged iff not (|rho| <= tau * sum_i |n[i]|*|ybar_i|)
+ * ybar: [G*(K+2)][n_out] -> y: [G*K][n_out]; bias[cout] (nullable) is added
+ * after decoding; *verdict (device) receives the summary.  HBM-bound. */
+DK_API dk_status dk_decode_verify(dk_ctx* ctx, const dk_problem* p, const float* ybar,
+                                  const float* C_host, const float* bias, float* y,
+                                  dk_verdict* verdict, void* stream);
+
+/* Encode -> linear -> decode -> verify for one layer in one call (flow steps
+ * 3-6 of Section 3.1 without leaving the device).  xbar_save (nullable)
+ * receives all K+2 encodings per group, [G*(K+2)][n_in], for later use by
+ * dk_linear_bwd_wgrad (Section 6, "Encoded Data Storage").  fault (host
+ * pointer, nullable) injects one wrong accelerator output.  Needs the
+ * workspace. */
+DK_API dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W,
+                                  const float* x, const float* r, const float* C_host,
+                                  const float* bias, float* y, float* xbar_save,
+                                  dk_verdict* verdict, const dk_fault* fault, void* stream);
+
+/* Eq. 4-6 summed over the virtual batches of the batch (Section 6, "Large
+ * Batch Aggregation"):
+ *   B[j][i] = (C_sq^{-1})[i][j] / gamma[g][j]          (the unique B of Eq. 5)
+ *   dW = scale * sum_g sum_{j<=K} gamma[g][j] * < sum_i B[j][i]*delta[g*K+i], xbar[g*rows+j] >
+ * delta: [G*K][n_out]; xbar holds `xbar_rows` (K+1 or K+2) encodings per
+ * group of which the first K+1 are used; gamma_host: [G][K+1], non-zero;
+ * dW has the shape of W.  Needs the workspace. */
+DK_API dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* delta,
+                                     const float* xbar, int32_t xbar_rows, const float* C_host,
+                                     const float* gamma_host, float scale, float* dW,
+                                     void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DK_H_ */

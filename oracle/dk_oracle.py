@@ -197,9 +197,10 @@ def verify(ybar: np.ndarray, C: np.ndarray, y: np.ndarray, z: np.ndarray,
     """Re-predict the redundant equation from the decoded unknowns.
 
     rho[g] = y_bar^(K+2) - sum_k C[K+1,k] y^(k) - C[K+1,K] z.  An element is
-    flagged iff |rho| > tau * sum_i |n_i| |y_bar^(i)| where n is the null
-    vector of the group's C.  The final comparison is taken in float32 (the
-    precision in which the GPU takes it).  Returns per-element arrays
+    flagged iff NOT(|rho| <= tau * sum_i |n_i| |y_bar^(i)|) where n is the null
+    vector of the group's C (written this way so that a NaN returned by the
+    accelerator is flagged too).  The final comparison is taken in float32
+    (the precision in which the GPU takes it).  Returns per-element arrays
     ``rho``, ``scale``, ``ratio`` = |rho|/scale and boolean ``flags`` of shape
     [G, ...].
     """
@@ -221,7 +222,8 @@ def verify(ybar: np.ndarray, C: np.ndarray, y: np.ndarray, z: np.ndarray,
         scale[g] = s
     with np.errstate(divide="ignore", invalid="ignore"):
         ratio = np.where(scale > 0, np.abs(rho) / scale, 0.0)
-    flags = np.abs(rho).astype(np.float32) > np.float32(tau) * scale.astype(np.float32)
+    with np.errstate(invalid="ignore"):
+        flags = ~(np.abs(rho).astype(np.float32) <= np.float32(tau) * scale.astype(np.float32))
     return {"rho": rho, "scale": scale, "ratio": ratio, "flags": flags}
 
 

@@ -1,0 +1,209 @@
+"""Thin ctypes binding over libdk.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (see include/dk.h).
+Tensors are torch CUDA tensors (fp32, contiguous) used purely as device
+memory; coefficient matrices are NumPy float32 arrays on the host.  Nothing
+here computes: if libdk.so is missing, loading the library fails loudly,
+there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdk.so")
+
+DK_FC, DK_CONV2D = 0, 1
+DK_NHWC, DK_NCHW = 0, 1
+DK_PREC_DEFAULT, DK_TF32X3, DK_FP32_SIMT = 0, 1, 2
+STATUS_NAMES = ["DK_OK", "DK_ERR_INVALID_ARG", "DK_ERR_SHAPE", "DK_ERR_SINGULAR", "DK_ERR_WORKSPACE",
+                "DK_ERR_CUDA", "DK_ERR_TIMEOUT", "DK_ERR_UNSUPPORTED"]
+
+
+class DkError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{where} failed with {name}")
+
+
+class dk_problem(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("layout", ctypes.c_int32),
+                ("cin", ctypes.c_int32), ("cout", ctypes.c_int32),
+                ("h", ctypes.c_int32), ("w", ctypes.c_int32),
+                ("kh", ctypes.c_int32), ("kw", ctypes.c_int32),
+                ("stride", ctypes.c_int32), ("pad", ctypes.c_int32),
+                ("K", ctypes.c_int32), ("G", ctypes.c_int32),
+                ("precision", ctypes.c_int32), ("tol", ctypes.c_float)]
+
+
+class dk_verdict(ctypes.Structure):
+    _fields_ = [("ok", ctypes.c_int32), ("n_flagged", ctypes.c_uint32),
+                ("first_index", ctypes.c_int64), ("max_ratio", ctypes.c_float),
+                ("status", ctypes.c_int32)]
+
+
+class dk_fault(ctypes.Structure):
+    _fields_ = [("group", ctypes.c_int32), ("enc", ctypes.c_int32),
+                ("out_index", ctypes.c_int64), ("delta", ctypes.c_float)]
+
+
+VERDICT_BYTES = ctypes.sizeof(dk_verdict)
+_lib = None
+
+
+def _signatures():
+    vp, i32 = ctypes.c_void_p, ctypes.c_int32
+    pp = ctypes.POINTER(dk_problem)
+    return {
+        "dk_create": [ctypes.POINTER(vp), ctypes.c_int],
+        "dk_destroy": [vp],
+        "dk_status_string": [ctypes.c_int],
+        "dk_workspace_bytes": [pp, ctypes.POINTER(ctypes.c_size_t)],
+        "dk_set_workspace": [vp, vp, ctypes.c_size_t],
+        "dk_encode": [vp, pp, vp, vp, vp, vp, vp],
+        "dk_linear_fwd": [vp, pp, vp, vp, vp, vp],
+        "dk_decode_verify": [vp, pp, vp, vp, vp, vp, vp, vp],
+        "dk_masked_linear": [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(dk_fault), vp],
+        "dk_linear_bwd_wgrad": [vp, pp, vp, vp, i32, vp, vp, ctypes.c_float, vp, vp],
+    }
+
+
+EXPORTS = list(_signatures().keys())
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libdk.so (once).  Raises if the library has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2207_00083_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, argtypes in _signatures().items():
+            fn = getattr(L, name)
+            fn.argtypes = argtypes
+            fn.restype = ctypes.c_char_p if name == "dk_status_string" else ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def problem_from_spec(spec, layout: int = DK_NHWC, precision: int = DK_PREC_DEFAULT,
+                      tol: float = 0.0, G: Optional[int] = None) -> dk_problem:
+    """dk_problem for a ``synth.LayerSpec``-like object."""
+    kind = DK_FC if spec.kind == "fc" else DK_CONV2D
+    return dk_problem(kind, layout, spec.cin, spec.cout, spec.h, spec.w, spec.kh, spec.kw,
+                      spec.stride, spec.pad, spec.K, spec.G if G is None else G, precision, tol)
+
+
+def _dev(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise ValueError("expected a contiguous fp32 CUDA tensor")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _host(a: np.ndarray):
+    if not (isinstance(a, np.ndarray) and a.dtype == np.float32 and a.flags["C_CONTIGUOUS"]):
+        raise ValueError("expected a C-contiguous float32 NumPy array")
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise DkError(status, where)
+
+
+class Context:
+    """Owns a dk_ctx and (optionally) a torch-allocated workspace."""
+
+    def __init__(self, device: int = 0):
+        self._h = ctypes.c_void_p()
+        self._ws = None
+        torch.cuda.init()
+        _check(lib().dk_create(ctypes.byref(self._h), device), "dk_create")
+        self.device = device
+
+    def close(self):
+        if self._h:
+            lib().dk_destroy(self._h)
+            self._h = ctypes.c_void_p()
+            self._ws = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def handle(self):
+        return self._h
+
+    def workspace_bytes(self, p: dk_problem) -> int:
+        n = ctypes.c_size_t()
+        _check(lib().dk_workspace_bytes(ctypes.byref(p), ctypes.byref(n)), "dk_workspace_bytes")
+        return n.value
+
+    def ensure_workspace(self, p: dk_problem):
+        """Grows the torch-owned workspace to what `p` needs and registers it."""
+        need = self.workspace_bytes(p)
+        if self._ws is None or self._ws.numel() < need + 256:
+            self._ws = None
+            self._ws = torch.empty(need + 256, dtype=torch.uint8, device=f"cuda:{self.device}")
+        base = self._ws.data_ptr()
+        off = (-base) % 256
+        _check(lib().dk_set_workspace(self._h, ctypes.c_void_p(base + off), self._ws.numel() - off),
+               "dk_set_workspace")
+
+
+def new_verdict(device: int = 0) -> torch.Tensor:
+    """Device storage for one dk_verdict."""
+    return torch.zeros(VERDICT_BYTES, dtype=torch.uint8, device=f"cuda:{device}")
+
+
+def read_verdict(v: torch.Tensor) -> dict:
+    """Synchronising device->host read of a dk_verdict."""
+    raw = v.cpu().numpy().tobytes()
+    s = dk_verdict.from_buffer_copy(raw)
+    return {"ok": int(s.ok), "n_flagged": int(s.n_flagged), "first_index": int(s.first_index),
+            "max_ratio": float(s.max_ratio), "status": int(s.status)}
+
+
+def dk_encode(ctx: Context, p: dk_problem, x, r, C: np.ndarray, xbar):
+    _check(lib().dk_encode(ctx.handle, ctypes.byref(p), _dev(x), _dev(r), _host(C), _dev(xbar), _stream()),
+           "dk_encode")
+
+
+def dk_linear_fwd(ctx: Context, p: dk_problem, W, xbar, ybar):
+    _check(lib().dk_linear_fwd(ctx.handle, ctypes.byref(p), _dev(W), _dev(xbar), _dev(ybar), _stream()),
+           "dk_linear_fwd")
+
+
+def dk_decode_verify(ctx: Context, p: dk_problem, ybar, C: np.ndarray, bias, y, verdict):
+    _check(lib().dk_decode_verify(ctx.handle, ctypes.byref(p), _dev(ybar), _host(C), _dev(bias), _dev(y),
+                                  ctypes.c_void_p(verdict.data_ptr()), _stream()), "dk_decode_verify")
+
+
+def dk_masked_linear(ctx: Context, p: dk_problem, W, x, r, C: np.ndarray, bias, y, xbar_save, verdict,
+                     fault: Optional[dk_fault] = None):
+    fp = ctypes.byref(fault) if fault is not None else None
+    _check(lib().dk_masked_linear(ctx.handle, ctypes.byref(p), _dev(W), _dev(x), _dev(r), _host(C),
+                                  _dev(bias), _dev(y), _dev(xbar_save),
+                                  ctypes.c_void_p(verdict.data_ptr()), fp, _stream()), "dk_masked_linear")
+
+
+def dk_linear_bwd_wgrad(ctx: Context, p: dk_problem, delta, xbar, xbar_rows: int, C: np.ndarray,
+                        gamma: np.ndarray, scale: float, dW):
+    _check(lib().dk_linear_bwd_wgrad(ctx.handle, ctypes.byref(p), _dev(delta), _dev(xbar), xbar_rows,
+                                     _host(C), _host(gamma), ctypes.c_float(scale), _dev(dW), _stream()),
+           "dk_linear_bwd_wgrad")

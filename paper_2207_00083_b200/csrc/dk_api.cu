@@ -1,0 +1,392 @@
+// C-ABI entry points of libdk: argument checks, fp64 coefficient algebra on
+// the host, workspace carving and kernel dispatch.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "dk_internal.h"
+
+namespace dk {
+
+dk_status make_geom(const dk_problem* p, Geom* g) {
+  if (!p || !g) return DK_ERR_INVALID_ARG;
+  if (p->kind != DK_FC && p->kind != DK_CONV2D) return DK_ERR_INVALID_ARG;
+  if (p->layout != DK_NHWC && p->layout != DK_NCHW) return DK_ERR_INVALID_ARG;
+  if (p->precision < DK_PREC_DEFAULT || p->precision > DK_FP32_SIMT) return DK_ERR_INVALID_ARG;
+  if (p->K < 1 || p->K > DK_MAX_K || p->G < 1) return DK_ERR_SHAPE;
+  if (p->cin < 1 || p->cout < 1) return DK_ERR_SHAPE;
+  memset(g, 0, sizeof(*g));
+  g->kind = p->kind;
+  g->layout = (p->kind == DK_FC) ? DK_NHWC : p->layout;
+  g->cin = p->cin;
+  g->cout = p->cout;
+  g->K = p->K;
+  g->G = p->G;
+  g->E = p->K + 2;
+  g->precision = p->precision == DK_PREC_DEFAULT ? DK_TF32X3 : p->precision;
+  g->tol = p->tol > 0.f ? p->tol : 1e-4f;
+  if (p->kind == DK_FC) {
+    g->h = g->w = g->kh = g->kw = g->stride = 1;
+    g->pad = 0;
+  } else {
+    if (p->h < 1 || p->w < 1 || p->kh < 1 || p->kw < 1 || p->stride < 1 || p->pad < 0)
+      return DK_ERR_SHAPE;
+    if (p->kh > 16 || p->kw > 16) return DK_ERR_SHAPE;
+    g->h = p->h; g->w = p->w; g->kh = p->kh; g->kw = p->kw;
+    g->stride = p->stride; g->pad = p->pad;
+  }
+  int eh = g->h + 2 * g->pad - g->kh, ew = g->w + 2 * g->pad - g->kw;
+  if (eh < 0 || ew < 0) return DK_ERR_SHAPE;
+  g->ho = eh / g->stride + 1;
+  g->wo = ew / g->stride + 1;
+  g->n_in = (long long)g->cin * g->h * g->w;
+  g->n_out = (long long)g->cout * g->ho * g->wo;
+  long long kc = (long long)g->cin * g->kh * g->kw;
+  if (kc > (1LL << 30)) return DK_ERR_SHAPE;
+  g->kc = (int)kc;
+  if ((long long)g->G * g->E * g->n_in >= (1LL << 40) ||
+      (long long)g->G * g->E * g->n_out >= (1LL << 40))
+    return DK_ERR_SHAPE;
+  if ((long long)g->G * g->E * g->ho * g->wo >= (1LL << 31)) return DK_ERR_SHAPE;
+  if (g->layout == DK_NHWC) {
+    g->xs_c = 1; g->xs_w = g->cin; g->xs_h = (long long)g->cin * g->w;
+    g->ws_c = 1; g->ws_v = g->cin; g->ws_u = (long long)g->cin * g->kw; g->ws_o = kc;
+    g->ys_c = 1; g->ys_w = g->cout; g->ys_h = (long long)g->cout * g->wo;
+  } else {
+    g->xs_w = 1; g->xs_h = g->w; g->xs_c = (long long)g->h * g->w;
+    g->ws_v = 1; g->ws_u = g->kw; g->ws_c = (long long)g->kh * g->kw; g->ws_o = kc;
+    g->ys_w = 1; g->ys_h = g->wo; g->ys_c = (long long)g->ho * g->wo;
+  }
+  return DK_OK;
+}
+
+// Gauss-Jordan inverse with partial pivoting, n <= DK_MAX_K+1, fp64.
+static bool invert_small(const double* M, int n, double* inv) {
+  double a[(DK_MAX_K + 1) * (DK_MAX_K + 1)];
+  double amax = 0.0;
+  for (int i = 0; i < n * n; ++i) { a[i] = M[i]; amax = fmax(amax, fabs(M[i])); }
+  if (!(amax > 0.0) || !isfinite(amax)) return false;
+  for (int i = 0; i < n; ++i)
+    for (int j = 0; j < n; ++j) inv[i * n + j] = (i == j) ? 1.0 : 0.0;
+  for (int c = 0; c < n; ++c) {
+    int piv = c;
+    for (int r = c + 1; r < n; ++r)
+      if (fabs(a[r * n + c]) > fabs(a[piv * n + c])) piv = r;
+    double pv = a[piv * n + c];
+    if (!(fabs(pv) > 1e-10 * amax)) return false;
+    if (piv != c)
+      for (int j = 0; j < n; ++j) {
+        double t = a[c * n + j]; a[c * n + j] = a[piv * n + j]; a[piv * n + j] = t;
+        t = inv[c * n + j]; inv[c * n + j] = inv[piv * n + j]; inv[piv * n + j] = t;
+      }
+    double ip = 1.0 / pv;
+    for (int j = 0; j < n; ++j) { a[c * n + j] *= ip; inv[c * n + j] *= ip; }
+    for (int r = 0; r < n; ++r) {
+      if (r == c) continue;
+      double f = a[r * n + c];
+      if (f == 0.0) continue;
+      for (int j = 0; j < n; ++j) {
+        a[r * n + j] -= f * a[c * n + j];
+        inv[r * n + j] -= f * inv[c * n + j];
+      }
+    }
+  }
+  return true;
+}
+
+dk_status upload_coefficients(dk_ctx* ctx, const Geom& g, const float* C_host,
+                              const float* gamma_host, bool want_dec, bool want_mix,
+                              cudaStream_t st, CoefView* view) {
+  const int K = g.K, K1 = K + 1, E = K + 2, G = g.G;
+  const size_t n_enc = (size_t)G * E * K1, n_dec = (size_t)G * K * K1, n_nul = (size_t)G * E,
+               n_mix = (size_t)G * K1 * K;
+  const size_t total = n_enc + 2 * n_dec + n_nul + n_mix;
+  if (total * sizeof(float) > kCoefSlotBytes) return DK_ERR_SHAPE;
+  if (!C_host) return DK_ERR_INVALID_ARG;
+  if (want_mix && !gamma_host) return DK_ERR_INVALID_ARG;
+
+  int s = ctx->cur_slot;
+  ctx->cur_slot = (s + 1) % kCoefSlots;
+  if (ctx->slot_used[s]) DK_CUDA_CHECK(cudaEventSynchronize(ctx->slot_ev[s]));
+  float* h = reinterpret_cast<float*>(ctx->h_stage + (size_t)s * kCoefSlotBytes);
+  float* d = reinterpret_cast<float*>(ctx->d_stage + (size_t)s * kCoefSlotBytes);
+  float* h_enc = h;
+  float* h_dec = h_enc + n_enc;
+  float* h_decl = h_dec + n_dec;
+  float* h_nul = h_decl + n_dec;
+  float* h_mix = h_nul + n_nul;
+  memcpy(h_enc, C_host, n_enc * sizeof(float));
+  memset(h_dec, 0, (2 * n_dec + n_nul + n_mix) * sizeof(float));
+
+  if (want_dec || want_mix) {
+    double sq[(DK_MAX_K + 1) * (DK_MAX_K + 1)], inv[(DK_MAX_K + 1) * (DK_MAX_K + 1)];
+    for (int gi = 0; gi < G; ++gi) {
+      const float* Cg = C_host + (size_t)gi * E * K1;
+      for (int i = 0; i < K1 * K1; ++i) sq[i] = (double)Cg[i];
+      if (!invert_small(sq, K1, inv)) return DK_ERR_SINGULAR;
+      // decode rows: y_k = sum_i inv[k][i] ybar_i
+      for (int k = 0; k < K; ++k)
+        for (int i = 0; i < K1; ++i) {
+          double v = inv[k * K1 + i];
+          float hi = (float)v;
+          h_dec[((size_t)gi * K + k) * K1 + i] = hi;
+          h_decl[((size_t)gi * K + k) * K1 + i] = (float)(v - (double)hi);
+        }
+      // null vector: n[0..K] = -C[K+1] . C_sq^{-1}, n[K+1] = 1
+      for (int i = 0; i < K1; ++i) {
+        double acc = 0.0;
+        for (int k = 0; k < K1; ++k) acc += (double)Cg[(size_t)K1 * K1 + k] * inv[k * K1 + i];
+        h_nul[(size_t)gi * E + i] = (float)(-acc);
+      }
+      h_nul[(size_t)gi * E + K1] = 1.f;
+      if (want_mix) {
+        // Eq. 5: B[j][i] = inv[i][j] / gamma[j]; mixing weight gamma[j]*B[j][i]
+        for (int j = 0; j < K1; ++j) {
+          double gm = (double)gamma_host[(size_t)gi * K1 + j];
+          if (gm == 0.0 || !isfinite(gm)) return DK_ERR_INVALID_ARG;
+          for (int i = 0; i < K; ++i) {
+            double B = inv[i * K1 + j] / gm;
+            h_mix[((size_t)gi * K1 + j) * K + i] = (float)(gm * B);
+          }
+        }
+      }
+    }
+  }
+  DK_CUDA_CHECK(cudaMemcpyAsync(d, h, total * sizeof(float), cudaMemcpyHostToDevice, st));
+  DK_CUDA_CHECK(cudaEventRecord(ctx->slot_ev[s], st));
+  ctx->slot_used[s] = true;
+  view->enc = d;
+  view->dec = d + n_enc;
+  view->decl = view->dec + n_dec;
+  view->nul = view->decl + n_dec;
+  view->dmix = view->nul + n_nul;
+  return DK_OK;
+}
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct WsPlan {
+  size_t xbar, ybar, dtil, total;
+};
+
+static WsPlan plan_workspace(const Geom& g) {
+  WsPlan w;
+  size_t off = 0;
+  w.xbar = off; off += align_up((size_t)g.G * g.E * g.n_in * sizeof(float), 256);
+  w.ybar = off; off += align_up((size_t)g.G * g.E * g.n_out * sizeof(float), 256);
+  w.dtil = off; off += align_up((size_t)g.G * (g.K + 1) * g.n_out * sizeof(float), 256);
+  w.total = off;
+  return w;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+struct DeviceGuard {
+  int prev;
+  bool ok;
+  explicit DeviceGuard(int dev) : prev(-1), ok(false) {
+    if (cudaGetDevice(&prev) != cudaSuccess) return;
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) return;
+    ok = true;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (ok && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+}  // namespace dk
+
+using namespace dk;
+
+extern "C" {
+
+const char* dk_status_string(dk_status s) {
+  switch (s) {
+    case DK_OK: return "DK_OK";
+    case DK_ERR_INVALID_ARG: return "DK_ERR_INVALID_ARG";
+    case DK_ERR_SHAPE: return "DK_ERR_SHAPE";
+    case DK_ERR_SINGULAR: return "DK_ERR_SINGULAR";
+    case DK_ERR_WORKSPACE: return "DK_ERR_WORKSPACE";
+    case DK_ERR_CUDA: return "DK_ERR_CUDA";
+    case DK_ERR_TIMEOUT: return "DK_ERR_TIMEOUT";
+    case DK_ERR_UNSUPPORTED: return "DK_ERR_UNSUPPORTED";
+  }
+  return "DK_ERR_UNKNOWN";
+}
+
+dk_status dk_create(dk_ctx** out, int device) {
+  if (!out) return DK_ERR_INVALID_ARG;
+  *out = nullptr;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return DK_ERR_CUDA;
+  DeviceGuard dg(device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  dk_ctx* c = new (std::nothrow) dk_ctx();
+  if (!c) return DK_ERR_CUDA;
+  memset(c, 0, sizeof(*c));
+  c->device = device;
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+    delete c;
+    return DK_ERR_CUDA;
+  }
+  c->sm_count = sms;
+  bool ok = cudaMallocHost(&c->h_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
+            cudaMalloc(&c->d_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
+            cudaMalloc(&c->d_counters, 256) == cudaSuccess &&
+            cudaMemset(c->d_counters, 0, 256) == cudaSuccess;
+  for (int i = 0; ok && i < kCoefSlots; ++i)
+    ok = cudaEventCreateWithFlags(&c->slot_ev[i], cudaEventDisableTiming) == cudaSuccess;
+  if (ok) ok = tc_init(c) == DK_OK;
+  if (!ok) { dk_destroy(c); return DK_ERR_CUDA; }
+  *out = c;
+  return DK_OK;
+}
+
+dk_status dk_destroy(dk_ctx* c) {
+  if (!c) return DK_OK;
+  DeviceGuard dg(c->device);
+  cudaDeviceSynchronize();
+  tc_destroy(c);
+  for (int i = 0; i < kCoefSlots; ++i)
+    if (c->slot_ev[i]) cudaEventDestroy(c->slot_ev[i]);
+  if (c->h_stage) cudaFreeHost(c->h_stage);
+  if (c->d_stage) cudaFree(c->d_stage);
+  if (c->d_counters) cudaFree(c->d_counters);
+  delete c;
+  return DK_OK;
+}
+
+dk_status dk_workspace_bytes(const dk_problem* p, size_t* bytes) {
+  if (!bytes) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  *bytes = plan_workspace(g).total;
+  return DK_OK;
+}
+
+dk_status dk_set_workspace(dk_ctx* ctx, void* dev_ptr, size_t bytes) {
+  if (!ctx) return DK_ERR_INVALID_ARG;
+  if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255)) return DK_ERR_INVALID_ARG;
+  ctx->ws = dev_ptr;
+  ctx->ws_bytes = dev_ptr ? bytes : 0;
+  return DK_OK;
+}
+
+dk_status dk_encode(dk_ctx* ctx, const dk_problem* p, const float* x, const float* r,
+                    const float* C_host, float* xbar, void* stream) {
+  if (!ctx || !x || !r || !C_host || !xbar) return DK_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(r) || !aligned16(xbar)) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  DeviceGuard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CoefView cv;
+  s = upload_coefficients(ctx, g, C_host, nullptr, false, false, st, &cv);
+  if (s != DK_OK) return s;
+  return launch_encode(g, x, r, cv.enc, xbar, ctx->sm_count, st);
+}
+
+dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W, const float* xbar,
+                        float* ybar, void* stream) {
+  if (!ctx || !W || !xbar || !ybar) return DK_ERR_INVALID_ARG;
+  if (!aligned16(W) || !aligned16(xbar) || !aligned16(ybar)) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  DeviceGuard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return launch_simt_fwd(g, W, xbar, ybar, g.G * g.E, st);
+}
+
+dk_status dk_decode_verify(dk_ctx* ctx, const dk_problem* p, const float* ybar,
+                           const float* C_host, const float* bias, float* y,
+                           dk_verdict* verdict, void* stream) {
+  if (!ctx || !ybar || !C_host || !y || !verdict) return DK_ERR_INVALID_ARG;
+  if (!aligned16(ybar) || !aligned16(y) || !aligned16(verdict)) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  DeviceGuard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CoefView cv;
+  s = upload_coefficients(ctx, g, C_host, nullptr, true, false, st, &cv);
+  if (s != DK_OK) return s;
+  s = launch_verdict_init(verdict, st);
+  if (s != DK_OK) return s;
+  return launch_decode_verify(g, ybar, cv, bias, y, verdict, ctx->d_counters, ctx->sm_count, st);
+}
+
+dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, const float* x,
+                           const float* r, const float* C_host, const float* bias, float* y,
+                           float* xbar_save, dk_verdict* verdict, const dk_fault* fault,
+                           void* stream) {
+  if (!ctx || !W || !x || !r || !C_host || !y || !verdict) return DK_ERR_INVALID_ARG;
+  if (!aligned16(W) || !aligned16(x) || !aligned16(r) || !aligned16(y) || !aligned16(verdict) ||
+      !aligned16(xbar_save))
+    return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  if (fault) {
+    if (fault->group < 0 || fault->group >= g.G || fault->enc < 0 || fault->enc >= g.E ||
+        fault->out_index < 0 || fault->out_index >= g.n_out)
+      return DK_ERR_INVALID_ARG;
+  }
+  WsPlan wp = plan_workspace(g);
+  if (!ctx->ws || ctx->ws_bytes < wp.total) return DK_ERR_WORKSPACE;
+  DeviceGuard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CoefView cv;
+  s = upload_coefficients(ctx, g, C_host, nullptr, true, false, st, &cv);
+  if (s != DK_OK) return s;
+  char* ws = static_cast<char*>(ctx->ws);
+  float* xbar = xbar_save ? xbar_save : reinterpret_cast<float*>(ws + wp.xbar);
+  float* ybar = reinterpret_cast<float*>(ws + wp.ybar);
+  s = launch_encode(g, x, r, cv.enc, xbar, ctx->sm_count, st);
+  if (s != DK_OK) return s;
+  s = launch_simt_fwd(g, W, xbar, ybar, g.G * g.E, st);
+  if (s != DK_OK) return s;
+  if (fault) {
+    long long idx = ((long long)fault->group * g.E + fault->enc) * g.n_out + fault->out_index;
+    s = launch_add_fault(ybar, idx, fault->delta, st);
+    if (s != DK_OK) return s;
+  }
+  s = launch_verdict_init(verdict, st);
+  if (s != DK_OK) return s;
+  return launch_decode_verify(g, ybar, cv, bias, y, verdict, ctx->d_counters, ctx->sm_count, st);
+}
+
+dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* delta,
+                              const float* xbar, int32_t xbar_rows, const float* C_host,
+                              const float* gamma_host, float scale, float* dW, void* stream) {
+  if (!ctx || !delta || !xbar || !C_host || !gamma_host || !dW) return DK_ERR_INVALID_ARG;
+  if (!aligned16(delta) || !aligned16(xbar) || !aligned16(dW)) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  if (xbar_rows != g.K + 1 && xbar_rows != g.K + 2) return DK_ERR_INVALID_ARG;
+  WsPlan wp = plan_workspace(g);
+  if (!ctx->ws || ctx->ws_bytes < wp.total) return DK_ERR_WORKSPACE;
+  DeviceGuard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CoefView cv;
+  s = upload_coefficients(ctx, g, C_host, gamma_host, true, true, st, &cv);
+  if (s != DK_OK) return s;
+  float* dtil = reinterpret_cast<float*>(static_cast<char*>(ctx->ws) + wp.dtil);
+  s = launch_mix_delta(g, delta, cv.dmix, dtil, ctx->sm_count, st);
+  if (s != DK_OK) return s;
+  return launch_simt_wgrad(g, dtil, xbar, xbar_rows, scale, dW, ctx->sm_count, st);
+}
+
+}  // extern "C"

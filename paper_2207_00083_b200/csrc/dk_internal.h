@@ -1,0 +1,99 @@
+// Internal declarations shared by the translation units of libdk.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "dk.h"
+
+namespace dk {
+
+// Geometry of one layer, derived once from dk_problem.
+struct Geom {
+  int kind, layout;
+  int cin, cout, h, w, kh, kw, stride, pad, ho, wo;
+  int K, G, E;              // E = K + 2
+  long long n_in, n_out;    // elements per input / output sample
+  int kc;                   // contraction length cin*kh*kw
+  int precision;
+  float tol;
+  // element strides of one sample: activation (channel, row, col), weights
+  // (cout, cin, u, v), output (channel, row, col)
+  long long xs_c, xs_h, xs_w;
+  long long ws_o, ws_c, ws_u, ws_v;
+  long long ys_c, ys_h, ys_w;
+};
+
+dk_status make_geom(const dk_problem* p, Geom* g);
+
+// Per-call coefficient tables in device memory (all fp32), one block per group.
+// enc : [G][K+2][K+1]   encoding coefficients as given
+// dec : [G][K][K+1]     rows 0..K-1 of C_sq^{-1}, fp32 head of the fp64 value
+// decl: [G][K][K+1]     fp32 remainder of the same fp64 value
+// nul : [G][K+2]        null vector n (n[K+1] = 1)
+// dmix: [G][K+1][K]     gamma[j]*B[j][i], the delta mixing weights of Eq. 4
+struct CoefView {
+  const float* enc;
+  const float* dec;
+  const float* decl;
+  const float* nul;
+  const float* dmix;
+};
+
+constexpr int kCoefSlots = 8;
+constexpr size_t kCoefSlotBytes = 512 * 1024;
+
+}  // namespace dk
+
+struct dk_ctx {
+  int device;
+  int sm_count;
+  void* ws;
+  size_t ws_bytes;
+  char* h_stage;   // pinned, kCoefSlots * kCoefSlotBytes
+  char* d_stage;   // device, same size
+  cudaEvent_t slot_ev[dk::kCoefSlots];
+  bool slot_used[dk::kCoefSlots];
+  int cur_slot;
+  unsigned int* d_counters;   // small zero-initialised scratch for last-block logic
+  void* tc_state;             // tensor-core path state
+};
+
+namespace dk {
+
+// Host-side coefficient algebra in fp64; fills a staging slot and enqueues
+// its upload.  want_dec / want_mix select which tables are derived.
+dk_status upload_coefficients(dk_ctx* ctx, const Geom& g, const float* C_host,
+                              const float* gamma_host, bool want_dec, bool want_mix,
+                              cudaStream_t st, CoefView* view);
+
+// elementwise kernels (dk_elementwise.cu)
+dk_status launch_encode(const Geom& g, const float* x, const float* r, const float* enc,
+                        float* xbar, int sm_count, cudaStream_t st);
+dk_status launch_verdict_init(dk_verdict* v, cudaStream_t st);
+dk_status launch_decode_verify(const Geom& g, const float* ybar, const CoefView& cv,
+                               const float* bias, float* y, dk_verdict* v,
+                               unsigned int* counter, int sm_count, cudaStream_t st);
+dk_status launch_add_fault(float* ybar, long long index, float delta, cudaStream_t st);
+dk_status launch_mix_delta(const Geom& g, const float* delta, const float* dmix, float* dtil,
+                           int sm_count, cudaStream_t st);
+
+// SIMT dense kernels (dk_simt.cu)
+dk_status launch_simt_fwd(const Geom& g, const float* W, const float* xbar, float* ybar,
+                          int nsamples, cudaStream_t st);
+// dW = scale * sum_n <dtil[n], xbar[row(n)]> with row(n) = (n/(K+1))*xbar_rows + n%(K+1)
+dk_status launch_simt_wgrad(const Geom& g, const float* dtil, const float* xbar, int xbar_rows,
+                            float scale, float* dW, int sm_count, cudaStream_t st);
+
+// tensor-core path (dk_tc.cu)
+dk_status tc_init(dk_ctx* ctx);
+void tc_destroy(dk_ctx* ctx);
+
+}  // namespace dk
+
+#define DK_CUDA_CHECK(expr)                      \
+  do {                                           \
+    cudaError_t _e = (expr);                     \
+    if (_e != cudaSuccess) return DK_ERR_CUDA;   \
+  } while (0)

@@ -24,3 +24,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """Compile libdk.so in-tree when it is missing or older than its sources
+    (nvcc cross-compiles without a GPU)."""
+    from paper_2207_00083_b200 import build as _b
+    _b.build()
+    yield

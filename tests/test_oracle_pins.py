@@ -282,6 +282,13 @@ def test_verify_threshold_is_relative_to_noise_scale():
         assert int(bad["flags"].sum()) == want
 
 
+def test_verify_flags_a_nan_from_the_accelerator():
+    spec = tiny_fc_spec(K=2, G=1)
+    d = synth.draw_layer(spec)
+    bad = O.masked_forward(d["W"], d["x"], d["r"], d["C"], fault=(3, (2,), float("nan")))
+    assert bad["flags"].sum() == 1 and bad["flags"][0, 2]
+
+
 # ---------------------------------------------------------------------------
 # wgrad (Eq. 4-6)
 # ---------------------------------------------------------------------------
