@@ -31,9 +31,9 @@ library float64 convolution and its autograd, the decode/encode round trip
 against the plain definition, closed forms for K = 1, the exact residual
 change n[i]*Delta under a single injected fault, and the Eq. 5 residual.
 Parity unpinned: the numerical threshold ``tau`` of ``verify`` and its
-noise-scale normaliser are constants of this implementation, not the paper's
-(the paper compares exactly in a finite field); nothing outside this file
-fixes them.
+noise-scale normaliser max(s_e, s_g) are choices of this implementation, not
+the paper's (the paper compares exactly in a finite field); nothing outside
+this file fixes them.
 """
 from __future__ import annotations
 
@@ -196,19 +196,34 @@ def verify(ybar: np.ndarray, C: np.ndarray, y: np.ndarray, z: np.ndarray,
            tau: float = 1e-4) -> Dict[str, np.ndarray]:
     """Re-predict the redundant equation from the decoded unknowns.
 
-    rho[g] = y_bar^(K+2) - sum_k C[K+1,k] y^(k) - C[K+1,K] z.  An element is
-    flagged iff NOT(|rho| <= tau * sum_i |n_i| |y_bar^(i)|) where n is the null
-    vector of the group's C (written this way so that a NaN returned by the
-    accelerator is flagged too).  The final comparison is taken in float32
-    (the precision in which the GPU takes it).  Returns per-element arrays
-    ``rho``, ``scale``, ``ratio`` = |rho|/scale and boolean ``flags`` of shape
-    [G, ...].
+    rho[g] = y_bar^(K+2) - sum_k C[K+1,k] y^(k) - C[K+1,K] z, which is zero in
+    exact arithmetic on an honest run.  In floating point it is compared with
+    the scale of the numbers it was formed from.  With n the null vector of
+    the group's C,
+
+        s_e = sum_i |n_i| |y_bar^(i)[e]|           (this element)
+        s_g = sum_i |n_i| rms_e(y_bar^(i))          (the group's whole sample)
+
+    an element is flagged iff NOT(|rho| <= tau * max(s_e, s_g)).  The group
+    term is needed because all K+2 encodings share the term <W, r>: where it
+    happens to be near zero every y_bar^(i)[e] is small at once while the
+    rounding error of the contraction is not.  Writing the test as NOT(<=)
+    flags a NaN returned by the accelerator; an element whose s_e is not
+    finite is flagged as well, and non-finite values are left out of the rms.
+    The comparison itself is taken in float32 (the precision in which the GPU
+    takes it).
+
+    Returns per-element arrays of shape [G, ...]: ``rho``, ``scale`` =
+    max(s_e, s_g), ``ratio`` = |rho|/scale (what is compared with tau),
+    ``ratio_group`` = |rho|/s_g (what the verdict reports as max_ratio) and
+    boolean ``flags``.
     """
     G, E, K1 = C.shape
     K = K1 - 1
     ybar = np.asarray(ybar, dtype=F64)
     rho = np.zeros((G,) + ybar.shape[1:], dtype=F64)
     scale = np.zeros_like(rho)
+    sgroup = np.zeros_like(rho)
     for g in range(G):
         c = np.asarray(C[g], dtype=F64)
         pred = c[K + 1, K] * z[g]
@@ -216,25 +231,32 @@ def verify(ybar: np.ndarray, C: np.ndarray, y: np.ndarray, z: np.ndarray,
             pred = pred + c[K + 1, k] * y[g * K + k]
         rho[g] = ybar[g * E + K + 1] - pred
         n = null_vector(c)
-        s = 0.0
+        s_e = 0.0
+        s_g = 0.0
         for i in range(E):
-            s = s + abs(n[i]) * np.abs(ybar[g * E + i])
-        scale[g] = s
+            row = ybar[g * E + i]
+            s_e = s_e + abs(n[i]) * np.abs(row)
+            fin = np.isfinite(row)
+            s_g = s_g + abs(n[i]) * np.sqrt(np.mean(np.where(fin, row, 0.0) ** 2))
+        sgroup[g] = s_g
+        with np.errstate(invalid="ignore"):
+            scale[g] = np.fmax(s_e, s_g)
     with np.errstate(divide="ignore", invalid="ignore"):
         ratio = np.where(scale > 0, np.abs(rho) / scale, 0.0)
-    with np.errstate(invalid="ignore"):
+        ratio_group = np.where(sgroup > 0, np.abs(rho) / sgroup, 0.0)
         flags = ~(np.abs(rho).astype(np.float32) <= np.float32(tau) * scale.astype(np.float32))
-    return {"rho": rho, "scale": scale, "ratio": ratio, "flags": flags}
+        flags |= ~np.isfinite(scale)
+    return {"rho": rho, "scale": scale, "ratio": ratio, "ratio_group": ratio_group, "flags": flags}
 
 
 def verdict(flags: np.ndarray, ratio: np.ndarray) -> Dict[str, float]:
     """Summary of a verify pass over arrays given in the memory order of the
     output tensor: ok, n_flagged, first flagged flat index (-1 if none) and
-    the largest ratio."""
+    the largest ratio (NaNs ignored)."""
     flat = np.flatnonzero(np.asarray(flags).reshape(-1))
     return {"ok": int(flat.size == 0), "n_flagged": int(flat.size),
             "first_index": int(flat[0]) if flat.size else -1,
-            "max_ratio": float(np.max(ratio)) if ratio.size else 0.0}
+            "max_ratio": float(np.nanmax(ratio)) if ratio.size else 0.0}
 
 
 # ---------------------------------------------------------------------------

@@ -46,6 +46,7 @@ dk_status make_geom(const dk_problem* p, Geom* g) {
   long long kc = (long long)g->cin * g->kh * g->kw;
   if (kc > (1LL << 30)) return DK_ERR_SHAPE;
   g->kc = (int)kc;
+  if ((size_t)g->G * (g->E + 1) > kVerifyStatFloats) return DK_ERR_SHAPE;
   if ((long long)g->G * g->E * g->n_in >= (1LL << 40) ||
       (long long)g->G * g->E * g->n_out >= (1LL << 40))
     return DK_ERR_SHAPE;
@@ -236,8 +237,8 @@ dk_status dk_create(dk_ctx** out, int device) {
   c->sm_count = sms;
   bool ok = cudaMallocHost(&c->h_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
-            cudaMalloc(&c->d_counters, 256) == cudaSuccess &&
-            cudaMemset(c->d_counters, 0, 256) == cudaSuccess;
+            cudaMalloc(&c->d_vstats, (kVerifyStatFloats + 64) * sizeof(float)) == cudaSuccess &&
+            cudaMalloc(&c->d_cand, kCandCap * sizeof(Candidate)) == cudaSuccess;
   for (int i = 0; ok && i < kCoefSlots; ++i)
     ok = cudaEventCreateWithFlags(&c->slot_ev[i], cudaEventDisableTiming) == cudaSuccess;
   if (ok) ok = tc_init(c) == DK_OK;
@@ -255,7 +256,8 @@ dk_status dk_destroy(dk_ctx* c) {
     if (c->slot_ev[i]) cudaEventDestroy(c->slot_ev[i]);
   if (c->h_stage) cudaFreeHost(c->h_stage);
   if (c->d_stage) cudaFree(c->d_stage);
-  if (c->d_counters) cudaFree(c->d_counters);
+  if (c->d_vstats) cudaFree(c->d_vstats);
+  if (c->d_cand) cudaFree(c->d_cand);
   delete c;
   return DK_OK;
 }
@@ -320,9 +322,12 @@ dk_status dk_decode_verify(dk_ctx* ctx, const dk_problem* p, const float* ybar,
   CoefView cv;
   s = upload_coefficients(ctx, g, C_host, nullptr, true, false, st, &cv);
   if (s != DK_OK) return s;
-  s = launch_verdict_init(verdict, st);
+  VerifyScratch vs = verify_scratch(ctx, g);
+  s = launch_verify_begin(g, vs, st);
   if (s != DK_OK) return s;
-  return launch_decode_verify(g, ybar, cv, bias, y, verdict, ctx->d_counters, ctx->sm_count, st);
+  s = launch_decode_verify(g, ybar, cv, bias, y, vs, ctx->sm_count, st);
+  if (s != DK_OK) return s;
+  return launch_verify_finalize(g, cv.nul, vs, verdict, st);
 }
 
 dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, const float* x,
@@ -361,9 +366,12 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     s = launch_add_fault(ybar, idx, fault->delta, st);
     if (s != DK_OK) return s;
   }
-  s = launch_verdict_init(verdict, st);
+  VerifyScratch vs = verify_scratch(ctx, g);
+  s = launch_verify_begin(g, vs, st);
   if (s != DK_OK) return s;
-  return launch_decode_verify(g, ybar, cv, bias, y, verdict, ctx->d_counters, ctx->sm_count, st);
+  s = launch_decode_verify(g, ybar, cv, bias, y, vs, ctx->sm_count, st);
+  if (s != DK_OK) return s;
+  return launch_verify_finalize(g, cv.nul, vs, verdict, st);
 }
 
 dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* delta,

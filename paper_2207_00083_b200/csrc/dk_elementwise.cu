@@ -79,25 +79,54 @@ mix_rows_kernel(const float* __restrict__ x, const float* __restrict__ r,
   }
 }
 
-__global__ void verdict_init_kernel(dk_verdict* v) {
-  v->ok = 1;
-  v->n_flagged = 0;
-  v->first_index = 0x7fffffffffffffffLL;
-  v->max_ratio = 0.f;
-  v->status = 0;
-}
-
 __global__ void add_fault_kernel(float* ybar, long long idx, float delta) { ybar[idx] += delta; }
 
-// Block-level merge of per-thread verify results into the device verdict;
-// the last block to finish turns an untouched first_index into -1.
-__device__ void verdict_merge(dk_verdict* vd, unsigned int* counter, unsigned int nflag,
-                              long long first, float maxr, unsigned int nblocks) {
-  __shared__ unsigned int s_n[32];
-  __shared__ long long s_f[32];
-  __shared__ float s_r[32];
+// Clears the per-call statistics of the integrity check.
+__global__ void verify_begin_kernel(float* stats, int nstats, unsigned int* count) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nstats; i += gridDim.x * blockDim.x)
+    stats[i] = 0.f;
+  if (blockIdx.x == 0 && threadIdx.x == 0) *count = 0u;
+}
+
+// s_g = sum_i |n_i| * rms(ybar_i) for group g from the accumulated sums of squares.
+__device__ __forceinline__ float group_scale(const float* sumsq, const float* nul, long long g,
+                                             int E, float inv_n) {
+  float s = 0.f;
+  for (int i = 0; i < E; ++i) s += fabsf(nul[g * E + i]) * sqrtf(sumsq[g * E + i] * inv_n);
+  return s;
+}
+
+// One block: final decision for every candidate, summary into *vd.
+__global__ void __launch_bounds__(256)
+verify_finalize_kernel(const float* sumsq, const int* maxrho, const unsigned int* count,
+                       const Candidate* cand, const float* nul, dk_verdict* vd, int G, int E,
+                       long long n_out, float tau) {
+  __shared__ unsigned int s_n[8];
+  __shared__ long long s_f[8];
+  __shared__ float s_r[8];
+  const float inv_n = 1.f / (float)n_out;
+  unsigned int nflag = 0;
+  long long first = 0x7fffffffffffffffLL;
+  float maxr = 0.f;
+  for (int g = threadIdx.x; g < G; g += blockDim.x) {
+    float sg = group_scale(sumsq, nul, g, E, inv_n);
+    float mr = __int_as_float(maxrho[g]);
+    if (sg > 0.f) maxr = fmaxf(maxr, mr / sg);
+  }
+  const unsigned int total = *count;
+  const unsigned int n = total < kCandCap ? total : kCandCap;
+  for (unsigned int c = threadIdx.x; c < n; c += blockDim.x) {
+    Candidate cd = cand[c];
+    long long g = cd.index / n_out;
+    float sg = group_scale(sumsq, nul, g, E, inv_n);
+    float scale = fmaxf(cd.s_e, sg);
+    bool bad = !(cd.absrho <= tau * scale) || !(cd.s_e < __int_as_float(0x7f800000));
+    if (bad) {
+      ++nflag;
+      first = cd.index < first ? cd.index : first;
+    }
+  }
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  const int nw = (blockDim.x + 31) >> 5;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     nflag += __shfl_xor_sync(0xffffffffu, nflag, o);
@@ -108,26 +137,51 @@ __device__ void verdict_merge(dk_verdict* vd, unsigned int* counter, unsigned in
   if (lane == 0) { s_n[wid] = nflag; s_f[wid] = first; s_r[wid] = maxr; }
   __syncthreads();
   if (threadIdx.x == 0) {
-    for (int w = 1; w < nw; ++w) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) {
       nflag += s_n[w];
       first = s_f[w] < first ? s_f[w] : first;
       maxr = fmaxf(maxr, s_r[w]);
     }
-    if (nflag) {
-      atomicAdd(&vd->n_flagged, nflag);
-      atomicMin(reinterpret_cast<unsigned long long*>(&vd->first_index), (unsigned long long)first);
-      atomicExch(&vd->ok, 0);
+    int status = 0;
+    if (total > kCandCap) {
+      // more suspects than the list holds: everything beyond it counts as flagged
+      nflag += total - kCandCap;
+      status = DK_ERR_WORKSPACE;
     }
-    if (maxr > 0.f) atomicMax(reinterpret_cast<int*>(&vd->max_ratio), __float_as_int(maxr));
-    __threadfence();
-    unsigned int done = atomicAdd(counter, 1u);
-    if (done == nblocks - 1) {
-      __threadfence();
-      unsigned long long fi =
-          atomicAdd(reinterpret_cast<unsigned long long*>(&vd->first_index), 0ULL);
-      if (fi == 0x7fffffffffffffffULL) vd->first_index = -1;
-      *counter = 0;
-    }
+    vd->ok = nflag == 0 ? 1 : 0;
+    vd->n_flagged = nflag;
+    vd->first_index = nflag ? first : -1;
+    vd->max_ratio = maxr;
+    vd->status = status;
+  }
+}
+
+// Per-block merge of the verify statistics: E sums of squares and max |rho|.
+template <int E>
+__device__ __forceinline__ void stats_merge(const VerifyScratch& vs, int g, float (&sq)[E],
+                                            float maxrho) {
+  __shared__ float s_sq[kThreads / 32][E + 1];
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+  for (int i = 0; i < E; ++i)
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq[i] += __shfl_xor_sync(0xffffffffu, sq[i], o);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) maxrho = fmaxf(maxrho, __shfl_xor_sync(0xffffffffu, maxrho, o));
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < E; ++i) s_sq[wid][i] = sq[i];
+    s_sq[wid][E] = maxrho;
+  }
+  __syncthreads();
+  if (threadIdx.x < E) {
+    float t = 0.f;
+    for (int w = 0; w < kThreads / 32; ++w) t += s_sq[w][threadIdx.x];
+    if (t != 0.f) atomicAdd(vs.sumsq + (size_t)g * E + threadIdx.x, t);
+  } else if (threadIdx.x == E) {
+    float t = 0.f;
+    for (int w = 0; w < kThreads / 32; ++w) t = fmaxf(t, s_sq[w][E]);
+    if (t > 0.f) atomicMax(vs.maxrho + g, __float_as_int(t));
   }
 }
 
@@ -135,8 +189,8 @@ template <int K, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 decode_verify_kernel(const float* __restrict__ ybar, const float* __restrict__ dec,
                      const float* __restrict__ decl, const float* __restrict__ nul,
-                     const float* __restrict__ bias, float* __restrict__ y, dk_verdict* vd,
-                     unsigned int* counter, long long n, float tau, int cout, long long cdiv) {
+                     const float* __restrict__ bias, float* __restrict__ y, VerifyScratch vs,
+                     long long n, float tau, int cout, long long cdiv) {
   constexpr int K1 = K + 1, E = K + 2;
   const int g = blockIdx.y;
   float dh[K][K1], dl[K][K1], nv[E];
@@ -151,9 +205,11 @@ decode_verify_kernel(const float* __restrict__ ybar, const float* __restrict__ d
   for (int i = 0; i < E; ++i) nv[i] = __ldg(nul + (size_t)g * E + i);
   const float* yb = ybar + (size_t)g * E * n;
   float* yo = y + (size_t)g * K * n;
-  unsigned int nflag = 0;
-  long long first = 0x7fffffffffffffffLL;
-  float maxr = 0.f;
+  float sq[E];
+#pragma unroll
+  for (int i = 0; i < E; ++i) sq[i] = 0.f;
+  float maxrho = 0.f;
+  const float kInf = __int_as_float(0x7f800000);
   const long long nvec = (n + 3) / 4;
   for (long long v = (long long)blockIdx.x * kThreads + threadIdx.x; v < nvec;
        v += (long long)gridDim.x * kThreads) {
@@ -188,20 +244,27 @@ decode_verify_kernel(const float* __restrict__ ybar, const float* __restrict__ d
         float rho = 0.f, sc = 0.f;
 #pragma unroll
         for (int i = 0; i < E; ++i) {
-          rho = fmaf(nv[i], in[i].v[q], rho);
-          sc = fmaf(fabsf(nv[i]), fabsf(in[i].v[q]), sc);
+          const float val = in[i].v[q];
+          rho = fmaf(nv[i], val, rho);
+          sc = fmaf(fabsf(nv[i]), fabsf(val), sc);
+          if (fabsf(val) < kInf) sq[i] = fmaf(val, val, sq[i]);
         }
         const float ar = fabsf(rho);
-        if (!(ar <= tau * sc)) {
-          ++nflag;
-          long long idx = (long long)g * n + e + q;
-          first = idx < first ? idx : first;
+        maxrho = fmaxf(maxrho, ar);
+        if (!(ar <= tau * sc) || !(sc < kInf)) {
+          unsigned int slot = atomicAdd(vs.count, 1u);
+          if (slot < kCandCap) {
+            Candidate cd;
+            cd.index = (long long)g * n + e + q;
+            cd.absrho = ar;
+            cd.s_e = sc;
+            vs.cand[slot] = cd;
+          }
         }
-        if (sc > 0.f) maxr = fmaxf(maxr, ar / sc);
       }
     }
   }
-  verdict_merge(vd, counter, nflag, first, maxr, gridDim.x * gridDim.y);
+  stats_merge<E>(vs, g, sq, maxrho);
 }
 
 inline int blocks_for(long long n, int G, int sm_count) {
@@ -229,17 +292,16 @@ dk_status launch_mix(const float* x, const float* r, const float* coef, float* o
 
 template <int K>
 dk_status launch_dv(const Geom& g, const float* ybar, const CoefView& cv, const float* bias,
-                    float* y, dk_verdict* v, unsigned int* counter, int sm_count,
-                    cudaStream_t st) {
+                    float* y, const VerifyScratch& vs, int sm_count, cudaStream_t st) {
   dim3 grid(blocks_for(g.n_out, g.G, sm_count), g.G);
   // channel of element e: (e / cdiv) % cout
   long long cdiv = (g.layout == DK_NCHW && g.kind == DK_CONV2D) ? (long long)g.ho * g.wo : 1;
   if (g.n_out % 4 == 0)
     decode_verify_kernel<K, true><<<grid, kThreads, 0, st>>>(
-        ybar, cv.dec, cv.decl, cv.nul, bias, y, v, counter, g.n_out, g.tol, g.cout, cdiv);
+        ybar, cv.dec, cv.decl, cv.nul, bias, y, vs, g.n_out, g.tol, g.cout, cdiv);
   else
     decode_verify_kernel<K, false><<<grid, kThreads, 0, st>>>(
-        ybar, cv.dec, cv.decl, cv.nul, bias, y, v, counter, g.n_out, g.tol, g.cout, cdiv);
+        ybar, cv.dec, cv.decl, cv.nul, bias, y, vs, g.n_out, g.tol, g.cout, cdiv);
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
 }
@@ -272,17 +334,37 @@ dk_status launch_mix_delta(const Geom& g, const float* delta, const float* dmix,
                                                           g.G, sm_count, st)));
 }
 
-dk_status launch_verdict_init(dk_verdict* v, cudaStream_t st) {
-  verdict_init_kernel<<<1, 1, 0, st>>>(v);
+VerifyScratch verify_scratch(const dk_ctx* ctx, const Geom& g) {
+  VerifyScratch vs;
+  vs.sumsq = ctx->d_vstats;
+  vs.maxrho = reinterpret_cast<int*>(ctx->d_vstats + (size_t)g.G * g.E);
+  vs.count = reinterpret_cast<unsigned int*>(ctx->d_vstats + kVerifyStatFloats);
+  vs.cand = ctx->d_cand;
+  return vs;
+}
+
+dk_status launch_verify_begin(const Geom& g, const VerifyScratch& vs, cudaStream_t st) {
+  int nstats = g.G * (g.E + 1);
+  int blocks = (nstats + 255) / 256;
+  if (blocks > 64) blocks = 64;
+  verify_begin_kernel<<<blocks, 256, 0, st>>>(vs.sumsq, nstats, vs.count);
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
 }
 
 dk_status launch_decode_verify(const Geom& g, const float* ybar, const CoefView& cv,
-                               const float* bias, float* y, dk_verdict* v,
-                               unsigned int* counter, int sm_count, cudaStream_t st) {
+                               const float* bias, float* y, const VerifyScratch& vs,
+                               int sm_count, cudaStream_t st) {
   if (g.G > 65535) return DK_ERR_SHAPE;
-  DK_DISPATCH_K(g.K, return (launch_dv<KK>(g, ybar, cv, bias, y, v, counter, sm_count, st)));
+  DK_DISPATCH_K(g.K, return (launch_dv<KK>(g, ybar, cv, bias, y, vs, sm_count, st)));
+}
+
+dk_status launch_verify_finalize(const Geom& g, const float* nul, const VerifyScratch& vs,
+                                 dk_verdict* v, cudaStream_t st) {
+  verify_finalize_kernel<<<1, 256, 0, st>>>(vs.sumsq, vs.maxrho, vs.count, vs.cand, nul, v, g.G,
+                                            g.E, g.n_out, g.tol);
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
 }
 
 dk_status launch_add_fault(float* ybar, long long index, float delta, cudaStream_t st) {

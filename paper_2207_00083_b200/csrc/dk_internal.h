@@ -44,6 +44,26 @@ struct CoefView {
 constexpr int kCoefSlots = 8;
 constexpr size_t kCoefSlotBytes = 512 * 1024;
 
+// Scratch of the integrity check.  The decision for an element needs the rms
+// of every encoded output row of its group, which is only known once the whole
+// tensor has been seen; so the pass that decodes accumulates the sums of
+// squares and appends every element that fails the per-element test to a
+// candidate list, and a one-block kernel takes the final decisions.
+struct Candidate {
+  long long index;   // g*n_out + e
+  float absrho;      // |rho|
+  float s_e;         // sum_i |n_i||ybar_i[e]|
+};
+constexpr unsigned int kCandCap = 1u << 16;
+constexpr size_t kVerifyStatFloats = 1u << 18;   // >= G*(K+3)
+
+struct VerifyScratch {
+  float* sumsq;          // [G][K+2] sum of squares of the finite values of each row
+  int* maxrho;           // [G] bit pattern of max |rho|
+  unsigned int* count;   // candidates appended (may exceed kCandCap)
+  Candidate* cand;       // [kCandCap]
+};
+
 }  // namespace dk
 
 struct dk_ctx {
@@ -56,7 +76,8 @@ struct dk_ctx {
   cudaEvent_t slot_ev[dk::kCoefSlots];
   bool slot_used[dk::kCoefSlots];
   int cur_slot;
-  unsigned int* d_counters;   // small zero-initialised scratch for last-block logic
+  float* d_vstats;            // kVerifyStatFloats floats + one counter
+  dk::Candidate* d_cand;      // kCandCap entries
   void* tc_state;             // tensor-core path state
 };
 
@@ -71,10 +92,14 @@ dk_status upload_coefficients(dk_ctx* ctx, const Geom& g, const float* C_host,
 // elementwise kernels (dk_elementwise.cu)
 dk_status launch_encode(const Geom& g, const float* x, const float* r, const float* enc,
                         float* xbar, int sm_count, cudaStream_t st);
-dk_status launch_verdict_init(dk_verdict* v, cudaStream_t st);
+VerifyScratch verify_scratch(const dk_ctx* ctx, const Geom& g);
+// begin: clears the statistics; finalize: decides the candidates, writes *v
+dk_status launch_verify_begin(const Geom& g, const VerifyScratch& vs, cudaStream_t st);
 dk_status launch_decode_verify(const Geom& g, const float* ybar, const CoefView& cv,
-                               const float* bias, float* y, dk_verdict* v,
-                               unsigned int* counter, int sm_count, cudaStream_t st);
+                               const float* bias, float* y, const VerifyScratch& vs,
+                               int sm_count, cudaStream_t st);
+dk_status launch_verify_finalize(const Geom& g, const float* nul, const VerifyScratch& vs,
+                                 dk_verdict* v, cudaStream_t st);
 dk_status launch_add_fault(float* ybar, long long index, float delta, cudaStream_t st);
 dk_status launch_mix_delta(const Geom& g, const float* delta, const float* dmix, float* dtil,
                            int sm_count, cudaStream_t st);

@@ -1,0 +1,326 @@
+"""GPU parity: every entry point of the C-ABI against the fp64 oracle on the
+same seeded inputs.  Floating-point bars: decoded outputs and gradients within
+1e-3 max-norm relative error (the encoded intermediates are held to tighter
+bars derived from fp32 rounding); integrity verdicts identical."""
+import ctypes
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dk_oracle as O
+from paper_2207_00083_b200 import binding as dk
+from paper_2207_00083_b200 import synth
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+
+TOL_DECODED = 1e-3      # decoded y and dW vs the oracle (max-norm relative)
+TOL_ENCODE = 1e-6       # x_bar: a handful of fp32 roundings of a K+1 term sum
+TOL_YBAR = 2e-5         # y_bar on identical fp32 inputs: fp32-class contraction
+
+
+def tiny(kind="conv", **kw):
+    base = dict(workload="tiny", name="t", kind=kind, cin=8, cout=12, K=2, G=2, sigma_r=100.0)
+    if kind == "conv":
+        base.update(h=9, w=7, kh=3, kw=3, stride=1, pad=1)
+    base.update(kw)
+    return synth.LayerSpec(**base)
+
+
+def small_cases():
+    L = synth.layer
+    return [
+        ("fc784", synth.layers("fc784")[0]),
+        ("fc_ragged_K1", tiny("fc", cin=37, cout=19, K=1, G=3)),
+        ("fc_K8", tiny("fc", cin=64, cout=130, K=8, G=2, sigma_r=1000.0, x_dist="normal")),
+        ("conv_tiny_K2", tiny()),
+        ("conv_ragged_K3", tiny(cin=5, cout=7, h=6, w=5, K=3, G=2)),
+        ("conv_7x7s2", tiny(cin=3, cout=16, h=20, w=20, kh=7, kw=7, stride=2, pad=3, K=4, G=1)),
+        ("conv_1x1s2", tiny(cin=16, cout=24, h=10, w=10, kh=1, kw=1, stride=2, pad=0, K=4, G=2)),
+        ("conv_3x3s2", tiny(cin=12, cout=20, h=11, w=11, stride=2, K=4, G=1)),
+        ("vgg_cifar_conv3_1_G2", L("vgg16_cifar", "conv3_1").with_groups(2)),
+        ("vgg_cifar_conv5_1_G3", L("vgg16_cifar", "conv5_1").with_groups(3)),
+        ("vgg_cifar_conv1_1_G2", L("vgg16_cifar", "conv1_1").with_groups(2)),
+        ("resnet_layer4_3x3_G2", L("resnet18_224", "layer4_3x3").with_groups(2)),
+        ("resnet_layer3_ds_G1", L("resnet18_224", "layer3_ds").with_groups(1)),
+        ("resnet_fc_G16", L("resnet18_224", "fc")),
+        ("mbv2_project_960_320_G2", L("mobilenetv2_pw", "project_960_320").with_groups(2)),
+        ("mbv2_expand_24_144_G1", dataclasses.replace(L("mobilenetv2_pw", "expand_24_144"), G=1, h=28, w=28)),
+        ("vgg224_fc7_G2", L("vgg16_224", "fc7").with_groups(2)),
+    ]
+
+
+CASES = small_cases()
+IDS = [c[0] for c in CASES]
+SPECS = [c[1] for c in CASES]
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = dk.Context(0)
+    yield c
+    c.close()
+
+
+@pytest.fixture(scope="module")
+def drawn():
+    cache = {}
+
+    def get(spec):
+        key = dataclasses.astuple(spec)
+        if key not in cache:
+            cache[key] = synth.draw_layer(spec)
+        return cache[key]
+    return get
+
+
+def lay(spec):
+    return dk.DK_NHWC
+
+
+# ---------------------------------------------------------------------------
+# dk_encode
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("spec", SPECS, ids=IDS)
+def test_encode_matches_oracle(ctx, drawn, spec):
+    d = drawn(spec)
+    p = dk.problem_from_spec(spec)
+    x, r = H.acts_to_dev(d["x"], lay(spec)), H.acts_to_dev(d["r"], lay(spec))
+    xbar = H.empty_acts(spec.G * (spec.K + 2), spec, "in", lay(spec))
+    dk.dk_encode(ctx, p, x, r, d["C"], xbar)
+    want = O.encode(d["x"], d["r"], d["C"])
+    assert H.max_rel(H.acts_from_dev(xbar, lay(spec)), want) < TOL_ENCODE
+
+
+# ---------------------------------------------------------------------------
+# dk_linear_fwd on identical fp32 encodings
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("prec", [dk.DK_PREC_DEFAULT, dk.DK_FP32_SIMT], ids=["default", "simt"])
+@pytest.mark.parametrize("spec", SPECS, ids=IDS)
+def test_linear_fwd_matches_oracle(ctx, drawn, spec, prec):
+    d = drawn(spec)
+    p = dk.problem_from_spec(spec, precision=prec)
+    xbar32 = O.encode(d["x"], d["r"], d["C"]).astype(np.float32)
+    W = H.weights_to_dev(d["W"], lay(spec))
+    xb = H.acts_to_dev(xbar32, lay(spec))
+    ybar = H.empty_acts(spec.G * (spec.K + 2), spec, "out", lay(spec))
+    ctx.ensure_workspace(p)
+    dk.dk_linear_fwd(ctx, p, W, xb, ybar)
+    want = O.linear(d["W"], xbar32, spec.stride, spec.pad)
+    assert H.max_rel(H.acts_from_dev(ybar, lay(spec)), want) < TOL_YBAR
+
+
+# ---------------------------------------------------------------------------
+# dk_decode_verify on identical fp32 y_bar, clean and with one wrong value
+# ---------------------------------------------------------------------------
+def _fault_list(spec):
+    E = spec.K + 2
+    out = [None]
+    last = (spec.cout - 1, spec.hout - 1, spec.wout - 1)
+    for enc in range(E):
+        g = enc % spec.G
+        pos = (enc % spec.cout, 0, 0) if enc % 2 == 0 else last
+        out.append((g, enc, pos))
+    return out
+
+
+@pytest.mark.parametrize("spec", SPECS, ids=IDS)
+def test_decode_verify_matches_oracle(ctx, drawn, spec):
+    d = drawn(spec)
+    K, E = spec.K, spec.K + 2
+    p = dk.problem_from_spec(spec, tol=H.TAU)
+    xbar = O.encode(d["x"], d["r"], d["C"])
+    ybar32 = O.linear(d["W"], xbar, spec.stride, spec.pad).astype(np.float32)
+    bias = np.linspace(-1.0, 1.0, spec.cout).astype(np.float32)
+    v = dk.new_verdict()
+    y = H.empty_acts(spec.G * K, spec, "out", lay(spec))
+    for fault in _fault_list(spec):
+        yb = ybar32.copy()
+        if fault is not None:
+            g, enc, (co, oh, ow) = fault
+            idx = (g * E + enc,) + H.logical_out_index(spec, co, oh, ow)
+            yb[idx] += np.float32(0.5 * float(np.sqrt(np.mean(yb[idx[0]].astype(np.float64) ** 2))))
+        yd, zd = O.decode(yb, d["C"])
+        chk = O.verify(yb, d["C"], yd, zd, H.TAU)
+        H.assert_no_gray_zone(chk["ratio"])
+        want_v = H.expected_verdict(chk["flags"], chk["ratio_group"], lay(spec))
+        dk.dk_decode_verify(ctx, p, H.acts_to_dev(yb, lay(spec)), d["C"], H.dev(bias), y, v)
+        got_v = dk.read_verdict(v)
+        assert got_v["status"] == 0
+        assert (got_v["ok"], got_v["n_flagged"], got_v["first_index"]) == \
+               (want_v["ok"], want_v["n_flagged"], want_v["first_index"])
+        if fault is None:
+            assert want_v["ok"] == 1 and got_v["max_ratio"] < H.TAU / 4
+            want_y = yd + (bias if yd.ndim == 2 else bias[None, :, None, None])
+            assert H.max_rel(H.acts_from_dev(y, lay(spec)), want_y) < TOL_DECODED
+        else:
+            g, enc, (co, oh, ow) = fault
+            assert want_v["n_flagged"] == 1
+            assert got_v["first_index"] == g * spec.n_out + H.flat_out_index(spec, lay(spec), co, oh, ow)
+            assert got_v["max_ratio"] == pytest.approx(want_v["max_ratio"], rel=1e-2)
+
+
+# ---------------------------------------------------------------------------
+# dk_masked_linear: decoded outputs vs the plain definition, verdicts
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("prec", [dk.DK_PREC_DEFAULT, dk.DK_FP32_SIMT], ids=["default", "simt"])
+@pytest.mark.parametrize("spec", SPECS, ids=IDS)
+def test_masked_linear_matches_oracle(ctx, drawn, spec, prec):
+    d = drawn(spec)
+    K, E = spec.K, spec.K + 2
+    p = dk.problem_from_spec(spec, precision=prec, tol=H.TAU)
+    ctx.ensure_workspace(p)
+    W = H.weights_to_dev(d["W"], lay(spec))
+    x, r = H.acts_to_dev(d["x"], lay(spec)), H.acts_to_dev(d["r"], lay(spec))
+    y = H.empty_acts(spec.G * K, spec, "out", lay(spec))
+    xsave = H.empty_acts(spec.G * E, spec, "in", lay(spec))
+    v = dk.new_verdict()
+    clean = O.masked_forward(d["W"], d["x"], d["r"], d["C"], spec.stride, spec.pad, H.TAU)
+    plain = O.linear_plain(d["W"], d["x"], spec.stride, spec.pad)
+
+    dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y, xsave, v)
+    got_v = dk.read_verdict(v)
+    assert (got_v["ok"], got_v["n_flagged"], got_v["first_index"], got_v["status"]) == (1, 0, -1, 0)
+    assert got_v["max_ratio"] < H.TAU / 4
+    got_y = H.acts_from_dev(y, lay(spec))
+    assert H.max_rel(got_y, plain) < TOL_DECODED
+    assert H.max_rel(got_y, clean["y"]) < TOL_DECODED
+    assert H.max_rel(H.acts_from_dev(xsave, lay(spec)), clean["xbar"]) < TOL_ENCODE
+
+    # without xbar_save the result is the same
+    y2 = torch.empty_like(y)
+    dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y2, None, v)
+    assert torch.equal(y, y2)
+
+    # one wrong accelerator output in every encoding row is flagged, exactly once
+    for fault in _fault_list(spec)[1:]:
+        g, enc, (co, oh, ow) = fault
+        row = g * E + enc
+        lidx = H.logical_out_index(spec, co, oh, ow)
+        delta = 0.5 * float(np.sqrt(np.mean(clean["ybar"][row] ** 2)))
+        bad = O.masked_forward(d["W"], d["x"], d["r"], d["C"], spec.stride, spec.pad, H.TAU,
+                               fault=(row, lidx, delta))
+        H.assert_no_gray_zone(bad["ratio"])
+        want_v = H.expected_verdict(bad["flags"], bad["ratio_group"], lay(spec))
+        f = dk.dk_fault(g, enc, H.flat_out_index(spec, lay(spec), co, oh, ow), delta)
+        dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y2, None, v, f)
+        got_v = dk.read_verdict(v)
+        assert (got_v["ok"], got_v["n_flagged"], got_v["first_index"]) == \
+               (want_v["ok"], want_v["n_flagged"], want_v["first_index"]) == \
+               (0, 1, g * spec.n_out + f.out_index)
+        assert got_v["max_ratio"] == pytest.approx(want_v["max_ratio"], rel=1e-2)
+
+
+# ---------------------------------------------------------------------------
+# dk_linear_bwd_wgrad
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("prec", [dk.DK_PREC_DEFAULT, dk.DK_FP32_SIMT], ids=["default", "simt"])
+@pytest.mark.parametrize("rows", ["K+2", "K+1"])
+@pytest.mark.parametrize("spec", SPECS, ids=IDS)
+def test_wgrad_matches_oracle(ctx, drawn, spec, rows, prec):
+    d = drawn(spec)
+    K, E = spec.K, spec.K + 2
+    p = dk.problem_from_spec(spec, precision=prec)
+    ctx.ensure_workspace(p)
+    xbar32 = O.encode(d["x"], d["r"], d["C"]).astype(np.float32)
+    nrows = E
+    if rows == "K+1":
+        keep = np.array([g * E + j for g in range(spec.G) for j in range(K + 1)])
+        xbar32 = xbar32[keep]
+        nrows = K + 1
+    scale = 1.0 / spec.batch
+    dW = H.empty_weights(spec, lay(spec))
+    dW.fill_(float("nan"))
+    dk.dk_linear_bwd_wgrad(ctx, p, H.acts_to_dev(d["delta"], lay(spec)), H.acts_to_dev(xbar32, lay(spec)),
+                           nrows, d["C"], d["gamma"], scale, dW)
+    got = H.weights_from_dev(dW, lay(spec))
+    plain = O.wgrad_plain(d["delta"], d["x"], scale, spec.kh, spec.kw, spec.stride, spec.pad)
+    masked = O.wgrad_masked(d["delta"], xbar32, d["C"], d["gamma"], scale, spec.kh, spec.kw,
+                            spec.stride, spec.pad, xbar_rows_per_group=nrows)
+    assert H.max_rel(got, masked) < TOL_DECODED
+    assert H.max_rel(got, plain) < TOL_DECODED
+
+
+# ---------------------------------------------------------------------------
+# channels-first layout (SIMT path) and bias in the fused call
+# ---------------------------------------------------------------------------
+def test_channels_first_layout_and_bias(ctx, drawn):
+    spec = tiny(cin=6, cout=10, h=8, w=9, K=2, G=2)
+    d = drawn(spec)
+    L = dk.DK_NCHW
+    p = dk.problem_from_spec(spec, layout=L, tol=H.TAU)
+    ctx.ensure_workspace(p)
+    bias = np.arange(spec.cout, dtype=np.float32) - 3
+    y = H.empty_acts(spec.batch, spec, "out", L)
+    xsave = H.empty_acts(spec.G * 4, spec, "in", L)
+    v = dk.new_verdict()
+    dk.dk_masked_linear(ctx, p, H.dev(d["W"]), H.dev(d["x"]), H.dev(d["r"]), d["C"], H.dev(bias), y, xsave, v)
+    want = O.linear_plain(d["W"], d["x"], spec.stride, spec.pad) + bias[None, :, None, None]
+    assert H.max_rel(y.cpu().numpy(), want) < TOL_DECODED
+    assert dk.read_verdict(v)["ok"] == 1
+    f = dk.dk_fault(1, 3, H.flat_out_index(spec, L, 4, 2, 5), 50.0)
+    dk.dk_masked_linear(ctx, p, H.dev(d["W"]), H.dev(d["x"]), H.dev(d["r"]), d["C"], None, y, None, v, f)
+    got = dk.read_verdict(v)
+    assert (got["ok"], got["n_flagged"], got["first_index"]) == (0, 1, spec.n_out + f.out_index)
+    dW = H.empty_weights(spec, L)
+    dk.dk_linear_bwd_wgrad(ctx, p, H.dev(d["delta"]), xsave, 4, d["C"], d["gamma"], 0.25, dW)
+    plain = O.wgrad_plain(d["delta"], d["x"], 0.25, 3, 3, 1, 1)
+    assert H.max_rel(dW.cpu().numpy(), plain) < TOL_DECODED
+
+
+# ---------------------------------------------------------------------------
+# error behaviour
+# ---------------------------------------------------------------------------
+def test_error_statuses(drawn):
+    spec = tiny("fc", cin=16, cout=8, K=2, G=1)
+    d = drawn(spec)
+    p = dk.problem_from_spec(spec)
+    c = dk.Context(0)
+    try:
+        x, r, W = H.dev(d["x"]), H.dev(d["r"]), H.dev(d["W"])
+        y = H.empty_acts(2, spec, "out", 0)
+        v = dk.new_verdict()
+        with pytest.raises(dk.DkError) as e:       # no workspace registered
+            dk.dk_masked_linear(c, p, W, x, r, d["C"], None, y, None, v)
+        assert e.value.status == 4
+        c.ensure_workspace(p)
+        Cs = d["C"].copy()
+        Cs[0, 1] = 2 * Cs[0, 0]                    # two dependent decode rows
+        with pytest.raises(dk.DkError) as e:
+            dk.dk_masked_linear(c, p, W, x, r, Cs, None, y, None, v)
+        assert e.value.status == 3
+        bad = dk.dk_fault(0, 9, 0, 1.0)            # encoding index out of range
+        with pytest.raises(dk.DkError) as e:
+            dk.dk_masked_linear(c, p, W, x, r, d["C"], None, y, None, v, bad)
+        assert e.value.status == 1
+        xb = torch.empty(4 * 16 + 1, device="cuda")[1:]   # 4-byte aligned only
+        rc = dk.lib().dk_encode(c.handle, ctypes.byref(p), ctypes.c_void_p(x.data_ptr()),
+                                ctypes.c_void_p(r.data_ptr()), ctypes.c_void_p(d["C"].ctypes.data),
+                                ctypes.c_void_p(xb.data_ptr()), None)
+        assert rc == 1
+        g0 = d["gamma"].copy()
+        g0[0, 1] = 0.0
+        with pytest.raises(dk.DkError) as e:
+            dk.dk_linear_bwd_wgrad(c, p, H.dev(d["delta"]), H.empty_acts(4, spec, "in", 0), 4, d["C"], g0,
+                                   1.0, H.empty_weights(spec, 0))
+        assert e.value.status == 1
+        # the context is still usable after refused calls
+        dk.dk_masked_linear(c, p, W, x, r, d["C"], None, y, None, v)
+        assert dk.read_verdict(v)["ok"] == 1
+    finally:
+        c.close()
+
+
+def test_nan_from_the_accelerator_is_flagged(ctx, drawn):
+    spec = tiny("fc", cin=16, cout=8, K=2, G=1)
+    d = drawn(spec)
+    p = dk.problem_from_spec(spec)
+    ybar = O.linear(d["W"], O.encode(d["x"], d["r"], d["C"])).astype(np.float32)
+    ybar[2, 5] = np.nan
+    v = dk.new_verdict()
+    y = H.empty_acts(2, spec, "out", 0)
+    dk.dk_decode_verify(ctx, p, H.dev(ybar), d["C"], None, y, v)
+    got = dk.read_verdict(v)
+    assert (got["ok"], got["n_flagged"], got["first_index"]) == (0, 1, 5)

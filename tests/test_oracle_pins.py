@@ -219,7 +219,7 @@ def test_verify_clean_run_has_zero_residual(K):
     m = O.masked_forward(d["W"], d["x"], d["r"], d["C"], spec.stride, spec.pad)
     assert m["ratio"].max() < 1e-10
     assert not m["flags"].any()
-    v = O.verdict(m["flags"], m["ratio"])
+    v = O.verdict(m["flags"], m["ratio_group"])
     assert v == {"ok": 1, "n_flagged": 0, "first_index": -1, "max_ratio": v["max_ratio"]}
 
 
@@ -280,6 +280,29 @@ def test_verify_threshold_is_relative_to_noise_scale():
         dlt = factor * 1e-4 * s / abs(n[0])
         bad = O.masked_forward(d["W"], d["x"], d["r"], d["C"], fault=(0, (1,), dlt))
         assert int(bad["flags"].sum()) == want
+
+
+def test_verify_does_not_flag_rounding_where_all_encodings_vanish():
+    """Where <W, r> and <W, x> vanish (a zero filter row) every y_bar is ~0 at
+    once; a rounding-sized residual there must not raise the flag, while the
+    same residual scaled up to the group's noise level must."""
+    spec = tiny_fc_spec(K=2, G=1, cin=32, cout=16)
+    d = synth.draw_layer(spec)
+    W = d["W"].copy()
+    W[3] = 0.0
+    clean = O.masked_forward(W, d["x"], d["r"], d["C"])
+    typical = float(np.sqrt(np.mean(clean["ybar"] ** 2)))
+    tiny_err = O.masked_forward(W, d["x"], d["r"], d["C"], fault=(1, (3,), 1e-7 * typical))
+    assert not tiny_err["flags"].any()
+    big_err = O.masked_forward(W, d["x"], d["r"], d["C"], fault=(1, (3,), 1e-1 * typical))
+    assert big_err["flags"].sum() == 1 and big_err["flags"][0, 3]
+
+
+def test_verify_flags_an_infinity_from_the_accelerator():
+    spec = tiny_fc_spec(K=2, G=1)
+    d = synth.draw_layer(spec)
+    bad = O.masked_forward(d["W"], d["x"], d["r"], d["C"], fault=(0, (1,), float("inf")))
+    assert bad["flags"].sum() == 1 and bad["flags"][0, 1]
 
 
 def test_verify_flags_a_nan_from_the_accelerator():
