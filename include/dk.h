@@ -170,6 +170,28 @@ DK_API dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const flo
                                      const float* gamma_host, float scale, float* dW,
                                      void* stream);
 
+/* Measurement aids (the paper reports time per class of operation, Table 3;
+ * these give the same breakdown per kernel class).  The library always counts
+ * the kernels it launches; with profiling enabled it also brackets every
+ * launch with CUDA events on the launching stream (up to a few thousand
+ * launches between two reads).  dk_profile_read synchronises on the recorded
+ * events, returns the time and number of timed launches of `kind` since the
+ * last reset together with the number of all launches of that kind, and
+ * leaves the records in place; dk_profile_reset clears records and counters. */
+enum {
+  DK_KERNEL_ENCODE = 0,
+  DK_KERNEL_LINEAR_FWD = 1,
+  DK_KERNEL_DECODE_VERIFY = 2,
+  DK_KERNEL_MIX_DELTA = 3,
+  DK_KERNEL_WGRAD = 4,
+  DK_KERNEL_OTHER = 5,
+  DK_KERNEL_KINDS = 6
+};
+DK_API dk_status dk_profile_enable(dk_ctx* ctx, int on);
+DK_API dk_status dk_profile_read(dk_ctx* ctx, int kind, double* ms_total, int64_t* timed_launches,
+                                 int64_t* all_launches);
+DK_API dk_status dk_profile_reset(dk_ctx* ctx);
+
 #ifdef __cplusplus
 }
 #endif

@@ -71,6 +71,10 @@ def _signatures():
         "dk_decode_verify": [vp, pp, vp, vp, vp, vp, vp, vp],
         "dk_masked_linear": [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(dk_fault), vp],
         "dk_linear_bwd_wgrad": [vp, pp, vp, vp, i32, vp, vp, ctypes.c_float, vp, vp],
+        "dk_profile_enable": [vp, ctypes.c_int],
+        "dk_profile_read": [vp, ctypes.c_int, ctypes.POINTER(ctypes.c_double),
+                            ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)],
+        "dk_profile_reset": [vp],
     }
 
 
@@ -164,6 +168,28 @@ class Context:
         off = (-base) % 256
         _check(lib().dk_set_workspace(self._h, ctypes.c_void_p(base + off), self._ws.numel() - off),
                "dk_set_workspace")
+
+
+KERNEL_KINDS = ["encode", "linear_fwd", "decode_verify", "mix_delta", "wgrad", "other"]
+
+
+def dk_profile_enable(ctx: Context, on: bool):
+    _check(lib().dk_profile_enable(ctx.handle, int(on)), "dk_profile_enable")
+
+
+def dk_profile_reset(ctx: Context):
+    _check(lib().dk_profile_reset(ctx.handle), "dk_profile_reset")
+
+
+def dk_profile_read(ctx: Context) -> dict:
+    """{kind: (ms_total, timed_launches, all_launches)} since the last reset."""
+    out = {}
+    for k, name in enumerate(KERNEL_KINDS):
+        ms, nt, na = ctypes.c_double(), ctypes.c_int64(), ctypes.c_int64()
+        _check(lib().dk_profile_read(ctx.handle, k, ctypes.byref(ms), ctypes.byref(nt), ctypes.byref(na)),
+               "dk_profile_read")
+        out[name] = (ms.value, nt.value, na.value)
+    return out
 
 
 def new_verdict(device: int = 0) -> torch.Tensor:

@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "dk_internal.h"
 
@@ -166,6 +167,34 @@ dk_status upload_coefficients(dk_ctx* ctx, const Geom& g, const float* C_host,
   return DK_OK;
 }
 
+struct ProfState {
+  bool on = false;
+  long long launches[DK_KERNEL_KINDS] = {0, 0, 0, 0, 0, 0};
+  std::vector<cudaEvent_t> ev;      // 2 per slot
+  std::vector<int> kind_of;         // per used slot
+  static constexpr size_t kMaxSlots = 8192;
+};
+
+ProfScope::ProfScope(dk_ctx* c, int kind, int nkernels, cudaStream_t s) : ctx(c), slot(-1), st(s) {
+  ProfState* ps = c->prof;
+  if (!ps) return;
+  ps->launches[kind] += nkernels;
+  if (!ps->on || ps->kind_of.size() >= ProfState::kMaxSlots) return;
+  size_t i = ps->kind_of.size();
+  while (ps->ev.size() < 2 * (i + 1)) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return;
+    ps->ev.push_back(e);
+  }
+  if (cudaEventRecord(ps->ev[2 * i], st) != cudaSuccess) return;
+  ps->kind_of.push_back(kind);
+  slot = (int)i;
+}
+
+ProfScope::~ProfScope() {
+  if (slot >= 0) cudaEventRecord(ctx->prof->ev[2 * slot + 1], st);
+}
+
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct WsPlan {
@@ -241,6 +270,8 @@ dk_status dk_create(dk_ctx** out, int device) {
             cudaMalloc(&c->d_cand, kCandCap * sizeof(Candidate)) == cudaSuccess;
   for (int i = 0; ok && i < kCoefSlots; ++i)
     ok = cudaEventCreateWithFlags(&c->slot_ev[i], cudaEventDisableTiming) == cudaSuccess;
+  c->prof = new (std::nothrow) ProfState();
+  ok = ok && c->prof != nullptr;
   if (ok) ok = tc_init(c) == DK_OK;
   if (!ok) { dk_destroy(c); return DK_ERR_CUDA; }
   *out = c;
@@ -254,6 +285,10 @@ dk_status dk_destroy(dk_ctx* c) {
   tc_destroy(c);
   for (int i = 0; i < kCoefSlots; ++i)
     if (c->slot_ev[i]) cudaEventDestroy(c->slot_ev[i]);
+  if (c->prof) {
+    for (cudaEvent_t e : c->prof->ev) cudaEventDestroy(e);
+    delete c->prof;
+  }
   if (c->h_stage) cudaFreeHost(c->h_stage);
   if (c->d_stage) cudaFree(c->d_stage);
   if (c->d_vstats) cudaFree(c->d_vstats);
@@ -292,6 +327,7 @@ dk_status dk_encode(dk_ctx* ctx, const dk_problem* p, const float* x, const floa
   CoefView cv;
   s = upload_coefficients(ctx, g, C_host, nullptr, false, false, st, &cv);
   if (s != DK_OK) return s;
+  ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
   return launch_encode(g, x, r, cv.enc, xbar, ctx->sm_count, st);
 }
 
@@ -305,6 +341,7 @@ dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W, const 
   DeviceGuard dg(ctx->device);
   if (!dg.ok) return DK_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
   return launch_simt_fwd(g, W, xbar, ybar, g.G * g.E, st);
 }
 
@@ -323,10 +360,17 @@ dk_status dk_decode_verify(dk_ctx* ctx, const dk_problem* p, const float* ybar,
   s = upload_coefficients(ctx, g, C_host, nullptr, true, false, st, &cv);
   if (s != DK_OK) return s;
   VerifyScratch vs = verify_scratch(ctx, g);
-  s = launch_verify_begin(g, vs, st);
+  {
+    ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+    s = launch_verify_begin(g, vs, st);
+  }
   if (s != DK_OK) return s;
-  s = launch_decode_verify(g, ybar, cv, bias, y, vs, ctx->sm_count, st);
+  {
+    ProfScope ps(ctx, DK_KERNEL_DECODE_VERIFY, 1, st);
+    s = launch_decode_verify(g, ybar, cv, bias, y, vs, ctx->sm_count, st);
+  }
   if (s != DK_OK) return s;
+  ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
   return launch_verify_finalize(g, cv.nul, vs, verdict, st);
 }
 
@@ -357,20 +401,34 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
   char* ws = static_cast<char*>(ctx->ws);
   float* xbar = xbar_save ? xbar_save : reinterpret_cast<float*>(ws + wp.xbar);
   float* ybar = reinterpret_cast<float*>(ws + wp.ybar);
-  s = launch_encode(g, x, r, cv.enc, xbar, ctx->sm_count, st);
+  {
+    ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
+    s = launch_encode(g, x, r, cv.enc, xbar, ctx->sm_count, st);
+  }
   if (s != DK_OK) return s;
-  s = launch_simt_fwd(g, W, xbar, ybar, g.G * g.E, st);
+  {
+    ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
+    s = launch_simt_fwd(g, W, xbar, ybar, g.G * g.E, st);
+  }
   if (s != DK_OK) return s;
   if (fault) {
     long long idx = ((long long)fault->group * g.E + fault->enc) * g.n_out + fault->out_index;
+    ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
     s = launch_add_fault(ybar, idx, fault->delta, st);
     if (s != DK_OK) return s;
   }
   VerifyScratch vs = verify_scratch(ctx, g);
-  s = launch_verify_begin(g, vs, st);
+  {
+    ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+    s = launch_verify_begin(g, vs, st);
+  }
   if (s != DK_OK) return s;
-  s = launch_decode_verify(g, ybar, cv, bias, y, vs, ctx->sm_count, st);
+  {
+    ProfScope ps(ctx, DK_KERNEL_DECODE_VERIFY, 1, st);
+    s = launch_decode_verify(g, ybar, cv, bias, y, vs, ctx->sm_count, st);
+  }
   if (s != DK_OK) return s;
+  ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
   return launch_verify_finalize(g, cv.nul, vs, verdict, st);
 }
 
@@ -392,9 +450,48 @@ dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* del
   s = upload_coefficients(ctx, g, C_host, gamma_host, true, true, st, &cv);
   if (s != DK_OK) return s;
   float* dtil = reinterpret_cast<float*>(static_cast<char*>(ctx->ws) + wp.dtil);
-  s = launch_mix_delta(g, delta, cv.dmix, dtil, ctx->sm_count, st);
+  {
+    ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
+    s = launch_mix_delta(g, delta, cv.dmix, dtil, ctx->sm_count, st);
+  }
   if (s != DK_OK) return s;
+  ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
   return launch_simt_wgrad(g, dtil, xbar, xbar_rows, scale, dW, ctx->sm_count, st);
+}
+
+dk_status dk_profile_enable(dk_ctx* ctx, int on) {
+  if (!ctx || !ctx->prof) return DK_ERR_INVALID_ARG;
+  ctx->prof->on = on != 0;
+  return DK_OK;
+}
+
+dk_status dk_profile_read(dk_ctx* ctx, int kind, double* ms_total, int64_t* timed_launches,
+                          int64_t* all_launches) {
+  if (!ctx || !ctx->prof || kind < 0 || kind >= DK_KERNEL_KINDS) return DK_ERR_INVALID_ARG;
+  DeviceGuard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  ProfState* ps = ctx->prof;
+  double ms = 0.0;
+  int64_t n = 0;
+  for (size_t i = 0; i < ps->kind_of.size(); ++i) {
+    if (ps->kind_of[i] != kind) continue;
+    float t = 0.f;
+    DK_CUDA_CHECK(cudaEventSynchronize(ps->ev[2 * i + 1]));
+    DK_CUDA_CHECK(cudaEventElapsedTime(&t, ps->ev[2 * i], ps->ev[2 * i + 1]));
+    ms += t;
+    ++n;
+  }
+  if (ms_total) *ms_total = ms;
+  if (timed_launches) *timed_launches = n;
+  if (all_launches) *all_launches = ps->launches[kind];
+  return DK_OK;
+}
+
+dk_status dk_profile_reset(dk_ctx* ctx) {
+  if (!ctx || !ctx->prof) return DK_ERR_INVALID_ARG;
+  ctx->prof->kind_of.clear();
+  for (int k = 0; k < DK_KERNEL_KINDS; ++k) ctx->prof->launches[k] = 0;
+  return DK_OK;
 }
 
 }  // extern "C"

@@ -64,6 +64,8 @@ struct VerifyScratch {
   Candidate* cand;       // [kCandCap]
 };
 
+struct ProfState;
+
 }  // namespace dk
 
 struct dk_ctx {
@@ -79,6 +81,7 @@ struct dk_ctx {
   float* d_vstats;            // kVerifyStatFloats floats + one counter
   dk::Candidate* d_cand;      // kCandCap entries
   void* tc_state;             // tensor-core path state
+  dk::ProfState* prof;        // launch counters and event records
 };
 
 namespace dk {
@@ -110,6 +113,16 @@ dk_status launch_simt_fwd(const Geom& g, const float* W, const float* xbar, floa
 // dW = scale * sum_n <dtil[n], xbar[row(n)]> with row(n) = (n/(K+1))*xbar_rows + n%(K+1)
 dk_status launch_simt_wgrad(const Geom& g, const float* dtil, const float* xbar, int xbar_rows,
                             float scale, float* dW, int sm_count, cudaStream_t st);
+
+// Launch accounting: counts `nkernels` launches of `kind` and, when profiling
+// is on, brackets them with a pair of events on `st`.
+struct ProfScope {
+  dk_ctx* ctx;
+  int slot;
+  cudaStream_t st;
+  ProfScope(dk_ctx* c, int kind, int nkernels, cudaStream_t s);
+  ~ProfScope();
+};
 
 // tensor-core path (dk_tc.cu)
 dk_status tc_init(dk_ctx* ctx);
