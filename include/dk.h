@@ -170,6 +170,29 @@ DK_API dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const flo
                                      const float* gamma_host, float scale, float* dW,
                                      void* stream);
 
+/* dk_decode_verify without allocation and without a context.  The paper has
+ * no counterpart for this call; it exists for callers that may not allocate
+ * device memory where they need the check: code confined to a fixed memory
+ * budget, sections where the device-wide synchronisation implied by an
+ * allocation is not acceptable, and processes that must not create a dk_ctx
+ * (dk_create allocates).  It computes exactly what dk_decode_verify computes,
+ * with the same arguments except that the CUDA device ordinal replaces the
+ * context.  All scratch memory (coefficient tables, per-group statistics, the
+ * suspect list) is one fixed array of about 1.2 MiB inside the library image,
+ * which every GPU that loads the library holds until the process exits.
+ *  - Limits: G*K*(K+1)*2 + G*(K+2) <= 16384 and G*(K+3) <= 16384; larger
+ *    problems are refused with DK_ERR_WORKSPACE and nothing is launched.
+ *  - The first call on a device looks up the array's device address (once per
+ *    device); make that first call outside any stream capture.
+ *  - Every call uses the same array: two calls whose kernels can overlap on
+ *    the GPU (different streams, different threads) race on it.  Calls on
+ *    one stream are safe; each call clears the state it needs.
+ *  - It calls no cudaMalloc/cudaFree and no allocating library routine; the
+ *    caller still provides ybar, y, bias and the dk_verdict on the device. */
+DK_API dk_status dk_decode_verify_static(int device, const dk_problem* p, const float* ybar,
+                                         const float* C_host, const float* bias, float* y,
+                                         dk_verdict* verdict, void* stream);
+
 /* Measurement aids (the paper reports time per class of operation, Table 3;
  * these give the same breakdown per kernel class).  The library always counts
  * the kernels it launches; with profiling enabled it also brackets every

@@ -71,6 +71,7 @@ def _signatures():
         "dk_decode_verify": [vp, pp, vp, vp, vp, vp, vp, vp],
         "dk_masked_linear": [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(dk_fault), vp],
         "dk_linear_bwd_wgrad": [vp, pp, vp, vp, i32, vp, vp, ctypes.c_float, vp, vp],
+        "dk_decode_verify_static": [ctypes.c_int, pp, vp, vp, vp, vp, vp, vp],
         "dk_profile_enable": [vp, ctypes.c_int],
         "dk_profile_read": [vp, ctypes.c_int, ctypes.POINTER(ctypes.c_double),
                             ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)],
@@ -218,6 +219,14 @@ def dk_linear_fwd(ctx: Context, p: dk_problem, W, xbar, ybar):
 def dk_decode_verify(ctx: Context, p: dk_problem, ybar, C: np.ndarray, bias, y, verdict):
     _check(lib().dk_decode_verify(ctx.handle, ctypes.byref(p), _dev(ybar), _host(C), _dev(bias), _dev(y),
                                   ctypes.c_void_p(verdict.data_ptr()), _stream()), "dk_decode_verify")
+
+
+def dk_decode_verify_static(device: int, p: dk_problem, ybar, C: np.ndarray, bias, y, verdict):
+    """Same result as dk_decode_verify, for callers that may not allocate: no
+    context, scratch in a fixed array inside the library (see include/dk.h)."""
+    _check(lib().dk_decode_verify_static(device, ctypes.byref(p), _dev(ybar), _host(C), _dev(bias), _dev(y),
+                                         ctypes.c_void_p(verdict.data_ptr()), _stream()),
+           "dk_decode_verify_static")
 
 
 def dk_masked_linear(ctx: Context, p: dk_problem, W, x, r, C: np.ndarray, bias, y, xbar_save, verdict,
