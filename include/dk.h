@@ -91,7 +91,7 @@ typedef struct {
   int32_t ok;           /* 1 = every element consistent, 0 = at least one flagged */
   uint32_t n_flagged;   /* number of flagged (group, output element) pairs        */
   int64_t first_index;  /* smallest flagged g*n_out + e (e in memory order), or -1 */
-  float max_ratio;      /* max |rho| / sum_i |n_i||ybar_i| over all elements      */
+  float max_ratio;      /* max over elements of |rho| / s_g (see dk_decode_verify) */
   int32_t status;       /* dk_status raised on the device (0 = none)              */
 } dk_verdict;
 
@@ -140,7 +140,10 @@ DK_API dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W,
 /* Eq. 2 and Section 4.4.  Per group and output element e:
  *   [y_0..y_{K-1}, z] = C_sq^{-1} . [ybar_0..ybar_K]      (z = <W,r> is dropped)
  *   rho = sum_i n[i]*ybar_i with n^T C = 0, n[K+1] = 1     (redundant equation)
- *   flagged iff not (|rho| <= tau * sum_i |n[i]|*|ybar_i|)
+ *   s_e = sum_i |n[i]|*|ybar_i[e]|,  s_g = sum_i |n[i]|*rms_e(ybar_i)
+ *   flagged iff not (|rho| <= tau * max(s_e, s_g)), or s_e is not finite
+ * (the paper compares exactly in a finite field; in floating point the
+ * residual is compared with the scale of the numbers it was formed from).
  * ybar: [G*(K+2)][n_out] -> y: [G*K][n_out]; bias[cout] (nullable) is added
  * after decoding; *verdict (device) receives the summary.  HBM-bound. */
 DK_API dk_status dk_decode_verify(dk_ctx* ctx, const dk_problem* p, const float* ybar,
