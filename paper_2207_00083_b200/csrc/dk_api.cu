@@ -198,15 +198,24 @@ ProfScope::~ProfScope() {
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct WsPlan {
-  size_t xbar, ybar, dtil, total;
+  size_t xbar, ybar, dtil, w_hi, w_lo, xb_hi, xb_lo, total;
 };
 
+// One layout serves every entry point: fp32 encodings (when the caller does
+// not store them), y_bar of the unfused path, mixed deltas of wgrad, and the
+// TF32 hi/lo split copies of W and x_bar that feed the tensor-core kernel.
 static WsPlan plan_workspace(const Geom& g) {
   WsPlan w;
   size_t off = 0;
-  w.xbar = off; off += align_up((size_t)g.G * g.E * g.n_in * sizeof(float), 256);
-  w.ybar = off; off += align_up((size_t)g.G * g.E * g.n_out * sizeof(float), 256);
-  w.dtil = off; off += align_up((size_t)g.G * (g.K + 1) * g.n_out * sizeof(float), 256);
+  const size_t xb = align_up((size_t)g.G * g.E * g.n_in * sizeof(float), 1024);
+  const size_t wb = align_up((size_t)g.cout * g.kc * sizeof(float), 1024);
+  w.xbar = off; off += xb;
+  w.ybar = off; off += align_up((size_t)g.G * g.E * g.n_out * sizeof(float), 1024);
+  w.dtil = off; off += align_up((size_t)g.G * (g.K + 1) * g.n_out * sizeof(float), 1024);
+  w.w_hi = off; off += wb;
+  w.w_lo = off; off += wb;
+  w.xb_hi = off; off += xb;
+  w.xb_lo = off; off += xb;
   w.total = off;
   return w;
 }
@@ -341,6 +350,23 @@ dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W, const 
   DeviceGuard dg(ctx->device);
   if (!dg.ok) return DK_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (tc_fwd_supported(ctx, g)) {
+    WsPlan wp = plan_workspace(g);
+    if (!ctx->ws || ctx->ws_bytes < wp.total) return DK_ERR_WORKSPACE;
+    char* ws = static_cast<char*>(ctx->ws);
+    float* w_hi = reinterpret_cast<float*>(ws + wp.w_hi);
+    float* w_lo = reinterpret_cast<float*>(ws + wp.w_lo);
+    float* xb_hi = reinterpret_cast<float*>(ws + wp.xb_hi);
+    float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
+    {
+      ProfScope ps(ctx, DK_KERNEL_OTHER, 2, st);
+      s = tc_split(W, w_hi, w_lo, (long long)g.cout * g.kc, ctx->sm_count, st);
+      if (s == DK_OK) s = tc_split(xbar, xb_hi, xb_lo, (long long)g.G * g.E * g.n_in, ctx->sm_count, st);
+    }
+    if (s != DK_OK) return s;
+    ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
+    return tc_linear_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, ybar, nullptr, st);
+  }
   ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
   return launch_simt_fwd(g, W, xbar, ybar, g.G * g.E, st);
 }
@@ -399,6 +425,34 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
   s = upload_coefficients(ctx, g, C_host, nullptr, true, false, st, &cv);
   if (s != DK_OK) return s;
   char* ws = static_cast<char*>(ctx->ws);
+  if (tc_fwd_supported(ctx, g)) {
+    // tensor-core path: encode+split pre-pass, then one GEMM whose epilogue
+    // decodes and gathers the integrity statistics; y_bar never reaches HBM
+    float* w_hi = reinterpret_cast<float*>(ws + wp.w_hi);
+    float* w_lo = reinterpret_cast<float*>(ws + wp.w_lo);
+    float* xb_hi = reinterpret_cast<float*>(ws + wp.xb_hi);
+    float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
+    VerifyScratch vs = verify_scratch(ctx, g);
+    {
+      ProfScope ps(ctx, DK_KERNEL_OTHER, 2, st);
+      s = tc_split(W, w_hi, w_lo, (long long)g.cout * g.kc, ctx->sm_count, st);
+      if (s == DK_OK) s = launch_verify_begin(g, vs, st);
+    }
+    if (s != DK_OK) return s;
+    {
+      ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
+      s = tc_encode_split(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, ctx->sm_count, st);
+    }
+    if (s != DK_OK) return s;
+    {
+      ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
+      s = tc_masked_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, cv, bias, y, vs,
+                        reinterpret_cast<int*>(vs.count + 1), fault, st);
+    }
+    if (s != DK_OK) return s;
+    ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+    return launch_verify_finalize(g, cv.nul, vs, verdict, st);
+  }
   float* xbar = xbar_save ? xbar_save : reinterpret_cast<float*>(ws + wp.xbar);
   float* ybar = reinterpret_cast<float*>(ws + wp.ybar);
   {

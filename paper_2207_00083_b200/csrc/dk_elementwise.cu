@@ -85,7 +85,10 @@ __global__ void add_fault_kernel(float* ybar, long long idx, float delta) { ybar
 __global__ void verify_begin_kernel(float* stats, int nstats, unsigned int* count) {
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nstats; i += gridDim.x * blockDim.x)
     stats[i] = 0.f;
-  if (blockIdx.x == 0 && threadIdx.x == 0) *count = 0u;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    count[0] = 0u;   // suspects appended
+    count[1] = 0u;   // status word a producing kernel may raise (DK_ERR_TIMEOUT)
+  }
 }
 
 // s_g = sum_i |n_i| * rms(ybar_i) for group g from the accumulated sums of squares.
@@ -142,15 +145,15 @@ verify_finalize_kernel(const float* sumsq, const int* maxrho, const unsigned int
       first = s_f[w] < first ? s_f[w] : first;
       maxr = fmaxf(maxr, s_r[w]);
     }
-    int status = 0;
+    int status = (int)count[1];   // raised by a producing kernel that gave up: nothing can be trusted
     if (total > kCandCap) {
       // more suspects than the list holds: everything beyond it counts as flagged
       nflag += total - kCandCap;
-      status = DK_ERR_WORKSPACE;
+      if (status == 0) status = DK_ERR_WORKSPACE;
     }
-    vd->ok = nflag == 0 ? 1 : 0;
+    vd->ok = (nflag == 0 && status == 0) ? 1 : 0;
     vd->n_flagged = nflag;
-    vd->first_index = nflag ? first : -1;
+    vd->first_index = (first != 0x7fffffffffffffffLL) ? first : -1;
     vd->max_ratio = maxr;
     vd->status = status;
   }

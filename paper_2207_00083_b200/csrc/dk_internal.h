@@ -127,6 +127,23 @@ struct ProfScope {
 // tensor-core path (dk_tc.cu)
 dk_status tc_init(dk_ctx* ctx);
 void tc_destroy(dk_ctx* ctx);
+// true when the tensor-core kernel takes this geometry (channels-last,
+// stride 1, cin % 4 == 0, not DK_FP32_SIMT)
+bool tc_fwd_supported(const dk_ctx* ctx, const Geom& g);
+// hi = tf32(src), lo = tf32(src - hi); n % 4 == 0
+dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_count, cudaStream_t st);
+// Eq. 1 with the split fused in; `full` (nullable) also receives the fp32 encodings
+dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const float* enc, float* full,
+                          float* hi, float* lo, int sm_count, cudaStream_t st);
+// y_bar = <W, x_bar> from split operands
+dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
+                        const float* xb_hi, const float* xb_lo, float* ybar, int* status_word,
+                        cudaStream_t st);
+// same contraction with decode + integrity statistics in the epilogue
+dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
+                        const float* xb_hi, const float* xb_lo, const CoefView& cv, const float* bias,
+                        float* y, const VerifyScratch& vs, int* status_word, const dk_fault* fault,
+                        cudaStream_t st);
 
 }  // namespace dk
 

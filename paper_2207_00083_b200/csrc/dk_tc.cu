@@ -1,9 +1,318 @@
-// Tensor-core path (tcgen05 / TMEM / TMA).
+// Host side of the tensor-core path: tensor maps, tile planning, launches, and
+// the HBM-bound pre-passes that write the TF32 hi/lo split operands.
+#include <cuda.h>
+
+#include <new>
+
 #include "dk_internal.h"
+#include "dk_tc_kernel.cuh"
 
 namespace dk {
+namespace {
 
-dk_status tc_init(dk_ctx* ctx) { ctx->tc_state = nullptr; return DK_OK; }
-void tc_destroy(dk_ctx*) {}
+using namespace tc;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+struct TcState {
+  EncodeTiledFn encode;
+  int smem_optin;
+};
+
+constexpr int kBK = 32;          // k-block: 32 fp32 = one 128-byte swizzle span per row
+constexpr int kChunk = 2;        // k-blocks accumulated in TMEM between promotions
+
+// ---------------------------------------------------------------------------
+// HBM-bound pre-passes: TF32 hi/lo split, alone or fused with the encoder
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+split_tf32_kernel(const float4* __restrict__ src, float4* __restrict__ hi, float4* __restrict__ lo, long long n4) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (long long)gridDim.x * blockDim.x) {
+    float4 v = __ldg(src + i), h, l;
+    h.x = to_tf32(v.x); l.x = to_tf32(v.x - h.x);
+    h.y = to_tf32(v.y); l.y = to_tf32(v.y - h.y);
+    h.z = to_tf32(v.z); l.z = to_tf32(v.z - h.z);
+    h.w = to_tf32(v.w); l.w = to_tf32(v.w - h.w);
+    hi[i] = h;
+    lo[i] = l;
+  }
+}
+
+// Eq. 1 with the split fused in: reads the K inputs and the noise once,
+// writes the K+2 encodings as hi/lo pairs (and in full when `full` is given).
+template <int K>
+__global__ void __launch_bounds__(256)
+encode_split_kernel(const float* __restrict__ x, const float* __restrict__ r, const float* __restrict__ enc,
+                    float* __restrict__ full, float* __restrict__ hi, float* __restrict__ lo, long long n) {
+  constexpr int K1 = K + 1, E = K + 2;
+  const int g = blockIdx.y;
+  float c[E][K1];
+#pragma unroll
+  for (int i = 0; i < E; ++i)
+#pragma unroll
+    for (int k = 0; k < K1; ++k) c[i][k] = __ldg(enc + ((size_t)g * E + i) * K1 + k);
+  const float* xg = x + (size_t)g * K * n;
+  const float* rg = r + (size_t)g * n;
+  const size_t ob = (size_t)g * E * n;
+  const long long n4 = n / 4;
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += (long long)gridDim.x * blockDim.x) {
+    float4 s[K1];
+#pragma unroll
+    for (int k = 0; k < K; ++k) s[k] = __ldg(reinterpret_cast<const float4*>(xg + (size_t)k * n) + q);
+    s[K] = __ldg(reinterpret_cast<const float4*>(rg) + q);
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+      float4 o, h, l;
+      o.x = c[i][K] * s[K].x; o.y = c[i][K] * s[K].y; o.z = c[i][K] * s[K].z; o.w = c[i][K] * s[K].w;
+#pragma unroll
+      for (int k = 0; k < K; ++k) {
+        o.x = fmaf(c[i][k], s[k].x, o.x); o.y = fmaf(c[i][k], s[k].y, o.y);
+        o.z = fmaf(c[i][k], s[k].z, o.z); o.w = fmaf(c[i][k], s[k].w, o.w);
+      }
+      h.x = to_tf32(o.x); l.x = to_tf32(o.x - h.x);
+      h.y = to_tf32(o.y); l.y = to_tf32(o.y - h.y);
+      h.z = to_tf32(o.z); l.z = to_tf32(o.z - h.z);
+      h.w = to_tf32(o.w); l.w = to_tf32(o.w - h.w);
+      const size_t off = ob + (size_t)i * n;
+      if (full != nullptr) reinterpret_cast<float4*>(full + off)[q] = o;
+      reinterpret_cast<float4*>(hi + off)[q] = h;
+      reinterpret_cast<float4*>(lo + off)[q] = l;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// tile planning
+// ---------------------------------------------------------------------------
+struct Tiling {
+  int P, bw, bh, bg, WT, HT, GT, MT, ntiles, KB, CB, nstages, BN;
+  size_t smem_bytes;
+};
+
+template <int BK>
+bool plan_tiling(const Geom& g, int smem_optin, Tiling* t) {
+  const int E = g.E;
+  const int P = tile_pixels(g.K);
+  // Box shape bw x bh x bg with bw*bh*bg = P (bw, bh powers of two): the one
+  // that covers the fewest out-of-range positions; ties go to wider rows.
+  t->P = P;
+  t->bw = t->bh = t->bg = 1;
+  long long best = -1;
+  for (int bw = 1; bw <= P; bw *= 2)
+    for (int bh = 1; bw * bh <= P; bh *= 2) {
+      if (P % (bw * bh)) continue;
+      const int bg = P / (bw * bh);
+      if (bg > 256) continue;
+      const long long cost = (long long)((g.wo + bw - 1) / bw) * bw * ((g.ho + bh - 1) / bh) * bh *
+                             ((g.G + bg - 1) / bg) * bg;
+      if (best < 0 || cost < best || (cost == best && (bw > t->bw || (bw == t->bw && bh > t->bh)))) {
+        best = cost; t->bw = bw; t->bh = bh; t->bg = bg;
+      }
+    }
+  if (best < 0) return false;
+  t->WT = (g.wo + t->bw - 1) / t->bw;
+  t->HT = (g.ho + t->bh - 1) / t->bh;
+  t->GT = (g.G + t->bg - 1) / t->bg;
+  t->MT = (g.cout + BM - 1) / BM;
+  long long nt = (long long)t->WT * t->HT * t->GT * t->MT;
+  if (nt > 0x7fffffffLL) return false;
+  t->ntiles = (int)nt;
+  t->CB = (g.cin + BK - 1) / BK;
+  t->KB = t->CB * g.kh * g.kw;
+  t->BN = E * P;
+  const size_t stage = 2 * ((size_t)BM * BK * 4 + (size_t)t->BN * BK * 4);
+  const size_t ctrl = 1024 + 256;   // alignment slack + barriers
+  int ns = (int)(((size_t)smem_optin - ctrl) / stage);
+  if (ns > kMaxStages) ns = kMaxStages;
+  if (ns < 2) return false;
+  t->nstages = ns;
+  t->smem_bytes = (size_t)ns * stage + ctrl;
+  return true;
+}
+
+bool encode_map(const TcState* ts, CUtensorMap* m, const void* base, int rank, const cuuint64_t* dims,
+                const cuuint64_t* strides_bytes, const cuuint32_t* box, int swz_bytes) {
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUtensorMapSwizzle sw = swz_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                           : (swz_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+  CUresult r = ts->encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<void*>(base), dims,
+                          strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <int BK, int MODE, int K>
+dk_status launch_one(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
+                     const float* xb_hi, const float* xb_lo, TcParams& prm, int sm_count, cudaStream_t st) {
+  CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo;
+  const int taps = g.kh * g.kw;
+  {
+    cuuint64_t dims[3] = {(cuuint64_t)g.cin, (cuuint64_t)taps, (cuuint64_t)g.cout};
+    cuuint64_t str[2] = {(cuuint64_t)g.cin * 4, (cuuint64_t)g.cin * taps * 4};
+    cuuint32_t box[3] = {(cuuint32_t)BK, 1, (cuuint32_t)BM};
+    if (!encode_map(ts, &ma_hi, w_hi, 3, dims, str, box, BK * 4) ||
+        !encode_map(ts, &ma_lo, w_lo, 3, dims, str, box, BK * 4))
+      return DK_ERR_CUDA;
+  }
+  {
+    cuuint64_t dims[5] = {(cuuint64_t)g.cin, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.E, (cuuint64_t)g.G};
+    cuuint64_t str[4] = {(cuuint64_t)g.cin * 4, (cuuint64_t)g.cin * g.w * 4, (cuuint64_t)g.n_in * 4,
+                         (cuuint64_t)g.n_in * g.E * 4};
+    cuuint32_t box[5] = {(cuuint32_t)BK, (cuuint32_t)tl.bw, (cuuint32_t)tl.bh, 1, (cuuint32_t)tl.bg};
+    if (!encode_map(ts, &mb_hi, xb_hi, 5, dims, str, box, BK * 4) ||
+        !encode_map(ts, &mb_lo, xb_lo, 5, dims, str, box, BK * 4))
+      return DK_ERR_CUDA;
+  }
+  auto kern = tc_fwd_kernel<BK, MODE, K>;
+  // The kernel re-partitions registers between its warpgroups and would wait
+  // forever if the pool it was launched with were smaller than it assumes.
+  cudaFuncAttributes fa;
+  DK_CUDA_CHECK(cudaFuncGetAttributes(&fa, kern));
+  if (fa.numRegs * kThreadsTc < 40 * 128 + 232 * 256) return DK_ERR_UNSUPPORTED;
+  DK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tl.smem_bytes));
+  int grid = tl.ntiles < sm_count ? tl.ntiles : sm_count;
+  kern<<<grid, kThreadsTc, tl.smem_bytes, st>>>(ma_hi, ma_lo, mb_hi, mb_lo, prm);
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+template <int BK, int MODE>
+dk_status launch_k(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
+                   const float* xb_hi, const float* xb_lo, TcParams& prm, int sm_count, cudaStream_t st) {
+  switch (g.K) {
+    case 1: return launch_one<BK, MODE, 1>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+    case 2: return launch_one<BK, MODE, 2>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+    case 3: return launch_one<BK, MODE, 3>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+    case 4: return launch_one<BK, MODE, 4>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+    case 5: return launch_one<BK, MODE, 5>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+    case 6: return launch_one<BK, MODE, 6>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+    case 7: return launch_one<BK, MODE, 7>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+    case 8: return launch_one<BK, MODE, 8>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+  }
+  return DK_ERR_SHAPE;
+}
+
+void fill_params(const Geom& g, const Tiling& tl, TcParams* p) {
+  p->bw = tl.bw; p->bh = tl.bh; p->bg = tl.bg;
+  p->WT = tl.WT; p->HT = tl.HT; p->GT = tl.GT; p->MT = tl.MT;
+  p->ntiles = tl.ntiles; p->KB = tl.KB; p->CB = tl.CB;
+  p->chunk = kChunk;
+  p->kw = g.kw; p->pad = g.pad; p->nstages = tl.nstages;
+  p->cout = g.cout; p->ho = g.ho; p->wo = g.wo; p->G = g.G;
+  p->n_out = g.n_out;
+  p->out = nullptr; p->dec = p->decl = p->nul = p->bias = nullptr;
+  p->vs.sumsq = nullptr; p->vs.maxrho = nullptr; p->vs.count = nullptr; p->vs.cand = nullptr;
+  p->tau = g.tol;
+  p->status = nullptr;
+  p->f_group = -1; p->f_enc = p->f_co = p->f_oh = p->f_ow = 0;
+  p->f_delta = 0.f;
+}
+
+}  // namespace
+
+dk_status tc_init(dk_ctx* ctx) {
+  TcState* ts = new (std::nothrow) TcState();
+  if (!ts) return DK_ERR_CUDA;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+    delete ts;
+    return DK_ERR_CUDA;
+  }
+  ts->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  int optin = 0;
+  if (cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device) != cudaSuccess) {
+    delete ts;
+    return DK_ERR_CUDA;
+  }
+  ts->smem_optin = optin;
+  ctx->tc_state = ts;
+  return DK_OK;
+}
+
+void tc_destroy(dk_ctx* ctx) {
+  delete static_cast<TcState*>(ctx->tc_state);
+  ctx->tc_state = nullptr;
+}
+
+bool tc_fwd_supported(const dk_ctx* ctx, const Geom& g) {
+  if (g.precision == DK_FP32_SIMT || ctx->tc_state == nullptr) return false;
+  if (g.layout != DK_NHWC || g.stride != 1 || (g.cin % 4) != 0) return false;
+  Tiling tl;
+  return plan_tiling<kBK>(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, &tl);
+}
+
+dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_count, cudaStream_t st) {
+  if (n % 4) return DK_ERR_SHAPE;
+  long long n4 = n / 4;
+  long long blocks = (n4 + 255) / 256;
+  if (blocks > (long long)sm_count * 16) blocks = (long long)sm_count * 16;
+  if (blocks < 1) blocks = 1;
+  split_tf32_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(src),
+                                                      reinterpret_cast<float4*>(hi), reinterpret_cast<float4*>(lo), n4);
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const float* enc, float* full,
+                          float* hi, float* lo, int sm_count, cudaStream_t st) {
+  if (g.n_in % 4 || g.G > 65535) return DK_ERR_SHAPE;
+  long long n4 = g.n_in / 4;
+  long long want = (n4 + 255) / 256;
+  long long cap = ((long long)sm_count * 16 + g.G - 1) / g.G;
+  if (want > cap) want = cap;
+  if (want < 1) want = 1;
+  dim3 grid((unsigned)want, (unsigned)g.G);
+#define DK_ENC_CASE(KK) \
+  case KK: encode_split_kernel<KK><<<grid, 256, 0, st>>>(x, r, enc, full, hi, lo, g.n_in); break;
+  switch (g.K) {
+    DK_ENC_CASE(1) DK_ENC_CASE(2) DK_ENC_CASE(3) DK_ENC_CASE(4)
+    DK_ENC_CASE(5) DK_ENC_CASE(6) DK_ENC_CASE(7) DK_ENC_CASE(8)
+    default: return DK_ERR_SHAPE;
+  }
+#undef DK_ENC_CASE
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
+                        const float* xb_lo, float* ybar, int* status_word, cudaStream_t st) {
+  TcState* ts = static_cast<TcState*>(ctx->tc_state);
+  Tiling tl;
+  if (!plan_tiling<kBK>(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
+  TcParams prm;
+  fill_params(g, tl, &prm);
+  prm.out = ybar;
+  prm.status = status_word;
+  return launch_k<kBK, MODE_YBAR>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
+}
+
+dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
+                        const float* xb_lo, const CoefView& cv, const float* bias, float* y,
+                        const VerifyScratch& vs, int* status_word, const dk_fault* fault, cudaStream_t st) {
+  TcState* ts = static_cast<TcState*>(ctx->tc_state);
+  Tiling tl;
+  if (!plan_tiling<kBK>(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
+  TcParams prm;
+  fill_params(g, tl, &prm);
+  prm.out = y;
+  prm.dec = cv.dec; prm.decl = cv.decl; prm.nul = cv.nul; prm.bias = bias;
+  prm.vs = vs;
+  prm.status = status_word;
+  if (fault) {
+    prm.f_group = fault->group;
+    prm.f_enc = fault->enc;
+    long long pix = fault->out_index / g.cout;
+    prm.f_co = (int)(fault->out_index - pix * g.cout);
+    prm.f_oh = (int)(pix / g.wo);
+    prm.f_ow = (int)(pix - (long long)prm.f_oh * g.wo);
+    prm.f_delta = fault->delta;
+  }
+  return launch_k<kBK, MODE_DECODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
+}
 
 }  // namespace dk

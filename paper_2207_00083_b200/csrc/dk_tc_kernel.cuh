@@ -1,0 +1,461 @@
+// Device side of the tensor-core path: PTX wrappers (TMA, mbarrier, tcgen05)
+// and the persistent warp-specialised 3xTF32 implicit-GEMM kernel.
+//
+// Arithmetic.  Every fp32 operand v is split as v = hi + lo with
+// hi = tf32(v), lo = tf32(v - hi) (round to nearest).  The product keeps
+// W_hi*x_hi + W_hi*x_lo + W_lo*x_hi and drops W_lo*x_lo (~2^-22 relative).
+// The tensor pipe adds into its fp32 accumulator with truncation; measured on
+// B200, a contraction of length 4608 accumulated entirely in TMEM is off by
+// 3.6e-5 (relative, max norm), which the decoder amplifies ~200x at noise
+// sigma 100.  So TMEM only ever accumulates a short chunk of k-blocks; the
+// epilogue warps add the chunks into fp32 registers with round-to-nearest.
+//
+// Tiling.  GEMM M = cout (128 rows of W per CTA tile = 128 TMEM lanes),
+// N = encodings x pixels.  One N tile holds P output pixels for ALL K+2
+// encodings of the same virtual batch(es): column e*P + p.  A thread of the
+// epilogue owns one TMEM lane (one output channel) and half of the pixels,
+// and sees every encoding of each of them: decoding and the redundant-equation
+// residual are thread-local.  The P pixels are a box bw x bh x bg (columns,
+// rows, groups) of the output; for filter tap (u,v) the operand tile is the
+// same box of the channels-last input shifted by (u-pad, v-pad), fetched by
+// one TMA box per encoding; out-of-image coordinates are zero-filled by the
+// TMA unit, which implements the zero padding.
+//
+// Pipeline.  Persistent CTAs (one per SM): warp 0 issues TMA loads into a ring
+// of shared-memory stages, warp 1 issues tcgen05.mma and commits, warps 4-11
+// (two warpgroups, which take the registers warpgroup 0 gives up) drain the
+// double-buffered TMEM accumulator chunk by chunk.  Every mbarrier
+// wait is bounded; on expiry the CTA raises DK_ERR_TIMEOUT in the status
+// word, lets in-flight copies land, frees TMEM and returns.
+#pragma once
+
+#include <cuda.h>
+
+#include "dk_internal.h"
+
+namespace dk {
+namespace tc {
+
+constexpr int BM = 128;            // output channels per tile = TMEM lanes
+constexpr int kEpiWarps = 8;
+constexpr int kThreadsTc = 32 * (4 + kEpiWarps);   // warpgroup 0: TMA, MMA, two idle warps
+constexpr int kMaxStages = 8;
+constexpr unsigned kSpinCap = 1u << 22;
+constexpr int MODE_YBAR = 0, MODE_DECODE = 1;
+
+// Pixels per encoding in one N tile, by virtual-batch size: (K+2)*P is a legal
+// UMMA N (multiple of 16, <= 256) and each epilogue thread keeps (K+2)*P/2
+// accumulators in registers.
+__host__ __device__ constexpr int tile_pixels(int K) {
+  return K == 1 ? 64 : K == 2 ? 48 : (K == 3 || K == 4) ? 32 : 16;
+}
+
+struct TcParams {
+  // tiling
+  int bw, bh, bg;              // box shape of the P pixels
+  int WT, HT, GT, MT;          // tiles along width, height, groups, cout
+  int ntiles;
+  int KB, CB;                  // k-blocks in total and per filter tap
+  int chunk;                   // k-blocks accumulated in TMEM before promotion
+  int kw, pad;
+  int nstages;
+  // problem
+  int cout, ho, wo, G;
+  long long n_out;
+  // outputs / epilogue inputs
+  float* out;                  // MODE_YBAR: ybar [G*E][ho][wo][cout]; MODE_DECODE: y [G*K][ho][wo][cout]
+  const float* dec;
+  const float* decl;
+  const float* nul;
+  const float* bias;
+  VerifyScratch vs;
+  float tau;
+  int* status;                 // device word that receives DK_ERR_TIMEOUT
+  // fault injection (MODE_DECODE): group < 0 disables
+  int f_group, f_enc, f_co, f_oh, f_ow;
+  float f_delta;
+};
+
+// ---------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when the
+// barrier did not complete within kSpinCap polls or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (unsigned i = 0; i < kSpinCap; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
+                                            int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
+                                            int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
+  uint32_t r[8];
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float to_tf32(float v) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+  return __uint_as_float(r);
+}
+
+// Shared-memory matrix descriptor of a K-major operand tile whose rows are
+// SWZ bytes long (one swizzle span per row), rows packed, 8-row groups SWZ*8
+// bytes apart.
+template <int SWZ>
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
+  constexpr uint64_t layout = (SWZ == 128) ? 2ull : (SWZ == 64 ? 4ull : 6ull);
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+  d |= (uint64_t)1 << 16;                             // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)((SWZ * 8) >> 4) << 32;              // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                             // descriptor version of this architecture
+  d |= layout << 61;
+  return d;
+}
+
+// ---------------------------------------------------------------------------
+// the GEMM kernel
+// ---------------------------------------------------------------------------
+template <int BK, int MODE, int K>
+__global__ void __launch_bounds__(kThreadsTc, 1)
+tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
+              const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
+              const TcParams p) {
+  constexpr int E = K + 2, K1 = K + 1;
+  constexpr int P = tile_pixels(K), PH = P / 2;
+  constexpr int BN = E * P;
+  constexpr int SWZ = BK * 4;
+  constexpr int A_BYTES = BM * BK * 4;
+  constexpr int B_BYTES = BN * BK * 4;
+  constexpr int STAGE_BYTES = 2 * (A_BYTES + B_BYTES);
+  static_assert(BN % 16 == 0 && BN <= 256 && PH % 8 == 0, "illegal tile");
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                                         ~static_cast<uintptr_t>(1023));
+  unsigned char* ctrl = smem + (size_t)p.nstages * STAGE_BYTES;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(ctrl);
+  uint64_t* empty_bar = full_bar + kMaxStages;
+  uint64_t* tfull_bar = empty_bar + kMaxStages;
+  uint64_t* tempty_bar = tfull_bar + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nchunks = (p.KB + p.chunk - 1) / p.chunk;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.nstages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + b, 1); mbar_init(tempty_bar + b, kEpiWarps); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // Register re-partitioning.  The CTA's register pool is fixed at launch
+  // (168 per thread x 384 threads for this launch bound); setmaxnreg.inc BLOCKS
+  // until the pool can serve it, so the two requests below must fit the pool.
+  static_assert(40 * 128 + 232 * 256 <= 168 * kThreadsTc, "setmaxnreg budget exceeds the CTA's register pool");
+  if (warp < 4) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      for (int t = blockIdx.x; alive && t < p.ntiles; t += gridDim.x) {
+        const int mt = t % p.MT;
+        int nt = t / p.MT;
+        const int wt = nt % p.WT; nt /= p.WT;
+        const int ht = nt % p.HT;
+        const int gt = nt / p.HT;
+        const int x0 = wt * p.bw - p.pad, y0 = ht * p.bh - p.pad, g0 = gt * p.bg, m0 = mt * BM;
+        for (int kb = 0; kb < p.KB; ++kb) {
+          if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) { alive = false; break; }
+          const int tap = kb / p.CB, c0 = (kb - tap * p.CB) * BK;
+          const int u = tap / p.kw, v = tap - u * p.kw;
+          unsigned char* st = smem + (size_t)stage * STAGE_BYTES;
+          mbar_expect_tx(full_bar + stage, (uint32_t)STAGE_BYTES);
+          tma_load_3d(st, &map_a_hi, full_bar + stage, c0, tap, m0);
+          tma_load_3d(st + A_BYTES, &map_a_lo, full_bar + stage, c0, tap, m0);
+          unsigned char* bh = st + 2 * A_BYTES;
+          unsigned char* bl = bh + B_BYTES;
+          constexpr int SUB = P * BK * 4;
+#pragma unroll 1
+          for (int e = 0; e < E; ++e) {
+            tma_load_5d(bh + e * SUB, &map_b_hi, full_bar + stage, c0, x0 + v, y0 + u, e, g0);
+            tma_load_5d(bl + e * SUB, &map_b_lo, full_bar + stage, c0, x0 + v, y0 + u, e, g0);
+          }
+          if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) |
+                                 ((uint32_t)(BM >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t acc_it = 0;     // chunks issued so far (all tiles)
+      bool alive = true;
+      for (int t = blockIdx.x; alive && t < p.ntiles; t += gridDim.x) {
+        for (int ci = 0; alive && ci < nchunks; ++ci, ++acc_it) {
+          const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
+          if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + buf * 256u;
+          const int kb_end = min(p.KB, (ci + 1) * p.chunk);
+          for (int kb = ci * p.chunk; kb < kb_end; ++kb) {
+            if (!mbar_wait(full_bar + stage, phase, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t st = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+            const uint64_t a_hi = make_desc<SWZ>(st), a_lo = make_desc<SWZ>(st + A_BYTES);
+            const uint64_t b_hi = make_desc<SWZ>(st + 2 * A_BYTES);
+            const uint64_t b_lo = make_desc<SWZ>(st + 2 * A_BYTES + B_BYTES);
+            const bool first = kb == ci * p.chunk;
+#pragma unroll
+            for (int kk = 0; kk < BK / 8; ++kk) {
+              const uint64_t adv = (uint64_t)(kk * 2);     // 32 bytes per k-step, in 16-byte units
+              tc_mma_tf32(d_tmem, a_hi + adv, b_hi + adv, idesc, (first && kk == 0) ? 0u : 1u);
+              tc_mma_tf32(d_tmem, a_hi + adv, b_lo + adv, idesc, 1u);
+              tc_mma_tf32(d_tmem, a_lo + adv, b_hi + adv, idesc, 1u);
+            }
+            tc_commit(empty_bar + stage);
+            if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+          }
+          if (alive) tc_commit(tfull_bar + buf);
+        }
+      }
+    }
+  }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 232;" ::: "memory");
+    // ---------------- epilogue: warps 4..11 ----------------
+    const int quad = warp & 3;                    // TMEM lane quadrant this warp may read
+    const int half = (warp - 4) >> 2;             // which half of the tile's pixels
+    const int S = p.bw * p.bh;                    // pixels of one group inside the tile
+    uint32_t acc_it = 0;
+    bool alive = true;
+    float acc[E][PH];
+    for (int t = blockIdx.x; alive && t < p.ntiles; t += gridDim.x) {
+      const int mt = t % p.MT;
+      int nt = t / p.MT;
+      const int wt = nt % p.WT; nt /= p.WT;
+      const int ht = nt % p.HT;
+      const int gt = nt / p.HT;
+      const int co = mt * BM + quad * 32 + lane;
+      const bool co_ok = co < p.cout;
+
+      // ---- sum the chunks of this tile in registers (round to nearest) ----
+      for (int ci = 0; ci < nchunks; ++ci, ++acc_it) {
+        const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
+        if (!mbar_wait(tfull_bar + buf, aphase, abort_flag)) { alive = false; break; }
+        tc_fence_after();
+        const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * PH);
+#pragma unroll
+        for (int e0 = 0; e0 < E; e0 += 2) {
+          float tmp[2][PH];
+#pragma unroll
+          for (int de = 0; de < 2; ++de)
+            if (e0 + de < E) {
+#pragma unroll
+              for (int c = 0; c < PH; c += 8) tc_ld8(tbase + (uint32_t)((e0 + de) * P + c), &tmp[de][c]);
+            }
+          tc_wait_ld();
+#pragma unroll
+          for (int de = 0; de < 2; ++de)
+            if (e0 + de < E) {
+#pragma unroll
+              for (int j = 0; j < PH; ++j)
+                acc[e0 + de][j] = (ci == 0) ? tmp[de][j] : acc[e0 + de][j] + tmp[de][j];
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar + buf);
+      }
+      if (!alive) break;
+
+      // ---- store / decode from registers ----
+      float sq[E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) sq[e] = 0.f;
+      float maxrho = 0.f;
+      int cur_g = -1;
+
+      auto flush_stats = [&](int g) {
+        if (MODE != MODE_DECODE || g < 0) return;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          float s = sq[e];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+          if (lane == 0 && s != 0.f) atomicAdd(p.vs.sumsq + (size_t)g * E + e, s);
+          sq[e] = 0.f;
+        }
+        float m = maxrho;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0 && m > 0.f) atomicMax(p.vs.maxrho + g, __float_as_int(m));
+        maxrho = 0.f;
+      };
+
+#pragma unroll
+      for (int j = 0; j < PH; ++j) {
+        const int pix = half * PH + j;
+        const int gl = pix / S, rem = pix - gl * S;
+        const int hl = rem / p.bw, wl = rem - hl * p.bw;
+        const int g = gt * p.bg + gl, oh = ht * p.bh + hl, ow = wt * p.bw + wl;
+        const bool in_range = g < p.G && oh < p.ho && ow < p.wo;      // warp-uniform
+        if (MODE == MODE_YBAR) {
+          if (in_range && co_ok) {
+            float* dst = p.out + ((size_t)g * E) * p.n_out + ((size_t)oh * p.wo + ow) * p.cout + co;
+#pragma unroll
+            for (int e = 0; e < E; ++e) dst[(size_t)e * p.n_out] = acc[e][j];
+          }
+        } else {
+          if (g != cur_g) {      // warp-uniform: g depends on the tile and the pixel only
+            flush_stats(cur_g);
+            cur_g = (g < p.G) ? g : -1;
+          }
+          if (in_range) {
+            float val[E];
+#pragma unroll
+            for (int e = 0; e < E; ++e) val[e] = co_ok ? acc[e][j] : 0.f;
+            if (g == p.f_group && oh == p.f_oh && ow == p.f_ow && co == p.f_co) {
+#pragma unroll
+              for (int e = 0; e < E; ++e)
+                if (e == p.f_enc) val[e] += p.f_delta;
+            }
+            const float* dh = p.dec + (size_t)g * K * K1;
+            const float* dl = p.decl + (size_t)g * K * K1;
+            const float* nv = p.nul + (size_t)g * E;
+            float* dst = p.out + ((size_t)g * K) * p.n_out + ((size_t)oh * p.wo + ow) * p.cout + co;
+            const float b = (p.bias != nullptr && co_ok) ? __ldg(p.bias + co) : 0.f;
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+              float hi = 0.f, lo = 0.f;
+#pragma unroll
+              for (int i = 0; i < K1; ++i) {
+                lo = fmaf(__ldg(dl + k * K1 + i), val[i], lo);
+                hi = fmaf(__ldg(dh + k * K1 + i), val[i], hi);
+              }
+              if (co_ok) dst[(size_t)k * p.n_out] = (hi + lo) + b;
+            }
+            float rho = 0.f, sc = 0.f;
+            const float kInf = __int_as_float(0x7f800000);
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+              const float n_e = __ldg(nv + e);
+              rho = fmaf(n_e, val[e], rho);
+              sc = fmaf(fabsf(n_e), fabsf(val[e]), sc);
+              if (fabsf(val[e]) < kInf) sq[e] = fmaf(val[e], val[e], sq[e]);
+            }
+            const float ar = fabsf(rho);
+            maxrho = fmaxf(maxrho, ar);
+            if (co_ok && (!(ar <= p.tau * sc) || !(sc < kInf))) {
+              unsigned int slot = atomicAdd(p.vs.count, 1u);
+              if (slot < kCandCap) {
+                Candidate cd;
+                cd.index = (long long)g * p.n_out + ((long long)oh * p.wo + ow) * p.cout + co;
+                cd.absrho = ar;
+                cd.s_e = sc;
+                p.vs.cand[slot] = cd;
+              }
+            }
+          }
+        }
+      }
+      if (MODE == MODE_DECODE) flush_stats(cur_g);
+    }
+  }
+
+  // ---------------- teardown ----------------
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // a bounded wait expired: report, give copies still in flight time to land
+    if (threadIdx.x == 0 && p.status != nullptr) atomicExch(p.status, (int)DK_ERR_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(16384);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+}  // namespace tc
+}  // namespace dk
