@@ -173,6 +173,13 @@ DK_API dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const flo
                                      const float* gamma_host, float scale, float* dW,
                                      void* stream);
 
+/* Errors raised ON THE DEVICE by calls that have no dk_verdict to carry them
+ * (dk_linear_fwd, dk_linear_bwd_wgrad): every wait inside the kernels is
+ * bounded, and a kernel whose wait expires stops, leaves its output incomplete
+ * and records DK_ERR_TIMEOUT.  dk_device_status synchronises the device,
+ * returns the recorded code (0 = none) in *status and clears it. */
+DK_API dk_status dk_device_status(dk_ctx* ctx, int32_t* status);
+
 /* dk_decode_verify without allocation and without a context.  The paper has
  * no counterpart for this call; it exists for callers that may not allocate
  * device memory where they need the check: code confined to a fixed memory

@@ -72,6 +72,7 @@ def _signatures():
         "dk_masked_linear": [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(dk_fault), vp],
         "dk_linear_bwd_wgrad": [vp, pp, vp, vp, i32, vp, vp, ctypes.c_float, vp, vp],
         "dk_decode_verify_static": [ctypes.c_int, pp, vp, vp, vp, vp, vp, vp],
+        "dk_device_status": [vp, ctypes.POINTER(ctypes.c_int32)],
         "dk_profile_enable": [vp, ctypes.c_int],
         "dk_profile_read": [vp, ctypes.c_int, ctypes.POINTER(ctypes.c_double),
                             ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)],
@@ -227,6 +228,14 @@ def dk_decode_verify_static(device: int, p: dk_problem, ybar, C: np.ndarray, bia
     _check(lib().dk_decode_verify_static(device, ctypes.byref(p), _dev(ybar), _host(C), _dev(bias), _dev(y),
                                          ctypes.c_void_p(verdict.data_ptr()), _stream()),
            "dk_decode_verify_static")
+
+
+def dk_device_status(ctx: Context) -> int:
+    """Synchronises and returns (then clears) the status raised on the device by
+    calls that have no verdict (0 = none)."""
+    v = ctypes.c_int32()
+    _check(lib().dk_device_status(ctx.handle, ctypes.byref(v)), "dk_device_status")
+    return v.value
 
 
 def dk_masked_linear(ctx: Context, p: dk_problem, W, x, r, C: np.ndarray, bias, y, xbar_save, verdict,

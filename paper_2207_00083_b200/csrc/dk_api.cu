@@ -220,6 +220,12 @@ static WsPlan plan_workspace(const Geom& g) {
   return w;
 }
 
+// Device word that kernels without a dk_verdict raise on a bounded-wait expiry
+// (third word after the verify statistics; read and cleared by dk_device_status).
+static int* ctx_status_word(dk_ctx* ctx) {
+  return reinterpret_cast<int*>(ctx->d_vstats + kVerifyStatFloats) + 2;
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 struct DeviceGuard {
@@ -276,6 +282,7 @@ dk_status dk_create(dk_ctx** out, int device) {
   bool ok = cudaMallocHost(&c->h_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_vstats, (kVerifyStatFloats + 64) * sizeof(float)) == cudaSuccess &&
+            cudaMemset(c->d_vstats, 0, (kVerifyStatFloats + 64) * sizeof(float)) == cudaSuccess &&
             cudaMalloc(&c->d_cand, kCandCap * sizeof(Candidate)) == cudaSuccess;
   for (int i = 0; ok && i < kCoefSlots; ++i)
     ok = cudaEventCreateWithFlags(&c->slot_ev[i], cudaEventDisableTiming) == cudaSuccess;
@@ -365,7 +372,7 @@ dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W, const 
     }
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
-    return tc_linear_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, ybar, nullptr, st);
+    return tc_linear_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, ybar, ctx_status_word(ctx), st);
   }
   ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
   return launch_simt_fwd(g, W, xbar, ybar, g.G * g.E, st);
@@ -504,6 +511,26 @@ dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* del
   s = upload_coefficients(ctx, g, C_host, gamma_host, true, true, st, &cv);
   if (s != DK_OK) return s;
   float* dtil = reinterpret_cast<float*>(static_cast<char*>(ctx->ws) + wp.dtil);
+  if (tc_wgrad_supported(ctx, g)) {
+    // tensor-core path: mixed deltas and encodings as TF32 hi/lo pairs (the
+    // y_bar region of the workspace, unused here, holds the lo part of dtil)
+    char* ws = static_cast<char*>(ctx->ws);
+    float* dt_lo = reinterpret_cast<float*>(ws + wp.ybar);
+    float* xb_hi = reinterpret_cast<float*>(ws + wp.xb_hi);
+    float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
+    {
+      ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
+      s = tc_mix_split(g, delta, cv.dmix, dtil, dt_lo, ctx->sm_count, st);
+    }
+    if (s != DK_OK) return s;
+    {
+      ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+      s = tc_split(xbar, xb_hi, xb_lo, (long long)g.G * xbar_rows * g.n_in, ctx->sm_count, st);
+    }
+    if (s != DK_OK) return s;
+    ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
+    return tc_wgrad(ctx, g, dtil, dt_lo, xb_hi, xb_lo, xbar_rows, scale, dW, ctx_status_word(ctx), st);
+  }
   {
     ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
     s = launch_mix_delta(g, delta, cv.dmix, dtil, ctx->sm_count, st);
@@ -511,6 +538,18 @@ dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* del
   if (s != DK_OK) return s;
   ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
   return launch_simt_wgrad(g, dtil, xbar, xbar_rows, scale, dW, ctx->sm_count, st);
+}
+
+dk_status dk_device_status(dk_ctx* ctx, int32_t* status) {
+  if (!ctx || !status) return DK_ERR_INVALID_ARG;
+  DeviceGuard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  int v = 0;
+  DK_CUDA_CHECK(cudaDeviceSynchronize());
+  DK_CUDA_CHECK(cudaMemcpy(&v, ctx_status_word(ctx), sizeof(int), cudaMemcpyDeviceToHost));
+  if (v != 0) DK_CUDA_CHECK(cudaMemset(ctx_status_word(ctx), 0, sizeof(int)));
+  *status = v;
+  return DK_OK;
 }
 
 dk_status dk_profile_enable(dk_ctx* ctx, int on) {

@@ -139,6 +139,15 @@ dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const f
 dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
                         const float* xb_hi, const float* xb_lo, float* ybar, int* status_word,
                         cudaStream_t st);
+// weight gradient on tensor cores (channels-last, stride 1, cin % 4 == 0, cout % 4 == 0)
+bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g);
+// Eq. 4 delta mixing written as a TF32 hi/lo pair, [G*(K+1)][n_out] each
+dk_status tc_mix_split(const Geom& g, const float* delta, const float* dmix, float* hi, float* lo,
+                       int sm_count, cudaStream_t st);
+// dW = scale * sum <dtil, xbar> from split operands (clears dW first)
+dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* dt_lo,
+                   const float* xb_hi, const float* xb_lo, int xbar_rows, float scale, float* dW,
+                   int* status_word, cudaStream_t st);
 // same contraction with decode + integrity statistics in the epilogue
 dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
                         const float* xb_hi, const float* xb_lo, const CoefView& cv, const float* bias,

@@ -6,6 +6,7 @@
 
 #include "dk_internal.h"
 #include "dk_tc_kernel.cuh"
+#include "dk_tc_wgrad.cuh"
 
 namespace dk {
 namespace {
@@ -22,6 +23,7 @@ struct TcState {
   int smem_optin;
 };
 
+constexpr int kSwz128Atom32 = 1128;
 constexpr int kBK = 32;          // k-block: 32 fp32 = one 128-byte swizzle span per row
 constexpr int kChunk = 2;        // k-blocks accumulated in TMEM between promotions
 
@@ -136,8 +138,12 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t) {
 bool encode_map(const TcState* ts, CUtensorMap* m, const void* base, int rank, const cuuint64_t* dims,
                 const cuuint64_t* strides_bytes, const cuuint32_t* box, int swz_bytes) {
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-  CUtensorMapSwizzle sw = swz_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
-                                           : (swz_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+  // swz_bytes: 32/64/128 = 16-byte chunks swizzled within that span (K-major
+  // operands); kSwz128Atom32 = 32-byte chunks within 128 bytes, the only layout
+  // the tensor core accepts for MN-major 32-bit operands
+  CUtensorMapSwizzle sw = swz_bytes == kSwz128Atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B
+                          : swz_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                          : (swz_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
   CUresult r = ts->encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<void*>(base), dims,
                           strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -313,6 +319,188 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
     prm.f_delta = fault->delta;
   }
   return launch_k<kBK, MODE_DECODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
+}
+
+// ---------------------------------------------------------------------------
+// weight gradient
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int kWgChunk = 1;      // k-blocks accumulated in TMEM between promotions
+
+// dtil[g*(K+1)+j] = sum_i dmix[g][j][i] * delta[g*K+i], written as a TF32 hi/lo pair (Eq. 4).
+template <int K>
+__global__ void __launch_bounds__(256)
+mix_split_kernel(const float* __restrict__ delta, const float* __restrict__ dmix, float* __restrict__ hi,
+                 float* __restrict__ lo, long long n) {
+  constexpr int K1 = K + 1;
+  const int g = blockIdx.y;
+  float c[K1][K];
+#pragma unroll
+  for (int j = 0; j < K1; ++j)
+#pragma unroll
+    for (int i = 0; i < K; ++i) c[j][i] = __ldg(dmix + ((size_t)g * K1 + j) * K + i);
+  const float* dg = delta + (size_t)g * K * n;
+  const size_t ob = (size_t)g * K1 * n;
+  const long long n4 = n / 4;
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n4; q += (long long)gridDim.x * blockDim.x) {
+    float4 s[K];
+#pragma unroll
+    for (int i = 0; i < K; ++i) s[i] = __ldg(reinterpret_cast<const float4*>(dg + (size_t)i * n) + q);
+#pragma unroll
+    for (int j = 0; j < K1; ++j) {
+      float4 o, h, l;
+      o.x = c[j][K - 1] * s[K - 1].x; o.y = c[j][K - 1] * s[K - 1].y;
+      o.z = c[j][K - 1] * s[K - 1].z; o.w = c[j][K - 1] * s[K - 1].w;
+#pragma unroll
+      for (int i = 0; i < K - 1; ++i) {
+        o.x = fmaf(c[j][i], s[i].x, o.x); o.y = fmaf(c[j][i], s[i].y, o.y);
+        o.z = fmaf(c[j][i], s[i].z, o.z); o.w = fmaf(c[j][i], s[i].w, o.w);
+      }
+      h.x = to_tf32(o.x); l.x = to_tf32(o.x - h.x);
+      h.y = to_tf32(o.y); l.y = to_tf32(o.y - h.y);
+      h.z = to_tf32(o.z); l.z = to_tf32(o.z - h.z);
+      h.w = to_tf32(o.w); l.w = to_tf32(o.w - h.w);
+      const size_t off = ob + (size_t)j * n;
+      reinterpret_cast<float4*>(hi + off)[q] = h;
+      reinterpret_cast<float4*>(lo + off)[q] = l;
+    }
+  }
+}
+
+struct WgPlan {
+  WgTcParams prm;
+  int BN;
+  size_t smem_bytes;
+};
+
+bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
+  WgTcParams& p = w->prm;
+  const int P = kWgPix;
+  long long best = -1;
+  p.bw = p.bh = p.bg = 1;
+  for (int bw = 1; bw <= P; bw *= 2)
+    for (int bh = 1; bw * bh <= P; bh *= 2) {
+      const int bg = P / (bw * bh);
+      const long long cost = (long long)((g.wo + bw - 1) / bw) * bw * ((g.ho + bh - 1) / bh) * bh *
+                             ((g.G + bg - 1) / bg) * bg;
+      if (best < 0 || cost < best || (cost == best && (bw > p.bw || (bw == p.bw && bh > p.bh)))) {
+        best = cost; p.bw = bw; p.bh = bh; p.bg = bg;
+      }
+    }
+  p.WT = (g.wo + p.bw - 1) / p.bw;
+  p.HT = (g.ho + p.bh - 1) / p.bh;
+  p.GT = (g.G + p.bg - 1) / p.bg;
+  long long pb = (long long)p.WT * p.HT * p.GT;
+  if (pb > 0x3fffffffLL) return false;
+  p.PB = (int)pb;
+  p.K1 = g.K + 1;
+  w->BN = g.cin <= 64 ? 64 : (g.cin <= 128 ? 128 : 256);
+  p.MT = (g.cout + BM - 1) / BM;
+  p.NB = (g.cin + w->BN - 1) / w->BN;
+  p.taps = g.kh * g.kw;
+  const long long base = (long long)p.MT * p.NB * p.taps;
+  long long nsplit = (2LL * sm_count + base - 1) / base;
+  if (nsplit > p.PB) nsplit = p.PB;
+  if (nsplit < 1) nsplit = 1;
+  p.pb_per_split = (int)((p.PB + nsplit - 1) / nsplit);
+  p.nsplit = (p.PB + p.pb_per_split - 1) / p.pb_per_split;
+  const long long items = base * p.nsplit;
+  if (items > 0x7fffffffLL) return false;
+  p.nitems = (int)items;
+  p.kw = g.kw; p.pad = g.pad;
+  p.chunk = kWgChunk;
+  p.cout = g.cout; p.cin = g.cin;
+  const size_t stage = 2 * ((size_t)(BM / 32) * kWgBox + (size_t)(w->BN / 32) * kWgBox);
+  const size_t ctrl = 1024 + 256;
+  int ns = (int)(((size_t)smem_optin - ctrl) / stage);
+  if (ns > kMaxStages) ns = kMaxStages;
+  if (ns < 2) return false;
+  p.nstages = ns;
+  w->smem_bytes = (size_t)ns * stage + ctrl;
+  return true;
+}
+
+template <int BN>
+dk_status launch_wgrad(const WgPlan& w, const CUtensorMap& md_hi, const CUtensorMap& md_lo,
+                       const CUtensorMap& mx_hi, const CUtensorMap& mx_lo, int sm_count, cudaStream_t st) {
+  auto kern = tc_wgrad_kernel<BN>;
+  cudaFuncAttributes fa;
+  DK_CUDA_CHECK(cudaFuncGetAttributes(&fa, kern));
+  if (fa.numRegs * kThreadsTc < 40 * 128 + 232 * 256) return DK_ERR_UNSUPPORTED;
+  DK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)w.smem_bytes));
+  int grid = w.prm.nitems < sm_count ? w.prm.nitems : sm_count;
+  kern<<<grid, kThreadsTc, w.smem_bytes, st>>>(md_hi, md_lo, mx_hi, mx_lo, w.prm);
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+}  // namespace
+
+bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g) {
+  if (g.precision == DK_FP32_SIMT || ctx->tc_state == nullptr) return false;
+  if (g.layout != DK_NHWC || g.stride != 1 || (g.cin % 4) != 0 || (g.cout % 4) != 0) return false;
+  WgPlan w;
+  return plan_wgrad(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, ctx->sm_count, &w);
+}
+
+dk_status tc_mix_split(const Geom& g, const float* delta, const float* dmix, float* hi, float* lo,
+                       int sm_count, cudaStream_t st) {
+  if (g.n_out % 4 || g.G > 65535) return DK_ERR_SHAPE;
+  long long n4 = g.n_out / 4;
+  long long want = (n4 + 255) / 256;
+  long long cap = ((long long)sm_count * 16 + g.G - 1) / g.G;
+  if (want > cap) want = cap;
+  if (want < 1) want = 1;
+  dim3 grid((unsigned)want, (unsigned)g.G);
+#define DK_MIX_CASE(KK) \
+  case KK: mix_split_kernel<KK><<<grid, 256, 0, st>>>(delta, dmix, hi, lo, g.n_out); break;
+  switch (g.K) {
+    DK_MIX_CASE(1) DK_MIX_CASE(2) DK_MIX_CASE(3) DK_MIX_CASE(4)
+    DK_MIX_CASE(5) DK_MIX_CASE(6) DK_MIX_CASE(7) DK_MIX_CASE(8)
+    default: return DK_ERR_SHAPE;
+  }
+#undef DK_MIX_CASE
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* dt_lo, const float* xb_hi,
+                   const float* xb_lo, int xbar_rows, float scale, float* dW, int* status_word,
+                   cudaStream_t st) {
+  TcState* ts = static_cast<TcState*>(ctx->tc_state);
+  WgPlan w;
+  if (!plan_wgrad(g, ts->smem_optin, ctx->sm_count, &w)) return DK_ERR_UNSUPPORTED;
+  w.prm.scale = scale;
+  w.prm.dW = dW;
+  w.prm.status = status_word;
+  CUtensorMap md_hi, md_lo, mx_hi, mx_lo;
+  {
+    cuuint64_t dims[5] = {(cuuint64_t)g.cout, (cuuint64_t)g.wo, (cuuint64_t)g.ho, (cuuint64_t)(g.K + 1),
+                          (cuuint64_t)g.G};
+    cuuint64_t str[4] = {(cuuint64_t)g.cout * 4, (cuuint64_t)g.cout * g.wo * 4, (cuuint64_t)g.n_out * 4,
+                         (cuuint64_t)g.n_out * (g.K + 1) * 4};
+    cuuint32_t box[5] = {32, (cuuint32_t)w.prm.bw, (cuuint32_t)w.prm.bh, 1, (cuuint32_t)w.prm.bg};
+    if (!encode_map(ts, &md_hi, dt_hi, 5, dims, str, box, kSwz128Atom32) ||
+        !encode_map(ts, &md_lo, dt_lo, 5, dims, str, box, kSwz128Atom32))
+      return DK_ERR_CUDA;
+  }
+  {
+    cuuint64_t dims[5] = {(cuuint64_t)g.cin, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)xbar_rows,
+                          (cuuint64_t)g.G};
+    cuuint64_t str[4] = {(cuuint64_t)g.cin * 4, (cuuint64_t)g.cin * g.w * 4, (cuuint64_t)g.n_in * 4,
+                         (cuuint64_t)g.n_in * xbar_rows * 4};
+    cuuint32_t box[5] = {32, (cuuint32_t)w.prm.bw, (cuuint32_t)w.prm.bh, 1, (cuuint32_t)w.prm.bg};
+    if (!encode_map(ts, &mx_hi, xb_hi, 5, dims, str, box, kSwz128Atom32) ||
+        !encode_map(ts, &mx_lo, xb_lo, 5, dims, str, box, kSwz128Atom32))
+      return DK_ERR_CUDA;
+  }
+  DK_CUDA_CHECK(cudaMemsetAsync(dW, 0, (size_t)g.cout * g.kc * sizeof(float), st));
+  switch (w.BN) {
+    case 64: return launch_wgrad<64>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
+    case 128: return launch_wgrad<128>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
+    default: return launch_wgrad<256>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
+  }
 }
 
 }  // namespace dk

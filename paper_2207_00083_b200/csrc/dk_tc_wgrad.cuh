@@ -1,0 +1,253 @@
+// Weight-gradient product of Eq. 4/6 on the tensor cores:
+//   dW[co][tap][ci] = scale * sum_{g, j<=K, pixel} dtil[g,j][pixel][co] * xbar[g,j][pixel + tap - pad][ci]
+// with dtil[g,j] = sum_i gamma_j B[j][i] delta[g,i] mixed beforehand.
+//
+// GEMM view: M = cout (128 per tile), N = a block of input channels of one
+// filter tap, contraction = (virtual batch, encoding, output pixel).  Both
+// operands are channels-last tensors, i.e. contiguous along M / N and strided
+// along the contraction: they are fetched by TMA as [32 pixels][32 channels]
+// boxes (128-byte rows, 32-byte chunks swizzled within the row) and fed to
+// tcgen05.mma as MN-major operands.  Same 3xTF32 split and the same pipeline as the forward kernel.
+//
+// Accuracy.  The K+1 encodings of a pixel block are consecutive k-blocks, so
+// the masking noise cancels every K+1 k-blocks and partial sums return to the
+// scale of the signal.  TMEM accumulates `chunk` k-blocks only (the tensor pipe
+// truncates when it adds into the accumulator); the epilogue warps sum the
+// chunks in registers with round-to-nearest.
+//
+// Parallelism.  Work item = (cout tile, tap, channel block, contraction
+// slice); persistent CTAs walk the items and add their slice into dW with
+// fp32 atomics (dW is cleared first).
+#pragma once
+
+#include "dk_tc_kernel.cuh"
+
+namespace dk {
+namespace tc {
+
+constexpr int kWgPix = 32;                 // contraction elements (pixels) per k-block
+constexpr int kWgBox = kWgPix * 128;       // bytes of one [32 pixels][32 channels] box
+
+struct WgTcParams {
+  int bw, bh, bg;              // box shape of the 32 pixels: columns, rows, groups
+  int WT, HT, GT;              // pixel blocks along width, height, groups
+  int PB;                      // WT*HT*GT
+  int K1;                      // encodings used (K+1)
+  int MT, NB, taps;            // cout tiles, channel blocks, filter taps
+  int nsplit, pb_per_split;    // contraction slices
+  int nitems;                  // MT*NB*taps*nsplit
+  int kw, pad;
+  int nstages, chunk;
+  int cout, cin;
+  float scale;
+  float* dW;                   // [cout][taps][cin]
+  int* status;
+};
+
+// Shared-memory descriptor of an MN-major 32-bit operand: [k][32 floats] boxes
+// of 128-byte rows whose 32-byte chunks are swizzled with a period of 4 rows
+// (the only MN-major layout the tensor core takes for 32-bit elements);
+// 4-row groups 512 bytes apart along k, column blocks `block_bytes` apart
+// along M/N.
+__device__ __forceinline__ uint64_t make_desc_mn(uint32_t smem_addr, uint32_t block_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+  d |= (uint64_t)((block_bytes >> 4) & 0x3FFF) << 16;   // leading byte offset: next 32-channel block
+  d |= (uint64_t)(512 >> 4) << 32;                      // stride byte offset: next 4 pixels
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)1 << 61;                               // 128-byte span, 32-byte swizzle atom
+  return d;
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kThreadsTc, 1)
+tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_constant__ CUtensorMap map_d_lo,
+                const __grid_constant__ CUtensorMap map_x_hi, const __grid_constant__ CUtensorMap map_x_lo,
+                const WgTcParams p) {
+  constexpr int NH = BN / 2;                     // accumulators per epilogue thread
+  constexpr int A_BYTES = (BM / 32) * kWgBox;    // 16 KiB
+  constexpr int B_BYTES = (BN / 32) * kWgBox;
+  constexpr int STAGE_BYTES = 2 * (A_BYTES + B_BYTES);
+  static_assert(BN % 64 == 0 && BN <= 256, "illegal channel block");
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                                         ~static_cast<uintptr_t>(1023));
+  unsigned char* ctrl = smem + (size_t)p.nstages * STAGE_BYTES;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(ctrl);
+  uint64_t* empty_bar = full_bar + kMaxStages;
+  uint64_t* tfull_bar = empty_bar + kMaxStages;
+  uint64_t* tempty_bar = tfull_bar + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.nstages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + b, 1); mbar_init(tempty_bar + b, kEpiWarps); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // item -> (mt, nb, tap, slice); k-blocks of an item = pixel blocks of its slice x K1 encodings
+  auto item_range = [&](int item, int& mt, int& nb, int& tap, int& pb_lo, int& pb_hi) {
+    mt = item % p.MT;
+    int r = item / p.MT;
+    nb = r % p.NB; r /= p.NB;
+    tap = r % p.taps;
+    const int s = r / p.taps;
+    pb_lo = s * p.pb_per_split;
+    pb_hi = min(p.PB, pb_lo + p.pb_per_split);
+  };
+
+  static_assert(40 * 128 + 232 * 256 <= 168 * kThreadsTc, "setmaxnreg budget exceeds the CTA's register pool");
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
+    if (warp == 0 && lane == 0) {
+      // ---------------- TMA producer ----------------
+      int stage = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; alive && item < p.nitems; item += gridDim.x) {
+        int mt, nb, tap, pb_lo, pb_hi;
+        item_range(item, mt, nb, tap, pb_lo, pb_hi);
+        const int u = tap / p.kw, v = tap - u * p.kw;
+        const int m0 = mt * BM, n0 = nb * BN;
+        for (int pb = pb_lo; alive && pb < pb_hi; ++pb) {
+          int r = pb;
+          const int wt = r % p.WT; r /= p.WT;
+          const int ht = r % p.HT;
+          const int gt = r / p.HT;
+          const int x0 = wt * p.bw, y0 = ht * p.bh, g0 = gt * p.bg;
+          for (int j = 0; j < p.K1; ++j) {
+            if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) { alive = false; break; }
+            unsigned char* st = smem + (size_t)stage * STAGE_BYTES;
+            mbar_expect_tx(full_bar + stage, (uint32_t)STAGE_BYTES);
+#pragma unroll 1
+            for (int cb = 0; cb < BM / 32; ++cb) {
+              tma_load_5d(st + cb * kWgBox, &map_d_hi, full_bar + stage, m0 + cb * 32, x0, y0, j, g0);
+              tma_load_5d(st + A_BYTES + cb * kWgBox, &map_d_lo, full_bar + stage, m0 + cb * 32, x0, y0, j, g0);
+            }
+            unsigned char* bh = st + 2 * A_BYTES;
+#pragma unroll 1
+            for (int cb = 0; cb < BN / 32; ++cb) {
+              tma_load_5d(bh + cb * kWgBox, &map_x_hi, full_bar + stage, n0 + cb * 32, x0 + v - p.pad,
+                          y0 + u - p.pad, j, g0);
+              tma_load_5d(bh + B_BYTES + cb * kWgBox, &map_x_lo, full_bar + stage, n0 + cb * 32, x0 + v - p.pad,
+                          y0 + u - p.pad, j, g0);
+            }
+            if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    } else if (warp == 1 && lane == 0) {
+      // ---------------- MMA issuer ----------------
+      constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | (1u << 16) |
+                                 ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t acc_it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; alive && item < p.nitems; item += gridDim.x) {
+        int mt, nb, tap, pb_lo, pb_hi;
+        item_range(item, mt, nb, tap, pb_lo, pb_hi);
+        const int KB = (pb_hi - pb_lo) * p.K1;
+        const int nchunks = (KB + p.chunk - 1) / p.chunk;
+        for (int ci = 0; alive && ci < nchunks; ++ci, ++acc_it) {
+          const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
+          if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + buf * 256u;
+          const int kb_end = min(KB, (ci + 1) * p.chunk);
+          for (int kb = ci * p.chunk; kb < kb_end; ++kb) {
+            if (!mbar_wait(full_bar + stage, phase, abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t st = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+            const uint64_t a_hi = make_desc_mn(st, kWgBox), a_lo = make_desc_mn(st + A_BYTES, kWgBox);
+            const uint64_t b_hi = make_desc_mn(st + 2 * A_BYTES, kWgBox);
+            const uint64_t b_lo = make_desc_mn(st + 2 * A_BYTES + B_BYTES, kWgBox);
+            const bool first = kb == ci * p.chunk;
+#pragma unroll
+            for (int kk = 0; kk < kWgPix / 8; ++kk) {
+              const uint64_t adv = (uint64_t)(kk * (1024 >> 4));   // 8 pixels = one 1024-byte row group
+              tc_mma_tf32(d_tmem, a_hi + adv, b_hi + adv, idesc, (first && kk == 0) ? 0u : 1u);
+              tc_mma_tf32(d_tmem, a_hi + adv, b_lo + adv, idesc, 1u);
+              tc_mma_tf32(d_tmem, a_lo + adv, b_hi + adv, idesc, 1u);
+            }
+            tc_commit(empty_bar + stage);
+            if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+          }
+          if (alive) tc_commit(tfull_bar + buf);
+        }
+      }
+    }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 232;" ::: "memory");
+    // ---------------- epilogue: warps 4..11 ----------------
+    const int quad = warp & 3;
+    const int half = (warp - 4) >> 2;
+    uint32_t acc_it = 0;
+    bool alive = true;
+    float acc[NH];
+    for (int item = blockIdx.x; alive && item < p.nitems; item += gridDim.x) {
+      int mt, nb, tap, pb_lo, pb_hi;
+      item_range(item, mt, nb, tap, pb_lo, pb_hi);
+      const int KB = (pb_hi - pb_lo) * p.K1;
+      const int nchunks = (KB + p.chunk - 1) / p.chunk;
+      for (int ci = 0; ci < nchunks; ++ci, ++acc_it) {
+        const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
+        if (!mbar_wait(tfull_bar + buf, aphase, abort_flag)) { alive = false; break; }
+        tc_fence_after();
+        const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * NH);
+#pragma unroll
+        for (int c0 = 0; c0 < NH; c0 += 32) {
+          float tmp[32];
+#pragma unroll
+          for (int c = 0; c < 32; c += 8) tc_ld8(tbase + (uint32_t)(c0 + c), &tmp[c]);
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) acc[c0 + c] = (ci == 0) ? tmp[c] : acc[c0 + c] + tmp[c];
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar + buf);
+      }
+      if (!alive) break;
+      const int co = mt * BM + quad * 32 + lane;
+      if (co < p.cout && nchunks > 0) {
+        float* dst = p.dW + ((size_t)co * p.taps + tap) * p.cin + nb * BN + half * NH;
+        const int nvalid = p.cin - (nb * BN + half * NH);
+#pragma unroll
+        for (int c = 0; c < NH; ++c)
+          if (c < nvalid) atomicAdd(dst + c, p.scale * acc[c]);
+      }
+    }
+  }
+
+  // ---------------- teardown ----------------
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0 && p.status != nullptr) atomicExch(p.status, (int)DK_ERR_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(16384);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+}  // namespace tc
+}  // namespace dk

@@ -108,6 +108,7 @@ def test_linear_fwd_matches_oracle(ctx, drawn, spec, prec):
     ybar = H.empty_acts(spec.G * (spec.K + 2), spec, "out", lay(spec))
     ctx.ensure_workspace(p)
     dk.dk_linear_fwd(ctx, p, W, xb, ybar)
+    assert dk.dk_device_status(ctx) == 0
     want = O.linear(d["W"], xbar32, spec.stride, spec.pad)
     assert H.max_rel(H.acts_from_dev(ybar, lay(spec)), want) < TOL_YBAR
 
@@ -235,6 +236,7 @@ def test_wgrad_matches_oracle(ctx, drawn, spec, rows, prec):
     dW.fill_(float("nan"))
     dk.dk_linear_bwd_wgrad(ctx, p, H.acts_to_dev(d["delta"], lay(spec)), H.acts_to_dev(xbar32, lay(spec)),
                            nrows, d["C"], d["gamma"], scale, dW)
+    assert dk.dk_device_status(ctx) == 0
     got = H.weights_from_dev(dW, lay(spec))
     plain = O.wgrad_plain(d["delta"], d["x"], scale, spec.kh, spec.kw, spec.stride, spec.pad)
     masked = O.wgrad_masked(d["delta"], xbar32, d["C"], d["gamma"], scale, spec.kh, spec.kw,

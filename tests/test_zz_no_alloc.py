@@ -51,7 +51,10 @@ def test_static_entry_point_matches_decode_verify_twice_in_a_row():
     try:
         # first call: clean run
         y_ref, v_ref, y_new, v_new = _both(ctx, spec, p, ybar, d["C"], bias)
-        assert v_new == v_ref and v_new["ok"] == 1 and v_new["first_index"] == -1
+        # the group rms behind max_ratio is summed with fp32 atomics: last bits may differ
+        assert v_new["max_ratio"] == pytest.approx(v_ref["max_ratio"], rel=1e-5)
+        assert (v_new["ok"], v_new["n_flagged"], v_new["first_index"], v_new["status"]) == \
+               (v_ref["ok"], v_ref["n_flagged"], v_ref["first_index"], v_ref["status"]) == (1, 0, -1, 0)
         got, want = y_new.cpu().numpy().astype(np.float64), y_ref.cpu().numpy().astype(np.float64)
         assert np.max(np.abs(got - want)) <= TOL_DECODED * np.max(np.abs(want))
         yd, _ = O.decode(ybar, d["C"])
