@@ -3,6 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--workload vgg16_cifar] [--no-cpu-baseline]
+    python bench.py --layer-table [--workload vgg16_224] [--layers conv3_2,conv4_2]
 
 One step = one pass of the whole path over one synthetic batch of the
 workload: for every layer the fused masked forward (encode, dense op on the
@@ -11,6 +12,10 @@ the masked weight gradient where the workload trains.  Prints ONE JSON line.
 
 `--impl reference` times the fp64 CPU oracle as it stands on a bounded sample
 of the same workload (one virtual batch of every layer per step).
+
+`--layer-table` times every layer of a workload on its own (forward call and
+wgrad call, CUDA events around the C-ABI call) and prints one JSON line with
+the per-layer table; it is a reporting aid, not the step metric.
 
 With N > 1 (under torchrun) every rank runs an independent replica of the
 workload on its own GPU: the path has no exchange step, nothing is sharded.
@@ -33,6 +38,7 @@ import numpy as np  # noqa: E402
 
 METRIC = "decoded masked-linear TFLOP/s & fraction of roofline; encode/decode GB/s"
 L2_FLUSH_BYTES = 512 << 20
+TF32_OVER_BF16 = 1.1 / 2.25      # nominal dense TF32 : BF16 tensor throughput
 
 
 def read_peaks():
@@ -113,7 +119,7 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------
-# our arm
+# helpers of our arm
 # ---------------------------------------------------------------------------
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -128,8 +134,9 @@ class ClockSampler:
     def start(self):
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.QUERY}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                       "--format=csv,noheader,nounits", "-lms", "50"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
+            time.sleep(0.3)      # let the sampler come up before the timed region
         except Exception:
             self.p = None
 
@@ -166,6 +173,156 @@ class ClockSampler:
         return out
 
 
+def shape_acts(n, s, which):
+    c, h, w = (s.cin, s.h, s.w) if which == "in" else (s.cout, s.hout, s.wout)
+    return (n, c) if s.kind == "fc" else (n, h, w, c)
+
+
+def shape_w(s):
+    return (s.cout, s.cin) if s.kind == "fc" else (s.cout, s.kh, s.kw, s.cin)
+
+
+def uses_tensor_cores(s):
+    """Mirror of the library's dispatch rule (channels-last, stride 1, cin % 4 == 0,
+    default arithmetic)."""
+    return s.stride == 1 and s.cin % 4 == 0 and getattr(s, "precision", "default") == "default"
+
+
+def make_layer(torch, dk, synth, ctx, s, dev, gen, rank, pinned):
+    """Device (and optionally pinned host) tensors of one layer, seeded."""
+    p = dk.problem_from_spec(s, tol=1e-4)
+    rng = synth._rng(s, "coef", rank)
+    L = {"spec": s, "p": p, "C": synth.draw_coefficients(rng, s.K, s.G),
+         "gamma": synth.draw_gamma(rng, s.K, s.G)}
+    x = torch.empty(shape_acts(s.batch, s, "in"), device=dev)
+    if s.x_dist == "uniform":
+        x.uniform_(0, 1, generator=gen)
+    else:
+        x.normal_(0, 1, generator=gen)
+    r = torch.empty(shape_acts(s.G, s, "in"), device=dev).normal_(0, s.sigma_r, generator=gen)
+    std = s.w_std if s.w_std is not None else (2.0 / s.kc) ** 0.5
+    L["x"], L["r"] = x, r
+    L["W"] = torch.randn(shape_w(s), device=dev, generator=gen) * std
+    L["y"] = torch.empty(shape_acts(s.batch, s, "out"), device=dev)
+    L["xsave"] = torch.empty(shape_acts(s.G * (s.K + 2), s, "in"), device=dev)
+    L["v"] = dk.new_verdict(dev.index)
+    L["h2d"] = L["d2h"] = 0
+    if s.wgrad:
+        L["delta"] = torch.empty(shape_acts(s.batch, s, "out"), device=dev).normal_(0, 1, generator=gen)
+        L["dW"] = torch.empty_like(L["W"])
+    if pinned:
+        L["hx"], L["hr"] = x.cpu().pin_memory(), r.cpu().pin_memory()
+        L["hy"] = torch.empty(L["y"].shape, dtype=torch.float32).pin_memory()
+        L["hv"] = torch.empty(dk.VERDICT_BYTES, dtype=torch.uint8).pin_memory()
+        L["h2d"] = (x.numel() + r.numel()) * 4
+        L["d2h"] = L["y"].numel() * 4 + dk.VERDICT_BYTES
+        if s.wgrad:
+            L["hdelta"] = L["delta"].cpu().pin_memory()
+            L["hdW"] = torch.empty(L["W"].shape, dtype=torch.float32).pin_memory()
+            L["h2d"] += L["delta"].numel() * 4
+            L["d2h"] += L["W"].numel() * 4
+    return L
+
+
+def measure_elementwise(torch, dk, synth, ctx, dev, peaks, iters=10):
+    """Standalone dk_encode / dk_decode_verify on tensors much larger than L2."""
+    K, G, n = 4, 32, 1 << 20
+    spec = synth.LayerSpec("elementwise", "stream", "fc", n, n, K=K, G=G)
+    p = dk.problem_from_spec(spec, tol=1e-4)
+    rng = np.random.default_rng(7)
+    C = synth.draw_coefficients(rng, K, G)
+    x = torch.rand((G * K, n), device=dev)
+    r = torch.randn((G, n), device=dev) * 100.0
+    xbar = torch.empty((G * (K + 2), n), device=dev)
+    y = torch.empty((G * K, n), device=dev)
+    v = dk.new_verdict(dev.index)
+    out = {}
+    for name, fn, bytes_per_pos in (
+            ("encode", lambda: dk.dk_encode(ctx, p, x, r, C, xbar), (2 * K + 3) * 4),
+            ("decode", lambda: dk.dk_decode_verify(ctx, p, xbar, C, None, y, v), (2 * K + 2) * 4)):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / iters
+        gbs = bytes_per_pos * G * n / (ms * 1e-3) / 1e9
+        out[name] = {"gbs": gbs, "frac_hbm": gbs / peaks["hbm_gbs"], "ms": ms,
+                     "bytes": bytes_per_pos * G * n, "shape": f"K={K} G={G} n={n} fp32"}
+    assert dk.read_verdict(v)["status"] == 0
+    return out
+
+
+def run_layer_table(args):
+    import torch
+    from paper_2207_00083_b200 import binding as dk
+    from paper_2207_00083_b200 import synth
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(0)
+    peaks = read_peaks()
+    tf32_peak = peaks["bf16_tflops"] * TF32_OVER_BF16
+    ctx = dk.Context(0)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(220700083)
+    flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)
+    want = set(args.layers.split(",")) if args.layers else None
+    rows = []
+    for s in synth.layers(args.workload):
+        if want and s.name not in want:
+            continue
+        L = make_layer(torch, dk, synth, ctx, s, dev, gen, 0, pinned=False)
+        ctx.ensure_workspace(L["p"])
+
+        def fwd():
+            dk.dk_masked_linear(ctx, L["p"], L["W"], L["x"], L["r"], L["C"], None, L["y"], L["xsave"], L["v"])
+
+        def wg():
+            dk.dk_linear_bwd_wgrad(ctx, L["p"], L["delta"], L["xsave"], s.K + 2, L["C"], L["gamma"],
+                                   1.0 / s.batch, L["dW"])
+        row = {"layer": s.name, "M": s.cout, "Kc": s.kc, "N_fwd": s.G * (s.K + 2) * s.hout * s.wout,
+               "tensor_cores": uses_tensor_cores(s)}
+        for name, fn, flops in (("fwd", fwd, s.fwd_flops()), ("wgrad", wg, s.wgrad_flops())):
+            if name == "wgrad" and not s.wgrad:
+                continue
+            for _ in range(2):
+                fn()
+            dk.dk_profile_reset(ctx)
+            dk.dk_profile_enable(ctx, True)
+            tot = 0.0
+            for _ in range(args.iters):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                tot += a.elapsed_time(b)
+            prof = dk.dk_profile_read(ctx)
+            dk.dk_profile_enable(ctx, False)
+            ms = tot / args.iters
+            kind = "linear_fwd" if name == "fwd" else "wgrad"
+            kms = prof[kind][0] / max(prof[kind][1], 1)
+            issued = 3.0 if uses_tensor_cores(s) else 1.0
+            row[name] = {"call_ms": round(ms, 4), "kernel_ms": round(kms, 4),
+                         "masked_tflops_call": round(flops / ms / 1e9, 2),
+                         "issued_tflops_kernel": round(issued * flops / kms / 1e9, 2),
+                         "frac_tf32_peak_kernel": round(issued * flops / kms / 1e9 / tf32_peak, 4),
+                         "other_kernels_ms": round(sum(v[0] for k, v in prof.items() if k != kind)
+                                                   / args.iters, 4)}
+        vd = dk.read_verdict(L["v"])
+        row["verdict_ok"] = vd["ok"]
+        rows.append(row)
+        del L
+        torch.cuda.empty_cache()
+    print(json.dumps({"layer_table": args.workload, "tf32_peak_tflops": tf32_peak, "peak_source": peaks["source"],
+                      "rows": rows}), flush=True)
+
+
+# ---------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -184,58 +341,13 @@ def run_ours(args):
 
     specs = synth.layers(args.workload)
     ctx = dk.Context(local)
-    E = specs[0].K + 2
     gen = torch.Generator(device=dev)
-    gen.manual_seed(2207_00083 + rank)
-
-    def shape_acts(n, s, which):
-        c, h, w = (s.cin, s.h, s.w) if which == "in" else (s.cout, s.hout, s.wout)
-        return (n, c) if s.kind == "fc" else (n, h, w, c)
-
-    def shape_w(s):
-        return (s.cout, s.cin) if s.kind == "fc" else (s.cout, s.kh, s.kw, s.cin)
-
-    layers = []
-    h2d = d2h = 0
-    for s in specs:
-        p = dk.problem_from_spec(s, tol=1e-4)
-        ctx.ensure_workspace(p)
-        rng = synth._rng(s, "coef", rank)
-        L = {"spec": s, "p": p,
-             "C": synth.draw_coefficients(rng, s.K, s.G), "gamma": synth.draw_gamma(rng, s.K, s.G)}
-        # pinned host copies (the end-to-end leg streams them in every step)
-        hx = torch.empty(shape_acts(s.batch, s, "in"), dtype=torch.float32).pin_memory()
-        hr = torch.empty(shape_acts(s.G, s, "in"), dtype=torch.float32).pin_memory()
-        cpu_gen = torch.Generator().manual_seed(1000 * rank + len(layers))
-        if s.x_dist == "uniform":
-            hx.uniform_(0, 1, generator=cpu_gen)
-        else:
-            hx.normal_(0, 1, generator=cpu_gen)
-        hr.normal_(0, s.sigma_r, generator=cpu_gen)
-        L["hx"], L["hr"] = hx, hr
-        L["x"], L["r"] = hx.to(dev), hr.to(dev)
-        std = s.w_std if s.w_std is not None else (2.0 / s.kc) ** 0.5
-        L["W"] = torch.randn(shape_w(s), device=dev, generator=gen) * std
-        L["y"] = torch.empty(shape_acts(s.batch, s, "out"), device=dev)
-        L["xsave"] = torch.empty(shape_acts(s.G * (s.K + 2), s, "in"), device=dev)
-        L["v"] = dk.new_verdict(local)
-        L["hy"] = torch.empty(shape_acts(s.batch, s, "out"), dtype=torch.float32).pin_memory()
-        L["hv"] = torch.empty(dk.VERDICT_BYTES, dtype=torch.uint8).pin_memory()
-        h2d += hx.numel() * 4 + hr.numel() * 4
-        d2h += L["hy"].numel() * 4 + dk.VERDICT_BYTES
-        if s.wgrad:
-            hd = torch.empty(shape_acts(s.batch, s, "out"), dtype=torch.float32).pin_memory()
-            hd.normal_(0, 1, generator=cpu_gen)
-            L["hdelta"], L["delta"] = hd, hd.to(dev)
-            L["dW"] = torch.empty_like(L["W"])
-            L["hdW"] = torch.empty(shape_w(s), dtype=torch.float32).pin_memory()
-            h2d += hd.numel() * 4
-            d2h += L["hdW"].numel() * 4
-        layers.append(L)
-    # the workspace may have been re-allocated while growing: register the final one per layer
+    gen.manual_seed(220700083 + rank)
+    layers = [make_layer(torch, dk, synth, ctx, s, dev, gen, rank, pinned=True) for s in specs]
+    h2d = sum(L["h2d"] for L in layers)
+    d2h = sum(L["d2h"] for L in layers)
     biggest = max(layers, key=lambda L: ctx.workspace_bytes(L["p"]))
     ctx.ensure_workspace(biggest["p"])
-
     flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)
 
     def step_device():
@@ -270,7 +382,6 @@ def run_ours(args):
             flush.zero_()
             fn()
         barrier()
-        total = 0.0
         evs = []
         for _ in range(steps):
             flush.zero_()                 # evict the previous step's tensors from L2 (untimed)
@@ -280,8 +391,7 @@ def run_ours(args):
             b.record()
             evs.append((a, b))
         barrier()
-        for a, b in evs:
-            total += a.elapsed_time(b)
+        total = sum(a.elapsed_time(b) for a, b in evs)
         t = torch.tensor([total], dtype=torch.float64, device=dev)
         if world > 1:
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -294,6 +404,7 @@ def run_ours(args):
 
     # ---- device-resident timing, with per-kernel events inside the library
     for _ in range(warmup):
+        flush.zero_()
         step_device()
     torch.cuda.synchronize()
     dk.dk_profile_reset(ctx)
@@ -306,12 +417,12 @@ def run_ours(args):
     prof = dk.dk_profile_read(ctx)
     dk.dk_profile_enable(ctx, False)
     launches = sum(v[2] for v in prof.values())
+    assert dk.dk_device_status(ctx) == 0
 
     # ---- end to end through host buffers
     ms_e2e = timed(step_e2e, steps, 1)
 
-    # every verdict of the last step must be clean
-    for L in layers:
+    for L in layers:        # every verdict of the last step must be clean
         vd = dk.read_verdict(L["v"])
         assert vd["ok"] == 1 and vd["status"] == 0, (L["spec"].name, vd)
 
@@ -323,53 +434,42 @@ def run_ours(args):
     value = world * step_flops * steps / (ms_total * 1e-3) / 1e12
     e2e_value = world * step_flops * steps / (ms_e2e * 1e-3) / 1e12
     K = specs[0].K
-
-    # roofline of the dominant kernel class
-    dom = max(prof, key=lambda k: prof[k][0])
+    ksum = max(sum(v[0] for v in prof.values()), 1e-9)
     kernel_ms = {k: round(v[0] / max(v[1], 1), 5) for k, v in prof.items() if v[1]}
-    share = {k: round(v[0] / max(sum(x[0] for x in prof.values()), 1e-9), 4) for k, v in prof.items() if v[1]}
-    issued_per_flop = 1.0   # SIMT fp32: one FMA per multiply-add
-    if dom in ("linear_fwd", "wgrad"):
-        flops_launch = (fwd_flops if dom == "linear_fwd" else wg_flops) / len(
-            [s for s in specs if (dom == "linear_fwd" or s.wgrad)])
-        avg_ms = prof[dom][0] / max(prof[dom][1], 1)
-        achieved = flops_launch * issued_per_flop / (avg_ms * 1e-3) / 1e12
-        peak = 148 * 128 * 2 * (clocks["sm_max_mhz"] or 1965.0) * 1e6 / 1e12
-        roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                    "frac": achieved / peak, "traffic": None, "kernel": dom,
-                    "peak_source": "148 SMs x 128 fp32 FMA lanes x 2 flop x max SM clock (derived)"}
-    else:
-        per_pos = {"encode": (K + 1 + K + 2) * 4, "decode_verify": (K + 2 + K) * 4, "mix_delta": (2 * K + 1) * 4}
-        nel = {"encode": sum(s.G * s.n_in for s in specs), "decode_verify": sum(s.G * s.n_out for s in specs),
-               "mix_delta": sum(s.G * s.n_out for s in specs if s.wgrad)}.get(dom, 0)
-        nl = len(specs)
-        avg_ms = prof[dom][0] / max(prof[dom][1], 1)
-        achieved = per_pos.get(dom, 0) * nel / nl / (avg_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": None, "kernel": dom,
-                    "peak_source": peaks["source"]}
+    share = {k: round(v[0] / ksum, 4) for k, v in prof.items() if v[1]}
 
-    def gbs(kind, bytes_per_pos, nel):
-        if kind not in prof or not prof[kind][1]:
-            return None
-        per_step_ms = prof[kind][0] / steps
-        return bytes_per_pos * nel / (per_step_ms * 1e-3) / 1e9
+    # roofline of the dominant kernel class (forward GEMM or wgrad GEMM)
+    dom = "linear_fwd" if prof["linear_fwd"][0] >= prof["wgrad"][0] else "wgrad"
+    dom_specs = [s for s in specs if dom == "linear_fwd" or s.wgrad]
+    tc_flops = sum((s.fwd_flops() if dom == "linear_fwd" else s.wgrad_flops()) for s in dom_specs
+                   if uses_tensor_cores(s))
+    simt_flops = sum((s.fwd_flops() if dom == "linear_fwd" else s.wgrad_flops()) for s in dom_specs
+                     if not uses_tensor_cores(s))
+    issued_per_launch = (3.0 * tc_flops + simt_flops) / len(dom_specs)
+    avg_ms = prof[dom][0] / max(prof[dom][1], 1)
+    tf32_peak = peaks["bf16_tflops"] * TF32_OVER_BF16
+    achieved = issued_per_launch / (avg_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": tf32_peak, "unit": "TFLOP/s",
+                "frac": achieved / tf32_peak, "traffic": None, "kernel": dom,
+                "launches_timed": prof[dom][1], "avg_launch_ms": avg_ms,
+                "flops": "issued TF32 flops = 3 x masked flops (3xTF32 split), averaged over the layers",
+                "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x nominal "
+                               f"TF32:BF16 ratio {TF32_OVER_BF16:.4f}"}
 
-    enc_gbs = gbs("encode", (2 * K + 3) * 4, sum(s.G * s.n_in for s in specs))
-    dec_gbs = gbs("decode_verify", (2 * K + 2) * 4, sum(s.G * s.n_out for s in specs))
+    elem = measure_elementwise(torch, dk, synth, ctx, dev, peaks)
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms_total / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "dtype": "tf32x3 (fp32 in/out)", "data": "synthetic",
         "config": {"workload": args.workload, "layers": len(specs), "batch": specs[0].batch, "K": K,
                    "G": specs[0].G, "flops": "masked (all K+2 fwd / K+1 wgrad encodings)",
                    "l2": f"flushed between steps ({L2_FLUSH_BYTES >> 20} MiB write, untimed)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "decoded_useful_tflops": value * (K / (K + 2) * fwd_flops + K / (K + 1) * wg_flops) / step_flops,
-        "encode_gbs": enc_gbs, "decode_gbs": dec_gbs,
-        "encode_frac_hbm": None if enc_gbs is None else enc_gbs / peaks["hbm_gbs"],
-        "decode_frac_hbm": None if dec_gbs is None else dec_gbs / peaks["hbm_gbs"],
+        "encode_gbs": elem["encode"]["gbs"], "decode_gbs": elem["decode"]["gbs"],
+        "encode_frac_hbm": elem["encode"]["frac_hbm"], "decode_frac_hbm": elem["decode"]["frac_hbm"],
+        "elementwise": elem,
         "kernel_ms_per_launch": kernel_ms, "kernel_time_share": share,
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -394,9 +494,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vgg16_cifar")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layer-table", action="store_true")
+    ap.add_argument("--layers", default="")
+    ap.add_argument("--iters", type=int, default=5)
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.layer_table:
+        run_layer_table(args)
     else:
         run_ours(args)
 
