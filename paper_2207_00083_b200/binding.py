@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libdk.so")
 
 DK_FC, DK_CONV2D = 0, 1
 DK_NHWC, DK_NCHW = 0, 1
-DK_PREC_DEFAULT, DK_TF32X3, DK_FP32_SIMT = 0, 1, 2
+DK_PREC_DEFAULT, DK_TF32X3, DK_FP32_SIMT, DK_FP64_SIMT = 0, 1, 2, 3
 STATUS_NAMES = ["DK_OK", "DK_ERR_INVALID_ARG", "DK_ERR_SHAPE", "DK_ERR_SINGULAR", "DK_ERR_WORKSPACE",
                 "DK_ERR_CUDA", "DK_ERR_TIMEOUT", "DK_ERR_UNSUPPORTED"]
 
@@ -98,10 +98,13 @@ def lib() -> ctypes.CDLL:
     return _lib
 
 
-def problem_from_spec(spec, layout: int = DK_NHWC, precision: int = DK_PREC_DEFAULT,
+def problem_from_spec(spec, layout: int = DK_NHWC, precision: Optional[int] = None,
                       tol: float = 0.0, G: Optional[int] = None) -> dk_problem:
-    """dk_problem for a ``synth.LayerSpec``-like object."""
+    """dk_problem for a ``synth.LayerSpec``-like object.  ``precision=None``
+    follows the spec's own hint (fp64 for the high-noise workload)."""
     kind = DK_FC if spec.kind == "fc" else DK_CONV2D
+    if precision is None:
+        precision = DK_FP64_SIMT if getattr(spec, "precision", "default") == "fp64" else DK_PREC_DEFAULT
     return dk_problem(kind, layout, spec.cin, spec.cout, spec.h, spec.w, spec.kh, spec.kw,
                       spec.stride, spec.pad, spec.K, spec.G if G is None else G, precision, tol)
 

@@ -15,7 +15,7 @@ dk_status make_geom(const dk_problem* p, Geom* g) {
   if (!p || !g) return DK_ERR_INVALID_ARG;
   if (p->kind != DK_FC && p->kind != DK_CONV2D) return DK_ERR_INVALID_ARG;
   if (p->layout != DK_NHWC && p->layout != DK_NCHW) return DK_ERR_INVALID_ARG;
-  if (p->precision < DK_PREC_DEFAULT || p->precision > DK_FP32_SIMT) return DK_ERR_INVALID_ARG;
+  if (p->precision < DK_PREC_DEFAULT || p->precision > DK_FP64_SIMT) return DK_ERR_INVALID_ARG;
   if (p->K < 1 || p->K > DK_MAX_K || p->G < 1) return DK_ERR_SHAPE;
   if (p->cin < 1 || p->cout < 1) return DK_ERR_SHAPE;
   memset(g, 0, sizeof(*g));
@@ -210,7 +210,8 @@ static WsPlan plan_workspace(const Geom& g) {
   const size_t xb = align_up((size_t)g.G * g.E * g.n_in * sizeof(float), 1024);
   const size_t wb = align_up((size_t)g.cout * g.kc * sizeof(float), 1024);
   w.xbar = off; off += xb;
-  w.ybar = off; off += align_up((size_t)g.G * g.E * g.n_out * sizeof(float), 1024);
+  // y_bar: sized for doubles (DK_FP64_SIMT keeps it in fp64)
+  w.ybar = off; off += align_up((size_t)g.G * g.E * g.n_out * sizeof(double), 1024);
   w.dtil = off; off += align_up((size_t)g.G * (g.K + 1) * g.n_out * sizeof(float), 1024);
   w.w_hi = off; off += wb;
   w.w_lo = off; off += wb;
@@ -455,6 +456,39 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
       ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
       s = tc_masked_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, cv, bias, y, vs,
                         reinterpret_cast<int*>(vs.count + 1), fault, st);
+    }
+    if (s != DK_OK) return s;
+    ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+    return launch_verify_finalize(g, cv.nul, vs, verdict, st);
+  }
+  if (g.precision == DK_FP64_SIMT) {
+    // beyond-fp32 path: encodings and y_bar stay in the workspace as doubles
+    // (the two adjacent hi/lo regions hold the fp64 encodings)
+    double* x64 = reinterpret_cast<double*>(ws + wp.xb_hi);
+    double* y64 = reinterpret_cast<double*>(ws + wp.ybar);
+    VerifyScratch vs = verify_scratch(ctx, g);
+    {
+      ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
+      s = launch_encode64(g, x, r, cv.enc, x64, xbar_save, ctx->sm_count, st);
+    }
+    if (s != DK_OK) return s;
+    {
+      ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
+      s = launch_simt_fwd64(g, W, x64, y64, g.G * g.E, st);
+    }
+    if (s != DK_OK) return s;
+    {
+      ProfScope ps(ctx, DK_KERNEL_OTHER, fault ? 2 : 1, st);
+      if (fault) {
+        long long idx = ((long long)fault->group * g.E + fault->enc) * g.n_out + fault->out_index;
+        s = launch_add_fault64(y64, idx, fault->delta, st);
+      }
+      if (s == DK_OK) s = launch_verify_begin(g, vs, st);
+    }
+    if (s != DK_OK) return s;
+    {
+      ProfScope ps(ctx, DK_KERNEL_DECODE_VERIFY, 1, st);
+      s = launch_decode_verify64(g, y64, cv, bias, y, vs, ctx->sm_count, st);
     }
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);

@@ -107,6 +107,15 @@ dk_status launch_add_fault(float* ybar, long long index, float delta, cudaStream
 dk_status launch_mix_delta(const Geom& g, const float* delta, const float* dmix, float* dtil,
                            int sm_count, cudaStream_t st);
 
+// fp64 variants for DK_FP64_SIMT (dk_fp64.cu, dk_simt.cu)
+dk_status launch_encode64(const Geom& g, const float* x, const float* r, const float* enc, double* out64,
+                          float* full32, int sm_count, cudaStream_t st);
+dk_status launch_decode_verify64(const Geom& g, const double* ybar, const CoefView& cv, const float* bias,
+                                 float* y, const VerifyScratch& vs, int sm_count, cudaStream_t st);
+dk_status launch_add_fault64(double* ybar, long long index, float delta, cudaStream_t st);
+dk_status launch_simt_fwd64(const Geom& g, const float* W, const double* xbar, double* ybar,
+                            int nsamples, cudaStream_t st);
+
 // SIMT dense kernels (dk_simt.cu)
 dk_status launch_simt_fwd(const Geom& g, const float* W, const float* xbar, float* ybar,
                           int nsamples, cudaStream_t st);

@@ -14,19 +14,26 @@ namespace {
 constexpr int BM = 64, BN = 64, BK = 16, NT = 256;
 constexpr int kFold = 4;   // fold the running sum every kFold k-tiles
 
+__device__ __forceinline__ float fma_t(float a, float b, float c) { return fmaf(a, b, c); }
+__device__ __forceinline__ double fma_t(double a, double b, double c) { return fma(a, b, c); }
+
+// T = type of the activations, of the accumulators and of the output: float,
+// or double for the regime in which fp32 cannot hold the signal next to the noise.
+template <typename T>
 struct FwdParams {
   const float* W;
-  const float* x;
-  float* y;
+  const T* x;
+  T* y;
   int cin, cout, h, w, kw, stride, pad, ho, wo, kc;
   long long N;           // samples * ho * wo
   long long n_in, n_out;
   long long xs_c, xs_h, xs_w, ws_o, ws_c, ws_u, ws_v, ys_c, ys_h, ys_w;
 };
 
-__global__ void __launch_bounds__(NT) simt_fwd_kernel(FwdParams p) {
-  __shared__ float As[BK][BM + 4];
-  __shared__ float Bs[BK][BN + 4];
+template <typename T>
+__global__ void __launch_bounds__(NT) simt_fwd_kernel(FwdParams<T> p) {
+  __shared__ T As[BK][BM + 4];
+  __shared__ T Bs[BK][BN + 4];
   const int t = threadIdx.x;
   const int tx = t % 16, ty = t / 16;
   const int m0 = blockIdx.y * BM;
@@ -56,11 +63,11 @@ __global__ void __launch_bounds__(NT) simt_fwd_kernel(FwdParams p) {
     b_iw0[i] = ow * p.stride - p.pad;
   }
 
-  float tot[4][4], acc[4][4];
+  T tot[4][4], acc[4][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) tot[i][j] = acc[i][j] = 0.f;
+    for (int j = 0; j < 4; ++j) tot[i][j] = acc[i][j] = T(0);
 
   int fold = 0;
   for (int k0 = 0; k0 < p.kc; k0 += BK) {
@@ -73,23 +80,23 @@ __global__ void __launch_bounds__(NT) simt_fwd_kernel(FwdParams p) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       int mm = t / BK + 16 * i;
-      As[kk][mm] = (kok && a_ok[i]) ? __ldg(p.W + a_off[i] + woff) : 0.f;
+      As[kk][mm] = (kok && a_ok[i]) ? T(__ldg(p.W + a_off[i] + woff)) : T(0);
       int ih = b_ih0[i] + u, iw = b_iw0[i] + v;
       bool ok = kok && b_ok[i] && ih >= 0 && ih < p.h && iw >= 0 && iw < p.w;
       Bs[kk][mm] = ok ? __ldg(p.x + b_base[i] + (long long)ci * p.xs_c + (long long)ih * p.xs_h +
                               (long long)iw * p.xs_w)
-                      : 0.f;
+                      : T(0);
     }
     __syncthreads();
 #pragma unroll
     for (int q = 0; q < BK; ++q) {
-      float a[4], b[4];
+      T a[4], b[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) { a[i] = As[q][ty * 4 + i]; b[i] = Bs[q][tx * 4 + i]; }
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        for (int j = 0; j < 4; ++j) acc[i][j] = fma_t(a[i], b[j], acc[i][j]);
     }
     __syncthreads();
     if (++fold == kFold) {
@@ -97,7 +104,7 @@ __global__ void __launch_bounds__(NT) simt_fwd_kernel(FwdParams p) {
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) { tot[i][j] += acc[i][j]; acc[i][j] = 0.f; }
+        for (int j = 0; j < 4; ++j) { tot[i][j] += acc[i][j]; acc[i][j] = T(0); }
     }
   }
 #pragma unroll
@@ -108,7 +115,7 @@ __global__ void __launch_bounds__(NT) simt_fwd_kernel(FwdParams p) {
     long long r = n / p.wo;
     int oh = (int)(r % p.ho);
     long long s = r / p.ho;
-    float* yo = p.y + s * p.n_out + (long long)oh * p.ys_h + (long long)ow * p.ys_w;
+    T* yo = p.y + s * p.n_out + (long long)oh * p.ys_h + (long long)ow * p.ys_w;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       int m = m0 + ty * 4 + i;
@@ -223,9 +230,11 @@ __global__ void __launch_bounds__(NT) simt_wgrad_kernel(WgParams p) {
 
 }  // namespace
 
-dk_status launch_simt_fwd(const Geom& g, const float* W, const float* xbar, float* ybar,
-                          int nsamples, cudaStream_t st) {
-  FwdParams p;
+namespace {
+template <typename T>
+dk_status launch_fwd_t(const Geom& g, const float* W, const T* xbar, T* ybar, int nsamples,
+                       cudaStream_t st) {
+  FwdParams<T> p;
   p.W = W; p.x = xbar; p.y = ybar;
   p.cin = g.cin; p.cout = g.cout; p.h = g.h; p.w = g.w; p.kw = g.kw; p.stride = g.stride;
   p.pad = g.pad; p.ho = g.ho; p.wo = g.wo; p.kc = g.kc;
@@ -238,9 +247,20 @@ dk_status launch_simt_fwd(const Geom& g, const float* W, const float* xbar, floa
   if (nb > 2147483647LL) return DK_ERR_SHAPE;
   dim3 grid((unsigned)nb, (unsigned)((g.cout + BM - 1) / BM));
   if (grid.y > 65535) return DK_ERR_SHAPE;
-  simt_fwd_kernel<<<grid, NT, 0, st>>>(p);
+  simt_fwd_kernel<T><<<grid, NT, 0, st>>>(p);
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
+}
+}  // namespace
+
+dk_status launch_simt_fwd(const Geom& g, const float* W, const float* xbar, float* ybar,
+                          int nsamples, cudaStream_t st) {
+  return launch_fwd_t<float>(g, W, xbar, ybar, nsamples, st);
+}
+
+dk_status launch_simt_fwd64(const Geom& g, const float* W, const double* xbar, double* ybar,
+                            int nsamples, cudaStream_t st) {
+  return launch_fwd_t<double>(g, W, xbar, ybar, nsamples, st);
 }
 
 dk_status launch_simt_wgrad(const Geom& g, const float* dtil, const float* xbar, int xbar_rows,

@@ -246,7 +246,7 @@ void tc_destroy(dk_ctx* ctx) {
 }
 
 bool tc_fwd_supported(const dk_ctx* ctx, const Geom& g) {
-  if (g.precision == DK_FP32_SIMT || ctx->tc_state == nullptr) return false;
+  if (g.precision != DK_TF32X3 || ctx->tc_state == nullptr) return false;
   if (g.layout != DK_NHWC || g.stride != 1 || (g.cin % 4) != 0) return false;
   Tiling tl;
   return plan_tiling<kBK>(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, &tl);
@@ -438,7 +438,7 @@ dk_status launch_wgrad(const WgPlan& w, const CUtensorMap& md_hi, const CUtensor
 }  // namespace
 
 bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g) {
-  if (g.precision == DK_FP32_SIMT || ctx->tc_state == nullptr) return false;
+  if (g.precision != DK_TF32X3 || ctx->tc_state == nullptr) return false;
   if (g.layout != DK_NHWC || g.stride != 1 || (g.cin % 4) != 0 || (g.cout % 4) != 0) return false;
   WgPlan w;
   return plan_wgrad(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, ctx->sm_count, &w);

@@ -61,6 +61,7 @@ class LayerSpec:
     w_std: Optional[float] = None   # None -> Kaiming normal sqrt(2/fan_in)
     wgrad: bool = True
     repeat: int = 1      # how many times this shape occurs in the network
+    precision: str = "default"   # arithmetic hint for the GPU path: "default" or "fp64"
 
     @property
     def hout(self) -> int:
@@ -145,7 +146,10 @@ def layers(workload: str) -> List[LayerSpec]:
             LayerSpec(wl, "fc", "fc", 512, 1000, **kw),
         ]
     if workload == "mobilenetv2_pw":
-        kw = dict(K=8, G=16, sigma_r=1000.0, x_dist="normal", wgrad=False, k=1, p=0)
+        # noise 1000x the activations with K = 8: one fp32 rounding of an encoded
+        # value is ~1e-4 of the decoded result per unit of decoder gain, so this
+        # workload asks the GPU path for its fp64 arithmetic
+        kw = dict(K=8, G=16, sigma_r=1000.0, x_dist="normal", wgrad=False, k=1, p=0, precision="fp64")
         wl = workload
         plan = [("expand_16_96", 16, 96, 112), ("project_96_24", 96, 24, 56),
                 ("expand_24_144", 24, 144, 56), ("project_144_24", 144, 24, 56),

@@ -34,7 +34,7 @@ def small_cases():
     return [
         ("fc784", synth.layers("fc784")[0]),
         ("fc_ragged_K1", tiny("fc", cin=37, cout=19, K=1, G=3)),
-        ("fc_K8", tiny("fc", cin=64, cout=130, K=8, G=2, sigma_r=1000.0, x_dist="normal")),
+        ("fc_K8", tiny("fc", cin=64, cout=130, K=8, G=2, sigma_r=1000.0, x_dist="normal", precision="fp64")),
         ("conv_tiny_K2", tiny()),
         ("conv_ragged_K3", tiny(cin=5, cout=7, h=6, w=5, K=3, G=2)),
         ("conv_7x7s2", tiny(cin=3, cout=16, h=20, w=20, kh=7, kw=7, stride=2, pad=3, K=4, G=1)),
@@ -97,7 +97,7 @@ def test_encode_matches_oracle(ctx, drawn, spec):
 # ---------------------------------------------------------------------------
 # dk_linear_fwd on identical fp32 encodings
 # ---------------------------------------------------------------------------
-@pytest.mark.parametrize("prec", [dk.DK_PREC_DEFAULT, dk.DK_FP32_SIMT], ids=["default", "simt"])
+@pytest.mark.parametrize("prec", [None, dk.DK_FP32_SIMT], ids=["default", "simt"])
 @pytest.mark.parametrize("spec", SPECS, ids=IDS)
 def test_linear_fwd_matches_oracle(ctx, drawn, spec, prec):
     d = drawn(spec)
@@ -166,7 +166,7 @@ def test_decode_verify_matches_oracle(ctx, drawn, spec):
 # ---------------------------------------------------------------------------
 # dk_masked_linear: decoded outputs vs the plain definition, verdicts
 # ---------------------------------------------------------------------------
-@pytest.mark.parametrize("prec", [dk.DK_PREC_DEFAULT, dk.DK_FP32_SIMT], ids=["default", "simt"])
+@pytest.mark.parametrize("prec", [None, dk.DK_FP32_SIMT], ids=["default", "simt"])
 @pytest.mark.parametrize("spec", SPECS, ids=IDS)
 def test_masked_linear_matches_oracle(ctx, drawn, spec, prec):
     d = drawn(spec)
@@ -217,7 +217,7 @@ def test_masked_linear_matches_oracle(ctx, drawn, spec, prec):
 # ---------------------------------------------------------------------------
 # dk_linear_bwd_wgrad
 # ---------------------------------------------------------------------------
-@pytest.mark.parametrize("prec", [dk.DK_PREC_DEFAULT, dk.DK_FP32_SIMT], ids=["default", "simt"])
+@pytest.mark.parametrize("prec", [None, dk.DK_FP32_SIMT], ids=["default", "simt"])
 @pytest.mark.parametrize("rows", ["K+2", "K+1"])
 @pytest.mark.parametrize("spec", SPECS, ids=IDS)
 def test_wgrad_matches_oracle(ctx, drawn, spec, rows, prec):
