@@ -373,7 +373,7 @@ dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W, const 
     }
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
-    return tc_linear_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, ybar, ctx_status_word(ctx), st);
+    return tc_linear_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, ybar, tc_fwd_ksplit(ctx, g), ctx_status_word(ctx), st);
   }
   ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
   return launch_simt_fwd(g, W, xbar, ybar, g.G * g.E, st);
@@ -452,6 +452,31 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
       s = tc_encode_split(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, ctx->sm_count, st);
     }
     if (s != DK_OK) return s;
+    const int ksplit = tc_fwd_ksplit(ctx, g);
+    if (ksplit > 1) {
+      // too few tiles to fill the GPU: slice the contraction, let the slices
+      // meet in y_bar (small here by construction) and decode in a second kernel
+      float* ybar = reinterpret_cast<float*>(ws + wp.ybar);
+      {
+        ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
+        s = tc_linear_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, ybar, ksplit,
+                          reinterpret_cast<int*>(vs.count + 1), st);
+      }
+      if (s != DK_OK) return s;
+      if (fault) {
+        long long idx = ((long long)fault->group * g.E + fault->enc) * g.n_out + fault->out_index;
+        ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+        s = launch_add_fault(ybar, idx, fault->delta, st);
+        if (s != DK_OK) return s;
+      }
+      {
+        ProfScope ps(ctx, DK_KERNEL_DECODE_VERIFY, 1, st);
+        s = launch_decode_verify(g, ybar, cv, bias, y, vs, ctx->sm_count, st);
+      }
+      if (s != DK_OK) return s;
+      ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+      return launch_verify_finalize(g, cv.nul, vs, verdict, st);
+    }
     {
       ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
       s = tc_masked_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, cv, bias, y, vs,

@@ -144,10 +144,12 @@ dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_c
 // Eq. 1 with the split fused in; `full` (nullable) also receives the fp32 encodings
 dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const float* enc, float* full,
                           float* hi, float* lo, int sm_count, cudaStream_t st);
-// y_bar = <W, x_bar> from split operands
+// y_bar = <W, x_bar> from split operands; ksplit > 1 slices the contraction
+// (y_bar is cleared and the slices add into it with atomics)
+int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g);
 dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
-                        const float* xb_hi, const float* xb_lo, float* ybar, int* status_word,
-                        cudaStream_t st);
+                        const float* xb_hi, const float* xb_lo, float* ybar, int ksplit,
+                        int* status_word, cudaStream_t st);
 // weight gradient on tensor cores (channels-last, stride 1, cin % 4 == 0, cout % 4 == 0)
 bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g);
 // Eq. 4 delta mixing written as a TF32 hi/lo pair, [G*(K+1)][n_out] each

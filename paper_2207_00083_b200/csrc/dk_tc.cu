@@ -2,6 +2,8 @@
 // the HBM-bound pre-passes that write the TF32 hi/lo split operands.
 #include <cuda.h>
 
+#include <stdlib.h>
+
 #include <new>
 
 #include "dk_internal.h"
@@ -26,6 +28,16 @@ struct TcState {
 constexpr int kSwz128Atom32 = 1128;
 constexpr int kBK = 32;          // k-block: 32 fp32 = one 128-byte swizzle span per row
 constexpr int kChunk = 2;        // k-blocks accumulated in TMEM between promotions
+
+// Tuning knobs read once from the environment (defaults are the measured best):
+//   DK_TC_CHUNK  k-blocks per TMEM chunk in the forward kernel
+//   DK_WG_CHUNK  k-blocks per TMEM chunk in the weight-gradient kernel
+int env_knob(const char* name, int dflt, int lo, int hi) {
+  const char* v = getenv(name);
+  if (!v || !*v) return dflt;
+  int x = atoi(v);
+  return x < lo ? lo : (x > hi ? hi : x);
+}
 
 // ---------------------------------------------------------------------------
 // HBM-bound pre-passes: TF32 hi/lo split, alone or fused with the encoder
@@ -179,7 +191,8 @@ dk_status launch_one(const TcState* ts, const Geom& g, const Tiling& tl, const f
   DK_CUDA_CHECK(cudaFuncGetAttributes(&fa, kern));
   if (fa.numRegs * kThreadsTc < 40 * 128 + 232 * 256) return DK_ERR_UNSUPPORTED;
   DK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tl.smem_bytes));
-  int grid = tl.ntiles < sm_count ? tl.ntiles : sm_count;
+  const long long nwork = (long long)tl.ntiles * prm.ksplit;
+  int grid = nwork < sm_count ? (int)nwork : sm_count;
   kern<<<grid, kThreadsTc, tl.smem_bytes, st>>>(ma_hi, ma_lo, mb_hi, mb_lo, prm);
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
@@ -205,7 +218,10 @@ void fill_params(const Geom& g, const Tiling& tl, TcParams* p) {
   p->bw = tl.bw; p->bh = tl.bh; p->bg = tl.bg;
   p->WT = tl.WT; p->HT = tl.HT; p->GT = tl.GT; p->MT = tl.MT;
   p->ntiles = tl.ntiles; p->KB = tl.KB; p->CB = tl.CB;
-  p->chunk = kChunk;
+  static const int chunk = env_knob("DK_TC_CHUNK", kChunk, 1, 64);
+  p->chunk = chunk;
+  p->ksplit = 1;
+  p->kb_per_split = tl.KB;
   p->kw = g.kw; p->pad = g.pad; p->nstages = tl.nstages;
   p->cout = g.cout; p->ho = g.ho; p->wo = g.wo; p->G = g.G;
   p->n_out = g.n_out;
@@ -285,13 +301,31 @@ dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const f
   return DK_OK;
 }
 
+// Contraction slices for problems with fewer tiles than SMs: each slice keeps
+// at least 8 k-blocks, and the slices of a tile add into y_bar with atomics.
+int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g) {
+  TcState* ts = static_cast<TcState*>(ctx->tc_state);
+  Tiling tl;
+  if (!ts || !plan_tiling<kBK>(g, ts->smem_optin, &tl)) return 1;
+  if (tl.ntiles * 2 > ctx->sm_count) return 1;
+  int want = (ctx->sm_count + tl.ntiles - 1) / tl.ntiles;
+  int cap = tl.KB / 8;
+  if (want > cap) want = cap;
+  return want < 1 ? 1 : want;
+}
+
 dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
-                        const float* xb_lo, float* ybar, int* status_word, cudaStream_t st) {
+                        const float* xb_lo, float* ybar, int ksplit, int* status_word, cudaStream_t st) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!plan_tiling<kBK>(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
   TcParams prm;
   fill_params(g, tl, &prm);
+  if (ksplit > 1) {
+    prm.kb_per_split = (tl.KB + ksplit - 1) / ksplit;
+    prm.ksplit = (tl.KB + prm.kb_per_split - 1) / prm.kb_per_split;
+    DK_CUDA_CHECK(cudaMemsetAsync(ybar, 0, (size_t)g.G * g.E * g.n_out * sizeof(float), st));
+  }
   prm.out = ybar;
   prm.status = status_word;
   return launch_k<kBK, MODE_YBAR>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
@@ -401,6 +435,9 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   p.taps = g.kh * g.kw;
   const long long base = (long long)p.MT * p.NB * p.taps;
   long long nsplit = (2LL * sm_count + base - 1) / base;
+  // every slice ends in cout x cin atomics: keep at least 16 k-blocks of work behind them
+  const long long by_work = ((long long)p.PB * p.K1) / 16;
+  if (nsplit > by_work) nsplit = by_work;
   if (nsplit > p.PB) nsplit = p.PB;
   if (nsplit < 1) nsplit = 1;
   p.pb_per_split = (int)((p.PB + nsplit - 1) / nsplit);
@@ -409,7 +446,8 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   if (items > 0x7fffffffLL) return false;
   p.nitems = (int)items;
   p.kw = g.kw; p.pad = g.pad;
-  p.chunk = kWgChunk;
+  static const int wg_chunk = env_knob("DK_WG_CHUNK", kWgChunk, 1, 64);
+  p.chunk = wg_chunk;
   p.cout = g.cout; p.cin = g.cin;
   const size_t stage = 2 * ((size_t)(BM / 32) * kWgBox + (size_t)(w->BN / 32) * kWgBox);
   const size_t ctrl = 1024 + 256;

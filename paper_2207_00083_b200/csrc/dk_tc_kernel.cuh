@@ -57,6 +57,7 @@ struct TcParams {
   int ntiles;
   int KB, CB;                  // k-blocks in total and per filter tap
   int chunk;                   // k-blocks accumulated in TMEM before promotion
+  int ksplit, kb_per_split;    // contraction slices per tile (slices add into `out` with atomics)
   int kw, pad;
   int nstages;
   // problem
@@ -202,7 +203,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nchunks = (p.KB + p.chunk - 1) / p.chunk;
+  const int nwork = p.ntiles * p.ksplit;     // work item = (tile, contraction slice)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.nstages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
@@ -230,33 +231,47 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
   asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
   if (warp == 0) {
     // ---------------- TMA producer ----------------
-    if (lane == 0) {
+    // The whole warp runs the loop: lane 0 waits for the stage and arms its
+    // barrier, then lanes 0..2E+1 issue one bulk tensor copy each, so that the
+    // 2E+2 copies of a stage are issued side by side instead of one after another.
+    {
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
-      for (int t = blockIdx.x; alive && t < p.ntiles; t += gridDim.x) {
+      for (int w = blockIdx.x; alive && w < nwork; w += gridDim.x) {
+        const int t = w / p.ksplit, ks = w - t * p.ksplit;
+        const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
         const int mt = t % p.MT;
         int nt = t / p.MT;
         const int wt = nt % p.WT; nt /= p.WT;
         const int ht = nt % p.HT;
         const int gt = nt / p.HT;
         const int x0 = wt * p.bw - p.pad, y0 = ht * p.bh - p.pad, g0 = gt * p.bg, m0 = mt * BM;
-        for (int kb = 0; kb < p.KB; ++kb) {
-          if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) { alive = false; break; }
+        for (int kb = kb_lo; kb < kb_hi; ++kb) {
+          int ok = 1;
+          if (lane == 0) {
+            ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag) ? 1 : 0;
+            if (ok) mbar_expect_tx(full_bar + stage, (uint32_t)STAGE_BYTES);
+          }
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) { alive = false; break; }
           const int tap = kb / p.CB, c0 = (kb - tap * p.CB) * BK;
           const int u = tap / p.kw, v = tap - u * p.kw;
           unsigned char* st = smem + (size_t)stage * STAGE_BYTES;
-          mbar_expect_tx(full_bar + stage, (uint32_t)STAGE_BYTES);
-          tma_load_3d(st, &map_a_hi, full_bar + stage, c0, tap, m0);
-          tma_load_3d(st + A_BYTES, &map_a_lo, full_bar + stage, c0, tap, m0);
-          unsigned char* bh = st + 2 * A_BYTES;
-          unsigned char* bl = bh + B_BYTES;
           constexpr int SUB = P * BK * 4;
-#pragma unroll 1
-          for (int e = 0; e < E; ++e) {
-            tma_load_5d(bh + e * SUB, &map_b_hi, full_bar + stage, c0, x0 + v, y0 + u, e, g0);
-            tma_load_5d(bl + e * SUB, &map_b_lo, full_bar + stage, c0, x0 + v, y0 + u, e, g0);
+          if (lane == 0) {
+            tma_load_3d(st, &map_a_hi, full_bar + stage, c0, tap, m0);
+          } else if (lane == 1) {
+            tma_load_3d(st + A_BYTES, &map_a_lo, full_bar + stage, c0, tap, m0);
+          } else if (lane < 2 + 2 * E) {
+            const int e = (lane - 2) >> 1;
+            if ((lane & 1) == 0)
+              tma_load_5d(st + 2 * A_BYTES + e * SUB, &map_b_hi, full_bar + stage, c0, x0 + v, y0 + u, e, g0);
+            else
+              tma_load_5d(st + 2 * A_BYTES + B_BYTES + e * SUB, &map_b_lo, full_bar + stage, c0, x0 + v, y0 + u,
+                          e, g0);
           }
+          __syncwarp();
           if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -270,21 +285,24 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
       uint32_t phase = 0;
       uint32_t acc_it = 0;     // chunks issued so far (all tiles)
       bool alive = true;
-      for (int t = blockIdx.x; alive && t < p.ntiles; t += gridDim.x) {
+      for (int w = blockIdx.x; alive && w < nwork; w += gridDim.x) {
+        const int ks = w % p.ksplit;
+        const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
+        const int nchunks = (kb_hi - kb_lo + p.chunk - 1) / p.chunk;
         for (int ci = 0; alive && ci < nchunks; ++ci, ++acc_it) {
           const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
           if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag)) { alive = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * 256u;
-          const int kb_end = min(p.KB, (ci + 1) * p.chunk);
-          for (int kb = ci * p.chunk; kb < kb_end; ++kb) {
+          const int kb_beg = kb_lo + ci * p.chunk, kb_end = min(kb_hi, kb_beg + p.chunk);
+          for (int kb = kb_beg; kb < kb_end; ++kb) {
             if (!mbar_wait(full_bar + stage, phase, abort_flag)) { alive = false; break; }
             tc_fence_after();
             const uint32_t st = smem_u32(smem + (size_t)stage * STAGE_BYTES);
             const uint64_t a_hi = make_desc<SWZ>(st), a_lo = make_desc<SWZ>(st + A_BYTES);
             const uint64_t b_hi = make_desc<SWZ>(st + 2 * A_BYTES);
             const uint64_t b_lo = make_desc<SWZ>(st + 2 * A_BYTES + B_BYTES);
-            const bool first = kb == ci * p.chunk;
+            const bool first = kb == kb_beg;
 #pragma unroll
             for (int kk = 0; kk < BK / 8; ++kk) {
               const uint64_t adv = (uint64_t)(kk * 2);     // 32 bytes per k-step, in 16-byte units
@@ -309,7 +327,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
     uint32_t acc_it = 0;
     bool alive = true;
     float acc[E][PH];
-    for (int t = blockIdx.x; alive && t < p.ntiles; t += gridDim.x) {
+    for (int w = blockIdx.x; alive && w < nwork; w += gridDim.x) {
+      const int t = w / p.ksplit, ks = w - t * p.ksplit;
+      const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
+      const int nchunks = (kb_hi - kb_lo + p.chunk - 1) / p.chunk;
       const int mt = t % p.MT;
       int nt = t / p.MT;
       const int wt = nt % p.WT; nt /= p.WT;
@@ -383,7 +404,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
           if (in_range && co_ok) {
             float* dst = p.out + ((size_t)g * E) * p.n_out + ((size_t)oh * p.wo + ow) * p.cout + co;
 #pragma unroll
-            for (int e = 0; e < E; ++e) dst[(size_t)e * p.n_out] = acc[e][j];
+            for (int e = 0; e < E; ++e) {
+              if (p.ksplit > 1) atomicAdd(dst + (size_t)e * p.n_out, acc[e][j]);   // `out` was cleared
+              else dst[(size_t)e * p.n_out] = acc[e][j];
+            }
           }
         } else {
           if (g != cur_g) {      // warp-uniform: g depends on the tile and the pixel only

@@ -114,11 +114,15 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
   static_assert(40 * 128 + 232 * 256 <= 168 * kThreadsTc, "setmaxnreg budget exceeds the CTA's register pool");
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
-    if (warp == 0 && lane == 0) {
+    if (warp == 0) {
       // ---------------- TMA producer ----------------
+      // whole warp: lane 0 arms the stage, then each lane issues its share of
+      // the 2*(BM+BN)/32 box copies so that they go out side by side
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
+      constexpr int NBOX = 2 * (BM / 32) + 2 * (BN / 32);
+      static_assert(NBOX <= 32, "one box per lane");
       for (int item = blockIdx.x; alive && item < p.nitems; item += gridDim.x) {
         int mt, nb, tap, pb_lo, pb_hi;
         item_range(item, mt, nb, tap, pb_lo, pb_hi);
@@ -131,22 +135,32 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
           const int gt = r / p.HT;
           const int x0 = wt * p.bw, y0 = ht * p.bh, g0 = gt * p.bg;
           for (int j = 0; j < p.K1; ++j) {
-            if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) { alive = false; break; }
+            int ok = 1;
+            if (lane == 0) {
+              ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag) ? 1 : 0;
+              if (ok) mbar_expect_tx(full_bar + stage, (uint32_t)STAGE_BYTES);
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) { alive = false; break; }
             unsigned char* st = smem + (size_t)stage * STAGE_BYTES;
-            mbar_expect_tx(full_bar + stage, (uint32_t)STAGE_BYTES);
-#pragma unroll 1
-            for (int cb = 0; cb < BM / 32; ++cb) {
-              tma_load_5d(st + cb * kWgBox, &map_d_hi, full_bar + stage, m0 + cb * 32, x0, y0, j, g0);
-              tma_load_5d(st + A_BYTES + cb * kWgBox, &map_d_lo, full_bar + stage, m0 + cb * 32, x0, y0, j, g0);
+            if (lane < 2 * (BM / 32)) {
+              const int cb = lane >> 1;
+              if ((lane & 1) == 0)
+                tma_load_5d(st + cb * kWgBox, &map_d_hi, full_bar + stage, m0 + cb * 32, x0, y0, j, g0);
+              else
+                tma_load_5d(st + A_BYTES + cb * kWgBox, &map_d_lo, full_bar + stage, m0 + cb * 32, x0, y0, j, g0);
+            } else if (lane < NBOX) {
+              const int q = lane - 2 * (BM / 32);
+              const int cb = q >> 1;
+              unsigned char* bh = st + 2 * A_BYTES;
+              if ((q & 1) == 0)
+                tma_load_5d(bh + cb * kWgBox, &map_x_hi, full_bar + stage, n0 + cb * 32, x0 + v - p.pad,
+                            y0 + u - p.pad, j, g0);
+              else
+                tma_load_5d(bh + B_BYTES + cb * kWgBox, &map_x_lo, full_bar + stage, n0 + cb * 32,
+                            x0 + v - p.pad, y0 + u - p.pad, j, g0);
             }
-            unsigned char* bh = st + 2 * A_BYTES;
-#pragma unroll 1
-            for (int cb = 0; cb < BN / 32; ++cb) {
-              tma_load_5d(bh + cb * kWgBox, &map_x_hi, full_bar + stage, n0 + cb * 32, x0 + v - p.pad,
-                          y0 + u - p.pad, j, g0);
-              tma_load_5d(bh + B_BYTES + cb * kWgBox, &map_x_lo, full_bar + stage, n0 + cb * 32, x0 + v - p.pad,
-                          y0 + u - p.pad, j, g0);
-            }
+            __syncwarp();
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
           }
         }

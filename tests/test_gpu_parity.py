@@ -190,10 +190,11 @@ def test_masked_linear_matches_oracle(ctx, drawn, spec, prec):
     assert H.max_rel(got_y, clean["y"]) < TOL_DECODED
     assert H.max_rel(H.acts_from_dev(xsave, lay(spec)), clean["xbar"]) < TOL_ENCODE
 
-    # without xbar_save the result is the same
+    # without xbar_save the result is the same (up to the order of the fp32
+    # atomics with which contraction slices of small problems meet in y_bar)
     y2 = torch.empty_like(y)
     dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y2, None, v)
-    assert torch.equal(y, y2)
+    assert float((y - y2).abs().max()) <= 1e-4 * float(y.abs().max())
 
     # one wrong accelerator output in every encoding row is flagged, exactly once
     for fault in _fault_list(spec)[1:]:
