@@ -27,7 +27,7 @@ struct TcState {
 
 constexpr int kSwz128Atom32 = 1128;
 constexpr int kBK = 32;          // k-block: 32 fp32 = one 128-byte swizzle span per row
-constexpr int kChunk = 2;        // k-blocks accumulated in TMEM between promotions
+constexpr int kChunk = 4;        // k-blocks accumulated in TMEM between promotions (error grows ~linearly with it)
 
 // Tuning knobs read once from the environment (defaults are the measured best):
 //   DK_TC_CHUNK  k-blocks per TMEM chunk in the forward kernel
@@ -360,7 +360,7 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
 // ---------------------------------------------------------------------------
 namespace {
 
-constexpr int kWgChunk = 1;      // k-blocks accumulated in TMEM between promotions
+constexpr int kWgChunk = 2;      // k-blocks accumulated in TMEM between promotions
 
 // dtil[g*(K+1)+j] = sum_i dmix[g][j][i] * delta[g*K+i], written as a TF32 hi/lo pair (Eq. 4).
 template <int K>

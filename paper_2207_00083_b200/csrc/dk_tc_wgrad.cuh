@@ -242,9 +242,14 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
       if (co < p.cout && nchunks > 0) {
         float* dst = p.dW + ((size_t)co * p.taps + tap) * p.cin + nb * BN + half * NH;
         const int nvalid = p.cin - (nb * BN + half * NH);
+        // 16-byte vector reductions: cin % 4 == 0 keeps every group of four
+        // either wholly inside or wholly outside the row, and dst 16-byte aligned
 #pragma unroll
-        for (int c = 0; c < NH; ++c)
-          if (c < nvalid) atomicAdd(dst + c, p.scale * acc[c]);
+        for (int c = 0; c < NH; c += 4)
+          if (c < nvalid)
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + c), "f"(p.scale * acc[c]),
+                         "f"(p.scale * acc[c + 1]), "f"(p.scale * acc[c + 2]), "f"(p.scale * acc[c + 3])
+                         : "memory");
       }
     }
   }

@@ -4,7 +4,8 @@
 
 For every small parity case: max-norm relative error of y_bar (dk_linear_fwd on
 identical fp32 encodings) and of the decoded y (dk_masked_linear against the
-plain definition), and the honest max_ratio of the integrity check, for the
+plain definition), the honest max_ratio of the integrity check and the error of dW
+(dk_linear_bwd_wgrad on fp32 encodings against the plain definition), for the
 tensor-core 3xTF32 mode, the fp32 SIMT mode and the fp64 mode.  Reporting aid
 for the choice of arithmetic; the pass/fail bars live in the test files."""
 import numpy as np
@@ -21,7 +22,8 @@ def main():
     extra = [("vgg_cifar_conv4_2_G4", synth.layer("vgg16_cifar", "conv4_2").with_groups(4)),
              ("vgg_cifar_conv1_2_G2", synth.layer("vgg16_cifar", "conv1_2").with_groups(2)),
              ("mbv2_expand_160_960_G2", synth.layer("mobilenetv2_pw", "expand_160_960").with_groups(2))]
-    print(f"{'case':28s} {'K':>2s} {'sigma':>6s} {'kc':>6s} {'mode':>5s} {'ybar':>9s} {'y':>9s} {'maxratio':>9s}")
+    print(f"{'case':28s} {'K':>2s} {'sigma':>6s} {'kc':>6s} {'mode':>6s} {'ybar':>9s} {'y':>9s} {'maxratio':>9s} "
+          f"{'dW':>9s}")
     for name, spec in CASES + extra:
         d = synth.draw_layer(spec)
         K, E = spec.K, spec.K + 2
@@ -41,8 +43,14 @@ def main():
                                 None, v)
             e2 = H.max_rel(H.acts_from_dev(y, 0), plain)
             vd = dk.read_verdict(v)
+            dW = H.empty_weights(spec, 0)
+            scale = 1.0 / spec.batch
+            dk.dk_linear_bwd_wgrad(ctx, p, H.acts_to_dev(d["delta"], 0), H.acts_to_dev(xbar32, 0), E, d["C"],
+                                   d["gamma"], scale, dW)
+            want_dw = O.wgrad_plain(d["delta"], d["x"], scale, spec.kh, spec.kw, spec.stride, spec.pad)
+            e3 = H.max_rel(H.weights_from_dev(dW, 0), want_dw)
             print(f"{name:28s} {K:2d} {spec.sigma_r:6.0f} {spec.kc:6d} {pn:>6s} {e1:9.2e} {e2:9.2e} "
-                  f"{vd['max_ratio']:9.2e} ok={vd['ok']}")
+                  f"{vd['max_ratio']:9.2e} {e3:9.2e} ok={vd['ok']}")
     ctx.close()
 
 
