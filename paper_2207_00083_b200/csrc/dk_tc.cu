@@ -39,6 +39,13 @@ int env_knob(const char* name, int dflt, int lo, int hi) {
   return x < lo ? lo : (x > hi ? hi : x);
 }
 
+// k-block of the forward kernel: 32 fp32 (128-byte rows, fewer and larger
+// stages) or 16 (64-byte rows, twice as many stages in the same shared memory)
+int fwd_bk() {
+  static const int bk = env_knob("DK_TC_BK", kBK, 16, 32) == 16 ? 16 : 32;
+  return bk;
+}
+
 // ---------------------------------------------------------------------------
 // HBM-bound pre-passes: TF32 hi/lo split, alone or fused with the encoder
 // ---------------------------------------------------------------------------
@@ -216,10 +223,12 @@ dk_status launch_k(const TcState* ts, const Geom& g, const Tiling& tl, const flo
 
 void fill_params(const Geom& g, const Tiling& tl, TcParams* p) {
   p->bw = tl.bw; p->bh = tl.bh; p->bg = tl.bg;
+  p->log2_bw = 0; while ((1 << p->log2_bw) < tl.bw) ++p->log2_bw;
+  p->log2_S = 0; while ((1 << p->log2_S) < tl.bw * tl.bh) ++p->log2_S;
   p->WT = tl.WT; p->HT = tl.HT; p->GT = tl.GT; p->MT = tl.MT;
   p->ntiles = tl.ntiles; p->KB = tl.KB; p->CB = tl.CB;
   static const int chunk = env_knob("DK_TC_CHUNK", kChunk, 1, 64);
-  p->chunk = chunk;
+  p->chunk = chunk * (32 / fwd_bk());   // the knob counts 32-wide k-blocks
   p->ksplit = 1;
   p->kb_per_split = tl.KB;
   p->kw = g.kw; p->pad = g.pad; p->nstages = tl.nstages;
@@ -231,6 +240,17 @@ void fill_params(const Geom& g, const Tiling& tl, TcParams* p) {
   p->status = nullptr;
   p->f_group = -1; p->f_enc = p->f_co = p->f_oh = p->f_ow = 0;
   p->f_delta = 0.f;
+}
+
+bool plan_fwd(const Geom& g, int smem_optin, Tiling* t) {
+  return fwd_bk() == 16 ? plan_tiling<16>(g, smem_optin, t) : plan_tiling<32>(g, smem_optin, t);
+}
+
+template <int MODE>
+dk_status launch_bk(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
+                    const float* xb_hi, const float* xb_lo, TcParams& prm, int sm_count, cudaStream_t st) {
+  return fwd_bk() == 16 ? launch_k<16, MODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st)
+                        : launch_k<32, MODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
 }
 
 }  // namespace
@@ -264,8 +284,9 @@ void tc_destroy(dk_ctx* ctx) {
 bool tc_fwd_supported(const dk_ctx* ctx, const Geom& g) {
   if (g.precision != DK_TF32X3 || ctx->tc_state == nullptr) return false;
   if (g.layout != DK_NHWC || g.stride != 1 || (g.cin % 4) != 0) return false;
+  if (g.n_out >= (1LL << 31)) return false;     // the epilogue keeps pixel offsets in 32 bits
   Tiling tl;
-  return plan_tiling<kBK>(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, &tl);
+  return plan_fwd(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, &tl);
 }
 
 dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_count, cudaStream_t st) {
@@ -306,10 +327,10 @@ dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const f
 int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
-  if (!ts || !plan_tiling<kBK>(g, ts->smem_optin, &tl)) return 1;
+  if (!ts || !plan_fwd(g, ts->smem_optin, &tl)) return 1;
   if (tl.ntiles * 2 > ctx->sm_count) return 1;
   int want = (ctx->sm_count + tl.ntiles - 1) / tl.ntiles;
-  int cap = tl.KB / 8;
+  int cap = tl.KB / (8 * (32 / fwd_bk()));
   if (want > cap) want = cap;
   return want < 1 ? 1 : want;
 }
@@ -318,7 +339,7 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
                         const float* xb_lo, float* ybar, int ksplit, int* status_word, cudaStream_t st) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
-  if (!plan_tiling<kBK>(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
+  if (!plan_fwd(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
   TcParams prm;
   fill_params(g, tl, &prm);
   if (ksplit > 1) {
@@ -328,7 +349,7 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   }
   prm.out = ybar;
   prm.status = status_word;
-  return launch_k<kBK, MODE_YBAR>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
+  return launch_bk<MODE_YBAR>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
 }
 
 dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
@@ -336,7 +357,7 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
                         const VerifyScratch& vs, int* status_word, const dk_fault* fault, cudaStream_t st) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
-  if (!plan_tiling<kBK>(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
+  if (!plan_fwd(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
   TcParams prm;
   fill_params(g, tl, &prm);
   prm.out = y;
@@ -352,7 +373,7 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
     prm.f_ow = (int)(pix - (long long)prm.f_oh * g.wo);
     prm.f_delta = fault->delta;
   }
-  return launch_k<kBK, MODE_DECODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
+  return launch_bk<MODE_DECODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
 }
 
 // ---------------------------------------------------------------------------
