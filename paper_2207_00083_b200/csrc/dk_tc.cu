@@ -8,6 +8,7 @@
 
 #include "dk_internal.h"
 #include "dk_tc_kernel.cuh"
+#include "dk_tc_pair.cuh"
 #include "dk_tc_wgrad.cuh"
 
 namespace dk {
@@ -110,11 +111,12 @@ encode_split_kernel(const float* __restrict__ x, const float* __restrict__ r, co
 // ---------------------------------------------------------------------------
 struct Tiling {
   int P, bw, bh, bg, WT, HT, GT, MT, ntiles, KB, CB, nstages, BN;
+  bool pair;               // tiles of 256 output channels on CTA pairs
   size_t smem_bytes;
 };
 
 template <int BK>
-bool plan_tiling(const Geom& g, int smem_optin, Tiling* t) {
+bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
   const int E = g.E;
   const int P = tile_pixels(g.K);
   // Box shape bw x bh x bg with bw*bh*bg = P (bw, bh powers of two): the one
@@ -137,14 +139,16 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t) {
   t->WT = (g.wo + t->bw - 1) / t->bw;
   t->HT = (g.ho + t->bh - 1) / t->bh;
   t->GT = (g.G + t->bg - 1) / t->bg;
-  t->MT = (g.cout + BM - 1) / BM;
+  t->pair = pair;
+  t->MT = pair ? (g.cout + BM2 - 1) / BM2 : (g.cout + BM - 1) / BM;
   long long nt = (long long)t->WT * t->HT * t->GT * t->MT;
   if (nt > 0x7fffffffLL) return false;
   t->ntiles = (int)nt;
   t->CB = (g.cin + BK - 1) / BK;
   t->KB = t->CB * g.kh * g.kw;
   t->BN = E * P;
-  const size_t stage = 2 * ((size_t)BM * BK * 4 + (size_t)t->BN * BK * 4);
+  // a CTA of a pair stages its own 128 rows of W and half of the activation rows
+  const size_t stage = 2 * ((size_t)BM * BK * 4 + (size_t)(pair ? t->BN / 2 : t->BN) * BK * 4);
   const size_t ctrl = 1024 + 256;   // alignment slack + barriers
   int ns = (int)(((size_t)smem_optin - ctrl) / stage);
   if (ns > kMaxStages) ns = kMaxStages;
@@ -169,28 +173,39 @@ bool encode_map(const TcState* ts, CUtensorMap* m, const void* base, int rank, c
   return r == CUDA_SUCCESS;
 }
 
-template <int BK, int MODE, int K>
-dk_status launch_one(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
-                     const float* xb_hi, const float* xb_lo, TcParams& prm, int sm_count, cudaStream_t st) {
-  CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo;
+// Tensor maps of the forward kernels: W as [cout][tap][cin] with a box of 128
+// output channels x one tap x BK channels; the encoded activations as
+// [G][E][h][w][cin] with one box of the tile's pixels per encoding.
+template <int BK>
+bool encode_fwd_maps(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
+                     const float* xb_hi, const float* xb_lo, CUtensorMap* ma_hi, CUtensorMap* ma_lo,
+                     CUtensorMap* mb_hi, CUtensorMap* mb_lo) {
   const int taps = g.kh * g.kw;
   {
     cuuint64_t dims[3] = {(cuuint64_t)g.cin, (cuuint64_t)taps, (cuuint64_t)g.cout};
     cuuint64_t str[2] = {(cuuint64_t)g.cin * 4, (cuuint64_t)g.cin * taps * 4};
     cuuint32_t box[3] = {(cuuint32_t)BK, 1, (cuuint32_t)BM};
-    if (!encode_map(ts, &ma_hi, w_hi, 3, dims, str, box, BK * 4) ||
-        !encode_map(ts, &ma_lo, w_lo, 3, dims, str, box, BK * 4))
-      return DK_ERR_CUDA;
+    if (!encode_map(ts, ma_hi, w_hi, 3, dims, str, box, BK * 4) ||
+        !encode_map(ts, ma_lo, w_lo, 3, dims, str, box, BK * 4))
+      return false;
   }
   {
     cuuint64_t dims[5] = {(cuuint64_t)g.cin, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.E, (cuuint64_t)g.G};
     cuuint64_t str[4] = {(cuuint64_t)g.cin * 4, (cuuint64_t)g.cin * g.w * 4, (cuuint64_t)g.n_in * 4,
                          (cuuint64_t)g.n_in * g.E * 4};
     cuuint32_t box[5] = {(cuuint32_t)BK, (cuuint32_t)tl.bw, (cuuint32_t)tl.bh, 1, (cuuint32_t)tl.bg};
-    if (!encode_map(ts, &mb_hi, xb_hi, 5, dims, str, box, BK * 4) ||
-        !encode_map(ts, &mb_lo, xb_lo, 5, dims, str, box, BK * 4))
-      return DK_ERR_CUDA;
+    if (!encode_map(ts, mb_hi, xb_hi, 5, dims, str, box, BK * 4) ||
+        !encode_map(ts, mb_lo, xb_lo, 5, dims, str, box, BK * 4))
+      return false;
   }
+  return true;
+}
+
+template <int BK, int MODE, int K>
+dk_status launch_one(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
+                     const float* xb_hi, const float* xb_lo, TcParams& prm, int sm_count, cudaStream_t st) {
+  CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo;
+  if (!encode_fwd_maps<BK>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, &ma_hi, &ma_lo, &mb_hi, &mb_lo)) return DK_ERR_CUDA;
   auto kern = tc_fwd_kernel<BK, MODE, K>;
   // The kernel re-partitions registers between its warpgroups and would wait
   // forever if the pool it was launched with were smaller than it assumes.
@@ -203,6 +218,41 @@ dk_status launch_one(const TcState* ts, const Geom& g, const Tiling& tl, const f
   kern<<<grid, kThreadsTc, tl.smem_bytes, st>>>(ma_hi, ma_lo, mb_hi, mb_lo, prm);
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
+}
+
+// CTA-pair kernel (even K only): grid = 2 x the number of resident pairs
+template <int MODE, int K>
+dk_status launch_pair_one(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
+                          const float* xb_hi, const float* xb_lo, TcParams& prm, int sm_count, cudaStream_t st) {
+  if constexpr (K % 2 != 0) {
+    return DK_ERR_UNSUPPORTED;
+  } else {
+    CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo;
+    if (!encode_fwd_maps<32>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, &ma_hi, &ma_lo, &mb_hi, &mb_lo)) return DK_ERR_CUDA;
+    auto kern = tc_fwd_pair_kernel<MODE, K>;
+    cudaFuncAttributes fa;
+    DK_CUDA_CHECK(cudaFuncGetAttributes(&fa, kern));
+    if (fa.numRegs * kThreadsTc < 40 * 128 + 232 * 256) return DK_ERR_UNSUPPORTED;
+    DK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tl.smem_bytes));
+    const long long nwork = (long long)tl.ntiles * prm.ksplit;
+    int pairs = sm_count / 2;
+    {
+      // pairs that can be resident together (a GPC with an odd SM leaves one out)
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)(2 * pairs));
+      cfg.blockDim = dim3(kThreadsTc);
+      cfg.dynamicSmemBytes = tl.smem_bytes;
+      int active = 0;
+      if (cudaOccupancyMaxActiveClusters(&active, kern, &cfg) == cudaSuccess && active > 0 && active < pairs)
+        pairs = active;
+      else
+        (void)cudaGetLastError();
+    }
+    if (nwork < pairs) pairs = (int)nwork;
+    kern<<<2 * pairs, kThreadsTc, tl.smem_bytes, st>>>(ma_hi, ma_lo, mb_hi, mb_lo, prm);
+    DK_CUDA_CHECK(cudaGetLastError());
+    return DK_OK;
+  }
 }
 
 template <int BK, int MODE>
@@ -242,13 +292,34 @@ void fill_params(const Geom& g, const Tiling& tl, TcParams* p) {
   p->f_delta = 0.f;
 }
 
+// CTA pairs serve layers with more than 128 output channels and an even
+// number of encodings (DK_TC_PAIR=0 switches them off)
+bool use_pair(const Geom& g) {
+  static const int on = env_knob("DK_TC_PAIR", 1, 0, 1);
+  return on && fwd_bk() == 32 && g.cout > BM && (g.E % 2) == 0;
+}
+
 bool plan_fwd(const Geom& g, int smem_optin, Tiling* t) {
+  if (use_pair(g) && plan_tiling<32>(g, smem_optin, t, true)) return true;
   return fwd_bk() == 16 ? plan_tiling<16>(g, smem_optin, t) : plan_tiling<32>(g, smem_optin, t);
+}
+
+template <int MODE>
+dk_status launch_pair(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
+                      const float* xb_hi, const float* xb_lo, TcParams& prm, int sm_count, cudaStream_t st) {
+  switch (g.K) {
+    case 2: return launch_pair_one<MODE, 2>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+    case 4: return launch_pair_one<MODE, 4>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+    case 6: return launch_pair_one<MODE, 6>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+    case 8: return launch_pair_one<MODE, 8>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
+  }
+  return DK_ERR_UNSUPPORTED;
 }
 
 template <int MODE>
 dk_status launch_bk(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
                     const float* xb_hi, const float* xb_lo, TcParams& prm, int sm_count, cudaStream_t st) {
+  if (tl.pair) return launch_pair<MODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
   return fwd_bk() == 16 ? launch_k<16, MODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st)
                         : launch_k<32, MODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
 }
@@ -328,8 +399,9 @@ int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!ts || !plan_fwd(g, ts->smem_optin, &tl)) return 1;
-  if (tl.ntiles * 2 > ctx->sm_count) return 1;
-  int want = (ctx->sm_count + tl.ntiles - 1) / tl.ntiles;
+  const int units = tl.pair ? ctx->sm_count / 2 : ctx->sm_count;     // CTAs or CTA pairs that run together
+  if (tl.ntiles * 2 > units) return 1;
+  int want = (units + tl.ntiles - 1) / tl.ntiles;
   int cap = tl.KB / (8 * (32 / fwd_bk()));
   if (want > cap) want = cap;
   return want < 1 ? 1 : want;

@@ -177,6 +177,267 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
 }
 
 // ---------------------------------------------------------------------------
+// Epilogue of one tile, from the fp32 sums in registers: stores the encoded
+// outputs (MODE_YBAR) or decodes them, evaluates the integrity residual and
+// collects the statistics of the check (MODE_DECODE).  Thread (quad, lane)
+// owns output channel `co`; `half` selects its PH of the tile's P pixels.
+// ---------------------------------------------------------------------------
+template <int MODE, int K>
+__device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K + 2][tile_pixels(K) / 2], int half,
+                                              int lane, int co, bool co_ok, int gt, int ht, int wt) {
+  constexpr int E = K + 2, K1 = K + 1;
+  constexpr int PH = tile_pixels(K) / 2;
+  const int S = p.bw * p.bh;                    // pixels of one group inside the tile
+  // position of this thread's j-th pixel; false when it lies outside the tensor
+  auto locate = [&](int j, int& g, int& oh, int& ow) -> bool {
+    const int pix = half * PH + j;
+    const int gl = pix >> p.log2_S, rem = pix & (S - 1);      // S and bw are powers of two
+    g = gt * p.bg + gl;
+    oh = ht * p.bh + (rem >> p.log2_bw);
+    ow = wt * p.bw + (rem & (p.bw - 1));
+    return g < p.G && oh < p.ho && ow < p.wo;                  // warp-uniform
+  };
+
+  // A tile that lies inside one group (every convolution whose image has at
+  // least P pixels) takes a branch-free walk over its pixels: the epilogue
+  // warps are few, so their speed depends on independent instructions from
+  // different pixels being in flight together.  Offsets fit 32 bits (n_out
+  // is checked on the host).
+  const bool one_group = p.bg == 1;
+  const int oh0 = ht * p.bh, ow0 = wt * p.bw;
+  auto pixel = [&](int j, int& off) -> bool {      // one_group only
+    const int pix = half * PH + j;
+    const int oh = oh0 + (pix >> p.log2_bw), ow = ow0 + (pix & (p.bw - 1));
+    off = (oh * p.wo + ow) * p.cout;
+    return oh < p.ho && ow < p.wo;
+  };
+
+  if (MODE == MODE_YBAR) {
+    if (one_group) {
+      float* base = p.out + ((size_t)gt * E) * p.n_out + co;
+#pragma unroll
+      for (int j = 0; j < PH; ++j) {
+        int off;
+        const bool ok = pixel(j, off) && co_ok;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          float* dst = base + (size_t)e * p.n_out + off;
+          if (ok) {
+            if (p.ksplit > 1) atomicAdd(dst, acc[e][j]);   // `out` was cleared
+            else *dst = acc[e][j];
+          }
+        }
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < PH; ++j) {
+        int g, oh, ow;
+        if (locate(j, g, oh, ow) && co_ok) {
+          float* dst = p.out + ((size_t)g * E) * p.n_out + ((size_t)oh * p.wo + ow) * p.cout + co;
+#pragma unroll
+          for (int e = 0; e < E; ++e) {
+            if (p.ksplit > 1) atomicAdd(dst + (size_t)e * p.n_out, acc[e][j]);   // `out` was cleared
+            else dst[(size_t)e * p.n_out] = acc[e][j];
+          }
+        }
+      }
+    }
+  } else {
+    if (p.f_group >= 0 && co == p.f_co) {      // fault hook: one element of one encoding
+      // (the per-encoding addend is formed first so that the accumulators
+      // are only ever indexed with compile-time constants)
+      float fd[E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) fd[e] = (e == p.f_enc) ? p.f_delta : 0.f;
+#pragma unroll
+      for (int j = 0; j < PH; ++j) {
+        int g, oh, ow;
+        const bool hit = locate(j, g, oh, ow) && g == p.f_group && oh == p.f_oh && ow == p.f_ow;
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e][j] += hit ? fd[e] : 0.f;
+      }
+    }
+    if (one_group) {
+      const int g = gt;
+      const float bias_co = (p.bias != nullptr && co_ok) ? __ldg(p.bias + co) : 0.f;
+#pragma unroll
+      for (int k = 0; k < K; ++k) {
+        float ch[K1], cl[K1];
+#pragma unroll
+        for (int i = 0; i < K1; ++i) {
+          ch[i] = __ldg(p.dec + ((size_t)g * K + k) * K1 + i);
+          cl[i] = __ldg(p.decl + ((size_t)g * K + k) * K1 + i);
+        }
+        float* base = p.out + ((size_t)g * K + k) * p.n_out + co;
+#pragma unroll
+        for (int j = 0; j < PH; ++j) {
+          int off;
+          const bool ok = pixel(j, off) && co_ok;
+          float hi = 0.f, lo = 0.f;
+#pragma unroll
+          for (int i = 0; i < K1; ++i) {
+            lo = fmaf(cl[i], acc[i][j], lo);
+            hi = fmaf(ch[i], acc[i][j], hi);
+          }
+          if (ok) base[off] = (hi + lo) + bias_co;
+        }
+      }
+      // integrity residual, statistics and candidates
+      float nv[E], sq[E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) { nv[e] = __ldg(p.nul + (size_t)g * E + e); sq[e] = 0.f; }
+      const float kInf = __int_as_float(0x7f800000);
+      float maxrho = 0.f;
+      uint32_t bad = 0;
+      auto residual = [&](int j, float& ar, float& sc) {
+        int off;
+        const bool ok = pixel(j, off) && co_ok;
+        float rho = 0.f;
+        sc = 0.f;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          const float v = ok ? acc[e][j] : 0.f;
+          rho = fmaf(nv[e], v, rho);
+          sc = fmaf(fabsf(nv[e]), fabsf(v), sc);
+        }
+        ar = fabsf(rho);
+      };
+#pragma unroll
+      for (int j = 0; j < PH; ++j) {
+        int off;
+        const bool ok = pixel(j, off) && co_ok;
+        float ar, sc;
+        residual(j, ar, sc);
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          const float v = ok ? acc[e][j] : 0.f;
+          sq[e] = fmaf(fabsf(v) < kInf ? v : 0.f, v, sq[e]);
+        }
+        maxrho = fmaxf(maxrho, ar);
+        bad |= (uint32_t)(!(ar <= p.tau * sc) || !(sc < kInf)) << j;
+      }
+      if (bad != 0u) {       // rare: append the candidates
+#pragma unroll
+        for (int j = 0; j < PH; ++j)
+          if ((bad >> j) & 1u) {
+            int off;
+            pixel(j, off);
+            float ar, sc;
+            residual(j, ar, sc);
+            unsigned int slot = atomicAdd(p.vs.count, 1u);
+            if (slot < kCandCap) {
+              Candidate cd;
+              cd.index = (long long)g * p.n_out + off + co;
+              cd.absrho = ar;
+              cd.s_e = sc;
+              p.vs.cand[slot] = cd;
+            }
+          }
+      }
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        float t = sq[e];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (lane == 0 && t != 0.f) atomicAdd(p.vs.sumsq + (size_t)g * E + e, t);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) maxrho = fmaxf(maxrho, __shfl_xor_sync(0xffffffffu, maxrho, o));
+      if (lane == 0 && maxrho > 0.f) atomicMax(p.vs.maxrho + g, __float_as_int(maxrho));
+    } else {
+      // The epilogue walks the pixels once per decoded row and once for the
+      // integrity residual, so that only one row of coefficients is live at a
+      // time; a row is re-read only when the group changes, and a tile of a
+      // convolution usually lies inside one group.
+      const float bias_co = (p.bias != nullptr && co_ok) ? __ldg(p.bias + co) : 0.f;
+#pragma unroll
+      for (int k = 0; k < K; ++k) {
+        int cg = -1;
+        float ch[K1], cl[K1];
+#pragma unroll
+        for (int j = 0; j < PH; ++j) {
+          int g, oh, ow;
+          if (!locate(j, g, oh, ow)) continue;
+          if (g != cg) {
+            const float* gh = p.dec + ((size_t)g * K + k) * K1;
+            const float* gl = p.decl + ((size_t)g * K + k) * K1;
+#pragma unroll
+            for (int i = 0; i < K1; ++i) { ch[i] = __ldg(gh + i); cl[i] = __ldg(gl + i); }
+            cg = g;
+          }
+          float hi = 0.f, lo = 0.f;
+#pragma unroll
+          for (int i = 0; i < K1; ++i) {
+            lo = fmaf(cl[i], acc[i][j], lo);
+            hi = fmaf(ch[i], acc[i][j], hi);
+          }
+          if (co_ok)
+            p.out[((size_t)g * K + k) * p.n_out + ((size_t)oh * p.wo + ow) * p.cout + co] = (hi + lo) + bias_co;
+        }
+      }
+      // integrity residual, statistics and candidates
+      float sq[E], nv[E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) sq[e] = 0.f;
+      float maxrho = 0.f;
+      int cur_g = -1, cg = -1;
+      auto flush_stats = [&](int g) {
+        if (g < 0) return;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          float s = sq[e];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+          if (lane == 0 && s != 0.f) atomicAdd(p.vs.sumsq + (size_t)g * E + e, s);
+          sq[e] = 0.f;
+        }
+        float m = maxrho;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0 && m > 0.f) atomicMax(p.vs.maxrho + g, __float_as_int(m));
+        maxrho = 0.f;
+      };
+      const float kInf = __int_as_float(0x7f800000);
+#pragma unroll
+      for (int j = 0; j < PH; ++j) {
+        int g, oh, ow;
+        const bool in_range = locate(j, g, oh, ow);
+        if (g != cur_g) {      // warp-uniform: g depends on the tile and the pixel only
+          flush_stats(cur_g);
+          cur_g = (g < p.G) ? g : -1;
+        }
+        if (!in_range) continue;
+        if (g != cg) {
+#pragma unroll
+          for (int e = 0; e < E; ++e) nv[e] = __ldg(p.nul + (size_t)g * E + e);
+          cg = g;
+        }
+        float rho = 0.f, sc = 0.f;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          const float v = co_ok ? acc[e][j] : 0.f;
+          rho = fmaf(nv[e], v, rho);
+          sc = fmaf(fabsf(nv[e]), fabsf(v), sc);
+          if (fabsf(v) < kInf) sq[e] = fmaf(v, v, sq[e]);
+        }
+        const float ar = fabsf(rho);
+        maxrho = fmaxf(maxrho, ar);
+        if (co_ok && (!(ar <= p.tau * sc) || !(sc < kInf))) {
+          unsigned int slot = atomicAdd(p.vs.count, 1u);
+          if (slot < kCandCap) {
+            Candidate cd;
+            cd.index = (long long)g * p.n_out + ((long long)oh * p.wo + ow) * p.cout + co;
+            cd.absrho = ar;
+            cd.s_e = sc;
+            p.vs.cand[slot] = cd;
+          }
+        }
+      }
+      flush_stats(cur_g);
+    }
+  }
+}
+// ---------------------------------------------------------------------------
 // the GEMM kernel
 // ---------------------------------------------------------------------------
 template <int BK, int MODE, int K>
@@ -324,7 +585,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
     // ---------------- epilogue: warps 4..11 ----------------
     const int quad = warp & 3;                    // TMEM lane quadrant this warp may read
     const int half = (warp - 4) >> 2;             // which half of the tile's pixels
-    const int S = p.bw * p.bh;                    // pixels of one group inside the tile
     uint32_t acc_it = 0;
     bool alive = true;
     float acc[E][PH];
@@ -370,255 +630,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
       }
       if (!alive) break;
 
-      // ---- store / decode from registers ----
-      // position of this thread's j-th pixel; false when it lies outside the tensor
-      auto locate = [&](int j, int& g, int& oh, int& ow) -> bool {
-        const int pix = half * PH + j;
-        const int gl = pix >> p.log2_S, rem = pix & (S - 1);      // S and bw are powers of two
-        g = gt * p.bg + gl;
-        oh = ht * p.bh + (rem >> p.log2_bw);
-        ow = wt * p.bw + (rem & (p.bw - 1));
-        return g < p.G && oh < p.ho && ow < p.wo;                  // warp-uniform
-      };
-
-      // A tile that lies inside one group (every convolution whose image has at
-      // least P pixels) takes a branch-free walk over its pixels: the epilogue
-      // warps are few, so their speed depends on independent instructions from
-      // different pixels being in flight together.  Offsets fit 32 bits (n_out
-      // is checked on the host).
-      const bool one_group = p.bg == 1;
-      const int oh0 = ht * p.bh, ow0 = wt * p.bw;
-      auto pixel = [&](int j, int& off) -> bool {      // one_group only
-        const int pix = half * PH + j;
-        const int oh = oh0 + (pix >> p.log2_bw), ow = ow0 + (pix & (p.bw - 1));
-        off = (oh * p.wo + ow) * p.cout;
-        return oh < p.ho && ow < p.wo;
-      };
-
-      if (MODE == MODE_YBAR) {
-        if (one_group) {
-          float* base = p.out + ((size_t)gt * E) * p.n_out + co;
-#pragma unroll
-          for (int j = 0; j < PH; ++j) {
-            int off;
-            const bool ok = pixel(j, off) && co_ok;
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-              float* dst = base + (size_t)e * p.n_out + off;
-              if (ok) {
-                if (p.ksplit > 1) atomicAdd(dst, acc[e][j]);   // `out` was cleared
-                else *dst = acc[e][j];
-              }
-            }
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < PH; ++j) {
-            int g, oh, ow;
-            if (locate(j, g, oh, ow) && co_ok) {
-              float* dst = p.out + ((size_t)g * E) * p.n_out + ((size_t)oh * p.wo + ow) * p.cout + co;
-#pragma unroll
-              for (int e = 0; e < E; ++e) {
-                if (p.ksplit > 1) atomicAdd(dst + (size_t)e * p.n_out, acc[e][j]);   // `out` was cleared
-                else dst[(size_t)e * p.n_out] = acc[e][j];
-              }
-            }
-          }
-        }
-      } else {
-        if (p.f_group >= 0 && co == p.f_co) {      // fault hook: one element of one encoding
-          // (the per-encoding addend is formed first so that the accumulators
-          // are only ever indexed with compile-time constants)
-          float fd[E];
-#pragma unroll
-          for (int e = 0; e < E; ++e) fd[e] = (e == p.f_enc) ? p.f_delta : 0.f;
-#pragma unroll
-          for (int j = 0; j < PH; ++j) {
-            int g, oh, ow;
-            const bool hit = locate(j, g, oh, ow) && g == p.f_group && oh == p.f_oh && ow == p.f_ow;
-#pragma unroll
-            for (int e = 0; e < E; ++e) acc[e][j] += hit ? fd[e] : 0.f;
-          }
-        }
-        if (one_group) {
-          const int g = gt;
-          const float bias_co = (p.bias != nullptr && co_ok) ? __ldg(p.bias + co) : 0.f;
-#pragma unroll
-          for (int k = 0; k < K; ++k) {
-            float ch[K1], cl[K1];
-#pragma unroll
-            for (int i = 0; i < K1; ++i) {
-              ch[i] = __ldg(p.dec + ((size_t)g * K + k) * K1 + i);
-              cl[i] = __ldg(p.decl + ((size_t)g * K + k) * K1 + i);
-            }
-            float* base = p.out + ((size_t)g * K + k) * p.n_out + co;
-#pragma unroll
-            for (int j = 0; j < PH; ++j) {
-              int off;
-              const bool ok = pixel(j, off) && co_ok;
-              float hi = 0.f, lo = 0.f;
-#pragma unroll
-              for (int i = 0; i < K1; ++i) {
-                lo = fmaf(cl[i], acc[i][j], lo);
-                hi = fmaf(ch[i], acc[i][j], hi);
-              }
-              if (ok) base[off] = (hi + lo) + bias_co;
-            }
-          }
-          // integrity residual, statistics and candidates
-          float nv[E], sq[E];
-#pragma unroll
-          for (int e = 0; e < E; ++e) { nv[e] = __ldg(p.nul + (size_t)g * E + e); sq[e] = 0.f; }
-          const float kInf = __int_as_float(0x7f800000);
-          float maxrho = 0.f;
-          uint32_t bad = 0;
-          auto residual = [&](int j, float& ar, float& sc) {
-            int off;
-            const bool ok = pixel(j, off) && co_ok;
-            float rho = 0.f;
-            sc = 0.f;
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-              const float v = ok ? acc[e][j] : 0.f;
-              rho = fmaf(nv[e], v, rho);
-              sc = fmaf(fabsf(nv[e]), fabsf(v), sc);
-            }
-            ar = fabsf(rho);
-          };
-#pragma unroll
-          for (int j = 0; j < PH; ++j) {
-            int off;
-            const bool ok = pixel(j, off) && co_ok;
-            float ar, sc;
-            residual(j, ar, sc);
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-              const float v = ok ? acc[e][j] : 0.f;
-              sq[e] = fmaf(fabsf(v) < kInf ? v : 0.f, v, sq[e]);
-            }
-            maxrho = fmaxf(maxrho, ar);
-            bad |= (uint32_t)(!(ar <= p.tau * sc) || !(sc < kInf)) << j;
-          }
-          if (bad != 0u) {       // rare: append the candidates
-#pragma unroll
-            for (int j = 0; j < PH; ++j)
-              if ((bad >> j) & 1u) {
-                int off;
-                pixel(j, off);
-                float ar, sc;
-                residual(j, ar, sc);
-                unsigned int slot = atomicAdd(p.vs.count, 1u);
-                if (slot < kCandCap) {
-                  Candidate cd;
-                  cd.index = (long long)g * p.n_out + off + co;
-                  cd.absrho = ar;
-                  cd.s_e = sc;
-                  p.vs.cand[slot] = cd;
-                }
-              }
-          }
-#pragma unroll
-          for (int e = 0; e < E; ++e) {
-            float t = sq[e];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-            if (lane == 0 && t != 0.f) atomicAdd(p.vs.sumsq + (size_t)g * E + e, t);
-          }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) maxrho = fmaxf(maxrho, __shfl_xor_sync(0xffffffffu, maxrho, o));
-          if (lane == 0 && maxrho > 0.f) atomicMax(p.vs.maxrho + g, __float_as_int(maxrho));
-        } else {
-          // The epilogue walks the pixels once per decoded row and once for the
-          // integrity residual, so that only one row of coefficients is live at a
-          // time; a row is re-read only when the group changes, and a tile of a
-          // convolution usually lies inside one group.
-          const float bias_co = (p.bias != nullptr && co_ok) ? __ldg(p.bias + co) : 0.f;
-#pragma unroll
-          for (int k = 0; k < K; ++k) {
-            int cg = -1;
-            float ch[K1], cl[K1];
-#pragma unroll
-            for (int j = 0; j < PH; ++j) {
-              int g, oh, ow;
-              if (!locate(j, g, oh, ow)) continue;
-              if (g != cg) {
-                const float* gh = p.dec + ((size_t)g * K + k) * K1;
-                const float* gl = p.decl + ((size_t)g * K + k) * K1;
-#pragma unroll
-                for (int i = 0; i < K1; ++i) { ch[i] = __ldg(gh + i); cl[i] = __ldg(gl + i); }
-                cg = g;
-              }
-              float hi = 0.f, lo = 0.f;
-#pragma unroll
-              for (int i = 0; i < K1; ++i) {
-                lo = fmaf(cl[i], acc[i][j], lo);
-                hi = fmaf(ch[i], acc[i][j], hi);
-              }
-              if (co_ok)
-                p.out[((size_t)g * K + k) * p.n_out + ((size_t)oh * p.wo + ow) * p.cout + co] = (hi + lo) + bias_co;
-            }
-          }
-          // integrity residual, statistics and candidates
-          float sq[E], nv[E];
-#pragma unroll
-          for (int e = 0; e < E; ++e) sq[e] = 0.f;
-          float maxrho = 0.f;
-          int cur_g = -1, cg = -1;
-          auto flush_stats = [&](int g) {
-            if (g < 0) return;
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-              float s = sq[e];
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-              if (lane == 0 && s != 0.f) atomicAdd(p.vs.sumsq + (size_t)g * E + e, s);
-              sq[e] = 0.f;
-            }
-            float m = maxrho;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-            if (lane == 0 && m > 0.f) atomicMax(p.vs.maxrho + g, __float_as_int(m));
-            maxrho = 0.f;
-          };
-          const float kInf = __int_as_float(0x7f800000);
-#pragma unroll
-          for (int j = 0; j < PH; ++j) {
-            int g, oh, ow;
-            const bool in_range = locate(j, g, oh, ow);
-            if (g != cur_g) {      // warp-uniform: g depends on the tile and the pixel only
-              flush_stats(cur_g);
-              cur_g = (g < p.G) ? g : -1;
-            }
-            if (!in_range) continue;
-            if (g != cg) {
-#pragma unroll
-              for (int e = 0; e < E; ++e) nv[e] = __ldg(p.nul + (size_t)g * E + e);
-              cg = g;
-            }
-            float rho = 0.f, sc = 0.f;
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-              const float v = co_ok ? acc[e][j] : 0.f;
-              rho = fmaf(nv[e], v, rho);
-              sc = fmaf(fabsf(nv[e]), fabsf(v), sc);
-              if (fabsf(v) < kInf) sq[e] = fmaf(v, v, sq[e]);
-            }
-            const float ar = fabsf(rho);
-            maxrho = fmaxf(maxrho, ar);
-            if (co_ok && (!(ar <= p.tau * sc) || !(sc < kInf))) {
-              unsigned int slot = atomicAdd(p.vs.count, 1u);
-              if (slot < kCandCap) {
-                Candidate cd;
-                cd.index = (long long)g * p.n_out + ((long long)oh * p.wo + ow) * p.cout + co;
-                cd.absrho = ar;
-                cd.s_e = sc;
-                p.vs.cand[slot] = cd;
-              }
-            }
-          }
-          flush_stats(cur_g);
-        }
-      }
+      tile_epilogue<MODE, K>(p, acc, half, lane, co, co_ok, gt, ht, wt);
     }
   }
 
