@@ -28,7 +28,7 @@ struct TcState {
 
 constexpr int kSwz128Atom32 = 1128;
 constexpr int kBK = 32;          // k-block: 32 fp32 = one 128-byte swizzle span per row
-constexpr int kChunk = 4;        // k-blocks accumulated in TMEM between promotions (error grows ~linearly with it)
+constexpr int kChunk = 8;        // 32-wide k-blocks accumulated in TMEM between promotions (error grows ~linearly with it)
 
 // Tuning knobs read once from the environment (defaults are the measured best):
 //   DK_TC_CHUNK  k-blocks per TMEM chunk in the forward kernel
