@@ -498,6 +498,7 @@ mix_split_kernel(const float* __restrict__ delta, const float* __restrict__ dmix
 struct WgPlan {
   WgTcParams prm;
   int BN;
+  bool pair;               // 256 output channels per work item on CTA pairs
   size_t smem_bytes;
 };
 
@@ -523,16 +524,32 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   p.PB = (int)pb;
   p.K1 = g.K + 1;
   w->BN = g.cin <= 64 ? 64 : (g.cin <= 128 ? 128 : 256);
-  p.MT = (g.cout + BM - 1) / BM;
+  static const int pair_on = env_knob("DK_WG_PAIR", 1, 0, 1);
+  w->pair = pair_on && g.cout > BM;
+  p.MT = w->pair ? (g.cout + BM2 - 1) / BM2 : (g.cout + BM - 1) / BM;
+  const int units = w->pair ? sm_count / 2 : sm_count;     // CTAs or CTA pairs that run together
   p.NB = (g.cin + w->BN - 1) / w->BN;
   p.taps = g.kh * g.kw;
   const long long base = (long long)p.MT * p.NB * p.taps;
-  long long nsplit = (2LL * sm_count + base - 1) / base;
-  // every slice ends in cout x cin atomics: keep at least 16 k-blocks of work behind them
-  const long long by_work = ((long long)p.PB * p.K1) / 16;
-  if (nsplit > by_work) nsplit = by_work;
-  if (nsplit > p.PB) nsplit = p.PB;
-  if (nsplit < 1) nsplit = 1;
+  // Slices of the pixel-block range per tile.  Work items are dealt round-robin to
+  // one CTA per SM, so the count that matters is how full the last round is:
+  // take the slice count (at most what keeps 16 k-blocks of work behind each
+  // slice's cout x cin atomics) with the best ratio items / (rounds * SMs),
+  // the smaller count on ties.
+  long long max_split = ((long long)p.PB * p.K1) / 16;
+  if (max_split > p.PB) max_split = p.PB;
+  if (max_split > 64) max_split = 64;
+  if (max_split < 1) max_split = 1;
+  long long nsplit = 1;
+  double best_eff = -1.0;
+  for (long long c = 1; c <= max_split; ++c) {
+    const long long per = (p.PB + c - 1) / c;
+    const long long eff_split = (p.PB + per - 1) / per;
+    const long long items_c = base * eff_split;
+    const long long rounds = (items_c + units - 1) / units;
+    const double eff = (double)items_c / (double)(rounds * units);
+    if (eff > best_eff + 0.02) { best_eff = eff; nsplit = c; }
+  }
   p.pb_per_split = (int)((p.PB + nsplit - 1) / nsplit);
   p.nsplit = (p.PB + p.pb_per_split - 1) / p.pb_per_split;
   const long long items = base * p.nsplit;
@@ -542,7 +559,7 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   static const int wg_chunk = env_knob("DK_WG_CHUNK", kWgChunk, 1, 64);
   p.chunk = wg_chunk;
   p.cout = g.cout; p.cin = g.cin;
-  const size_t stage = 2 * ((size_t)(BM / 32) * kWgBox + (size_t)(w->BN / 32) * kWgBox);
+  const size_t stage = 2 * ((size_t)(BM / 32) * kWgBox + (size_t)((w->pair ? w->BN / 2 : w->BN) / 32) * kWgBox);
   const size_t ctrl = 1024 + 256;
   int ns = (int)(((size_t)smem_optin - ctrl) / stage);
   if (ns > kMaxStages) ns = kMaxStages;
@@ -552,17 +569,40 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   return true;
 }
 
-template <int BN>
+template <int BN, bool PAIR>
 dk_status launch_wgrad(const WgPlan& w, const CUtensorMap& md_hi, const CUtensorMap& md_lo,
                        const CUtensorMap& mx_hi, const CUtensorMap& mx_lo, int sm_count, cudaStream_t st) {
-  auto kern = tc_wgrad_kernel<BN>;
+  auto kern = tc_wgrad_kernel<BN, PAIR>;
   cudaFuncAttributes fa;
   DK_CUDA_CHECK(cudaFuncGetAttributes(&fa, kern));
   if (fa.numRegs * kThreadsTc < 40 * 128 + 232 * 256) return DK_ERR_UNSUPPORTED;
   DK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)w.smem_bytes));
-  int grid = w.prm.nitems < sm_count ? w.prm.nitems : sm_count;
-  kern<<<grid, kThreadsTc, w.smem_bytes, st>>>(md_hi, md_lo, mx_hi, mx_lo, w.prm);
-  DK_CUDA_CHECK(cudaGetLastError());
+  if (!PAIR) {
+    int grid = w.prm.nitems < sm_count ? w.prm.nitems : sm_count;
+    kern<<<grid, kThreadsTc, w.smem_bytes, st>>>(md_hi, md_lo, mx_hi, mx_lo, w.prm);
+    DK_CUDA_CHECK(cudaGetLastError());
+    return DK_OK;
+  }
+  // clusters of two CTAs; as many pairs as can be resident together
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg = {};
+  int pairs = sm_count / 2;
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  cfg.blockDim = dim3(kThreadsTc);
+  cfg.dynamicSmemBytes = w.smem_bytes;
+  cfg.stream = st;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  int active = 0;
+  if (cudaOccupancyMaxActiveClusters(&active, kern, &cfg) == cudaSuccess && active > 0 && active < pairs)
+    pairs = active;
+  else
+    (void)cudaGetLastError();
+  if (w.prm.nitems < pairs) pairs = w.prm.nitems;
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  DK_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kern, md_hi, md_lo, mx_hi, mx_lo, w.prm));
   return DK_OK;
 }
 
@@ -628,9 +668,12 @@ dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* 
   }
   DK_CUDA_CHECK(cudaMemsetAsync(dW, 0, (size_t)g.cout * g.kc * sizeof(float), st));
   switch (w.BN) {
-    case 64: return launch_wgrad<64>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
-    case 128: return launch_wgrad<128>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
-    default: return launch_wgrad<256>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
+    case 64: return w.pair ? launch_wgrad<64, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st)
+                           : launch_wgrad<64, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
+    case 128: return w.pair ? launch_wgrad<128, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st)
+                            : launch_wgrad<128, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
+    default: return w.pair ? launch_wgrad<256, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st)
+                           : launch_wgrad<256, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
   }
 }
 

@@ -18,9 +18,14 @@
 // Parallelism.  Work item = (cout tile, tap, channel block, contraction
 // slice); persistent CTAs walk the items and add their slice into dW with
 // fp32 atomics (dW is cleared first).
+//
+// PAIR = true runs the same pipeline on clusters of two CTAs with
+// tcgen05 cta_group::2 (see dk_tc_pair.cuh): a pair owns 256 output channels,
+// each CTA stages its own 128 columns of dtil and half of the channel block
+// of xbar, the leader issues the MMAs for both.
 #pragma once
 
-#include "dk_tc_kernel.cuh"
+#include "dk_tc_pair.cuh"
 
 namespace dk {
 namespace tc {
@@ -59,15 +64,17 @@ __device__ __forceinline__ uint64_t make_desc_mn(uint32_t smem_addr, uint32_t bl
   return d;
 }
 
-template <int BN>
+template <int BN, bool PAIR>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_constant__ CUtensorMap map_d_lo,
                 const __grid_constant__ CUtensorMap map_x_hi, const __grid_constant__ CUtensorMap map_x_lo,
                 const WgTcParams p) {
   constexpr int NH = BN / 2;                     // accumulators per epilogue thread
   constexpr int A_BYTES = (BM / 32) * kWgBox;    // 16 KiB
-  constexpr int B_BYTES = (BN / 32) * kWgBox;
+  constexpr int BNL = PAIR ? BN / 2 : BN;        // channels of xbar this CTA stages
+  constexpr int B_BYTES = (BNL / 32) * kWgBox;
   constexpr int STAGE_BYTES = 2 * (A_BYTES + B_BYTES);
+  constexpr int MROWS = PAIR ? 2 * BM : BM;      // output channels of a work item
   static_assert(BN % 64 == 0 && BN <= 256, "illegal channel block");
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -81,22 +88,36 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const int first_item = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int item_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.nstages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + b, 1); mbar_init(tempty_bar + b, kEpiWarps); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull_bar + b, 1);
+      mbar_init(tempty_bar + b, PAIR ? 2 * kEpiWarps : kEpiWarps);     // a pair's chunks are released on the leader
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(512u)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (PAIR) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(512u)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(512u)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -121,13 +142,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
-      constexpr int NBOX = 2 * (BM / 32) + 2 * (BN / 32);
+      constexpr int NBOX = 2 * (BM / 32) + 2 * (BNL / 32);
       static_assert(NBOX <= 32, "one box per lane");
-      for (int item = blockIdx.x; alive && item < p.nitems; item += gridDim.x) {
+      for (int item = first_item; alive && item < p.nitems; item += item_step) {
         int mt, nb, tap, pb_lo, pb_hi;
         item_range(item, mt, nb, tap, pb_lo, pb_hi);
         const int u = tap / p.kw, v = tap - u * p.kw;
-        const int m0 = mt * BM, n0 = nb * BN;
+        const int m0 = mt * MROWS + (int)rank * BM, n0 = nb * BN + (int)rank * (PAIR ? BNL : 0);
         for (int pb = pb_lo; alive && pb < pb_hi; ++pb) {
           int r = pb;
           const int wt = r % p.WT; r /= p.WT;
@@ -138,42 +159,50 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
             int ok = 1;
             if (lane == 0) {
               ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag) ? 1 : 0;
-              if (ok) mbar_expect_tx(full_bar + stage, (uint32_t)STAGE_BYTES);
+              // the bytes of both CTAs of a pair are counted on the leader's barrier
+              if (ok && rank == 0) mbar_expect_tx(full_bar + stage, (uint32_t)((PAIR ? 2 : 1) * STAGE_BYTES));
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) { alive = false; break; }
             unsigned char* st = smem + (size_t)stage * STAGE_BYTES;
+            const uint32_t pbar = PAIR ? mapa_shared(smem_u32(full_bar + stage), 0u) : 0u;
+            auto load = [&](void* dst, const CUtensorMap* map, int c0, int c1, int c2) {
+              if constexpr (PAIR) tma_pair_load_5d(dst, map, pbar, c0, c1, c2, j, g0);
+              else tma_load_5d(dst, map, full_bar + stage, c0, c1, c2, j, g0);
+            };
             if (lane < 2 * (BM / 32)) {
               const int cb = lane >> 1;
-              if ((lane & 1) == 0)
-                tma_load_5d(st + cb * kWgBox, &map_d_hi, full_bar + stage, m0 + cb * 32, x0, y0, j, g0);
-              else
-                tma_load_5d(st + A_BYTES + cb * kWgBox, &map_d_lo, full_bar + stage, m0 + cb * 32, x0, y0, j, g0);
+              if ((lane & 1) == 0) load(st + cb * kWgBox, &map_d_hi, m0 + cb * 32, x0, y0);
+              else load(st + A_BYTES + cb * kWgBox, &map_d_lo, m0 + cb * 32, x0, y0);
             } else if (lane < NBOX) {
               const int q = lane - 2 * (BM / 32);
               const int cb = q >> 1;
               unsigned char* bh = st + 2 * A_BYTES;
-              if ((q & 1) == 0)
-                tma_load_5d(bh + cb * kWgBox, &map_x_hi, full_bar + stage, n0 + cb * 32, x0 + v - p.pad,
-                            y0 + u - p.pad, j, g0);
-              else
-                tma_load_5d(bh + B_BYTES + cb * kWgBox, &map_x_lo, full_bar + stage, n0 + cb * 32,
-                            x0 + v - p.pad, y0 + u - p.pad, j, g0);
+              if ((q & 1) == 0) load(bh + cb * kWgBox, &map_x_hi, n0 + cb * 32, x0 + v - p.pad, y0 + u - p.pad);
+              else load(bh + B_BYTES + cb * kWgBox, &map_x_lo, n0 + cb * 32, x0 + v - p.pad, y0 + u - p.pad);
             }
             __syncwarp();
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
           }
         }
       }
-    } else if (warp == 1 && lane == 0) {
-      // ---------------- MMA issuer ----------------
+    } else if (warp == 1 && lane == 0 && rank == 0) {
+      // ---------------- MMA issuer (of a pair: the leader only) ----------------
       constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | (1u << 16) |
-                                 ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                                 ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(MROWS >> 4) << 24);
+      auto mma = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t acc) {
+        if constexpr (PAIR) tc_pair_mma_tf32(d, a, b, idesc, acc);
+        else tc_mma_tf32(d, a, b, idesc, acc);
+      };
+      auto commit = [&](uint64_t* bar) {
+        if constexpr (PAIR) tc_pair_commit(bar);
+        else tc_commit(bar);
+      };
       int stage = 0;
       uint32_t phase = 0;
       uint32_t acc_it = 0;
       bool alive = true;
-      for (int item = blockIdx.x; alive && item < p.nitems; item += gridDim.x) {
+      for (int item = first_item; alive && item < p.nitems; item += item_step) {
         int mt, nb, tap, pb_lo, pb_hi;
         item_range(item, mt, nb, tap, pb_lo, pb_hi);
         const int KB = (pb_hi - pb_lo) * p.K1;
@@ -195,14 +224,14 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
 #pragma unroll
             for (int kk = 0; kk < kWgPix / 8; ++kk) {
               const uint64_t adv = (uint64_t)(kk * (1024 >> 4));   // 8 pixels = one 1024-byte row group
-              tc_mma_tf32(d_tmem, a_hi + adv, b_hi + adv, idesc, (first && kk == 0) ? 0u : 1u);
-              tc_mma_tf32(d_tmem, a_hi + adv, b_lo + adv, idesc, 1u);
-              tc_mma_tf32(d_tmem, a_lo + adv, b_hi + adv, idesc, 1u);
+              mma(d_tmem, a_hi + adv, b_hi + adv, (first && kk == 0) ? 0u : 1u);
+              mma(d_tmem, a_hi + adv, b_lo + adv, 1u);
+              mma(d_tmem, a_lo + adv, b_hi + adv, 1u);
             }
-            tc_commit(empty_bar + stage);
+            commit(empty_bar + stage);
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
           }
-          if (alive) tc_commit(tfull_bar + buf);
+          if (alive) commit(tfull_bar + buf);
         }
       }
     }
@@ -214,7 +243,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
     uint32_t acc_it = 0;
     bool alive = true;
     float acc[NH];
-    for (int item = blockIdx.x; alive && item < p.nitems; item += gridDim.x) {
+    for (int item = first_item; alive && item < p.nitems; item += item_step) {
       int mt, nb, tap, pb_lo, pb_hi;
       item_range(item, mt, nb, tap, pb_lo, pb_hi);
       const int KB = (pb_hi - pb_lo) * p.K1;
@@ -224,21 +253,25 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
         if (!mbar_wait(tfull_bar + buf, aphase, abort_flag)) { alive = false; break; }
         tc_fence_after();
         const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * NH);
+        constexpr int TS = NH > 96 ? 16 : 32;      // columns per round trip (fewer when the sums fill the registers)
 #pragma unroll
-        for (int c0 = 0; c0 < NH; c0 += 32) {
-          float tmp[32];
+        for (int c0 = 0; c0 < NH; c0 += TS) {
+          float tmp[TS];
 #pragma unroll
-          for (int c = 0; c < 32; c += 8) tc_ld8(tbase + (uint32_t)(c0 + c), &tmp[c]);
+          for (int c = 0; c < TS; c += 8) tc_ld8(tbase + (uint32_t)(c0 + c), &tmp[c]);
           tc_wait_ld();
 #pragma unroll
-          for (int c = 0; c < 32; ++c) acc[c0 + c] = (ci == 0) ? tmp[c] : acc[c0 + c] + tmp[c];
+          for (int c = 0; c < TS; ++c) acc[c0 + c] = (ci == 0) ? tmp[c] : acc[c0 + c] + tmp[c];
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar + buf);
+        if (lane == 0) {
+          if constexpr (PAIR) mbar_arrive_cluster(mapa_shared(smem_u32(tempty_bar + buf), 0u));
+          else mbar_arrive(tempty_bar + buf);
+        }
       }
       if (!alive) break;
-      const int co = mt * BM + quad * 32 + lane;
+      const int co = mt * MROWS + (int)rank * BM + quad * 32 + lane;
       if (co < p.cout && nchunks > 0) {
         float* dst = p.dW + ((size_t)co * p.taps + tap) * p.cin + nb * BN + half * NH;
         const int nvalid = p.cin - (nb * BN + half * NH);
@@ -262,9 +295,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
     for (int i = 0; i < 64; ++i) __nanosleep(16384);
     __syncthreads();
   }
+  if constexpr (PAIR) cluster_sync_all();     // neither CTA frees TMEM or exits while its peer may still use the pair's resources
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    if constexpr (PAIR)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 
