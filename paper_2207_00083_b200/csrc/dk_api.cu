@@ -442,14 +442,9 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
     VerifyScratch vs = verify_scratch(ctx, g);
     {
-      ProfScope ps(ctx, DK_KERNEL_OTHER, 2, st);
-      s = tc_split(W, w_hi, w_lo, (long long)g.cout * g.kc, ctx->sm_count, st);
-      if (s == DK_OK) s = launch_verify_begin(g, vs, st);
-    }
-    if (s != DK_OK) return s;
-    {
+      // one launch: encodings and weights as hi/lo pairs, integrity statistics cleared
       ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
-      s = tc_encode_split(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, ctx->sm_count, st);
+      s = tc_fwd_prepass(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, W, w_hi, w_lo, vs, ctx->sm_count, st);
     }
     if (s != DK_OK) return s;
     const int ksplit = tc_fwd_ksplit(ctx, g);
@@ -578,13 +573,10 @@ dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* del
     float* xb_hi = reinterpret_cast<float*>(ws + wp.xb_hi);
     float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
     {
+      // one launch: mixed deltas and stored encodings as hi/lo pairs, dW cleared
       ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
-      s = tc_mix_split(g, delta, cv.dmix, dtil, dt_lo, ctx->sm_count, st);
-    }
-    if (s != DK_OK) return s;
-    {
-      ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
-      s = tc_split(xbar, xb_hi, xb_lo, (long long)g.G * xbar_rows * g.n_in, ctx->sm_count, st);
+      s = tc_wgrad_prepass(g, delta, cv.dmix, dtil, dt_lo, xbar, (long long)g.G * xbar_rows * g.n_in, xb_hi, xb_lo,
+                           dW, ctx->sm_count, st);
     }
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);

@@ -155,10 +155,22 @@ bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g);
 // Eq. 4 delta mixing written as a TF32 hi/lo pair, [G*(K+1)][n_out] each
 dk_status tc_mix_split(const Geom& g, const float* delta, const float* dmix, float* hi, float* lo,
                        int sm_count, cudaStream_t st);
-// dW = scale * sum <dtil, xbar> from split operands (clears dW first)
+// dW = scale * sum <dtil, xbar> from split operands; adds into dW, which the
+// caller has cleared (tc_wgrad_prepass does)
 dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* dt_lo,
                    const float* xb_hi, const float* xb_lo, int xbar_rows, float scale, float* dW,
                    int* status_word, cudaStream_t st);
+// One launch for everything a masked forward call prepares (dk_tc_prepass.cu):
+// Eq. 1 encodings as hi/lo pairs (and in full when `full` is given), W as a
+// hi/lo pair, cleared integrity statistics.
+dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const float* enc, float* full,
+                         float* xb_hi, float* xb_lo, const float* W, float* w_hi, float* w_lo,
+                         const VerifyScratch& vs, int sm_count, cudaStream_t st);
+// One launch for what a weight-gradient call prepares: Eq. 4 delta mixing and
+// the stored encodings as hi/lo pairs, dW cleared.
+dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix, float* dt_hi, float* dt_lo,
+                           const float* xbar, long long xbar_elems, float* xb_hi, float* xb_lo, float* dW,
+                           int sm_count, cudaStream_t st);
 // same contraction with decode + integrity statistics in the epilogue
 dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
                         const float* xb_hi, const float* xb_lo, const CoefView& cv, const float* bias,

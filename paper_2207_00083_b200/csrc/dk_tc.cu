@@ -24,7 +24,62 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct TcState {
   EncodeTiledFn encode;
   int smem_optin;
+  int device;
 };
+
+// What the launch of one kernel instantiation needs to know about it, looked
+// up once per device instead of on every call (each query costs microseconds
+// of host time, which small layers cannot hide).
+constexpr int kMaxDevices = 64;
+struct KernelCache {
+  int regs[kMaxDevices];          // registers per thread, 0 = not queried yet
+  size_t smem[kMaxDevices];       // dynamic shared memory limit already set
+  int pairs[kMaxDevices];         // resident CTA pairs, 0 = not queried yet
+};
+
+// Checks the register pool the kernel's setmaxnreg split relies on and raises
+// the dynamic shared memory limit to `smem` when it is not there yet.
+template <typename Kern>
+dk_status prepare_kernel(Kern kern, KernelCache& kc, int dev, size_t smem) {
+  if (dev < 0 || dev >= kMaxDevices) return DK_ERR_UNSUPPORTED;
+  if (kc.regs[dev] == 0) {
+    cudaFuncAttributes fa;
+    DK_CUDA_CHECK(cudaFuncGetAttributes(&fa, kern));
+    kc.regs[dev] = fa.numRegs;
+  }
+  // The kernels re-partition registers between their warpgroups and would wait
+  // forever if the pool they were launched with were smaller than they assume.
+  if (kc.regs[dev] * kThreadsTc < 40 * 128 + 232 * 256) return DK_ERR_UNSUPPORTED;
+  if (kc.smem[dev] < smem) {
+    DK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kc.smem[dev] = smem;
+  }
+  return DK_OK;
+}
+
+// CTA pairs of `kern` that can be resident together (a GPC with an odd number
+// of SMs leaves one out), at most sm_count / 2.
+template <typename Kern>
+int resident_pairs(Kern kern, KernelCache& kc, int dev, size_t smem, int sm_count, bool cluster_attr) {
+  if (kc.pairs[dev] == 0) {
+    int pairs = sm_count / 2;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    cfg.blockDim = dim3(kThreadsTc);
+    cfg.dynamicSmemBytes = smem;
+    if (cluster_attr) { cfg.attrs = &attr; cfg.numAttrs = 1; }
+    int active = 0;
+    if (cudaOccupancyMaxActiveClusters(&active, kern, &cfg) == cudaSuccess && active > 0 && active < pairs)
+      pairs = active;
+    else
+      (void)cudaGetLastError();
+    kc.pairs[dev] = pairs;
+  }
+  return kc.pairs[dev];
+}
 
 constexpr int kSwz128Atom32 = 1128;
 constexpr int kBK = 32;          // k-block: 32 fp32 = one 128-byte swizzle span per row
@@ -207,12 +262,8 @@ dk_status launch_one(const TcState* ts, const Geom& g, const Tiling& tl, const f
   CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo;
   if (!encode_fwd_maps<BK>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, &ma_hi, &ma_lo, &mb_hi, &mb_lo)) return DK_ERR_CUDA;
   auto kern = tc_fwd_kernel<BK, MODE, K>;
-  // The kernel re-partitions registers between its warpgroups and would wait
-  // forever if the pool it was launched with were smaller than it assumes.
-  cudaFuncAttributes fa;
-  DK_CUDA_CHECK(cudaFuncGetAttributes(&fa, kern));
-  if (fa.numRegs * kThreadsTc < 40 * 128 + 232 * 256) return DK_ERR_UNSUPPORTED;
-  DK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tl.smem_bytes));
+  static KernelCache kc = {};
+  if (dk_status e = prepare_kernel(kern, kc, ts->device, tl.smem_bytes)) return e;
   const long long nwork = (long long)tl.ntiles * prm.ksplit;
   int grid = nwork < sm_count ? (int)nwork : sm_count;
   kern<<<grid, kThreadsTc, tl.smem_bytes, st>>>(ma_hi, ma_lo, mb_hi, mb_lo, prm);
@@ -230,24 +281,10 @@ dk_status launch_pair_one(const TcState* ts, const Geom& g, const Tiling& tl, co
     CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo;
     if (!encode_fwd_maps<32>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, &ma_hi, &ma_lo, &mb_hi, &mb_lo)) return DK_ERR_CUDA;
     auto kern = tc_fwd_pair_kernel<MODE, K>;
-    cudaFuncAttributes fa;
-    DK_CUDA_CHECK(cudaFuncGetAttributes(&fa, kern));
-    if (fa.numRegs * kThreadsTc < 40 * 128 + 232 * 256) return DK_ERR_UNSUPPORTED;
-    DK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tl.smem_bytes));
+    static KernelCache kc = {};
+    if (dk_status e = prepare_kernel(kern, kc, ts->device, tl.smem_bytes)) return e;
     const long long nwork = (long long)tl.ntiles * prm.ksplit;
-    int pairs = sm_count / 2;
-    {
-      // pairs that can be resident together (a GPC with an odd SM leaves one out)
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3((unsigned)(2 * pairs));
-      cfg.blockDim = dim3(kThreadsTc);
-      cfg.dynamicSmemBytes = tl.smem_bytes;
-      int active = 0;
-      if (cudaOccupancyMaxActiveClusters(&active, kern, &cfg) == cudaSuccess && active > 0 && active < pairs)
-        pairs = active;
-      else
-        (void)cudaGetLastError();
-    }
+    int pairs = resident_pairs(kern, kc, ts->device, tl.smem_bytes, sm_count, false);
     if (nwork < pairs) pairs = (int)nwork;
     kern<<<2 * pairs, kThreadsTc, tl.smem_bytes, st>>>(ma_hi, ma_lo, mb_hi, mb_lo, prm);
     DK_CUDA_CHECK(cudaGetLastError());
@@ -343,6 +380,7 @@ dk_status tc_init(dk_ctx* ctx) {
     return DK_ERR_CUDA;
   }
   ts->smem_optin = optin;
+  ts->device = ctx->device;
   ctx->tc_state = ts;
   return DK_OK;
 }
@@ -571,12 +609,10 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
 
 template <int BN, bool PAIR>
 dk_status launch_wgrad(const WgPlan& w, const CUtensorMap& md_hi, const CUtensorMap& md_lo,
-                       const CUtensorMap& mx_hi, const CUtensorMap& mx_lo, int sm_count, cudaStream_t st) {
+                       const CUtensorMap& mx_hi, const CUtensorMap& mx_lo, int dev, int sm_count, cudaStream_t st) {
   auto kern = tc_wgrad_kernel<BN, PAIR>;
-  cudaFuncAttributes fa;
-  DK_CUDA_CHECK(cudaFuncGetAttributes(&fa, kern));
-  if (fa.numRegs * kThreadsTc < 40 * 128 + 232 * 256) return DK_ERR_UNSUPPORTED;
-  DK_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)w.smem_bytes));
+  static KernelCache kc = {};
+  if (dk_status e = prepare_kernel(kern, kc, dev, w.smem_bytes)) return e;
   if (!PAIR) {
     int grid = w.prm.nitems < sm_count ? w.prm.nitems : sm_count;
     kern<<<grid, kThreadsTc, w.smem_bytes, st>>>(md_hi, md_lo, mx_hi, mx_lo, w.prm);
@@ -584,22 +620,16 @@ dk_status launch_wgrad(const WgPlan& w, const CUtensorMap& md_hi, const CUtensor
     return DK_OK;
   }
   // clusters of two CTAs; as many pairs as can be resident together
+  int pairs = resident_pairs(kern, kc, dev, w.smem_bytes, sm_count, true);
   cudaLaunchAttribute attr;
   attr.id = cudaLaunchAttributeClusterDimension;
   attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg = {};
-  int pairs = sm_count / 2;
-  cfg.gridDim = dim3((unsigned)(2 * pairs));
   cfg.blockDim = dim3(kThreadsTc);
   cfg.dynamicSmemBytes = w.smem_bytes;
   cfg.stream = st;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  int active = 0;
-  if (cudaOccupancyMaxActiveClusters(&active, kern, &cfg) == cudaSuccess && active > 0 && active < pairs)
-    pairs = active;
-  else
-    (void)cudaGetLastError();
   if (w.prm.nitems < pairs) pairs = w.prm.nitems;
   cfg.gridDim = dim3((unsigned)(2 * pairs));
   DK_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kern, md_hi, md_lo, mx_hi, mx_lo, w.prm));
@@ -666,14 +696,13 @@ dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* 
         !encode_map(ts, &mx_lo, xb_lo, 5, dims, str, box, kSwz128Atom32))
       return DK_ERR_CUDA;
   }
-  DK_CUDA_CHECK(cudaMemsetAsync(dW, 0, (size_t)g.cout * g.kc * sizeof(float), st));
   switch (w.BN) {
-    case 64: return w.pair ? launch_wgrad<64, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st)
-                           : launch_wgrad<64, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
-    case 128: return w.pair ? launch_wgrad<128, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st)
-                            : launch_wgrad<128, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
-    default: return w.pair ? launch_wgrad<256, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st)
-                           : launch_wgrad<256, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->sm_count, st);
+    case 64: return w.pair ? launch_wgrad<64, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st)
+                           : launch_wgrad<64, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st);
+    case 128: return w.pair ? launch_wgrad<128, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st)
+                            : launch_wgrad<128, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st);
+    default: return w.pair ? launch_wgrad<256, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st)
+                           : launch_wgrad<256, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st);
   }
 }
 
