@@ -39,6 +39,10 @@ import numpy as np  # noqa: E402
 METRIC = "decoded masked-linear TFLOP/s & fraction of roofline; encode/decode GB/s"
 L2_FLUSH_BYTES = 512 << 20
 TF32_OVER_BF16 = 1.1 / 2.25      # nominal dense TF32 : BF16 tensor throughput
+# DRAM bytes (read + write) per launch of the GEMM kernel classes, from one ncu capture of this command's
+# launches (profiles/dram_traffic_gemm_kernels_bench_vgg16_cifar.md); None = not captured since the kernels
+# last changed.
+NCU_TRAFFIC_BYTES = {"vgg16_cifar": {"linear_fwd": None, "wgrad": None}}
 
 
 def read_peaks():
@@ -449,8 +453,19 @@ def run_ours(args):
     avg_ms = prof[dom][0] / max(prof[dom][1], 1)
     tf32_peak = peaks["bf16_tflops"] * TF32_OVER_BF16
     achieved = issued_per_launch / (avg_ms * 1e-3) / 1e12
+    # bytes one launch of the dominant GEMM kernel must move (averaged over the layers): its two operands
+    # as TF32 hi/lo pairs once, its result once
+    if dom == "linear_fwd":
+        alg_bytes = sum(8 * (s.G * (s.K + 2) * s.n_in + s.cout * s.kc) + 4 * s.G * s.K * s.n_out
+                        for s in dom_specs) / len(dom_specs)
+    else:
+        alg_bytes = sum(8 * s.G * (s.K + 1) * (s.n_in + s.n_out) + 4 * s.cout * s.kc
+                        for s in dom_specs) / len(dom_specs)
+    traffic = NCU_TRAFFIC_BYTES.get(args.workload, {}).get(dom)
     roofline = {"bound": "tensor", "achieved": achieved, "peak": tf32_peak, "unit": "TFLOP/s",
-                "frac": achieved / tf32_peak, "traffic": None, "kernel": dom,
+                "frac": achieved / tf32_peak, "traffic": traffic, "traffic_unit": "bytes per launch (ncu, "
+                "dram read + write, average over the layers' launches)", "algorithmic_bytes": alg_bytes,
+                "kernel": dom,
                 "launches_timed": prof[dom][1], "avg_launch_ms": avg_ms,
                 "flops": "issued TF32 flops = 3 x masked flops (3xTF32 split), averaged over the layers",
                 "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x nominal "

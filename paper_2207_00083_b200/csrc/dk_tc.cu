@@ -561,14 +561,30 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   if (pb > 0x3fffffffLL) return false;
   p.PB = (int)pb;
   p.K1 = g.K + 1;
-  w->BN = g.cin <= 64 ? 64 : (g.cin <= 128 ? 128 : 256);
+  // N tile = tpn tap slots of cb channels.  Few input channels would make a
+  // narrow tile (N = 64 or 128 re-reads the 128 rows of dtil from shared memory
+  // once per 64 or 128 columns); putting several filter taps side by side keeps
+  // N at 192 or 256.
+  p.taps = g.kh * g.kw;
+  static const int pack_on = env_knob("DK_WG_PACK", 1, 0, 1);
+  if (g.cin <= 64) {
+    p.cb = 64;
+    p.tpn = !pack_on || p.taps == 1 ? 1 : (p.taps % 3 == 0 || p.taps < 4 ? (p.taps < 3 ? p.taps : 3) : 4);
+  } else if (g.cin <= 128) {
+    p.cb = 128;
+    p.tpn = !pack_on || p.taps == 1 ? 1 : 2;
+  } else {
+    p.cb = 256;
+    p.tpn = 1;
+  }
+  w->BN = p.cb * p.tpn;
+  p.TG = (p.taps + p.tpn - 1) / p.tpn;
   static const int pair_on = env_knob("DK_WG_PAIR", 1, 0, 1);
   w->pair = pair_on && g.cout > BM;
   p.MT = w->pair ? (g.cout + BM2 - 1) / BM2 : (g.cout + BM - 1) / BM;
   const int units = w->pair ? sm_count / 2 : sm_count;     // CTAs or CTA pairs that run together
-  p.NB = (g.cin + w->BN - 1) / w->BN;
-  p.taps = g.kh * g.kw;
-  const long long base = (long long)p.MT * p.NB * p.taps;
+  p.NB = (g.cin + p.cb - 1) / p.cb;
+  const long long base = (long long)p.MT * p.NB * p.TG;
   // Slices of the pixel-block range per tile.  Work items are dealt round-robin to
   // one CTA per SM, so the count that matters is how full the last round is:
   // take the slice count (at most what keeps 16 k-blocks of work behind each
@@ -699,6 +715,8 @@ dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* 
   switch (w.BN) {
     case 64: return w.pair ? launch_wgrad<64, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st)
                            : launch_wgrad<64, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st);
+    case 192: return w.pair ? launch_wgrad<192, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st)
+                            : launch_wgrad<192, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st);
     case 128: return w.pair ? launch_wgrad<128, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st)
                             : launch_wgrad<128, false>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st);
     default: return w.pair ? launch_wgrad<256, true>(w, md_hi, md_lo, mx_hi, mx_lo, ctx->device, ctx->sm_count, st)

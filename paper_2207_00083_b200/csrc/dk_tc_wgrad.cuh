@@ -39,6 +39,7 @@ struct WgTcParams {
   int PB;                      // WT*HT*GT
   int K1;                      // encodings used (K+1)
   int MT, NB, taps;            // cout tiles, channel blocks, filter taps
+  int cb, tpn, TG;             // channels per tap slot, tap slots per N tile (BN = cb*tpn), tap groups
   int nsplit, pb_per_split;    // contraction slices
   int nitems;                  // MT*NB*taps*nsplit
   int kw, pad;
@@ -121,13 +122,16 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // item -> (mt, nb, tap, slice); k-blocks of an item = pixel blocks of its slice x K1 encodings
-  auto item_range = [&](int item, int& mt, int& nb, int& tap, int& pb_lo, int& pb_hi) {
+  // item -> (mt, nb, tap group, slice); k-blocks of an item = pixel blocks of its slice x K1 encodings.
+  // The N tile of an item is tpn slots of cb channels: slot t holds channels
+  // [nb*cb, nb*cb + cb) of filter tap tg*tpn + t (layers with few input channels
+  // put several taps side by side so that the tile stays wide).
+  auto item_range = [&](int item, int& mt, int& nb, int& tg, int& pb_lo, int& pb_hi) {
     mt = item % p.MT;
     int r = item / p.MT;
     nb = r % p.NB; r /= p.NB;
-    tap = r % p.taps;
-    const int s = r / p.taps;
+    tg = r % p.TG;
+    const int s = r / p.TG;
     pb_lo = s * p.pb_per_split;
     pb_hi = min(p.PB, pb_lo + p.pb_per_split);
   };
@@ -145,10 +149,21 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
       constexpr int NBOX = 2 * (BM / 32) + 2 * (BNL / 32);
       static_assert(NBOX <= 32, "one box per lane");
       for (int item = first_item; alive && item < p.nitems; item += item_step) {
-        int mt, nb, tap, pb_lo, pb_hi;
-        item_range(item, mt, nb, tap, pb_lo, pb_hi);
-        const int u = tap / p.kw, v = tap - u * p.kw;
-        const int m0 = mt * MROWS + (int)rank * BM, n0 = nb * BN + (int)rank * (PAIR ? BNL : 0);
+        int mt, nb, tg, pb_lo, pb_hi;
+        item_range(item, mt, nb, tg, pb_lo, pb_hi);
+        const int m0 = mt * MROWS + (int)rank * BM;
+        // this lane's box of x_bar: 32 channels of one tap slot (a slot past the
+        // last tap reads from beyond the channel range, i.e. zeros)
+        int bx_c = 0, bx_u = 0, bx_v = 0;
+        if (lane >= 2 * (BM / 32) && lane < NBOX) {
+          const int gb = (int)rank * (PAIR ? BNL / 32 : 0) + ((lane - 2 * (BM / 32)) >> 1);
+          const int slot = (gb * 32) / p.cb;
+          const int tap = tg * p.tpn + slot;
+          bx_c = tap < p.taps ? nb * p.cb + (gb * 32 - slot * p.cb) : p.cin;
+          const int tt = tap < p.taps ? tap : 0;
+          bx_u = tt / p.kw;
+          bx_v = tt - bx_u * p.kw;
+        }
         for (int pb = pb_lo; alive && pb < pb_hi; ++pb) {
           int r = pb;
           const int wt = r % p.WT; r /= p.WT;
@@ -178,8 +193,8 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
               const int q = lane - 2 * (BM / 32);
               const int cb = q >> 1;
               unsigned char* bh = st + 2 * A_BYTES;
-              if ((q & 1) == 0) load(bh + cb * kWgBox, &map_x_hi, n0 + cb * 32, x0 + v - p.pad, y0 + u - p.pad);
-              else load(bh + B_BYTES + cb * kWgBox, &map_x_lo, n0 + cb * 32, x0 + v - p.pad, y0 + u - p.pad);
+              if ((q & 1) == 0) load(bh + cb * kWgBox, &map_x_hi, bx_c, x0 + bx_v - p.pad, y0 + bx_u - p.pad);
+              else load(bh + B_BYTES + cb * kWgBox, &map_x_lo, bx_c, x0 + bx_v - p.pad, y0 + bx_u - p.pad);
             }
             __syncwarp();
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
@@ -203,8 +218,8 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
       uint32_t acc_it = 0;
       bool alive = true;
       for (int item = first_item; alive && item < p.nitems; item += item_step) {
-        int mt, nb, tap, pb_lo, pb_hi;
-        item_range(item, mt, nb, tap, pb_lo, pb_hi);
+        int mt, nb, tg, pb_lo, pb_hi;
+        item_range(item, mt, nb, tg, pb_lo, pb_hi);
         const int KB = (pb_hi - pb_lo) * p.K1;
         const int nchunks = (KB + p.chunk - 1) / p.chunk;
         for (int ci = 0; alive && ci < nchunks; ++ci, ++acc_it) {
@@ -244,8 +259,8 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
     bool alive = true;
     float acc[NH];
     for (int item = first_item; alive && item < p.nitems; item += item_step) {
-      int mt, nb, tap, pb_lo, pb_hi;
-      item_range(item, mt, nb, tap, pb_lo, pb_hi);
+      int mt, nb, tg, pb_lo, pb_hi;
+      item_range(item, mt, nb, tg, pb_lo, pb_hi);
       const int KB = (pb_hi - pb_lo) * p.K1;
       const int nchunks = (KB + p.chunk - 1) / p.chunk;
       for (int ci = 0; ci < nchunks; ++ci, ++acc_it) {
@@ -273,16 +288,22 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
       if (!alive) break;
       const int co = mt * MROWS + (int)rank * BM + quad * 32 + lane;
       if (co < p.cout && nchunks > 0) {
-        float* dst = p.dW + ((size_t)co * p.taps + tap) * p.cin + nb * BN + half * NH;
-        const int nvalid = p.cin - (nb * BN + half * NH);
-        // 16-byte vector reductions: cin % 4 == 0 keeps every group of four
-        // either wholly inside or wholly outside the row, and dst 16-byte aligned
+        float* row = p.dW + (size_t)co * p.taps * p.cin;
+        // 16-byte vector reductions: cin % 4 == 0 and cb % 4 == 0 keep every group
+        // of four inside one tap slot, wholly inside or outside the channel range,
+        // and its address 16-byte aligned
 #pragma unroll
-        for (int c = 0; c < NH; c += 4)
-          if (c < nvalid)
-            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + c), "f"(p.scale * acc[c]),
-                         "f"(p.scale * acc[c + 1]), "f"(p.scale * acc[c + 2]), "f"(p.scale * acc[c + 3])
+        for (int c = 0; c < NH; c += 4) {
+          const int col = half * NH + c;
+          const int slot = col / p.cb;
+          const int tap = tg * p.tpn + slot;
+          const int ch = nb * p.cb + (col - slot * p.cb);
+          if (tap < p.taps && ch < p.cin)
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(row + (size_t)tap * p.cin + ch),
+                         "f"(p.scale * acc[c]), "f"(p.scale * acc[c + 1]), "f"(p.scale * acc[c + 2]),
+                         "f"(p.scale * acc[c + 3])
                          : "memory");
+        }
       }
     }
   }
