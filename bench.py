@@ -187,9 +187,9 @@ def shape_w(s):
 
 
 def uses_tensor_cores(s):
-    """Mirror of the library's dispatch rule (channels-last, stride 1, cin % 4 == 0,
+    """Mirror of the library's dispatch rule (channels-last, stride <= 4, cin % 4 == 0,
     default arithmetic)."""
-    return s.stride == 1 and s.cin % 4 == 0 and getattr(s, "precision", "default") == "default"
+    return s.stride <= 4 and s.cin % 4 == 0 and getattr(s, "precision", "default") == "default"
 
 
 def make_layer(torch, dk, synth, ctx, s, dev, gen, rank, pinned):

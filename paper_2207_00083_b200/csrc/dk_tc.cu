@@ -214,8 +214,11 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
 }
 
 bool encode_map(const TcState* ts, CUtensorMap* m, const void* base, int rank, const cuuint64_t* dims,
-                const cuuint64_t* strides_bytes, const cuuint32_t* box, int swz_bytes) {
-  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+                const cuuint64_t* strides_bytes, const cuuint32_t* box, int swz_bytes, int step_wh = 1) {
+  // step_wh > 1: every step_wh-th column and row (dimensions 1 and 2), the input
+  // positions a strided convolution reads; such a box spans box*step_wh positions
+  cuuint32_t estr[5] = {1, (cuuint32_t)step_wh, (cuuint32_t)step_wh, 1, 1};
+  if (rank < 3) estr[1] = estr[2] = 1;
   // swz_bytes: 32/64/128 = 16-byte chunks swizzled within that span (K-major
   // operands); kSwz128Atom32 = 32-byte chunks within 128 bytes, the only layout
   // the tensor core accepts for MN-major 32-bit operands
@@ -248,9 +251,10 @@ bool encode_fwd_maps(const TcState* ts, const Geom& g, const Tiling& tl, const f
     cuuint64_t dims[5] = {(cuuint64_t)g.cin, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.E, (cuuint64_t)g.G};
     cuuint64_t str[4] = {(cuuint64_t)g.cin * 4, (cuuint64_t)g.cin * g.w * 4, (cuuint64_t)g.n_in * 4,
                          (cuuint64_t)g.n_in * g.E * 4};
-    cuuint32_t box[5] = {(cuuint32_t)BK, (cuuint32_t)tl.bw, (cuuint32_t)tl.bh, 1, (cuuint32_t)tl.bg};
-    if (!encode_map(ts, mb_hi, xb_hi, 5, dims, str, box, BK * 4) ||
-        !encode_map(ts, mb_lo, xb_lo, 5, dims, str, box, BK * 4))
+    cuuint32_t box[5] = {(cuuint32_t)BK, (cuuint32_t)(tl.bw * g.stride), (cuuint32_t)(tl.bh * g.stride), 1,
+                         (cuuint32_t)tl.bg};
+    if (!encode_map(ts, mb_hi, xb_hi, 5, dims, str, box, BK * 4, g.stride) ||
+        !encode_map(ts, mb_lo, xb_lo, 5, dims, str, box, BK * 4, g.stride))
       return false;
   }
   return true;
@@ -318,7 +322,7 @@ void fill_params(const Geom& g, const Tiling& tl, TcParams* p) {
   p->chunk = chunk * (32 / fwd_bk());   // the knob counts 32-wide k-blocks
   p->ksplit = 1;
   p->kb_per_split = tl.KB;
-  p->kw = g.kw; p->pad = g.pad; p->nstages = tl.nstages;
+  p->kw = g.kw; p->pad = g.pad; p->stride = g.stride; p->nstages = tl.nstages;
   p->cout = g.cout; p->ho = g.ho; p->wo = g.wo; p->G = g.G;
   p->n_out = g.n_out;
   p->out = nullptr; p->dec = p->decl = p->nul = p->bias = nullptr;
@@ -392,7 +396,7 @@ void tc_destroy(dk_ctx* ctx) {
 
 bool tc_fwd_supported(const dk_ctx* ctx, const Geom& g) {
   if (g.precision != DK_TF32X3 || ctx->tc_state == nullptr) return false;
-  if (g.layout != DK_NHWC || g.stride != 1 || (g.cin % 4) != 0) return false;
+  if (g.layout != DK_NHWC || g.stride < 1 || g.stride > 4 || (g.cin % 4) != 0) return false;
   if (g.n_out >= (1LL << 31)) return false;     // the epilogue keeps pixel offsets in 32 bits
   Tiling tl;
   return plan_fwd(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, &tl);
@@ -609,7 +613,7 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   const long long items = base * p.nsplit;
   if (items > 0x7fffffffLL) return false;
   p.nitems = (int)items;
-  p.kw = g.kw; p.pad = g.pad;
+  p.kw = g.kw; p.pad = g.pad; p.stride = g.stride;
   static const int wg_chunk = env_knob("DK_WG_CHUNK", kWgChunk, 1, 64);
   p.chunk = wg_chunk;
   p.cout = g.cout; p.cin = g.cin;
@@ -656,7 +660,7 @@ dk_status launch_wgrad(const WgPlan& w, const CUtensorMap& md_hi, const CUtensor
 
 bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g) {
   if (g.precision != DK_TF32X3 || ctx->tc_state == nullptr) return false;
-  if (g.layout != DK_NHWC || g.stride != 1 || (g.cin % 4) != 0 || (g.cout % 4) != 0) return false;
+  if (g.layout != DK_NHWC || g.stride < 1 || g.stride > 4 || (g.cin % 4) != 0 || (g.cout % 4) != 0) return false;
   WgPlan w;
   return plan_wgrad(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, ctx->sm_count, &w);
 }
@@ -707,9 +711,10 @@ dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* 
                           (cuuint64_t)g.G};
     cuuint64_t str[4] = {(cuuint64_t)g.cin * 4, (cuuint64_t)g.cin * g.w * 4, (cuuint64_t)g.n_in * 4,
                          (cuuint64_t)g.n_in * xbar_rows * 4};
-    cuuint32_t box[5] = {32, (cuuint32_t)w.prm.bw, (cuuint32_t)w.prm.bh, 1, (cuuint32_t)w.prm.bg};
-    if (!encode_map(ts, &mx_hi, xb_hi, 5, dims, str, box, kSwz128Atom32) ||
-        !encode_map(ts, &mx_lo, xb_lo, 5, dims, str, box, kSwz128Atom32))
+    cuuint32_t box[5] = {32, (cuuint32_t)(w.prm.bw * g.stride), (cuuint32_t)(w.prm.bh * g.stride), 1,
+                         (cuuint32_t)w.prm.bg};
+    if (!encode_map(ts, &mx_hi, xb_hi, 5, dims, str, box, kSwz128Atom32, g.stride) ||
+        !encode_map(ts, &mx_lo, xb_lo, 5, dims, str, box, kSwz128Atom32, g.stride))
       return DK_ERR_CUDA;
   }
   switch (w.BN) {

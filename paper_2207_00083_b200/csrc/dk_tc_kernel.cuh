@@ -59,7 +59,7 @@ struct TcParams {
   int KB, CB;                  // k-blocks in total and per filter tap
   int chunk;                   // k-blocks accumulated in TMEM before promotion
   int ksplit, kb_per_split;    // contraction slices per tile (slices add into `out` with atomics)
-  int kw, pad;
+  int kw, pad, stride;
   int nstages;
   // problem
   int cout, ho, wo, G;
@@ -508,7 +508,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
         const int wt = nt % p.WT; nt /= p.WT;
         const int ht = nt % p.HT;
         const int gt = nt / p.HT;
-        const int x0 = wt * p.bw - p.pad, y0 = ht * p.bh - p.pad, g0 = gt * p.bg, m0 = mt * BM;
+        const int x0 = wt * p.bw * p.stride - p.pad, y0 = ht * p.bh * p.stride - p.pad;     // input position of tap (0,0)
+        const int g0 = gt * p.bg, m0 = mt * BM;
         for (int kb = kb_lo; kb < kb_hi; ++kb) {
           int ok = 1;
           if (lane == 0) {

@@ -148,7 +148,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
       const int wt = nt % p.WT; nt /= p.WT;
       const int ht = nt % p.HT;
       const int gt = nt / p.HT;
-      const int x0 = wt * p.bw - p.pad, y0 = ht * p.bh - p.pad, g0 = gt * p.bg;
+      const int x0 = wt * p.bw * p.stride - p.pad, y0 = ht * p.bh * p.stride - p.pad, g0 = gt * p.bg;
       const int m0 = mt * BM2 + (int)rank * BM;
       for (int kb = kb_lo; kb < kb_hi; ++kb) {
         int ok = 1;

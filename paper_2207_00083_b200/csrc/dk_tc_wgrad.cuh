@@ -42,7 +42,7 @@ struct WgTcParams {
   int cb, tpn, TG;             // channels per tap slot, tap slots per N tile (BN = cb*tpn), tap groups
   int nsplit, pb_per_split;    // contraction slices
   int nitems;                  // MT*NB*taps*nsplit
-  int kw, pad;
+  int kw, pad, stride;
   int nstages, chunk;
   int cout, cin;
   float scale;
@@ -193,8 +193,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
               const int q = lane - 2 * (BM / 32);
               const int cb = q >> 1;
               unsigned char* bh = st + 2 * A_BYTES;
-              if ((q & 1) == 0) load(bh + cb * kWgBox, &map_x_hi, bx_c, x0 + bx_v - p.pad, y0 + bx_u - p.pad);
-              else load(bh + B_BYTES + cb * kWgBox, &map_x_lo, bx_c, x0 + bx_v - p.pad, y0 + bx_u - p.pad);
+              const int xi = x0 * p.stride + bx_v - p.pad, yi = y0 * p.stride + bx_u - p.pad;   // input position
+              if ((q & 1) == 0) load(bh + cb * kWgBox, &map_x_hi, bx_c, xi, yi);
+              else load(bh + B_BYTES + cb * kWgBox, &map_x_lo, bx_c, xi, yi);
             }
             __syncwarp();
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
