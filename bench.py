@@ -406,22 +406,29 @@ def run_ours(args):
     wg_flops = sum(s.wgrad_flops() for s in specs if s.wgrad)
     step_flops = fwd_flops + wg_flops
 
-    # ---- device-resident timing, with per-kernel events inside the library
+    # ---- device-resident timing (the library only counts its launches here)
     for _ in range(warmup):
         flush.zero_()
         step_device()
     torch.cuda.synchronize()
     dk.dk_profile_reset(ctx)
-    dk.dk_profile_enable(ctx, True)
+    dk.dk_profile_enable(ctx, False)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     ms_total = timed(step_device, steps, 0)
     clocks = sampler.stop() if rank == 0 else None
+    launches = sum(v[2] for v in dk.dk_profile_read(ctx).values())
+    assert dk.dk_device_status(ctx) == 0
+
+    # ---- a second, untimed-for-the-metric pass with the library's per-kernel events on: kernel shares and
+    # the dominant kernel's average launch duration (the event pairs themselves cost a little, so the step
+    # metric above is taken without them)
+    dk.dk_profile_reset(ctx)
+    dk.dk_profile_enable(ctx, True)
+    timed(step_device, min(steps, 10), 0)
     prof = dk.dk_profile_read(ctx)
     dk.dk_profile_enable(ctx, False)
-    launches = sum(v[2] for v in prof.values())
-    assert dk.dk_device_status(ctx) == 0
 
     # ---- end to end through host buffers
     ms_e2e = timed(step_e2e, steps, 1)

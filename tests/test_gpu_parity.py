@@ -49,6 +49,18 @@ def small_cases():
         ("mbv2_project_960_320_G2", L("mobilenetv2_pw", "project_960_320").with_groups(2)),
         ("mbv2_expand_24_144_G1", dataclasses.replace(L("mobilenetv2_pw", "expand_24_144"), G=1, h=28, w=28)),
         ("vgg224_fc7_G2", L("vgg16_224", "fc7").with_groups(2)),
+        # CTA-pair kernels (cout > 128) at the other even K, ragged cout, a stride
+        ("pair_K2_cout200", tiny(cin=32, cout=200, h=12, w=10, K=2, G=3)),
+        ("pair_K6_cout256", tiny(cin=64, cout=256, h=8, w=8, K=6, G=2)),
+        ("pair_K8_cout384_s100", tiny(cin=32, cout=384, h=6, w=6, K=8, G=2)),
+        ("pair_s2_cout256", tiny(cin=64, cout=256, h=14, w=14, stride=2, K=4, G=2)),
+        # odd K keeps the single-CTA kernel even with many output channels
+        ("single_K3_cout160", tiny(cin=16, cout=160, h=7, w=9, K=3, G=2)),
+        # weight-gradient N tiles: 3 taps x 64 with a partly filled slot (cin 48),
+        # 2 taps x 128 (cin 96, odd tap count), 4 taps of a 2x2 filter
+        ("wg_pack_cin48", tiny(cin=48, cout=64, h=10, w=10, K=4, G=2)),
+        ("wg_pack_cin96", tiny(cin=96, cout=136, h=9, w=9, K=4, G=2)),
+        ("wg_pack_2x2", tiny(cin=16, cout=32, h=8, w=8, kh=2, kw=2, pad=0, K=2, G=2)),
     ]
 
 
