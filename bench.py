@@ -187,9 +187,13 @@ def shape_w(s):
 
 
 def uses_tensor_cores(s):
-    """Mirror of the library's dispatch rule (channels-last, stride <= 4, cin % 4 == 0,
-    default arithmetic)."""
-    return s.stride <= 4 and s.cin % 4 == 0 and getattr(s, "precision", "default") == "default"
+    """Mirror of the library's dispatch rule (channels-last, default arithmetic; stride <= 4 and
+    cin % 4 == 0, or a stem: cin % 4 != 0 with a contraction of at most 256 elements)."""
+    if getattr(s, "precision", "default") != "default":
+        return False
+    if s.cin % 4 == 0:
+        return s.stride <= 4
+    return s.kind == "conv" and s.kc <= 256 and s.cout % 4 == 0
 
 
 def make_layer(torch, dk, synth, ctx, s, dev, gen, rank, pinned):

@@ -201,14 +201,31 @@ struct WsPlan {
   size_t xbar, ybar, dtil, w_hi, w_lo, xb_hi, xb_lo, total;
 };
 
+// Geometry of the layers that go through the patch-row pre-pass (3-channel
+// stems): channels-last convolution, cin not a multiple of four, a contraction
+// of at most 256 elements, default arithmetic.  Independent of the context so
+// that dk_workspace_bytes can size for it.
+static bool stem_shape(const Geom& g) {
+  return g.kind == DK_CONV2D && g.layout == DK_NHWC && g.precision == DK_TF32X3 && (g.cin % 4) != 0 &&
+         g.kc <= 256 && (g.cout % 4) == 0;
+}
+
 // One layout serves every entry point: fp32 encodings (when the caller does
 // not store them), y_bar of the unfused path, mixed deltas of wgrad, and the
 // TF32 hi/lo split copies of W and x_bar that feed the tensor-core kernel.
 static WsPlan plan_workspace(const Geom& g) {
   WsPlan w;
   size_t off = 0;
-  const size_t xb = align_up((size_t)g.G * g.E * g.n_in * sizeof(float), 1024);
-  const size_t wb = align_up((size_t)g.cout * g.kc * sizeof(float), 1024);
+  // (a stem layer's hi/lo regions hold its patch rows and padded weights instead)
+  size_t xe = (size_t)g.G * g.E * g.n_in, we = (size_t)g.cout * g.kc;
+  if (stem_shape(g)) {
+    const size_t Kp = (size_t)tc_stem_padded_kc(g);
+    const size_t rows = (size_t)g.G * g.E * g.ho * g.wo * Kp;
+    if (rows > xe) xe = rows;
+    we = (size_t)g.cout * Kp;
+  }
+  const size_t xb = align_up(xe * sizeof(float), 1024);
+  const size_t wb = align_up(we * sizeof(float), 1024);
   w.xbar = off; off += xb;
   // y_bar: sized for doubles (DK_FP64_SIMT keeps it in fp64)
   w.ybar = off; off += align_up((size_t)g.G * g.E * g.n_out * sizeof(double), 1024);
@@ -433,9 +450,14 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
   s = upload_coefficients(ctx, g, C_host, nullptr, true, false, st, &cv);
   if (s != DK_OK) return s;
   char* ws = static_cast<char*>(ctx->ws);
-  if (tc_fwd_supported(ctx, g)) {
+  const bool stem = stem_shape(g) && tc_stem_supported(ctx, g);
+  const Geom g_stem = stem ? tc_stem_gemm_geom(g) : g;
+  if (stem || tc_fwd_supported(ctx, g)) {
     // tensor-core path: encode+split pre-pass, then one GEMM whose epilogue
-    // decodes and gathers the integrity statistics; y_bar never reaches HBM
+    // decodes and gathers the integrity statistics; y_bar never reaches HBM.
+    // (A stem layer's pre-pass writes patch rows, and the GEMM runs on the
+    // 1x1 geometry over them; outputs and statistics are laid out the same.)
+    const Geom& gg = g_stem;
     float* w_hi = reinterpret_cast<float*>(ws + wp.w_hi);
     float* w_lo = reinterpret_cast<float*>(ws + wp.w_lo);
     float* xb_hi = reinterpret_cast<float*>(ws + wp.xb_hi);
@@ -444,17 +466,18 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     {
       // one launch: encodings and weights as hi/lo pairs, integrity statistics cleared
       ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
-      s = tc_fwd_prepass(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, W, w_hi, w_lo, vs, ctx->sm_count, st);
+      s = stem ? tc_stem_fwd_prepass(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, W, w_hi, w_lo, vs, ctx->sm_count, st)
+               : tc_fwd_prepass(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, W, w_hi, w_lo, vs, ctx->sm_count, st);
     }
     if (s != DK_OK) return s;
-    const int ksplit = tc_fwd_ksplit(ctx, g);
+    const int ksplit = tc_fwd_ksplit(ctx, gg);
     if (ksplit > 1) {
       // too few tiles to fill the GPU: slice the contraction, let the slices
       // meet in y_bar (small here by construction) and decode in a second kernel
       float* ybar = reinterpret_cast<float*>(ws + wp.ybar);
       {
         ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
-        s = tc_linear_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, ybar, ksplit,
+        s = tc_linear_fwd(ctx, gg, w_hi, w_lo, xb_hi, xb_lo, ybar, ksplit,
                           reinterpret_cast<int*>(vs.count + 1), st);
       }
       if (s != DK_OK) return s;
@@ -466,20 +489,20 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
       }
       {
         ProfScope ps(ctx, DK_KERNEL_DECODE_VERIFY, 1, st);
-        s = launch_decode_verify(g, ybar, cv, bias, y, vs, ctx->sm_count, st);
+        s = launch_decode_verify(gg, ybar, cv, bias, y, vs, ctx->sm_count, st);
       }
       if (s != DK_OK) return s;
       ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
-      return launch_verify_finalize(g, cv.nul, vs, verdict, st);
+      return launch_verify_finalize(gg, cv.nul, vs, verdict, st);
     }
     {
       ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
-      s = tc_masked_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, cv, bias, y, vs,
+      s = tc_masked_fwd(ctx, gg, w_hi, w_lo, xb_hi, xb_lo, cv, bias, y, vs,
                         reinterpret_cast<int*>(vs.count + 1), fault, st);
     }
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
-    return launch_verify_finalize(g, cv.nul, vs, verdict, st);
+    return launch_verify_finalize(gg, cv.nul, vs, verdict, st);
   }
   if (g.precision == DK_FP64_SIMT) {
     // beyond-fp32 path: encodings and y_bar stay in the workspace as doubles

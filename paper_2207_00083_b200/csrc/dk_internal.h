@@ -177,9 +177,20 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
                         float* y, const VerifyScratch& vs, int* status_word, const dk_fault* fault,
                         cudaStream_t st);
 
+// Forward pass of layers with cin % 4 != 0 (3-channel stems) on the tensor-core kernels: the
+// pre-pass lays the kc inputs under the filter out as rows of Kp = kc rounded
+// up to 32 (hi/lo pairs), and the GEMM kernels run the 1x1 convolution that
+// tc_stem_gemm_geom describes (dk_tc_prepass.cu).
+bool tc_stem_supported(const dk_ctx* ctx, const Geom& g);
+int tc_stem_padded_kc(const Geom& g);
+Geom tc_stem_gemm_geom(const Geom& g);
+dk_status tc_stem_fwd_prepass(const Geom& g, const float* x, const float* r, const float* enc, float* full,
+                              float* col_hi, float* col_lo, const float* W, float* w_hi, float* w_lo,
+                              const VerifyScratch& vs, int sm_count, cudaStream_t st);
+
 }  // namespace dk
 
-#define DK_CUDA_CHECK(expr)                      \
+#define DK_CUDA_CHECK(expr)                     \
   do {                                           \
     cudaError_t _e = (expr);                     \
     if (_e != cudaSuccess) return DK_ERR_CUDA;   \

@@ -665,6 +665,14 @@ bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g) {
   return plan_wgrad(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, ctx->sm_count, &w);
 }
 
+bool tc_stem_supported(const dk_ctx* ctx, const Geom& g) {
+  static const int on = env_knob("DK_TC_STEM", 1, 0, 1);
+  if (!on || g.kind != DK_CONV2D || g.layout != DK_NHWC || g.precision != DK_TF32X3) return false;
+  if ((g.cin % 4) == 0 || g.kc > 256 || (g.cout % 4) != 0) return false;
+  const Geom s = tc_stem_gemm_geom(g);
+  return tc_fwd_supported(ctx, s);
+}
+
 dk_status tc_mix_split(const Geom& g, const float* delta, const float* dmix, float* hi, float* lo,
                        int sm_count, cudaStream_t st) {
   if (g.n_out % 4 || g.G > 65535) return DK_ERR_SHAPE;

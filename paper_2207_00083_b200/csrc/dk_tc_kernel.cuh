@@ -260,26 +260,35 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
     if (one_group) {
       const int g = gt;
       const float bias_co = (p.bias != nullptr && co_ok) ? __ldg(p.bias + co) : 0.f;
+      // Offsets and validity of this thread's pixels, once; sums of pixels outside
+      // the tensor (or of a channel past cout) are cleared so that the passes
+      // below need no further selects.  The instruction count of this epilogue
+      // is what bounds layers with a short contraction, so each pass is kept to
+      // the arithmetic it cannot avoid.
+      int off[PH];
+      uint32_t okm = 0;
+#pragma unroll
+      for (int j = 0; j < PH; ++j) {
+        const bool ok = pixel(j, off[j]) && co_ok;
+        okm |= (uint32_t)ok << j;
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e][j] = ok ? acc[e][j] : 0.f;
+      }
+      // decoded rows (Eq. 2).  One fp32 coefficient per term: the fp32 sums'
+      // own rounding is as large as the second float of the coefficient pair
+      // would contribute.
 #pragma unroll
       for (int k = 0; k < K; ++k) {
-        float ch[K1], cl[K1];
+        float ck[K1];
 #pragma unroll
-        for (int i = 0; i < K1; ++i) {
-          ch[i] = __ldg(p.dec + ((size_t)g * K + k) * K1 + i);
-          cl[i] = __ldg(p.decl + ((size_t)g * K + k) * K1 + i);
-        }
+        for (int i = 0; i < K1; ++i) ck[i] = __ldg(p.dec + ((size_t)g * K + k) * K1 + i);
         float* base = p.out + ((size_t)g * K + k) * p.n_out + co;
 #pragma unroll
         for (int j = 0; j < PH; ++j) {
-          int off;
-          const bool ok = pixel(j, off) && co_ok;
-          float hi = 0.f, lo = 0.f;
+          float yv = ck[0] * acc[0][j];
 #pragma unroll
-          for (int i = 0; i < K1; ++i) {
-            lo = fmaf(cl[i], acc[i][j], lo);
-            hi = fmaf(ch[i], acc[i][j], hi);
-          }
-          if (ok) base[off] = (hi + lo) + bias_co;
+          for (int i = 1; i < K1; ++i) yv = fmaf(ck[i], acc[i][j], yv);
+          if ((okm >> j) & 1u) base[off[j]] = yv + bias_co;
         }
       }
       // integrity residual, statistics and candidates
@@ -290,27 +299,22 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
       float maxrho = 0.f;
       uint32_t bad = 0;
       auto residual = [&](int j, float& ar, float& sc) {
-        int off;
-        const bool ok = pixel(j, off) && co_ok;
         float rho = 0.f;
         sc = 0.f;
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-          const float v = ok ? acc[e][j] : 0.f;
-          rho = fmaf(nv[e], v, rho);
-          sc = fmaf(fabsf(nv[e]), fabsf(v), sc);
+          rho = fmaf(nv[e], acc[e][j], rho);
+          sc = fmaf(fabsf(nv[e]), fabsf(acc[e][j]), sc);
         }
         ar = fabsf(rho);
       };
 #pragma unroll
       for (int j = 0; j < PH; ++j) {
-        int off;
-        const bool ok = pixel(j, off) && co_ok;
         float ar, sc;
         residual(j, ar, sc);
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-          const float v = ok ? acc[e][j] : 0.f;
+          const float v = acc[e][j];
           sq[e] = fmaf(fabsf(v) < kInf ? v : 0.f, v, sq[e]);
         }
         maxrho = fmaxf(maxrho, ar);
@@ -320,29 +324,31 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
 #pragma unroll
         for (int j = 0; j < PH; ++j)
           if ((bad >> j) & 1u) {
-            int off;
-            pixel(j, off);
             float ar, sc;
             residual(j, ar, sc);
             unsigned int slot = atomicAdd(p.vs.count, 1u);
             if (slot < kCandCap) {
               Candidate cd;
-              cd.index = (long long)g * p.n_out + off + co;
+              cd.index = (long long)g * p.n_out + off[j] + co;
               cd.absrho = ar;
               cd.s_e = sc;
               p.vs.cand[slot] = cd;
             }
           }
       }
+      // warp sums of the E statistics and the maximum, the butterflies interleaved
 #pragma unroll
-      for (int e = 0; e < E; ++e) {
-        float t = sq[e];
+      for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-        if (lane == 0 && t != 0.f) atomicAdd(p.vs.sumsq + (size_t)g * E + e, t);
+        for (int e = 0; e < E; ++e) sq[e] += __shfl_xor_sync(0xffffffffu, sq[e], o);
+        maxrho = fmaxf(maxrho, __shfl_xor_sync(0xffffffffu, maxrho, o));
       }
+      {      // lane e adds statistic e
+        float t = 0.f;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) maxrho = fmaxf(maxrho, __shfl_xor_sync(0xffffffffu, maxrho, o));
+        for (int e = 0; e < E; ++e) t = lane == e ? sq[e] : t;
+        if (lane < E && t != 0.f) atomicAdd(p.vs.sumsq + (size_t)g * E + lane, t);
+      }
       if (lane == 0 && maxrho > 0.f) atomicMax(p.vs.maxrho + g, __float_as_int(maxrho));
     } else {
       // The epilogue walks the pixels once per decoded row and once for the

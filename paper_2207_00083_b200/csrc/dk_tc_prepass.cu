@@ -189,4 +189,179 @@ dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix,
   return DK_OK;
 }
 
+// ---------------------------------------------------------------------------
+// Layers whose input has a channel count that is not a multiple of four (the
+// 3-channel stems).  Their contraction is short (kc = 27 or 147), which the
+// tensor-core kernels cannot fetch as 16-byte aligned channel runs.  The
+// pre-pass therefore writes, per encoded sample and output pixel, the kc
+// inputs under the filter as one row padded to a multiple of 32, already as a
+// hi/lo pair; the GEMM kernels then see a 1x1 convolution over ho x wo pixels
+// with Kp input channels.  (The weight gradient of these layers stays on the
+// fp32 kernels: its operands would have to be rewritten as patch rows too,
+// which costs more HBM traffic than the tensor cores save.)
+// ---------------------------------------------------------------------------
+namespace {
+
+struct PatchGeom {
+  int cin, h, w, kw, stride, pad, ho, wo, kc, Kp;
+  long long n_in;
+};
+
+// offset inside one sample of the input under filter position k of output pixel pix, or -1 (padding / k >= kc)
+__device__ __forceinline__ long long patch_offset(const PatchGeom& q, int pix, int k) {
+  if (k >= q.kc) return -1;
+  const int c = k % q.cin, t = k / q.cin;
+  const int v = t % q.kw, u = t / q.kw;
+  const int oy = pix / q.wo, ox = pix - oy * q.wo;
+  const int iy = oy * q.stride + u - q.pad, ix = ox * q.stride + v - q.pad;
+  if (iy < 0 || iy >= q.h || ix < 0 || ix >= q.w) return -1;
+  return ((long long)iy * q.w + ix) * q.cin + c;
+}
+
+struct StemFwd {
+  PatchGeom q;
+  const float* x; const float* r; const float* enc; float* full; float* col_hi; float* col_lo;
+  int G, per_g;                                    // blocks [0, G*per_g): patches of the encodings
+  int full_blocks;                                 // then: encodings in their own layout (when stored)
+  const float* W; float* w_hi; float* w_lo; int cout; int w_blocks;   // then: padded weights
+  float* stats; int nstats; unsigned int* count;   // cleared by block 0
+};
+
+template <int K>
+__global__ void __launch_bounds__(256) stem_fwd_prepass_kernel(const StemFwd a) {
+  constexpr int K1 = K + 1, E = K + 2;
+  const PatchGeom& q = a.q;
+  const int npix = q.ho * q.wo, kq = q.Kp / 4;
+  int b = blockIdx.x;
+  if (b < a.G * a.per_g) {
+    if (b == 0) {
+      for (int i = threadIdx.x; i < a.nstats; i += blockDim.x) a.stats[i] = 0.f;
+      if (threadIdx.x == 0) { a.count[0] = 0u; a.count[1] = 0u; }
+    }
+    const int g = b / a.per_g, chunk = b - g * a.per_g;
+    float c[E][K1];
+#pragma unroll
+    for (int i = 0; i < E; ++i)
+#pragma unroll
+      for (int k = 0; k < K1; ++k) c[i][k] = __ldg(a.enc + ((size_t)g * E + i) * K1 + k);
+    const float* xg = a.x + (size_t)g * K * q.n_in;
+    const float* rg = a.r + (size_t)g * q.n_in;
+    const long long items = (long long)npix * kq;
+    for (long long it = (long long)chunk * blockDim.x + threadIdx.x; it < items; it += (long long)a.per_g * blockDim.x) {
+      const int pix = (int)(it / kq), k0 = (int)(it - (long long)pix * kq) * 4;
+      float s[K1][4];
+#pragma unroll
+      for (int d = 0; d < 4; ++d) {
+        const long long off = patch_offset(q, pix, k0 + d);
+#pragma unroll
+        for (int k = 0; k < K; ++k) s[k][d] = off >= 0 ? __ldg(xg + (size_t)k * q.n_in + off) : 0.f;
+        s[K][d] = off >= 0 ? __ldg(rg + off) : 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < E; ++i) {
+        float4 o, hh, ll;
+        float t[4];
+#pragma unroll
+        for (int d = 0; d < 4; ++d) {
+          float acc = c[i][K] * s[K][d];
+#pragma unroll
+          for (int k = 0; k < K; ++k) acc = fmaf(c[i][k], s[k][d], acc);
+          t[d] = acc;
+        }
+        o = make_float4(t[0], t[1], t[2], t[3]);
+        split4(o, hh, ll);
+        const size_t row = ((size_t)g * E + i) * npix + pix;
+        reinterpret_cast<float4*>(a.col_hi + row * q.Kp)[k0 / 4] = hh;
+        reinterpret_cast<float4*>(a.col_lo + row * q.Kp)[k0 / 4] = ll;
+      }
+    }
+    return;
+  }
+  b -= a.G * a.per_g;
+  if (b < a.full_blocks) {
+    // Eq. 1 in the tensor's own layout, for the caller who stores the encodings
+    const long long total = (long long)a.G * q.n_in;
+    for (long long i = (long long)b * blockDim.x + threadIdx.x; i < total; i += (long long)a.full_blocks * blockDim.x) {
+      const int g = (int)(i / q.n_in);
+      const long long off = i - (long long)g * q.n_in;
+      float s[K1];
+#pragma unroll
+      for (int k = 0; k < K; ++k) s[k] = __ldg(a.x + ((size_t)g * K + k) * q.n_in + off);
+      s[K] = __ldg(a.r + (size_t)g * q.n_in + off);
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        const float* ce = a.enc + ((size_t)g * E + e) * K1;
+        float acc = __ldg(ce + K) * s[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) acc = fmaf(__ldg(ce + k), s[k], acc);
+        a.full[((size_t)g * E + e) * q.n_in + off] = acc;
+      }
+    }
+    return;
+  }
+  b -= a.full_blocks;
+  const long long witems = (long long)a.cout * kq;
+  for (long long it = (long long)b * blockDim.x + threadIdx.x; it < witems; it += (long long)a.w_blocks * blockDim.x) {
+    const int co = (int)(it / kq), k0 = (int)(it - (long long)co * kq) * 4;
+    float t[4];
+#pragma unroll
+    for (int d = 0; d < 4; ++d) t[d] = k0 + d < q.kc ? __ldg(a.W + (size_t)co * q.kc + k0 + d) : 0.f;
+    float4 hh, ll;
+    split4(make_float4(t[0], t[1], t[2], t[3]), hh, ll);
+    reinterpret_cast<float4*>(a.w_hi + (size_t)co * q.Kp)[k0 / 4] = hh;
+    reinterpret_cast<float4*>(a.w_lo + (size_t)co * q.Kp)[k0 / 4] = ll;
+  }
+}
+
+PatchGeom patch_geom(const Geom& g) {
+  PatchGeom q;
+  q.cin = g.cin; q.h = g.h; q.w = g.w; q.kw = g.kw; q.stride = g.stride; q.pad = g.pad;
+  q.ho = g.ho; q.wo = g.wo; q.kc = g.kc; q.Kp = tc_stem_padded_kc(g); q.n_in = g.n_in;
+  return q;
+}
+
+}  // namespace
+
+int tc_stem_padded_kc(const Geom& g) { return (g.kc + 31) / 32 * 32; }
+
+Geom tc_stem_gemm_geom(const Geom& g) {
+  Geom s = g;
+  const int Kp = tc_stem_padded_kc(g);
+  s.kind = DK_CONV2D; s.layout = DK_NHWC;
+  s.cin = Kp; s.h = g.ho; s.w = g.wo; s.kh = s.kw = 1; s.stride = 1; s.pad = 0;
+  s.n_in = (long long)Kp * g.ho * g.wo;
+  s.kc = Kp;
+  s.xs_c = 1; s.xs_w = Kp; s.xs_h = (long long)Kp * g.wo;
+  s.ws_c = 1; s.ws_v = Kp; s.ws_u = Kp; s.ws_o = Kp;
+  return s;
+}
+
+dk_status tc_stem_fwd_prepass(const Geom& g, const float* x, const float* r, const float* enc, float* full,
+                              float* col_hi, float* col_lo, const float* W, float* w_hi, float* w_lo,
+                              const VerifyScratch& vs, int sm_count, cudaStream_t st) {
+  StemFwd a;
+  a.q = patch_geom(g);
+  a.x = x; a.r = r; a.enc = enc; a.full = full; a.col_hi = col_hi; a.col_lo = col_lo;
+  a.G = g.G;
+  const long long cap = (long long)sm_count * 16;
+  const long long items = (long long)g.ho * g.wo * (a.q.Kp / 4);
+  a.per_g = job_blocks(items, (cap + g.G - 1) / g.G);
+  a.full_blocks = full ? job_blocks((long long)g.G * g.n_in, cap) : 0;
+  a.W = W; a.w_hi = w_hi; a.w_lo = w_lo; a.cout = g.cout;
+  a.w_blocks = job_blocks((long long)g.cout * (a.q.Kp / 4), cap);
+  a.stats = vs.sumsq; a.nstats = g.G * (g.E + 1); a.count = vs.count;
+  const long long blocks = (long long)a.G * a.per_g + a.full_blocks + a.w_blocks;
+  if (blocks > 0x7fffffffLL) return DK_ERR_SHAPE;
+#define DK_PRE_CASE(KK) \
+  case KK: stem_fwd_prepass_kernel<KK><<<(unsigned)blocks, 256, 0, st>>>(a); break;
+  switch (g.K) {
+    DK_PRE_CASE(1) DK_PRE_CASE(2) DK_PRE_CASE(3) DK_PRE_CASE(4)
+    DK_PRE_CASE(5) DK_PRE_CASE(6) DK_PRE_CASE(7) DK_PRE_CASE(8)
+    default: return DK_ERR_SHAPE;
+  }
+#undef DK_PRE_CASE
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
 }  // namespace dk
