@@ -328,6 +328,23 @@ def run_layer_table(args):
                       "rows": rows}), flush=True)
 
 
+def max_over_ranks(value, world, device):
+    """Device-timed milliseconds of this rank -> the slowest rank's figure (every rank gets it).
+    The replicas share nothing, so this and the barriers are the only communication of a multi-GPU run."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(flops_per_step, steps, world, ms_total):
+    """Aggregate throughput of `world` replicas that each ran `steps` steps of `flops_per_step` masked
+    flops within `ms_total` (the slowest rank's time), in TFLOP/s."""
+    return world * flops_per_step * steps / (ms_total * 1e-3) / 1e12
+
+
 # ---------------------------------------------------------------------------
 # our arm
 # ---------------------------------------------------------------------------
@@ -400,10 +417,7 @@ def run_ours(args):
             evs.append((a, b))
         barrier()
         total = sum(a.elapsed_time(b) for a, b in evs)
-        t = torch.tensor([total], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return max_over_ranks(total, world, dev)
 
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     fwd_flops = sum(s.fwd_flops() for s in specs)
@@ -446,8 +460,8 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    value = world * step_flops * steps / (ms_total * 1e-3) / 1e12
-    e2e_value = world * step_flops * steps / (ms_e2e * 1e-3) / 1e12
+    value = whole_job_value(step_flops, steps, world, ms_total)
+    e2e_value = whole_job_value(step_flops, steps, world, ms_e2e)
     K = specs[0].K
     ksum = max(sum(v[0] for v in prof.values()), 1e-9)
     kernel_ms = {k: round(v[0] / max(v[1], 1), 5) for k, v in prof.items() if v[1]}
