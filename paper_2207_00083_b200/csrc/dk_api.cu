@@ -498,11 +498,9 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     {
       ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
       s = tc_masked_fwd(ctx, gg, w_hi, w_lo, xb_hi, xb_lo, cv, bias, y, vs,
-                        reinterpret_cast<int*>(vs.count + 1), fault, st);
+                        reinterpret_cast<int*>(vs.count + 1), fault, verdict, st);
     }
-    if (s != DK_OK) return s;
-    ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
-    return launch_verify_finalize(gg, cv.nul, vs, verdict, st);
+    return s;      // the kernel's last CTA has written the verdict
   }
   if (g.precision == DK_FP64_SIMT) {
     // beyond-fp32 path: encodings and y_bar stay in the workspace as doubles

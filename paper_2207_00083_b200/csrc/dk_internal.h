@@ -171,11 +171,12 @@ dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const fl
 dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix, float* dt_hi, float* dt_lo,
                            const float* xbar, long long xbar_elems, float* xb_hi, float* xb_lo, float* dW,
                            int sm_count, cudaStream_t st);
-// same contraction with decode + integrity statistics in the epilogue
+// same contraction with decode + integrity statistics in the epilogue; when
+// `verdict` is given the kernel's last CTA also writes it (no finalize launch)
 dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
                         const float* xb_hi, const float* xb_lo, const CoefView& cv, const float* bias,
                         float* y, const VerifyScratch& vs, int* status_word, const dk_fault* fault,
-                        cudaStream_t st);
+                        dk_verdict* verdict, cudaStream_t st);
 
 // Forward pass of layers with cin % 4 != 0 (3-channel stems) on the tensor-core kernels: the
 // pre-pass lays the kc inputs under the filter out as rows of Kp = kc rounded

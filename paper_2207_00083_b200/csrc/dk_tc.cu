@@ -329,6 +329,7 @@ void fill_params(const Geom& g, const Tiling& tl, TcParams* p) {
   p->vs.sumsq = nullptr; p->vs.maxrho = nullptr; p->vs.count = nullptr; p->vs.cand = nullptr;
   p->tau = g.tol;
   p->status = nullptr;
+  p->verdict = nullptr; p->done = nullptr;
   p->f_group = -1; p->f_enc = p->f_co = p->f_oh = p->f_ow = 0;
   p->f_delta = 0.f;
 }
@@ -468,7 +469,8 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
 
 dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
                         const float* xb_lo, const CoefView& cv, const float* bias, float* y,
-                        const VerifyScratch& vs, int* status_word, const dk_fault* fault, cudaStream_t st) {
+                        const VerifyScratch& vs, int* status_word, const dk_fault* fault, dk_verdict* verdict,
+                        cudaStream_t st) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!plan_fwd(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
@@ -478,6 +480,8 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   prm.dec = cv.dec; prm.decl = cv.decl; prm.nul = cv.nul; prm.bias = bias;
   prm.vs = vs;
   prm.status = status_word;
+  prm.verdict = verdict;
+  prm.done = vs.count + 3;      // fourth word after the statistics: zero between calls
   if (fault) {
     prm.f_group = fault->group;
     prm.f_enc = fault->enc;

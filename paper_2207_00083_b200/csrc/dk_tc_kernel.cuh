@@ -32,6 +32,7 @@
 #include <cuda.h>
 
 #include "dk_internal.h"
+#include "dk_verify.cuh"
 
 namespace dk {
 namespace tc {
@@ -73,6 +74,11 @@ struct TcParams {
   VerifyScratch vs;
   float tau;
   int* status;                 // device word that receives DK_ERR_TIMEOUT
+  // MODE_DECODE: when `verdict` is given, the CTA that finishes last takes the
+  // final decisions of the check (`done` counts finished CTAs, starts at zero
+  // and is left at zero)
+  dk_verdict* verdict;
+  unsigned int* done;
   // fault injection (MODE_DECODE): group < 0 disables
   int f_group, f_enc, f_co, f_oh, f_ow;
   float f_delta;
@@ -444,6 +450,29 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
   }
 }
 // ---------------------------------------------------------------------------
+// After its last tile a CTA's 256 epilogue threads (tid 0..255) come here.  The
+// CTA that arrives last has every statistic of the integrity check in front of
+// it and writes the verdict, which saves the separate one-block launch.
+// `alive` = false: this warp's wait expired; the status is raised before the
+// count so that whoever decides sees it.
+// ---------------------------------------------------------------------------
+template <int MODE, int K>
+__device__ __forceinline__ void tail_finalize(const TcParams& p, int tid, bool alive, volatile int* last_flag) {
+  if (MODE != MODE_DECODE || p.verdict == nullptr) return;
+  if (!alive && p.status != nullptr) atomicExch(p.status, (int)DK_ERR_TIMEOUT);
+  __threadfence();
+  asm volatile("bar.sync 1, 256;" ::: "memory");
+  if (tid == 0) *last_flag = (atomicAdd(p.done, 1u) == gridDim.x - 1) ? 1 : 0;
+  asm volatile("bar.sync 1, 256;" ::: "memory");
+  if (*last_flag) {
+    __threadfence();
+    verify_finalize_block(tid, p.vs.sumsq, p.vs.maxrho, p.vs.count, p.vs.cand, p.nul, p.verdict, p.G, K + 2,
+                          p.n_out, p.tau);
+    if (tid == 0) *p.done = 0u;
+  }
+}
+
+// ---------------------------------------------------------------------------
 // the GEMM kernel
 // ---------------------------------------------------------------------------
 template <int BK, int MODE, int K>
@@ -639,6 +668,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
 
       tile_epilogue<MODE, K>(p, acc, half, lane, co, co_ok, gt, ht, wt);
     }
+    tail_finalize<MODE, K>(p, (int)threadIdx.x - 128, alive, abort_flag + 1);
   }
 
   // ---------------- teardown ----------------

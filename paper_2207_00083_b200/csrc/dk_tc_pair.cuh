@@ -268,6 +268,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
       if (!alive) break;
       tile_epilogue<MODE, K>(p, acc, half, lane, co, co_ok, gt, ht, wt);
     }
+    tail_finalize<MODE, K>(p, (int)threadIdx.x - 128, alive, abort_flag + 1);
   }
 
   // ---------------- teardown ----------------
