@@ -383,19 +383,46 @@ def run_ours(args):
                 dk.dk_linear_bwd_wgrad(ctx, L["p"], L["delta"], L["xsave"], s.K + 2, L["C"], L["gamma"],
                                        1.0 / s.batch, L["dW"])
 
+    h2d_stream, d2h_stream = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+
     def step_e2e():
+        """The same step through host buffers: every layer's inputs come from pinned host memory and its
+        results go back there.  Uploads, the library's calls and downloads run on three streams chained by
+        events, layer by layer, so that the copies of one layer overlap the kernels of its neighbours; the
+        step starts after everything before it and ends when the last download has landed."""
+        main = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(main)
+        h2d_stream.wait_event(start)
+        d2h_stream.wait_event(start)
         for L in layers:
             s = L["spec"]
-            L["x"].copy_(L["hx"], non_blocking=True)
-            L["r"].copy_(L["hr"], non_blocking=True)
+            with torch.cuda.stream(h2d_stream):
+                L["x"].copy_(L["hx"], non_blocking=True)
+                L["r"].copy_(L["hr"], non_blocking=True)
+                if s.wgrad:
+                    L["delta"].copy_(L["hdelta"], non_blocking=True)
+                up = torch.cuda.Event()
+                up.record(h2d_stream)
+            main.wait_event(up)
             dk.dk_masked_linear(ctx, L["p"], L["W"], L["x"], L["r"], L["C"], None, L["y"], L["xsave"], L["v"])
-            L["hy"].copy_(L["y"], non_blocking=True)
-            L["hv"].copy_(L["v"], non_blocking=True)
+            fwd_done = torch.cuda.Event()
+            fwd_done.record(main)
+            d2h_stream.wait_event(fwd_done)
+            with torch.cuda.stream(d2h_stream):
+                L["hy"].copy_(L["y"], non_blocking=True)
+                L["hv"].copy_(L["v"], non_blocking=True)
             if s.wgrad:
-                L["delta"].copy_(L["hdelta"], non_blocking=True)
                 dk.dk_linear_bwd_wgrad(ctx, L["p"], L["delta"], L["xsave"], s.K + 2, L["C"], L["gamma"],
                                        1.0 / s.batch, L["dW"])
-                L["hdW"].copy_(L["dW"], non_blocking=True)
+                wg_done = torch.cuda.Event()
+                wg_done.record(main)
+                d2h_stream.wait_event(wg_done)
+                with torch.cuda.stream(d2h_stream):
+                    L["hdW"].copy_(L["dW"], non_blocking=True)
+        down = torch.cuda.Event()
+        down.record(d2h_stream)
+        main.wait_event(down)
 
     def barrier():
         if world > 1:
