@@ -390,7 +390,8 @@ dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W, const 
     }
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
-    return tc_linear_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, ybar, tc_fwd_ksplit(ctx, g), ctx_status_word(ctx), st);
+    return tc_linear_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, ybar, tc_fwd_ksplit(ctx, g), false, ctx_status_word(ctx),
+                         st);
   }
   ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
   return launch_simt_fwd(g, W, xbar, ybar, g.G * g.E, st);
@@ -463,21 +464,23 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     float* xb_hi = reinterpret_cast<float*>(ws + wp.xb_hi);
     float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
     VerifyScratch vs = verify_scratch(ctx, g);
+    const int ksplit = tc_fwd_ksplit(ctx, gg);
+    float* ybar = reinterpret_cast<float*>(ws + wp.ybar);
+    const bool prepass_clears = ksplit > 1 && !stem;     // the pre-pass also clears y_bar for the slices
     {
       // one launch: encodings and weights as hi/lo pairs, integrity statistics cleared
       ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
       s = stem ? tc_stem_fwd_prepass(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, W, w_hi, w_lo, vs, ctx->sm_count, st)
-               : tc_fwd_prepass(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, W, w_hi, w_lo, vs, ctx->sm_count, st);
+               : tc_fwd_prepass(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, W, w_hi, w_lo, vs,
+                                prepass_clears ? ybar : nullptr, ctx->sm_count, st);
     }
     if (s != DK_OK) return s;
-    const int ksplit = tc_fwd_ksplit(ctx, gg);
     if (ksplit > 1) {
       // too few tiles to fill the GPU: slice the contraction, let the slices
       // meet in y_bar (small here by construction) and decode in a second kernel
-      float* ybar = reinterpret_cast<float*>(ws + wp.ybar);
       {
         ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
-        s = tc_linear_fwd(ctx, gg, w_hi, w_lo, xb_hi, xb_lo, ybar, ksplit,
+        s = tc_linear_fwd(ctx, gg, w_hi, w_lo, xb_hi, xb_lo, ybar, ksplit, prepass_clears,
                           reinterpret_cast<int*>(vs.count + 1), st);
       }
       if (s != DK_OK) return s;

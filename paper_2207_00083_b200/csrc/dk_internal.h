@@ -145,10 +145,10 @@ dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_c
 dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const float* enc, float* full,
                           float* hi, float* lo, int sm_count, cudaStream_t st);
 // y_bar = <W, x_bar> from split operands; ksplit > 1 slices the contraction
-// (y_bar is cleared and the slices add into it with atomics)
+// (the slices add into y_bar with atomics; it is cleared here unless the caller has done so)
 int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g);
 dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
-                        const float* xb_hi, const float* xb_lo, float* ybar, int ksplit,
+                        const float* xb_hi, const float* xb_lo, float* ybar, int ksplit, bool ybar_cleared,
                         int* status_word, cudaStream_t st);
 // weight gradient on tensor cores (channels-last, stride 1, cin % 4 == 0, cout % 4 == 0)
 bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g);
@@ -162,10 +162,11 @@ dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* 
                    int* status_word, cudaStream_t st);
 // One launch for everything a masked forward call prepares (dk_tc_prepass.cu):
 // Eq. 1 encodings as hi/lo pairs (and in full when `full` is given), W as a
-// hi/lo pair, cleared integrity statistics.
+// hi/lo pair, cleared integrity statistics, and (ybar_clear != nullptr) the
+// y_bar buffer of a split-K call cleared.
 dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const float* enc, float* full,
                          float* xb_hi, float* xb_lo, const float* W, float* w_hi, float* w_lo,
-                         const VerifyScratch& vs, int sm_count, cudaStream_t st);
+                         const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st);
 // One launch for what a weight-gradient call prepares: Eq. 4 delta mixing and
 // the stored encodings as hi/lo pairs, dW cleared.
 dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix, float* dt_hi, float* dt_lo,

@@ -436,22 +436,38 @@ dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const f
   return DK_OK;
 }
 
-// Contraction slices for problems with fewer tiles than SMs: each slice keeps
-// at least 8 k-blocks, and the slices of a tile add into y_bar with atomics.
+// Contraction slices for problems with fewer tiles than SMs.  Work items are
+// dealt round-robin to the resident CTAs (or pairs), so a slice count costs
+// rounds x (k-blocks per slice + a fixed per-item part: pipeline fill, epilogue
+// atomics), plus, for any count above one, the launches of the unfused path
+// (y_bar cleared, decode in a second kernel).  The cheapest count wins; slices
+// keep at least 8 k-blocks.  All figures in units of one k-block's time.
 int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!ts || !plan_fwd(g, ts->smem_optin, &tl)) return 1;
   const int units = tl.pair ? ctx->sm_count / 2 : ctx->sm_count;     // CTAs or CTA pairs that run together
-  if (tl.ntiles * 2 > units) return 1;
-  int want = (units + tl.ntiles - 1) / tl.ntiles;
-  int cap = tl.KB / (8 * (32 / fwd_bk()));
-  if (want > cap) want = cap;
-  return want < 1 ? 1 : want;
+  if (tl.ntiles >= units) return 1;
+  const int unit_kb = 32 / fwd_bk();             // k-blocks per 32 contraction elements
+  const int cap = tl.KB / (8 * unit_kb);
+  const long long kItem = 6 * unit_kb, kUnfused = 20 * unit_kb;
+  int best = 1;
+  long long best_cost = (long long)((tl.ntiles + units - 1) / units) * (tl.KB + kItem);
+  for (int c = 2; c <= cap; ++c) {
+    const int per = (tl.KB + c - 1) / c;
+    const int eff = (tl.KB + per - 1) / per;
+    if (eff != c) continue;                      // same slices as a smaller count
+    const long long items = (long long)tl.ntiles * eff;
+    const long long rounds = (items + units - 1) / units;
+    const long long cost = rounds * (per + kItem) + kUnfused;
+    if (cost < best_cost) { best_cost = cost; best = c; }
+  }
+  return best;
 }
 
 dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
-                        const float* xb_lo, float* ybar, int ksplit, int* status_word, cudaStream_t st) {
+                        const float* xb_lo, float* ybar, int ksplit, bool ybar_cleared, int* status_word,
+                        cudaStream_t st) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!plan_fwd(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
@@ -460,7 +476,8 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   if (ksplit > 1) {
     prm.kb_per_split = (tl.KB + ksplit - 1) / ksplit;
     prm.ksplit = (tl.KB + prm.kb_per_split - 1) / prm.kb_per_split;
-    DK_CUDA_CHECK(cudaMemsetAsync(ybar, 0, (size_t)g.G * g.E * g.n_out * sizeof(float), st));
+    if (!ybar_cleared)
+      DK_CUDA_CHECK(cudaMemsetAsync(ybar, 0, (size_t)g.G * g.E * g.n_out * sizeof(float), st));
   }
   prm.out = ybar;
   prm.status = status_word;

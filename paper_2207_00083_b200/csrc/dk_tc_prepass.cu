@@ -79,11 +79,19 @@ struct FwdPrepass {
   long long n_in; int G, per_g;                    // blocks [0, G*per_g): encode
   const float* W; float* w_hi; float* w_lo; long long w4; int w_blocks;   // then w_blocks blocks: split W
   float* stats; int nstats; unsigned int* count;   // cleared by block 0
+  float4* zero; long long z4; int z_blocks;        // then z_blocks blocks: clear y_bar (split-K calls)
 };
 
 template <int K>
 __global__ void __launch_bounds__(256) fwd_prepass_kernel(const FwdPrepass a) {
   const int enc_blocks = a.G * a.per_g;
+  if ((int)blockIdx.x >= enc_blocks + a.w_blocks) {
+    const int b = (int)blockIdx.x - enc_blocks - a.w_blocks;
+    const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (long long i = (long long)b * blockDim.x + threadIdx.x; i < a.z4; i += (long long)a.z_blocks * blockDim.x)
+      a.zero[i] = z;
+    return;
+  }
   if ((int)blockIdx.x < enc_blocks) {
     if (blockIdx.x == 0) {
       for (int i = threadIdx.x; i < a.nstats; i += blockDim.x) a.stats[i] = 0.f;
@@ -136,10 +144,14 @@ int job_blocks(long long n4, long long cap) {
 
 dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const float* enc, float* full,
                          float* xb_hi, float* xb_lo, const float* W, float* w_hi, float* w_lo,
-                         const VerifyScratch& vs, int sm_count, cudaStream_t st) {
+                         const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st) {
   const long long wn = (long long)g.cout * g.kc;
   if (g.n_in % 4 || wn % 4) return DK_ERR_SHAPE;
   FwdPrepass a;
+  const long long yn = (long long)g.G * g.E * g.n_out;
+  a.zero = reinterpret_cast<float4*>(ybar_clear);
+  a.z4 = ybar_clear ? (yn + 3) / 4 : 0;           // the y_bar region is padded to 1 KiB
+  a.z_blocks = ybar_clear ? job_blocks(a.z4, (long long)sm_count * 4) : 0;
   a.x = x; a.r = r; a.enc = enc; a.full = full; a.xb_hi = xb_hi; a.xb_lo = xb_lo;
   a.n_in = g.n_in; a.G = g.G;
   const long long cap = (long long)sm_count * 16;
@@ -147,7 +159,7 @@ dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const fl
   a.W = W; a.w_hi = w_hi; a.w_lo = w_lo; a.w4 = wn / 4;
   a.w_blocks = job_blocks(a.w4, cap);
   a.stats = vs.sumsq; a.nstats = g.G * (g.E + 1); a.count = vs.count;
-  const long long blocks = (long long)a.G * a.per_g + a.w_blocks;
+  const long long blocks = (long long)a.G * a.per_g + a.w_blocks + a.z_blocks;
   if (blocks > 0x7fffffffLL) return DK_ERR_SHAPE;
 #define DK_PRE_CASE(KK) \
   case KK: fwd_prepass_kernel<KK><<<(unsigned)blocks, 256, 0, st>>>(a); break;
