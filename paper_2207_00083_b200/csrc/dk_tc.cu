@@ -611,23 +611,22 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   p.NB = (g.cin + p.cb - 1) / p.cb;
   const long long base = (long long)p.MT * p.NB * p.TG;
   // Slices of the pixel-block range per tile.  Work items are dealt round-robin to
-  // one CTA per SM, so the count that matters is how full the last round is:
-  // take the slice count (at most what keeps 16 k-blocks of work behind each
-  // slice's cout x cin atomics) with the best ratio items / (rounds * SMs),
-  // the smaller count on ties.
-  long long max_split = ((long long)p.PB * p.K1) / 16;
-  if (max_split > p.PB) max_split = p.PB;
-  if (max_split > 64) max_split = 64;
+  // the resident CTAs (or pairs), so a slice count costs rounds x (k-blocks per
+  // slice + a fixed per-item part: pipeline fill and the cout x cin reductions
+  // into dW), in units of one k-block's time.  The cheapest count (at most 64
+  // slices) wins, the smaller one on ties.
+  long long max_split = p.PB < 64 ? p.PB : 64;
   if (max_split < 1) max_split = 1;
-  long long nsplit = 1;
-  double best_eff = -1.0;
+  const long long kItem = 10;
+  long long nsplit = 1, best_cost = -1;
   for (long long c = 1; c <= max_split; ++c) {
     const long long per = (p.PB + c - 1) / c;
     const long long eff_split = (p.PB + per - 1) / per;
+    if (eff_split != c) continue;               // same slices as a smaller count
     const long long items_c = base * eff_split;
     const long long rounds = (items_c + units - 1) / units;
-    const double eff = (double)items_c / (double)(rounds * units);
-    if (eff > best_eff + 0.02) { best_eff = eff; nsplit = c; }
+    const long long cost = rounds * (per * p.K1 + kItem);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; nsplit = c; }
   }
   p.pb_per_split = (int)((p.PB + nsplit - 1) / nsplit);
   p.nsplit = (p.PB + p.pb_per_split - 1) / p.pb_per_split;
