@@ -137,14 +137,14 @@ decode_verify_kernel(const float* __restrict__ ybar, const float* __restrict__ d
                      long long n, float tau, int cout, long long cdiv) {
   constexpr int K1 = K + 1, E = K + 2;
   const int g = blockIdx.y;
-  float dh[K][K1], dl[K][K1], nv[E];
+  // One fp32 coefficient per term: the fp32 sum's own rounding is as large as
+  // what the second float of the coefficient pair (decl) would contribute.
+  (void)decl;
+  float dh[K][K1], nv[E];
 #pragma unroll
   for (int k = 0; k < K; ++k)
 #pragma unroll
-    for (int i = 0; i < K1; ++i) {
-      dh[k][i] = __ldg(dec + ((size_t)g * K + k) * K1 + i);
-      dl[k][i] = __ldg(decl + ((size_t)g * K + k) * K1 + i);
-    }
+    for (int i = 0; i < K1; ++i) dh[k][i] = __ldg(dec + ((size_t)g * K + k) * K1 + i);
 #pragma unroll
   for (int i = 0; i < E; ++i) nv[i] = __ldg(nul + (size_t)g * E + i);
   const float* yb = ybar + (size_t)g * E * n;
@@ -172,13 +172,10 @@ decode_verify_kernel(const float* __restrict__ ybar, const float* __restrict__ d
       f4 o;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        float lo = 0.f, hi = 0.f;
+        float acc = dh[k][0] * in[0].v[q];
 #pragma unroll
-        for (int i = 0; i < K1; ++i) {
-          lo = fmaf(dl[k][i], in[i].v[q], lo);
-          hi = fmaf(dh[k][i], in[i].v[q], hi);
-        }
-        o.v[q] = (hi + lo) + b.v[q];
+        for (int i = 1; i < K1; ++i) acc = fmaf(dh[k][i], in[i].v[q], acc);
+        o.v[q] = acc + b.v[q];
       }
       store4<VEC>(yo + (size_t)k * n, e, n, o);
     }
