@@ -42,7 +42,7 @@ TF32_OVER_BF16 = 1.1 / 2.25      # nominal dense TF32 : BF16 tensor throughput
 # DRAM bytes (read + write) per launch of the GEMM kernel classes, from one ncu capture of this command's
 # launches (profiles/dram_traffic_gemm_kernels_bench_vgg16_cifar.md); None = not captured since the kernels
 # last changed.
-NCU_TRAFFIC_BYTES = {"vgg16_cifar": {"linear_fwd": 37150876, "wgrad": 47628064}}
+NCU_TRAFFIC_BYTES = {"vgg16_cifar": {"linear_fwd": 37150685, "wgrad": 47604374}}
 
 
 def read_peaks():
