@@ -28,6 +28,14 @@
  *    encoding i.  Rows 0..K are the square, invertible part used for
  *    decoding (the transpose of the paper's A in X_bar = X.A); row K+1 is
  *    the redundant encoding used only by the integrity check.
+ *  - Colluding accelerators (Section 4.5: M noise vectors, S = K_p + M
+ *    encodings of K_p private inputs, plus the redundant one).  No separate
+ *    entry point is needed: call with K = K_p + M - 1, store per group the
+ *    K_p private inputs followed by the first M - 1 noise vectors in x, the
+ *    M-th noise vector in r, and pass C[g] = [A^T; redundant row] with
+ *    A = [A1; A2].  Rows K_p..K-1 of each group's y then hold <W, r_m>
+ *    (to be dropped), and dk_linear_bwd_wgrad takes zero deltas for those rows.
+ *    K_p + M - 1 <= DK_MAX_K.
  *  - An integrity violation is a RESULT (dk_verdict.ok = 0), not an error:
  *    the call still returns DK_OK.
  *  - The library allocates only small per-context buffers in dk_create.

@@ -20,6 +20,9 @@ steps in order, without blocking or fusion:
 * ``wgrad_masked``      Eq. 4 and Eq. 6, summed over virtual batches
 * ``linear_plain`` / ``wgrad_plain``   the unmasked definitions (Eq. 3) that
                         the method must reproduce exactly in exact arithmetic
+* ``encode_colluding`` / ``decode_colluding`` / ``wgrad_colluding`` /
+  ``colluding_subsets_full_rank``   the M-noise-vector scheme of Section 4.5
+                        (X_bar = X.A1 + R.A2, S = K + M encodings)
 
 Coefficient convention: ``C[g, i, k]`` = coefficient of source k (k < K the
 private inputs, k = K the noise) in encoding i; rows 0..K are the decodable
@@ -371,3 +374,82 @@ def masked_forward(W, x, r, C, stride=1, pad=0, tau=1e-4, fault=None, bias=None)
     out = {"xbar": xbar, "ybar": ybar, "y": y, "z": z}
     out.update(chk)
     return out
+
+
+# ---------------------------------------------------------------------------
+# Colluding GPUs (Section 4.5): M noise vectors, S = K + M encodings
+# ---------------------------------------------------------------------------
+def encode_colluding(x: np.ndarray, R: np.ndarray, A1: np.ndarray, A2: np.ndarray) -> np.ndarray:
+    """X_bar = X . A1 + R . A2 for ONE virtual batch (first equation of Section 4.5).
+
+    x: [K, ...] private inputs, R: [M, ...] noise vectors, A1: [K, S], A2: [M, S]
+    with S = K + M.  Returns x_bar [S, ...]: encoding j is
+    sum_i A1[i, j] x[i] + sum_m A2[m, j] R[m].
+    """
+    x = np.asarray(x, dtype=np.float64)
+    R = np.asarray(R, dtype=np.float64)
+    K, M = x.shape[0], R.shape[0]
+    S = A1.shape[1]
+    assert A1.shape == (K, S) and A2.shape == (M, S) and S == K + M
+    out = np.zeros((S,) + x.shape[1:], dtype=np.float64)
+    for j in range(S):
+        for i in range(K):
+            out[j] += A1[i, j] * x[i]
+        for m in range(M):
+            out[j] += A2[m, j] * R[m]
+    return out
+
+
+def decode_colluding(ybar: np.ndarray, A1: np.ndarray, A2: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Y_bar = [Y | Z] . A with A = [A1; A2] square (S x S): recover Y = <W, X>
+    (K results) and Z = <W, R> (M results, dropped by the caller) from the S
+    encoded results of one virtual batch, element by element."""
+    ybar = np.asarray(ybar, dtype=np.float64)
+    A = np.concatenate([A1, A2], axis=0)
+    K = A1.shape[0]
+    Ainv = invert(A)
+    flat = ybar.reshape(ybar.shape[0], -1)            # [S, elements]
+    sol = np.zeros_like(flat)
+    for u in range(A.shape[0]):                       # unknown u = sum_j ybar[j] * Ainv[j, u]
+        for j in range(A.shape[0]):
+            sol[u] += Ainv[j, u] * flat[j]
+    sol = sol.reshape(ybar.shape)
+    return sol[:K], sol[K:]
+
+
+def colluding_subsets_full_rank(A2: np.ndarray, tol: float = 1e-9) -> bool:
+    """The condition Section 5 needs of A2 for M colluders: every choice of M of
+    its S columns is a full-rank M x M block, so that no linear combination of
+    the encodings a coalition holds is free of noise."""
+    import itertools
+    M, S = A2.shape
+    for cols in itertools.combinations(range(S), M):
+        sub = A2[:, cols]
+        if np.linalg.matrix_rank(sub, tol=tol) < M:
+            return False
+    return True
+
+
+def wgrad_colluding(delta: np.ndarray, xbar: np.ndarray, A1: np.ndarray, A2: np.ndarray,
+                    gamma: np.ndarray, scale: float, kh: int = 1, kw: int = 1, stride: int = 1,
+                    pad: int = 0) -> np.ndarray:
+    """grad W = scale * sum_{j<=S} gamma_j <sum_{i<=K} beta_{j,i} delta^(i), x_bar^(j)> for one
+    virtual batch, with B the solution of B^T . Gamma . A = [I_K | 0] (the K x S
+    condition of Section 4.5 with A = [A1; A2] as X_bar = [X | R] . A)."""
+    A = np.concatenate([A1, A2], axis=0)              # [S, S], rows = sources, columns = encodings
+    K, S = A1.shape[0], A.shape[0]
+    Ainv = invert(A)
+    # B^T Gamma A^T-of-the-sources: with X_bar^T = A^T [X|R]^T the condition reads
+    # sum_j B[j,i] gamma_j A[u,j] = [u == i]; hence B[j,i] = Ainv[j,i] / gamma_j
+    B = np.zeros((S, K))
+    for j in range(S):
+        for i in range(K):
+            B[j, i] = Ainv[j, i] / gamma[j]
+    total = None
+    for j in range(S):
+        mixed = np.zeros_like(np.asarray(delta[0], dtype=np.float64))
+        for i in range(K):
+            mixed = mixed + B[j, i] * np.asarray(delta[i], dtype=np.float64)
+        eq = bilinear_wgrad(mixed, xbar[j], kh, kw, stride, pad)
+        total = gamma[j] * eq if total is None else total + gamma[j] * eq
+    return scale * total

@@ -260,6 +260,43 @@ def draw_layer(spec: LayerSpec, with_delta: bool = True) -> Dict[str, np.ndarray
     return out
 
 
+def draw_colluding(spec: LayerSpec, K: int, M: int) -> Dict[str, np.ndarray]:
+    """Inputs of the M-noise-vector scheme for colluding accelerators (the paper's
+    X_bar = X.A1 + R.A2 with S = K + M encodings), laid out so that the library's
+    (K_lib + 2) x (K_lib + 1) interface with K_lib = K + M - 1 expresses it:
+
+    * ``x``  [G*K_lib, ...]: per group the K private inputs followed by the first
+      M - 1 noise vectors; ``r`` [G, ...]: the M-th noise vector; ``C`` as usual.
+    * ``delta`` [G*K_lib, ...]: output gradients of the K private inputs, zeros for
+      the rows that stand for noise.
+    * the same coefficients and data in the paper's notation: ``A1`` [G, K, S],
+      ``A2`` [G, M, S] (rows = sources, columns = encodings, i.e. the transpose of
+      the square part of C), ``x_private`` [G, K, ...], ``R`` [G, M, ...],
+      ``delta_private`` [G, K, ...].
+
+    Pure relabelling and drawing: nothing of the method is computed here.
+    """
+    assert spec.K == K + M - 1 and M >= 1
+    d = draw_layer(spec, with_delta=True)
+    G, KL, S = spec.G, spec.K, K + M
+    x = d["x"].reshape((G, KL) + d["x"].shape[1:]).copy()
+    if M > 1:
+        extra = (_rng(spec, "r", 1).standard_normal((G, M - 1) + x.shape[2:], dtype=np.float32)
+                 * np.float32(spec.sigma_r))
+        x[:, K:] = extra
+    delta = d["delta"].reshape((G, KL) + d["delta"].shape[1:]).copy()
+    delta[:, K:] = 0
+    A = np.transpose(d["C"][:, :S, :], (0, 2, 1)).astype(np.float64)     # A[g, source, encoding]
+    out = dict(d)
+    out["x"] = x.reshape(d["x"].shape)
+    out["delta"] = delta.reshape(d["delta"].shape)
+    out["A1"], out["A2"] = A[:, :K], A[:, K:]
+    out["x_private"] = x[:, :K].copy()
+    out["R"] = np.concatenate([x[:, K:], d["r"][:, None]], axis=1)
+    out["delta_private"] = delta[:, :K].copy()
+    return out
+
+
 def sample_coordinates(spec: LayerSpec, n: int, what: str = "y") -> np.ndarray:
     """Seeded sample of coordinates used for spot checks on large layers.
 
