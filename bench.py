@@ -40,8 +40,7 @@ METRIC = "decoded masked-linear TFLOP/s & fraction of roofline; encode/decode GB
 L2_FLUSH_BYTES = 512 << 20
 TF32_OVER_BF16 = 1.1 / 2.25      # nominal dense TF32 : BF16 tensor throughput
 # DRAM bytes (read + write) per launch of the GEMM kernel classes, from one ncu capture of this command's
-# launches (profiles/dram_traffic_gemm_kernels_bench_vgg16_cifar.md); None = not captured since the kernels
-# last changed.
+# launches (summary with the command under profiles/); None = not captured since the kernels last changed.
 NCU_TRAFFIC_BYTES = {"vgg16_cifar": {"linear_fwd": 37150685, "wgrad": 47604374}}
 
 
