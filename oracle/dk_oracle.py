@@ -20,6 +20,9 @@ steps in order, without blocking or fusion:
 * ``wgrad_masked``      Eq. 4 and Eq. 6, summed over virtual batches
 * ``linear_plain`` / ``wgrad_plain``   the unmasked definitions (Eq. 3) that
                         the method must reproduce exactly in exact arithmetic
+* ``wgrad_redundant``   the "two sets of equations" idea of Section 4.4 applied
+                        to the weight gradient: decode it from encodings
+                        1..K+1 and again from encodings 2..K+2, compare
 * ``encode_colluding`` / ``decode_colluding`` / ``wgrad_colluding`` /
   ``colluding_subsets_full_rank``   the M-noise-vector scheme of Section 4.5
                         (X_bar = X.A1 + R.A2, S = K + M encodings)
@@ -34,9 +37,10 @@ library float64 convolution and its autograd, the decode/encode round trip
 against the plain definition, closed forms for K = 1, the exact residual
 change n[i]*Delta under a single injected fault, and the Eq. 5 residual.
 Parity unpinned: the numerical threshold ``tau`` of ``verify`` and its
-noise-scale normaliser max(s_e, s_g) are choices of this implementation, not
-the paper's (the paper compares exactly in a finite field); nothing outside
-this file fixes them.
+noise-scale normaliser max(s_e, s_g), and the threshold and rms normaliser of
+``wgrad_redundant`` (a check the paper does not describe for the backward
+pass), are choices of this implementation, not the paper's (the paper
+compares exactly in a finite field); nothing outside this file fixes them.
 """
 from __future__ import annotations
 
@@ -374,6 +378,49 @@ def masked_forward(W, x, r, C, stride=1, pad=0, tau=1e-4, fault=None, bias=None)
     out = {"xbar": xbar, "ybar": ybar, "y": y, "z": z}
     out.update(chk)
     return out
+
+
+# ---------------------------------------------------------------------------
+# Section 4.4 applied to the weight gradient: two sets of equations
+# ---------------------------------------------------------------------------
+def second_equation_set(C: np.ndarray, gamma: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Coefficients of the equation set that uses encodings 2..K+2 instead of
+    1..K+1: per group the rows of C moved up by one (the first encoding becomes
+    the unused last row), and the same for the K+1 gammas (rotated)."""
+    C2 = np.concatenate([C[:, 1:], C[:, :1]], axis=1)
+    g2 = np.concatenate([gamma[:, 1:], gamma[:, :1]], axis=1)
+    return C2, g2
+
+
+def wgrad_redundant(delta: np.ndarray, xbar: np.ndarray, C: np.ndarray, gamma: np.ndarray,
+                    scale: float, kh: int = 1, kw: int = 1, stride: int = 1, pad: int = 0,
+                    tau_w: float = 1e-2, fault=None) -> Dict[str, np.ndarray]:
+    """grad W decoded twice, from two different sets of K+1 of the K+2 stored
+    encodings (Eq. 4-6 with the B of each set), and compared: consistent results
+    mean that no term <delta_bar, x_bar^(j)> came back wrong (Section 4.4's
+    "computing it redundantly at least twice using at least two sets of
+    equations", which the paper states for the forward results only).
+
+    ``xbar`` holds all K+2 encodings per group.  ``fault`` = (which, index
+    tuple, value) adds ``value`` to one element of result ``which`` (0 or 1)
+    before the comparison.  An element is flagged iff
+    not(|dW_0 - dW_1| <= tau_w * rms(dW_0)).
+    """
+    G, E, K1 = C.shape
+    xbar = np.asarray(xbar, dtype=F64)
+    first = wgrad_masked(delta, xbar, C, gamma, scale, kh, kw, stride, pad, xbar_rows_per_group=E)
+    # the second set: per group encodings 1..K+1, then (unused) encoding 0
+    order = np.array([g * E + (i + 1) % E for g in range(G) for i in range(E)])
+    C2, g2 = second_equation_set(C, gamma)
+    second = wgrad_masked(delta, xbar[order], C2, g2, scale, kh, kw, stride, pad, xbar_rows_per_group=E)
+    if fault is not None:
+        which, idx, val = fault
+        (first if which == 0 else second)[tuple(idx)] += val
+    rms = float(np.sqrt(np.mean(first ** 2)))
+    diff = np.abs(first - second)
+    ratio = diff / rms if rms > 0 else np.where(diff > 0, np.inf, 0.0)
+    flags = ~(diff <= tau_w * rms)
+    return {"dW": first, "dW_second": second, "ratio": ratio, "flags": flags, "rms": rms}
 
 
 # ---------------------------------------------------------------------------
