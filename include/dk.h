@@ -188,6 +188,32 @@ DK_API dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const flo
                                      const float* gamma_host, float scale, float* dW,
                                      void* stream);
 
+/* The weight gradient with an integrity check.  Section 4.4 verifies a result
+ * "by computing it redundantly at least twice using at least two sets of
+ * equations" and states this for the forward outputs; this call applies the
+ * same idea to Eq. 4-6: dW is decoded from encodings 0..K of every group (as
+ * dk_linear_bwd_wgrad does) and a second time, into workspace scratch, from
+ * encodings 1..K+1 with the B of that set (square part = rows 1..K+1 of C,
+ * gammas rotated by one); any K+1 rows of C are independent because no
+ * component of its null vector vanishes.  The two agree up to rounding unless a
+ * term <delta_bar, x_bar^(j)> came back wrong.  Element e is flagged iff
+ *   not (|dW[e] - dW_second[e]| <= tol_w * rms(dW)),
+ * and *verdict (device) receives ok, the number of flagged elements, the
+ * smallest flagged index into dW as stored, max |difference| / rms(dW), and
+ * the device status.  tol_w > 0; honest fp32-class differences are ~1e-3 of
+ * rms(dW), 1e-2 is a reasonable setting (the threshold and the normaliser are
+ * this library's choice, the paper gives none).  xbar: all K+2 encodings per
+ * group, [G*(K+2)][n_in], n_in a multiple of 4 (else DK_ERR_UNSUPPORTED).
+ * fault (host pointer, nullable) adds fault->delta to element fault->out_index
+ * of result fault->enc (0: dW, 1: the second one) before the comparison;
+ * fault->group is ignored.  Costs two weight-gradient products.  Needs the
+ * workspace. */
+DK_API dk_status dk_linear_bwd_wgrad_verify(dk_ctx* ctx, const dk_problem* p, const float* delta,
+                                            const float* xbar, const float* C_host,
+                                            const float* gamma_host, float scale, float tol_w,
+                                            float* dW, dk_verdict* verdict, const dk_fault* fault,
+                                            void* stream);
+
 /* Errors raised ON THE DEVICE by calls that have no dk_verdict to carry them
  * (dk_linear_fwd, dk_linear_bwd_wgrad): every wait inside the kernels is
  * bounded, and a kernel whose wait expires stops, leaves its output incomplete

@@ -71,6 +71,8 @@ def _signatures():
         "dk_decode_verify": [vp, pp, vp, vp, vp, vp, vp, vp],
         "dk_masked_linear": [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(dk_fault), vp],
         "dk_linear_bwd_wgrad": [vp, pp, vp, vp, i32, vp, vp, ctypes.c_float, vp, vp],
+        "dk_linear_bwd_wgrad_verify": [vp, pp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, vp,
+                                       ctypes.POINTER(dk_fault), vp],
         "dk_decode_verify_static": [ctypes.c_int, pp, vp, vp, vp, vp, vp, vp],
         "dk_device_status": [vp, ctypes.POINTER(ctypes.c_int32)],
         "dk_profile_enable": [vp, ctypes.c_int],
@@ -247,6 +249,15 @@ def dk_masked_linear(ctx: Context, p: dk_problem, W, x, r, C: np.ndarray, bias, 
     _check(lib().dk_masked_linear(ctx.handle, ctypes.byref(p), _dev(W), _dev(x), _dev(r), _host(C),
                                   _dev(bias), _dev(y), _dev(xbar_save),
                                   ctypes.c_void_p(verdict.data_ptr()), fp, _stream()), "dk_masked_linear")
+
+
+def dk_linear_bwd_wgrad_verify(ctx: Context, p: dk_problem, delta, xbar, C: np.ndarray, gamma: np.ndarray,
+                               scale: float, tol_w: float, dW, verdict, fault=None):
+    fp = ctypes.byref(fault) if fault is not None else None
+    _check(lib().dk_linear_bwd_wgrad_verify(ctx.handle, ctypes.byref(p), _dev(delta), _dev(xbar), _host(C),
+                                            _host(gamma), ctypes.c_float(scale), ctypes.c_float(tol_w), _dev(dW),
+                                            ctypes.c_void_p(verdict.data_ptr()), fp, _stream()),
+           "dk_linear_bwd_wgrad_verify")
 
 
 def dk_linear_bwd_wgrad(ctx: Context, p: dk_problem, delta, xbar, xbar_rows: int, C: np.ndarray,

@@ -571,6 +571,40 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
   return launch_verify_finalize(g, cv.nul, vs, verdict, st);
 }
 
+// Eq. 4-6 on encodings 0..K of every group of `xbar` (xbar_rows rows per group,
+// `xbar_elems` readable elements from `xbar` on).
+static dk_status wgrad_impl(dk_ctx* ctx, const Geom& g, const WsPlan& wp, const float* delta, const float* xbar,
+                            int xbar_rows, long long xbar_elems, const float* C_host, const float* gamma_host,
+                            float scale, float* dW, cudaStream_t st) {
+  CoefView cv;
+  dk_status s = upload_coefficients(ctx, g, C_host, gamma_host, true, true, st, &cv);
+  if (s != DK_OK) return s;
+  float* dtil = reinterpret_cast<float*>(static_cast<char*>(ctx->ws) + wp.dtil);
+  if (tc_wgrad_supported(ctx, g)) {
+    // tensor-core path: mixed deltas and encodings as TF32 hi/lo pairs (the
+    // y_bar region of the workspace, unused here, holds the lo part of dtil)
+    char* ws = static_cast<char*>(ctx->ws);
+    float* dt_lo = reinterpret_cast<float*>(ws + wp.ybar);
+    float* xb_hi = reinterpret_cast<float*>(ws + wp.xb_hi);
+    float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
+    {
+      // one launch: mixed deltas and stored encodings as hi/lo pairs, dW cleared
+      ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
+      s = tc_wgrad_prepass(g, delta, cv.dmix, dtil, dt_lo, xbar, xbar_elems, xb_hi, xb_lo, dW, ctx->sm_count, st);
+    }
+    if (s != DK_OK) return s;
+    ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
+    return tc_wgrad(ctx, g, dtil, dt_lo, xb_hi, xb_lo, xbar_rows, scale, dW, ctx_status_word(ctx), st);
+  }
+  {
+    ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
+    s = launch_mix_delta(g, delta, cv.dmix, dtil, ctx->sm_count, st);
+  }
+  if (s != DK_OK) return s;
+  ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
+  return launch_simt_wgrad(g, dtil, xbar, xbar_rows, scale, dW, ctx->sm_count, st);
+}
+
 dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* delta,
                               const float* xbar, int32_t xbar_rows, const float* C_host,
                               const float* gamma_host, float scale, float* dW, void* stream) {
@@ -584,35 +618,53 @@ dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* del
   if (!ctx->ws || ctx->ws_bytes < wp.total) return DK_ERR_WORKSPACE;
   DeviceGuard dg(ctx->device);
   if (!dg.ok) return DK_ERR_CUDA;
+  return wgrad_impl(ctx, g, wp, delta, xbar, xbar_rows, (long long)g.G * xbar_rows * g.n_in, C_host, gamma_host,
+                    scale, dW, static_cast<cudaStream_t>(stream));
+}
+
+dk_status dk_linear_bwd_wgrad_verify(dk_ctx* ctx, const dk_problem* p, const float* delta, const float* xbar,
+                                     const float* C_host, const float* gamma_host, float scale, float tol_w,
+                                     float* dW, dk_verdict* verdict, const dk_fault* fault, void* stream) {
+  if (!ctx || !delta || !xbar || !C_host || !gamma_host || !dW || !verdict) return DK_ERR_INVALID_ARG;
+  if (!aligned16(delta) || !aligned16(xbar) || !aligned16(dW) || !aligned16(verdict)) return DK_ERR_INVALID_ARG;
+  if (!(tol_w > 0.f)) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  if (g.n_in % 4) return DK_ERR_UNSUPPORTED;      // the second set starts one row into xbar: keep it 16-byte aligned
+  const long long n_dw = (long long)g.cout * g.kc;
+  if (fault && (fault->enc < 0 || fault->enc > 1 || fault->out_index < 0 || fault->out_index >= n_dw))
+    return DK_ERR_INVALID_ARG;
+  WsPlan wp = plan_workspace(g);
+  if (!ctx->ws || ctx->ws_bytes < wp.total) return DK_ERR_WORKSPACE;
+  DeviceGuard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  CoefView cv;
-  s = upload_coefficients(ctx, g, C_host, gamma_host, true, true, st, &cv);
+  const int K1 = g.K + 1, E = g.E;
+  // first set: encodings 0..K with C and gamma as given
+  s = wgrad_impl(ctx, g, wp, delta, xbar, E, (long long)g.G * E * g.n_in, C_host, gamma_host, scale, dW, st);
   if (s != DK_OK) return s;
-  float* dtil = reinterpret_cast<float*>(static_cast<char*>(ctx->ws) + wp.dtil);
-  if (tc_wgrad_supported(ctx, g)) {
-    // tensor-core path: mixed deltas and encodings as TF32 hi/lo pairs (the
-    // y_bar region of the workspace, unused here, holds the lo part of dtil)
-    char* ws = static_cast<char*>(ctx->ws);
-    float* dt_lo = reinterpret_cast<float*>(ws + wp.ybar);
-    float* xb_hi = reinterpret_cast<float*>(ws + wp.xb_hi);
-    float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
-    {
-      // one launch: mixed deltas and stored encodings as hi/lo pairs, dW cleared
-      ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
-      s = tc_wgrad_prepass(g, delta, cv.dmix, dtil, dt_lo, xbar, (long long)g.G * xbar_rows * g.n_in, xb_hi, xb_lo,
-                           dW, ctx->sm_count, st);
-    }
+  // second set: encodings 1..K+1 = rows 0..K of the tensor that starts one row
+  // later; its square coefficient part is rows 1..K+1 of C, its gammas rotated
+  std::vector<float> C2((size_t)g.G * E * K1), g2((size_t)g.G * K1);
+  for (int gi = 0; gi < g.G; ++gi) {
+    for (int i = 0; i < E; ++i)
+      for (int k = 0; k < K1; ++k)
+        C2[((size_t)gi * E + i) * K1 + k] = C_host[((size_t)gi * E + (i + 1) % E) * K1 + k];
+    for (int j = 0; j < K1; ++j) g2[(size_t)gi * K1 + j] = gamma_host[(size_t)gi * K1 + (j + 1) % K1];
+  }
+  float* dW2 = reinterpret_cast<float*>(static_cast<char*>(ctx->ws) + wp.w_hi);      // unused by the wgrad path
+  s = wgrad_impl(ctx, g, wp, delta, xbar + g.n_in, E, ((long long)g.G * E - 1) * g.n_in, C2.data(), g2.data(), scale,
+                 dW2, st);
+  if (s != DK_OK) return s;
+  ProfScope ps(ctx, DK_KERNEL_OTHER, fault ? 4 : 3, st);
+  if (fault) {
+    s = launch_add_fault(fault->enc == 0 ? dW : dW2, fault->out_index, fault->delta, st);
     if (s != DK_OK) return s;
-    ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
-    return tc_wgrad(ctx, g, dtil, dt_lo, xb_hi, xb_lo, xbar_rows, scale, dW, ctx_status_word(ctx), st);
   }
-  {
-    ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
-    s = launch_mix_delta(g, delta, cv.dmix, dtil, ctx->sm_count, st);
-  }
-  if (s != DK_OK) return s;
-  ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
-  return launch_simt_wgrad(g, dtil, xbar, xbar_rows, scale, dW, ctx->sm_count, st);
+  // 32 bytes of scratch behind the integrity statistics' counters
+  void* scratch = ctx->d_vstats + kVerifyStatFloats + 16;
+  return launch_wgrad_compare(dW, dW2, n_dw, tol_w, scratch, ctx_status_word(ctx), verdict, ctx->sm_count, st);
 }
 
 dk_status dk_device_status(dk_ctx* ctx, int32_t* status) {

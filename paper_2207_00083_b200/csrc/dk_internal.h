@@ -107,6 +107,12 @@ dk_status launch_add_fault(float* ybar, long long index, float delta, cudaStream
 dk_status launch_mix_delta(const Geom& g, const float* delta, const float* dmix, float* dtil,
                            int sm_count, cudaStream_t st);
 
+// dk_wgverify.cu: elementwise comparison of two weight gradients (n elements)
+// against tol * rms(a); `scratch32` = 32 bytes of device scratch; the verdict
+// also carries *status_word when that is given
+dk_status launch_wgrad_compare(const float* a, const float* b, long long n, float tol, void* scratch32,
+                               const int* status_word, dk_verdict* v, int sm_count, cudaStream_t st);
+
 // fp64 variants for DK_FP64_SIMT (dk_fp64.cu, dk_simt.cu)
 dk_status launch_encode64(const Geom& g, const float* x, const float* r, const float* enc, double* out64,
                           float* full32, int sm_count, cudaStream_t st);
