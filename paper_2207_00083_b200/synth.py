@@ -297,6 +297,26 @@ def draw_colluding(spec: LayerSpec, K: int, M: int) -> Dict[str, np.ndarray]:
     return out
 
 
+def draw_field_layer(spec: LayerSpec, p: int, with_delta: bool = True) -> Dict[str, np.ndarray]:
+    """Inputs of one layer for the finite-field arithmetic of the paper's
+    Section 5: the same floating-point x, W and delta as ``draw_layer`` plus a
+    bias, and what that section draws in the field itself, uniformly: the noise
+    ``rq`` [G, ...] over [0, p), the coefficients ``Cq`` [G, K+2, K+1] and the
+    diagonal ``gammaq`` [G, K+1] over [1, p).  The coefficient blocks are not
+    screened: a singular square part or a vanishing null-space component has
+    probability of order K/p.  Quantisation is part of the method and is not
+    done here."""
+    d = draw_layer(spec, with_delta=with_delta)
+    out = {"x": d["x"], "W": d["W"]}
+    if with_delta:
+        out["delta"] = d["delta"]
+    out["bias"] = _rng(spec, "bias").standard_normal(spec.cout, dtype=np.float32) * np.float32(0.1)
+    out["rq"] = _rng(spec, "r", 7).integers(0, p, size=_x_shape(spec, spec.G), dtype=np.int64)
+    out["Cq"] = _rng(spec, "coef", 7).integers(1, p, size=(spec.G, spec.K + 2, spec.K + 1), dtype=np.int64)
+    out["gammaq"] = _rng(spec, "gamma", 7).integers(1, p, size=(spec.G, spec.K + 1), dtype=np.int64)
+    return out
+
+
 def sample_coordinates(spec: LayerSpec, n: int, what: str = "y") -> np.ndarray:
     """Seeded sample of coordinates used for spot checks on large layers.
 
