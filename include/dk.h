@@ -244,6 +244,108 @@ DK_API dk_status dk_decode_verify_static(int device, const dk_problem* p, const 
                                          const float* C_host, const float* bias, float* y,
                                          dk_verdict* verdict, void* stream);
 
+/* ---------------------------------------------------------------------------
+ * The same path in the finite field F_p (Section 5, "Privacy Guarantee", and
+ * Algorithm 1).  The paper quantises inputs and weights to l fractional bits
+ * (l = 8), maps them to residues modulo the prime p = 2^25 - 39, draws the
+ * noise, the coefficients A and Gamma uniformly in F_p and runs Eq. 1, the
+ * linear operation, Eq. 2 and Eq. 4-6 modulo p; a result then decodes exactly
+ * and the integrity test of Section 4.4 is an exact comparison.
+ *  - Residues are uint32 in [0, p) on the device, laid out like their fp32
+ *    counterparts.  `prime` must be an odd prime below 2^30 (checked by trial
+ *    division; DK_ERR_INVALID_ARG otherwise).  Coefficient arrays C_host
+ *    [G][K+2][K+1] and gamma_host [G][K+1] are HOST arrays of residues
+ *    (gamma non-zero); the index convention is the one of the fp32 calls.
+ *  - DK_ERR_SINGULAR: a group's square block is not invertible modulo p, or a
+ *    component of its null vector is zero (a fault in that encoding would be
+ *    invisible to the redundant equation).
+ *  - A decoded value is meaningful as a number only while the true integer
+ *    result lies in (-p/2, p/2); the calls compute modulo p regardless, so
+ *    keeping the scaled values in range is the caller's job (the paper
+ *    normalises VGG activations for this reason).
+ *  - dk_verdict: ok, n_flagged and first_index as for the fp32 calls;
+ *    max_ratio is 0 when clean and 1 otherwise (the comparison is exact).
+ *  - dk_field_masked_linear and dk_field_linear_bwd_wgrad need a workspace of
+ *    dk_field_workspace_bytes registered with dk_set_workspace.
+ * ------------------------------------------------------------------------- */
+
+/* An accelerator that returns one wrong residue: delta (mod p) is added to
+ * ybar[group*(K+2)+enc][out_index] before decoding. */
+typedef struct {
+  int32_t group, enc;
+  int64_t out_index;
+  uint32_t delta;
+} dk_field_fault;
+
+DK_API dk_status dk_field_workspace_bytes(const dk_problem* p, size_t* bytes);
+
+/* Algorithm 1, procedures Round and Field: vq[i] = Field(Round(v[i]*2^scale_bits)),
+ * Round(t) = floor(t) if t - floor(t) < 0.5 else floor(t) + 1, Field = residue
+ * in [0, p).  scale_bits = l for inputs, weights and output gradients, 2l for a
+ * bias.  v: n fp32 values (device), finite; a value whose scaled magnitude
+ * is not below 4e18 maps to 0.  HBM-bound. */
+DK_API dk_status dk_field_quantize(dk_ctx* ctx, const float* v, int64_t n, int32_t scale_bits,
+                                   uint32_t prime, uint32_t* vq, void* stream);
+
+/* The way back for a tensor of residues (Section 5: "subtracts p from all the
+ * elements larger than p/2 to restore negative numbers"): v[i] = c*2^-scale_bits
+ * with c the representative of vq[i] in (-p/2, p/2).  Used for the weight
+ * gradient, whose residues carry 2l fractional bits. */
+DK_API dk_status dk_field_dequantize(dk_ctx* ctx, const uint32_t* vq, int64_t n, int32_t scale_bits,
+                                     uint32_t prime, float* v, void* stream);
+
+/* Eq. 1 and the redundant encoding of Section 4.4 modulo p:
+ *   xbar[g*(K+2)+i][e] = sum_{k<K} C[g][i][k]*xq[g*K+k][e] + C[g][i][K]*rq[g][e]  (mod p)
+ * xq: [G*K][n_in], rq: [G][n_in] (uniform residues drawn by the caller)
+ * -> xbar: [G*(K+2)][n_in]. */
+DK_API dk_status dk_field_encode(dk_ctx* ctx, const dk_problem* p, uint32_t prime, const uint32_t* xq,
+                                 const uint32_t* rq, const uint32_t* C_host, uint32_t* xbar, void* stream);
+
+/* The bilinear operation of Section 4.1 on residues (step "GPUs compute" of
+ * Algorithm 1): ybar = <Wq, xbar> modulo p for all G*(K+2) encoded samples,
+ * FC or convolution as in dk_linear_fwd, every layout and stride.  Exact:
+ * products are accumulated in 64 bits and reduced before they can overflow. */
+DK_API dk_status dk_field_linear_fwd(dk_ctx* ctx, const dk_problem* p, uint32_t prime, const uint32_t* Wq,
+                                     const uint32_t* xbar, uint32_t* ybar, void* stream);
+
+/* Eq. 2 and Section 4.4 modulo p, then the last steps of Algorithm 1.  Per
+ * group and output element e:
+ *   [y_0..y_{K-1}, z] = C_sq^{-1} . [ybar_0..ybar_K]  (mod p),  z dropped
+ *   flagged iff sum_i n[i]*ybar_i != 0 (mod p), n^T C = 0, n[K+1] = 1
+ *   y_k += bias_q[channel(e)] (mod p) when bias_q is given (device, [cout],
+ *          residues quantised with 2l bits)
+ *   yq (nullable, int32 [G*K][n_out]) = representative of y_k in (-p/2, p/2)
+ *   y  (nullable, fp32  [G*K][n_out]) = Round(yq*2^-l)*2^-l
+ * At least one of yq, y must be given.  *verdict (device) receives the summary. */
+DK_API dk_status dk_field_decode_verify(dk_ctx* ctx, const dk_problem* p, uint32_t prime, int32_t l,
+                                        const uint32_t* ybar, const uint32_t* C_host,
+                                        const uint32_t* bias_q, int32_t* yq, float* y,
+                                        dk_verdict* verdict, void* stream);
+
+/* Procedure "Linear Operations" of Algorithm 1 in one call: quantise W, x
+ * (l bits) and bias (2l bits, nullable, fp32 [cout]), encode with the noise rq,
+ * run the linear operation on the encodings, decode, check, return to floating
+ * point.  W, x: fp32 as in dk_masked_linear; xbar_save (nullable) receives the
+ * K+2 encodings per group as residues for dk_field_linear_bwd_wgrad; fault
+ * (host pointer, nullable) injects one wrong accelerator output. */
+DK_API dk_status dk_field_masked_linear(dk_ctx* ctx, const dk_problem* p, uint32_t prime, int32_t l,
+                                        const float* W, const float* x, const uint32_t* rq,
+                                        const uint32_t* C_host, const float* bias, float* y, int32_t* yq,
+                                        uint32_t* xbar_save, dk_verdict* verdict,
+                                        const dk_field_fault* fault, void* stream);
+
+/* Eq. 4-6 modulo p, summed over the virtual batches:
+ *   B[j][i] = (C_sq^{-1})[i][j] / gamma[g][j]                       (mod p)
+ *   dWq = sum_g sum_{j<=K} gamma[g][j] * < sum_i B[j][i]*deltaq[g*K+i], xbar[g*rows+j] >  (mod p)
+ * deltaq: [G*K][n_out] residues (quantise the output gradients with
+ * dk_field_quantize); xbar: xbar_rows (K+1 or K+2) encodings per group; dWq has
+ * the shape of W and equals sum_i <deltaq_i, xq_i> modulo p exactly; apply
+ * dk_field_dequantize with 2l bits and the batch scale afterwards. */
+DK_API dk_status dk_field_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, uint32_t prime,
+                                           const uint32_t* deltaq, const uint32_t* xbar, int32_t xbar_rows,
+                                           const uint32_t* C_host, const uint32_t* gamma_host,
+                                           uint32_t* dWq, void* stream);
+
 /* Measurement aids (the paper reports time per class of operation, Table 3;
  * these give the same breakdown per kernel class).  The library always counts
  * the kernels it launches; with profiling enabled it also brackets every

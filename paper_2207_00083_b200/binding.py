@@ -53,6 +53,11 @@ class dk_fault(ctypes.Structure):
                 ("out_index", ctypes.c_int64), ("delta", ctypes.c_float)]
 
 
+class dk_field_fault(ctypes.Structure):
+    _fields_ = [("group", ctypes.c_int32), ("enc", ctypes.c_int32),
+                ("out_index", ctypes.c_int64), ("delta", ctypes.c_uint32)]
+
+
 VERDICT_BYTES = ctypes.sizeof(dk_verdict)
 _lib = None
 
@@ -75,6 +80,15 @@ def _signatures():
                                        ctypes.POINTER(dk_fault), vp],
         "dk_decode_verify_static": [ctypes.c_int, pp, vp, vp, vp, vp, vp, vp],
         "dk_device_status": [vp, ctypes.POINTER(ctypes.c_int32)],
+        "dk_field_workspace_bytes": [pp, ctypes.POINTER(ctypes.c_size_t)],
+        "dk_field_quantize": [vp, vp, ctypes.c_int64, i32, ctypes.c_uint32, vp, vp],
+        "dk_field_dequantize": [vp, vp, ctypes.c_int64, i32, ctypes.c_uint32, vp, vp],
+        "dk_field_encode": [vp, pp, ctypes.c_uint32, vp, vp, vp, vp, vp],
+        "dk_field_linear_fwd": [vp, pp, ctypes.c_uint32, vp, vp, vp, vp],
+        "dk_field_decode_verify": [vp, pp, ctypes.c_uint32, i32, vp, vp, vp, vp, vp, vp, vp],
+        "dk_field_masked_linear": [vp, pp, ctypes.c_uint32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                   ctypes.POINTER(dk_field_fault), vp],
+        "dk_field_linear_bwd_wgrad": [vp, pp, ctypes.c_uint32, vp, vp, i32, vp, vp, vp, vp],
         "dk_profile_enable": [vp, ctypes.c_int],
         "dk_profile_read": [vp, ctypes.c_int, ctypes.POINTER(ctypes.c_double),
                             ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)],
@@ -165,9 +179,15 @@ class Context:
         _check(lib().dk_workspace_bytes(ctypes.byref(p), ctypes.byref(n)), "dk_workspace_bytes")
         return n.value
 
-    def ensure_workspace(self, p: dk_problem):
-        """Grows the torch-owned workspace to what `p` needs and registers it."""
-        need = self.workspace_bytes(p)
+    def field_workspace_bytes(self, p: dk_problem) -> int:
+        n = ctypes.c_size_t()
+        _check(lib().dk_field_workspace_bytes(ctypes.byref(p), ctypes.byref(n)), "dk_field_workspace_bytes")
+        return n.value
+
+    def ensure_workspace(self, p: dk_problem, field: bool = False):
+        """Grows the torch-owned workspace to what `p` needs and registers it
+        (``field=True``: what the finite-field calls need)."""
+        need = self.field_workspace_bytes(p) if field else self.workspace_bytes(p)
         if self._ws is None or self._ws.numel() < need + 256:
             self._ws = None
             self._ws = torch.empty(need + 256, dtype=torch.uint8, device=f"cuda:{self.device}")
@@ -265,3 +285,64 @@ def dk_linear_bwd_wgrad(ctx: Context, p: dk_problem, delta, xbar, xbar_rows: int
     _check(lib().dk_linear_bwd_wgrad(ctx.handle, ctypes.byref(p), _dev(delta), _dev(xbar), xbar_rows,
                                      _host(C), _host(gamma), ctypes.c_float(scale), _dev(dW), _stream()),
            "dk_linear_bwd_wgrad")
+
+
+# ---------------------------------------------------------------------------
+# finite-field calls: residues are int32 CUDA tensors holding values in [0, p)
+# (the library reads them as uint32), coefficient arrays NumPy uint32 on the host
+# ---------------------------------------------------------------------------
+def _res(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()):
+        raise ValueError("expected a contiguous int32 CUDA tensor of residues")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _host_u32(a: np.ndarray):
+    if not (isinstance(a, np.ndarray) and a.dtype == np.uint32 and a.flags["C_CONTIGUOUS"]):
+        raise ValueError("expected a C-contiguous uint32 NumPy array")
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def dk_field_quantize(ctx: Context, v, scale_bits: int, prime: int, vq):
+    _check(lib().dk_field_quantize(ctx.handle, _dev(v), v.numel(), scale_bits, prime, _res(vq), _stream()),
+           "dk_field_quantize")
+
+
+def dk_field_dequantize(ctx: Context, vq, scale_bits: int, prime: int, v):
+    _check(lib().dk_field_dequantize(ctx.handle, _res(vq), vq.numel(), scale_bits, prime, _dev(v), _stream()),
+           "dk_field_dequantize")
+
+
+def dk_field_encode(ctx: Context, p: dk_problem, prime: int, xq, rq, C: np.ndarray, xbar):
+    _check(lib().dk_field_encode(ctx.handle, ctypes.byref(p), prime, _res(xq), _res(rq), _host_u32(C),
+                                 _res(xbar), _stream()), "dk_field_encode")
+
+
+def dk_field_linear_fwd(ctx: Context, p: dk_problem, prime: int, Wq, xbar, ybar):
+    _check(lib().dk_field_linear_fwd(ctx.handle, ctypes.byref(p), prime, _res(Wq), _res(xbar), _res(ybar),
+                                     _stream()), "dk_field_linear_fwd")
+
+
+def dk_field_decode_verify(ctx: Context, p: dk_problem, prime: int, l: int, ybar, C: np.ndarray, bias_q, yq, y,
+                           verdict):
+    _check(lib().dk_field_decode_verify(ctx.handle, ctypes.byref(p), prime, l, _res(ybar), _host_u32(C),
+                                        _res(bias_q), _res(yq), _dev(y), ctypes.c_void_p(verdict.data_ptr()),
+                                        _stream()), "dk_field_decode_verify")
+
+
+def dk_field_masked_linear(ctx: Context, p: dk_problem, prime: int, l: int, W, x, rq, C: np.ndarray, bias, y, yq,
+                           xbar_save, verdict, fault: Optional[dk_field_fault] = None):
+    fp = ctypes.byref(fault) if fault is not None else None
+    _check(lib().dk_field_masked_linear(ctx.handle, ctypes.byref(p), prime, l, _dev(W), _dev(x), _res(rq),
+                                        _host_u32(C), _dev(bias), _dev(y), _res(yq), _res(xbar_save),
+                                        ctypes.c_void_p(verdict.data_ptr()), fp, _stream()),
+           "dk_field_masked_linear")
+
+
+def dk_field_linear_bwd_wgrad(ctx: Context, p: dk_problem, prime: int, deltaq, xbar, xbar_rows: int, C: np.ndarray,
+                              gamma: np.ndarray, dWq):
+    _check(lib().dk_field_linear_bwd_wgrad(ctx.handle, ctypes.byref(p), prime, _res(deltaq), _res(xbar), xbar_rows,
+                                           _host_u32(C), _host_u32(gamma), _res(dWq), _stream()),
+           "dk_field_linear_bwd_wgrad")

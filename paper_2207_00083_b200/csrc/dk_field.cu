@@ -1,0 +1,996 @@
+// The masked path in the finite field F_p (Section 5 of the paper, Algorithm 1):
+// quantisation to residues, Eq. 1 / Eq. 2 / the redundant equation of
+// Section 4.4 and Eq. 4-6 modulo a prime p, with an exact equality test.
+//
+// Residues are uint32 in [0, p), p < 2^30.  A product of two residues is below
+// 2^60; every contraction accumulates such products in uint64 and reduces
+// before the sum can pass 2^64 (the host derives how many terms fit).
+// Reduction is Barrett's: q = mulhi(x, floor(2^64 / p)) is the true quotient
+// or one less, so x - q*p lies in [0, 2p).
+#include <stdlib.h>
+#include <string.h>
+
+#include <vector>
+
+#include "dk_internal.h"
+
+namespace dk {
+namespace {
+
+typedef unsigned int u32;
+typedef unsigned long long u64;
+
+struct Modulus {
+  u64 m;   // floor(2^64 / p)
+  u32 p;
+};
+
+__host__ __device__ __forceinline__ u32 reduce64(u64 x, Modulus md) {
+#ifdef __CUDA_ARCH__
+  u64 q = __umul64hi(x, md.m);
+#else
+  u64 q = (u64)(((unsigned __int128)x * md.m) >> 64);
+#endif
+  u64 r = x - q * md.p;
+  if (r >= md.p) r -= md.p;
+  if (r >= md.p) r -= md.p;
+  return (u32)r;
+}
+
+// ---------------------------------------------------------------------------
+// host-side algebra in F_p (tiny matrices)
+// ---------------------------------------------------------------------------
+bool prime_by_trial_division(u32 p) {
+  if (p < 3 || (p & 1) == 0) return false;
+  for (u32 d = 3; (u64)d * d <= p; d += 2)
+    if (p % d == 0) return false;
+  return true;
+}
+
+u32 mulmod(u32 a, u32 b, u32 p) { return (u32)(((u64)a * b) % p); }
+
+// a^(p-2) mod p: the inverse by Fermat's little theorem
+u32 invmod(u32 a, u32 p) {
+  u32 result = 1, base = a % p;
+  u32 e = p - 2;
+  while (e) {
+    if (e & 1) result = mulmod(result, base, p);
+    base = mulmod(base, base, p);
+    e >>= 1;
+  }
+  return result;
+}
+
+// Gauss-Jordan elimination over F_p; false when singular.
+bool invert_mod(const u32* M, int n, u32 p, u32* inv) {
+  u32 a[(DK_MAX_K + 1) * (DK_MAX_K + 1)];
+  for (int i = 0; i < n * n; ++i) a[i] = M[i] % p;
+  for (int i = 0; i < n; ++i)
+    for (int j = 0; j < n; ++j) inv[i * n + j] = (i == j);
+  for (int c = 0; c < n; ++c) {
+    int piv = -1;
+    for (int r = c; r < n && piv < 0; ++r)
+      if (a[r * n + c]) piv = r;
+    if (piv < 0) return false;
+    if (piv != c)
+      for (int j = 0; j < n; ++j) {
+        u32 t = a[c * n + j]; a[c * n + j] = a[piv * n + j]; a[piv * n + j] = t;
+        t = inv[c * n + j]; inv[c * n + j] = inv[piv * n + j]; inv[piv * n + j] = t;
+      }
+    const u32 ip = invmod(a[c * n + c], p);
+    for (int j = 0; j < n; ++j) {
+      a[c * n + j] = mulmod(a[c * n + j], ip, p);
+      inv[c * n + j] = mulmod(inv[c * n + j], ip, p);
+    }
+    for (int r = 0; r < n; ++r) {
+      if (r == c || a[r * n + c] == 0) continue;
+      const u32 f = a[r * n + c];
+      for (int j = 0; j < n; ++j) {
+        a[r * n + j] = (a[r * n + j] + p - mulmod(f, a[c * n + j], p)) % p;
+        inv[r * n + j] = (inv[r * n + j] + p - mulmod(f, inv[c * n + j], p)) % p;
+      }
+    }
+  }
+  return true;
+}
+
+// Per-call tables in device memory, one block per group (all residues):
+// enc [G][K+2][K+1] as given; dec [G][K][K+1] rows 0..K-1 of C_sq^{-1};
+// nul [G][K+2] with nul^T C = 0, nul[K+1] = 1; mix [G][K+1][K] = gamma_j*B[j][i].
+struct FieldCoef {
+  const u32* enc;
+  const u32* dec;
+  const u32* nul;
+  const u32* mix;
+};
+
+dk_status upload_field_coefficients(dk_ctx* ctx, const Geom& g, u32 p, const u32* C_host,
+                                    const u32* gamma_host, bool want_dec, bool want_mix,
+                                    cudaStream_t st, FieldCoef* view) {
+  const int K = g.K, K1 = K + 1, E = K + 2, G = g.G;
+  const size_t n_enc = (size_t)G * E * K1, n_dec = (size_t)G * K * K1, n_nul = (size_t)G * E,
+               n_mix = (size_t)G * K1 * K;
+  const size_t total = n_enc + n_dec + n_nul + n_mix;
+  if (total * sizeof(u32) > kCoefSlotBytes) return DK_ERR_SHAPE;
+  for (size_t i = 0; i < n_enc; ++i)
+    if (C_host[i] >= p) return DK_ERR_INVALID_ARG;
+
+  int s = ctx->cur_slot;
+  ctx->cur_slot = (s + 1) % kCoefSlots;
+  if (ctx->slot_used[s]) DK_CUDA_CHECK(cudaEventSynchronize(ctx->slot_ev[s]));
+  u32* h = reinterpret_cast<u32*>(ctx->h_stage + (size_t)s * kCoefSlotBytes);
+  u32* d = reinterpret_cast<u32*>(ctx->d_stage + (size_t)s * kCoefSlotBytes);
+  u32* h_enc = h;
+  u32* h_dec = h_enc + n_enc;
+  u32* h_nul = h_dec + n_dec;
+  u32* h_mix = h_nul + n_nul;
+  memcpy(h_enc, C_host, n_enc * sizeof(u32));
+  memset(h_dec, 0, (n_dec + n_nul + n_mix) * sizeof(u32));
+  if (want_dec || want_mix) {
+    u32 inv[(DK_MAX_K + 1) * (DK_MAX_K + 1)];
+    for (int gi = 0; gi < G; ++gi) {
+      const u32* Cg = C_host + (size_t)gi * E * K1;
+      if (!invert_mod(Cg, K1, p, inv)) return DK_ERR_SINGULAR;
+      for (int k = 0; k < K; ++k)
+        for (int i = 0; i < K1; ++i) h_dec[((size_t)gi * K + k) * K1 + i] = inv[k * K1 + i];
+      // null vector: n[0..K] = -C[K+1] . C_sq^{-1}, n[K+1] = 1.  A zero
+      // component would hide a fault in that encoding from the check.
+      for (int i = 0; i < K1; ++i) {
+        u64 acc = 0;
+        for (int k = 0; k < K1; ++k) acc = (acc + (u64)Cg[(size_t)K1 * K1 + k] * inv[k * K1 + i]) % p;
+        const u32 ni = (u32)((p - acc) % p);
+        if (ni == 0) return DK_ERR_SINGULAR;
+        h_nul[(size_t)gi * E + i] = ni;
+      }
+      h_nul[(size_t)gi * E + K1] = 1;
+      if (want_mix) {
+        // Eq. 5: B[j][i] = inv[i][j] / gamma[j]; the kernels use gamma[j]*B[j][i]
+        for (int j = 0; j < K1; ++j) {
+          const u32 gm = gamma_host[(size_t)gi * K1 + j];
+          if (gm == 0 || gm >= p) return DK_ERR_INVALID_ARG;
+          const u32 gi_inv = invmod(gm, p);
+          for (int i = 0; i < K; ++i) {
+            const u32 B = mulmod(inv[i * K1 + j], gi_inv, p);
+            h_mix[((size_t)gi * K1 + j) * K + i] = mulmod(gm, B, p);
+          }
+        }
+      }
+    }
+  }
+  DK_CUDA_CHECK(cudaMemcpyAsync(d, h, total * sizeof(u32), cudaMemcpyHostToDevice, st));
+  DK_CUDA_CHECK(cudaEventRecord(ctx->slot_ev[s], st));
+  ctx->slot_used[s] = true;
+  view->enc = d;
+  view->dec = d + n_enc;
+  view->nul = view->dec + n_dec;
+  view->mix = view->nul + n_nul;
+  return DK_OK;
+}
+
+// ---------------------------------------------------------------------------
+// elementwise kernels
+// ---------------------------------------------------------------------------
+
+// Field(Round(v * scale)), Algorithm 1: floor when the fractional part is
+// below one half, floor + 1 otherwise; then the residue in [0, p).  v * scale
+// (a power of two) and the fractional part are exact in fp32.
+__global__ void __launch_bounds__(256) field_quantize_kernel(const float* __restrict__ v, long long n, float scale,
+                                                            u32 p, u32* __restrict__ out) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const float t = v[i] * scale;
+    const float f = floorf(t);
+    const float q = (t - f < 0.5f) ? f : f + 1.0f;
+    u32 res = 0;
+    if (fabsf(q) < 2.0e9f) {        // the usual case: 32-bit remainder
+      int m = (int)q % (int)p;
+      if (m < 0) m += (int)p;
+      res = (u32)m;
+    } else if (fabsf(q) < 4.0e18f) {      // also false for NaN
+      long long m = (long long)q % (long long)p;
+      if (m < 0) m += p;
+      res = (u32)m;
+    }
+    out[i] = res;
+  }
+}
+
+// value = centred residue * 2^-shift
+__global__ void __launch_bounds__(256) field_dequantize_kernel(const u32* __restrict__ vq, long long n, u32 p,
+                                                              double inv_scale, float* __restrict__ out) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const u32 r = vq[i];
+    const long long c = (2ull * r > p) ? (long long)r - (long long)p : (long long)r;
+    out[i] = (float)((double)c * inv_scale);
+  }
+}
+
+template <int VEC>
+struct Vec;
+template <>
+struct Vec<1> {
+  u32 v[1];
+  __device__ __forceinline__ void load(const u32* p) { v[0] = __ldg(p); }
+  __device__ __forceinline__ void store(u32* p) const { *p = v[0]; }
+};
+template <>
+struct Vec<4> {
+  u32 v[4];
+  __device__ __forceinline__ void load(const u32* p) {
+    const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  }
+  __device__ __forceinline__ void store(u32* p) const {
+    *reinterpret_cast<uint4*>(p) = make_uint4(v[0], v[1], v[2], v[3]);
+  }
+};
+
+// out[g*ROUT + i][e] = sum_{k<RA} T[g][i][k]*a[g*RA + k][e] (+ T[g][i][RA]*b[g][e] when b is given).
+// Serves Eq. 1 (a = inputs, b = noise, ROUT = K+2) and the delta mixing of
+// Eq. 4 (a = deltas, no b, ROUT = K+1).  RIN = RA + (b ? 1 : 0) <= 9 terms below
+// 2^60 each: the sum stays below 2^64.
+template <int RIN, int VEC>
+__global__ void __launch_bounds__(256) field_mix_rows_kernel(const u32* __restrict__ a, const u32* __restrict__ b,
+                                                            const u32* __restrict__ table, u32* __restrict__ out,
+                                                            long long n, int rout, Modulus md) {
+  __shared__ u32 T[(DK_MAX_K + 2) * (DK_MAX_K + 1)];
+  const int g = blockIdx.y;
+  const int RA = b ? RIN - 1 : RIN;
+  for (int i = threadIdx.x; i < rout * RIN; i += blockDim.x) T[i] = table[(size_t)g * rout * RIN + i];
+  __syncthreads();
+  const long long nvec = n / VEC;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+    Vec<VEC> src[RIN];
+#pragma unroll
+    for (int k = 0; k < RIN; ++k) {
+      if (k < RA) src[k].load(a + ((long long)g * RA + k) * n + i * VEC);
+      else src[k].load(b + (long long)g * n + i * VEC);
+    }
+    for (int r = 0; r < rout; ++r) {
+      u64 acc[VEC];
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) acc[v] = 0;
+#pragma unroll
+      for (int k = 0; k < RIN; ++k) {
+        const u32 c = T[r * RIN + k];
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) acc[v] += (u64)c * src[k].v[v];
+      }
+      Vec<VEC> o;
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) o.v[v] = reduce64(acc[v], md);
+      o.store(out + ((long long)g * rout + r) * n + i * VEC);
+    }
+  }
+}
+
+template <int VEC>
+dk_status launch_mix_rows(int rin, const u32* a, const u32* b, const u32* table, u32* out, long long n, int rout,
+                          int G, Modulus md, int sm_count, cudaStream_t st) {
+  long long nvec = n / VEC;
+  long long bx = (nvec + 255) / 256;
+  const long long cap = (16LL * sm_count + G - 1) / G;
+  if (bx > cap) bx = cap;
+  if (bx < 1) bx = 1;
+  dim3 grid((unsigned)bx, (unsigned)G);
+  switch (rin) {
+#define DK_CASE(R) \
+  case R: field_mix_rows_kernel<R, VEC><<<grid, 256, 0, st>>>(a, b, table, out, n, rout, md); break;
+    DK_CASE(1) DK_CASE(2) DK_CASE(3) DK_CASE(4) DK_CASE(5) DK_CASE(6) DK_CASE(7) DK_CASE(8) DK_CASE(9)
+#undef DK_CASE
+    default: return DK_ERR_SHAPE;
+  }
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+dk_status mix_rows(int rin, const u32* a, const u32* b, const u32* table, u32* out, long long n, int rout, int G,
+                   Modulus md, int sm_count, cudaStream_t st) {
+  if (G > 65535) return DK_ERR_SHAPE;
+  const bool vec4 = (n % 4) == 0 && ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) |
+                                      reinterpret_cast<uintptr_t>(out)) & 15) == 0;
+  return vec4 ? launch_mix_rows<4>(rin, a, b, table, out, n, rout, G, md, sm_count, st)
+              : launch_mix_rows<1>(rin, a, b, table, out, n, rout, G, md, sm_count, st);
+}
+
+// Eq. 2 and the redundant equation in F_p.  One thread decodes VEC output
+// positions of one group: it reads the K+2 encoded values, forms
+// rho = sum_i nul[i]*ybar_i (mod p), which is zero exactly when the redundant
+// equation agrees with the other K+1, decodes y_k = sum_i dec[k][i]*ybar_i
+// (+ bias) and writes the centred integer and/or Round(y*2^-l)*2^-l.
+// Flagged positions are counted per warp and reported with one atomic each.
+struct DecodeParams {
+  const u32* ybar;
+  const u32* dec;
+  const u32* nul;
+  const u32* bias;   // residues, [cout], nullable
+  int* yq;           // nullable
+  float* y;          // nullable
+  dk_verdict* v;
+  long long n;       // positions per sample
+  long long ch_div;  // channel of position e = (e / ch_div) % cout
+  int cout;
+  double inv_scale;  // 2^-l
+  Modulus md;
+};
+
+template <int K, int VEC>
+__global__ void __launch_bounds__(256) field_decode_verify_kernel(DecodeParams p) {
+  constexpr int K1 = K + 1, E = K + 2;
+  __shared__ u32 D[K * K1];
+  __shared__ u32 N[E];
+  const int g = blockIdx.y;
+  for (int i = threadIdx.x; i < K * K1; i += blockDim.x) D[i] = p.dec[(size_t)g * K * K1 + i];
+  for (int i = threadIdx.x; i < E; i += blockDim.x) N[i] = p.nul[(size_t)g * E + i];
+  __syncthreads();
+  const long long nvec = p.n / VEC;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long first = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long lane0 = first - (threadIdx.x & 31);
+  // every lane of a warp runs the same number of rounds (the ballot below is warp-wide)
+  for (long long i0 = lane0; i0 < nvec; i0 += stride) {
+    const long long i = i0 + (threadIdx.x & 31);
+    const bool act = i < nvec;
+    unsigned int nbad = 0;
+    long long firstbad = 0x7fffffffffffffffLL;
+    if (act) {
+      Vec<VEC> yb[E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) yb[e].load(p.ybar + ((long long)g * E + e) * p.n + i * VEC);
+      u64 rho[VEC];
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) rho[v] = 0;
+#pragma unroll
+      for (int e = 0; e < E; ++e)
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) rho[v] += (u64)N[e] * yb[e].v[v];
+#pragma unroll
+      for (int v = VEC - 1; v >= 0; --v)
+        if (reduce64(rho[v], p.md) != 0) {
+          ++nbad;
+          firstbad = (long long)g * p.n + i * VEC + v;
+        }
+#pragma unroll
+      for (int k = 0; k < K; ++k) {
+        u64 acc[VEC];
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) acc[v] = 0;
+#pragma unroll
+        for (int e = 0; e < K1; ++e) {
+          const u32 c = D[k * K1 + e];
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) acc[v] += (u64)c * yb[e].v[v];
+        }
+        const long long o = ((long long)g * K + k) * p.n + i * VEC;
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) {
+          u32 r = reduce64(acc[v], p.md);
+          if (p.bias) {
+            const long long e = i * VEC + v;
+            r += __ldg(p.bias + (int)((e / p.ch_div) % p.cout));
+            if (r >= p.md.p) r -= p.md.p;
+          }
+          const long long c = (2ull * r > p.md.p) ? (long long)r - (long long)p.md.p : (long long)r;
+          if (p.yq) p.yq[o + v] = (int)c;
+          if (p.y) {
+            const double t = (double)c * p.inv_scale;
+            const double f = floor(t);
+            p.y[o + v] = (float)(((t - f < 0.5) ? f : f + 1.0) * p.inv_scale);
+          }
+        }
+      }
+    }
+    const unsigned int any = __ballot_sync(0xffffffffu, nbad != 0);
+    if (any) {
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) {
+        nbad += __shfl_xor_sync(0xffffffffu, nbad, s);
+        const long long other = __shfl_xor_sync(0xffffffffu, firstbad, s);
+        firstbad = other < firstbad ? other : firstbad;
+      }
+      if ((threadIdx.x & 31) == 0) {
+        atomicAdd(&p.v->n_flagged, nbad);
+        atomicMin(reinterpret_cast<u64*>(&p.v->first_index), (u64)firstbad);
+        atomicExch(&p.v->ok, 0);
+        p.v->max_ratio = 1.0f;
+      }
+    }
+  }
+}
+
+__global__ void field_verdict_begin_kernel(dk_verdict* v) {
+  v->ok = 1;
+  v->n_flagged = 0;
+  v->first_index = -1;      // all ones: also the identity of the unsigned minimum
+  v->max_ratio = 0.f;
+  v->status = 0;
+}
+
+__global__ void field_add_fault_kernel(u32* ybar, long long index, u32 delta, u32 p) {
+  ybar[index] = (u32)(((u64)ybar[index] + delta) % p);
+}
+
+template <int VEC>
+dk_status launch_decode_t(int K, const DecodeParams& p, int G, int sm_count, cudaStream_t st) {
+  long long nvec = p.n / VEC;
+  long long bx = (nvec + 255) / 256;
+  const long long cap = (16LL * sm_count + G - 1) / G;
+  if (bx > cap) bx = cap;
+  if (bx < 1) bx = 1;
+  dim3 grid((unsigned)bx, (unsigned)G);
+  switch (K) {
+#define DK_CASE(KK) \
+  case KK: field_decode_verify_kernel<KK, VEC><<<grid, 256, 0, st>>>(p); break;
+    DK_CASE(1) DK_CASE(2) DK_CASE(3) DK_CASE(4) DK_CASE(5) DK_CASE(6) DK_CASE(7) DK_CASE(8)
+#undef DK_CASE
+    default: return DK_ERR_SHAPE;
+  }
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+// ---------------------------------------------------------------------------
+// the contraction <W_q, x_bar> modulo p (implicit GEMM, every geometry/layout)
+// ---------------------------------------------------------------------------
+constexpr int BM = 64, BN = 64, BK = 16, NT = 256;
+
+struct FwdParams {
+  const u32* W;
+  const u32* x;
+  u32* y;
+  int cin, cout, h, w, kw, stride, pad, ho, wo, kc;
+  long long N;           // samples * ho * wo
+  long long n_in, n_out;
+  long long xs_c, xs_h, xs_w, ws_o, ws_c, ws_u, ws_v, ys_c, ys_h, ys_w;
+  int fold_tiles;        // k-tiles between two reductions
+  Modulus md;
+};
+
+__global__ void __launch_bounds__(NT) field_fwd_kernel(FwdParams p) {
+  __shared__ __align__(16) u32 As[BK][BM + 4];
+  __shared__ __align__(16) u32 Bs[BK][BN + 4];
+  const int t = threadIdx.x;
+  const int tx = t % 16, ty = t / 16;
+  const int m0 = blockIdx.y * BM;
+  const long long n0 = (long long)blockIdx.x * BN;
+
+  // load slots: element (kk, mm) with kk = t % 16, mm = t / 16 + 16*i
+  const int kk = t % BK;
+  long long a_off[4];
+  bool a_ok[4];
+  long long b_base[4];
+  int b_ih0[4], b_iw0[4];
+  bool b_ok[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int mm = t / BK + 16 * i;
+    a_ok[i] = (m0 + mm) < p.cout;
+    a_off[i] = (long long)(m0 + mm) * p.ws_o;
+    const long long n = n0 + mm;
+    b_ok[i] = n < p.N;
+    const long long nn = b_ok[i] ? n : 0;
+    const int ow = (int)(nn % p.wo);
+    const long long r = nn / p.wo;
+    const int oh = (int)(r % p.ho);
+    const long long s = r / p.ho;
+    b_base[i] = s * p.n_in;
+    b_ih0[i] = oh * p.stride - p.pad;
+    b_iw0[i] = ow * p.stride - p.pad;
+  }
+
+  u64 acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0;
+
+  int fold = 0;
+  for (int k0 = 0; k0 < p.kc; k0 += BK) {
+    const int k = k0 + kk;
+    const bool kok = k < p.kc;
+    const int tap = kok ? k / p.cin : 0;
+    const int ci = kok ? k - tap * p.cin : 0;
+    const int u = tap / p.kw, v = tap - u * p.kw;
+    const long long woff = (long long)ci * p.ws_c + (long long)u * p.ws_u + (long long)v * p.ws_v;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int mm = t / BK + 16 * i;
+      As[kk][mm] = (kok && a_ok[i]) ? __ldg(p.W + a_off[i] + woff) : 0u;
+      const int ih = b_ih0[i] + u, iw = b_iw0[i] + v;
+      const bool ok = kok && b_ok[i] && ih >= 0 && ih < p.h && iw >= 0 && iw < p.w;
+      Bs[kk][mm] = ok ? __ldg(p.x + b_base[i] + (long long)ci * p.xs_c + (long long)ih * p.xs_h +
+                              (long long)iw * p.xs_w)
+                      : 0u;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < BK; ++q) {
+      const uint4 a4 = *reinterpret_cast<const uint4*>(&As[q][ty * 4]);
+      const uint4 b4 = *reinterpret_cast<const uint4*>(&Bs[q][tx * 4]);
+      const u32 a[4] = {a4.x, a4.y, a4.z, a4.w};
+      const u32 b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] += (u64)a[i] * b[j];
+    }
+    __syncthreads();
+    if (++fold == p.fold_tiles) {
+      fold = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = reduce64(acc[i][j], p.md);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const long long n = n0 + tx * 4 + j;
+    if (n >= p.N) continue;
+    const int ow = (int)(n % p.wo);
+    const long long r = n / p.wo;
+    const int oh = (int)(r % p.ho);
+    const long long s = r / p.ho;
+    u32* yo = p.y + s * p.n_out + (long long)oh * p.ys_h + (long long)ow * p.ys_w;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int m = m0 + ty * 4 + i;
+      if (m < p.cout) yo[(long long)m * p.ys_c] = reduce64(acc[i][j], p.md);
+    }
+  }
+}
+
+// How many products of two residues may be added to one residue in a uint64.
+long long terms_per_reduction(u32 p) {
+  const u64 pm = (u64)p - 1;
+  return (long long)((~0ull - pm) / (pm * pm));
+}
+
+dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* ybar, int nsamples, Modulus md,
+                           cudaStream_t st) {
+  FwdParams p;
+  p.W = W; p.x = xbar; p.y = ybar;
+  p.cin = g.cin; p.cout = g.cout; p.h = g.h; p.w = g.w; p.kw = g.kw; p.stride = g.stride;
+  p.pad = g.pad; p.ho = g.ho; p.wo = g.wo; p.kc = g.kc;
+  p.N = (long long)nsamples * g.ho * g.wo;
+  p.n_in = g.n_in; p.n_out = g.n_out;
+  p.xs_c = g.xs_c; p.xs_h = g.xs_h; p.xs_w = g.xs_w;
+  p.ws_o = g.ws_o; p.ws_c = g.ws_c; p.ws_u = g.ws_u; p.ws_v = g.ws_v;
+  p.ys_c = g.ys_c; p.ys_h = g.ys_h; p.ys_w = g.ys_w;
+  long long ft = terms_per_reduction(md.p) / BK;
+  if (ft < 1) return DK_ERR_UNSUPPORTED;
+  if (ft > 256) ft = 256;
+  p.fold_tiles = (int)ft;
+  p.md = md;
+  const long long nb = (p.N + BN - 1) / BN;
+  if (nb > 2147483647LL) return DK_ERR_SHAPE;
+  dim3 grid((unsigned)nb, (unsigned)((g.cout + BM - 1) / BM));
+  if (grid.y > 65535) return DK_ERR_SHAPE;
+  field_fwd_kernel<<<grid, NT, 0, st>>>(p);
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+// ---------------------------------------------------------------------------
+// the weight-gradient contraction modulo p
+// ---------------------------------------------------------------------------
+struct WgParams {
+  const u32* d;     // mixed deltas [G*(K+1)][n_out]
+  const u32* x;     // encodings, xbar_rows per group
+  u64* acc;         // [cout*kc] partial sums of residues, cleared by the caller
+  int cin, cout, h, w, kw, stride, pad, ho, wo, kc;
+  int K1, xbar_rows, P, PC;   // P = ho*wo pixels, PC = ceil(P/BK)
+  long long GP;               // G * PC contraction blocks
+  long long per_split;
+  int fold_blocks;            // contraction blocks between two reductions
+  long long n_in, n_out;
+  long long xs_c, xs_h, xs_w, ws_o, ws_c, ws_u, ws_v, ys_c, ys_h, ys_w;
+  Modulus md;
+};
+
+__global__ void __launch_bounds__(NT) field_wgrad_kernel(WgParams p) {
+  __shared__ __align__(16) u32 As[BK][BM + 4];
+  __shared__ __align__(16) u32 Bs[BK][BN + 4];
+  const int t = threadIdx.x;
+  const int tx = t % 16, ty = t / 16;
+  const int m0 = blockIdx.y * BM;
+  const int kb0 = blockIdx.x * BN;
+  const long long gp_lo = (long long)blockIdx.z * p.per_split;
+  long long gp_hi = gp_lo + p.per_split;
+  if (gp_hi > p.GP) gp_hi = p.GP;
+
+  // load slots: (pixel pp = t / 64 + 4*i, column cc = t % 64)
+  const int cc = t % 64;
+  const bool a_ok = (m0 + cc) < p.cout;
+  const long long a_off = (long long)(m0 + cc) * p.ys_c;
+  const int kcol = kb0 + cc;
+  const bool b_ok = kcol < p.kc;
+  const int tap = b_ok ? kcol / p.cin : 0;
+  const int ci = b_ok ? kcol - tap * p.cin : 0;
+  const int u = tap / p.kw, v = tap - u * p.kw;
+  const long long b_off = (long long)ci * p.xs_c;
+
+  u64 acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0;
+
+  int fold = 0;
+  for (long long gp = gp_lo; gp < gp_hi; ++gp) {
+    const long long g = gp / p.PC;
+    const int pc = (int)(gp - g * p.PC);
+    int oh[4], ow[4];
+    bool pok[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int pix = pc * BK + t / 64 + 4 * i;
+      pok[i] = pix < p.P;
+      const int pp = pok[i] ? pix : 0;
+      oh[i] = pp / p.wo;
+      ow[i] = pp - oh[i] * p.wo;
+    }
+    for (int j = 0; j < p.K1; ++j) {
+      const u32* dj = p.d + (g * p.K1 + j) * p.n_out;
+      const u32* xj = p.x + (g * p.xbar_rows + j) * p.n_in;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int pp = t / 64 + 4 * i;
+        As[pp][cc] = (pok[i] && a_ok)
+                         ? __ldg(dj + a_off + (long long)oh[i] * p.ys_h + (long long)ow[i] * p.ys_w)
+                         : 0u;
+        const int ih = oh[i] * p.stride + u - p.pad, iw = ow[i] * p.stride + v - p.pad;
+        const bool ok = pok[i] && b_ok && ih >= 0 && ih < p.h && iw >= 0 && iw < p.w;
+        Bs[pp][cc] = ok ? __ldg(xj + b_off + (long long)ih * p.xs_h + (long long)iw * p.xs_w) : 0u;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int q = 0; q < BK; ++q) {
+        const uint4 a4 = *reinterpret_cast<const uint4*>(&As[q][ty * 4]);
+        const uint4 b4 = *reinterpret_cast<const uint4*>(&Bs[q][tx * 4]);
+        const u32 a[4] = {a4.x, a4.y, a4.z, a4.w};
+        const u32 b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) acc[i][jj] += (u64)a[i] * b[jj];
+      }
+      __syncthreads();
+    }
+    if (++fold == p.fold_blocks) {
+      fold = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) acc[i][jj] = reduce64(acc[i][jj], p.md);
+    }
+  }
+#pragma unroll
+  for (int jj = 0; jj < 4; ++jj) {
+    const int kcol2 = kb0 + tx * 4 + jj;
+    if (kcol2 >= p.kc) continue;
+    const int tap2 = kcol2 / p.cin, ci2 = kcol2 - tap2 * p.cin;
+    const int u2 = tap2 / p.kw, v2 = tap2 - u2 * p.kw;
+    const long long woff = (long long)ci2 * p.ws_c + (long long)u2 * p.ws_u + (long long)v2 * p.ws_v;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int m = m0 + ty * 4 + i;
+      if (m < p.cout) atomicAdd(p.acc + (long long)m * p.ws_o + woff, (u64)reduce64(acc[i][jj], p.md));
+    }
+  }
+}
+
+// the slices' residues (at most 65535 of them, each below p) summed in uint64 -> residue
+__global__ void __launch_bounds__(256) field_reduce_kernel(const u64* __restrict__ acc, long long n, Modulus md,
+                                                          u32* __restrict__ out) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+    out[i] = reduce64(acc[i], md);
+}
+
+int ew_blocks(long long n, int sm_count) {
+  long long b = (n + 255) / 256;
+  if (b > 16LL * sm_count) b = 16LL * sm_count;
+  return (int)(b < 1 ? 1 : b);
+}
+
+struct FieldWs {
+  size_t wq, xq, xbar, ybar, bq, dtil, acc64, total;
+};
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+FieldWs plan_field_ws(const Geom& g) {
+  FieldWs w;
+  size_t off = 0;
+  w.wq = off; off += align_up((size_t)g.cout * g.kc * sizeof(u32), 1024);
+  w.xq = off; off += align_up((size_t)g.G * g.K * g.n_in * sizeof(u32), 1024);
+  w.xbar = off; off += align_up((size_t)g.G * g.E * g.n_in * sizeof(u32), 1024);
+  w.ybar = off; off += align_up((size_t)g.G * g.E * g.n_out * sizeof(u32), 1024);
+  w.bq = off; off += align_up((size_t)g.cout * sizeof(u32), 1024);
+  w.dtil = off; off += align_up((size_t)g.G * (g.K + 1) * g.n_out * sizeof(u32), 1024);
+  w.acc64 = off; off += align_up((size_t)g.cout * g.kc * sizeof(u64), 1024);
+  w.total = off;
+  return w;
+}
+
+struct Guard {
+  int prev;
+  bool ok;
+  explicit Guard(int dev) : prev(-1), ok(false) {
+    if (cudaGetDevice(&prev) != cudaSuccess) return;
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) return;
+    ok = true;
+  }
+  ~Guard() {
+    int cur = -1;
+    if (ok && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+dk_status make_modulus(uint32_t p, Modulus* md) {
+  if (p >= (1u << 30) || !prime_by_trial_division(p)) return DK_ERR_INVALID_ARG;
+  md->p = p;
+  md->m = ~0ull / p;      // = floor(2^64 / p): p is odd, so it does not divide 2^64
+  return DK_OK;
+}
+
+dk_status quantize_launch(const float* v, long long n, int scale_bits, u32 p, u32* out, int sm_count,
+                          cudaStream_t st) {
+  if (n == 0) return DK_OK;
+  field_quantize_kernel<<<ew_blocks(n, sm_count), 256, 0, st>>>(v, n, ldexpf(1.0f, scale_bits), p, out);
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+dk_status decode_verify_launch(dk_ctx* ctx, const Geom& g, int l, const u32* ybar, const FieldCoef& fc,
+                               const u32* bias_q, int* yq, float* y, dk_verdict* verdict, Modulus md,
+                               cudaStream_t st) {
+  {
+    ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+    field_verdict_begin_kernel<<<1, 1, 0, st>>>(verdict);
+    DK_CUDA_CHECK(cudaGetLastError());
+  }
+  DecodeParams dp;
+  dp.ybar = ybar; dp.dec = fc.dec; dp.nul = fc.nul; dp.bias = bias_q; dp.yq = yq; dp.y = y; dp.v = verdict;
+  dp.n = g.n_out;
+  dp.ch_div = (g.layout == DK_NCHW) ? (long long)g.ho * g.wo : 1;
+  dp.cout = g.cout;
+  dp.inv_scale = ldexp(1.0, -l);
+  dp.md = md;
+  const bool vec4 = (g.n_out % 4) == 0 && aligned16(ybar) && aligned16(yq) && aligned16(y);
+  ProfScope ps(ctx, DK_KERNEL_DECODE_VERIFY, 1, st);
+  return vec4 ? launch_decode_t<4>(g.K, dp, g.G, ctx->sm_count, st)
+              : launch_decode_t<1>(g.K, dp, g.G, ctx->sm_count, st);
+}
+
+}  // namespace
+}  // namespace dk
+
+using namespace dk;
+
+extern "C" {
+
+dk_status dk_field_workspace_bytes(const dk_problem* p, size_t* bytes) {
+  if (!bytes) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  *bytes = plan_field_ws(g).total;
+  return DK_OK;
+}
+
+dk_status dk_field_quantize(dk_ctx* ctx, const float* v, int64_t n, int32_t scale_bits, uint32_t prime,
+                            uint32_t* vq, void* stream) {
+  if (!ctx || n < 0 || (n > 0 && (!v || !vq)) || scale_bits < 0 || scale_bits > 60) return DK_ERR_INVALID_ARG;
+  Modulus md;
+  dk_status s = make_modulus(prime, &md);
+  if (s != DK_OK) return s;
+  Guard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+  return quantize_launch(v, n, scale_bits, prime, vq, ctx->sm_count, st);
+}
+
+dk_status dk_field_dequantize(dk_ctx* ctx, const uint32_t* vq, int64_t n, int32_t scale_bits, uint32_t prime,
+                              float* v, void* stream) {
+  if (!ctx || n < 0 || (n > 0 && (!v || !vq)) || scale_bits < 0 || scale_bits > 60) return DK_ERR_INVALID_ARG;
+  Modulus md;
+  dk_status s = make_modulus(prime, &md);
+  if (s != DK_OK) return s;
+  if (n == 0) return DK_OK;
+  Guard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+  field_dequantize_kernel<<<ew_blocks(n, ctx->sm_count), 256, 0, st>>>(vq, n, prime, ldexp(1.0, -scale_bits), v);
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+dk_status dk_field_encode(dk_ctx* ctx, const dk_problem* p, uint32_t prime, const uint32_t* xq,
+                          const uint32_t* rq, const uint32_t* C_host, uint32_t* xbar, void* stream) {
+  if (!ctx || !xq || !rq || !C_host || !xbar) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  Modulus md;
+  s = make_modulus(prime, &md);
+  if (s != DK_OK) return s;
+  Guard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FieldCoef fc;
+  s = upload_field_coefficients(ctx, g, prime, C_host, nullptr, false, false, st, &fc);
+  if (s != DK_OK) return s;
+  ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
+  return mix_rows(g.K + 1, xq, rq, fc.enc, xbar, g.n_in, g.E, g.G, md, ctx->sm_count, st);
+}
+
+dk_status dk_field_linear_fwd(dk_ctx* ctx, const dk_problem* p, uint32_t prime, const uint32_t* Wq,
+                              const uint32_t* xbar, uint32_t* ybar, void* stream) {
+  if (!ctx || !Wq || !xbar || !ybar) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  Modulus md;
+  s = make_modulus(prime, &md);
+  if (s != DK_OK) return s;
+  Guard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
+  return launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, st);
+}
+
+dk_status dk_field_decode_verify(dk_ctx* ctx, const dk_problem* p, uint32_t prime, int32_t l,
+                                 const uint32_t* ybar, const uint32_t* C_host, const uint32_t* bias_q,
+                                 int32_t* yq, float* y, dk_verdict* verdict, void* stream) {
+  if (!ctx || !ybar || !C_host || !verdict || (!yq && !y) || l < 0 || l > 30) return DK_ERR_INVALID_ARG;
+  if (!aligned16(verdict)) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  Modulus md;
+  s = make_modulus(prime, &md);
+  if (s != DK_OK) return s;
+  Guard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FieldCoef fc;
+  s = upload_field_coefficients(ctx, g, prime, C_host, nullptr, true, false, st, &fc);
+  if (s != DK_OK) return s;
+  return decode_verify_launch(ctx, g, l, ybar, fc, bias_q, yq, y, verdict, md, st);
+}
+
+dk_status dk_field_masked_linear(dk_ctx* ctx, const dk_problem* p, uint32_t prime, int32_t l, const float* W,
+                                 const float* x, const uint32_t* rq, const uint32_t* C_host, const float* bias,
+                                 float* y, int32_t* yq, uint32_t* xbar_save, dk_verdict* verdict,
+                                 const dk_field_fault* fault, void* stream) {
+  if (!ctx || !W || !x || !rq || !C_host || !verdict || (!yq && !y) || l < 0 || l > 30) return DK_ERR_INVALID_ARG;
+  if (!aligned16(verdict)) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  Modulus md;
+  s = make_modulus(prime, &md);
+  if (s != DK_OK) return s;
+  if (fault) {
+    if (fault->group < 0 || fault->group >= g.G || fault->enc < 0 || fault->enc >= g.E ||
+        fault->out_index < 0 || fault->out_index >= g.n_out)
+      return DK_ERR_INVALID_ARG;
+  }
+  const FieldWs wp = plan_field_ws(g);
+  if (!ctx->ws || ctx->ws_bytes < wp.total) return DK_ERR_WORKSPACE;
+  Guard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FieldCoef fc;
+  s = upload_field_coefficients(ctx, g, prime, C_host, nullptr, true, false, st, &fc);
+  if (s != DK_OK) return s;
+  char* ws = static_cast<char*>(ctx->ws);
+  u32* Wq = reinterpret_cast<u32*>(ws + wp.wq);
+  u32* xq = reinterpret_cast<u32*>(ws + wp.xq);
+  u32* xbar = xbar_save ? xbar_save : reinterpret_cast<u32*>(ws + wp.xbar);
+  u32* ybar = reinterpret_cast<u32*>(ws + wp.ybar);
+  u32* bq = bias ? reinterpret_cast<u32*>(ws + wp.bq) : nullptr;
+  {
+    // Algorithm 1: W_q = Field(Round(W*2^l)), X_q likewise, b_q with 2l bits
+    ProfScope ps(ctx, DK_KERNEL_OTHER, bias ? 3 : 2, st);
+    s = quantize_launch(W, (long long)g.cout * g.kc, l, prime, Wq, ctx->sm_count, st);
+    if (s == DK_OK) s = quantize_launch(x, (long long)g.G * g.K * g.n_in, l, prime, xq, ctx->sm_count, st);
+    if (s == DK_OK && bias) s = quantize_launch(bias, g.cout, 2 * l, prime, bq, ctx->sm_count, st);
+  }
+  if (s != DK_OK) return s;
+  {
+    ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
+    s = mix_rows(g.K + 1, xq, rq, fc.enc, xbar, g.n_in, g.E, g.G, md, ctx->sm_count, st);
+  }
+  if (s != DK_OK) return s;
+  {
+    ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
+    s = launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, st);
+  }
+  if (s != DK_OK) return s;
+  if (fault) {
+    ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+    field_add_fault_kernel<<<1, 1, 0, st>>>(ybar, ((long long)fault->group * g.E + fault->enc) * g.n_out +
+                                                      fault->out_index, fault->delta % prime, prime);
+    DK_CUDA_CHECK(cudaGetLastError());
+  }
+  return decode_verify_launch(ctx, g, l, ybar, fc, bq, yq, y, verdict, md, st);
+}
+
+dk_status dk_field_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, uint32_t prime, const uint32_t* deltaq,
+                                    const uint32_t* xbar, int32_t xbar_rows, const uint32_t* C_host,
+                                    const uint32_t* gamma_host, uint32_t* dWq, void* stream) {
+  if (!ctx || !deltaq || !xbar || !C_host || !gamma_host || !dWq) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  if (xbar_rows != g.K + 1 && xbar_rows != g.K + 2) return DK_ERR_INVALID_ARG;
+  Modulus md;
+  s = make_modulus(prime, &md);
+  if (s != DK_OK) return s;
+  const FieldWs wp = plan_field_ws(g);
+  if (!ctx->ws || ctx->ws_bytes < wp.total) return DK_ERR_WORKSPACE;
+  Guard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FieldCoef fc;
+  s = upload_field_coefficients(ctx, g, prime, C_host, gamma_host, true, true, st, &fc);
+  if (s != DK_OK) return s;
+  char* ws = static_cast<char*>(ctx->ws);
+  u32* dtil = reinterpret_cast<u32*>(ws + wp.dtil);
+  u64* acc = reinterpret_cast<u64*>(ws + wp.acc64);
+  {
+    // Eq. 4: delta_bar^(j) = sum_i B[j][i] delta^(i), with gamma_j folded in
+    ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
+    s = mix_rows(g.K, deltaq, nullptr, fc.mix, dtil, g.n_out, g.K + 1, g.G, md, ctx->sm_count, st);
+  }
+  if (s != DK_OK) return s;
+  WgParams wg;
+  wg.d = dtil; wg.x = xbar; wg.acc = acc;
+  wg.cin = g.cin; wg.cout = g.cout; wg.h = g.h; wg.w = g.w; wg.kw = g.kw; wg.stride = g.stride;
+  wg.pad = g.pad; wg.ho = g.ho; wg.wo = g.wo; wg.kc = g.kc;
+  wg.K1 = g.K + 1; wg.xbar_rows = xbar_rows;
+  wg.P = g.ho * g.wo;
+  wg.PC = (wg.P + BK - 1) / BK;
+  wg.GP = (long long)g.G * wg.PC;
+  wg.n_in = g.n_in; wg.n_out = g.n_out;
+  wg.xs_c = g.xs_c; wg.xs_h = g.xs_h; wg.xs_w = g.xs_w;
+  wg.ws_o = g.ws_o; wg.ws_c = g.ws_c; wg.ws_u = g.ws_u; wg.ws_v = g.ws_v;
+  wg.ys_c = g.ys_c; wg.ys_h = g.ys_h; wg.ys_w = g.ys_w;
+  wg.md = md;
+  long long fb = terms_per_reduction(prime) / ((long long)BK * wg.K1);
+  if (fb < 1) return DK_ERR_UNSUPPORTED;
+  if (fb > 64) fb = 64;
+  wg.fold_blocks = (int)fb;
+  const long long tiles = (long long)((g.cout + BM - 1) / BM) * ((g.kc + BN - 1) / BN);
+  long long splits = (4LL * ctx->sm_count + tiles - 1) / tiles;
+  if (splits > wg.GP) splits = wg.GP;
+  if (splits > 65535) splits = 65535;
+  if (splits < 1) splits = 1;
+  wg.per_split = (wg.GP + splits - 1) / splits;
+  splits = (wg.GP + wg.per_split - 1) / wg.per_split;
+  const long long n_dw = (long long)g.cout * g.kc;
+  dim3 grid((unsigned)((g.kc + BN - 1) / BN), (unsigned)((g.cout + BM - 1) / BM), (unsigned)splits);
+  if (grid.y > 65535) return DK_ERR_SHAPE;
+  {
+    ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
+    DK_CUDA_CHECK(cudaMemsetAsync(acc, 0, (size_t)n_dw * sizeof(u64), st));
+    field_wgrad_kernel<<<grid, NT, 0, st>>>(wg);
+    DK_CUDA_CHECK(cudaGetLastError());
+  }
+  ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+  field_reduce_kernel<<<ew_blocks(n_dw, ctx->sm_count), 256, 0, st>>>(acc, n_dw, md, dWq);
+  DK_CUDA_CHECK(cudaGetLastError());
+  return DK_OK;
+}
+
+}  // extern "C"
