@@ -4,6 +4,7 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--workload vgg16_cifar] [--no-cpu-baseline]
     python bench.py --layer-table [--workload vgg16_224] [--layers conv3_2,conv4_2]
+    python bench.py --field-table [--workload vgg16_cifar] [--layers conv3_2,conv4_2]
 
 One step = one pass of the whole path over one synthetic batch of the
 workload: for every layer the fused masked forward (encode, dense op on the
@@ -16,6 +17,10 @@ of the same workload (one virtual batch of every layer per step).
 `--layer-table` times every layer of a workload on its own (forward call and
 wgrad call, CUDA events around the C-ABI call) and prints one JSON line with
 the per-layer table; it is a reporting aid, not the step metric.
+
+`--field-table` does the same for the finite-field calls (Section 5 of the
+paper: residues modulo p = 2^25 - 39), in exact modular multiply-accumulates
+per second against the integer-ALU peak.
 
 With N > 1 (under torchrun) every rank runs an independent replica of the
 workload on its own GPU: the path has no exchange step, nothing is sharded.
@@ -327,6 +332,129 @@ def run_layer_table(args):
                       "rows": rows}), flush=True)
 
 
+P_FIELD, L_FIELD = 2 ** 25 - 39, 8     # the prime and the fractional bits the paper uses (Section 5)
+# Integer multiply-add lanes: 64 per SM and clock (32-bit IMAD).  One exact multiply-accumulate of two
+# 25-bit residues is a 32x32->64-bit multiply with a 64-bit add, i.e. two passes of the 32-bit multiplier.
+INT_LANES_PER_SM, SMS, IMAD_PER_FIELD_MAC = 64, 148, 2
+
+
+def run_field_table(args):
+    """Per-layer timing of the finite-field calls (dk_field_masked_linear, dk_field_linear_bwd_wgrad) and of
+    the standalone field encode / decode_verify, in exact modular multiply-accumulates per second against the
+    integer-ALU peak; a reporting aid like --layer-table."""
+    import torch
+    from paper_2207_00083_b200 import binding as dk
+    from paper_2207_00083_b200 import synth
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(0)
+    peaks = read_peaks()
+    ctx = dk.Context(0)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(220700083)
+    flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)
+    want = set(args.layers.split(",")) if args.layers else None
+    sampler = ClockSampler(0)
+    sampler.start()
+    rows = []
+
+    def residues(shape):
+        return torch.randint(0, P_FIELD, shape, dtype=torch.int32, device=dev, generator=gen)
+
+    def timeit(fn, iters):
+        for _ in range(2):
+            fn()
+        tot = 0.0
+        for _ in range(iters):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            tot += a.elapsed_time(b)
+        return tot / iters
+
+    for s in synth.layers(args.workload):
+        if want and s.name not in want:
+            continue
+        p = dk.problem_from_spec(s)
+        ctx.ensure_workspace(p, field=True)
+        rng = synth._rng(s, "coef", 7)
+        C = rng.integers(1, P_FIELD, size=(s.G, s.K + 2, s.K + 1)).astype(np.uint32)
+        gamma = rng.integers(1, P_FIELD, size=(s.G, s.K + 1)).astype(np.uint32)
+        x = torch.empty(shape_acts(s.batch, s, "in"), device=dev)
+        x.uniform_(0, 1, generator=gen) if s.x_dist == "uniform" else x.normal_(0, 1, generator=gen)
+        W = torch.randn(shape_w(s), device=dev, generator=gen) * (s.w_std or (2.0 / s.kc) ** 0.5)
+        rq = residues(shape_acts(s.G, s, "in"))
+        y = torch.empty(shape_acts(s.batch, s, "out"), device=dev)
+        xsave = torch.empty(shape_acts(s.G * (s.K + 2), s, "in"), dtype=torch.int32, device=dev)
+        v = dk.new_verdict(0)
+
+        def fwd():
+            dk.dk_field_masked_linear(ctx, p, P_FIELD, L_FIELD, W, x, rq, C, None, y, None, xsave, v)
+        row = {"layer": s.name, "M": s.cout, "Kc": s.kc, "N_fwd": s.G * (s.K + 2) * s.hout * s.wout}
+        calls = [("fwd", fwd, s.fwd_flops() / 2, "linear_fwd")]
+        if s.wgrad:
+            dq = residues(shape_acts(s.batch, s, "out"))
+            dWq = torch.empty(shape_w(s), dtype=torch.int32, device=dev)
+
+            def wg():
+                dk.dk_field_linear_bwd_wgrad(ctx, p, P_FIELD, dq, xsave, s.K + 2, C, gamma, dWq)
+            calls.append(("wgrad", wg, s.wgrad_flops() / 2, "wgrad"))
+        for name, fn, macs, kind in calls:
+            fn()
+            dk.dk_profile_reset(ctx)
+            dk.dk_profile_enable(ctx, True)
+            ms = timeit(fn, args.iters)
+            prof = dk.dk_profile_read(ctx)
+            dk.dk_profile_enable(ctx, False)
+            kms = prof[kind][0] / max(prof[kind][1], 1)
+            row[name] = {"call_ms": round(ms, 4), "kernel_ms": round(kms, 4),
+                         "tmacs_call": round(macs / ms / 1e9, 3), "tmacs_kernel": round(macs / kms / 1e9, 3)}
+        vd = dk.read_verdict(v)
+        row["verdict_ok"] = vd["ok"]
+        rows.append(row)
+        torch.cuda.empty_cache()
+
+    # standalone field encode / decode_verify on tensors much larger than L2 (uint32 residues: the same
+    # bytes per position as the fp32 calls)
+    K, G, n = 4, 32, 1 << 20
+    spec = synth.LayerSpec("elementwise", "stream", "fc", n, n, K=K, G=G)
+    p = dk.problem_from_spec(spec)
+    C = np.random.default_rng(7).integers(1, P_FIELD, size=(G, K + 2, K + 1)).astype(np.uint32)
+    xq, rq = residues((G * K, n)), residues((G, n))
+    xbar = torch.empty((G * (K + 2), n), dtype=torch.int32, device=dev)
+    yq = torch.empty((G * K, n), dtype=torch.int32, device=dev)
+    v = dk.new_verdict(0)
+    elem = {}
+    for name, fn, bpp in (("encode", lambda: dk.dk_field_encode(ctx, p, P_FIELD, xq, rq, C, xbar), (2 * K + 3) * 4),
+                          ("decode", lambda: dk.dk_field_decode_verify(ctx, p, P_FIELD, L_FIELD, xbar, C, None, yq,
+                                                                       None, v), (2 * K + 2) * 4)):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(10):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / 10
+        gbs = bpp * G * n / (ms * 1e-3) / 1e9
+        elem[name] = {"gbs": round(gbs, 1), "frac_hbm": round(gbs / peaks["hbm_gbs"], 4), "ms": round(ms, 4)}
+    assert dk.read_verdict(v)["ok"] == 1      # decode of encode-only data: rho = n . C . [x; r] = 0
+    clocks = sampler.stop()
+    mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+    peak = SMS * INT_LANES_PER_SM * mhz * 1e6 / IMAD_PER_FIELD_MAC / 1e12
+    for row in rows:
+        for name in ("fwd", "wgrad"):
+            if name in row:
+                row[name]["frac_alu_peak_kernel"] = round(row[name]["tmacs_kernel"] / peak, 4)
+    print(json.dumps({"field_table": args.workload, "prime": P_FIELD, "l": L_FIELD, "unit": "T exact modular MAC/s",
+                      "alu_peak_tmacs": round(peak, 3),
+                      "alu_peak_source": f"{SMS} SMs x {INT_LANES_PER_SM} int32 multiply-add lanes x {mhz} MHz / "
+                                         f"{IMAD_PER_FIELD_MAC} multiplier passes per 64-bit multiply-accumulate",
+                      "elementwise": elem, "clocks": clocks, "rows": rows}), flush=True)
+
+
 def max_over_ranks(value, world, device):
     """Device-timed milliseconds of this rank -> the slowest rank's figure (every rank gets it).
     The replicas share nothing, so this and the barriers are the only communication of a multi-GPU run."""
@@ -561,6 +689,7 @@ def main():
     ap.add_argument("--workload", default="vgg16_cifar")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layer-table", action="store_true")
+    ap.add_argument("--field-table", action="store_true")
     ap.add_argument("--layers", default="")
     ap.add_argument("--iters", type=int, default=5)
     args = ap.parse_args()
@@ -568,6 +697,8 @@ def main():
         run_reference(args)
     elif args.layer_table:
         run_layer_table(args)
+    elif args.field_table:
+        run_field_table(args)
     else:
         run_ours(args)
 

@@ -542,10 +542,226 @@ __global__ void __launch_bounds__(NT) field_fwd_kernel(FwdParams p) {
   }
 }
 
+// ---------------------------------------------------------------------------
+// The same contraction on the integer tensor cores.  A residue below 2^32 is
+// four base-256 digits, which are the four bytes of its uint32 as stored, so
+// <W_q, x_bar> = sum_{a,b<4} 2^{8(a+b)} * sum_k Wdigit_a[k] * xdigit_b[k]:
+// sixteen u8 x u8 -> s32 matrix products (mma.sync m16n8k32), accumulated in
+// seven s32 accumulators by weight class a+b and folded modulo p into uint64
+// totals before a class can overflow (255^2 * 4 pairs * 4096 terms < 2^31).
+// The digit planes are formed in registers by a 4x4 byte transpose of four
+// consecutive k-elements; operands sit in shared memory as plain residues.
+// ---------------------------------------------------------------------------
+constexpr int MMA_BM = 64, MMA_BN = 64, MMA_BK = 32;
+constexpr int kMmaFoldTiles = 4096 / MMA_BK;
+constexpr int kMmaStageWords = (MMA_BM + MMA_BN) * MMA_BK;     // one pipeline stage: A tile then B tile
+
+struct RowInfo {        // one output pixel (column of the GEMM) of the block's tile
+  long long base;       // offset of its sample in x, or -1 when past the end
+  int ih0, iw0;
+};
+
+// Word k of row r of a 32-word tile row.  Odd rows swap their two 16-word
+// halves, so that the 16-byte fragment reads of a quarter warp (rows r, r+1,
+// four chunks each) fall into distinct banks.
+__device__ __forceinline__ int tile_word(int r, int k) { return r * MMA_BK + (k ^ ((r & 1) << 4)); }
+
+// Asynchronous global -> shared copy of BYTES (4 or 16); `valid` false writes zeros and reads nothing.
+template <int BYTES>
+__device__ __forceinline__ void copy_async(u32* smem_dst, const u32* gsrc, bool valid) {
+  const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+  const int n = valid ? BYTES : 0;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;\n" ::"r"(d), "l"(gsrc), "n"(BYTES), "r"(n));
+}
+__device__ __forceinline__ void copy_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void copy_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+__device__ __forceinline__ void digit_planes(const uint4 w, u32 (&pl)[4]) {
+  const u32 t0 = __byte_perm(w.x, w.y, 0x5140), t1 = __byte_perm(w.z, w.w, 0x5140);
+  const u32 u0 = __byte_perm(w.x, w.y, 0x7362), u1 = __byte_perm(w.z, w.w, 0x7362);
+  pl[0] = __byte_perm(t0, t1, 0x5410);
+  pl[1] = __byte_perm(t0, t1, 0x7632);
+  pl[2] = __byte_perm(u0, u1, 0x5410);
+  pl[3] = __byte_perm(u0, u1, 0x7632);
+}
+
+__device__ __forceinline__ void mma_u8(int (&d)[4], const u32 a0, const u32 a1, const u32 a2, const u32 a3,
+                                       const u32 b0, const u32 b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+struct MmaConsts {
+  u32 pow32;   // 2^32 mod p
+};
+
+// total = (total + sum_c acc_c * 2^{8c}) mod p for the seven class sums of one output element
+__device__ __forceinline__ u32 fold_classes(u32 total, const int (&c)[7], Modulus md, u32 pow32) {
+  const u64 lo = (u64)(u32)c[0] + ((u64)(u32)c[1] << 8) + ((u64)(u32)c[2] << 16) + ((u64)(u32)c[3] << 24);
+  const u64 hi = (u64)(u32)c[4] + ((u64)(u32)c[5] << 8) + ((u64)(u32)c[6] << 16);     // weight 2^32
+  const u64 t = (u64)total + reduce64(lo, md) + (u64)reduce64(hi, md) * pow32;
+  return reduce64(t, md);
+}
+
+// VEC = 4: channels are contiguous in W and x and cin % 4 == 0, so four
+// consecutive k-elements are 16 contiguous bytes of one filter tap; VEC = 1:
+// every geometry and layout, one element per copy.
+template <int VEC>
+__global__ void __launch_bounds__(256, 1) field_fwd_mma_kernel(FwdParams p, MmaConsts mc) {
+  __shared__ __align__(16) u32 tiles[2 * kMmaStageWords];
+  __shared__ RowInfo rows[MMA_BN];
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int g = lane >> 2, tig = lane & 3;
+  const int wm = warp & 3, wn = warp >> 2;          // warp tile: rows 16*wm.., columns 32*wn..
+  const int m0 = blockIdx.y * MMA_BM;
+  const long long n0 = (long long)blockIdx.x * MMA_BN;
+
+  if (t < MMA_BN) {
+    const long long n = n0 + t;
+    RowInfo ri;
+    if (n < p.N) {
+      const int ow = (int)(n % p.wo);
+      const long long r = n / p.wo;
+      const int oh = (int)(r % p.ho);
+      ri.base = (r / p.ho) * p.n_in;
+      ri.ih0 = oh * p.stride - p.pad;
+      ri.iw0 = ow * p.stride - p.pad;
+    } else {
+      ri.base = -1; ri.ih0 = 0; ri.iw0 = 0;
+    }
+    rows[t] = ri;
+  }
+  __syncthreads();
+
+  // loader: a thread copies elements k = kq .. kq+VEC-1 of rows r0 + RSTEP*i of both tiles
+  constexpr int CPR = MMA_BK / VEC;              // copies per tile row
+  constexpr int RSTEP = 256 / CPR, NCOPY = MMA_BM / RSTEP;
+  const int kq = (t % CPR) * VEC, r0 = t / CPR;
+  auto load_tile = [&](int k0, u32* stage) {
+    const int k = k0 + kq;
+    const bool kok = k < p.kc;
+    const int tap = kok ? k / p.cin : 0;
+    const int ci = kok ? k - tap * p.cin : 0;
+    const int u = tap / p.kw, v = tap - u * p.kw;
+    const long long woff = (long long)ci * p.ws_c + (long long)u * p.ws_u + (long long)v * p.ws_v;
+    const long long xoff = (long long)ci * p.xs_c;
+    u32* as = stage;
+    u32* bs = stage + MMA_BM * MMA_BK;
+#pragma unroll
+    for (int i = 0; i < NCOPY; ++i) {
+      const int mm = r0 + RSTEP * i;
+      const bool aok = kok && (m0 + mm) < p.cout;
+      copy_async<4 * VEC>(as + tile_word(mm, kq), aok ? p.W + (long long)(m0 + mm) * p.ws_o + woff : p.W, aok);
+      const RowInfo ri = rows[mm];
+      const int ih = ri.ih0 + u, iw = ri.iw0 + v;
+      const bool ok = kok && ri.base >= 0 && ih >= 0 && ih < p.h && iw >= 0 && iw < p.w;
+      copy_async<4 * VEC>(bs + tile_word(mm, kq),
+                          ok ? p.x + ri.base + xoff + (long long)ih * p.xs_h + (long long)iw * p.xs_w : p.x, ok);
+    }
+    copy_async_commit();
+  };
+
+  int acc[7][4][4];       // [weight class][n-tile][fragment register]
+  u32 tot[4][4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      tot[j][r] = 0;
+#pragma unroll
+      for (int c = 0; c < 7; ++c) acc[c][j][r] = 0;
+    }
+
+  const int ntiles = (p.kc + MMA_BK - 1) / MMA_BK;
+  load_tile(0, tiles);
+  int fold = 0;
+  for (int kt = 0; kt < ntiles; ++kt) {
+    u32* stage = tiles + (kt & 1) * kMmaStageWords;
+    if (kt + 1 < ntiles) {
+      load_tile((kt + 1) * MMA_BK, tiles + ((kt + 1) & 1) * kMmaStageWords);
+      copy_async_wait<1>();
+    } else {
+      copy_async_wait<0>();
+    }
+    __syncthreads();
+    {
+      const u32* as = stage;
+      const u32* bs = stage + MMA_BM * MMA_BK;
+      u32 a[4][4];       // [fragment register][digit]
+      const int ra = wm * 16 + g;      // rows ra and ra + 8 have the same parity
+      digit_planes(*reinterpret_cast<const uint4*>(as + tile_word(ra, 4 * tig)), a[0]);
+      digit_planes(*reinterpret_cast<const uint4*>(as + tile_word(ra + 8, 4 * tig)), a[1]);
+      digit_planes(*reinterpret_cast<const uint4*>(as + tile_word(ra, 16 + 4 * tig)), a[2]);
+      digit_planes(*reinterpret_cast<const uint4*>(as + tile_word(ra + 8, 16 + 4 * tig)), a[3]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        u32 b[2][4];
+        const int rb = wn * 32 + j * 8 + g;
+        digit_planes(*reinterpret_cast<const uint4*>(bs + tile_word(rb, 4 * tig)), b[0]);
+        digit_planes(*reinterpret_cast<const uint4*>(bs + tile_word(rb, 16 + 4 * tig)), b[1]);
+#pragma unroll
+        for (int da = 0; da < 4; ++da)
+#pragma unroll
+          for (int db = 0; db < 4; ++db)
+            mma_u8(acc[da + db][j], a[0][da], a[1][da], a[2][da], a[3][da], b[0][db], b[1][db]);
+      }
+    }
+    __syncthreads();
+    if (++fold == kMmaFoldTiles) {
+      fold = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const int c[7] = {acc[0][j][r], acc[1][j][r], acc[2][j][r], acc[3][j][r],
+                            acc[4][j][r], acc[5][j][r], acc[6][j][r]};
+          tot[j][r] = fold_classes(tot[j][r], c, p.md, mc.pow32);
+#pragma unroll
+          for (int cc = 0; cc < 7; ++cc) acc[cc][j][r] = 0;
+        }
+    }
+  }
+  // fragment register r of n-tile j: row g + 8*(r >> 1), column 2*tig + (r & 1)
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int cb = 0; cb < 2; ++cb) {
+      const long long n = n0 + wn * 32 + j * 8 + 2 * tig + cb;
+      if (n >= p.N) continue;
+      const int ow = (int)(n % p.wo);
+      const long long rr = n / p.wo;
+      const int oh = (int)(rr % p.ho);
+      u32* yo = p.y + (rr / p.ho) * p.n_out + (long long)oh * p.ys_h + (long long)ow * p.ys_w;
+#pragma unroll
+      for (int rb = 0; rb < 2; ++rb) {
+        const int r = rb * 2 + cb;
+        const int m = m0 + wm * 16 + g + 8 * rb;
+        if (m >= p.cout) continue;
+        const int c[7] = {acc[0][j][r], acc[1][j][r], acc[2][j][r], acc[3][j][r],
+                          acc[4][j][r], acc[5][j][r], acc[6][j][r]};
+        yo[(long long)m * p.ys_c] = fold_classes(tot[j][r], c, p.md, mc.pow32);
+      }
+    }
+}
+
 // How many products of two residues may be added to one residue in a uint64.
 long long terms_per_reduction(u32 p) {
   const u64 pm = (u64)p - 1;
   return (long long)((~0ull - pm) / (pm * pm));
+}
+
+bool aligned16(const void* p);
+
+// DK_FIELD_SIMT=1 selects the 64-bit integer-ALU kernel instead of the tensor-core one (a cross-check).
+bool field_use_simt() {
+  static const bool v = [] {
+    const char* e = getenv("DK_FIELD_SIMT");
+    return e && e[0] == '1';
+  }();
+  return v;
 }
 
 dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* ybar, int nsamples, Modulus md,
@@ -568,7 +784,16 @@ dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* yb
   if (nb > 2147483647LL) return DK_ERR_SHAPE;
   dim3 grid((unsigned)nb, (unsigned)((g.cout + BM - 1) / BM));
   if (grid.y > 65535) return DK_ERR_SHAPE;
-  field_fwd_kernel<<<grid, NT, 0, st>>>(p);
+  static_assert(BM == MMA_BM && BN == MMA_BN, "one grid shape serves both kernels");
+  if (field_use_simt()) {
+    field_fwd_kernel<<<grid, NT, 0, st>>>(p);
+  } else {
+    MmaConsts mc;
+    mc.pow32 = (u32)((1ull << 32) % md.p);
+    const bool vec4 = g.xs_c == 1 && g.ws_c == 1 && (g.cin % 4) == 0 && aligned16(W) && aligned16(xbar);
+    if (vec4) field_fwd_mma_kernel<4><<<grid, 256, 0, st>>>(p, mc);
+    else field_fwd_mma_kernel<1><<<grid, 256, 0, st>>>(p, mc);
+  }
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
 }
