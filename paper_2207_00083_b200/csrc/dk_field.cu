@@ -555,6 +555,8 @@ __global__ void __launch_bounds__(NT) field_fwd_kernel(FwdParams p) {
 constexpr int MMA_BM = 64, MMA_BN = 64, MMA_BK = 32;
 constexpr int kMmaFoldTiles = 4096 / MMA_BK;
 constexpr int kMmaStageWords = (MMA_BM + MMA_BN) * MMA_BK;     // one pipeline stage: A tile then B tile
+constexpr int kMmaStages = 4;
+constexpr size_t kMmaSmemBytes = (size_t)kMmaStages * kMmaStageWords * sizeof(u32);
 
 struct RowInfo {        // one output pixel (column of the GEMM) of the block's tile
   long long base;       // offset of its sample in x, or -1 when past the end
@@ -611,7 +613,7 @@ __device__ __forceinline__ u32 fold_classes(u32 total, const int (&c)[7], Modulu
 // every geometry and layout, one element per copy.
 template <int VEC>
 __global__ void __launch_bounds__(256, 1) field_fwd_mma_kernel(FwdParams p, MmaConsts mc) {
-  __shared__ __align__(16) u32 tiles[2 * kMmaStageWords];
+  extern __shared__ __align__(16) u32 tiles[];      // kMmaStages pipeline stages
   __shared__ RowInfo rows[MMA_BN];
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   const int g = lane >> 2, tig = lane & 3;
@@ -675,18 +677,27 @@ __global__ void __launch_bounds__(256, 1) field_fwd_mma_kernel(FwdParams p, MmaC
       for (int c = 0; c < 7; ++c) acc[c][j][r] = 0;
     }
 
+  // Multi-stage pipeline with one barrier per k-tile: tiles kt+1 .. kt+S-2 are in
+  // flight while tile kt is multiplied; the stage refilled in iteration kt is the
+  // one every warp finished reading before it arrived at this iteration's barrier.
+  // (A group is committed every iteration, empty past the end, so that
+  // "all but the newest S-2 groups" always means "tile kt has landed".)
   const int ntiles = (p.kc + MMA_BK - 1) / MMA_BK;
-  load_tile(0, tiles);
+#pragma unroll
+  for (int s = 0; s < kMmaStages - 1; ++s) {
+    if (s < ntiles) load_tile(s * MMA_BK, tiles + s * kMmaStageWords);
+    else copy_async_commit();
+  }
   int fold = 0;
   for (int kt = 0; kt < ntiles; ++kt) {
-    u32* stage = tiles + (kt & 1) * kMmaStageWords;
-    if (kt + 1 < ntiles) {
-      load_tile((kt + 1) * MMA_BK, tiles + ((kt + 1) & 1) * kMmaStageWords);
-      copy_async_wait<1>();
-    } else {
-      copy_async_wait<0>();
-    }
+    u32* stage = tiles + (kt % kMmaStages) * kMmaStageWords;
+    copy_async_wait<kMmaStages - 2>();
     __syncthreads();
+    {
+      const int nt = kt + kMmaStages - 1;
+      if (nt < ntiles) load_tile(nt * MMA_BK, tiles + (nt % kMmaStages) * kMmaStageWords);
+      else copy_async_commit();
+    }
     {
       const u32* as = stage;
       const u32* bs = stage + MMA_BM * MMA_BK;
@@ -709,7 +720,6 @@ __global__ void __launch_bounds__(256, 1) field_fwd_mma_kernel(FwdParams p, MmaC
             mma_u8(acc[da + db][j], a[0][da], a[1][da], a[2][da], a[3][da], b[0][db], b[1][db]);
       }
     }
-    __syncthreads();
     if (++fold == kMmaFoldTiles) {
       fold = 0;
 #pragma unroll
@@ -791,8 +801,15 @@ dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* yb
     MmaConsts mc;
     mc.pow32 = (u32)((1ull << 32) % md.p);
     const bool vec4 = g.xs_c == 1 && g.ws_c == 1 && (g.cin % 4) == 0 && aligned16(W) && aligned16(xbar);
-    if (vec4) field_fwd_mma_kernel<4><<<grid, 256, 0, st>>>(p, mc);
-    else field_fwd_mma_kernel<1><<<grid, 256, 0, st>>>(p, mc);
+    static const bool attr_ok = [] {
+      return cudaFuncSetAttribute(field_fwd_mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)kMmaSmemBytes) == cudaSuccess &&
+             cudaFuncSetAttribute(field_fwd_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)kMmaSmemBytes) == cudaSuccess;
+    }();
+    if (!attr_ok) return DK_ERR_CUDA;
+    if (vec4) field_fwd_mma_kernel<4><<<grid, 256, kMmaSmemBytes, st>>>(p, mc);
+    else field_fwd_mma_kernel<1><<<grid, 256, kMmaSmemBytes, st>>>(p, mc);
   }
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
@@ -905,6 +922,182 @@ __global__ void __launch_bounds__(NT) field_wgrad_kernel(WgParams p) {
       if (m < p.cout) atomicAdd(p.acc + (long long)m * p.ws_o + woff, (u64)reduce64(acc[i][jj], p.md));
     }
   }
+}
+
+// The weight-gradient contraction on the integer tensor cores.  The contraction
+// index r runs over (group, encoding, output pixel) flattened; both operands are
+// stored with the channel contiguous, so a tile is kept in shared memory as it
+// arrives, [r][column], and a thread gathers the four consecutive r of one
+// column with four 32-bit reads (row pitch == 2 mod 32 words: conflict-free)
+// before the same byte transpose into digit planes as in the forward kernel.
+constexpr int WG_LD = MMA_BM + 2;
+constexpr int kWgStageWords = 2 * MMA_BK * WG_LD;
+constexpr size_t kWgSmemBytes = (size_t)kMmaStages * kWgStageWords * sizeof(u32);
+
+// n / d for 0 <= n < 2^32 by multiplication (Granlund-Montgomery round-up
+// method): s = ceil(log2 d), m = floor(2^32 (2^s - d) / d) + 1, q = (mulhi(n, m) + n) >> s.
+struct FastDiv {
+  u32 m;
+  int s;
+};
+FastDiv make_fastdiv(u32 d) {
+  FastDiv f;
+  f.s = 0;
+  while ((1ull << f.s) < d) ++f.s;
+  f.m = (u32)((((1ull << f.s) - d) << 32) / d + 1);
+  return f;
+}
+__device__ __forceinline__ u32 fastdiv(u32 n, FastDiv f) { return (u32)(((u64)__umulhi(n, f.m) + n) >> f.s); }
+
+struct WgMmaParams {
+  FastDiv div_P, div_K1, div_wo;
+  const u32* d;     // mixed deltas [G*(K+1)][n_out]
+  const u32* x;     // encodings, xbar_rows per group
+  u64* acc;         // [cout*kc] sums of the slices' residues, cleared by the caller
+  int cin, cout, h, w, kw, stride, pad, ho, wo, kc;
+  int K1, xbar_rows, P;
+  long long R;                // G * (K+1) * P contraction elements
+  int tiles_per_split, ntiles;
+  long long n_in, n_out;
+  long long xs_c, xs_h, xs_w, ws_o, ws_c, ws_u, ws_v, ys_c, ys_h, ys_w;
+  Modulus md;
+  u32 pow32;
+};
+
+__device__ __forceinline__ uint4 gather4(const u32* col) {
+  return make_uint4(col[0], col[WG_LD], col[2 * WG_LD], col[3 * WG_LD]);
+}
+
+template <int VEC>
+__global__ void __launch_bounds__(256, 1) field_wgrad_mma_kernel(WgMmaParams p) {
+  extern __shared__ __align__(16) u32 tiles[];
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int g = lane >> 2, tig = lane & 3;
+  const int wm = warp & 3, wn = warp >> 2;
+  const int m0 = blockIdx.y * MMA_BM;
+  const int kb0 = blockIdx.x * MMA_BN;
+  const int t_lo = blockIdx.z * p.tiles_per_split;
+  const int t_hi = min(t_lo + p.tiles_per_split, p.ntiles);
+
+  // loader: VEC columns starting at `col` of the r-rows rr0 + RSTEP*i of both tiles
+  constexpr int CPR = MMA_BM / VEC, RSTEP = 256 / CPR, NCOPY = MMA_BK / RSTEP;
+  const int col = (t % CPR) * VEC, rr0 = t / CPR;
+  const bool a_ok = (m0 + col) < p.cout;
+  const long long a_off = (long long)(m0 + col) * p.ys_c;
+  const int kcol = kb0 + col;
+  const bool b_ok = kcol < p.kc;
+  const int tap = b_ok ? kcol / p.cin : 0;
+  const int ci = b_ok ? kcol - tap * p.cin : 0;
+  const int u = tap / p.kw, v = tap - u * p.kw;
+  const long long b_off = (long long)ci * p.xs_c;
+  auto load_tile = [&](int rt, u32* stage) {
+    u32* as = stage;
+    u32* bs = stage + MMA_BK * WG_LD;
+#pragma unroll
+    for (int i = 0; i < NCOPY; ++i) {
+      const int rr = rr0 + RSTEP * i;
+      const u32 r = (u32)rt * MMA_BK + rr;
+      const bool rok = r < (u32)p.R;
+      const u32 gj = rok ? fastdiv(r, p.div_P) : 0;
+      const int pix = rok ? (int)(r - gj * p.P) : 0;
+      const long long gg = fastdiv(gj, p.div_K1);
+      const int j = (int)(gj - (u32)gg * p.K1);
+      const int oh = (int)fastdiv((u32)pix, p.div_wo), ow = pix - oh * p.wo;
+      const bool aok = rok && a_ok;
+      copy_async<4 * VEC>(as + rr * WG_LD + col,
+                          aok ? p.d + (gg * p.K1 + j) * p.n_out + a_off + (long long)oh * p.ys_h + (long long)ow * p.ys_w
+                              : p.d, aok);
+      const int ih = oh * p.stride + u - p.pad, iw = ow * p.stride + v - p.pad;
+      const bool bok = rok && b_ok && ih >= 0 && ih < p.h && iw >= 0 && iw < p.w;
+      copy_async<4 * VEC>(bs + rr * WG_LD + col,
+                          bok ? p.x + (gg * p.xbar_rows + j) * p.n_in + b_off + (long long)ih * p.xs_h +
+                                    (long long)iw * p.xs_w
+                              : p.x, bok);
+    }
+    copy_async_commit();
+  };
+
+  int acc[7][4][4];
+  u32 tot[4][4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      tot[j][r] = 0;
+#pragma unroll
+      for (int c = 0; c < 7; ++c) acc[c][j][r] = 0;
+    }
+
+  const int ntiles = t_hi - t_lo;
+#pragma unroll
+  for (int s = 0; s < kMmaStages - 1; ++s) {
+    if (s < ntiles) load_tile(t_lo + s, tiles + s * kWgStageWords);
+    else copy_async_commit();
+  }
+  int fold = 0;
+  for (int kt = 0; kt < ntiles; ++kt) {
+    const u32* as = tiles + (kt % kMmaStages) * kWgStageWords;
+    const u32* bs = as + MMA_BK * WG_LD;
+    copy_async_wait<kMmaStages - 2>();
+    __syncthreads();
+    {
+      const int nt = kt + kMmaStages - 1;
+      if (nt < ntiles) load_tile(t_lo + nt, tiles + (nt % kMmaStages) * kWgStageWords);
+      else copy_async_commit();
+    }
+    {
+      u32 a[4][4];
+      const u32* ac = as + (4 * tig) * WG_LD + wm * 16 + g;
+      digit_planes(gather4(ac), a[0]);
+      digit_planes(gather4(ac + 8), a[1]);
+      digit_planes(gather4(ac + 16 * WG_LD), a[2]);
+      digit_planes(gather4(ac + 16 * WG_LD + 8), a[3]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        u32 b[2][4];
+        const u32* bc = bs + (4 * tig) * WG_LD + wn * 32 + j * 8 + g;
+        digit_planes(gather4(bc), b[0]);
+        digit_planes(gather4(bc + 16 * WG_LD), b[1]);
+#pragma unroll
+        for (int da = 0; da < 4; ++da)
+#pragma unroll
+          for (int db = 0; db < 4; ++db)
+            mma_u8(acc[da + db][j], a[0][da], a[1][da], a[2][da], a[3][da], b[0][db], b[1][db]);
+      }
+    }
+    if (++fold == kMmaFoldTiles) {
+      fold = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const int c[7] = {acc[0][j][r], acc[1][j][r], acc[2][j][r], acc[3][j][r],
+                            acc[4][j][r], acc[5][j][r], acc[6][j][r]};
+          tot[j][r] = fold_classes(tot[j][r], c, p.md, p.pow32);
+#pragma unroll
+          for (int cc = 0; cc < 7; ++cc) acc[cc][j][r] = 0;
+        }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int cb = 0; cb < 2; ++cb) {
+      const int kcol2 = kb0 + wn * 32 + j * 8 + 2 * tig + cb;
+      if (kcol2 >= p.kc) continue;
+      const int tap2 = kcol2 / p.cin, ci2 = kcol2 - tap2 * p.cin;
+      const int u2 = tap2 / p.kw, v2 = tap2 - u2 * p.kw;
+      const long long woff = (long long)ci2 * p.ws_c + (long long)u2 * p.ws_u + (long long)v2 * p.ws_v;
+#pragma unroll
+      for (int rb = 0; rb < 2; ++rb) {
+        const int r = rb * 2 + cb;
+        const int m = m0 + wm * 16 + g + 8 * rb;
+        if (m >= p.cout) continue;
+        const int c[7] = {acc[0][j][r], acc[1][j][r], acc[2][j][r], acc[3][j][r],
+                          acc[4][j][r], acc[5][j][r], acc[6][j][r]};
+        atomicAdd(p.acc + (long long)m * p.ws_o + woff, (u64)fold_classes(tot[j][r], c, p.md, p.pow32));
+      }
+    }
 }
 
 // the slices' residues (at most 65535 of them, each below p) summed in uint64 -> residue
@@ -1179,37 +1372,79 @@ dk_status dk_field_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, uint32_t p
     s = mix_rows(g.K, deltaq, nullptr, fc.mix, dtil, g.n_out, g.K + 1, g.G, md, ctx->sm_count, st);
   }
   if (s != DK_OK) return s;
-  WgParams wg;
-  wg.d = dtil; wg.x = xbar; wg.acc = acc;
-  wg.cin = g.cin; wg.cout = g.cout; wg.h = g.h; wg.w = g.w; wg.kw = g.kw; wg.stride = g.stride;
-  wg.pad = g.pad; wg.ho = g.ho; wg.wo = g.wo; wg.kc = g.kc;
-  wg.K1 = g.K + 1; wg.xbar_rows = xbar_rows;
-  wg.P = g.ho * g.wo;
-  wg.PC = (wg.P + BK - 1) / BK;
-  wg.GP = (long long)g.G * wg.PC;
-  wg.n_in = g.n_in; wg.n_out = g.n_out;
-  wg.xs_c = g.xs_c; wg.xs_h = g.xs_h; wg.xs_w = g.xs_w;
-  wg.ws_o = g.ws_o; wg.ws_c = g.ws_c; wg.ws_u = g.ws_u; wg.ws_v = g.ws_v;
-  wg.ys_c = g.ys_c; wg.ys_h = g.ys_h; wg.ys_w = g.ys_w;
-  wg.md = md;
-  long long fb = terms_per_reduction(prime) / ((long long)BK * wg.K1);
-  if (fb < 1) return DK_ERR_UNSUPPORTED;
-  if (fb > 64) fb = 64;
-  wg.fold_blocks = (int)fb;
-  const long long tiles = (long long)((g.cout + BM - 1) / BM) * ((g.kc + BN - 1) / BN);
-  long long splits = (4LL * ctx->sm_count + tiles - 1) / tiles;
-  if (splits > wg.GP) splits = wg.GP;
-  if (splits > 65535) splits = 65535;
-  if (splits < 1) splits = 1;
-  wg.per_split = (wg.GP + splits - 1) / splits;
-  splits = (wg.GP + wg.per_split - 1) / wg.per_split;
   const long long n_dw = (long long)g.cout * g.kc;
-  dim3 grid((unsigned)((g.kc + BN - 1) / BN), (unsigned)((g.cout + BM - 1) / BM), (unsigned)splits);
-  if (grid.y > 65535) return DK_ERR_SHAPE;
-  {
+  const long long tiles = (long long)((g.cout + BM - 1) / BM) * ((g.kc + BN - 1) / BN);
+  if ((g.cout + BM - 1) / BM > 65535) return DK_ERR_SHAPE;
+  if (field_use_simt()) {
+    WgParams wg;
+    wg.d = dtil; wg.x = xbar; wg.acc = acc;
+    wg.cin = g.cin; wg.cout = g.cout; wg.h = g.h; wg.w = g.w; wg.kw = g.kw; wg.stride = g.stride;
+    wg.pad = g.pad; wg.ho = g.ho; wg.wo = g.wo; wg.kc = g.kc;
+    wg.K1 = g.K + 1; wg.xbar_rows = xbar_rows;
+    wg.P = g.ho * g.wo;
+    wg.PC = (wg.P + BK - 1) / BK;
+    wg.GP = (long long)g.G * wg.PC;
+    wg.n_in = g.n_in; wg.n_out = g.n_out;
+    wg.xs_c = g.xs_c; wg.xs_h = g.xs_h; wg.xs_w = g.xs_w;
+    wg.ws_o = g.ws_o; wg.ws_c = g.ws_c; wg.ws_u = g.ws_u; wg.ws_v = g.ws_v;
+    wg.ys_c = g.ys_c; wg.ys_h = g.ys_h; wg.ys_w = g.ys_w;
+    wg.md = md;
+    long long fb = terms_per_reduction(prime) / ((long long)BK * wg.K1);
+    if (fb < 1) return DK_ERR_UNSUPPORTED;
+    if (fb > 64) fb = 64;
+    wg.fold_blocks = (int)fb;
+    long long splits = (4LL * ctx->sm_count + tiles - 1) / tiles;
+    if (splits > wg.GP) splits = wg.GP;
+    if (splits > 65535) splits = 65535;
+    if (splits < 1) splits = 1;
+    wg.per_split = (wg.GP + splits - 1) / splits;
+    splits = (wg.GP + wg.per_split - 1) / wg.per_split;
+    dim3 grid((unsigned)((g.kc + BN - 1) / BN), (unsigned)((g.cout + BM - 1) / BM), (unsigned)splits);
     ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
     DK_CUDA_CHECK(cudaMemsetAsync(acc, 0, (size_t)n_dw * sizeof(u64), st));
     field_wgrad_kernel<<<grid, NT, 0, st>>>(wg);
+    DK_CUDA_CHECK(cudaGetLastError());
+  } else {
+    WgMmaParams wg;
+    wg.d = dtil; wg.x = xbar; wg.acc = acc;
+    wg.cin = g.cin; wg.cout = g.cout; wg.h = g.h; wg.w = g.w; wg.kw = g.kw; wg.stride = g.stride;
+    wg.pad = g.pad; wg.ho = g.ho; wg.wo = g.wo; wg.kc = g.kc;
+    wg.K1 = g.K + 1; wg.xbar_rows = xbar_rows;
+    wg.P = g.ho * g.wo;
+    wg.R = (long long)g.G * wg.K1 * wg.P;
+    const long long nt = (wg.R + MMA_BK - 1) / MMA_BK;
+    if (wg.R >= (1LL << 31)) return DK_ERR_SHAPE;
+    wg.div_P = make_fastdiv((u32)wg.P);
+    wg.div_K1 = make_fastdiv((u32)wg.K1);
+    wg.div_wo = make_fastdiv((u32)g.wo);
+    wg.ntiles = (int)nt;
+    wg.n_in = g.n_in; wg.n_out = g.n_out;
+    wg.xs_c = g.xs_c; wg.xs_h = g.xs_h; wg.xs_w = g.xs_w;
+    wg.ws_o = g.ws_o; wg.ws_c = g.ws_c; wg.ws_u = g.ws_u; wg.ws_v = g.ws_v;
+    wg.ys_c = g.ys_c; wg.ys_h = g.ys_h; wg.ys_w = g.ys_w;
+    wg.md = md;
+    wg.pow32 = (u32)((1ull << 32) % md.p);
+    // slices of the contraction: about two rounds of blocks on the device, at least 8 tiles each
+    long long splits = (2LL * ctx->sm_count + tiles - 1) / tiles;
+    if (splits > (nt + 7) / 8) splits = (nt + 7) / 8;
+    if (splits > 65535) splits = 65535;
+    if (splits < 1) splits = 1;
+    wg.tiles_per_split = (int)((nt + splits - 1) / splits);
+    splits = (nt + wg.tiles_per_split - 1) / wg.tiles_per_split;
+    dim3 grid((unsigned)((g.kc + BN - 1) / BN), (unsigned)((g.cout + BM - 1) / BM), (unsigned)splits);
+    static const bool attr_ok = [] {
+      return cudaFuncSetAttribute(field_wgrad_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)kWgSmemBytes) == cudaSuccess &&
+             cudaFuncSetAttribute(field_wgrad_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)kWgSmemBytes) == cudaSuccess;
+    }();
+    if (!attr_ok) return DK_ERR_CUDA;
+    const bool vec2 = g.xs_c == 1 && g.ys_c == 1 && (g.cin % 2) == 0 && (g.cout % 2) == 0 &&
+                      ((reinterpret_cast<uintptr_t>(dtil) | reinterpret_cast<uintptr_t>(xbar)) & 7) == 0;
+    ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
+    DK_CUDA_CHECK(cudaMemsetAsync(acc, 0, (size_t)n_dw * sizeof(u64), st));
+    if (vec2) field_wgrad_mma_kernel<2><<<grid, 256, kWgSmemBytes, st>>>(wg);
+    else field_wgrad_mma_kernel<1><<<grid, 256, kWgSmemBytes, st>>>(wg);
     DK_CUDA_CHECK(cudaGetLastError());
   }
   ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
