@@ -26,7 +26,9 @@ first, then channels, rows, columns.
 * ``field_derive_B`` / ``field_mix_delta`` / ``field_wgrad_masked``
                          Eq. 4-6 in F_p
 * ``field_linear_plain`` / ``field_wgrad_plain``   what the masked results must
-                         equal, residue for residue
+                         equal, residue for residue (``field_linear_at`` /
+                         ``field_wgrad_plain_at``: one element of them, for
+                         spot checks on large layers)
 * ``field_masked_forward``   procedure Linear Operations of Algorithm 1
 
 Coefficient convention: ``C[g, i, k]`` as in the floating-point oracle (rows
@@ -218,6 +220,26 @@ def field_linear(Wq: np.ndarray, xq: np.ndarray, p: int, stride: int = 1, pad: i
     return y
 
 
+def field_linear_at(Wq: np.ndarray, x_one: np.ndarray, co: int, oh: int, ow: int, p: int,
+                    stride: int = 1, pad: int = 0) -> int:
+    """One output element of ``field_linear`` for one sample, in Python integers."""
+    if x_one.ndim == 1:
+        return sum(int(a) * int(b) for a, b in zip(Wq[co], x_one)) % p
+    cin, h, w = x_one.shape
+    _, _, kh, kw = Wq.shape
+    acc = 0
+    for u in range(kh):
+        ih = oh * stride + u - pad
+        if ih < 0 or ih >= h:
+            continue
+        for v in range(kw):
+            iw = ow * stride + v - pad
+            if iw < 0 or iw >= w:
+                continue
+            acc += sum(int(a) * int(b) for a, b in zip(Wq[co, :, u, v], x_one[:, ih, iw]))
+    return acc % p
+
+
 def field_linear_plain(Wq, xq, p, stride=1, pad=0):
     """What decoding must return: the same operation on the unencoded residues."""
     return field_linear(Wq, xq, p, stride, pad)
@@ -330,6 +352,26 @@ def field_wgrad_plain(deltaq: np.ndarray, xq: np.ndarray, p: int, kh: int = 1, k
         term = field_bilinear_wgrad(deltaq[i], xq[i], p, kh, kw, stride, pad)
         total = term if total is None else (total + term) % I64(p)
     return total
+
+
+def field_wgrad_plain_at(deltaq: np.ndarray, xq: np.ndarray, co: int, ci: int, u: int, v: int, p: int,
+                         stride: int = 1, pad: int = 0) -> int:
+    """One element of ``field_wgrad_plain``, in Python integers."""
+    if xq.ndim == 2:
+        return sum(int(a) * int(b) for a, b in zip(deltaq[:, co], xq[:, ci])) % p
+    n, _, h, w = xq.shape
+    _, _, ho, wo = deltaq.shape
+    acc = 0
+    for a in range(ho):
+        ih = a * stride + u - pad
+        if ih < 0 or ih >= h:
+            continue
+        for b in range(wo):
+            iw = b * stride + v - pad
+            if iw < 0 or iw >= w:
+                continue
+            acc += sum(int(s) * int(t) for s, t in zip(deltaq[:, co, a, b], xq[:, ci, ih, iw]))
+    return acc % p
 
 
 # ---------------------------------------------------------------------------

@@ -556,6 +556,11 @@ constexpr int MMA_BM = 64, MMA_BN = 64, MMA_BK = 32;
 constexpr int kMmaFoldTiles = 4096 / MMA_BK;
 constexpr int kMmaStageWords = (MMA_BM + MMA_BN) * MMA_BK;     // one pipeline stage: A tile then B tile
 constexpr int kMmaStages = 4;
+// Warp tile 16 x (8*kMmaNT): 4 x (8/kMmaNT) warps cover the 64 x 64 block tile.  Measured on conv layers of
+// 64-512 channels: 4 n-tiles per warp (8 warps, 255 registers) 11-12 T modular MAC/s, 2 n-tiles (16 warps,
+// 128 registers) 10-11: the rate does not follow occupancy, the tensor pipe reads 33 % busy in both.
+constexpr int kMmaNT = 4;
+constexpr int kMmaThreads = 1024 / kMmaNT;
 constexpr size_t kMmaSmemBytes = (size_t)kMmaStages * kMmaStageWords * sizeof(u32);
 
 struct RowInfo {        // one output pixel (column of the GEMM) of the block's tile
@@ -590,8 +595,7 @@ __device__ __forceinline__ void digit_planes(const uint4 w, u32 (&pl)[4]) {
 
 __device__ __forceinline__ void mma_u8(int (&d)[4], const u32 a0, const u32 a1, const u32 a2, const u32 a3,
                                        const u32 b0, const u32 b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
       : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -612,12 +616,12 @@ __device__ __forceinline__ u32 fold_classes(u32 total, const int (&c)[7], Modulu
 // consecutive k-elements are 16 contiguous bytes of one filter tap; VEC = 1:
 // every geometry and layout, one element per copy.
 template <int VEC>
-__global__ void __launch_bounds__(256, 1) field_fwd_mma_kernel(FwdParams p, MmaConsts mc) {
+__global__ void __launch_bounds__(kMmaThreads, 1) field_fwd_mma_kernel(FwdParams p, MmaConsts mc) {
   extern __shared__ __align__(16) u32 tiles[];      // kMmaStages pipeline stages
   __shared__ RowInfo rows[MMA_BN];
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   const int g = lane >> 2, tig = lane & 3;
-  const int wm = warp & 3, wn = warp >> 2;          // warp tile: rows 16*wm.., columns 32*wn..
+  const int wm = warp & 3, wn = warp >> 2;          // warp tile: rows 16*wm.., columns 8*kMmaNT*wn..
   const int m0 = blockIdx.y * MMA_BM;
   const long long n0 = (long long)blockIdx.x * MMA_BN;
 
@@ -640,7 +644,7 @@ __global__ void __launch_bounds__(256, 1) field_fwd_mma_kernel(FwdParams p, MmaC
 
   // loader: a thread copies elements k = kq .. kq+VEC-1 of rows r0 + RSTEP*i of both tiles
   constexpr int CPR = MMA_BK / VEC;              // copies per tile row
-  constexpr int RSTEP = 256 / CPR, NCOPY = MMA_BM / RSTEP;
+  constexpr int RSTEP = kMmaThreads / CPR, NCOPY = MMA_BM / RSTEP;
   const int kq = (t % CPR) * VEC, r0 = t / CPR;
   auto load_tile = [&](int k0, u32* stage) {
     const int k = k0 + kq;
@@ -666,10 +670,10 @@ __global__ void __launch_bounds__(256, 1) field_fwd_mma_kernel(FwdParams p, MmaC
     copy_async_commit();
   };
 
-  int acc[7][4][4];       // [weight class][n-tile][fragment register]
-  u32 tot[4][4];
+  int acc[7][kMmaNT][4];       // [weight class][n-tile][fragment register]
+  u32 tot[kMmaNT][4];
 #pragma unroll
-  for (int j = 0; j < 4; ++j)
+  for (int j = 0; j < kMmaNT; ++j)
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       tot[j][r] = 0;
@@ -708,22 +712,25 @@ __global__ void __launch_bounds__(256, 1) field_fwd_mma_kernel(FwdParams p, MmaC
       digit_planes(*reinterpret_cast<const uint4*>(as + tile_word(ra, 16 + 4 * tig)), a[2]);
       digit_planes(*reinterpret_cast<const uint4*>(as + tile_word(ra + 8, 16 + 4 * tig)), a[3]);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < kMmaNT; ++j) {
         u32 b[2][4];
-        const int rb = wn * 32 + j * 8 + g;
+        const int rb = wn * (8 * kMmaNT) + j * 8 + g;
         digit_planes(*reinterpret_cast<const uint4*>(bs + tile_word(rb, 4 * tig)), b[0]);
         digit_planes(*reinterpret_cast<const uint4*>(bs + tile_word(rb, 16 + 4 * tig)), b[1]);
+        // digit pairs in an order that keeps two products of one weight class four instructions apart
 #pragma unroll
         for (int da = 0; da < 4; ++da)
 #pragma unroll
-          for (int db = 0; db < 4; ++db)
+          for (int i = 0; i < 4; ++i) {
+            const int db = (i + 4 - da) & 3;
             mma_u8(acc[da + db][j], a[0][da], a[1][da], a[2][da], a[3][da], b[0][db], b[1][db]);
+          }
       }
     }
     if (++fold == kMmaFoldTiles) {
       fold = 0;
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
+      for (int j = 0; j < kMmaNT; ++j)
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
           const int c[7] = {acc[0][j][r], acc[1][j][r], acc[2][j][r], acc[3][j][r],
@@ -736,10 +743,10 @@ __global__ void __launch_bounds__(256, 1) field_fwd_mma_kernel(FwdParams p, MmaC
   }
   // fragment register r of n-tile j: row g + 8*(r >> 1), column 2*tig + (r & 1)
 #pragma unroll
-  for (int j = 0; j < 4; ++j)
+  for (int j = 0; j < kMmaNT; ++j)
 #pragma unroll
     for (int cb = 0; cb < 2; ++cb) {
-      const long long n = n0 + wn * 32 + j * 8 + 2 * tig + cb;
+      const long long n = n0 + wn * (8 * kMmaNT) + j * 8 + 2 * tig + cb;
       if (n >= p.N) continue;
       const int ow = (int)(n % p.wo);
       const long long rr = n / p.wo;
@@ -808,8 +815,8 @@ dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* yb
                                   (int)kMmaSmemBytes) == cudaSuccess;
     }();
     if (!attr_ok) return DK_ERR_CUDA;
-    if (vec4) field_fwd_mma_kernel<4><<<grid, 256, kMmaSmemBytes, st>>>(p, mc);
-    else field_fwd_mma_kernel<1><<<grid, 256, kMmaSmemBytes, st>>>(p, mc);
+    if (vec4) field_fwd_mma_kernel<4><<<grid, kMmaThreads, kMmaSmemBytes, st>>>(p, mc);
+    else field_fwd_mma_kernel<1><<<grid, kMmaThreads, kMmaSmemBytes, st>>>(p, mc);
   }
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
@@ -969,7 +976,7 @@ __device__ __forceinline__ uint4 gather4(const u32* col) {
 }
 
 template <int VEC>
-__global__ void __launch_bounds__(256, 1) field_wgrad_mma_kernel(WgMmaParams p) {
+__global__ void __launch_bounds__(kMmaThreads, 1) field_wgrad_mma_kernel(WgMmaParams p) {
   extern __shared__ __align__(16) u32 tiles[];
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   const int g = lane >> 2, tig = lane & 3;
@@ -980,7 +987,7 @@ __global__ void __launch_bounds__(256, 1) field_wgrad_mma_kernel(WgMmaParams p) 
   const int t_hi = min(t_lo + p.tiles_per_split, p.ntiles);
 
   // loader: VEC columns starting at `col` of the r-rows rr0 + RSTEP*i of both tiles
-  constexpr int CPR = MMA_BM / VEC, RSTEP = 256 / CPR, NCOPY = MMA_BK / RSTEP;
+  constexpr int CPR = MMA_BM / VEC, RSTEP = kMmaThreads / CPR, NCOPY = MMA_BK / RSTEP;
   const int col = (t % CPR) * VEC, rr0 = t / CPR;
   const bool a_ok = (m0 + col) < p.cout;
   const long long a_off = (long long)(m0 + col) * p.ys_c;
@@ -1017,10 +1024,10 @@ __global__ void __launch_bounds__(256, 1) field_wgrad_mma_kernel(WgMmaParams p) 
     copy_async_commit();
   };
 
-  int acc[7][4][4];
-  u32 tot[4][4];
+  int acc[7][kMmaNT][4];
+  u32 tot[kMmaNT][4];
 #pragma unroll
-  for (int j = 0; j < 4; ++j)
+  for (int j = 0; j < kMmaNT; ++j)
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       tot[j][r] = 0;
@@ -1053,22 +1060,25 @@ __global__ void __launch_bounds__(256, 1) field_wgrad_mma_kernel(WgMmaParams p) 
       digit_planes(gather4(ac + 16 * WG_LD), a[2]);
       digit_planes(gather4(ac + 16 * WG_LD + 8), a[3]);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < kMmaNT; ++j) {
         u32 b[2][4];
-        const u32* bc = bs + (4 * tig) * WG_LD + wn * 32 + j * 8 + g;
+        const u32* bc = bs + (4 * tig) * WG_LD + wn * (8 * kMmaNT) + j * 8 + g;
         digit_planes(gather4(bc), b[0]);
         digit_planes(gather4(bc + 16 * WG_LD), b[1]);
+        // digit pairs in an order that keeps two products of one weight class four instructions apart
 #pragma unroll
         for (int da = 0; da < 4; ++da)
 #pragma unroll
-          for (int db = 0; db < 4; ++db)
+          for (int i = 0; i < 4; ++i) {
+            const int db = (i + 4 - da) & 3;
             mma_u8(acc[da + db][j], a[0][da], a[1][da], a[2][da], a[3][da], b[0][db], b[1][db]);
+          }
       }
     }
     if (++fold == kMmaFoldTiles) {
       fold = 0;
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
+      for (int j = 0; j < kMmaNT; ++j)
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
           const int c[7] = {acc[0][j][r], acc[1][j][r], acc[2][j][r], acc[3][j][r],
@@ -1080,10 +1090,10 @@ __global__ void __launch_bounds__(256, 1) field_wgrad_mma_kernel(WgMmaParams p) 
     }
   }
 #pragma unroll
-  for (int j = 0; j < 4; ++j)
+  for (int j = 0; j < kMmaNT; ++j)
 #pragma unroll
     for (int cb = 0; cb < 2; ++cb) {
-      const int kcol2 = kb0 + wn * 32 + j * 8 + 2 * tig + cb;
+      const int kcol2 = kb0 + wn * (8 * kMmaNT) + j * 8 + 2 * tig + cb;
       if (kcol2 >= p.kc) continue;
       const int tap2 = kcol2 / p.cin, ci2 = kcol2 - tap2 * p.cin;
       const int u2 = tap2 / p.kw, v2 = tap2 - u2 * p.kw;
@@ -1443,8 +1453,8 @@ dk_status dk_field_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, uint32_t p
                       ((reinterpret_cast<uintptr_t>(dtil) | reinterpret_cast<uintptr_t>(xbar)) & 7) == 0;
     ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
     DK_CUDA_CHECK(cudaMemsetAsync(acc, 0, (size_t)n_dw * sizeof(u64), st));
-    if (vec2) field_wgrad_mma_kernel<2><<<grid, 256, kWgSmemBytes, st>>>(wg);
-    else field_wgrad_mma_kernel<1><<<grid, 256, kWgSmemBytes, st>>>(wg);
+    if (vec2) field_wgrad_mma_kernel<2><<<grid, kMmaThreads, kWgSmemBytes, st>>>(wg);
+    else field_wgrad_mma_kernel<1><<<grid, kMmaThreads, kWgSmemBytes, st>>>(wg);
     DK_CUDA_CHECK(cudaGetLastError());
   }
   ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);

@@ -273,3 +273,20 @@ def test_one_time_pad_bijection_on_a_tiny_field():
         Cq = np.array([[[3, c_noise], [5, 1], [2, 7]]])
         seen = sorted(int(F.field_encode(np.array([[4]]), np.array([[r]]), Cq, p)[0, 0]) for r in range(p))
         assert seen == list(range(p))
+
+
+def test_single_element_functions_agree_with_the_full_ones():
+    spec = _spec("conv", K=2, G=2, stride=2, pad=1)
+    d = synth.draw_field_layer(spec, P)
+    Wq, xq, dq = F.quantize(d["W"], L, P), F.quantize(d["x"], L, P), F.quantize(d["delta"], L, P)
+    full = F.field_linear(Wq, xq, P, spec.stride, spec.pad)
+    fullw = F.field_wgrad_plain(dq, xq, P, spec.kh, spec.kw, spec.stride, spec.pad)
+    for s, co, oh, ow in [(0, 0, 0, 0), (3, 3, spec.hout - 1, spec.wout - 1), (2, 1, 1, 2)]:
+        assert F.field_linear_at(Wq, xq[s], co, oh, ow, P, spec.stride, spec.pad) == full[s, co, oh, ow]
+    for co, ci, u, v in [(0, 0, 0, 0), (3, 4, 2, 2), (1, 2, 0, 1)]:
+        assert F.field_wgrad_plain_at(dq, xq, co, ci, u, v, P, spec.stride, spec.pad) == fullw[co, ci, u, v]
+    fc = _spec("fc", K=2, G=2)
+    d = synth.draw_field_layer(fc, P)
+    Wq, xq, dq = F.quantize(d["W"], L, P), F.quantize(d["x"], L, P), F.quantize(d["delta"], L, P)
+    assert F.field_linear_at(Wq, xq[1], 2, 0, 0, P) == F.field_linear(Wq, xq, P)[1, 2]
+    assert F.field_wgrad_plain_at(dq, xq, 3, 1, 0, 0, P) == F.field_wgrad_plain(dq, xq, P)[3, 1]

@@ -2,6 +2,10 @@
 exact CPU oracle on the same seeded inputs.  Everything here is integer work:
 residues, decoded integers, verdicts and the dequantised outputs (exact
 multiples of 2^-l) must match bit for bit."""
+import os
+import subprocess
+import sys
+
 import numpy as np
 import pytest
 import torch
@@ -225,3 +229,59 @@ def test_argument_errors_are_reported_without_launching(ctx):
     with pytest.raises(dk.DkError) as ei:
         dk.dk_field_decode_verify(ctx, p, P, L, ybar, C, None, yq, None, v)
     assert ei.value.status == 3
+
+
+@pytest.mark.parametrize("layer", ["conv2_2", "conv5_1"])
+def test_full_size_layer_sampled_against_the_oracle(ctx, layer):
+    """A whole layer of the CIFAR-shaped VGG-16 workload (all 32 virtual batches, the
+    configuration `bench.py --field-table` times): decoded integers and weight-gradient
+    residues at sampled coordinates against single elements computed in Python integers;
+    the verdict must be clean and an injected fault found."""
+    spec = synth.layer("vgg16_cifar", layer)
+    d = synth.draw_field_layer(spec, P)
+    p = dk.problem_from_spec(spec)
+    ctx.ensure_workspace(p, field=True)
+    E = spec.K + 2
+    C, gamma = u32(d["Cq"]), u32(d["gammaq"])
+    W_dev, x_dev = H.weights_to_dev(d["W"], dk.DK_NHWC), H.acts_to_dev(d["x"], dk.DK_NHWC)
+    rq_dev = res_acts_to_dev(d["rq"], dk.DK_NHWC)
+    yq_dev = torch.empty(H.empty_acts(spec.batch, spec, "out", dk.DK_NHWC).shape, dtype=torch.int32, device="cuda")
+    xsave = torch.empty((spec.G * E,) + tuple(x_dev.shape[1:]), dtype=torch.int32, device="cuda")
+    v = dk.new_verdict()
+    dk.dk_field_masked_linear(ctx, p, P, L, W_dev, x_dev, rq_dev, C, None, None, yq_dev, xsave, v)
+    got = dk.read_verdict(v)
+    assert (got["ok"], got["n_flagged"], got["first_index"]) == (1, 0, -1)
+    Wq, xq = F.quantize(d["W"], L, P), F.quantize(d["x"], L, P)
+    yq = res_acts_from_dev(yq_dev, dk.DK_NHWC)
+    for g, co, oh, ow in synth.sample_coordinates(spec, 24, "y"):
+        for k in (0, spec.K - 1):
+            s = int(g) * spec.K + k
+            want = F.centre(np.array(F.field_linear_at(Wq, xq[s], co, oh, ow, P, spec.stride, spec.pad)), P)
+            assert yq[s, co, oh, ow] == want
+    f = dk.dk_field_fault(spec.G - 1, 1, 77, 1)
+    dk.dk_field_masked_linear(ctx, p, P, L, W_dev, x_dev, rq_dev, C, None, None, yq_dev, None, v, f)
+    got = dk.read_verdict(v)
+    assert (got["ok"], got["n_flagged"], got["first_index"]) == (0, 1, (spec.G - 1) * spec.n_out + 77)
+
+    delta_dev = H.acts_to_dev(d["delta"], dk.DK_NHWC)
+    dq_dev = empty_res(delta_dev)
+    dk.dk_field_quantize(ctx, delta_dev, L, P, dq_dev)
+    dWq_dev = torch.empty(H.empty_weights(spec, dk.DK_NHWC).shape, dtype=torch.int32, device="cuda")
+    dk.dk_field_linear_bwd_wgrad(ctx, p, P, dq_dev, xsave, E, C, gamma, dWq_dev)
+    dWq = res_weights_from_dev(dWq_dev, dk.DK_NHWC)
+    dq = F.quantize(d["delta"], L, P)
+    for co, ci, u, vv in synth.sample_coordinates(spec, 12, "dw"):
+        assert dWq[co, ci, u, vv] == F.field_wgrad_plain_at(dq, xq, co, ci, u, vv, P, spec.stride, spec.pad)
+
+
+def test_integer_alu_kernels_give_the_same_residues():
+    """DK_FIELD_SIMT=1 selects the 64-bit integer-ALU contraction kernels instead of the tensor-core ones
+    (the switch is read once per process): a few parity cases re-run in a child process under it."""
+    if os.environ.get("DK_FIELD_SIMT") == "1":
+        pytest.skip("already running under the switch")
+    env = dict(os.environ, DK_FIELD_SIMT="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", os.path.abspath(__file__), "-k",
+                        "conv_tiny_K2 or fc_K8_long or conv_3x3s2_K5 or conv_ragged_K3_nchw"],
+                       cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
