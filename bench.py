@@ -20,7 +20,7 @@ the per-layer table; it is a reporting aid, not the step metric.
 
 `--field-table` does the same for the finite-field calls (Section 5 of the
 paper: residues modulo p = 2^25 - 39), in exact modular multiply-accumulates
-per second against the integer-ALU peak.
+per second against the peak of the integer tensor pipe they run on.
 
 With N > 1 (under torchrun) every rank runs an independent replica of the
 workload on its own GPU: the path has no exchange step, nothing is sharded.
@@ -333,15 +333,17 @@ def run_layer_table(args):
 
 
 P_FIELD, L_FIELD = 2 ** 25 - 39, 8     # the prime and the fractional bits the paper uses (Section 5)
-# Integer multiply-add lanes: 64 per SM and clock (32-bit IMAD).  One exact multiply-accumulate of two
-# 25-bit residues is a 32x32->64-bit multiply with a 64-bit add, i.e. two passes of the 32-bit multiplier.
-INT_LANES_PER_SM, SMS, IMAD_PER_FIELD_MAC = 64, 148, 2
+# Peaks of the integer tensor pipes in int8 operations (2 per multiply-accumulate) per clock and SM, as ncu states
+# them for this part (sm__ops_path_tensor_op_{imma,utcimma}_src_int8_sparsity_off peak_sustained): the mma.sync
+# path the field kernels use, and the tcgen05 path.  One exact multiply-accumulate of two residues costs
+# sixteen u8 x u8 multiply-accumulates (four base-256 digits each).
+SMS, IMMA_OPS_PER_CLK_SM, UTCIMMA_OPS_PER_CLK_SM, INT8_OPS_PER_FIELD_MAC = 148, 4096, 16384, 32
 
 
 def run_field_table(args):
     """Per-layer timing of the finite-field calls (dk_field_masked_linear, dk_field_linear_bwd_wgrad) and of
     the standalone field encode / decode_verify, in exact modular multiply-accumulates per second against the
-    integer-ALU peak; a reporting aid like --layer-table."""
+    int8 tensor peak of the mma.sync path; a reporting aid like --layer-table."""
     import torch
     from paper_2207_00083_b200 import binding as dk
     from paper_2207_00083_b200 import synth
@@ -443,17 +445,18 @@ def run_field_table(args):
     assert dk.read_verdict(v)["ok"] == 1      # decode of encode-only data: rho = n . C . [x; r] = 0
     clocks = sampler.stop()
     mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
-    peak = SMS * INT_LANES_PER_SM * mhz * 1e6 / IMAD_PER_FIELD_MAC / 1e12
+    peak = SMS * IMMA_OPS_PER_CLK_SM * mhz * 1e6 / INT8_OPS_PER_FIELD_MAC / 1e12
+    peak_tc5 = SMS * UTCIMMA_OPS_PER_CLK_SM * mhz * 1e6 / INT8_OPS_PER_FIELD_MAC / 1e12
     for row in rows:
         for name in ("fwd", "wgrad"):
             if name in row:
-                row[name]["frac_alu_peak_kernel"] = round(row[name]["tmacs_kernel"] / peak, 4)
+                row[name]["frac_int8_mma_sync_peak_kernel"] = round(row[name]["tmacs_kernel"] / peak, 4)
     print(json.dumps({"field_table": args.workload, "prime": P_FIELD, "l": L_FIELD, "unit": "T exact modular MAC/s",
-                      "alu_peak_tmacs": round(peak, 3),
-                      "alu_peak_source": f"{SMS} SMs x {INT_LANES_PER_SM} int32 multiply-add lanes x {mhz} MHz / "
-                                         f"{IMAD_PER_FIELD_MAC} multiplier passes per 64-bit multiply-accumulate",
+                      "bound": "tensor (int8, mma.sync path)", "peak_tmacs": round(peak, 2),
+                      "peak_source": f"{SMS} SMs x {IMMA_OPS_PER_CLK_SM} int8 ops per clock and SM (ncu's peak for "
+                                     f"mma.sync int8) x {mhz} MHz / {INT8_OPS_PER_FIELD_MAC} int8 ops per modular MAC",
+                      "tcgen05_int8_peak_tmacs": round(peak_tc5, 2),
                       "elementwise": elem, "clocks": clocks, "rows": rows}), flush=True)
-
 
 def max_over_ranks(value, world, device):
     """Device-timed milliseconds of this rank -> the slowest rank's figure (every rank gets it).
