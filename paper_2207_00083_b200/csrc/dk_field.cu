@@ -21,8 +21,10 @@ typedef unsigned int u32;
 typedef unsigned long long u64;
 
 struct Modulus {
-  u64 m;   // floor(2^64 / p)
+  u64 m;     // floor(2^64 / p)
   u32 p;
+  u32 m32;   // floor(2^(32+s) / p) with 2^s <= p < 2^(s+1); valid when s >= 0
+  int s;     // -1 when p >= 2^27 (the short reduction is not offered)
 };
 
 __host__ __device__ __forceinline__ u32 reduce64(u64 x, Modulus md) {
@@ -35,6 +37,21 @@ __host__ __device__ __forceinline__ u32 reduce64(u64 x, Modulus md) {
   if (r >= md.p) r -= md.p;
   if (r >= md.p) r -= md.p;
   return (u32)r;
+}
+
+// Short Barrett reduction for x < 2^(32+s): q = mulhi32(x >> s, m32) is the true
+// quotient or up to two less, and x - q*p < 3p < 2^32 needs only the low words.
+// The elementwise kernels' sums qualify when p < 2^27: at most 16 products
+// below p^2 < 2^(2s+2) stay below 2^(32+s).
+__device__ __forceinline__ u32 reduce_short(u64 x, Modulus md) {
+  const u32 q = __umulhi((u32)(x >> md.s), md.m32);
+  u32 r = (u32)x - q * md.p;
+  if (r >= md.p) r -= md.p;
+  if (r >= md.p) r -= md.p;
+  return r;
+}
+__device__ __forceinline__ u32 reduce_sum(u64 x, Modulus md) {
+  return md.s >= 0 ? reduce_short(x, md) : reduce64(x, md);
 }
 
 // ---------------------------------------------------------------------------
@@ -260,7 +277,7 @@ __global__ void __launch_bounds__(256) field_mix_rows_kernel(const u32* __restri
       }
       Vec<VEC> o;
 #pragma unroll
-      for (int v = 0; v < VEC; ++v) o.v[v] = reduce64(acc[v], md);
+      for (int v = 0; v < VEC; ++v) o.v[v] = reduce_sum(acc[v], md);
       o.store(out + ((long long)g * rout + r) * n + i * VEC);
     }
   }
@@ -348,7 +365,7 @@ __global__ void __launch_bounds__(256) field_decode_verify_kernel(DecodeParams p
         for (int v = 0; v < VEC; ++v) rho[v] += (u64)N[e] * yb[e].v[v];
 #pragma unroll
       for (int v = VEC - 1; v >= 0; --v)
-        if (reduce64(rho[v], p.md) != 0) {
+        if (reduce_sum(rho[v], p.md) != 0) {
           ++nbad;
           firstbad = (long long)g * p.n + i * VEC + v;
         }
@@ -364,21 +381,31 @@ __global__ void __launch_bounds__(256) field_decode_verify_kernel(DecodeParams p
           for (int v = 0; v < VEC; ++v) acc[v] += (u64)c * yb[e].v[v];
         }
         const long long o = ((long long)g * K + k) * p.n + i * VEC;
+        int cq[VEC];
 #pragma unroll
         for (int v = 0; v < VEC; ++v) {
-          u32 r = reduce64(acc[v], p.md);
+          u32 r = reduce_sum(acc[v], p.md);
           if (p.bias) {
             const long long e = i * VEC + v;
             r += __ldg(p.bias + (int)((e / p.ch_div) % p.cout));
             if (r >= p.md.p) r -= p.md.p;
           }
-          const long long c = (2ull * r > p.md.p) ? (long long)r - (long long)p.md.p : (long long)r;
-          if (p.yq) p.yq[o + v] = (int)c;
-          if (p.y) {
-            const double t = (double)c * p.inv_scale;
+          cq[v] = (2u * r > p.md.p) ? (int)r - (int)p.md.p : (int)r;      // p < 2^30: no overflow
+        }
+        if (p.yq) {
+          if (VEC == 4) *reinterpret_cast<int4*>(p.yq + o) = make_int4(cq[0], cq[1], cq[2], cq[3 % VEC]);
+          else p.yq[o] = cq[0];
+        }
+        if (p.y) {
+          float yv[VEC];
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) {
+            const double t = (double)cq[v] * p.inv_scale;
             const double f = floor(t);
-            p.y[o + v] = (float)(((t - f < 0.5) ? f : f + 1.0) * p.inv_scale);
+            yv[v] = (float)(((t - f < 0.5) ? f : f + 1.0) * p.inv_scale);
           }
+          if (VEC == 4) *reinterpret_cast<float4*>(p.y + o) = make_float4(yv[0], yv[1], yv[2], yv[3 % VEC]);
+          else p.y[o] = yv[0];
         }
       }
     }
@@ -833,7 +860,7 @@ struct WgParams {
   int K1, xbar_rows, P, PC;   // P = ho*wo pixels, PC = ceil(P/BK)
   long long GP;               // G * PC contraction blocks
   long long per_split;
-  int fold_blocks;            // contraction blocks between two reductions
+  int fold_blocks;            // contraction blocks between two reductions (0: after every k-tile)
   long long n_in, n_out;
   long long xs_c, xs_h, xs_w, ws_o, ws_c, ws_u, ws_v, ys_c, ys_h, ys_w;
   Modulus md;
@@ -907,6 +934,12 @@ __global__ void __launch_bounds__(NT) field_wgrad_kernel(WgParams p) {
           for (int jj = 0; jj < 4; ++jj) acc[i][jj] += (u64)a[i] * b[jj];
       }
       __syncthreads();
+      if (p.fold_blocks == 0) {      // large p: only one k-tile of products fits between reductions
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) acc[i][jj] = reduce64(acc[i][jj], p.md);
+      }
     }
     if (++fold == p.fold_blocks) {
       fold = 0;
@@ -1164,6 +1197,14 @@ dk_status make_modulus(uint32_t p, Modulus* md) {
   if (p >= (1u << 30) || !prime_by_trial_division(p)) return DK_ERR_INVALID_ARG;
   md->p = p;
   md->m = ~0ull / p;      // = floor(2^64 / p): p is odd, so it does not divide 2^64
+  md->s = -1;
+  md->m32 = 0;
+  if (p < (1u << 27)) {
+    int s = 0;
+    while ((2u << s) <= p) ++s;      // 2^s <= p < 2^(s+1)
+    md->s = s;
+    md->m32 = (u32)((1ull << (32 + s)) / p);      // in (2^31, 2^32): p is not a power of two
+  }
   return DK_OK;
 }
 
@@ -1399,8 +1440,8 @@ dk_status dk_field_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, uint32_t p
     wg.ws_o = g.ws_o; wg.ws_c = g.ws_c; wg.ws_u = g.ws_u; wg.ws_v = g.ws_v;
     wg.ys_c = g.ys_c; wg.ys_h = g.ys_h; wg.ys_w = g.ys_w;
     wg.md = md;
-    long long fb = terms_per_reduction(prime) / ((long long)BK * wg.K1);
-    if (fb < 1) return DK_ERR_UNSUPPORTED;
+    if (terms_per_reduction(prime) < BK) return DK_ERR_UNSUPPORTED;
+    long long fb = terms_per_reduction(prime) / ((long long)BK * wg.K1);      // 0: reduce after every k-tile
     if (fb > 64) fb = 64;
     wg.fold_blocks = (int)fb;
     long long splits = (4LL * ctx->sm_count + tiles - 1) / tiles;

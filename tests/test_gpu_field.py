@@ -212,6 +212,44 @@ def test_masked_linear_and_wgrad_match_the_oracle(ctx, name, spec, layout):
                           F.centre(want_dw, P).astype(np.float64) / 4 ** L)
 
 
+@pytest.mark.parametrize("prime", [65537, 2 ** 27 - 39, 2 ** 29 - 3])
+@pytest.mark.parametrize("kind", ["fc", "conv"])
+def test_other_primes(ctx, prime, kind):
+    """Any odd prime below 2^30 is served: a small one (the decoded integers wrap, parity is modulo p all the
+    same), the largest one below 2^27 (the last to take the short reduction in the elementwise kernels) and one
+    above it (64-bit reductions everywhere)."""
+    spec = tiny("fc", cin=300, cout=21, K=3, G=2) if kind == "fc" else tiny(cin=6, cout=10, h=7, w=6, K=8, G=1)
+    d = synth.draw_field_layer(spec, prime)
+    p = dk.problem_from_spec(spec)
+    ctx.ensure_workspace(p, field=True)
+    E = spec.K + 2
+    C, gamma = u32(d["Cq"]), u32(d["gammaq"])
+    W_dev, x_dev = H.weights_to_dev(d["W"], dk.DK_NHWC), H.acts_to_dev(d["x"], dk.DK_NHWC)
+    rq_dev = res_acts_to_dev(d["rq"], dk.DK_NHWC)
+    y_dev = H.empty_acts(spec.batch, spec, "out", dk.DK_NHWC)
+    yq_dev = torch.empty(y_dev.shape, dtype=torch.int32, device="cuda")
+    xsave = torch.empty((spec.G * E,) + tuple(x_dev.shape[1:]), dtype=torch.int32, device="cuda")
+    v = dk.new_verdict()
+    dk.dk_field_masked_linear(ctx, p, prime, L, W_dev, x_dev, rq_dev, C, H.dev(d["bias"]), y_dev, yq_dev, xsave, v)
+    want = F.field_masked_forward(d["W"], d["x"], d["rq"], d["Cq"], L, prime, spec.stride, spec.pad, bias=d["bias"])
+    assert np.array_equal(res_acts_from_dev(xsave, dk.DK_NHWC), want["xbar"])
+    assert np.array_equal(res_acts_from_dev(yq_dev, dk.DK_NHWC), want["yq"])
+    assert np.array_equal(H.acts_from_dev(y_dev, dk.DK_NHWC).astype(np.float64), want["y"])
+    assert dk.read_verdict(v)["ok"] == 1
+    f = dk.dk_field_fault(spec.G - 1, spec.K + 1, 5, 1)
+    dk.dk_field_masked_linear(ctx, p, prime, L, W_dev, x_dev, rq_dev, C, None, None, yq_dev, None, v, f)
+    got = dk.read_verdict(v)
+    assert (got["ok"], got["n_flagged"], got["first_index"]) == (0, 1, (spec.G - 1) * spec.n_out + 5)
+    delta_dev = H.acts_to_dev(d["delta"], dk.DK_NHWC)
+    dq_dev = empty_res(delta_dev)
+    dk.dk_field_quantize(ctx, delta_dev, L, prime, dq_dev)
+    dWq_dev = torch.empty(H.empty_weights(spec, dk.DK_NHWC).shape, dtype=torch.int32, device="cuda")
+    dk.dk_field_linear_bwd_wgrad(ctx, p, prime, dq_dev, xsave, E, C, gamma, dWq_dev)
+    dq = F.quantize(d["delta"], L, prime)
+    assert np.array_equal(res_weights_from_dev(dWq_dev, dk.DK_NHWC),
+                          F.field_wgrad_plain(dq, want["xq"], prime, spec.kh, spec.kw, spec.stride, spec.pad))
+
+
 def test_argument_errors_are_reported_without_launching(ctx):
     spec = tiny("fc", cin=8, cout=4, K=2, G=1)
     p = dk.problem_from_spec(spec)
@@ -282,6 +320,6 @@ def test_integer_alu_kernels_give_the_same_residues():
     env = dict(os.environ, DK_FIELD_SIMT="1")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", os.path.abspath(__file__), "-k",
-                        "conv_tiny_K2 or fc_K8_long or conv_3x3s2_K5 or conv_ragged_K3_nchw"],
+                        "conv_tiny_K2 or fc_K8_long or conv_3x3s2_K5 or conv_ragged_K3_nchw or other_primes"],
                        cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
