@@ -349,13 +349,17 @@ def run_field_table(args):
     from paper_2207_00083_b200 import synth
     dev = torch.device("cuda:0")
     torch.cuda.set_device(0)
-    peaks = read_peaks()
     ctx = dk.Context(0)
+    flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)
+    out = measure_field(torch, dk, synth, ctx, dev, read_peaks(), flush, args.workload,
+                        set(args.layers.split(",")) if args.layers else None, args.iters)
+    print(json.dumps(out), flush=True)
+
+
+def measure_field(torch, dk, synth, ctx, dev, peaks, flush, workload, want, iters):
     gen = torch.Generator(device=dev)
     gen.manual_seed(220700083)
-    flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)
-    want = set(args.layers.split(",")) if args.layers else None
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(dev.index or 0)
     sampler.start()
     rows = []
 
@@ -374,7 +378,7 @@ def run_field_table(args):
             tot += a.elapsed_time(b)
         return tot / iters
 
-    for s in synth.layers(args.workload):
+    for s in synth.layers(workload):
         if want and s.name not in want:
             continue
         p = dk.problem_from_spec(s)
@@ -388,7 +392,7 @@ def run_field_table(args):
         rq = residues(shape_acts(s.G, s, "in"))
         y = torch.empty(shape_acts(s.batch, s, "out"), device=dev)
         xsave = torch.empty(shape_acts(s.G * (s.K + 2), s, "in"), dtype=torch.int32, device=dev)
-        v = dk.new_verdict(0)
+        v = dk.new_verdict(dev.index or 0)
 
         def fwd():
             dk.dk_field_masked_linear(ctx, p, P_FIELD, L_FIELD, W, x, rq, C, None, y, None, xsave, v)
@@ -405,7 +409,7 @@ def run_field_table(args):
             fn()
             dk.dk_profile_reset(ctx)
             dk.dk_profile_enable(ctx, True)
-            ms = timeit(fn, args.iters)
+            ms = timeit(fn, iters)
             prof = dk.dk_profile_read(ctx)
             dk.dk_profile_enable(ctx, False)
             kms = prof[kind][0] / max(prof[kind][1], 1)
@@ -425,7 +429,7 @@ def run_field_table(args):
     xq, rq = residues((G * K, n)), residues((G, n))
     xbar = torch.empty((G * (K + 2), n), dtype=torch.int32, device=dev)
     yq = torch.empty((G * K, n), dtype=torch.int32, device=dev)
-    v = dk.new_verdict(0)
+    v = dk.new_verdict(dev.index or 0)
     elem = {}
     for name, fn, bpp in (("encode", lambda: dk.dk_field_encode(ctx, p, P_FIELD, xq, rq, C, xbar), (2 * K + 3) * 4),
                           ("decode", lambda: dk.dk_field_decode_verify(ctx, p, P_FIELD, L_FIELD, xbar, C, None, yq,
@@ -451,12 +455,12 @@ def run_field_table(args):
         for name in ("fwd", "wgrad"):
             if name in row:
                 row[name]["frac_int8_mma_sync_peak_kernel"] = round(row[name]["tmacs_kernel"] / peak, 4)
-    print(json.dumps({"field_table": args.workload, "prime": P_FIELD, "l": L_FIELD, "unit": "T exact modular MAC/s",
-                      "bound": "tensor (int8, mma.sync path)", "peak_tmacs": round(peak, 2),
-                      "peak_source": f"{SMS} SMs x {IMMA_OPS_PER_CLK_SM} int8 ops per clock and SM (ncu's peak for "
-                                     f"mma.sync int8) x {mhz} MHz / {INT8_OPS_PER_FIELD_MAC} int8 ops per modular MAC",
-                      "tcgen05_int8_peak_tmacs": round(peak_tc5, 2),
-                      "elementwise": elem, "clocks": clocks, "rows": rows}), flush=True)
+    return {"field_table": workload, "prime": P_FIELD, "l": L_FIELD, "unit": "T exact modular MAC/s",
+            "bound": "tensor (int8, mma.sync path)", "peak_tmacs": round(peak, 2),
+            "peak_source": f"{SMS} SMs x {IMMA_OPS_PER_CLK_SM} int8 ops per clock and SM (ncu's peak for "
+                           f"mma.sync int8) x {mhz} MHz / {INT8_OPS_PER_FIELD_MAC} int8 ops per modular MAC",
+            "tcgen05_int8_peak_tmacs": round(peak_tc5, 2),
+            "elementwise": elem, "clocks": clocks, "rows": rows}
 
 def max_over_ranks(value, world, device):
     """Device-timed milliseconds of this rank -> the slowest rank's figure (every rank gets it).
@@ -674,6 +678,14 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
+    if world == 1:
+        # the finite-field calls on one mid-sized layer of the same workload (reported beside the metric,
+        # measured after it; `--field-table` gives every layer)
+        names = [s.name for s in specs]
+        pick = "conv3_2" if "conv3_2" in names else names[len(names) // 2]
+        fm = measure_field(torch, dk, synth, ctx, dev, peaks, flush, args.workload, {pick}, 5)
+        line["field_path"] = {k: fm[k] for k in ("prime", "l", "unit", "bound", "peak_tmacs", "peak_source",
+                                                  "elementwise", "rows")}
     if not args.no_cpu_baseline and world == 1:
         r = time_oracle(args.workload, 500, 1, budget_s=12.0)
         line["cpu_baseline"] = {"value": r["value"], "unit": "TFLOP/s", "cores": r["cores"], "kind": "oracle",
