@@ -791,6 +791,289 @@ __global__ void __launch_bounds__(kMmaThreads, 1) field_fwd_mma_kernel(FwdParams
     }
 }
 
+// ---------------------------------------------------------------------------
+// The forward contraction on the tcgen05 integer tensor path.  Same digit
+// decomposition as above, but the sixteen u8 x u8 products of a k-step are
+// tcgen05.mma.kind::i8 instructions on digit PLANES in shared memory (K-major,
+// 128-byte swizzle: one row = 128 contraction elements of one digit), and the
+// seven weight-class sums live in tensor memory (7 x 64 columns of s32).
+//
+//   tile: 128 output channels (TMEM lanes) x 64 pixels, k-tiles of 128 elements
+//   all 8 warps: load residues (16-byte groups of one filter tap), split them
+//                into digit planes, store the planes swizzled; two stages
+//   thread 0:    64 MMAs per k-tile (16 digit pairs x 4 k-steps of 32), commit
+//   all 8 warps: at the end (and every 64 k-tiles, before a class sum can pass
+//                2^31) read the class sums with tcgen05.ld and fold them mod p
+// Every mbarrier wait is bounded; on expiry the CTA stops issuing, reports
+// DK_ERR_TIMEOUT in *status, still frees its tensor memory and returns.
+// ---------------------------------------------------------------------------
+namespace tcf {
+constexpr int TM = 128, TN = 64, TK = 128;
+constexpr int kThreads = 256;
+constexpr int A_PLANE = TM * TK, B_PLANE = TN * TK;              // bytes per digit plane
+constexpr int STAGE = 4 * A_PLANE + 4 * B_PLANE;                 // 96 KB
+constexpr int kStages = 2;
+constexpr size_t kSmem = (size_t)kStages * STAGE + 1024;         // + slack for 1024-byte alignment
+constexpr int kFoldTiles = 8192 / TK;                            // 4 pairs * 255^2 * 8192 < 2^31
+constexpr unsigned kSpin = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (unsigned i = 0; i < kSpin; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void ld8(uint32_t taddr, int (&v)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr)
+               : "memory");
+}
+// K-major operand plane, rows of 128 bytes (one swizzle span), 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t plane_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= 2ull << 61;                 // 128-byte swizzle
+  return d;
+}
+}  // namespace tcf
+
+__global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParams p, MmaConsts mc, int* status) {
+  using namespace tcf;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t mma_done[kStages];
+  __shared__ uint32_t tmem_slot[2];          // [0] TMEM base address, [1] abort flag
+  __shared__ RowInfo rows[TN];
+  __shared__ long long out_off[TN];
+  uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int m0 = blockIdx.y * TM;
+  const long long n0 = (long long)blockIdx.x * TN;
+
+  if (t == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(mma_done + s, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (t < TN) {
+    const long long n = n0 + t;
+    RowInfo ri;
+    long long oo = -1;
+    if (n < p.N) {
+      const int ow = (int)(n % p.wo);
+      const long long r = n / p.wo;
+      const int oh = (int)(r % p.ho);
+      const long long smp = r / p.ho;
+      ri.base = smp * p.n_in;
+      ri.ih0 = oh * p.stride - p.pad;
+      ri.iw0 = ow * p.stride - p.pad;
+      oo = smp * p.n_out + (long long)oh * p.ys_h + (long long)ow * p.ys_w;
+    } else {
+      ri.base = -1; ri.ih0 = 0; ri.iw0 = 0;
+    }
+    rows[t] = ri;
+    out_off[t] = oo;
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_slot[0];
+
+  // this thread's part of the result: TMEM lane (output channel) 32*(warp & 3) + lane, columns 32*(warp >> 2) ..
+  const int q = warp & 3, h = warp >> 2;
+  u32 tot[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) tot[j] = 0;
+
+  // S32 accumulator, unsigned 8-bit A and B, both K-major, N = 64, M = 128
+  constexpr uint32_t idesc = (2u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(TN >> 3) << 17) |
+                             ((uint32_t)(TM >> 4) << 24);
+
+  const int ntiles = (p.kc + TK - 1) / TK;
+  uint32_t started = 0;                // bit c: class c has received its first product since the last fold
+  bool alive = true;
+  for (int kt = 0; kt < ntiles; ++kt) {
+    const int stage = kt & 1;
+    uint8_t* st = smem + (size_t)stage * STAGE;
+    // the products that read this stage two k-tiles ago must have completed
+    if (kt >= kStages) {
+      if (!mbar_wait(mma_done + stage, (uint32_t)((kt / kStages - 1) & 1), abort_flag)) alive = false;
+    }
+    if (alive) {
+      // units of 16 contraction elements of one row: 128 rows of W, then 64 pixels of x.  A thread's
+      // units all sit in the same 16-element column c = t & 7 of the k-tile, so the filter taps of its
+      // four 4-element groups are worked out once per k-tile.
+      const int c = t & 7;
+      int g_ci[4], g_u[4], g_v[4];
+      bool g_ok[4];
+      {
+        int k = kt * TK + c * 16;
+        int tap = k / p.cin;
+        int ci = k - tap * p.cin;
+        int u = tap / p.kw, v = tap - u * p.kw;
+#pragma unroll
+        for (int gq = 0; gq < 4; ++gq) {
+          g_ok[gq] = k < p.kc;
+          g_ci[gq] = ci; g_u[gq] = u; g_v[gq] = v;
+          k += 4; ci += 4;
+          if (ci >= p.cin) {
+            ci -= p.cin;
+            if (++v == p.kw) { v = 0; ++u; }
+          }
+        }
+      }
+      for (int uidx = t; uidx < (TM + TN) * 8; uidx += kThreads) {
+        const bool isA = uidx < TM * 8;
+        const int row = isA ? (uidx >> 3) : ((uidx - TM * 8) >> 3);
+        uint4 w[4];
+        if (isA) {
+          const bool rok = m0 + row < p.cout;
+          const u32* wr = p.W + (long long)(m0 + row) * p.ws_o;
+#pragma unroll
+          for (int gq = 0; gq < 4; ++gq)
+            w[gq] = (rok && g_ok[gq])
+                        ? __ldg(reinterpret_cast<const uint4*>(wr + g_ci[gq] + (long long)g_u[gq] * p.ws_u +
+                                                               (long long)g_v[gq] * p.ws_v))
+                        : make_uint4(0u, 0u, 0u, 0u);
+        } else {
+          const RowInfo ri = rows[row];
+#pragma unroll
+          for (int gq = 0; gq < 4; ++gq) {
+            const int ih = ri.ih0 + g_u[gq], iw = ri.iw0 + g_v[gq];
+            const bool ok = g_ok[gq] && ri.base >= 0 && ih >= 0 && ih < p.h && iw >= 0 && iw < p.w;
+            w[gq] = ok ? __ldg(reinterpret_cast<const uint4*>(p.x + ri.base + g_ci[gq] + (long long)ih * p.xs_h +
+                                                              (long long)iw * p.xs_w))
+                       : make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+        u32 pl[4][4];      // [group of four elements][digit]
+#pragma unroll
+        for (int gq = 0; gq < 4; ++gq) digit_planes(w[gq], pl[gq]);
+        uint8_t* base = st + (isA ? 0 : 4 * A_PLANE) + row * TK + ((c ^ (row & 7)) << 4);
+        const int plane = isA ? A_PLANE : B_PLANE;
+#pragma unroll
+        for (int dg = 0; dg < 4; ++dg)
+          *reinterpret_cast<uint4*>(base + dg * plane) = make_uint4(pl[0][dg], pl[1][dg], pl[2][dg], pl[3][dg]);
+      }
+      // make the planes visible to the tensor core's (asynchronous-proxy) reads
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    if (*abort_flag) alive = false;
+    if (alive && t == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t sa = smem_u32(st), sb = sa + 4 * A_PLANE;
+#pragma unroll
+      for (int ks = 0; ks < TK / 32; ++ks) {
+        const uint64_t adv = (uint64_t)(ks * 2);       // 32 bytes per k-step, in 16-byte units
+#pragma unroll
+        for (int da = 0; da < 4; ++da)
+#pragma unroll
+          for (int db = 0; db < 4; ++db) {
+            const int c = da + db;
+            mma_i8(tmem_base + (uint32_t)(c * TN), plane_desc(sa + da * A_PLANE) + adv,
+                   plane_desc(sb + db * B_PLANE) + adv, idesc, (started >> c) & 1u);
+            started |= 1u << c;
+          }
+      }
+      commit(mma_done + stage);
+    }
+    // fold before a class sum can overflow, and at the end
+    const bool last = kt + 1 == ntiles;
+    if (last || ((kt + 1) % kFoldTiles) == 0) {
+      // every product issued so far: the newest commit of each stage in use
+      const int kprev = kt - 1;
+      if (alive && kprev >= 0 &&
+          !mbar_wait(mma_done + (kprev & 1), (uint32_t)((kprev / kStages) & 1), abort_flag))
+        alive = false;
+      if (alive && !mbar_wait(mma_done + stage, (uint32_t)((kt / kStages) & 1), abort_flag)) alive = false;
+      __syncthreads();
+      if (*abort_flag) alive = false;
+      if (alive) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+        for (int cg = 0; cg < 4; ++cg) {
+          int cls[7][8];
+#pragma unroll
+          for (int c = 0; c < 7; ++c)
+            ld8(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * TN + h * 32 + cg * 8), cls[c]);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int cc[7] = {cls[0][j], cls[1][j], cls[2][j], cls[3][j], cls[4][j], cls[5][j], cls[6][j]};
+            tot[cg * 8 + j] = fold_classes(tot[cg * 8 + j], cc, p.md, mc.pow32);
+          }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      }
+      __syncthreads();
+      started = 0;
+    }
+  }
+  if (alive) {
+    const int m = m0 + q * 32 + lane;
+    if (m < p.cout) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const long long oo = out_off[h * 32 + j];
+        if (oo >= 0) p.y[oo + (long long)m * p.ys_c] = tot[j];
+      }
+    }
+  }
+  __syncthreads();
+  if (*abort_flag) {
+    // a bounded wait expired: report, and give products still in flight time to retire
+    if (t == 0 && status != nullptr) atomicExch(status, (int)DK_ERR_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(16384);
+    __syncthreads();
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // How many products of two residues may be added to one residue in a uint64.
 long long terms_per_reduction(u32 p) {
   const u64 pm = (u64)p - 1;
@@ -808,8 +1091,17 @@ bool field_use_simt() {
   return v;
 }
 
+// DK_FIELD_MMA_SYNC=1 keeps the forward contraction on the mma.sync kernel (a cross-check of the tcgen05 one).
+bool field_use_mma_sync() {
+  static const bool v = [] {
+    const char* e = getenv("DK_FIELD_MMA_SYNC");
+    return e && e[0] == '1';
+  }();
+  return v;
+}
+
 dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* ybar, int nsamples, Modulus md,
-                           cudaStream_t st) {
+                           int* status, cudaStream_t st) {
   FwdParams p;
   p.W = W; p.x = xbar; p.y = ybar;
   p.cin = g.cin; p.cout = g.cout; p.h = g.h; p.w = g.w; p.kw = g.kw; p.stride = g.stride;
@@ -835,6 +1127,17 @@ dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* yb
     MmaConsts mc;
     mc.pow32 = (u32)((1ull << 32) % md.p);
     const bool vec4 = g.xs_c == 1 && g.ws_c == 1 && (g.cin % 4) == 0 && aligned16(W) && aligned16(xbar);
+    if (vec4 && !field_use_mma_sync()) {
+      static const bool tc_attr_ok =
+          cudaFuncSetAttribute(field_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)tcf::kSmem) == cudaSuccess;
+      if (!tc_attr_ok) return DK_ERR_CUDA;
+      const long long tnb = (p.N + tcf::TN - 1) / tcf::TN;
+      dim3 tgrid((unsigned)tnb, (unsigned)((g.cout + tcf::TM - 1) / tcf::TM));
+      field_fwd_tc_kernel<<<tgrid, tcf::kThreads, tcf::kSmem, st>>>(p, mc, status);
+      DK_CUDA_CHECK(cudaGetLastError());
+      return DK_OK;
+    }
     static const bool attr_ok = [] {
       return cudaFuncSetAttribute(field_fwd_mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)kMmaSmemBytes) == cudaSuccess &&
@@ -1157,6 +1460,9 @@ int ew_blocks(long long n, int sm_count) {
   return (int)(b < 1 ? 1 : b);
 }
 
+// The context's device status word (read and cleared by dk_device_status).
+int* field_status_word(dk_ctx* ctx) { return reinterpret_cast<int*>(ctx->d_vstats + kVerifyStatFloats) + 2; }
+
 struct FieldWs {
   size_t wq, xq, xbar, ybar, bq, dtil, acc64, total;
 };
@@ -1314,7 +1620,7 @@ dk_status dk_field_linear_fwd(dk_ctx* ctx, const dk_problem* p, uint32_t prime, 
   if (!dg.ok) return DK_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
-  return launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, st);
+  return launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, field_status_word(ctx), st);
 }
 
 dk_status dk_field_decode_verify(dk_ctx* ctx, const dk_problem* p, uint32_t prime, int32_t l,
@@ -1383,7 +1689,7 @@ dk_status dk_field_masked_linear(dk_ctx* ctx, const dk_problem* p, uint32_t prim
   if (s != DK_OK) return s;
   {
     ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
-    s = launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, st);
+    s = launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, field_status_word(ctx), st);
   }
   if (s != DK_OK) return s;
   if (fault) {
