@@ -799,17 +799,18 @@ __global__ void __launch_bounds__(kMmaThreads, 1) field_fwd_mma_kernel(FwdParams
 // seven weight-class sums live in tensor memory (7 x 64 columns of s32).
 //
 //   tile: 128 output channels (TMEM lanes) x 64 pixels, k-tiles of 128 elements
-//   all 8 warps: load residues (16-byte groups of one filter tap), split them
+//   all 16 warps: load residues (16-byte groups of one filter tap), split them
 //                into digit planes, store the planes swizzled; two stages
 //   thread 0:    64 MMAs per k-tile (16 digit pairs x 4 k-steps of 32), commit
-//   all 8 warps: at the end (and every 64 k-tiles, before a class sum can pass
-//                2^31) read the class sums with tcgen05.ld and fold them mod p
+//   all 16 warps: at the end (and every 64 k-tiles, before a class sum can pass
+//                2^31) read the class sums with tcgen05.ld and fold them mod p;
+//                between two folds the partial residues wait in the output buffer
 // Every mbarrier wait is bounded; on expiry the CTA stops issuing, reports
 // DK_ERR_TIMEOUT in *status, still frees its tensor memory and returns.
 // ---------------------------------------------------------------------------
 namespace tcf {
 constexpr int TM = 128, TN = 64, TK = 128;
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 constexpr int A_PLANE = TM * TK, B_PLANE = TN * TK;              // bytes per digit plane
 constexpr int STAGE = 4 * A_PLANE + 4 * B_PLANE;                 // 96 KB
 constexpr int kStages = 2;
@@ -920,11 +921,9 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_slot[0];
 
-  // this thread's part of the result: TMEM lane (output channel) 32*(warp & 3) + lane, columns 32*(warp >> 2) ..
+  // this thread's part of the result: TMEM lane (output channel) 32*(warp & 3) + lane, columns 16*(warp >> 2) ..
   const int q = warp & 3, h = warp >> 2;
-  u32 tot[32];
-#pragma unroll
-  for (int j = 0; j < 32; ++j) tot[j] = 0;
+  bool folded = false;           // a partial result is already in y
 
   // S32 accumulator, unsigned 8-bit A and B, both K-major, N = 64, M = 128
   constexpr uint32_t idesc = (2u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(TN >> 3) << 17) |
@@ -963,33 +962,42 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
           }
         }
       }
-      for (int uidx = t; uidx < (TM + TN) * 8; uidx += kThreads) {
+      constexpr int UPT = (TM + TN) * 8 / kThreads;      // units per thread
+      uint4 w[UPT][4];
+#pragma unroll
+      for (int ui = 0; ui < UPT; ++ui) {                 // all loads first: one exposed latency per k-tile
+        const int uidx = t + ui * kThreads;
         const bool isA = uidx < TM * 8;
         const int row = isA ? (uidx >> 3) : ((uidx - TM * 8) >> 3);
-        uint4 w[4];
         if (isA) {
           const bool rok = m0 + row < p.cout;
           const u32* wr = p.W + (long long)(m0 + row) * p.ws_o;
 #pragma unroll
           for (int gq = 0; gq < 4; ++gq)
-            w[gq] = (rok && g_ok[gq])
-                        ? __ldg(reinterpret_cast<const uint4*>(wr + g_ci[gq] + (long long)g_u[gq] * p.ws_u +
-                                                               (long long)g_v[gq] * p.ws_v))
-                        : make_uint4(0u, 0u, 0u, 0u);
+            w[ui][gq] = (rok && g_ok[gq])
+                            ? __ldg(reinterpret_cast<const uint4*>(wr + g_ci[gq] + (long long)g_u[gq] * p.ws_u +
+                                                                   (long long)g_v[gq] * p.ws_v))
+                            : make_uint4(0u, 0u, 0u, 0u);
         } else {
           const RowInfo ri = rows[row];
 #pragma unroll
           for (int gq = 0; gq < 4; ++gq) {
             const int ih = ri.ih0 + g_u[gq], iw = ri.iw0 + g_v[gq];
             const bool ok = g_ok[gq] && ri.base >= 0 && ih >= 0 && ih < p.h && iw >= 0 && iw < p.w;
-            w[gq] = ok ? __ldg(reinterpret_cast<const uint4*>(p.x + ri.base + g_ci[gq] + (long long)ih * p.xs_h +
-                                                              (long long)iw * p.xs_w))
-                       : make_uint4(0u, 0u, 0u, 0u);
+            w[ui][gq] = ok ? __ldg(reinterpret_cast<const uint4*>(p.x + ri.base + g_ci[gq] +
+                                                                  (long long)ih * p.xs_h + (long long)iw * p.xs_w))
+                           : make_uint4(0u, 0u, 0u, 0u);
           }
         }
+      }
+#pragma unroll
+      for (int ui = 0; ui < UPT; ++ui) {
+        const int uidx = t + ui * kThreads;
+        const bool isA = uidx < TM * 8;
+        const int row = isA ? (uidx >> 3) : ((uidx - TM * 8) >> 3);
         u32 pl[4][4];      // [group of four elements][digit]
 #pragma unroll
-        for (int gq = 0; gq < 4; ++gq) digit_planes(w[gq], pl[gq]);
+        for (int gq = 0; gq < 4; ++gq) digit_planes(w[ui][gq], pl[gq]);
         uint8_t* base = st + (isA ? 0 : 4 * A_PLANE) + row * TK + ((c ^ (row & 7)) << 4);
         const int plane = isA ? A_PLANE : B_PLANE;
 #pragma unroll
@@ -1032,33 +1040,28 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
       if (*abort_flag) alive = false;
       if (alive) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int m = m0 + q * 32 + lane;
 #pragma unroll
-        for (int cg = 0; cg < 4; ++cg) {
+        for (int cg = 0; cg < 2; ++cg) {
           int cls[7][8];
 #pragma unroll
           for (int c = 0; c < 7; ++c)
-            ld8(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * TN + h * 32 + cg * 8), cls[c]);
+            ld8(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * TN + h * 16 + cg * 8), cls[c]);
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
+            const long long oo = out_off[h * 16 + cg * 8 + j];
+            if (oo < 0 || m >= p.cout) continue;
+            u32* dst = p.y + oo + (long long)m * p.ys_c;
             const int cc[7] = {cls[0][j], cls[1][j], cls[2][j], cls[3][j], cls[4][j], cls[5][j], cls[6][j]};
-            tot[cg * 8 + j] = fold_classes(tot[cg * 8 + j], cc, p.md, mc.pow32);
+            *dst = fold_classes(folded ? *dst : 0u, cc, p.md, mc.pow32);
           }
         }
+        folded = true;
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       }
       __syncthreads();
       started = 0;
-    }
-  }
-  if (alive) {
-    const int m = m0 + q * 32 + lane;
-    if (m < p.cout) {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const long long oo = out_off[h * 32 + j];
-        if (oo >= 0) p.y[oo + (long long)m * p.ys_c] = tot[j];
-      }
     }
   }
   __syncthreads();
