@@ -872,7 +872,33 @@ __device__ __forceinline__ uint64_t plane_desc(uint32_t smem_addr) {
 }
 }  // namespace tcf
 
-__global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParams p, MmaConsts mc, int* status) {
+// W as four digit planes, [digit][cout][kcp] bytes with kcp = kc rounded up to the k-tile (zero filled):
+// written once per call, so that every CTA fetches its rows of W as ready 16-byte chunks.
+__global__ void __launch_bounds__(256) field_w_planes_kernel(const u32* __restrict__ W, int cout, int kc, int kcp,
+                                                            uint8_t* __restrict__ planes) {
+  const long long chunks = (long long)cout * (kcp / 16);
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < chunks; i += stride) {
+    const int m = (int)(i / (kcp / 16));
+    const int k0 = (int)(i - (long long)m * (kcp / 16)) * 16;
+    u32 pl[4][4];
+#pragma unroll
+    for (int gq = 0; gq < 4; ++gq) {
+      const int k = k0 + gq * 4;
+      const uint4 w = k < kc ? __ldg(reinterpret_cast<const uint4*>(W + (long long)m * kc + k))
+                             : make_uint4(0u, 0u, 0u, 0u);
+      digit_planes(w, pl[gq]);
+    }
+#pragma unroll
+    for (int dg = 0; dg < 4; ++dg)
+      *reinterpret_cast<uint4*>(planes + ((long long)dg * cout + m) * kcp + k0) =
+          make_uint4(pl[0][dg], pl[1][dg], pl[2][dg], pl[3][dg]);
+  }
+}
+
+__global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParams p, MmaConsts mc,
+                                                                       const uint8_t* __restrict__ wplanes, int kcp,
+                                                                       int* status) {
   using namespace tcf;
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t mma_done[kStages];
@@ -962,48 +988,41 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
           }
         }
       }
-      constexpr int UPT = (TM + TN) * 8 / kThreads;      // units per thread
-      uint4 w[UPT][4];
+      // rows of W: ready digit planes, copied asynchronously chunk by chunk into the swizzled layout
 #pragma unroll
-      for (int ui = 0; ui < UPT; ++ui) {                 // all loads first: one exposed latency per k-tile
-        const int uidx = t + ui * kThreads;
-        const bool isA = uidx < TM * 8;
-        const int row = isA ? (uidx >> 3) : ((uidx - TM * 8) >> 3);
-        if (isA) {
-          const bool rok = m0 + row < p.cout;
-          const u32* wr = p.W + (long long)(m0 + row) * p.ws_o;
-#pragma unroll
-          for (int gq = 0; gq < 4; ++gq)
-            w[ui][gq] = (rok && g_ok[gq])
-                            ? __ldg(reinterpret_cast<const uint4*>(wr + g_ci[gq] + (long long)g_u[gq] * p.ws_u +
-                                                                   (long long)g_v[gq] * p.ws_v))
-                            : make_uint4(0u, 0u, 0u, 0u);
-        } else {
-          const RowInfo ri = rows[row];
-#pragma unroll
-          for (int gq = 0; gq < 4; ++gq) {
-            const int ih = ri.ih0 + g_u[gq], iw = ri.iw0 + g_v[gq];
-            const bool ok = g_ok[gq] && ri.base >= 0 && ih >= 0 && ih < p.h && iw >= 0 && iw < p.w;
-            w[ui][gq] = ok ? __ldg(reinterpret_cast<const uint4*>(p.x + ri.base + g_ci[gq] +
-                                                                  (long long)ih * p.xs_h + (long long)iw * p.xs_w))
-                           : make_uint4(0u, 0u, 0u, 0u);
-          }
-        }
+      for (int i = 0; i < 4 * TM * 8 / kThreads; ++i) {
+        const int idx = t + i * kThreads;            // (digit, row, chunk)
+        const int dg = idx / (TM * 8), row = (idx >> 3) & (TM - 1);
+        const bool rok = m0 + row < p.cout;
+        const uint8_t* src = wplanes + ((long long)dg * p.cout + (rok ? m0 + row : 0)) * kcp + kt * TK + c * 16;
+        const unsigned dst = smem_u32(st + dg * A_PLANE + row * TK + ((c ^ (row & 7)) << 4));
+        const int nbytes = rok ? 16 : 0;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(nbytes));
       }
+      asm volatile("cp.async.commit_group;\n" ::);
+      // pixels of x: one unit of 16 contraction elements per thread
+      {
+        static_assert(TN * 8 == kThreads, "one x unit per thread");
+        const int row = t >> 3;
+        const RowInfo ri = rows[row];
+        uint4 w[4];
 #pragma unroll
-      for (int ui = 0; ui < UPT; ++ui) {
-        const int uidx = t + ui * kThreads;
-        const bool isA = uidx < TM * 8;
-        const int row = isA ? (uidx >> 3) : ((uidx - TM * 8) >> 3);
+        for (int gq = 0; gq < 4; ++gq) {
+          const int ih = ri.ih0 + g_u[gq], iw = ri.iw0 + g_v[gq];
+          const bool ok = g_ok[gq] && ri.base >= 0 && ih >= 0 && ih < p.h && iw >= 0 && iw < p.w;
+          w[gq] = ok ? __ldg(reinterpret_cast<const uint4*>(p.x + ri.base + g_ci[gq] + (long long)ih * p.xs_h +
+                                                            (long long)iw * p.xs_w))
+                     : make_uint4(0u, 0u, 0u, 0u);
+        }
         u32 pl[4][4];      // [group of four elements][digit]
 #pragma unroll
-        for (int gq = 0; gq < 4; ++gq) digit_planes(w[ui][gq], pl[gq]);
-        uint8_t* base = st + (isA ? 0 : 4 * A_PLANE) + row * TK + ((c ^ (row & 7)) << 4);
-        const int plane = isA ? A_PLANE : B_PLANE;
+        for (int gq = 0; gq < 4; ++gq) digit_planes(w[gq], pl[gq]);
+        uint8_t* base = st + 4 * A_PLANE + row * TK + ((c ^ (row & 7)) << 4);
 #pragma unroll
         for (int dg = 0; dg < 4; ++dg)
-          *reinterpret_cast<uint4*>(base + dg * plane) = make_uint4(pl[0][dg], pl[1][dg], pl[2][dg], pl[3][dg]);
+          *reinterpret_cast<uint4*>(base + dg * B_PLANE) = make_uint4(pl[0][dg], pl[1][dg], pl[2][dg], pl[3][dg]);
       }
+      asm volatile("cp.async.wait_group 0;\n" ::);
       // make the planes visible to the tensor core's (asynchronous-proxy) reads
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -1103,8 +1122,10 @@ bool field_use_mma_sync() {
   return v;
 }
 
+// `wplanes` (nullable): device scratch of at least 4 * cout * round_up(kc, 128) bytes for the digit planes of W;
+// without it the contraction runs on the mma.sync kernel.
 dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* ybar, int nsamples, Modulus md,
-                           int* status, cudaStream_t st) {
+                           uint8_t* wplanes, size_t wplanes_bytes, int* status, cudaStream_t st) {
   FwdParams p;
   p.W = W; p.x = xbar; p.y = ybar;
   p.cin = g.cin; p.cout = g.cout; p.h = g.h; p.w = g.w; p.kw = g.kw; p.stride = g.stride;
@@ -1130,14 +1151,18 @@ dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* yb
     MmaConsts mc;
     mc.pow32 = (u32)((1ull << 32) % md.p);
     const bool vec4 = g.xs_c == 1 && g.ws_c == 1 && (g.cin % 4) == 0 && aligned16(W) && aligned16(xbar);
-    if (vec4 && !field_use_mma_sync()) {
+    const int kcp = (g.kc + tcf::TK - 1) / tcf::TK * tcf::TK;
+    if (vec4 && !field_use_mma_sync() && wplanes != nullptr && wplanes_bytes >= (size_t)4 * g.cout * kcp) {
       static const bool tc_attr_ok =
           cudaFuncSetAttribute(field_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)tcf::kSmem) == cudaSuccess;
       if (!tc_attr_ok) return DK_ERR_CUDA;
       const long long tnb = (p.N + tcf::TN - 1) / tcf::TN;
       dim3 tgrid((unsigned)tnb, (unsigned)((g.cout + tcf::TM - 1) / tcf::TM));
-      field_fwd_tc_kernel<<<tgrid, tcf::kThreads, tcf::kSmem, st>>>(p, mc, status);
+      const long long chunks = (long long)g.cout * (kcp / 16);
+      field_w_planes_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(W, g.cout, g.kc, kcp, wplanes);
+      DK_CUDA_CHECK(cudaGetLastError());
+      field_fwd_tc_kernel<<<tgrid, tcf::kThreads, tcf::kSmem, st>>>(p, mc, wplanes, kcp, status);
       DK_CUDA_CHECK(cudaGetLastError());
       return DK_OK;
     }
@@ -1467,7 +1492,7 @@ int ew_blocks(long long n, int sm_count) {
 int* field_status_word(dk_ctx* ctx) { return reinterpret_cast<int*>(ctx->d_vstats + kVerifyStatFloats) + 2; }
 
 struct FieldWs {
-  size_t wq, xq, xbar, ybar, bq, dtil, acc64, total;
+  size_t wq, wpl, wpl_bytes, xq, xbar, ybar, bq, dtil, acc64, total;
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -1476,6 +1501,8 @@ FieldWs plan_field_ws(const Geom& g) {
   FieldWs w;
   size_t off = 0;
   w.wq = off; off += align_up((size_t)g.cout * g.kc * sizeof(u32), 1024);
+  w.wpl_bytes = (size_t)4 * g.cout * ((g.kc + 127) / 128 * 128);      // digit planes of W_q
+  w.wpl = off; off += align_up(w.wpl_bytes, 1024);
   w.xq = off; off += align_up((size_t)g.G * g.K * g.n_in * sizeof(u32), 1024);
   w.xbar = off; off += align_up((size_t)g.G * g.E * g.n_in * sizeof(u32), 1024);
   w.ybar = off; off += align_up((size_t)g.G * g.E * g.n_out * sizeof(u32), 1024);
@@ -1623,7 +1650,11 @@ dk_status dk_field_linear_fwd(dk_ctx* ctx, const dk_problem* p, uint32_t prime, 
   if (!dg.ok) return DK_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
-  return launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, field_status_word(ctx), st);
+  const FieldWs wp = plan_field_ws(g);
+  const bool have_ws = ctx->ws && ctx->ws_bytes >= wp.total;
+  return launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md,
+                          have_ws ? reinterpret_cast<uint8_t*>(static_cast<char*>(ctx->ws) + wp.wpl) : nullptr,
+                          have_ws ? wp.wpl_bytes : 0, field_status_word(ctx), st);
 }
 
 dk_status dk_field_decode_verify(dk_ctx* ctx, const dk_problem* p, uint32_t prime, int32_t l,
@@ -1692,7 +1723,8 @@ dk_status dk_field_masked_linear(dk_ctx* ctx, const dk_problem* p, uint32_t prim
   if (s != DK_OK) return s;
   {
     ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
-    s = launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, field_status_word(ctx), st);
+    s = launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, reinterpret_cast<uint8_t*>(ws + wp.wpl), wp.wpl_bytes,
+                         field_status_word(ctx), st);
   }
   if (s != DK_OK) return s;
   if (fault) {
