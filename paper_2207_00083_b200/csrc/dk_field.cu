@@ -799,10 +799,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) field_fwd_mma_kernel(FwdParams
 // seven weight-class sums live in tensor memory (7 x 64 columns of s32).
 //
 //   tile: 128 output channels (TMEM lanes) x 64 pixels, k-tiles of 128 elements
-//   all 16 warps: load residues (16-byte groups of one filter tap), split them
-//                into digit planes, store the planes swizzled; two stages
-//   thread 0:    64 MMAs per k-tile (16 digit pairs x 4 k-steps of 32), commit
-//   all 16 warps: at the end (and every 64 k-tiles, before a class sum can pass
+//   16 producer warps: fetch W's digit planes (cp.async), load residues of x
+//                (16-byte groups of one filter tap), split them into digit planes,
+//                store the planes swizzled; two stages, handed over by mbarriers
+//   one thread of a 17th warp: 64 MMAs per k-tile (16 digit pairs x 4 k-steps of 32), commit
+//   the producer warps: at the end (and every 64 k-tiles, before a class sum can pass
 //                2^31) read the class sums with tcgen05.ld and fold them mod p;
 //                between two folds the partial residues wait in the output buffer
 // Every mbarrier wait is bounded; on expiry the CTA stops issuing, reports
@@ -810,7 +811,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) field_fwd_mma_kernel(FwdParams
 // ---------------------------------------------------------------------------
 namespace tcf {
 constexpr int TM = 128, TN = 64, TK = 128;
-constexpr int kThreads = 512;
+constexpr int kProducers = 512;                 // 16 warps fill the stages and read the sums
+constexpr int kThreads = kProducers + 32;       // + one warp whose first lane issues the products
 constexpr int A_PLANE = TM * TK, B_PLANE = TN * TK;              // bytes per digit plane
 constexpr int STAGE = 4 * A_PLANE + 4 * B_PLANE;                 // 96 KB
 constexpr int kStages = 2;
@@ -901,7 +903,8 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
                                                                        int* status) {
   using namespace tcf;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t mma_done[kStages];
+  __shared__ uint64_t full_bar[kStages];     // a stage's planes are in shared memory (kProducers arrivals)
+  __shared__ uint64_t mma_done[kStages];     // the products that read a stage have completed (one commit)
   __shared__ uint32_t tmem_slot[2];          // [0] TMEM base address, [1] abort flag
   __shared__ RowInfo rows[TN];
   __shared__ long long out_off[TN];
@@ -913,7 +916,7 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
   const long long n0 = (long long)blockIdx.x * TN;
 
   if (t == 0) {
-    for (int s = 0; s < kStages; ++s) mbar_init(mma_done + s, 1);
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar + s, kProducers); mbar_init(mma_done + s, 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -946,29 +949,53 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_slot[0];
-
-  // this thread's part of the result: TMEM lane (output channel) 32*(warp & 3) + lane, columns 16*(warp >> 2) ..
-  const int q = warp & 3, h = warp >> 2;
-  bool folded = false;           // a partial result is already in y
-
-  // S32 accumulator, unsigned 8-bit A and B, both K-major, N = 64, M = 128
-  constexpr uint32_t idesc = (2u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(TN >> 3) << 17) |
-                             ((uint32_t)(TM >> 4) << 24);
-
   const int ntiles = (p.kc + TK - 1) / TK;
-  uint32_t started = 0;                // bit c: class c has received its first product since the last fold
-  bool alive = true;
-  for (int kt = 0; kt < ntiles; ++kt) {
-    const int stage = kt & 1;
-    uint8_t* st = smem + (size_t)stage * STAGE;
-    // the products that read this stage two k-tiles ago must have completed
-    if (kt >= kStages) {
-      if (!mbar_wait(mma_done + stage, (uint32_t)((kt / kStages - 1) & 1), abort_flag)) alive = false;
+
+  if (warp == kProducers / 32) {
+    // ---------------- MMA issuer: one thread ----------------
+    if (lane == 0) {
+      // S32 accumulator, unsigned 8-bit A and B, both K-major, N = 64, M = 128
+      constexpr uint32_t idesc = (2u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(TN >> 3) << 17) |
+                                 ((uint32_t)(TM >> 4) << 24);
+      uint32_t started = 0;            // bit c: class c has received its first product since the last fold
+      for (int kt = 0; kt < ntiles; ++kt) {
+        const int stage = kt & 1;
+        if (!mbar_wait(full_bar + stage, (uint32_t)((kt / kStages) & 1), abort_flag)) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE), sb = sa + 4 * A_PLANE;
+#pragma unroll
+        for (int ks = 0; ks < TK / 32; ++ks) {
+          const uint64_t adv = (uint64_t)(ks * 2);       // 32 bytes per k-step, in 16-byte units
+#pragma unroll
+          for (int da = 0; da < 4; ++da)
+#pragma unroll
+            for (int db = 0; db < 4; ++db) {
+              const int c = da + db;
+              mma_i8(tmem_base + (uint32_t)(c * TN), plane_desc(sa + da * A_PLANE) + adv,
+                     plane_desc(sb + db * B_PLANE) + adv, idesc, (started >> c) & 1u);
+              started |= 1u << c;
+            }
+        }
+        commit(mma_done + stage);
+        if (((kt + 1) % kFoldTiles) == 0) started = 0;      // the producers fold and restart the sums here
+      }
     }
-    if (alive) {
-      // units of 16 contraction elements of one row: 128 rows of W, then 64 pixels of x.  A thread's
-      // units all sit in the same 16-element column c = t & 7 of the k-tile, so the filter taps of its
-      // four 4-element groups are worked out once per k-tile.
+  } else {
+    // ---------------- producers (and, at a fold, readers of the sums): 16 warps ----------------
+    // this thread's part of the result: TMEM lane (output channel) 32*(warp & 3) + lane, columns 16*(warp >> 2) ..
+    const int q = warp & 3, h = warp >> 2;
+    bool folded = false;           // a partial result is already in y
+    bool alive = true;
+    for (int kt = 0; alive && kt < ntiles; ++kt) {
+      const int stage = kt & 1;
+      uint8_t* st = smem + (size_t)stage * STAGE;
+      // the products that read this stage two k-tiles ago must have completed
+      if (kt >= kStages && !mbar_wait(mma_done + stage, (uint32_t)((kt / kStages - 1) & 1), abort_flag)) {
+        alive = false;
+        break;
+      }
+      // units of 16 contraction elements of one row.  A thread's units all sit in the same 16-element
+      // column c = t & 7 of the k-tile, so the filter taps of its four 4-element groups are worked out once.
       const int c = t & 7;
       int g_ci[4], g_u[4], g_v[4];
       bool g_ok[4];
@@ -990,8 +1017,8 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
       }
       // rows of W: ready digit planes, copied asynchronously chunk by chunk into the swizzled layout
 #pragma unroll
-      for (int i = 0; i < 4 * TM * 8 / kThreads; ++i) {
-        const int idx = t + i * kThreads;            // (digit, row, chunk)
+      for (int i = 0; i < 4 * TM * 8 / kProducers; ++i) {
+        const int idx = t + i * kProducers;            // (digit, row, chunk)
         const int dg = idx / (TM * 8), row = (idx >> 3) & (TM - 1);
         const bool rok = m0 + row < p.cout;
         const uint8_t* src = wplanes + ((long long)dg * p.cout + (rok ? m0 + row : 0)) * kcp + kt * TK + c * 16;
@@ -1002,7 +1029,7 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
       asm volatile("cp.async.commit_group;\n" ::);
       // pixels of x: one unit of 16 contraction elements per thread
       {
-        static_assert(TN * 8 == kThreads, "one x unit per thread");
+        static_assert(TN * 8 == kProducers, "one x unit per thread");
         const int row = t >> 3;
         const RowInfo ri = rows[row];
         uint4 w[4];
@@ -1023,41 +1050,19 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
           *reinterpret_cast<uint4*>(base + dg * B_PLANE) = make_uint4(pl[0][dg], pl[1][dg], pl[2][dg], pl[3][dg]);
       }
       asm volatile("cp.async.wait_group 0;\n" ::);
-      // make the planes visible to the tensor core's (asynchronous-proxy) reads
+      // make the planes visible to the tensor core's (asynchronous-proxy) reads, then hand the stage over
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncthreads();
-    if (*abort_flag) alive = false;
-    if (alive && t == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t sa = smem_u32(st), sb = sa + 4 * A_PLANE;
-#pragma unroll
-      for (int ks = 0; ks < TK / 32; ++ks) {
-        const uint64_t adv = (uint64_t)(ks * 2);       // 32 bytes per k-step, in 16-byte units
-#pragma unroll
-        for (int da = 0; da < 4; ++da)
-#pragma unroll
-          for (int db = 0; db < 4; ++db) {
-            const int c = da + db;
-            mma_i8(tmem_base + (uint32_t)(c * TN), plane_desc(sa + da * A_PLANE) + adv,
-                   plane_desc(sb + db * B_PLANE) + adv, idesc, (started >> c) & 1u);
-            started |= 1u << c;
-          }
-      }
-      commit(mma_done + stage);
-    }
-    // fold before a class sum can overflow, and at the end
-    const bool last = kt + 1 == ntiles;
-    if (last || ((kt + 1) % kFoldTiles) == 0) {
-      // every product issued so far: the newest commit of each stage in use
-      const int kprev = kt - 1;
-      if (alive && kprev >= 0 &&
-          !mbar_wait(mma_done + (kprev & 1), (uint32_t)((kprev / kStages) & 1), abort_flag))
-        alive = false;
-      if (alive && !mbar_wait(mma_done + stage, (uint32_t)((kt / kStages) & 1), abort_flag)) alive = false;
-      __syncthreads();
-      if (*abort_flag) alive = false;
-      if (alive) {
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(full_bar + stage)) : "memory");
+
+      // fold before a class sum can overflow, and at the end
+      const bool last = kt + 1 == ntiles;
+      if (last || ((kt + 1) % kFoldTiles) == 0) {
+        // every product issued so far has completed once the commit of this k-tile has arrived
+        // (a commit covers all earlier products of the issuing thread)
+        if (!mbar_wait(mma_done + stage, (uint32_t)((kt / kStages) & 1), abort_flag)) {
+          alive = false;
+          break;
+        }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int m = m0 + q * 32 + lane;
 #pragma unroll
@@ -1077,10 +1082,9 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
           }
         }
         folded = true;
+        // the next arrival on a full barrier orders these reads before the products that overwrite the sums
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       }
-      __syncthreads();
-      started = 0;
     }
   }
   __syncthreads();
