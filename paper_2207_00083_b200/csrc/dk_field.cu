@@ -954,30 +954,40 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
   if (warp == kProducers / 32) {
     // ---------------- MMA issuer: one thread ----------------
     if (lane == 0) {
-      // S32 accumulator, unsigned 8-bit A and B, both K-major, N = 64, M = 128
-      constexpr uint32_t idesc = (2u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(TN >> 3) << 17) |
-                                 ((uint32_t)(TM >> 4) << 24);
-      uint32_t started = 0;            // bit c: class c has received its first product since the last fold
+      // S32 accumulator, unsigned 8-bit A and B, both K-major, M = 128; N = 64 columns per weight class.
+      // The four digit planes of x lie one after the other in shared memory, so W's digit a against ALL of
+      // them is one instruction with N = 256 whose result columns are the classes a .. a+3, which are
+      // adjacent in tensor memory too: four instructions per k-step instead of sixteen.  Only the first
+      // k-step after a fold, where some of those classes must be overwritten and others added to, is split.
+      auto idesc_n = [](int n) {
+        return (2u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+      };
+      bool fresh = true;               // no product since the last fold
       for (int kt = 0; kt < ntiles; ++kt) {
         const int stage = kt & 1;
         if (!mbar_wait(full_bar + stage, (uint32_t)((kt / kStages) & 1), abort_flag)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE), sb = sa + 4 * A_PLANE;
+        const uint64_t bdesc = plane_desc(sb);
 #pragma unroll
         for (int ks = 0; ks < TK / 32; ++ks) {
           const uint64_t adv = (uint64_t)(ks * 2);       // 32 bytes per k-step, in 16-byte units
 #pragma unroll
-          for (int da = 0; da < 4; ++da)
-#pragma unroll
-            for (int db = 0; db < 4; ++db) {
-              const int c = da + db;
-              mma_i8(tmem_base + (uint32_t)(c * TN), plane_desc(sa + da * A_PLANE) + adv,
-                     plane_desc(sb + db * B_PLANE) + adv, idesc, (started >> c) & 1u);
-              started |= 1u << c;
+          for (int da = 0; da < 4; ++da) {
+            const uint64_t adesc = plane_desc(sa + da * A_PLANE) + adv;
+            const uint32_t d = tmem_base + (uint32_t)(da * TN);
+            if (fresh && ks == 0 && da > 0) {
+              // classes da .. da+2 have a product already, class da+3 has none
+              mma_i8(d, adesc, bdesc + adv, idesc_n(3 * TN), 1u);
+              mma_i8(d + 3 * TN, adesc, plane_desc(sb + 3 * B_PLANE) + adv, idesc_n(TN), 0u);
+            } else {
+              mma_i8(d, adesc, bdesc + adv, idesc_n(4 * TN), (fresh && ks == 0) ? 0u : 1u);
             }
+          }
         }
+        fresh = false;
         commit(mma_done + stage);
-        if (((kt + 1) % kFoldTiles) == 0) started = 0;      // the producers fold and restart the sums here
+        if (((kt + 1) % kFoldTiles) == 0) fresh = true;      // the producers fold and restart the sums here
       }
     }
   } else {
