@@ -304,7 +304,13 @@ DK_API dk_status dk_field_encode(dk_ctx* ctx, const dk_problem* p, uint32_t prim
 /* The bilinear operation of Section 4.1 on residues (step "GPUs compute" of
  * Algorithm 1): ybar = <Wq, xbar> modulo p for all G*(K+2) encoded samples,
  * FC or convolution as in dk_linear_fwd, every layout and stride.  Exact:
- * products are accumulated in 64 bits and reduced before they can overflow. */
+ * residues are multiplied digit by digit (base 256) on the integer tensor
+ * cores and the partial sums reduced modulo p before they can overflow.
+ * Shapes with contiguous channels (DK_FC, DK_NHWC with cin % 4 == 0) run on
+ * the tcgen05 path when a workspace of dk_field_workspace_bytes is registered
+ * (it holds W_q's digit planes); others, or calls without a workspace, run
+ * on the mma.sync path.  A bounded device-side wait that expires is reported
+ * by dk_device_status as DK_ERR_TIMEOUT. */
 DK_API dk_status dk_field_linear_fwd(dk_ctx* ctx, const dk_problem* p, uint32_t prime, const uint32_t* Wq,
                                      const uint32_t* xbar, uint32_t* ybar, void* stream);
 

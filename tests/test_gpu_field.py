@@ -33,6 +33,7 @@ CASES = [
     ("fc784", synth.layers("fc784")[0], dk.DK_NHWC),
     ("fc_ragged_K1", tiny("fc", cin=37, cout=19, K=1, G=3), dk.DK_NHWC),
     ("fc_K8_long", tiny("fc", cin=20011, cout=70, K=8, G=1), dk.DK_NHWC),     # several reductions per sum
+    ("fc_long_tc", tiny("fc", cin=20012, cout=130, K=2, G=1), dk.DK_NHWC),    # tcgen05 kernel: folds at 8192 and 16384
     ("conv_tiny_K2", tiny(), dk.DK_NHWC),
     ("conv_ragged_K3_nchw", tiny(cin=5, cout=7, h=6, w=5, K=3, G=2), dk.DK_NCHW),
     ("conv_7x7s2_stem", tiny(cin=3, cout=16, h=20, w=20, kh=7, kw=7, stride=2, pad=3, K=4, G=1), dk.DK_NHWC),
@@ -312,14 +313,17 @@ def test_full_size_layer_sampled_against_the_oracle(ctx, layer):
         assert dWq[co, ci, u, vv] == F.field_wgrad_plain_at(dq, xq, co, ci, u, vv, P, spec.stride, spec.pad)
 
 
-def test_integer_alu_kernels_give_the_same_residues():
-    """DK_FIELD_SIMT=1 selects the 64-bit integer-ALU contraction kernels instead of the tensor-core ones
-    (the switch is read once per process): a few parity cases re-run in a child process under it."""
-    if os.environ.get("DK_FIELD_SIMT") == "1":
+@pytest.mark.parametrize("switch", ["DK_FIELD_SIMT", "DK_FIELD_MMA_SYNC"])
+def test_cross_check_kernels_give_the_same_residues(switch):
+    """DK_FIELD_SIMT=1 selects the 64-bit integer-ALU contraction kernels, DK_FIELD_MMA_SYNC=1 keeps the forward
+    contraction on the mma.sync kernel instead of the tcgen05 one (both switches are read once per process):
+    a few parity cases re-run in a child process under each."""
+    if os.environ.get(switch) == "1":
         pytest.skip("already running under the switch")
-    env = dict(os.environ, DK_FIELD_SIMT="1")
+    env = dict(os.environ, **{switch: "1"})
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", os.path.abspath(__file__), "-k",
-                        "conv_tiny_K2 or fc_K8_long or conv_3x3s2_K5 or conv_ragged_K3_nchw or other_primes"],
-                       cwd=root, env=env, capture_output=True, text=True, timeout=600)
+                        "conv_tiny_K2 or fc_K8_long or conv_3x3s2_K5 or conv_ragged_K3_nchw or other_primes "
+                        "or vgg_cifar_conv3_1"],
+                       cwd=root, env=env, capture_output=True, text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
