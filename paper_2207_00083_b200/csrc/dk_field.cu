@@ -900,6 +900,7 @@ __global__ void __launch_bounds__(256) field_w_planes_kernel(const u32* __restri
 
 __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParams p, MmaConsts mc,
                                                                        const uint8_t* __restrict__ wplanes, int kcp,
+                                                                       u64* split_acc, int tiles_per_split,
                                                                        int* status) {
   using namespace tcf;
   extern __shared__ uint8_t smem_raw[];
@@ -949,7 +950,10 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_slot[0];
-  const int ntiles = (p.kc + TK - 1) / TK;
+  // this CTA's slice of the contraction: k-tiles kt0 .. kt0 + ntiles - 1 (the whole of it unless the launch
+  // is split; slices meet as residues in split_acc, a uint64 per output element that the caller cleared)
+  const int kt0 = blockIdx.z * tiles_per_split;
+  const int ntiles = min(tiles_per_split, (p.kc + TK - 1) / TK - kt0);
 
   if (warp == kProducers / 32) {
     // ---------------- MMA issuer: one thread ----------------
@@ -1010,7 +1014,7 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
       int g_ci[4], g_u[4], g_v[4];
       bool g_ok[4];
       {
-        int k = kt * TK + c * 16;
+        int k = (kt0 + kt) * TK + c * 16;
         int tap = k / p.cin;
         int ci = k - tap * p.cin;
         int u = tap / p.kw, v = tap - u * p.kw;
@@ -1031,7 +1035,7 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
         const int idx = t + i * kProducers;            // (digit, row, chunk)
         const int dg = idx / (TM * 8), row = (idx >> 3) & (TM - 1);
         const bool rok = m0 + row < p.cout;
-        const uint8_t* src = wplanes + ((long long)dg * p.cout + (rok ? m0 + row : 0)) * kcp + kt * TK + c * 16;
+        const uint8_t* src = wplanes + ((long long)dg * p.cout + (rok ? m0 + row : 0)) * kcp + (kt0 + kt) * TK + c * 16;
         const unsigned dst = smem_u32(st + dg * A_PLANE + row * TK + ((c ^ (row & 7)) << 4));
         const int nbytes = rok ? 16 : 0;
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(nbytes));
@@ -1088,7 +1092,8 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
             if (oo < 0 || m >= p.cout) continue;
             u32* dst = p.y + oo + (long long)m * p.ys_c;
             const int cc[7] = {cls[0][j], cls[1][j], cls[2][j], cls[3][j], cls[4][j], cls[5][j], cls[6][j]};
-            *dst = fold_classes(folded ? *dst : 0u, cc, p.md, mc.pow32);
+            if (split_acc != nullptr) atomicAdd(split_acc + (dst - p.y), (u64)fold_classes(0u, cc, p.md, mc.pow32));
+            else *dst = fold_classes(folded ? *dst : 0u, cc, p.md, mc.pow32);
           }
         }
         folded = true;
@@ -1138,8 +1143,29 @@ bool field_use_mma_sync() {
 
 // `wplanes` (nullable): device scratch of at least 4 * cout * round_up(kc, 128) bytes for the digit planes of W;
 // without it the contraction runs on the mma.sync kernel.
+__global__ void field_reduce_kernel(const u64* __restrict__ acc, long long n, Modulus md, u32* __restrict__ out);
+int ew_blocks(long long n, int sm_count);
+
+// Slices of the contraction for the tcgen05 kernel: `ctas` output tiles of `ntiles` k-tiles on `sms` SMs.
+// Cost of ns slices = rounds of CTAs x (k-tiles per slice + a fixed part of about three k-tiles for set-up,
+// the fold and the write-out); slices keep at least four k-tiles.
+int field_fwd_slices(long long ctas, int ntiles, int sms) {
+  int best = 1;
+  double best_cost = 1e300;
+  for (int ns = 1; ns <= 16 && ntiles / ns >= 4; ++ns) {
+    const long long rounds = (ctas * ns + sms - 1) / sms;
+    const double cost = (double)rounds * ((double)((ntiles + ns - 1) / ns) + 3.0) + (ns > 1 ? 1.0 : 0.0);
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = ns; }
+  }
+  return best;
+}
+
+// `wplanes` (nullable): device scratch of at least 4 * cout * round_up(kc, 128) bytes for the digit planes of W;
+// without it the contraction runs on the mma.sync kernel.  `split_acc` (nullable, split_bytes): uint64 scratch
+// in which slices of the contraction meet when a layer has too few output tiles to fill the device.
 dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* ybar, int nsamples, Modulus md,
-                           uint8_t* wplanes, size_t wplanes_bytes, int* status, cudaStream_t st) {
+                           uint8_t* wplanes, size_t wplanes_bytes, u64* split_acc, size_t split_bytes, int sm_count,
+                           int* status, cudaStream_t st) {
   FwdParams p;
   p.W = W; p.x = xbar; p.y = ybar;
   p.cin = g.cin; p.cout = g.cout; p.h = g.h; p.w = g.w; p.kw = g.kw; p.stride = g.stride;
@@ -1176,7 +1202,21 @@ dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* yb
       const long long chunks = (long long)g.cout * (kcp / 16);
       field_w_planes_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(W, g.cout, g.kc, kcp, wplanes);
       DK_CUDA_CHECK(cudaGetLastError());
-      field_fwd_tc_kernel<<<tgrid, tcf::kThreads, tcf::kSmem, st>>>(p, mc, wplanes, kcp, status);
+      const int ntiles = kcp / tcf::TK;
+      const long long n_y = (long long)nsamples * g.n_out;
+      int ns = field_fwd_slices((long long)tgrid.x * tgrid.y, ntiles, sm_count);
+      if (split_acc == nullptr || split_bytes < (size_t)n_y * sizeof(u64)) ns = 1;
+      if (ns > 1) {
+        tgrid.z = (unsigned)ns;
+        const int tps = (ntiles + ns - 1) / ns;
+        tgrid.z = (unsigned)((ntiles + tps - 1) / tps);
+        DK_CUDA_CHECK(cudaMemsetAsync(split_acc, 0, (size_t)n_y * sizeof(u64), st));
+        field_fwd_tc_kernel<<<tgrid, tcf::kThreads, tcf::kSmem, st>>>(p, mc, wplanes, kcp, split_acc, tps, status);
+        DK_CUDA_CHECK(cudaGetLastError());
+        field_reduce_kernel<<<ew_blocks(n_y, sm_count), 256, 0, st>>>(split_acc, n_y, md, ybar);
+      } else {
+        field_fwd_tc_kernel<<<tgrid, tcf::kThreads, tcf::kSmem, st>>>(p, mc, wplanes, kcp, nullptr, ntiles, status);
+      }
       DK_CUDA_CHECK(cudaGetLastError());
       return DK_OK;
     }
@@ -1668,7 +1708,9 @@ dk_status dk_field_linear_fwd(dk_ctx* ctx, const dk_problem* p, uint32_t prime, 
   const bool have_ws = ctx->ws && ctx->ws_bytes >= wp.total;
   return launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md,
                           have_ws ? reinterpret_cast<uint8_t*>(static_cast<char*>(ctx->ws) + wp.wpl) : nullptr,
-                          have_ws ? wp.wpl_bytes : 0, field_status_word(ctx), st);
+                          have_ws ? wp.wpl_bytes : 0,
+                          have_ws ? reinterpret_cast<u64*>(static_cast<char*>(ctx->ws) + wp.acc64) : nullptr,
+                          have_ws ? wp.total - wp.acc64 : 0, ctx->sm_count, field_status_word(ctx), st);
 }
 
 dk_status dk_field_decode_verify(dk_ctx* ctx, const dk_problem* p, uint32_t prime, int32_t l,
@@ -1738,6 +1780,7 @@ dk_status dk_field_masked_linear(dk_ctx* ctx, const dk_problem* p, uint32_t prim
   {
     ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
     s = launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, reinterpret_cast<uint8_t*>(ws + wp.wpl), wp.wpl_bytes,
+                         reinterpret_cast<u64*>(ws + wp.acc64), wp.total - wp.acc64, ctx->sm_count,
                          field_status_word(ctx), st);
   }
   if (s != DK_OK) return s;
