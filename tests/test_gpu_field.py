@@ -33,7 +33,9 @@ CASES = [
     ("fc784", synth.layers("fc784")[0], dk.DK_NHWC),
     ("fc_ragged_K1", tiny("fc", cin=37, cout=19, K=1, G=3), dk.DK_NHWC),
     ("fc_K8_long", tiny("fc", cin=20011, cout=70, K=8, G=1), dk.DK_NHWC),     # several reductions per sum
-    ("fc_long_tc", tiny("fc", cin=20012, cout=130, K=2, G=1), dk.DK_NHWC),    # tcgen05 kernel: folds at 8192 and 16384
+    ("fc_long_tc", tiny("fc", cin=20012, cout=130, K=2, G=1), dk.DK_NHWC),    # tcgen05 kernel, sliced contraction
+    # 1025 k-tiles in 16 slices of 65: each slice folds its class sums once before its end
+    ("fc_very_long_tc", tiny("fc", cin=131076, cout=8, K=1, G=1), dk.DK_NHWC),
     ("conv_tiny_K2", tiny(), dk.DK_NHWC),
     ("conv_ragged_K3_nchw", tiny(cin=5, cout=7, h=6, w=5, K=3, G=2), dk.DK_NCHW),
     ("conv_7x7s2_stem", tiny(cin=3, cout=16, h=20, w=20, kh=7, kw=7, stride=2, pad=3, K=4, G=1), dk.DK_NHWC),
