@@ -143,11 +143,11 @@ def linear(W: np.ndarray, x: np.ndarray, stride: int = 1, pad: int = 0) -> np.nd
 
 def linear_at(W: np.ndarray, x_one: np.ndarray, co: int, oh: int, ow: int,
               stride: int = 1, pad: int = 0) -> float:
-    """One output element of ``linear`` for one sample (x_one has no batch axis)."""
-    W = np.asarray(W, dtype=F64)
-    x_one = np.asarray(x_one, dtype=F64)
+    """One output element of ``linear`` for one sample (x_one has no batch axis).
+    Only the filter row and the input columns under it are converted to
+    float64, so that a single element of a large layer stays cheap."""
     if x_one.ndim == 1:
-        return float(W[co] @ x_one)
+        return float(np.asarray(W[co], dtype=F64) @ np.asarray(x_one, dtype=F64))
     cin, h, w = x_one.shape
     _, _, kh, kw = W.shape
     acc = 0.0
@@ -159,7 +159,7 @@ def linear_at(W: np.ndarray, x_one: np.ndarray, co: int, oh: int, ow: int,
             iw = ow * stride + v - pad
             if iw < 0 or iw >= w:
                 continue
-            acc += float(W[co, :, u, v] @ x_one[:, ih, iw])
+            acc += float(np.asarray(W[co, :, u, v], dtype=F64) @ np.asarray(x_one[:, ih, iw], dtype=F64))
     return acc
 
 
@@ -344,15 +344,15 @@ def wgrad_plain(delta: np.ndarray, x: np.ndarray, scale: float, kh: int = 1, kw:
 
 def wgrad_plain_at(delta: np.ndarray, x: np.ndarray, scale: float, co: int, ci: int,
                    u: int = 0, v: int = 0, stride: int = 1, pad: int = 0) -> float:
-    """One element of ``wgrad_plain``."""
-    d = np.asarray(delta, dtype=F64)
-    x = np.asarray(x, dtype=F64)
+    """One element of ``wgrad_plain`` (only output channel ``co`` of delta and
+    input channel ``ci`` of x are converted to float64)."""
     if x.ndim == 2:
-        return scale * float(d[:, co] @ x[:, ci])
-    _, _, ho, wo = d.shape
-    xp = _pad(x[:, ci:ci + 1], pad)[:, 0]
+        return scale * float(np.asarray(delta[:, co], dtype=F64) @ np.asarray(x[:, ci], dtype=F64))
+    d = np.asarray(delta[:, co], dtype=F64)
+    _, ho, wo = d.shape
+    xp = _pad(np.asarray(x[:, ci:ci + 1], dtype=F64), pad)[:, 0]
     win = xp[:, u:u + (ho - 1) * stride + 1:stride, v:v + (wo - 1) * stride + 1:stride]
-    return scale * float(np.sum(d[:, co] * win))
+    return scale * float(np.sum(d * win))
 
 
 # ---------------------------------------------------------------------------
