@@ -2,17 +2,25 @@
 """Benchmark of the masked linear-algebra path.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload vgg16_cifar] [--no-cpu-baseline]
+                    [--workload vgg16_224] [--no-cpu-baseline] [--no-field]
     python bench.py --layer-table [--workload vgg16_224] [--layers conv3_2,conv4_2]
     python bench.py --field-table [--workload vgg16_cifar] [--layers conv3_2,conv4_2]
+    python bench.py --schedule [--workload vgg16_224]
 
 One step = one pass of the whole path over one synthetic batch of the
 workload: for every layer the fused masked forward (encode, dense op on the
 K+2 encodings, decode, integrity check, with the encodings stored) followed by
 the masked weight gradient where the workload trains.  Prints ONE JSON line.
 
+The default workload is the full VGG-16 step at 224 x 224, batch 256 (13
+convolutions and 3 fully connected layers, all resident).  Beside the step
+metric the line carries, per layer and call, the roof that binds it (tensor
+or HBM) and the fraction reached; the ten-step schedule with one injected
+wrong accelerator output and what the integrity check said; and the smallest
+wrong value the floating-point check flags, measured through the C-ABI.
+
 `--impl reference` times the fp64 CPU oracle as it stands on a bounded sample
-of the same workload (one virtual batch of every layer per step).
+of the same workload (step i = one virtual batch of layer i mod L).
 
 `--layer-table` times every layer of a workload on its own (forward call and
 wgrad call, CUDA events around the C-ABI call) and prints one JSON line with
@@ -44,9 +52,11 @@ import numpy as np  # noqa: E402
 METRIC = "decoded masked-linear TFLOP/s & fraction of roofline; encode/decode GB/s"
 L2_FLUSH_BYTES = 512 << 20
 TF32_OVER_BF16 = 1.1 / 2.25      # nominal dense TF32 : BF16 tensor throughput
-# DRAM bytes (read + write) per launch of the GEMM kernel classes, from one ncu capture of this command's
-# launches (summary with the command under profiles/); None = not captured since the kernels last changed.
-NCU_TRAFFIC_BYTES = {"vgg16_cifar": {"linear_fwd": 37150685, "wgrad": 47604374}}
+FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # SMs x FMA lanes x 2 x max SM clock
+# DRAM bytes (read + write) per launch of the GEMM kernel classes, average over the layers' launches, from
+# ncu captures of these kernels (summaries with their commands under profiles/); a workload or class that is
+# absent here has not been captured since the kernels last changed and reports null.
+NCU_TRAFFIC_BYTES = {}
 
 
 def read_peaks():
@@ -63,18 +73,16 @@ def read_peaks():
 # ---------------------------------------------------------------------------
 # reference arm / CPU baseline: the oracle on one virtual batch of every layer
 # ---------------------------------------------------------------------------
-def oracle_sample_step(specs, drawn):
-    """Runs the oracle's masked forward (+ wgrad) on one group of every layer.
-    Returns the masked flops it covered."""
+def oracle_layer_sample(spec, d):
+    """The oracle's masked forward (+ check, + masked wgrad where the workload trains) on ONE virtual batch
+    (G = 1) of one layer.  Returns the masked flops it covered."""
     from oracle import dk_oracle as O
-    flops = 0.0
-    for spec, d in zip(specs, drawn):
-        m = O.masked_forward(d["W"], d["x"], d["r"], d["C"], spec.stride, spec.pad)
-        flops += spec.fwd_flops()
-        if spec.wgrad:
-            O.wgrad_masked(d["delta"], m["xbar"], d["C"], d["gamma"], 1.0 / spec.batch,
-                           spec.kh, spec.kw, spec.stride, spec.pad)
-            flops += spec.wgrad_flops()
+    m = O.masked_forward(d["W"], d["x"], d["r"], d["C"], spec.stride, spec.pad)
+    flops = spec.fwd_flops()
+    if spec.wgrad:
+        O.wgrad_masked(d["delta"], m["xbar"], d["C"], d["gamma"], 1.0 / spec.batch,
+                       spec.kh, spec.kw, spec.stride, spec.pad)
+        flops += spec.wgrad_flops()
     return flops
 
 
@@ -90,23 +98,39 @@ def cpu_threads():
 
 
 def time_oracle(workload, steps, warmup, budget_s=None):
+    """Times the oracle as it stands on a bounded sample of the workload: step i runs one virtual batch
+    (G = 1) of layer (i mod L) of the workload's L layers, so that L consecutive steps cover one group of
+    every layer; with `budget_s` the run stops at the first step boundary past the budget."""
     from paper_2207_00083_b200 import synth
     specs = [s.with_groups(1) for s in synth.layers(workload)]
-    drawn = [synth.draw_layer(s) for s in specs]
-    for _ in range(warmup):
-        oracle_sample_step(specs, drawn)
-    t0 = time.perf_counter()
-    flops = 0.0
-    done = 0
-    for _ in range(steps):
-        flops += oracle_sample_step(specs, drawn)
+    n = len(specs)
+    drawn = {}
+
+    def one(i):
+        li = i % n
+        if li not in drawn:
+            drawn[li] = synth.draw_layer(specs[li], with_delta=specs[li].wgrad)
+        return oracle_layer_sample(specs[li], drawn[li])
+
+    for i in range(warmup):
+        one(i)
+    for i in range(warmup, warmup + steps):      # inputs are drawn outside the timed region
+        li = i % n
+        if li not in drawn:
+            drawn[li] = synth.draw_layer(specs[li], with_delta=specs[li].wgrad)
+    flops, done, dt = 0.0, 0, 0.0
+    for i in range(warmup, warmup + steps):
+        t0 = time.perf_counter()
+        flops += one(i)
+        dt += time.perf_counter() - t0
         done += 1
-        if budget_s is not None and time.perf_counter() - t0 > budget_s:
+        if budget_s is not None and dt > budget_s:
             break
-    dt = time.perf_counter() - t0
+    covered = [specs[i % n].name for i in range(warmup, warmup + done)]
     return {"value": flops / dt / 1e12, "ms_per_step": dt / done * 1e3, "steps": done,
-            "sample": f"one virtual batch (G=1) of each of the {len(specs)} layers of {workload} per step, "
-                      f"masked forward+verify" + (" and masked wgrad" if specs[0].wgrad else ""),
+            "sample": f"{done} steps, step i = one virtual batch (G=1) of layer (i mod {n}) of {workload}: masked "
+                      f"forward+verify" + (" and masked wgrad" if specs[0].wgrad else "") +
+                      f"; layers covered: {','.join(covered)}",
             "cores": cpu_threads()}
 
 
@@ -201,7 +225,7 @@ def uses_tensor_cores(s):
 
 
 def make_layer(torch, dk, synth, ctx, s, dev, gen, rank, pinned):
-    """Device (and optionally pinned host) tensors of one layer, seeded."""
+    """Device tensors of one layer, seeded (`pinned` is unused: host copies are made by measure_e2e)."""
     p = dk.problem_from_spec(s, tol=1e-4)
     rng = synth._rng(s, "coef", rank)
     L = {"spec": s, "p": p, "C": synth.draw_coefficients(rng, s.K, s.G),
@@ -218,21 +242,9 @@ def make_layer(torch, dk, synth, ctx, s, dev, gen, rank, pinned):
     L["y"] = torch.empty(shape_acts(s.batch, s, "out"), device=dev)
     L["xsave"] = torch.empty(shape_acts(s.G * (s.K + 2), s, "in"), device=dev)
     L["v"] = dk.new_verdict(dev.index)
-    L["h2d"] = L["d2h"] = 0
     if s.wgrad:
         L["delta"] = torch.empty(shape_acts(s.batch, s, "out"), device=dev).normal_(0, 1, generator=gen)
         L["dW"] = torch.empty_like(L["W"])
-    if pinned:
-        L["hx"], L["hr"] = x.cpu().pin_memory(), r.cpu().pin_memory()
-        L["hy"] = torch.empty(L["y"].shape, dtype=torch.float32).pin_memory()
-        L["hv"] = torch.empty(dk.VERDICT_BYTES, dtype=torch.uint8).pin_memory()
-        L["h2d"] = (x.numel() + r.numel()) * 4
-        L["d2h"] = L["y"].numel() * 4 + dk.VERDICT_BYTES
-        if s.wgrad:
-            L["hdelta"] = L["delta"].cpu().pin_memory()
-            L["hdW"] = torch.empty(L["W"].shape, dtype=torch.float32).pin_memory()
-            L["h2d"] += L["delta"].numel() * 4
-            L["d2h"] += L["W"].numel() * 4
     return L
 
 
@@ -270,6 +282,7 @@ def measure_elementwise(torch, dk, synth, ctx, dev, peaks, iters=10):
 
 
 def run_layer_table(args):
+    """Every layer of a workload on its own (one layer resident at a time): see profile_layers."""
     import torch
     from paper_2207_00083_b200 import binding as dk
     from paper_2207_00083_b200 import synth
@@ -288,47 +301,13 @@ def run_layer_table(args):
             continue
         L = make_layer(torch, dk, synth, ctx, s, dev, gen, 0, pinned=False)
         ctx.ensure_workspace(L["p"])
-
-        def fwd():
-            dk.dk_masked_linear(ctx, L["p"], L["W"], L["x"], L["r"], L["C"], None, L["y"], L["xsave"], L["v"])
-
-        def wg():
-            dk.dk_linear_bwd_wgrad(ctx, L["p"], L["delta"], L["xsave"], s.K + 2, L["C"], L["gamma"],
-                                   1.0 / s.batch, L["dW"])
-        row = {"layer": s.name, "M": s.cout, "Kc": s.kc, "N_fwd": s.G * (s.K + 2) * s.hout * s.wout,
-               "tensor_cores": uses_tensor_cores(s)}
-        for name, fn, flops in (("fwd", fwd, s.fwd_flops()), ("wgrad", wg, s.wgrad_flops())):
-            if name == "wgrad" and not s.wgrad:
-                continue
-            for _ in range(2):
-                fn()
-            dk.dk_profile_reset(ctx)
-            dk.dk_profile_enable(ctx, True)
-            tot = 0.0
-            for _ in range(args.iters):
-                flush.zero_()
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(); fn(); b.record()
-                torch.cuda.synchronize()
-                tot += a.elapsed_time(b)
-            prof = dk.dk_profile_read(ctx)
-            dk.dk_profile_enable(ctx, False)
-            ms = tot / args.iters
-            kind = "linear_fwd" if name == "fwd" else "wgrad"
-            kms = prof[kind][0] / max(prof[kind][1], 1)
-            issued = 3.0 if uses_tensor_cores(s) else 1.0
-            row[name] = {"call_ms": round(ms, 4), "kernel_ms": round(kms, 4),
-                         "masked_tflops_call": round(flops / ms / 1e9, 2),
-                         "issued_tflops_kernel": round(issued * flops / kms / 1e9, 2),
-                         "frac_tf32_peak_kernel": round(issued * flops / kms / 1e9 / tf32_peak, 4),
-                         "other_kernels_ms": round(sum(v[0] for k, v in prof.items() if k != kind)
-                                                   / args.iters, 4)}
-        vd = dk.read_verdict(L["v"])
-        row["verdict_ok"] = vd["ok"]
+        row = profile_layers(torch, dk, ctx, [L], peaks, tf32_peak, flush, iters=args.iters)[0]
+        row["verdict_ok"] = dk.read_verdict(L["v"])["ok"]
         rows.append(row)
         del L
         torch.cuda.empty_cache()
-    print(json.dumps({"layer_table": args.workload, "tf32_peak_tflops": tf32_peak, "peak_source": peaks["source"],
+    print(json.dumps({"layer_table": args.workload, "tf32_peak_tflops": tf32_peak, "hbm_gbs": peaks["hbm_gbs"],
+                      "fp32_alu_peak_tflops": FP32_ALU_PEAK_TFLOPS, "peak_source": peaks["source"],
                       "rows": rows}), flush=True)
 
 
@@ -487,6 +466,166 @@ def whole_job_value(flops_per_step, steps, world, ms_total):
 
 
 # ---------------------------------------------------------------------------
+# per-layer accounting: which roof binds, algorithmic bytes, issued flops
+# ---------------------------------------------------------------------------
+def wgrad_on_tensor_cores(s):
+    """Mirror of the library's dispatch rule for the weight gradient (channels-last, default arithmetic,
+    cin % 4 == 0, cout % 4 == 0, stride <= 4); everything else runs on the fp32 kernel."""
+    return (getattr(s, "precision", "default") == "default" and s.cin % 4 == 0 and s.cout % 4 == 0
+            and s.stride <= 4)
+
+
+def algorithmic_bytes(s, call):
+    """Bytes a call must move at least (fp32): the fused forward reads the K private inputs and the noise
+    of every group and W once, writes the K decoded outputs and the K+1 encodings the backward pass needs;
+    the weight gradient reads the K output gradients and those K+1 encodings, writes dW once."""
+    if call == "fwd":
+        return 4.0 * (s.G * (s.K + 1) * s.n_in + s.cout * s.kc + s.G * s.K * s.n_out + s.G * (s.K + 1) * s.n_in)
+    return 4.0 * (s.G * s.K * s.n_out + s.G * (s.K + 1) * s.n_in + s.cout * s.kc)
+
+
+def layer_roofs(s, call, peaks, tf32_peak):
+    """Time floors of one call (ms) under the tensor roof (issued 3xTF32 flops, or fp32 FMAs for the
+    kernels that do not use the tensor cores) and under the HBM roof (algorithmic bytes), and which binds."""
+    flops = s.fwd_flops() if call == "fwd" else s.wgrad_flops()
+    tensor = uses_tensor_cores(s) if call == "fwd" else wgrad_on_tensor_cores(s)
+    issued = 3.0 * flops if tensor else flops
+    t_compute = issued / ((tf32_peak if tensor else FP32_ALU_PEAK_TFLOPS) * 1e12) * 1e3
+    t_hbm = algorithmic_bytes(s, call) / (peaks["hbm_gbs"] * 1e9) * 1e3
+    bound = ("tensor" if tensor else "alu") if t_compute >= t_hbm else "hbm"
+    return {"bound": bound, "floor_ms": max(t_compute, t_hbm), "tensor_floor_ms": t_compute,
+            "hbm_floor_ms": t_hbm, "issued_flops": issued, "tensor_cores": tensor}
+
+
+def fwd_call(dk, ctx, L, fault=None):
+    dk.dk_masked_linear(ctx, L["p"], L["W"], L["x"], L["r"], L["C"], None, L["y"], L["xsave"], L["v"], fault)
+
+
+def wgrad_call(dk, ctx, L):
+    s = L["spec"]
+    dk.dk_linear_bwd_wgrad(ctx, L["p"], L["delta"], L["xsave"], s.K + 2, L["C"], L["gamma"], 1.0 / s.batch, L["dW"])
+
+
+def profile_layers(torch, dk, ctx, layers, peaks, tf32_peak, flush, iters=2):
+    """One call at a time with the library's own event pairs on: per layer and call the time of the whole
+    call, of its GEMM kernel and of everything else it launches, against the roof that binds the layer."""
+    rows = []
+    for L in layers:
+        s = L["spec"]
+        row = {"layer": s.name, "M": s.cout, "Kc": s.kc, "N_fwd": s.G * (s.K + 2) * s.hout * s.wout}
+        for call, fn, kind in (("fwd", lambda: fwd_call(dk, ctx, L), "linear_fwd"),
+                               ("wgrad", lambda: wgrad_call(dk, ctx, L), "wgrad")):
+            if call == "wgrad" and not s.wgrad:
+                continue
+            fn()
+            dk.dk_profile_reset(ctx)
+            dk.dk_profile_enable(ctx, True)
+            tot = 0.0
+            for _ in range(iters):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                tot += a.elapsed_time(b)
+            prof = dk.dk_profile_read(ctx)
+            dk.dk_profile_enable(ctx, False)
+            ms = tot / iters
+            kms = prof[kind][0] / max(prof[kind][1], 1)
+            roof = layer_roofs(s, call, peaks, tf32_peak)
+            flops = s.fwd_flops() if call == "fwd" else s.wgrad_flops()
+            row[call] = {"bound": roof["bound"], "call_ms": round(ms, 4), "kernel_ms": round(kms, 4),
+                         "other_kernels_ms": round(sum(v[0] for k, v in prof.items() if k != kind) / iters, 4),
+                         "floor_ms": round(roof["floor_ms"], 4),
+                         "frac_of_roof_call": round(roof["floor_ms"] / ms, 4),
+                         "frac_of_roof_kernel": round(roof["floor_ms"] / kms, 4) if kms > 0 else None,
+                         "masked_tflops_call": round(flops / ms / 1e9, 2),
+                         "issued_tflops_kernel": round(roof["issued_flops"] / kms / 1e9, 2) if kms > 0 else None,
+                         "algorithmic_gbs_call": round(algorithmic_bytes(s, call) / ms / 1e6, 1)}
+        rows.append(row)
+    return rows
+
+
+# ---------------------------------------------------------------------------
+# the ten-step schedule with one wrong accelerator output
+# ---------------------------------------------------------------------------
+def run_fault_schedule(dk, ctx, layers, steps=10, seed=2207):
+    """`steps` passes of the whole path over all layers (fused forward with the integrity check, then the
+    weight gradient); in ONE seeded (step, layer) the accelerator returns one wrong value (dk_fault).
+    Returns the fault and what the verdicts said: every other call must be clean, the faulted call must
+    flag exactly that element."""
+    rng = np.random.default_rng(seed)
+    f_step = int(rng.integers(0, steps))
+    f_layer = int(rng.integers(0, len(layers)))
+    s = layers[f_layer]["spec"]
+    f_group, f_enc = int(rng.integers(0, s.G)), int(rng.integers(0, s.K + 2))
+    f_index = int(rng.integers(0, s.n_out))
+    fault = dk.dk_fault(f_group, f_enc, f_index, 500.0)
+    clean_calls, bad_clean, flagged = 0, [], None
+    for step in range(steps):
+        for li, L in enumerate(layers):
+            hit = step == f_step and li == f_layer
+            fwd_call(dk, ctx, L, fault if hit else None)
+            vd = dk.read_verdict(L["v"])
+            if hit:
+                flagged = vd
+            elif (vd["ok"], vd["n_flagged"], vd["first_index"], vd["status"]) == (1, 0, -1, 0):
+                clean_calls += 1
+            else:
+                bad_clean.append({"step": step, "layer": L["spec"].name, "verdict": vd})
+            if L["spec"].wgrad:
+                wgrad_call(dk, ctx, L)
+    status = dk.dk_device_status(ctx)
+    want_index = f_group * s.n_out + f_index
+    ok = (not bad_clean and status == 0 and flagged is not None and
+          (flagged["ok"], flagged["n_flagged"], flagged["first_index"]) == (0, 1, want_index))
+    return {"steps": steps, "layers": len(layers), "calls_checked": steps * len(layers),
+            "fault": {"step": f_step, "layer": s.name, "group": f_group, "enc": f_enc, "out_index": f_index,
+                      "delta": 500.0, "expected_first_index": want_index},
+            "clean_calls": clean_calls, "unexpected": bad_clean, "faulted_verdict": flagged,
+            "device_status": status, "as_expected": bool(ok)}
+
+
+# ---------------------------------------------------------------------------
+# detection floor of the floating-point integrity check, measured through the C-ABI
+# ---------------------------------------------------------------------------
+def detection_floor(torch, dk, ctx, L, positions=3, iters=26):
+    """Smallest wrong value that the check flags, per encoding row, found by bisection on dk_fault.delta
+    (each probe is one dk_masked_linear call) at a few output elements of one layer, in units of the rms of
+    that encoded output row (taken from dk_encode + dk_linear_fwd).  The paper's exact comparison has no
+    such floor; the floating-point rule flags |rho| > tau * max(s_e, s_g)."""
+    s, p = L["spec"], L["p"]
+    E = s.K + 2
+    dev = L["x"].device
+    xbar = torch.empty(shape_acts(s.G * E, s, "in"), device=dev)
+    ybar = torch.empty(shape_acts(s.G * E, s, "out"), device=dev)
+    dk.dk_encode(ctx, p, L["x"], L["r"], L["C"], xbar)
+    dk.dk_linear_fwd(ctx, p, L["W"], xbar, ybar)
+    rows_rms = ybar.reshape(s.G * E, -1).square().mean(dim=1).sqrt().cpu().numpy()
+    rng = np.random.default_rng(83)
+    out = []
+    for enc in range(E):
+        floors = []
+        for _ in range(positions):
+            g, idx = int(rng.integers(0, s.G)), int(rng.integers(0, s.n_out))
+            rms = float(rows_rms[g * E + enc])
+            lo, hi = 1e-9 * rms, 1e2 * rms           # lo passes, hi is flagged
+            for _ in range(iters):
+                mid = (lo * hi) ** 0.5
+                dk.dk_masked_linear(ctx, p, L["W"], L["x"], L["r"], L["C"], None, L["y"], None, L["v"],
+                                    dk.dk_fault(g, enc, idx, mid))
+                if dk.read_verdict(L["v"])["n_flagged"] >= 1:
+                    hi = mid
+                else:
+                    lo = mid
+            floors.append(hi / rms)
+        out.append({"enc": enc, "floor_over_row_rms_median": float(np.median(floors)),
+                    "floor_over_row_rms_max": float(max(floors))})
+    dk.dk_masked_linear(ctx, p, L["W"], L["x"], L["r"], L["C"], None, L["y"], L["xsave"], L["v"])
+    return {"layer": s.name, "tau": 1e-4, "rule": "flagged iff not(|rho| <= tau*max(s_e, s_g))",
+            "positions_per_row": positions, "unit": "smallest flagged |delta| / rms(y_bar row)", "rows": out}
+
+
+# ---------------------------------------------------------------------------
 # our arm
 # ---------------------------------------------------------------------------
 def run_ours(args):
@@ -509,61 +648,16 @@ def run_ours(args):
     ctx = dk.Context(local)
     gen = torch.Generator(device=dev)
     gen.manual_seed(220700083 + rank)
-    layers = [make_layer(torch, dk, synth, ctx, s, dev, gen, rank, pinned=True) for s in specs]
-    h2d = sum(L["h2d"] for L in layers)
-    d2h = sum(L["d2h"] for L in layers)
+    layers = [make_layer(torch, dk, synth, ctx, s, dev, gen, rank, pinned=False) for s in specs]
     biggest = max(layers, key=lambda L: ctx.workspace_bytes(L["p"]))
     ctx.ensure_workspace(biggest["p"])
     flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)
 
     def step_device():
         for L in layers:
-            s = L["spec"]
-            dk.dk_masked_linear(ctx, L["p"], L["W"], L["x"], L["r"], L["C"], None, L["y"], L["xsave"], L["v"])
-            if s.wgrad:
-                dk.dk_linear_bwd_wgrad(ctx, L["p"], L["delta"], L["xsave"], s.K + 2, L["C"], L["gamma"],
-                                       1.0 / s.batch, L["dW"])
-
-    h2d_stream, d2h_stream = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-
-    def step_e2e():
-        """The same step through host buffers: every layer's inputs come from pinned host memory and its
-        results go back there.  Uploads, the library's calls and downloads run on three streams chained by
-        events, layer by layer, so that the copies of one layer overlap the kernels of its neighbours; the
-        step starts after everything before it and ends when the last download has landed."""
-        main = torch.cuda.current_stream()
-        start = torch.cuda.Event()
-        start.record(main)
-        h2d_stream.wait_event(start)
-        d2h_stream.wait_event(start)
-        for L in layers:
-            s = L["spec"]
-            with torch.cuda.stream(h2d_stream):
-                L["x"].copy_(L["hx"], non_blocking=True)
-                L["r"].copy_(L["hr"], non_blocking=True)
-                if s.wgrad:
-                    L["delta"].copy_(L["hdelta"], non_blocking=True)
-                up = torch.cuda.Event()
-                up.record(h2d_stream)
-            main.wait_event(up)
-            dk.dk_masked_linear(ctx, L["p"], L["W"], L["x"], L["r"], L["C"], None, L["y"], L["xsave"], L["v"])
-            fwd_done = torch.cuda.Event()
-            fwd_done.record(main)
-            d2h_stream.wait_event(fwd_done)
-            with torch.cuda.stream(d2h_stream):
-                L["hy"].copy_(L["y"], non_blocking=True)
-                L["hv"].copy_(L["v"], non_blocking=True)
-            if s.wgrad:
-                dk.dk_linear_bwd_wgrad(ctx, L["p"], L["delta"], L["xsave"], s.K + 2, L["C"], L["gamma"],
-                                       1.0 / s.batch, L["dW"])
-                wg_done = torch.cuda.Event()
-                wg_done.record(main)
-                d2h_stream.wait_event(wg_done)
-                with torch.cuda.stream(d2h_stream):
-                    L["hdW"].copy_(L["dW"], non_blocking=True)
-        down = torch.cuda.Event()
-        down.record(d2h_stream)
-        main.wait_event(down)
+            fwd_call(dk, ctx, L)
+            if L["spec"].wgrad:
+                wgrad_call(dk, ctx, L)
 
     def barrier():
         if world > 1:
@@ -607,21 +701,22 @@ def run_ours(args):
     launches = sum(v[2] for v in dk.dk_profile_read(ctx).values())
     assert dk.dk_device_status(ctx) == 0
 
-    # ---- a second, untimed-for-the-metric pass with the library's per-kernel events on: kernel shares and
-    # the dominant kernel's average launch duration (the event pairs themselves cost a little, so the step
-    # metric above is taken without them)
+    # ---- a second pass with the library's per-kernel events on (the event pairs cost a little, so the step
+    # metric above is taken without them): kernel shares and the dominant kernel's average launch duration,
+    # measured inside the same back-to-back step
     dk.dk_profile_reset(ctx)
     dk.dk_profile_enable(ctx, True)
-    timed(step_device, min(steps, 10), 0)
+    prof_steps = min(steps, 10)
+    timed(step_device, prof_steps, 0)
     prof = dk.dk_profile_read(ctx)
     dk.dk_profile_enable(ctx, False)
-
-    # ---- end to end through host buffers
-    ms_e2e = timed(step_e2e, steps, 1)
 
     for L in layers:        # every verdict of the last step must be clean
         vd = dk.read_verdict(L["v"])
         assert vd["ok"] == 1 and vd["status"] == 0, (L["spec"].name, vd)
+
+    # ---- end to end through host buffers: pinned host copies of every layer's inputs and results
+    e2e = measure_e2e(torch, dk, ctx, layers, dev, timed, min(steps, args.e2e_steps), step_flops, world)
 
     if rank != 0:
         if world > 1:
@@ -629,42 +724,46 @@ def run_ours(args):
         return
 
     value = whole_job_value(step_flops, steps, world, ms_total)
-    e2e_value = whole_job_value(step_flops, steps, world, ms_e2e)
     K = specs[0].K
     ksum = max(sum(v[0] for v in prof.values()), 1e-9)
     kernel_ms = {k: round(v[0] / max(v[1], 1), 5) for k, v in prof.items() if v[1]}
     share = {k: round(v[0] / ksum, 4) for k, v in prof.items() if v[1]}
 
-    # roofline of the dominant kernel class (forward GEMM or wgrad GEMM)
+    # roofline of the dominant kernel class (forward GEMM or wgrad GEMM), timed inside the long step: the
+    # sustained tensor figure is the denominator, the burst one is given beside it
+    long_step = ms_total / steps * (warmup + steps) > 1000.0
+    bf16 = peaks["bf16_tflops_sustained"] if long_step else peaks["bf16_tflops"]
+    tf32_peak = bf16 * TF32_OVER_BF16
+    tf32_burst = peaks["bf16_tflops"] * TF32_OVER_BF16
     dom = "linear_fwd" if prof["linear_fwd"][0] >= prof["wgrad"][0] else "wgrad"
-    dom_specs = [s for s in specs if dom == "linear_fwd" or s.wgrad]
-    tc_flops = sum((s.fwd_flops() if dom == "linear_fwd" else s.wgrad_flops()) for s in dom_specs
-                   if uses_tensor_cores(s))
-    simt_flops = sum((s.fwd_flops() if dom == "linear_fwd" else s.wgrad_flops()) for s in dom_specs
-                     if not uses_tensor_cores(s))
-    issued_per_launch = (3.0 * tc_flops + simt_flops) / len(dom_specs)
+    call = "fwd" if dom == "linear_fwd" else "wgrad"
+    dom_specs = [s for s in specs if call == "fwd" or s.wgrad]
+    roofs = [layer_roofs(s, call, peaks, tf32_peak) for s in dom_specs]
+    issued_per_launch = sum(r["issued_flops"] for r in roofs) / len(dom_specs)
     avg_ms = prof[dom][0] / max(prof[dom][1], 1)
-    tf32_peak = peaks["bf16_tflops"] * TF32_OVER_BF16
     achieved = issued_per_launch / (avg_ms * 1e-3) / 1e12
-    # bytes one launch of the dominant GEMM kernel must move (averaged over the layers): its two operands
-    # as TF32 hi/lo pairs once, its result once
-    if dom == "linear_fwd":
-        alg_bytes = sum(8 * (s.G * (s.K + 2) * s.n_in + s.cout * s.kc) + 4 * s.G * s.K * s.n_out
-                        for s in dom_specs) / len(dom_specs)
-    else:
-        alg_bytes = sum(8 * s.G * (s.K + 1) * (s.n_in + s.n_out) + 4 * s.cout * s.kc
-                        for s in dom_specs) / len(dom_specs)
+    alg_bytes = sum(algorithmic_bytes(s, call) for s in dom_specs) / len(dom_specs)
     traffic = NCU_TRAFFIC_BYTES.get(args.workload, {}).get(dom)
     roofline = {"bound": "tensor", "achieved": achieved, "peak": tf32_peak, "unit": "TFLOP/s",
-                "frac": achieved / tf32_peak, "traffic": traffic, "traffic_unit": "bytes per launch (ncu, "
-                "dram read + write, average over the layers' launches)", "algorithmic_bytes": alg_bytes,
-                "kernel": dom,
-                "launches_timed": prof[dom][1], "avg_launch_ms": avg_ms,
-                "flops": "issued TF32 flops = 3 x masked flops (3xTF32 split), averaged over the layers",
-                "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x nominal "
-                               f"TF32:BF16 ratio {TF32_OVER_BF16:.4f}"}
+                "frac": achieved / tf32_peak, "frac_of_burst_peak": achieved / tf32_burst,
+                "traffic": traffic, "traffic_unit": "bytes per launch (ncu, dram read + write, average over "
+                "the layers' launches)", "algorithmic_bytes": alg_bytes,
+                "algorithmic_bytes_rule": "per call, fp32: fused forward reads (K+1) inputs per group and W, "
+                "writes K outputs and K+1 stored encodings; wgrad reads K gradients and K+1 encodings, writes dW",
+                "kernel": dom, "launches_timed": prof[dom][1], "avg_launch_ms": avg_ms,
+                "flops_per_launch": issued_per_launch,
+                "flops": "issued flops per launch = 3 x masked flops on the tensor-core kernels (3xTF32 split), "
+                         "1 x on the fp32 kernels, averaged over the layers (each launched once per step)",
+                "peak_source": f"{peaks['source']} bf16 {'sustained' if long_step else 'burst'} {bf16} TFLOP/s "
+                               f"x nominal TF32:BF16 ratio {TF32_OVER_BF16:.4f} (kernel timed inside a "
+                               f"{'long' if long_step else 'short'} step)"}
 
+    layer_rows = profile_layers(torch, dk, ctx, layers, peaks, tf32_burst, flush)
+    big = [r for r in layer_rows if r["fwd"]["bound"] == "tensor"]
     elem = measure_elementwise(torch, dk, synth, ctx, dev, peaks)
+    schedule = run_fault_schedule(dk, ctx, layers, steps=10)
+    floor_layer = next((L for L in layers if L["spec"].name in ("fc7", "conv5_3", "layer4_3x3", "fc")), layers[-1])
+    floor = detection_floor(torch, dk, ctx, floor_layer)
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
@@ -672,7 +771,8 @@ def run_ours(args):
         "dtype": "tf32x3 (fp32 in/out)", "data": "synthetic",
         "config": {"workload": args.workload, "layers": len(specs), "batch": specs[0].batch, "K": K,
                    "G": specs[0].G, "flops": "masked (all K+2 fwd / K+1 wgrad encodings)",
-                   "l2": f"flushed between steps ({L2_FLUSH_BYTES >> 20} MiB write, untimed)",
+                   "l2": f"flushed between steps ({L2_FLUSH_BYTES >> 20} MiB write, untimed); every large "
+                         f"layer's tensors exceed L2 by themselves",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "decoded_useful_tflops": value * (K / (K + 2) * fwd_flops + K / (K + 1) * wg_flops) / step_flops,
         "encode_gbs": elem["encode"]["gbs"], "decode_gbs": elem["decode"]["gbs"],
@@ -680,26 +780,113 @@ def run_ours(args):
         "elementwise": elem,
         "kernel_ms_per_launch": kernel_ms, "kernel_time_share": share,
         "roofline": roofline,
-        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": ms_e2e / steps},
+        "layers": layer_rows,
+        "layers_note": "one call at a time, L2 flushed before each, roofs from the burst tensor figure "
+                       f"({tf32_burst:.1f} TFLOP/s TF32) and the measured copy bandwidth; 'bound' = the larger "
+                       "of the two time floors of the call",
+        "tensor_bound_layers_min_frac_kernel": min((r["fwd"]["frac_of_roof_kernel"] for r in big), default=None),
+        "e2e": e2e,
         "gpu_launches": int(launches),
         "clocks": clocks,
+        "fault_schedule": schedule,
+        "verify": {"detection_floor": floor},
     }
-    if world == 1:
-        # the finite-field calls on one mid-sized layer of the same workload (reported beside the metric,
-        # measured after it; `--field-table` gives every layer)
-        names = [s.name for s in specs]
-        pick = "conv3_2" if "conv3_2" in names else names[len(names) // 2]
-        fm = measure_field(torch, dk, synth, ctx, dev, peaks, flush, args.workload, {pick}, 5)
-        line["field_path"] = {k: fm[k] for k in ("prime", "l", "unit", "bound", "peak_tmacs", "peak_source",
-                                                  "mma_sync_peak_tmacs", "elementwise", "rows")}
+    if world == 1 and not args.no_field:
+        # the finite-field calls on one mid-sized layer (reported beside the metric, measured after it;
+        # `--field-table` gives every layer of a workload)
+        fm = measure_field(torch, dk, synth, ctx, dev, peaks, flush, "vgg16_cifar", {"conv3_2"}, 5)
+        line["field_path"] = {k: fm[k] for k in ("field_table", "prime", "l", "unit", "bound", "peak_tmacs",
+                                                  "peak_source", "mma_sync_peak_tmacs", "elementwise", "rows")}
     if not args.no_cpu_baseline and world == 1:
-        r = time_oracle(args.workload, 500, 1, budget_s=12.0)
+        del layers
+        torch.cuda.empty_cache()
+        r = time_oracle(args.workload, len(specs), 0, budget_s=20.0)
         line["cpu_baseline"] = {"value": r["value"], "unit": "TFLOP/s", "cores": r["cores"], "kind": "oracle",
                                 "sample": r["sample"]}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def measure_e2e(torch, dk, ctx, layers, dev, timed, steps, step_flops, world):
+    """The same step through host buffers: every layer's inputs come from pinned host memory and its
+    results go back there.  Uploads, the library's calls and downloads run on three streams chained by
+    events, layer by layer, so that the copies of one layer overlap the kernels of its neighbours; a step
+    starts after everything before it and ends when the last download has landed."""
+    h2d = d2h = 0
+    for L in layers:
+        s = L["spec"]
+        L["hx"] = torch.empty(L["x"].shape, dtype=torch.float32, pin_memory=True).copy_(L["x"])
+        L["hr"] = torch.empty(L["r"].shape, dtype=torch.float32, pin_memory=True).copy_(L["r"])
+        L["hy"] = torch.empty(L["y"].shape, dtype=torch.float32, pin_memory=True)
+        L["hv"] = torch.empty(dk.VERDICT_BYTES, dtype=torch.uint8, pin_memory=True)
+        h2d += (L["x"].numel() + L["r"].numel()) * 4
+        d2h += L["y"].numel() * 4 + dk.VERDICT_BYTES
+        if s.wgrad:
+            L["hdelta"] = torch.empty(L["delta"].shape, dtype=torch.float32, pin_memory=True).copy_(L["delta"])
+            L["hdW"] = torch.empty(L["W"].shape, dtype=torch.float32, pin_memory=True)
+            h2d += L["delta"].numel() * 4
+            d2h += L["W"].numel() * 4
+    h2d_stream, d2h_stream = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+
+    def step_e2e():
+        main = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(main)
+        h2d_stream.wait_event(start)
+        d2h_stream.wait_event(start)
+        for L in layers:
+            s = L["spec"]
+            with torch.cuda.stream(h2d_stream):
+                L["x"].copy_(L["hx"], non_blocking=True)
+                L["r"].copy_(L["hr"], non_blocking=True)
+                if s.wgrad:
+                    L["delta"].copy_(L["hdelta"], non_blocking=True)
+                up = torch.cuda.Event()
+                up.record(h2d_stream)
+            main.wait_event(up)
+            fwd_call(dk, ctx, L)
+            fwd_done = torch.cuda.Event()
+            fwd_done.record(main)
+            d2h_stream.wait_event(fwd_done)
+            with torch.cuda.stream(d2h_stream):
+                L["hy"].copy_(L["y"], non_blocking=True)
+                L["hv"].copy_(L["v"], non_blocking=True)
+            if s.wgrad:
+                wgrad_call(dk, ctx, L)
+                wg_done = torch.cuda.Event()
+                wg_done.record(main)
+                d2h_stream.wait_event(wg_done)
+                with torch.cuda.stream(d2h_stream):
+                    L["hdW"].copy_(L["dW"], non_blocking=True)
+        down = torch.cuda.Event()
+        down.record(d2h_stream)
+        main.wait_event(down)
+
+    steps = max(1, steps)
+    ms = timed(step_e2e, steps, 1)
+    for L in layers:
+        for k in ("hx", "hr", "hy", "hv", "hdelta", "hdW"):
+            L.pop(k, None)
+    return {"value": whole_job_value(step_flops, steps, world, ms), "unit": "TFLOP/s",
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms / steps, "steps": steps}
+
+
+def run_schedule(args):
+    """`--schedule`: only the ten-step schedule with one injected fault, as one JSON line."""
+    import torch
+    from paper_2207_00083_b200 import binding as dk
+    from paper_2207_00083_b200 import synth
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(0)
+    ctx = dk.Context(0)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(220700083)
+    layers = [make_layer(torch, dk, synth, ctx, s, dev, gen, 0, pinned=False) for s in synth.layers(args.workload)]
+    ctx.ensure_workspace(max(layers, key=lambda L: ctx.workspace_bytes(L["p"]))["p"])
+    out = run_fault_schedule(dk, ctx, layers, steps=10)
+    out["workload"] = args.workload
+    print(json.dumps(out), flush=True)
 
 
 def main():
@@ -708,7 +895,10 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="vgg16_cifar")
+    ap.add_argument("--workload", default="vgg16_224")
+    ap.add_argument("--e2e-steps", type=int, default=3, help="timed steps of the host-buffer measurement")
+    ap.add_argument("--no-field", action="store_true")
+    ap.add_argument("--schedule", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layer-table", action="store_true")
     ap.add_argument("--field-table", action="store_true")
@@ -721,6 +911,8 @@ def main():
         run_layer_table(args)
     elif args.field_table:
         run_field_table(args)
+    elif args.schedule:
+        run_schedule(args)
     else:
         run_ours(args)
 

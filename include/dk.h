@@ -147,8 +147,10 @@ DK_API dk_status dk_encode(dk_ctx* ctx, const dk_problem* p, const float* x, con
  *   FC:   ybar[n][o] = sum_c W[o][c]*xbar[n][c]
  *   conv: ybar[n][o][p][q] = sum_{c,u,v} W[o][c][u][v]*xbar[n][c][p*s+u-pad][q*s+v-pad]
  * (cross-correlation, zero padding).  The tensor-core path serves DK_FC and
- * DK_CONV2D/DK_NHWC with stride 1 and cin % 4 == 0 and needs the workspace;
- * everything else runs on the SIMT path. */
+ * DK_CONV2D/DK_NHWC with stride <= 4 and cin % 4 == 0 and needs the workspace
+ * (in dk_masked_linear also the 3-channel stems: cin % 4 != 0 with a
+ * contraction of at most 256 elements and cout % 4 == 0); everything else runs
+ * on the SIMT path. */
 DK_API dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W,
                                const float* xbar, float* ybar, void* stream);
 
@@ -234,7 +236,12 @@ DK_API dk_status dk_device_status(dk_ctx* ctx, int32_t* status);
  *  - Limits: G*K*(K+1)*2 + G*(K+2) <= 16384 and G*(K+3) <= 16384; larger
  *    problems are refused with DK_ERR_WORKSPACE and nothing is launched.
  *  - The first call on a device looks up the array's device address (once per
- *    device); make that first call outside any stream capture.
+ *    device); make that first call outside any stream capture.  No call may
+ *    be made on a stream that is being captured: the coefficient tables are
+ *    copied from the call's own stack frame, so such a call is refused with
+ *    DK_ERR_UNSUPPORTED.  The call needs about 70 KiB of host stack.
+ *  - The one-time address look-up is not synchronised: make the first call on
+ *    a device from one thread.
  *  - Every call uses the same array: two calls whose kernels can overlap on
  *    the GPU (different streams, different threads) race on it.  Calls on
  *    one stream are safe; each call clears the state it needs.

@@ -95,6 +95,13 @@ extern "C" dk_status dk_decode_verify_static(int device, const dk_problem* p, co
   if (prev != device && cudaSetDevice(device) != cudaSuccess) return DK_ERR_CUDA;
   s = setup_device(device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The coefficient tables below are copied from this call's stack frame; a
+  // copy recorded by a stream capture would read the frame after it is gone.
+  if (s == DK_OK) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) s = DK_ERR_CUDA;
+    else if (cap != cudaStreamCaptureStatusNone) s = DK_ERR_UNSUPPORTED;
+  }
   if (s == DK_OK) {
     // decode rows (two-float split of the fp64 inverse) and null vector, on the stack
     float tab[kCoefFloats];

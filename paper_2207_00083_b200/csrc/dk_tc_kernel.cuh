@@ -320,8 +320,8 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
         residual(j, ar, sc);
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-          const float v = acc[e][j];
-          sq[e] = fmaf(fabsf(v) < kInf ? v : 0.f, v, sq[e]);
+          const float vf = fabsf(acc[e][j]) < kInf ? acc[e][j] : 0.f;     // non-finite values stay out of the rms
+          sq[e] = fmaf(vf, vf, sq[e]);
         }
         maxrho = fmaxf(maxrho, ar);
         bad |= (uint32_t)(!(ar <= p.tau * sc) || !(sc < kInf)) << j;

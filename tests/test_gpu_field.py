@@ -329,3 +329,58 @@ def test_cross_check_kernels_give_the_same_residues(switch):
                         "or vgg_cifar_conv3_1"],
                        cwd=root, env=env, capture_output=True, text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+# ---------------------------------------------------------------------------
+# Adversarial residues: every operand equal to p - 1, the value with the largest
+# base-256 digits, at contraction lengths around the fold interval of the
+# tensor-core kernels (8192 terms per class sum) and for a prime close to the
+# 2^30 limit.  The expected results are closed forms in Python integers:
+# (p-1)^2 = 1 (mod p), so a contraction of n such products is n mod p.
+# ---------------------------------------------------------------------------
+ADV_PRIMES = [2 ** 25 - 39, 2 ** 30 - 35]
+ADV_LENGTHS = [8188, 8191, 8192, 8193, 8196, 16380, 16385, 16388, 24580]     # multiples of 4 take the tcgen05 kernel
+
+
+@pytest.mark.parametrize("prime", ADV_PRIMES)
+@pytest.mark.parametrize("n", ADV_LENGTHS)
+def test_linear_fwd_on_maximal_residues(ctx, prime, n):
+    assert F.is_prime(prime)
+    for cout, use_ws in ((130, True), (24, False)):           # tcgen05 kernel (workspace) / mma.sync kernel
+        spec = tiny("fc", cin=n, cout=cout, K=2, G=1)
+        p = dk.problem_from_spec(spec)
+        if use_ws:
+            ctx.ensure_workspace(p, field=True)
+        Wq = torch.full((cout, n), prime - 1, dtype=torch.int64).to(torch.int32).cuda()
+        xbar = torch.full((spec.G * (spec.K + 2), n), prime - 1, dtype=torch.int64).to(torch.int32).cuda()
+        ybar = torch.empty((spec.G * (spec.K + 2), cout), dtype=torch.int32, device="cuda")
+        dk.dk_field_linear_fwd(ctx, p, prime, Wq, xbar, ybar)
+        assert dk.dk_device_status(ctx) == 0
+        want = (n * pow(prime - 1, 2, prime)) % prime
+        got = ybar.cpu().numpy().astype(np.int64) & 0xFFFFFFFF
+        assert np.all(got == want), (prime, n, cout, int(got.flat[0]), want)
+
+
+@pytest.mark.parametrize("prime", ADV_PRIMES)
+@pytest.mark.parametrize("pixels", [8191, 8193, 16385])
+def test_wgrad_on_maximal_residues(ctx, prime, pixels):
+    """K = 1 with the identity as square coefficient block: B = [[1/gamma_0], [0]], so the mixed gradient of
+    encoding 0 is delta itself and that of encoding 1 is zero.  With delta = x_bar = p - 1 everywhere the
+    1x1 convolution's weight gradient is (number of pixels) * (p-1)^2 = pixels (mod p) in every element."""
+    spec = tiny("conv", cin=16, cout=24, h=1, w=pixels, kh=1, kw=1, pad=0, K=1, G=1)
+    p = dk.problem_from_spec(spec)
+    ctx.ensure_workspace(p, field=True)
+    C = np.array([[[1, 0], [0, 1], [5, 7]]], dtype=np.uint32)
+    gamma = np.array([[3, 11]], dtype=np.uint32)
+    dq = torch.full((1, 1, pixels, spec.cout), prime - 1, dtype=torch.int64).to(torch.int32).cuda()
+    xbar = torch.full((3, 1, pixels, spec.cin), prime - 1, dtype=torch.int64).to(torch.int32).cuda()
+    dWq = torch.empty((spec.cout, 1, 1, spec.cin), dtype=torch.int32, device="cuda")
+    dk.dk_field_linear_bwd_wgrad(ctx, p, prime, dq, xbar, 3, C, gamma, dWq)
+    assert dk.dk_device_status(ctx) == 0
+    want = (pixels * pow(prime - 1, 2, prime)) % prime
+    got = dWq.cpu().numpy().astype(np.int64) & 0xFFFFFFFF
+    assert np.all(got == want), (prime, pixels, int(got.flat[0]), want)
+    # the same through the oracle's own single-element routine
+    d64 = np.full((1, spec.cout, 1, pixels), prime - 1, dtype=np.int64)
+    x64 = np.full((1, spec.cin, 1, pixels), prime - 1, dtype=np.int64)
+    assert F.field_wgrad_plain_at(d64, x64, 3, 5, 0, 0, prime, 1, 0) == want

@@ -227,6 +227,38 @@ def test_masked_linear_matches_oracle(ctx, drawn, spec, prec):
         assert got_v["max_ratio"] == pytest.approx(want_v["max_ratio"], rel=1e-2)
 
 
+@pytest.mark.parametrize("bad_value", [float("inf"), float("-inf"), float("nan")], ids=["inf", "-inf", "nan"])
+@pytest.mark.parametrize("name", ["vgg_cifar_conv3_1_G2", "conv_tiny_K2", "pair_K6_cout256", "vgg_cifar_conv5_1_G3"])
+def test_masked_linear_flags_a_non_finite_accelerator_output(ctx, drawn, name, bad_value):
+    """A non-finite value returned by the accelerator is flagged (NOT(|rho| <= ...) is true for NaN, an
+    infinite s_e is flagged) and stays out of the group's rms, through the fused epilogue as well as
+    through the split-K path; same verdict as the oracle."""
+    spec = SPECS[IDS.index(name)]
+    d = drawn(spec)
+    E = spec.K + 2
+    p = dk.problem_from_spec(spec, tol=H.TAU)
+    ctx.ensure_workspace(p)
+    W = H.weights_to_dev(d["W"], lay(spec))
+    x, r = H.acts_to_dev(d["x"], lay(spec)), H.acts_to_dev(d["r"], lay(spec))
+    y = H.empty_acts(spec.G * spec.K, spec, "out", lay(spec))
+    v = dk.new_verdict()
+    g, enc, (co, oh, ow) = spec.G - 1, 1, (3, spec.hout - 1, 0)
+    bad = O.masked_forward(d["W"], d["x"], d["r"], d["C"], spec.stride, spec.pad, H.TAU,
+                           fault=(g * E + enc, H.logical_out_index(spec, co, oh, ow), bad_value))
+    want_v = H.expected_verdict(bad["flags"], bad["ratio_group"], lay(spec))
+    assert want_v["n_flagged"] == 1
+    f = dk.dk_fault(g, enc, H.flat_out_index(spec, lay(spec), co, oh, ow), bad_value)
+    dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y, None, v, f)
+    got_v = dk.read_verdict(v)
+    assert (got_v["ok"], got_v["n_flagged"], got_v["first_index"], got_v["status"]) == \
+           (0, 1, g * spec.n_out + f.out_index, 0)
+    assert got_v["first_index"] == want_v["first_index"]
+    if np.isinf(bad_value):
+        assert np.isinf(got_v["max_ratio"]) and np.isinf(want_v["max_ratio"])
+    else:
+        assert got_v["max_ratio"] == pytest.approx(want_v["max_ratio"], rel=0.05, abs=1e-7)
+
+
 # ---------------------------------------------------------------------------
 # dk_linear_bwd_wgrad
 # ---------------------------------------------------------------------------

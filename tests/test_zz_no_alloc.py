@@ -82,6 +82,50 @@ def test_static_entry_point_matches_decode_verify_twice_in_a_row():
         ctx.close()
 
 
+def test_static_entry_point_leaves_free_device_memory_unchanged():
+    """What the call exists for: with no context alive, a warmed-up call must not change the amount of
+    free device memory (no allocation by the call itself or by anything it uses)."""
+    spec = synth.layer("vgg16_cifar", "conv4_1").with_groups(2)
+    p = dk.problem_from_spec(spec, tol=H.TAU)
+    d, ybar = _inputs(spec)
+    yb = H.acts_to_dev(ybar, dk.DK_NHWC)
+    y = H.empty_acts(spec.batch, spec, "out", dk.DK_NHWC)
+    v = dk.new_verdict()
+    dk.dk_decode_verify_static(0, p, yb, d["C"], None, y, v)      # first call on the device: address look-up
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        dk.dk_decode_verify_static(0, p, yb, d["C"], None, y, v)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert dk.read_verdict(v)["ok"] == 1
+
+
+def test_static_entry_point_refuses_a_capturing_stream():
+    """The tables are copied from the call's stack frame, so a call on a capturing stream is refused."""
+    spec = synth.layer("vgg16_cifar", "conv5_1").with_groups(1)
+    p = dk.problem_from_spec(spec, tol=H.TAU)
+    d, ybar = _inputs(spec)
+    yb = H.acts_to_dev(ybar, dk.DK_NHWC)
+    y = H.empty_acts(spec.batch, spec, "out", dk.DK_NHWC)
+    v = dk.new_verdict()
+    dk.dk_decode_verify_static(0, p, yb, d["C"], None, y, v)
+    torch.cuda.synchronize()
+    C = np.ascontiguousarray(d["C"], dtype=np.float32)
+    st = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        graph.capture_begin()
+        rc = dk.lib().dk_decode_verify_static(0, ctypes.byref(p), ctypes.c_void_p(yb.data_ptr()),
+                                              ctypes.c_void_p(C.ctypes.data), None, ctypes.c_void_p(y.data_ptr()),
+                                              ctypes.c_void_p(v.data_ptr()), ctypes.c_void_p(st.cuda_stream))
+        graph.capture_end()
+    assert rc == 7      # DK_ERR_UNSUPPORTED, nothing recorded
+    dk.dk_decode_verify_static(0, p, yb, d["C"], None, y, v)      # and the entry point still works afterwards
+    assert dk.read_verdict(v)["ok"] == 1
+
+
 def test_static_entry_point_refuses_what_does_not_fit():
     spec = synth.LayerSpec("tiny", "t", "fc", 16, 8, K=8, G=400)      # tables beyond the fixed array
     p = dk.problem_from_spec(spec)
