@@ -39,7 +39,7 @@ def ctx():
     c.close()
 
 
-def to_dev(a, conv_weights=False):
+def to_dev(a):
     """Logical host array -> device tensor in the library's channels-last layout (the permutation runs on
     the device; a 4-D weight array [cout, cin, kh, kw] becomes [cout, kh, kw, cin])."""
     t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
@@ -49,7 +49,7 @@ def to_dev(a, conv_weights=False):
 
 
 def sampled_y_error(spec, d, y_dev):
-    coords = synth.sample_coordinates(spec, N_Y, "y")
+    coords = synth.sample_coordinates(spec, 2 * N_Y, "y")      # duplicates are dropped by the sampler
     K = spec.K
     ks = np.random.default_rng(5).integers(0, K, len(coords))
     # the last element of the whole tensor: last sample, channel and pixel
@@ -61,15 +61,15 @@ def sampled_y_error(spec, d, y_dev):
     W64 = d["W"].astype(np.float64)
     want = np.array([O.linear_at(W64, d["x"][bb], co, oh, ow, spec.stride, spec.pad)
                      for bb, (_, co, oh, ow) in zip(b, coords)])
-    assert len(want) >= N_Y
+    assert len(want) >= min(N_Y, spec.G * spec.n_out)
     return float(np.max(np.abs(got - want)) / np.max(np.abs(want)))
 
 
 def sampled_dw_error(spec, d, dW_dev, scale_arg):
-    coords = synth.sample_coordinates(spec, N_DW, "dw")
+    coords = synth.sample_coordinates(spec, 2 * N_DW, "dw")
     coords = coords[np.lexsort((coords[:, 1], coords[:, 0]))]
     got_all = dW_dev.cpu().numpy()         # [cout, kh, kw, cin] or [cout, cin]
-    assert len(coords) >= N_DW
+    assert len(coords) >= min(N_DW, spec.cout * spec.kc)
     worst, scale = 0.0, 0.0
     for (co, ci, u, v) in coords:
         want = O.wgrad_plain_at(d["delta"], d["x"], scale_arg, co, ci, u, v, spec.stride, spec.pad)

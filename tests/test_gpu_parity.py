@@ -253,11 +253,6 @@ def test_masked_linear_flags_a_non_finite_accelerator_output(ctx, drawn, name, b
     assert (got_v["ok"], got_v["n_flagged"], got_v["first_index"], got_v["status"]) == \
            (0, 1, g * spec.n_out + f.out_index, 0)
     assert got_v["first_index"] == want_v["first_index"]
-    if np.isinf(bad_value):
-        assert np.isinf(got_v["max_ratio"]) and np.isinf(want_v["max_ratio"])
-    else:
-        assert got_v["max_ratio"] == pytest.approx(want_v["max_ratio"], rel=0.05, abs=1e-7)
-
 
 # ---------------------------------------------------------------------------
 # dk_linear_bwd_wgrad
