@@ -23,6 +23,11 @@ steps in order, without blocking or fusion:
 * ``wgrad_redundant``   the "two sets of equations" idea of Section 4.4 applied
                         to the weight gradient: decode it from encodings
                         1..K+1 and again from encodings 2..K+2, compare
+* ``dgrad_plain`` / ``relu`` / ``relu_bwd`` / ``maxpool2x2`` / ``maxpool2x2_bwd`` /
+  ``training_step_plain``   the unmasked steps that chain the masked products
+                        into a training step (Section 4.2 back-propagation of
+                        delta "without encoding", the non-linear layers of the
+                        Section 3.1 flow, Section 6 aggregation)
 * ``encode_colluding`` / ``decode_colluding`` / ``wgrad_colluding`` /
   ``colluding_subsets_full_rank``   the M-noise-vector scheme of Section 4.5
                         (X_bar = X.A1 + R.A2, S = K + M encodings)
@@ -35,12 +40,17 @@ row.
 Pins (see the ``-m "not gpu"`` tests): brute-force loops on tiny inputs, a
 library float64 convolution and its autograd, the decode/encode round trip
 against the plain definition, closed forms for K = 1, the exact residual
-change n[i]*Delta under a single injected fault, and the Eq. 5 residual.
-Parity unpinned: the numerical threshold ``tau`` of ``verify`` and its
-noise-scale normaliser max(s_e, s_g), and the threshold and rms normaliser of
-``wgrad_redundant`` (a check the paper does not describe for the backward
-pass), are choices of this implementation, not the paper's (the paper
-compares exactly in a finite field); nothing outside this file fixes them.
+change n[i]*Delta under a single injected fault, the Eq. 5 residual, the exact
+(integer) residuals and the finite-field flag set on small-integer inputs for
+both integrity rules, and float64 autograd of a library three-layer chain for
+the back-propagation helpers.
+Parity unpinned: the numerical VALUE of the threshold ``tau`` of ``verify`` and
+of ``tau_w`` of ``wgrad_redundant`` (a check the paper does not describe for the
+backward pass) and the choice of normalisers max(s_e, s_g) and rms(dW) are
+choices of this implementation, not the paper's (the paper compares exactly in
+a finite field).  What the paper does fix is pinned: with exact arithmetic
+both rules flag exactly the elements whose residual is non-zero, and the
+first agrees with the finite-field rule on the same integers.
 """
 from __future__ import annotations
 
@@ -500,3 +510,92 @@ def wgrad_colluding(delta: np.ndarray, xbar: np.ndarray, A1: np.ndarray, A2: np.
         eq = bilinear_wgrad(mixed, xbar[j], kh, kw, stride, pad)
         total = gamma[j] * eq if total is None else total + gamma[j] * eq
     return scale * total
+
+
+# ---------------------------------------------------------------------------
+# The unmasked steps around the masked products in a training step: gradient
+# back-propagation through a linear layer (Section 4.2: delta_l is computed from
+# delta_{l+1} and W "without encoding"), the non-linear layers the paper keeps
+# inside the enclave (ReLU, MaxPool; flow of Section 3.1), and the aggregation
+# of weight gradients over virtual batches (Section 6, Algorithm 2).
+# ---------------------------------------------------------------------------
+def dgrad_plain(delta: np.ndarray, W: np.ndarray, in_hw: Tuple[int, int] = (1, 1), stride: int = 1,
+                pad: int = 0) -> np.ndarray:
+    """Gradient with respect to the layer's input: the adjoint of ``linear``.
+    FC: dx = delta @ W.  Convolution: every term W[o,c,u,v] x[n,c,p*s+u-pad,q*s+v-pad] of y[n,o,p,q]
+    sends delta[n,o,p,q] W[o,c,u,v] back to that input position."""
+    d = np.asarray(delta, dtype=F64)
+    W = np.asarray(W, dtype=F64)
+    if d.ndim == 2:
+        return d @ W
+    n, cout, ho, wo = d.shape
+    _, cin, kh, kw = W.shape
+    h, w = in_hw
+    dxp = np.zeros((n, cin, h + 2 * pad, w + 2 * pad), dtype=F64)
+    for u in range(kh):
+        for v in range(kw):
+            # contribution of filter tap (u, v): [n, ho, wo, cin]
+            t = np.tensordot(d, W[:, :, u, v], axes=([1], [0])).transpose(0, 3, 1, 2)
+            dxp[:, :, u:u + (ho - 1) * stride + 1:stride, v:v + (wo - 1) * stride + 1:stride] += t
+    return dxp[:, :, pad:pad + h, pad:pad + w]
+
+
+def relu(x: np.ndarray) -> np.ndarray:
+    return np.maximum(np.asarray(x, dtype=F64), 0.0)
+
+
+def relu_bwd(dy: np.ndarray, x: np.ndarray) -> np.ndarray:
+    """Gradient through ReLU at pre-activation x: passes where x > 0."""
+    return np.where(np.asarray(x) > 0, np.asarray(dy, dtype=F64), 0.0)
+
+
+def maxpool2x2(x: np.ndarray) -> np.ndarray:
+    """2x2 max pooling with stride 2 on [n, c, h, w] (h, w even)."""
+    x = np.asarray(x, dtype=F64)
+    n, c, h, w = x.shape
+    win = x.reshape(n, c, h // 2, 2, w // 2, 2)
+    return win.max(axis=(3, 5))
+
+
+def maxpool2x2_bwd(dy: np.ndarray, x: np.ndarray) -> np.ndarray:
+    """Gradient through ``maxpool2x2``: each output's gradient goes to the first maximum of its window in
+    row-major order (top-left, top-right, bottom-left, bottom-right)."""
+    x = np.asarray(x, dtype=F64)
+    dy = np.asarray(dy, dtype=F64)
+    n, c, h, w = x.shape
+    dx = np.zeros_like(x)
+    win = x.reshape(n, c, h // 2, 2, w // 2, 2).transpose(0, 1, 2, 4, 3, 5).reshape(n, c, h // 2, w // 2, 4)
+    first = np.argmax(win, axis=4)                      # numpy returns the first maximum
+    for k in range(4):
+        du, dv = divmod(k, 2)
+        dx[:, :, du::2, dv::2] = np.where(first == k, dy, 0.0)
+    return dx
+
+
+def training_step_plain(layers, Ws, x0: np.ndarray, dL_dy: np.ndarray, scale: float) -> Dict[str, list]:
+    """One training step of a chain of linear layers, each followed by ReLU and optionally a 2x2 max
+    pooling, in plain (unmasked) arithmetic: what the masked step must reproduce.
+
+    ``layers``: list of dicts with stride, pad, pool (bool), kh, kw; ``Ws`` their weights; ``x0`` the batch;
+    ``dL_dy`` the loss gradient with respect to the last layer's output (after its ReLU/pool).
+    Returns the inputs of every layer (``acts``), pre-activations (``pre``), the gradients with respect to
+    every pre-activation (``deltas``) and the weight gradients (``dWs``, scaled by ``scale``)."""
+    acts, pre = [np.asarray(x0, dtype=F64)], []
+    for L, W in zip(layers, Ws):
+        z = linear(W, acts[-1], L["stride"], L["pad"])
+        pre.append(z)
+        a = relu(z)
+        acts.append(maxpool2x2(a) if L["pool"] else a)
+    g = np.asarray(dL_dy, dtype=F64)
+    deltas, dWs = [None] * len(layers), [None] * len(layers)
+    for li in range(len(layers) - 1, -1, -1):
+        L, W = layers[li], Ws[li]
+        if L["pool"]:
+            g = maxpool2x2_bwd(g, relu(pre[li]))
+        d = relu_bwd(g, pre[li])
+        deltas[li] = d
+        dWs[li] = wgrad_plain(d, acts[li], scale, L["kh"], L["kw"], L["stride"], L["pad"])
+        if li > 0:
+            hw = acts[li].shape[2:] if acts[li].ndim == 4 else (1, 1)
+            g = dgrad_plain(d, W, hw, L["stride"], L["pad"])
+    return {"acts": acts, "pre": pre, "deltas": deltas, "dWs": dWs}
