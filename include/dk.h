@@ -216,6 +216,46 @@ DK_API dk_status dk_linear_bwd_wgrad_verify(dk_ctx* ctx, const dk_problem* p, co
                                             float* dW, dk_verdict* verdict, const dk_fault* fault,
                                             void* stream);
 
+/* dk_linear_bwd_wgrad that ADDS to what dW holds instead of overwriting it:
+ *   dW += scale * sum_g sum_{j<=K} gamma[g][j] * < ... >       (same terms)
+ * Section 6, "Large Batch Aggregation" (Algorithm 2): the gradient of a batch
+ * is the sum of the gradients of its virtual batches, so a batch larger than
+ * what one call holds is processed as several calls on slices of its groups,
+ * the first through dk_linear_bwd_wgrad and the others through this call (the
+ * paper's paging of partial sums in and out of the enclave is not needed
+ * here: the running sum stays in device memory). */
+DK_API dk_status dk_linear_bwd_wgrad_accumulate(dk_ctx* ctx, const dk_problem* p, const float* delta,
+                                                const float* xbar, int32_t xbar_rows, const float* C_host,
+                                                const float* gamma_host, float scale, float* dW,
+                                                void* stream);
+
+/* Back-propagation of the output gradient through the layer (Section 4.2: the
+ * gradient with respect to the layer's input is computed from delta and W
+ * "without encoding", since neither is private):
+ *   FC:   dx[n][c] = sum_o delta[n][o]*W[o][c]
+ *   conv: dx[n][c][i][j] = sum over (o,u,v,p,q) with i = p*s+u-pad, j = q*s+v-pad
+ *                          of delta[n][o][p][q]*W[o][c][u][v]
+ * (the adjoint of dk_linear_fwd's operation).  delta: [G*K][n_out], dx:
+ * [G*K][n_in], layouts as in dk_problem.  Stride-1 channels-last layers with
+ * cin % 4 == 0 and cout % 4 == 0 run on the tensor-core kernel (plain 3xTF32;
+ * needs the workspace of dk_workspace_bytes(p)); others run in fp32 FMAs. */
+DK_API dk_status dk_linear_bwd_dgrad(dk_ctx* ctx, const dk_problem* p, const float* W, const float* delta,
+                                     float* dx, void* stream);
+
+/* The non-linear layers between the masked products (the paper keeps ReLU and
+ * MaxPool on the trusted side, Section 3.1 flow; here they run on the same
+ * device).  x: [n][h][w][c] channels-last (a vector per sample: h = w = 1).
+ *   fwd: y = relu(x), or with pool != 0 the 2x2/stride-2 max pooling of relu(x),
+ *        y: [n][h/2][w/2][c] (a last odd row or column is dropped).
+ *   bwd: dx = dy where x > 0, else 0; with pool != 0, dy[n][p][q][c] goes to the
+ *        first maximum of relu(x) in its 2x2 window (row-major order) if that
+ *        x > 0, every other position gets 0.  dy has the shape of y, dx of x.
+ * HBM-bound. */
+DK_API dk_status dk_relu_pool_fwd(dk_ctx* ctx, const float* x, int64_t n, int32_t h, int32_t w, int32_t c,
+                                  int32_t pool, float* y, void* stream);
+DK_API dk_status dk_relu_pool_bwd(dk_ctx* ctx, const float* dy, const float* x, int64_t n, int32_t h, int32_t w,
+                                  int32_t c, int32_t pool, float* dx, void* stream);
+
 /* Errors raised ON THE DEVICE by calls that have no dk_verdict to carry them
  * (dk_linear_fwd, dk_linear_bwd_wgrad): every wait inside the kernels is
  * bounded, and a kernel whose wait expires stops, leaves its output incomplete

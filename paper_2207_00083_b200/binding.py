@@ -76,6 +76,10 @@ def _signatures():
         "dk_decode_verify": [vp, pp, vp, vp, vp, vp, vp, vp],
         "dk_masked_linear": [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(dk_fault), vp],
         "dk_linear_bwd_wgrad": [vp, pp, vp, vp, i32, vp, vp, ctypes.c_float, vp, vp],
+        "dk_linear_bwd_wgrad_accumulate": [vp, pp, vp, vp, i32, vp, vp, ctypes.c_float, vp, vp],
+        "dk_linear_bwd_dgrad": [vp, pp, vp, vp, vp, vp],
+        "dk_relu_pool_fwd": [vp, vp, ctypes.c_int64, i32, i32, i32, i32, vp, vp],
+        "dk_relu_pool_bwd": [vp, vp, vp, ctypes.c_int64, i32, i32, i32, i32, vp, vp],
         "dk_linear_bwd_wgrad_verify": [vp, pp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, vp,
                                        ctypes.POINTER(dk_fault), vp],
         "dk_decode_verify_static": [ctypes.c_int, pp, vp, vp, vp, vp, vp, vp],
@@ -285,6 +289,28 @@ def dk_linear_bwd_wgrad(ctx: Context, p: dk_problem, delta, xbar, xbar_rows: int
     _check(lib().dk_linear_bwd_wgrad(ctx.handle, ctypes.byref(p), _dev(delta), _dev(xbar), xbar_rows,
                                      _host(C), _host(gamma), ctypes.c_float(scale), _dev(dW), _stream()),
            "dk_linear_bwd_wgrad")
+
+
+def dk_linear_bwd_wgrad_accumulate(ctx: Context, p: dk_problem, delta, xbar, xbar_rows: int, C: np.ndarray,
+                                   gamma: np.ndarray, scale: float, dW):
+    _check(lib().dk_linear_bwd_wgrad_accumulate(ctx.handle, ctypes.byref(p), _dev(delta), _dev(xbar), xbar_rows,
+                                                _host(C), _host(gamma), ctypes.c_float(scale), _dev(dW),
+                                                _stream()), "dk_linear_bwd_wgrad_accumulate")
+
+
+def dk_linear_bwd_dgrad(ctx: Context, p: dk_problem, W, delta, dx):
+    _check(lib().dk_linear_bwd_dgrad(ctx.handle, ctypes.byref(p), _dev(W), _dev(delta), _dev(dx), _stream()),
+           "dk_linear_bwd_dgrad")
+
+
+def dk_relu_pool_fwd(ctx: Context, x, n: int, h: int, w: int, c: int, pool: bool, y):
+    _check(lib().dk_relu_pool_fwd(ctx.handle, _dev(x), n, h, w, c, int(pool), _dev(y), _stream()),
+           "dk_relu_pool_fwd")
+
+
+def dk_relu_pool_bwd(ctx: Context, dy, x, n: int, h: int, w: int, c: int, pool: bool, dx):
+    _check(lib().dk_relu_pool_bwd(ctx.handle, _dev(dy), _dev(x), n, h, w, c, int(pool), _dev(dx), _stream()),
+           "dk_relu_pool_bwd")
 
 
 # ---------------------------------------------------------------------------

@@ -243,6 +243,12 @@ static WsPlan plan_workspace(const Geom& g) {
 static int* ctx_status_word(dk_ctx* ctx) {
   return reinterpret_cast<int*>(ctx->d_vstats + kVerifyStatFloats) + 2;
 }
+int* device_status_word(dk_ctx* ctx) { return ctx_status_word(ctx); }
+
+void workspace_offsets(const Geom& g, size_t* ybar, size_t* w_hi, size_t* w_lo) {
+  const WsPlan wp = plan_workspace(g);
+  *ybar = wp.ybar; *w_hi = wp.w_hi; *w_lo = wp.w_lo;
+}
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
@@ -575,7 +581,7 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
 // `xbar_elems` readable elements from `xbar` on).
 static dk_status wgrad_impl(dk_ctx* ctx, const Geom& g, const WsPlan& wp, const float* delta, const float* xbar,
                             int xbar_rows, long long xbar_elems, const float* C_host, const float* gamma_host,
-                            float scale, float* dW, cudaStream_t st) {
+                            float scale, float* dW, cudaStream_t st, bool accumulate = false) {
   CoefView cv;
   dk_status s = upload_coefficients(ctx, g, C_host, gamma_host, true, true, st, &cv);
   if (s != DK_OK) return s;
@@ -590,7 +596,8 @@ static dk_status wgrad_impl(dk_ctx* ctx, const Geom& g, const WsPlan& wp, const 
     {
       // one launch: mixed deltas and stored encodings as hi/lo pairs, dW cleared
       ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
-      s = tc_wgrad_prepass(g, delta, cv.dmix, dtil, dt_lo, xbar, xbar_elems, xb_hi, xb_lo, dW, ctx->sm_count, st);
+      s = tc_wgrad_prepass(g, delta, cv.dmix, dtil, dt_lo, xbar, xbar_elems, xb_hi, xb_lo,
+                           accumulate ? nullptr : dW, ctx->sm_count, st);
     }
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
@@ -602,7 +609,7 @@ static dk_status wgrad_impl(dk_ctx* ctx, const Geom& g, const WsPlan& wp, const 
   }
   if (s != DK_OK) return s;
   ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
-  return launch_simt_wgrad(g, dtil, xbar, xbar_rows, scale, dW, ctx->sm_count, st);
+  return launch_simt_wgrad(g, dtil, xbar, xbar_rows, scale, dW, ctx->sm_count, st, !accumulate);
 }
 
 dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* delta,
@@ -620,6 +627,23 @@ dk_status dk_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, const float* del
   if (!dg.ok) return DK_ERR_CUDA;
   return wgrad_impl(ctx, g, wp, delta, xbar, xbar_rows, (long long)g.G * xbar_rows * g.n_in, C_host, gamma_host,
                     scale, dW, static_cast<cudaStream_t>(stream));
+}
+
+dk_status dk_linear_bwd_wgrad_accumulate(dk_ctx* ctx, const dk_problem* p, const float* delta, const float* xbar,
+                                         int32_t xbar_rows, const float* C_host, const float* gamma_host,
+                                         float scale, float* dW, void* stream) {
+  if (!ctx || !delta || !xbar || !C_host || !gamma_host || !dW) return DK_ERR_INVALID_ARG;
+  if (!aligned16(delta) || !aligned16(xbar) || !aligned16(dW)) return DK_ERR_INVALID_ARG;
+  Geom g;
+  dk_status s = make_geom(p, &g);
+  if (s != DK_OK) return s;
+  if (xbar_rows != g.K + 1 && xbar_rows != g.K + 2) return DK_ERR_INVALID_ARG;
+  WsPlan wp = plan_workspace(g);
+  if (!ctx->ws || ctx->ws_bytes < wp.total) return DK_ERR_WORKSPACE;
+  DeviceGuard dg(ctx->device);
+  if (!dg.ok) return DK_ERR_CUDA;
+  return wgrad_impl(ctx, g, wp, delta, xbar, xbar_rows, (long long)g.G * xbar_rows * g.n_in, C_host, gamma_host,
+                    scale, dW, static_cast<cudaStream_t>(stream), true);
 }
 
 dk_status dk_linear_bwd_wgrad_verify(dk_ctx* ctx, const dk_problem* p, const float* delta, const float* xbar,

@@ -126,8 +126,14 @@ dk_status launch_simt_fwd64(const Geom& g, const float* W, const double* xbar, d
 dk_status launch_simt_fwd(const Geom& g, const float* W, const float* xbar, float* ybar,
                           int nsamples, cudaStream_t st);
 // dW = scale * sum_n <dtil[n], xbar[row(n)]> with row(n) = (n/(K+1))*xbar_rows + n%(K+1)
+// (clear = false adds to what dW holds)
 dk_status launch_simt_wgrad(const Geom& g, const float* dtil, const float* xbar, int xbar_rows,
-                            float scale, float* dW, int sm_count, cudaStream_t st);
+                            float scale, float* dW, int sm_count, cudaStream_t st, bool clear = true);
+
+// the context's status word (see dk_device_status) and the offsets of workspace regions that
+// other translation units borrow (dk_api.cu)
+int* device_status_word(dk_ctx* ctx);
+void workspace_offsets(const Geom& g, size_t* ybar, size_t* w_hi, size_t* w_lo);
 
 // Launch accounting: counts `nkernels` launches of `kind` and, when profiling
 // is on, brackets them with a pair of events on `st`.
@@ -174,7 +180,7 @@ dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const fl
                          float* xb_hi, float* xb_lo, const float* W, float* w_hi, float* w_lo,
                          const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st);
 // One launch for what a weight-gradient call prepares: Eq. 4 delta mixing and
-// the stored encodings as hi/lo pairs, dW cleared.
+// the stored encodings as hi/lo pairs, dW cleared (dW = nullptr: left as it is).
 dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix, float* dt_hi, float* dt_lo,
                            const float* xbar, long long xbar_elems, float* xb_hi, float* xb_lo, float* dW,
                            int sm_count, cudaStream_t st);

@@ -264,7 +264,7 @@ dk_status launch_simt_fwd64(const Geom& g, const float* W, const double* xbar, d
 }
 
 dk_status launch_simt_wgrad(const Geom& g, const float* dtil, const float* xbar, int xbar_rows,
-                            float scale, float* dW, int sm_count, cudaStream_t st) {
+                            float scale, float* dW, int sm_count, cudaStream_t st, bool clear) {
   WgParams p;
   p.d = dtil; p.x = xbar; p.dW = dW;
   p.cin = g.cin; p.cout = g.cout; p.h = g.h; p.w = g.w; p.kw = g.kw; p.stride = g.stride;
@@ -285,7 +285,7 @@ dk_status launch_simt_wgrad(const Geom& g, const float* dtil, const float* xbar,
   if (splits < 1) splits = 1;
   p.per_split = (p.GP + splits - 1) / splits;
   splits = (p.GP + p.per_split - 1) / p.per_split;
-  DK_CUDA_CHECK(cudaMemsetAsync(dW, 0, (size_t)g.cout * g.kc * sizeof(float), st));
+  if (clear) DK_CUDA_CHECK(cudaMemsetAsync(dW, 0, (size_t)g.cout * g.kc * sizeof(float), st));
   dim3 grid((unsigned)((g.kc + BN - 1) / BN), (unsigned)((g.cout + BM - 1) / BM), (unsigned)splits);
   if (grid.y > 65535) return DK_ERR_SHAPE;
   simt_wgrad_kernel<<<grid, NT, 0, st>>>(p);

@@ -185,8 +185,8 @@ dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix,
   a.per_g = job_blocks(g.n_out / 4, (cap + g.G - 1) / g.G);
   a.xbar = xbar; a.xb_hi = xb_hi; a.xb_lo = xb_lo; a.x4 = xbar_elems / 4;
   a.x_blocks = job_blocks(a.x4, cap);
-  a.dW = reinterpret_cast<float4*>(dW); a.dw4 = dwn / 4;
-  a.z_blocks = job_blocks(a.dw4, (long long)sm_count * 4);
+  a.dW = reinterpret_cast<float4*>(dW); a.dw4 = dW ? dwn / 4 : 0;
+  a.z_blocks = dW ? job_blocks(a.dw4, (long long)sm_count * 4) : 0;
   const long long blocks = (long long)a.G * a.per_g + a.x_blocks + a.z_blocks;
   if (blocks > 0x7fffffffLL) return DK_ERR_SHAPE;
 #define DK_PRE_CASE(KK) \
