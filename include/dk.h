@@ -43,6 +43,9 @@
  *    dk_set_workspace (size from dk_workspace_bytes).
  *  - A context is not thread-safe, and calls that share a context but run
  *    on different streams race on its scratch buffers.
+ *  - The library reads no environment variable and keeps no state outside its
+ *    contexts (dk_decode_verify_static's fixed scratch array excepted); what
+ *    can be tuned is a per-context option (dk_set_option).
  */
 #ifndef DK_H_
 #define DK_H_
@@ -125,6 +128,44 @@ typedef struct dk_ctx dk_ctx;
  * a few MB of device and pinned host memory for coefficient upload. */
 DK_API dk_status dk_create(dk_ctx** ctx, int device);
 DK_API dk_status dk_destroy(dk_ctx* ctx);
+
+/* Per-context options.  None is needed in normal use: the defaults are the
+ * measured best.  They exist for measurements (what a tiling choice costs), for
+ * cross-checks in the tests (another kernel for the same result) and for the
+ * failure-handling test.  A value outside an option's range is clamped.
+ *   DK_OPT_TC_CHUNK   32-wide k-blocks accumulated in tensor memory between two
+ *                     promotions to fp32 registers in the forward kernels
+ *                     (default 8, 1..64).  CHANGES THE ARITHMETIC: the tensor
+ *                     pipe truncates when it adds, so the error of y_bar grows
+ *                     with the chunk length.
+ *   DK_OPT_WG_CHUNK   the same for the weight-gradient kernel (default 2, 1..64);
+ *                     changes the arithmetic likewise.
+ *   DK_OPT_TC_BK      k-block of the forward kernel: 32 (default) or 16 floats.
+ *   DK_OPT_TC_PAIR    1 (default): layers with more than 128 output channels and
+ *                     even K run on pairs of CTAs; 0: one CTA per tile.
+ *   DK_OPT_WG_PACK    1 (default): the weight-gradient kernel puts several filter
+ *                     taps side by side for layers with few input channels.
+ *   DK_OPT_WG_PAIR    1 (default): CTA pairs in the weight-gradient kernel.
+ *   DK_OPT_TC_STEM    1 (default): 3-channel stems run on the tensor-core kernels
+ *                     through patch rows; 0: on the fp32 kernels.
+ *   DK_OPT_FIELD_PATH contraction kernels of the finite-field calls: 0 (default)
+ *                     tensor cores (tcgen05 where the shape allows, else mma.sync),
+ *                     1 the 64-bit integer-ALU kernels, 2 mma.sync only.
+ *   DK_OPT_SPIN_LIMIT polls after which a device-side wait gives up and the call
+ *                     reports DK_ERR_TIMEOUT (default 2^22, 2^10..2^26).
+ *   DK_OPT_TEST_WITHHOLD  test hook, default -1 (off): the producer warp of the
+ *                     next tensor-core forward or weight-gradient kernel arms the
+ *                     barrier of its n-th pipeline stage but issues no copy for
+ *                     it and stops, so every consumer's wait runs out; nothing is
+ *                     read or written out of bounds.  The option switches itself
+ *                     off after one launch. */
+enum {
+  DK_OPT_TC_CHUNK = 0, DK_OPT_WG_CHUNK = 1, DK_OPT_TC_BK = 2, DK_OPT_TC_PAIR = 3, DK_OPT_WG_PACK = 4,
+  DK_OPT_WG_PAIR = 5, DK_OPT_TC_STEM = 6, DK_OPT_FIELD_PATH = 7, DK_OPT_SPIN_LIMIT = 8,
+  DK_OPT_TEST_WITHHOLD = 9, DK_OPT_COUNT = 10
+};
+DK_API dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value);
+DK_API dk_status dk_get_option(dk_ctx* ctx, int32_t option, int32_t* value);
 
 /* Human-readable name of a status code (static storage). */
 DK_API const char* dk_status_string(dk_status s);

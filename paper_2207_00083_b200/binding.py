@@ -21,6 +21,9 @@ LIB_PATH = os.path.join(_HERE, "libdk.so")
 DK_FC, DK_CONV2D = 0, 1
 DK_NHWC, DK_NCHW = 0, 1
 DK_PREC_DEFAULT, DK_TF32X3, DK_FP32_SIMT, DK_FP64_SIMT = 0, 1, 2, 3
+(DK_OPT_TC_CHUNK, DK_OPT_WG_CHUNK, DK_OPT_TC_BK, DK_OPT_TC_PAIR, DK_OPT_WG_PACK, DK_OPT_WG_PAIR, DK_OPT_TC_STEM,
+ DK_OPT_FIELD_PATH, DK_OPT_SPIN_LIMIT, DK_OPT_TEST_WITHHOLD) = range(10)
+DK_ERR_TIMEOUT = 6
 STATUS_NAMES = ["DK_OK", "DK_ERR_INVALID_ARG", "DK_ERR_SHAPE", "DK_ERR_SINGULAR", "DK_ERR_WORKSPACE",
                 "DK_ERR_CUDA", "DK_ERR_TIMEOUT", "DK_ERR_UNSUPPORTED"]
 
@@ -71,6 +74,8 @@ def _signatures():
         "dk_status_string": [ctypes.c_int],
         "dk_workspace_bytes": [pp, ctypes.POINTER(ctypes.c_size_t)],
         "dk_set_workspace": [vp, vp, ctypes.c_size_t],
+        "dk_set_option": [vp, i32, i32],
+        "dk_get_option": [vp, i32, ctypes.POINTER(i32)],
         "dk_encode": [vp, pp, vp, vp, vp, vp, vp],
         "dk_linear_fwd": [vp, pp, vp, vp, vp, vp],
         "dk_decode_verify": [vp, pp, vp, vp, vp, vp, vp, vp],
@@ -199,6 +204,16 @@ class Context:
         off = (-base) % 256
         _check(lib().dk_set_workspace(self._h, ctypes.c_void_p(base + off), self._ws.numel() - off),
                "dk_set_workspace")
+
+
+def dk_set_option(ctx: Context, option: int, value: int):
+    _check(lib().dk_set_option(ctx.handle, option, value), "dk_set_option")
+
+
+def dk_get_option(ctx: Context, option: int) -> int:
+    v = ctypes.c_int32()
+    _check(lib().dk_get_option(ctx.handle, option, ctypes.byref(v)), "dk_get_option")
+    return v.value
 
 
 KERNEL_KINDS = ["encode", "linear_fwd", "decode_verify", "mix_delta", "wgrad", "other"]

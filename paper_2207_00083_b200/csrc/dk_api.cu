@@ -303,6 +303,8 @@ dk_status dk_create(dk_ctx** out, int device) {
     return DK_ERR_CUDA;
   }
   c->sm_count = sms;
+  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1};
+  for (int i = 0; i < DK_OPT_COUNT; ++i) c->opt.v[i] = kOptDefault[i];
   bool ok = cudaMallocHost(&c->h_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_vstats, (kVerifyStatFloats + 64) * sizeof(float)) == cudaSuccess &&
@@ -334,6 +336,22 @@ dk_status dk_destroy(dk_ctx* c) {
   if (c->d_vstats) cudaFree(c->d_vstats);
   if (c->d_cand) cudaFree(c->d_cand);
   delete c;
+  return DK_OK;
+}
+
+dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value) {
+  if (!ctx || option < 0 || option >= DK_OPT_COUNT) return DK_ERR_INVALID_ARG;
+  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1};
+  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 1, 2, 1 << 26, 1 << 20};
+  int v = value < lo[option] ? lo[option] : (value > hi[option] ? hi[option] : value);
+  if (option == DK_OPT_TC_BK) v = v == 16 ? 16 : 32;
+  ctx->opt.v[option] = v;
+  return DK_OK;
+}
+
+dk_status dk_get_option(dk_ctx* ctx, int32_t option, int32_t* value) {
+  if (!ctx || !value || option < 0 || option >= DK_OPT_COUNT) return DK_ERR_INVALID_ARG;
+  *value = ctx->opt.v[option];
   return DK_OK;
 }
 

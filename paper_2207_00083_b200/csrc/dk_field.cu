@@ -818,7 +818,6 @@ constexpr int STAGE = 4 * A_PLANE + 4 * B_PLANE;                 // 96 KB
 constexpr int kStages = 2;
 constexpr size_t kSmem = (size_t)kStages * STAGE + 1024;         // + slack for 1024-byte alignment
 constexpr int kFoldTiles = 8192 / TK;                            // 4 pairs * 255^2 * 8192 < 2^31
-constexpr unsigned kSpin = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -835,8 +834,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (unsigned i = 0; i < kSpin; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned cap) {
+  for (unsigned i = 0; i < cap; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u && *abort_flag) return false;
   }
@@ -901,7 +900,9 @@ __global__ void __launch_bounds__(256) field_w_planes_kernel(const u32* __restri
 __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParams p, MmaConsts mc,
                                                                        const uint8_t* __restrict__ wplanes, int kcp,
                                                                        u64* split_acc, int tiles_per_split,
-                                                                       int* status) {
+                                                                       int* status, unsigned spin_cap, int withhold) {
+  // spin_cap: polls after which a wait gives up; withhold (test hook, -1 = off): thread 0 does not arrive
+  // for that k-tile's stage and stops, so every other role's wait runs out
   using namespace tcf;
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[kStages];     // a stage's planes are in shared memory (kProducers arrivals)
@@ -969,7 +970,7 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
       bool fresh = true;               // no product since the last fold
       for (int kt = 0; kt < ntiles; ++kt) {
         const int stage = kt & 1;
-        if (!mbar_wait(full_bar + stage, (uint32_t)((kt / kStages) & 1), abort_flag)) break;
+        if (!mbar_wait(full_bar + stage, (uint32_t)((kt / kStages) & 1), abort_flag, spin_cap)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE), sb = sa + 4 * A_PLANE;
         const uint64_t bdesc = plane_desc(sb);
@@ -1004,7 +1005,7 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
       const int stage = kt & 1;
       uint8_t* st = smem + (size_t)stage * STAGE;
       // the products that read this stage two k-tiles ago must have completed
-      if (kt >= kStages && !mbar_wait(mma_done + stage, (uint32_t)((kt / kStages - 1) & 1), abort_flag)) {
+      if (kt >= kStages && !mbar_wait(mma_done + stage, (uint32_t)((kt / kStages - 1) & 1), abort_flag, spin_cap)) {
         alive = false;
         break;
       }
@@ -1066,6 +1067,7 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
       asm volatile("cp.async.wait_group 0;\n" ::);
       // make the planes visible to the tensor core's (asynchronous-proxy) reads, then hand the stage over
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      if (t == 0 && kt == withhold) { alive = false; break; }      // test hook: this stage never becomes full
       asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(full_bar + stage)) : "memory");
 
       // fold before a class sum can overflow, and at the end
@@ -1073,7 +1075,7 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
       if (last || ((kt + 1) % kFoldTiles) == 0) {
         // every product issued so far has completed once the commit of this k-tile has arrived
         // (a commit covers all earlier products of the issuing thread)
-        if (!mbar_wait(mma_done + stage, (uint32_t)((kt / kStages) & 1), abort_flag)) {
+        if (!mbar_wait(mma_done + stage, (uint32_t)((kt / kStages) & 1), abort_flag, spin_cap)) {
           alive = false;
           break;
         }
@@ -1123,24 +1125,15 @@ long long terms_per_reduction(u32 p) {
 
 bool aligned16(const void* p);
 
-// DK_FIELD_SIMT=1 selects the 64-bit integer-ALU kernel instead of the tensor-core one (a cross-check).
-bool field_use_simt() {
-  static const bool v = [] {
-    const char* e = getenv("DK_FIELD_SIMT");
-    return e && e[0] == '1';
-  }();
-  return v;
+// the test hook DK_OPT_TEST_WITHHOLD serves one launch
+int take_withhold(dk_ctx* ctx) {
+  const int w = ctx->opt.v[DK_OPT_TEST_WITHHOLD];
+  ctx->opt.v[DK_OPT_TEST_WITHHOLD] = -1;
+  return w;
 }
 
-// DK_FIELD_MMA_SYNC=1 keeps the forward contraction on the mma.sync kernel (a cross-check of the tcgen05 one).
-bool field_use_mma_sync() {
-  static const bool v = [] {
-    const char* e = getenv("DK_FIELD_MMA_SYNC");
-    return e && e[0] == '1';
-  }();
-  return v;
-}
-
+// `path` (option DK_OPT_FIELD_PATH): 0 = tensor cores (tcgen05 where the shape allows, else mma.sync),
+// 1 = the 64-bit integer-ALU kernels, 2 = mma.sync only (1 and 2 are cross-checks of the default).
 // `wplanes` (nullable): device scratch of at least 4 * cout * round_up(kc, 128) bytes for the digit planes of W;
 // without it the contraction runs on the mma.sync kernel.
 __global__ void field_reduce_kernel(const u64* __restrict__ acc, long long n, Modulus md, u32* __restrict__ out);
@@ -1165,7 +1158,7 @@ int field_fwd_slices(long long ctas, int ntiles, int sms) {
 // in which slices of the contraction meet when a layer has too few output tiles to fill the device.
 dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* ybar, int nsamples, Modulus md,
                            uint8_t* wplanes, size_t wplanes_bytes, u64* split_acc, size_t split_bytes, int sm_count,
-                           int* status, cudaStream_t st) {
+                           int* status, int path, unsigned spin_cap, int withhold, cudaStream_t st) {
   FwdParams p;
   p.W = W; p.x = xbar; p.y = ybar;
   p.cin = g.cin; p.cout = g.cout; p.h = g.h; p.w = g.w; p.kw = g.kw; p.stride = g.stride;
@@ -1185,14 +1178,14 @@ dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* yb
   dim3 grid((unsigned)nb, (unsigned)((g.cout + BM - 1) / BM));
   if (grid.y > 65535) return DK_ERR_SHAPE;
   static_assert(BM == MMA_BM && BN == MMA_BN, "one grid shape serves both kernels");
-  if (field_use_simt()) {
+  if (path == 1) {
     field_fwd_kernel<<<grid, NT, 0, st>>>(p);
   } else {
     MmaConsts mc;
     mc.pow32 = (u32)((1ull << 32) % md.p);
     const bool vec4 = g.xs_c == 1 && g.ws_c == 1 && (g.cin % 4) == 0 && aligned16(W) && aligned16(xbar);
     const int kcp = (g.kc + tcf::TK - 1) / tcf::TK * tcf::TK;
-    if (vec4 && !field_use_mma_sync() && wplanes != nullptr && wplanes_bytes >= (size_t)4 * g.cout * kcp) {
+    if (vec4 && path != 2 && wplanes != nullptr && wplanes_bytes >= (size_t)4 * g.cout * kcp) {
       static const bool tc_attr_ok =
           cudaFuncSetAttribute(field_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)tcf::kSmem) == cudaSuccess;
@@ -1211,11 +1204,11 @@ dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* yb
         const int tps = (ntiles + ns - 1) / ns;
         tgrid.z = (unsigned)((ntiles + tps - 1) / tps);
         DK_CUDA_CHECK(cudaMemsetAsync(split_acc, 0, (size_t)n_y * sizeof(u64), st));
-        field_fwd_tc_kernel<<<tgrid, tcf::kThreads, tcf::kSmem, st>>>(p, mc, wplanes, kcp, split_acc, tps, status);
+        field_fwd_tc_kernel<<<tgrid, tcf::kThreads, tcf::kSmem, st>>>(p, mc, wplanes, kcp, split_acc, tps, status, spin_cap, withhold);
         DK_CUDA_CHECK(cudaGetLastError());
         field_reduce_kernel<<<ew_blocks(n_y, sm_count), 256, 0, st>>>(split_acc, n_y, md, ybar);
       } else {
-        field_fwd_tc_kernel<<<tgrid, tcf::kThreads, tcf::kSmem, st>>>(p, mc, wplanes, kcp, nullptr, ntiles, status);
+        field_fwd_tc_kernel<<<tgrid, tcf::kThreads, tcf::kSmem, st>>>(p, mc, wplanes, kcp, nullptr, ntiles, status, spin_cap, withhold);
       }
       DK_CUDA_CHECK(cudaGetLastError());
       return DK_OK;
@@ -1710,7 +1703,8 @@ dk_status dk_field_linear_fwd(dk_ctx* ctx, const dk_problem* p, uint32_t prime, 
                           have_ws ? reinterpret_cast<uint8_t*>(static_cast<char*>(ctx->ws) + wp.wpl) : nullptr,
                           have_ws ? wp.wpl_bytes : 0,
                           have_ws ? reinterpret_cast<u64*>(static_cast<char*>(ctx->ws) + wp.acc64) : nullptr,
-                          have_ws ? wp.total - wp.acc64 : 0, ctx->sm_count, field_status_word(ctx), st);
+                          have_ws ? wp.total - wp.acc64 : 0, ctx->sm_count, field_status_word(ctx), ctx->opt.v[DK_OPT_FIELD_PATH], (unsigned)ctx->opt.v[DK_OPT_SPIN_LIMIT],
+                          take_withhold(ctx), st);
 }
 
 dk_status dk_field_decode_verify(dk_ctx* ctx, const dk_problem* p, uint32_t prime, int32_t l,
@@ -1781,7 +1775,8 @@ dk_status dk_field_masked_linear(dk_ctx* ctx, const dk_problem* p, uint32_t prim
     ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
     s = launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, reinterpret_cast<uint8_t*>(ws + wp.wpl), wp.wpl_bytes,
                          reinterpret_cast<u64*>(ws + wp.acc64), wp.total - wp.acc64, ctx->sm_count,
-                         field_status_word(ctx), st);
+                         field_status_word(ctx), ctx->opt.v[DK_OPT_FIELD_PATH], (unsigned)ctx->opt.v[DK_OPT_SPIN_LIMIT],
+                          take_withhold(ctx), st);
   }
   if (s != DK_OK) return s;
   if (fault) {
@@ -1824,7 +1819,7 @@ dk_status dk_field_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, uint32_t p
   const long long n_dw = (long long)g.cout * g.kc;
   const long long tiles = (long long)((g.cout + BM - 1) / BM) * ((g.kc + BN - 1) / BN);
   if ((g.cout + BM - 1) / BM > 65535) return DK_ERR_SHAPE;
-  if (field_use_simt()) {
+  if (ctx->opt.v[DK_OPT_FIELD_PATH] == 1) {
     WgParams wg;
     wg.d = dtil; wg.x = xbar; wg.acc = acc;
     wg.cin = g.cin; wg.cout = g.cout; wg.h = g.h; wg.w = g.w; wg.kw = g.kw; wg.stride = g.stride;

@@ -66,6 +66,11 @@ struct VerifyScratch {
 
 struct ProfState;
 
+// Per-context options (dk_set_option), indexed by DK_OPT_*.
+struct Options {
+  int v[DK_OPT_COUNT];
+};
+
 }  // namespace dk
 
 struct dk_ctx {
@@ -82,6 +87,7 @@ struct dk_ctx {
   dk::Candidate* d_cand;      // kCandCap entries
   void* tc_state;             // tensor-core path state
   dk::ProfState* prof;        // launch counters and event records
+  dk::Options opt;
 };
 
 namespace dk {

@@ -2,8 +2,6 @@
 // the HBM-bound pre-passes that write the TF32 hi/lo split operands.
 #include <cuda.h>
 
-#include <stdlib.h>
-
 #include <new>
 
 #include "dk_internal.h"
@@ -25,6 +23,7 @@ struct TcState {
   EncodeTiledFn encode;
   int smem_optin;
   int device;
+  Options* opt;             // the context's options (dk_set_option)
 };
 
 // What the launch of one kernel instantiation needs to know about it, looked
@@ -83,24 +82,10 @@ int resident_pairs(Kern kern, KernelCache& kc, int dev, size_t smem, int sm_coun
 
 constexpr int kSwz128Atom32 = 1128;
 constexpr int kBK = 32;          // k-block: 32 fp32 = one 128-byte swizzle span per row
-constexpr int kChunk = 8;        // 32-wide k-blocks accumulated in TMEM between promotions (error grows ~linearly with it)
-
-// Tuning knobs read once from the environment (defaults are the measured best):
-//   DK_TC_CHUNK  k-blocks per TMEM chunk in the forward kernel
-//   DK_WG_CHUNK  k-blocks per TMEM chunk in the weight-gradient kernel
-int env_knob(const char* name, int dflt, int lo, int hi) {
-  const char* v = getenv(name);
-  if (!v || !*v) return dflt;
-  int x = atoi(v);
-  return x < lo ? lo : (x > hi ? hi : x);
-}
 
 // k-block of the forward kernel: 32 fp32 (128-byte rows, fewer and larger
 // stages) or 16 (64-byte rows, twice as many stages in the same shared memory)
-int fwd_bk() {
-  static const int bk = env_knob("DK_TC_BK", kBK, 16, 32) == 16 ? 16 : 32;
-  return bk;
-}
+int fwd_bk(const TcState* ts) { return ts->opt->v[DK_OPT_TC_BK] == 16 ? 16 : 32; }
 
 // ---------------------------------------------------------------------------
 // HBM-bound pre-passes: TF32 hi/lo split, alone or fused with the encoder
@@ -312,14 +297,17 @@ dk_status launch_k(const TcState* ts, const Geom& g, const Tiling& tl, const flo
   return DK_ERR_SHAPE;
 }
 
-void fill_params(const Geom& g, const Tiling& tl, TcParams* p) {
+void fill_params(const TcState* ts, const Geom& g, const Tiling& tl, TcParams* p) {
   p->bw = tl.bw; p->bh = tl.bh; p->bg = tl.bg;
   p->log2_bw = 0; while ((1 << p->log2_bw) < tl.bw) ++p->log2_bw;
   p->log2_S = 0; while ((1 << p->log2_S) < tl.bw * tl.bh) ++p->log2_S;
   p->WT = tl.WT; p->HT = tl.HT; p->GT = tl.GT; p->MT = tl.MT;
   p->ntiles = tl.ntiles; p->KB = tl.KB; p->CB = tl.CB;
-  static const int chunk = env_knob("DK_TC_CHUNK", kChunk, 1, 64);
-  p->chunk = chunk * (32 / fwd_bk());   // the knob counts 32-wide k-blocks
+  // 32-wide k-blocks accumulated in TMEM between promotions (the error grows ~linearly with it)
+  p->chunk = ts->opt->v[DK_OPT_TC_CHUNK] * (32 / fwd_bk(ts));
+  p->spin_cap = (unsigned)ts->opt->v[DK_OPT_SPIN_LIMIT];
+  p->withhold = ts->opt->v[DK_OPT_TEST_WITHHOLD];
+  ts->opt->v[DK_OPT_TEST_WITHHOLD] = -1;      // the hook serves one launch
   p->ksplit = 1;
   p->kb_per_split = tl.KB;
   p->kw = g.kw; p->pad = g.pad; p->stride = g.stride; p->nstages = tl.nstages;
@@ -335,15 +323,15 @@ void fill_params(const Geom& g, const Tiling& tl, TcParams* p) {
 }
 
 // CTA pairs serve layers with more than 128 output channels and an even
-// number of encodings (DK_TC_PAIR=0 switches them off)
-bool use_pair(const Geom& g) {
-  static const int on = env_knob("DK_TC_PAIR", 1, 0, 1);
-  return on && fwd_bk() == 32 && g.cout > BM && (g.E % 2) == 0;
+// number of encodings (option DK_OPT_TC_PAIR switches them off)
+bool use_pair(const TcState* ts, const Geom& g) {
+  return ts->opt->v[DK_OPT_TC_PAIR] && fwd_bk(ts) == 32 && g.cout > BM && (g.E % 2) == 0;
 }
 
-bool plan_fwd(const Geom& g, int smem_optin, Tiling* t) {
-  if (use_pair(g) && plan_tiling<32>(g, smem_optin, t, true)) return true;
-  return fwd_bk() == 16 ? plan_tiling<16>(g, smem_optin, t) : plan_tiling<32>(g, smem_optin, t);
+bool plan_fwd(const TcState* ts, const Geom& g, Tiling* t) {
+  const int smem_optin = ts->smem_optin;
+  if (use_pair(ts, g) && plan_tiling<32>(g, smem_optin, t, true)) return true;
+  return fwd_bk(ts) == 16 ? plan_tiling<16>(g, smem_optin, t) : plan_tiling<32>(g, smem_optin, t);
 }
 
 template <int MODE>
@@ -362,7 +350,7 @@ template <int MODE>
 dk_status launch_bk(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
                     const float* xb_hi, const float* xb_lo, TcParams& prm, int sm_count, cudaStream_t st) {
   if (tl.pair) return launch_pair<MODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
-  return fwd_bk() == 16 ? launch_k<16, MODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st)
+  return fwd_bk(ts) == 16 ? launch_k<16, MODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st)
                         : launch_k<32, MODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, sm_count, st);
 }
 
@@ -386,6 +374,7 @@ dk_status tc_init(dk_ctx* ctx) {
   }
   ts->smem_optin = optin;
   ts->device = ctx->device;
+  ts->opt = &ctx->opt;
   ctx->tc_state = ts;
   return DK_OK;
 }
@@ -400,7 +389,7 @@ bool tc_fwd_supported(const dk_ctx* ctx, const Geom& g) {
   if (g.layout != DK_NHWC || g.stride < 1 || g.stride > 4 || (g.cin % 4) != 0) return false;
   if (g.n_out >= (1LL << 31)) return false;     // the epilogue keeps pixel offsets in 32 bits
   Tiling tl;
-  return plan_fwd(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, &tl);
+  return plan_fwd(static_cast<TcState*>(ctx->tc_state), g, &tl);
 }
 
 dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_count, cudaStream_t st) {
@@ -445,10 +434,10 @@ dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const f
 int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
-  if (!ts || !plan_fwd(g, ts->smem_optin, &tl)) return 1;
+  if (!ts || !plan_fwd(ts, g, &tl)) return 1;
   const int units = tl.pair ? ctx->sm_count / 2 : ctx->sm_count;     // CTAs or CTA pairs that run together
   if (tl.ntiles >= units) return 1;
-  const int unit_kb = 32 / fwd_bk();             // k-blocks per 32 contraction elements
+  const int unit_kb = 32 / fwd_bk(ts);           // k-blocks per 32 contraction elements
   const int cap = tl.KB / (8 * unit_kb);
   const long long kItem = 6 * unit_kb, kUnfused = 20 * unit_kb;
   int best = 1;
@@ -470,9 +459,9 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
                         cudaStream_t st) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
-  if (!plan_fwd(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
+  if (!plan_fwd(ts, g, &tl)) return DK_ERR_UNSUPPORTED;
   TcParams prm;
-  fill_params(g, tl, &prm);
+  fill_params(ts, g, tl, &prm);
   if (ksplit > 1) {
     prm.kb_per_split = (tl.KB + ksplit - 1) / ksplit;
     prm.ksplit = (tl.KB + prm.kb_per_split - 1) / prm.kb_per_split;
@@ -490,9 +479,9 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
                         cudaStream_t st) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
-  if (!plan_fwd(g, ts->smem_optin, &tl)) return DK_ERR_UNSUPPORTED;
+  if (!plan_fwd(ts, g, &tl)) return DK_ERR_UNSUPPORTED;
   TcParams prm;
-  fill_params(g, tl, &prm);
+  fill_params(ts, g, tl, &prm);
   prm.out = y;
   prm.dec = cv.dec; prm.decl = cv.decl; prm.nul = cv.nul; prm.bias = bias;
   prm.vs = vs;
@@ -516,7 +505,6 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
 // ---------------------------------------------------------------------------
 namespace {
 
-constexpr int kWgChunk = 2;      // k-blocks accumulated in TMEM between promotions
 
 // dtil[g*(K+1)+j] = sum_i dmix[g][j][i] * delta[g*K+i], written as a TF32 hi/lo pair (Eq. 4).
 template <int K>
@@ -565,7 +553,7 @@ struct WgPlan {
   size_t smem_bytes;
 };
 
-bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
+bool plan_wgrad(const Options& opt, const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   WgTcParams& p = w->prm;
   const int P = kWgPix;
   long long best = -1;
@@ -591,7 +579,7 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   // once per 64 or 128 columns); putting several filter taps side by side keeps
   // N at 192 or 256.
   p.taps = g.kh * g.kw;
-  static const int pack_on = env_knob("DK_WG_PACK", 1, 0, 1);
+  const int pack_on = opt.v[DK_OPT_WG_PACK];
   if (g.cin <= 64) {
     p.cb = 64;
     p.tpn = !pack_on || p.taps == 1 ? 1 : (p.taps % 3 == 0 || p.taps < 4 ? (p.taps < 3 ? p.taps : 3) : 4);
@@ -604,7 +592,7 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   }
   w->BN = p.cb * p.tpn;
   p.TG = (p.taps + p.tpn - 1) / p.tpn;
-  static const int pair_on = env_knob("DK_WG_PAIR", 1, 0, 1);
+  const int pair_on = opt.v[DK_OPT_WG_PAIR];
   w->pair = pair_on && g.cout > BM;
   p.MT = w->pair ? (g.cout + BM2 - 1) / BM2 : (g.cout + BM - 1) / BM;
   const int units = w->pair ? sm_count / 2 : sm_count;     // CTAs or CTA pairs that run together
@@ -634,8 +622,9 @@ bool plan_wgrad(const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
   if (items > 0x7fffffffLL) return false;
   p.nitems = (int)items;
   p.kw = g.kw; p.pad = g.pad; p.stride = g.stride;
-  static const int wg_chunk = env_knob("DK_WG_CHUNK", kWgChunk, 1, 64);
-  p.chunk = wg_chunk;
+  p.chunk = opt.v[DK_OPT_WG_CHUNK];      // k-blocks accumulated in TMEM between promotions
+  p.spin_cap = (unsigned)opt.v[DK_OPT_SPIN_LIMIT];
+  p.withhold = -1;
   p.cout = g.cout; p.cin = g.cin;
   const size_t stage = 2 * ((size_t)(BM / 32) * kWgBox + (size_t)((w->pair ? w->BN / 2 : w->BN) / 32) * kWgBox);
   const size_t ctrl = 1024 + 256;
@@ -682,12 +671,11 @@ bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g) {
   if (g.precision != DK_TF32X3 || ctx->tc_state == nullptr) return false;
   if (g.layout != DK_NHWC || g.stride < 1 || g.stride > 4 || (g.cin % 4) != 0 || (g.cout % 4) != 0) return false;
   WgPlan w;
-  return plan_wgrad(g, static_cast<TcState*>(ctx->tc_state)->smem_optin, ctx->sm_count, &w);
+  return plan_wgrad(ctx->opt, g, static_cast<TcState*>(ctx->tc_state)->smem_optin, ctx->sm_count, &w);
 }
 
 bool tc_stem_supported(const dk_ctx* ctx, const Geom& g) {
-  static const int on = env_knob("DK_TC_STEM", 1, 0, 1);
-  if (!on || g.kind != DK_CONV2D || g.layout != DK_NHWC || g.precision != DK_TF32X3) return false;
+  if (!ctx->opt.v[DK_OPT_TC_STEM] || g.kind != DK_CONV2D || g.layout != DK_NHWC || g.precision != DK_TF32X3) return false;
   if ((g.cin % 4) == 0 || g.kc > 256 || (g.cout % 4) != 0) return false;
   const Geom s = tc_stem_gemm_geom(g);
   return tc_fwd_supported(ctx, s);
@@ -719,7 +707,9 @@ dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* 
                    cudaStream_t st) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   WgPlan w;
-  if (!plan_wgrad(g, ts->smem_optin, ctx->sm_count, &w)) return DK_ERR_UNSUPPORTED;
+  if (!plan_wgrad(ctx->opt, g, ts->smem_optin, ctx->sm_count, &w)) return DK_ERR_UNSUPPORTED;
+  w.prm.withhold = ctx->opt.v[DK_OPT_TEST_WITHHOLD];
+  ctx->opt.v[DK_OPT_TEST_WITHHOLD] = -1;      // the hook serves one launch
   w.prm.scale = scale;
   w.prm.dW = dW;
   w.prm.status = status_word;

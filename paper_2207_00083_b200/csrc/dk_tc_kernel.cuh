@@ -41,7 +41,6 @@ constexpr int BM = 128;            // output channels per tile = TMEM lanes
 constexpr int kEpiWarps = 8;
 constexpr int kThreadsTc = 32 * (4 + kEpiWarps);   // warpgroup 0: TMA, MMA, two idle warps
 constexpr int kMaxStages = 8;
-constexpr unsigned kSpinCap = 1u << 22;
 constexpr int MODE_YBAR = 0, MODE_DECODE = 1;
 
 // Pixels per encoding in one N tile, by virtual-batch size: (K+2)*P is a legal
@@ -62,6 +61,8 @@ struct TcParams {
   int ksplit, kb_per_split;    // contraction slices per tile (slices add into `out` with atomics)
   int kw, pad, stride;
   int nstages;
+  unsigned spin_cap;           // polls after which a wait gives up
+  int withhold;                // test hook: the producer arms its n-th stage but issues no copy (-1 = off)
   // problem
   int cout, ho, wo, G;
   long long n_out;
@@ -112,9 +113,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false (and raises the CTA's abort flag) when the
-// barrier did not complete within kSpinCap polls or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (unsigned i = 0; i < kSpinCap; ++i) {
+// barrier did not complete within `cap` polls or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned cap) {
+  for (unsigned i = 0; i < cap; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u && *abort_flag) return false;
   }
@@ -532,7 +533,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
     // barrier, then lanes 0..2E+1 issue one bulk tensor copy each, so that the
     // 2E+2 copies of a stage are issued side by side instead of one after another.
     {
-      int stage = 0;
+      int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool alive = true;
       for (int w = blockIdx.x; alive && w < nwork; w += gridDim.x) {
@@ -548,11 +549,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
         for (int kb = kb_lo; kb < kb_hi; ++kb) {
           int ok = 1;
           if (lane == 0) {
-            ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag) ? 1 : 0;
+            ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
             if (ok) mbar_expect_tx(full_bar + stage, (uint32_t)STAGE_BYTES);
           }
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) { alive = false; break; }
+          if (issued++ == p.withhold) { alive = false; break; }      // test hook: armed, nothing copied
           const int tap = kb / p.CB, c0 = (kb - tap * p.CB) * BK;
           const int u = tap / p.kw, v = tap - u * p.kw;
           unsigned char* st = smem + (size_t)stage * STAGE_BYTES;
@@ -589,12 +591,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
         const int nchunks = (kb_hi - kb_lo + p.chunk - 1) / p.chunk;
         for (int ci = 0; alive && ci < nchunks; ++ci, ++acc_it) {
           const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
-          if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag)) { alive = false; break; }
+          if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag, p.spin_cap)) { alive = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * 256u;
           const int kb_beg = kb_lo + ci * p.chunk, kb_end = min(kb_hi, kb_beg + p.chunk);
           for (int kb = kb_beg; kb < kb_end; ++kb) {
-            if (!mbar_wait(full_bar + stage, phase, abort_flag)) { alive = false; break; }
+            if (!mbar_wait(full_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
             tc_fence_after();
             const uint32_t st = smem_u32(smem + (size_t)stage * STAGE_BYTES);
             const uint64_t a_hi = make_desc<SWZ>(st), a_lo = make_desc<SWZ>(st + A_BYTES);
@@ -639,7 +641,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
       // ---- sum the chunks of this tile in registers (round to nearest) ----
       for (int ci = 0; ci < nchunks; ++ci, ++acc_it) {
         const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
-        if (!mbar_wait(tfull_bar + buf, aphase, abort_flag)) { alive = false; break; }
+        if (!mbar_wait(tfull_bar + buf, aphase, abort_flag, p.spin_cap)) { alive = false; break; }
         tc_fence_after();
         const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * PH);
 #pragma unroll

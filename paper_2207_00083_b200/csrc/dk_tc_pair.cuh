@@ -137,7 +137,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
   asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
   if (warp == 0) {
     // ---------------- TMA producer (both CTAs) ----------------
-    int stage = 0;
+    int stage = 0, issued = 0;
     uint32_t phase = 0;
     bool alive = true;
     for (int w = pair; alive && w < nwork; w += npairs) {
@@ -153,11 +153,12 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
       for (int kb = kb_lo; kb < kb_hi; ++kb) {
         int ok = 1;
         if (lane == 0) {
-          ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag) ? 1 : 0;
+          ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
           if (ok && rank == 0) mbar_expect_tx(full_bar + stage, (uint32_t)(2 * STAGE_BYTES));
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) { alive = false; break; }
+        if (issued++ == p.withhold) { alive = false; break; }      // test hook: armed, nothing copied
         const int tap = kb / p.CB, c0 = (kb - tap * p.CB) * BK;
         const int u = tap / p.kw, v = tap - u * p.kw;
         unsigned char* st = smem + (size_t)stage * STAGE_BYTES;
@@ -193,12 +194,12 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         const int nchunks = (kb_hi - kb_lo + p.chunk - 1) / p.chunk;
         for (int ci = 0; alive && ci < nchunks; ++ci, ++acc_it) {
           const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
-          if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag)) { alive = false; break; }
+          if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag, p.spin_cap)) { alive = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * 256u;
           const int kb_beg = kb_lo + ci * p.chunk, kb_end = min(kb_hi, kb_beg + p.chunk);
           for (int kb = kb_beg; kb < kb_end; ++kb) {
-            if (!mbar_wait(full_bar + stage, phase, abort_flag)) { alive = false; break; }
+            if (!mbar_wait(full_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
             tc_fence_after();
             const uint32_t st = smem_u32(smem + (size_t)stage * STAGE_BYTES);
             const uint64_t a_hi = make_desc<SWZ>(st), a_lo = make_desc<SWZ>(st + A_BYTES);
@@ -242,7 +243,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
 
       for (int ci = 0; ci < nchunks; ++ci, ++acc_it) {
         const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
-        if (!mbar_wait(tfull_bar + buf, aphase, abort_flag)) { alive = false; break; }
+        if (!mbar_wait(tfull_bar + buf, aphase, abort_flag, p.spin_cap)) { alive = false; break; }
         tc_fence_after();
         const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * PH);
 #pragma unroll

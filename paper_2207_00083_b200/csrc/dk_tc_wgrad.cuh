@@ -44,6 +44,8 @@ struct WgTcParams {
   int nitems;                  // MT*NB*taps*nsplit
   int kw, pad, stride;
   int nstages, chunk;
+  unsigned spin_cap;           // polls after which a wait gives up
+  int withhold;                // test hook: the producer arms its n-th stage but issues no copy (-1 = off)
   int cout, cin;
   float scale;
   float* dW;                   // [cout][taps][cin]
@@ -143,7 +145,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
       // ---------------- TMA producer ----------------
       // whole warp: lane 0 arms the stage, then each lane issues its share of
       // the 2*(BM+BN)/32 box copies so that they go out side by side
-      int stage = 0;
+      int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool alive = true;
       constexpr int NBOX = 2 * (BM / 32) + 2 * (BNL / 32);
@@ -173,12 +175,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
           for (int j = 0; j < p.K1; ++j) {
             int ok = 1;
             if (lane == 0) {
-              ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag) ? 1 : 0;
+              ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
               // the bytes of both CTAs of a pair are counted on the leader's barrier
               if (ok && rank == 0) mbar_expect_tx(full_bar + stage, (uint32_t)((PAIR ? 2 : 1) * STAGE_BYTES));
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) { alive = false; break; }
+            if (issued++ == p.withhold) { alive = false; break; }      // test hook: armed, nothing copied
             unsigned char* st = smem + (size_t)stage * STAGE_BYTES;
             const uint32_t pbar = PAIR ? mapa_shared(smem_u32(full_bar + stage), 0u) : 0u;
             auto load = [&](void* dst, const CUtensorMap* map, int c0, int c1, int c2) {
@@ -225,12 +228,12 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
         const int nchunks = (KB + p.chunk - 1) / p.chunk;
         for (int ci = 0; alive && ci < nchunks; ++ci, ++acc_it) {
           const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
-          if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag)) { alive = false; break; }
+          if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag, p.spin_cap)) { alive = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * 256u;
           const int kb_end = min(KB, (ci + 1) * p.chunk);
           for (int kb = ci * p.chunk; kb < kb_end; ++kb) {
-            if (!mbar_wait(full_bar + stage, phase, abort_flag)) { alive = false; break; }
+            if (!mbar_wait(full_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
             tc_fence_after();
             const uint32_t st = smem_u32(smem + (size_t)stage * STAGE_BYTES);
             const uint64_t a_hi = make_desc_mn(st, kWgBox), a_lo = make_desc_mn(st + A_BYTES, kWgBox);
@@ -266,7 +269,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
       const int nchunks = (KB + p.chunk - 1) / p.chunk;
       for (int ci = 0; ci < nchunks; ++ci, ++acc_it) {
         const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
-        if (!mbar_wait(tfull_bar + buf, aphase, abort_flag)) { alive = false; break; }
+        if (!mbar_wait(tfull_bar + buf, aphase, abort_flag, p.spin_cap)) { alive = false; break; }
         tc_fence_after();
         const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * NH);
         constexpr int TS = NH > 96 ? 16 : 32;      // columns per round trip (fewer when the sums fill the registers)

@@ -2,10 +2,6 @@
 exact CPU oracle on the same seeded inputs.  Everything here is integer work:
 residues, decoded integers, verdicts and the dequantised outputs (exact
 multiples of 2^-l) must match bit for bit."""
-import os
-import subprocess
-import sys
-
 import numpy as np
 import pytest
 import torch
@@ -315,20 +311,38 @@ def test_full_size_layer_sampled_against_the_oracle(ctx, layer):
         assert dWq[co, ci, u, vv] == F.field_wgrad_plain_at(dq, xq, co, ci, u, vv, P, spec.stride, spec.pad)
 
 
-@pytest.mark.parametrize("switch", ["DK_FIELD_SIMT", "DK_FIELD_MMA_SYNC"])
-def test_cross_check_kernels_give_the_same_residues(switch):
-    """DK_FIELD_SIMT=1 selects the 64-bit integer-ALU contraction kernels, DK_FIELD_MMA_SYNC=1 keeps the forward
-    contraction on the mma.sync kernel instead of the tcgen05 one (both switches are read once per process):
-    a few parity cases re-run in a child process under each."""
-    if os.environ.get(switch) == "1":
-        pytest.skip("already running under the switch")
-    env = dict(os.environ, **{switch: "1"})
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", os.path.abspath(__file__), "-k",
-                        "conv_tiny_K2 or fc_K8_long or conv_3x3s2_K5 or conv_ragged_K3_nchw or other_primes "
-                        "or vgg_cifar_conv3_1"],
-                       cwd=root, env=env, capture_output=True, text=True, timeout=900)
-    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+CROSS_CHECK = [c for c in CASES if c[0] in ("conv_tiny_K2", "fc_K8_long", "conv_3x3s2_K5", "conv_ragged_K3_nchw",
+                                            "vgg_cifar_conv3_1_G2", "fc_long_tc")]
+
+
+@pytest.mark.parametrize("path", [1, 2], ids=["integer_alu", "mma_sync"])
+@pytest.mark.parametrize("name,spec,layout", CROSS_CHECK, ids=[c[0] for c in CROSS_CHECK])
+def test_cross_check_kernels_give_the_same_residues(name, spec, layout, path):
+    """Option DK_OPT_FIELD_PATH = 1 selects the 64-bit integer-ALU contraction kernels, 2 keeps the forward
+    contraction on the mma.sync kernel instead of the tcgen05 one: the encoded outputs and the weight
+    gradient are the same residues as the oracle's under each."""
+    c = dk.Context(0)
+    try:
+        dk.dk_set_option(c, dk.DK_OPT_FIELD_PATH, path)
+        d = synth.draw_field_layer(spec, P)
+        p = dk.problem_from_spec(spec, layout=layout)
+        c.ensure_workspace(p, field=True)
+        E = spec.K + 2
+        Wq, xq = F.quantize(d["W"], L, P), F.quantize(d["x"], L, P)
+        xbar = F.field_encode(xq, d["rq"], d["Cq"], P)
+        want_ybar = F.field_linear(Wq, xbar, P, spec.stride, spec.pad)
+        ybar_dev = empty_res(res_acts_to_dev(want_ybar, layout))
+        dk.dk_field_linear_fwd(c, p, P, res_weights_to_dev(Wq, layout), res_acts_to_dev(xbar, layout), ybar_dev)
+        assert np.array_equal(res_acts_from_dev(ybar_dev, layout), want_ybar)
+        dq = F.quantize(d["delta"], L, P)
+        dWq = empty_res(res_weights_to_dev(Wq, layout))
+        dk.dk_field_linear_bwd_wgrad(c, p, P, res_acts_to_dev(dq, layout), res_acts_to_dev(xbar, layout), E,
+                                     u32(d["Cq"]), u32(d["gammaq"]), dWq)
+        assert dk.dk_device_status(c) == 0
+        assert np.array_equal(res_weights_from_dev(dWq, layout),
+                              F.field_wgrad_plain(dq, xq, P, spec.kh, spec.kw, spec.stride, spec.pad))
+    finally:
+        c.close()
 
 
 # ---------------------------------------------------------------------------
