@@ -53,6 +53,9 @@ METRIC = "decoded masked-linear TFLOP/s & fraction of roofline; encode/decode GB
 L2_FLUSH_BYTES = 512 << 20
 TF32_OVER_BF16 = 1.1 / 2.25      # nominal dense TF32 : BF16 tensor throughput
 FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # SMs x FMA lanes x 2 x max SM clock
+# fp64 rate of this part: 148 SMs x 64 fp64 FMA lanes x 2 x 1.965 GHz = 37.2 TFLOP/s; a register-resident loop of
+# mma.sync.m8n8k4.f64 measured 37.0 and one of plain fp64 FMAs 36.6 on this machine
+FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
 # DRAM bytes (read + write) per launch of the GEMM kernel classes, average over the layers' launches, from
 # ncu captures of these kernels (summaries with their commands under profiles/); a workload or class that is
 # absent here has not been captured since the kernels last changed and reports null.
@@ -490,7 +493,9 @@ def layer_roofs(s, call, peaks, tf32_peak):
     flops = s.fwd_flops() if call == "fwd" else s.wgrad_flops()
     tensor = uses_tensor_cores(s) if call == "fwd" else wgrad_on_tensor_cores(s)
     issued = 3.0 * flops if tensor else flops
-    t_compute = issued / ((tf32_peak if tensor else FP32_ALU_PEAK_TFLOPS) * 1e12) * 1e3
+    fp64 = getattr(s, "precision", "default") == "fp64" and call == "fwd"     # the fp64 regime: fp64 units bind
+    alu_peak = FP64_PEAK_TFLOPS if fp64 else FP32_ALU_PEAK_TFLOPS
+    t_compute = issued / ((tf32_peak if tensor else alu_peak) * 1e12) * 1e3
     t_hbm = algorithmic_bytes(s, call) / (peaks["hbm_gbs"] * 1e9) * 1e3
     bound = ("tensor" if tensor else "alu") if t_compute >= t_hbm else "hbm"
     return {"bound": bound, "floor_ms": max(t_compute, t_hbm), "tensor_floor_ms": t_compute,

@@ -529,6 +529,23 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     }
     return s;      // the kernel's last CTA has written the verdict
   }
+  if (g.precision == DK_FP64_SIMT && fused64_supported(g)) {
+    // pointwise layers: one kernel encodes, contracts and decodes in fp64; nothing but x, r, W and y
+    // (and the fp32 encodings, when stored) touches memory
+    VerifyScratch vs = verify_scratch(ctx, g);
+    {
+      ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+      s = launch_verify_begin(g, vs, st);
+    }
+    if (s != DK_OK) return s;
+    {
+      ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
+      s = launch_fused64(g, W, x, r, cv, bias, y, xbar_save, vs, fault, ctx->sm_count, st);
+    }
+    if (s != DK_OK) return s;
+    ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+    return launch_verify_finalize(g, cv.nul, vs, verdict, st);
+  }
   if (g.precision == DK_FP64_SIMT) {
     // beyond-fp32 path: encodings and y_bar stay in the workspace as doubles
     // (the two adjacent hi/lo regions hold the fp64 encodings)

@@ -128,6 +128,13 @@ dk_status launch_add_fault64(double* ybar, long long index, float delta, cudaStr
 dk_status launch_simt_fwd64(const Geom& g, const float* W, const double* xbar, double* ybar,
                             int nsamples, cudaStream_t st);
 
+// DK_FP64_SIMT for pointwise convolutions in one kernel (dk_fp64_fused.cu): Eq. 1 in the prologue, the
+// contraction on the fp64 tensor path, Eq. 2 and the integrity statistics in the epilogue
+bool fused64_supported(const Geom& g);
+dk_status launch_fused64(const Geom& g, const float* W, const float* x, const float* r, const CoefView& cv,
+                         const float* bias, float* y, float* xsave, const VerifyScratch& vs, const dk_fault* fault,
+                         int sm_count, cudaStream_t st);
+
 // SIMT dense kernels (dk_simt.cu)
 dk_status launch_simt_fwd(const Geom& g, const float* W, const float* xbar, float* ybar,
                           int nsamples, cudaStream_t st);

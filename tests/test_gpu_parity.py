@@ -61,6 +61,18 @@ def small_cases():
         ("wg_pack_cin48", tiny(cin=48, cout=64, h=10, w=10, K=4, G=2)),
         ("wg_pack_cin96", tiny(cin=96, cout=136, h=9, w=9, K=4, G=2)),
         ("wg_pack_2x2", tiny(cin=16, cout=32, h=8, w=8, kh=2, kw=2, pad=0, K=2, G=2)),
+        # the fused fp64 kernel of pointwise layers: ragged pixel tiles, ragged channel blocks, a ragged last
+        # chunk of the contraction (cin 24), every warp layout (cout 8 .. 300), K = 1 .. 8
+        ("f64_K8_ragged", tiny(cin=24, cout=40, h=7, w=7, kh=1, kw=1, pad=0, K=8, G=2, sigma_r=1000.0,
+                               x_dist="normal", precision="fp64")),
+        ("f64_K4_cout144", tiny(cin=32, cout=144, h=5, w=6, kh=1, kw=1, pad=0, K=4, G=3, sigma_r=1000.0,
+                                x_dist="normal", precision="fp64")),
+        ("f64_K1_cout8", tiny(cin=4, cout=8, h=9, w=9, kh=1, kw=1, pad=0, K=1, G=2, sigma_r=1000.0,
+                              x_dist="normal", precision="fp64")),
+        ("f64_K6_cout300", tiny(cin=72, cout=300, h=3, w=3, kh=1, kw=1, pad=0, K=6, G=2, sigma_r=1000.0,
+                                x_dist="normal", precision="fp64")),
+        ("f64_K2_cout20", tiny(cin=16, cout=20, h=11, w=13, kh=1, kw=1, pad=0, K=2, G=1, sigma_r=1000.0,
+                               x_dist="normal", precision="fp64")),
     ]
 
 
@@ -181,6 +193,8 @@ def test_decode_verify_matches_oracle(ctx, drawn, spec):
 @pytest.mark.parametrize("prec", [None, dk.DK_FP32_SIMT], ids=["default", "simt"])
 @pytest.mark.parametrize("spec", SPECS, ids=IDS)
 def test_masked_linear_matches_oracle(ctx, drawn, spec, prec):
+    if prec == dk.DK_FP32_SIMT and spec.name == "t" and spec.precision == "fp64" and spec.kind == "conv":
+        pytest.skip("fp32 arithmetic cannot hold 1e-3 at noise 1000x the inputs (the error table records it)")
     d = drawn(spec)
     K, E = spec.K, spec.K + 2
     p = dk.problem_from_spec(spec, precision=prec, tol=H.TAU)
