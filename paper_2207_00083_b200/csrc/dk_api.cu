@@ -303,7 +303,7 @@ dk_status dk_create(dk_ctx** out, int device) {
     return DK_ERR_CUDA;
   }
   c->sm_count = sms;
-  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1};
+  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1};
   for (int i = 0; i < DK_OPT_COUNT; ++i) c->opt.v[i] = kOptDefault[i];
   bool ok = cudaMallocHost(&c->h_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
@@ -341,8 +341,8 @@ dk_status dk_destroy(dk_ctx* c) {
 
 dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx || option < 0 || option >= DK_OPT_COUNT) return DK_ERR_INVALID_ARG;
-  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1};
-  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 1, 2, 1 << 26, 1 << 20};
+  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0};
+  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 1, 2, 1 << 26, 1 << 20, 1};
   int v = value < lo[option] ? lo[option] : (value > hi[option] ? hi[option] : value);
   if (option == DK_OPT_TC_BK) v = v == 16 ? 16 : 32;
   ctx->opt.v[option] = v;
@@ -409,8 +409,11 @@ dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W, const 
     float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
     {
       ProfScope ps(ctx, DK_KERNEL_OTHER, 2, st);
+      const int raw = ctx->opt.v[DK_OPT_XBAR_HI];
       s = tc_split(W, w_hi, w_lo, (long long)g.cout * g.kc, ctx->sm_count, st);
-      if (s == DK_OK) s = tc_split(xbar, xb_hi, xb_lo, (long long)g.G * g.E * g.n_in, ctx->sm_count, st);
+      if (s == DK_OK)
+        s = tc_split(xbar, raw ? nullptr : xb_hi, xb_lo, (long long)g.G * g.E * g.n_in, ctx->sm_count, st, raw);
+      if (raw) xb_hi = const_cast<float*>(xbar);      // the kernel reads the caller's encodings as leading term
     }
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
@@ -491,12 +494,18 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     const int ksplit = tc_fwd_ksplit(ctx, gg);
     float* ybar = reinterpret_cast<float*>(ws + wp.ybar);
     const bool prepass_clears = ksplit > 1 && !stem;     // the pre-pass also clears y_bar for the slices
+    // leading TF32 term of the encodings: the fp32 encodings themselves (stored by the caller, or in the
+    // workspace), or a rounded copy
+    const int raw = stem ? 0 : ctx->opt.v[DK_OPT_XBAR_HI];
+    float* full = xbar_save;
+    if (raw && !full) full = reinterpret_cast<float*>(ws + wp.xbar);
     {
       // one launch: encodings and weights as hi/lo pairs, integrity statistics cleared
       ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
       s = stem ? tc_stem_fwd_prepass(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, W, w_hi, w_lo, vs, ctx->sm_count, st)
-               : tc_fwd_prepass(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, W, w_hi, w_lo, vs,
-                                prepass_clears ? ybar : nullptr, ctx->sm_count, st);
+               : tc_fwd_prepass(g, x, r, cv.enc, full, raw ? nullptr : xb_hi, xb_lo, W, w_hi, w_lo, vs,
+                                prepass_clears ? ybar : nullptr, ctx->sm_count, st, raw);
+      if (raw) xb_hi = full;
     }
     if (s != DK_OK) return s;
     if (ksplit > 1) {
@@ -631,8 +640,10 @@ static dk_status wgrad_impl(dk_ctx* ctx, const Geom& g, const WsPlan& wp, const 
     {
       // one launch: mixed deltas and stored encodings as hi/lo pairs, dW cleared
       ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
-      s = tc_wgrad_prepass(g, delta, cv.dmix, dtil, dt_lo, xbar, xbar_elems, xb_hi, xb_lo,
-                           accumulate ? nullptr : dW, ctx->sm_count, st);
+      const int raw = ctx->opt.v[DK_OPT_XBAR_HI];
+      s = tc_wgrad_prepass(g, delta, cv.dmix, dtil, dt_lo, xbar, xbar_elems, raw ? nullptr : xb_hi, xb_lo,
+                           accumulate ? nullptr : dW, ctx->sm_count, st, raw, xbar_rows);
+      if (raw) xb_hi = const_cast<float*>(xbar);      // the stored encodings are the leading term
     }
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);

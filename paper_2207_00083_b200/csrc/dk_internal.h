@@ -165,7 +165,8 @@ void tc_destroy(dk_ctx* ctx);
 // stride 1, cin % 4 == 0, not DK_FP32_SIMT)
 bool tc_fwd_supported(const dk_ctx* ctx, const Geom& g);
 // hi = tf32(src), lo = tf32(src - hi); n % 4 == 0
-dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_count, cudaStream_t st);
+// (hi = nullptr, raw = 1: only lo = tf32(src - trunc(src)) is written, the reader takes src itself as hi)
+dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_count, cudaStream_t st, int raw = 0);
 // Eq. 1 with the split fused in; `full` (nullable) also receives the fp32 encodings
 dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const float* enc, float* full,
                           float* hi, float* lo, int sm_count, cudaStream_t st);
@@ -191,12 +192,15 @@ dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* 
 // y_bar buffer of a split-K call cleared.
 dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const float* enc, float* full,
                          float* xb_hi, float* xb_lo, const float* W, float* w_hi, float* w_lo,
-                         const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st);
+                         const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st, int raw = 0);
+// (raw != 0: xb_hi is not written; the reader takes the fp32 encodings in `full` as leading term and
+// xb_lo holds tf32(v - trunc(v)))
 // One launch for what a weight-gradient call prepares: Eq. 4 delta mixing and
 // the stored encodings as hi/lo pairs, dW cleared (dW = nullptr: left as it is).
 dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix, float* dt_hi, float* dt_lo,
                            const float* xbar, long long xbar_elems, float* xb_hi, float* xb_lo, float* dW,
-                           int sm_count, cudaStream_t st);
+                           int sm_count, cudaStream_t st, int raw = 0, int xbar_rows = 0);
+// (raw != 0: only xb_lo is written, and only for the K+1 encodings of each group that Eq. 4 uses)
 // same contraction with decode + integrity statistics in the epilogue; when
 // `verdict` is given the kernel's last CTA also writes it (no finalize launch)
 dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,

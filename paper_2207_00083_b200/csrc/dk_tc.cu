@@ -91,9 +91,20 @@ int fwd_bk(const TcState* ts) { return ts->opt->v[DK_OPT_TC_BK] == 16 ? 16 : 32;
 // HBM-bound pre-passes: TF32 hi/lo split, alone or fused with the encoder
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-split_tf32_kernel(const float4* __restrict__ src, float4* __restrict__ hi, float4* __restrict__ lo, long long n4) {
+split_tf32_kernel(const float4* __restrict__ src, float4* __restrict__ hi, float4* __restrict__ lo, long long n4,
+                  int raw) {
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (long long)gridDim.x * blockDim.x) {
     float4 v = __ldg(src + i), h, l;
+    if (raw) {
+      // only the second term; the reader takes src itself as the first (the tensor core ignores the 13 low
+      // mantissa bits of a TF32 operand, i.e. it sees trunc(src))
+      l.x = to_tf32(v.x - __uint_as_float(__float_as_uint(v.x) & 0xffffe000u));
+      l.y = to_tf32(v.y - __uint_as_float(__float_as_uint(v.y) & 0xffffe000u));
+      l.z = to_tf32(v.z - __uint_as_float(__float_as_uint(v.z) & 0xffffe000u));
+      l.w = to_tf32(v.w - __uint_as_float(__float_as_uint(v.w) & 0xffffe000u));
+      lo[i] = l;
+      continue;
+    }
     h.x = to_tf32(v.x); l.x = to_tf32(v.x - h.x);
     h.y = to_tf32(v.y); l.y = to_tf32(v.y - h.y);
     h.z = to_tf32(v.z); l.z = to_tf32(v.z - h.z);
@@ -392,14 +403,15 @@ bool tc_fwd_supported(const dk_ctx* ctx, const Geom& g) {
   return plan_fwd(static_cast<TcState*>(ctx->tc_state), g, &tl);
 }
 
-dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_count, cudaStream_t st) {
+dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_count, cudaStream_t st, int raw) {
+  if ((raw != 0) != (hi == nullptr)) return DK_ERR_INVALID_ARG;
   if (n % 4) return DK_ERR_SHAPE;
   long long n4 = n / 4;
   long long blocks = (n4 + 255) / 256;
   if (blocks > (long long)sm_count * 16) blocks = (long long)sm_count * 16;
   if (blocks < 1) blocks = 1;
   split_tf32_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(src),
-                                                      reinterpret_cast<float4*>(hi), reinterpret_cast<float4*>(lo), n4);
+                                                      reinterpret_cast<float4*>(hi), reinterpret_cast<float4*>(lo), n4, raw);
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
 }

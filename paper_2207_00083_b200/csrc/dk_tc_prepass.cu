@@ -22,10 +22,29 @@ __device__ __forceinline__ void split4(const float4& v, float4& h, float4& l) {
   h.w = to_tf32(v.w); l.w = to_tf32(v.w - h.w);
 }
 
-// blocks [first, first + nblocks) split src into hi = tf32(src), lo = tf32(src - hi)
+// The second TF32 term when the reader takes the fp32 value itself as the first: the tensor core ignores
+// the 13 low mantissa bits of a TF32 operand, i.e. it sees trunc(v).  (Measured: with the term
+// tf32(v - tf32(v)), which would be right if it rounded, y_bar is off by 5e-4; with this one the error
+// equals that of a separately stored rounded first term.)
+__device__ __forceinline__ float lo_of_raw(float v) {
+  return to_tf32(v - __uint_as_float(__float_as_uint(v) & 0xffffe000u));
+}
+__device__ __forceinline__ float4 lo4_of_raw(const float4& v) {
+  return make_float4(lo_of_raw(v.x), lo_of_raw(v.y), lo_of_raw(v.z), lo_of_raw(v.w));
+}
+
+// blocks [first, first + nblocks) split src into hi = tf32(src), lo = tf32(src - hi); with raw != 0 only the
+// second term (see lo_of_raw) is written, and rows (of row4 vectors) whose index modulo `period` is >= `used`
+// are skipped
 __device__ __forceinline__ void split_job(const float4* __restrict__ src, float4* __restrict__ hi,
-                                          float4* __restrict__ lo, long long n4, int block, int nblocks) {
+                                          float4* __restrict__ lo, long long n4, int block, int nblocks, int raw = 0,
+                                          long long row4 = 0, int period = 1, int used = 1) {
   for (long long i = (long long)block * blockDim.x + threadIdx.x; i < n4; i += (long long)nblocks * blockDim.x) {
+    if (raw) {
+      if (period > used && (int)((i / row4) % period) >= used) continue;
+      lo[i] = lo4_of_raw(__ldg(src + i));
+      continue;
+    }
     float4 h, l;
     split4(__ldg(src + i), h, l);
     hi[i] = h;
@@ -40,7 +59,7 @@ template <int ROWS, int COLS, bool LAST_SEPARATE>
 __device__ __forceinline__ void mix_job(const float* __restrict__ in, const float* __restrict__ last,
                                         const float* __restrict__ coef, float* __restrict__ full,
                                         float* __restrict__ hi, float* __restrict__ lo, long long n, int g,
-                                        int chunk, int nchunks) {
+                                        int chunk, int nchunks, int raw = 0) {
   float c[ROWS][COLS];
 #pragma unroll
   for (int i = 0; i < ROWS; ++i)
@@ -65,11 +84,15 @@ __device__ __forceinline__ void mix_job(const float* __restrict__ in, const floa
         o.x = fmaf(c[i][k], s[k].x, o.x); o.y = fmaf(c[i][k], s[k].y, o.y);
         o.z = fmaf(c[i][k], s[k].z, o.z); o.w = fmaf(c[i][k], s[k].w, o.w);
       }
-      split4(o, h, l);
       const size_t off = ob + (size_t)i * n;
       if (full != nullptr) reinterpret_cast<float4*>(full + off)[q] = o;
-      reinterpret_cast<float4*>(hi + off)[q] = h;
-      reinterpret_cast<float4*>(lo + off)[q] = l;
+      if (raw) {
+        reinterpret_cast<float4*>(lo + off)[q] = lo4_of_raw(o);
+      } else {
+        split4(o, h, l);
+        reinterpret_cast<float4*>(hi + off)[q] = h;
+        reinterpret_cast<float4*>(lo + off)[q] = l;
+      }
     }
   }
 }
@@ -80,6 +103,7 @@ struct FwdPrepass {
   const float* W; float* w_hi; float* w_lo; long long w4; int w_blocks;   // then w_blocks blocks: split W
   float* stats; int nstats; unsigned int* count;   // cleared by block 0
   float4* zero; long long z4; int z_blocks;        // then z_blocks blocks: clear y_bar (split-K calls)
+  int raw;                                         // the encodings in `full` serve as leading term (see lo_of_raw)
 };
 
 template <int K>
@@ -98,7 +122,7 @@ __global__ void __launch_bounds__(256) fwd_prepass_kernel(const FwdPrepass a) {
       if (threadIdx.x == 0) { a.count[0] = 0u; a.count[1] = 0u; }
     }
     const int g = blockIdx.x / a.per_g, chunk = blockIdx.x - g * a.per_g;
-    mix_job<K + 2, K + 1, true>(a.x, a.r, a.enc, a.full, a.xb_hi, a.xb_lo, a.n_in, g, chunk, a.per_g);
+    mix_job<K + 2, K + 1, true>(a.x, a.r, a.enc, a.full, a.xb_hi, a.xb_lo, a.n_in, g, chunk, a.per_g, a.raw);
   } else {
     split_job(reinterpret_cast<const float4*>(a.W), reinterpret_cast<float4*>(a.w_hi),
               reinterpret_cast<float4*>(a.w_lo), a.w4, (int)blockIdx.x - enc_blocks, a.w_blocks);
@@ -110,6 +134,7 @@ struct WgPrepass {
   long long n_out; int G, per_g;                   // blocks [0, G*per_g): delta mixing
   const float* xbar; float* xb_hi; float* xb_lo; long long x4; int x_blocks;   // then: split xbar
   float4* dW; long long dw4; int z_blocks;         // then: clear dW
+  int raw; long long row4; int period, used;       // raw: only the second term of the used encodings is written
 };
 
 template <int K>
@@ -124,7 +149,7 @@ __global__ void __launch_bounds__(256) wgrad_prepass_kernel(const WgPrepass a) {
   b -= mix_blocks;
   if (b < a.x_blocks) {
     split_job(reinterpret_cast<const float4*>(a.xbar), reinterpret_cast<float4*>(a.xb_hi),
-              reinterpret_cast<float4*>(a.xb_lo), a.x4, b, a.x_blocks);
+              reinterpret_cast<float4*>(a.xb_lo), a.x4, b, a.x_blocks, a.raw, a.row4, a.period, a.used);
     return;
   }
   b -= a.x_blocks;
@@ -144,10 +169,12 @@ int job_blocks(long long n4, long long cap) {
 
 dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const float* enc, float* full,
                          float* xb_hi, float* xb_lo, const float* W, float* w_hi, float* w_lo,
-                         const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st) {
+                         const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st, int raw) {
   const long long wn = (long long)g.cout * g.kc;
   if (g.n_in % 4 || wn % 4) return DK_ERR_SHAPE;
+  if (raw && full == nullptr) return DK_ERR_INVALID_ARG;
   FwdPrepass a;
+  a.raw = raw;
   const long long yn = (long long)g.G * g.E * g.n_out;
   a.zero = reinterpret_cast<float4*>(ybar_clear);
   a.z4 = ybar_clear ? (yn + 3) / 4 : 0;           // the y_bar region is padded to 1 KiB
@@ -175,10 +202,11 @@ dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const fl
 
 dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix, float* dt_hi, float* dt_lo,
                            const float* xbar, long long xbar_elems, float* xb_hi, float* xb_lo, float* dW,
-                           int sm_count, cudaStream_t st) {
+                           int sm_count, cudaStream_t st, int raw, int xbar_rows) {
   const long long dwn = (long long)g.cout * g.kc;
-  if (g.n_out % 4 || xbar_elems % 4 || dwn % 4) return DK_ERR_SHAPE;
+  if (g.n_out % 4 || xbar_elems % 4 || dwn % 4 || g.n_in % 4) return DK_ERR_SHAPE;
   WgPrepass a;
+  a.raw = raw; a.row4 = g.n_in / 4; a.period = xbar_rows > 0 ? xbar_rows : 1; a.used = xbar_rows > 0 ? g.K + 1 : 1;
   a.delta = delta; a.dmix = dmix; a.dt_hi = dt_hi; a.dt_lo = dt_lo;
   a.n_out = g.n_out; a.G = g.G;
   const long long cap = (long long)sm_count * 16;
