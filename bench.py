@@ -502,8 +502,8 @@ def layer_roofs(s, call, peaks, tf32_peak):
             "hbm_floor_ms": t_hbm, "issued_flops": issued, "tensor_cores": tensor}
 
 
-def fwd_call(dk, ctx, L, fault=None):
-    dk.dk_masked_linear(ctx, L["p"], L["W"], L["x"], L["r"], L["C"], None, L["y"], L["xsave"], L["v"], fault)
+def fwd_call(dk, ctx, L, fault=None, p=None):
+    dk.dk_masked_linear(ctx, p or L["p"], L["W"], L["x"], L["r"], L["C"], None, L["y"], L["xsave"], L["v"], fault)
 
 
 def wgrad_call(dk, ctx, L):
@@ -518,9 +518,12 @@ def profile_layers(torch, dk, ctx, layers, peaks, tf32_peak, flush, iters=2):
     for L in layers:
         s = L["spec"]
         row = {"layer": s.name, "M": s.cout, "Kc": s.kc, "N_fwd": s.G * (s.K + 2) * s.hout * s.wout}
+        # the opt-in forward mode with W as one TF32 term (two products per step), where the tensor cores serve
+        p_x2 = dk.problem_from_spec(s, precision=dk.DK_TF32X2_WUNSPLIT, tol=1e-4) if uses_tensor_cores(s) else None
         for call, fn, kind in (("fwd", lambda: fwd_call(dk, ctx, L), "linear_fwd"),
+                               ("fwd_tf32x2w", lambda: fwd_call(dk, ctx, L, p=p_x2), "linear_fwd"),
                                ("wgrad", lambda: wgrad_call(dk, ctx, L), "wgrad")):
-            if call == "wgrad" and not s.wgrad:
+            if (call == "wgrad" and not s.wgrad) or (call == "fwd_tf32x2w" and p_x2 is None):
                 continue
             fn()
             dk.dk_profile_reset(ctx)
@@ -536,6 +539,11 @@ def profile_layers(torch, dk, ctx, layers, peaks, tf32_peak, flush, iters=2):
             dk.dk_profile_enable(ctx, False)
             ms = tot / iters
             kms = prof[kind][0] / max(prof[kind][1], 1)
+            if call == "fwd_tf32x2w":
+                row[call] = {"call_ms": round(ms, 4), "kernel_ms": round(kms, 4),
+                             "issued_tflops_kernel": round(2.0 * s.fwd_flops() / kms / 1e9, 2) if kms > 0 else None,
+                             "masked_tflops_call": round(s.fwd_flops() / ms / 1e9, 2)}
+                continue
             roof = layer_roofs(s, call, peaks, tf32_peak)
             flops = s.fwd_flops() if call == "fwd" else s.wgrad_flops()
             row[call] = {"bound": roof["bound"], "call_ms": round(ms, 4), "kernel_ms": round(kms, 4),

@@ -81,8 +81,14 @@ enum { DK_NHWC = 0, DK_NCHW = 1 };
  * products kept (error ~2^-22 per product); DK_FP32_SIMT uses plain fp32 FMAs
  * and accepts every geometry.  A request the tensor-core path cannot serve
  * (see dk_linear_fwd) is executed by the SIMT path. */
-enum { DK_PREC_DEFAULT = 0, DK_TF32X3 = 1, DK_FP32_SIMT = 2, DK_FP64_SIMT = 3 };
-/* DK_FP64_SIMT exists for the regime in which fp32 itself cannot hold the
+enum { DK_PREC_DEFAULT = 0, DK_TF32X3 = 1, DK_FP32_SIMT = 2, DK_FP64_SIMT = 3, DK_TF32X2_WUNSPLIT = 4 };
+/* DK_TF32X2_WUNSPLIT (forward calls only; the weight gradient and everything the
+ * tensor-core kernels do not take run as under DK_TF32X3): W enters as ONE TF32
+ * term, the encodings stay split, two products per step instead of three.
+ * Rounding W is exact under decoding, decode(<W', x_bar>) = <W', x>: the result
+ * is the layer's output for weights rounded to 11 significant bits, an error of
+ * ~1e-4 of the output's scale that does not grow with the noise.  Opt-in.
+ * DK_FP64_SIMT exists for the regime in which fp32 itself cannot hold the
  * signal next to the noise: with noise 1000x the inputs and K = 8, one fp32
  * rounding of an encoded value (2^-24 * 2000) decodes to ~1e-3 of the result.
  * In dk_masked_linear it encodes, contracts and decodes in fp64 (encodings and
@@ -100,7 +106,7 @@ typedef struct {
   int32_t kh, kw;     /* filter size (FC: 1, 1)                                   */
   int32_t stride, pad;/* same in both directions (FC: 1, 0)                       */
   int32_t K, G;       /* virtual batch size (1..DK_MAX_K), number of groups       */
-  int32_t precision;  /* DK_PREC_DEFAULT | DK_TF32X3 | DK_FP32_SIMT | DK_FP64_SIMT */
+  int32_t precision;  /* DK_PREC_DEFAULT | DK_TF32X3 | DK_FP32_SIMT | DK_FP64_SIMT | DK_TF32X2_WUNSPLIT */
   float tol;          /* integrity threshold tau; <= 0 selects 1e-4               */
 } dk_problem;
 

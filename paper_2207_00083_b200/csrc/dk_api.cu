@@ -15,7 +15,7 @@ dk_status make_geom(const dk_problem* p, Geom* g) {
   if (!p || !g) return DK_ERR_INVALID_ARG;
   if (p->kind != DK_FC && p->kind != DK_CONV2D) return DK_ERR_INVALID_ARG;
   if (p->layout != DK_NHWC && p->layout != DK_NCHW) return DK_ERR_INVALID_ARG;
-  if (p->precision < DK_PREC_DEFAULT || p->precision > DK_FP64_SIMT) return DK_ERR_INVALID_ARG;
+  if (p->precision < DK_PREC_DEFAULT || p->precision > DK_TF32X2_WUNSPLIT) return DK_ERR_INVALID_ARG;
   if (p->K < 1 || p->K > DK_MAX_K || p->G < 1) return DK_ERR_SHAPE;
   if (p->cin < 1 || p->cout < 1) return DK_ERR_SHAPE;
   memset(g, 0, sizeof(*g));
@@ -26,7 +26,8 @@ dk_status make_geom(const dk_problem* p, Geom* g) {
   g->K = p->K;
   g->G = p->G;
   g->E = p->K + 2;
-  g->precision = p->precision == DK_PREC_DEFAULT ? DK_TF32X3 : p->precision;
+  g->precision = (p->precision == DK_PREC_DEFAULT || p->precision == DK_TF32X2_WUNSPLIT) ? DK_TF32X3 : p->precision;
+  g->nprod = p->precision == DK_TF32X2_WUNSPLIT ? 2 : 3;
   g->tol = p->tol > 0.f ? p->tol : 1e-4f;
   if (p->kind == DK_FC) {
     g->h = g->w = g->kh = g->kw = g->stride = 1;

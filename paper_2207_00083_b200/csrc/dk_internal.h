@@ -17,6 +17,7 @@ struct Geom {
   long long n_in, n_out;    // elements per input / output sample
   int kc;                   // contraction length cin*kh*kw
   int precision;
+  int nprod;                // TF32 products per step of the forward tensor-core kernels: 3, or 2 (W as one term)
   float tol;
   // element strides of one sample: activation (channel, row, col), weights
   // (cout, cin, u, v), output (channel, row, col)

@@ -318,6 +318,7 @@ void fill_params(const TcState* ts, const Geom& g, const Tiling& tl, TcParams* p
   p->chunk = ts->opt->v[DK_OPT_TC_CHUNK] * (32 / fwd_bk(ts));
   p->spin_cap = (unsigned)ts->opt->v[DK_OPT_SPIN_LIMIT];
   p->withhold = ts->opt->v[DK_OPT_TEST_WITHHOLD];
+  p->nprod = g.nprod == 2 ? 2 : 3;
   ts->opt->v[DK_OPT_TEST_WITHHOLD] = -1;      // the hook serves one launch
   p->ksplit = 1;
   p->kb_per_split = tl.KB;

@@ -63,6 +63,7 @@ struct TcParams {
   int nstages;
   unsigned spin_cap;           // polls after which a wait gives up
   int withhold;                // test hook: the producer arms its n-th stage but issues no copy (-1 = off)
+  int nprod;                   // 3: W_hi.x_hi + W_hi.x_lo + W_lo.x_hi; 2: W as one TF32 term, W_lo neither loaded nor used
   // problem
   int cout, ho, wo, G;
   long long n_out;
@@ -550,7 +551,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
           int ok = 1;
           if (lane == 0) {
             ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
-            if (ok) mbar_expect_tx(full_bar + stage, (uint32_t)STAGE_BYTES);
+            if (ok) mbar_expect_tx(full_bar + stage, (uint32_t)(STAGE_BYTES - (p.nprod == 2 ? A_BYTES : 0)));
           }
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) { alive = false; break; }
@@ -562,7 +563,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
           if (lane == 0) {
             tma_load_3d(st, &map_a_hi, full_bar + stage, c0, tap, m0);
           } else if (lane == 1) {
-            tma_load_3d(st + A_BYTES, &map_a_lo, full_bar + stage, c0, tap, m0);
+            if (p.nprod == 3) tma_load_3d(st + A_BYTES, &map_a_lo, full_bar + stage, c0, tap, m0);
           } else if (lane < 2 + 2 * E) {
             const int e = (lane - 2) >> 1;
             if ((lane & 1) == 0)
@@ -608,7 +609,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
               const uint64_t adv = (uint64_t)(kk * 2);     // 32 bytes per k-step, in 16-byte units
               tc_mma_tf32(d_tmem, a_hi + adv, b_hi + adv, idesc, (first && kk == 0) ? 0u : 1u);
               tc_mma_tf32(d_tmem, a_hi + adv, b_lo + adv, idesc, 1u);
-              tc_mma_tf32(d_tmem, a_lo + adv, b_hi + adv, idesc, 1u);
+              if (p.nprod == 3) tc_mma_tf32(d_tmem, a_lo + adv, b_hi + adv, idesc, 1u);
             }
             tc_commit(empty_bar + stage);
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }

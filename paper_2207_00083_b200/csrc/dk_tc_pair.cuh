@@ -154,7 +154,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         int ok = 1;
         if (lane == 0) {
           ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
-          if (ok && rank == 0) mbar_expect_tx(full_bar + stage, (uint32_t)(2 * STAGE_BYTES));
+          if (ok && rank == 0) mbar_expect_tx(full_bar + stage, (uint32_t)(2 * (STAGE_BYTES - (p.nprod == 2 ? A_BYTES : 0))));
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) { alive = false; break; }
@@ -166,7 +166,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         if (lane == 0) {
           tma_pair_load_3d(st, &map_a_hi, bar, c0, tap, m0);
         } else if (lane == 1) {
-          tma_pair_load_3d(st + A_BYTES, &map_a_lo, bar, c0, tap, m0);
+          if (p.nprod == 3) tma_pair_load_3d(st + A_BYTES, &map_a_lo, bar, c0, tap, m0);
         } else if (lane < 2 + 2 * EH) {
           const int i = (lane - 2) >> 1;
           const int e = (int)rank * EH + i;
@@ -211,7 +211,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
               const uint64_t adv = (uint64_t)(kk * 2);     // 32 bytes per k-step, in 16-byte units
               tc_pair_mma_tf32(d_tmem, a_hi + adv, b_hi + adv, idesc, (first && kk == 0) ? 0u : 1u);
               tc_pair_mma_tf32(d_tmem, a_hi + adv, b_lo + adv, idesc, 1u);
-              tc_pair_mma_tf32(d_tmem, a_lo + adv, b_hi + adv, idesc, 1u);
+              if (p.nprod == 3) tc_pair_mma_tf32(d_tmem, a_lo + adv, b_hi + adv, idesc, 1u);
             }
             tc_pair_commit(empty_bar + stage);
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }

@@ -122,3 +122,32 @@ def test_full_size_layer_matches_oracle_on_samples(ctx, spec):
         assert sampled_dw_error(spec, d, dW, scale) < TOL_DECODED
     del W, x, r, y, xsave
     torch.cuda.empty_cache()
+
+
+X2_SPECS = [synth.layer("vgg16_cifar", "conv1_2"), synth.layer("vgg16_cifar", "conv4_2"), synth.layer("resnet18_224", "layer2_3x3s2"),
+            synth.layer("resnet18_224", "layer4_3x3"), synth.layer("vgg16_224", "conv3_2"), synth.layer("vgg16_224", "conv5_1"),
+            synth.layer("vgg16_224", "fc6"), synth.layer("vgg16_224", "fc8")]
+
+
+@pytest.mark.parametrize("spec", X2_SPECS, ids=[f"{s.workload}:{s.name}" for s in X2_SPECS])
+def test_full_size_forward_with_unsplit_weights(ctx, spec):
+    """DK_TF32X2_WUNSPLIT (W as one TF32 term, two products per step) at full size: sampled decoded outputs
+    within 5e-4 of the oracle (the bar the mode is offered under), clean verdict, fault flagged."""
+    d = synth.draw_layer(spec, with_delta=False)
+    E = spec.K + 2
+    p = dk.problem_from_spec(spec, precision=dk.DK_TF32X2_WUNSPLIT, tol=H.TAU)
+    ctx.ensure_workspace(p)
+    W, x, r = to_dev(d["W"]), to_dev(d["x"]), to_dev(d["r"])
+    y = H.empty_acts(spec.batch, spec, "out", dk.DK_NHWC)
+    v = dk.new_verdict()
+    dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y, None, v)
+    vd = dk.read_verdict(v)
+    assert (vd["ok"], vd["n_flagged"], vd["first_index"], vd["status"]) == (1, 0, -1, 0)
+    assert vd["max_ratio"] < H.TAU / 4
+    assert sampled_y_error(spec, d, y) < 5e-4
+    f = dk.dk_fault(1, 2, spec.n_out // 3, 500.0)
+    dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y, None, v, f)
+    vd = dk.read_verdict(v)
+    assert (vd["ok"], vd["n_flagged"], vd["first_index"]) == (0, 1, 1 * spec.n_out + f.out_index)
+    del W, x, r, y
+    torch.cuda.empty_cache()
