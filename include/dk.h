@@ -152,8 +152,11 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  *   DK_OPT_WG_PACK    1 (default): the weight-gradient kernel puts several filter
  *                     taps side by side for layers with few input channels.
  *   DK_OPT_WG_PAIR    1 (default): CTA pairs in the weight-gradient kernel.
- *   DK_OPT_TC_STEM    1 (default): 3-channel stems run on the tensor-core kernels
- *                     through patch rows; 0: on the fp32 kernels.
+ *   DK_OPT_TC_STEM    forward pass of layers with 1-3 input channels (the stems):
+ *                     1 (default) one fused fp32 kernel (encode, contraction, decode
+ *                     and check in registers and shared memory) when the contraction
+ *                     has at most 64 elements, else the tensor-core kernels through
+ *                     patch rows; 2 always the latter; 0 the generic fp32 kernels.
  *   DK_OPT_FIELD_PATH contraction kernels of the finite-field calls: 0 (default)
  *                     tensor cores (tcgen05 where the shape allows, else mma.sync),
  *                     1 the 64-bit integer-ALU kernels, 2 mma.sync only.

@@ -15,7 +15,7 @@ INCLUDE = os.path.join(ROOT, "include")
 OBJ_DIR = os.path.join(ROOT, "_build")
 LIB_PATH = os.path.join(PKG, "libdk.so")
 
-SOURCES = ["dk_api.cu", "dk_elementwise.cu", "dk_simt.cu", "dk_tc.cu", "dk_tc_prepass.cu", "dk_static.cu", "dk_fp64.cu", "dk_fp64_fused.cu", "dk_wgverify.cu", "dk_field.cu", "dk_chain.cu"]
+SOURCES = ["dk_api.cu", "dk_elementwise.cu", "dk_simt.cu", "dk_tc.cu", "dk_tc_prepass.cu", "dk_static.cu", "dk_fp64.cu", "dk_fp64_fused.cu", "dk_wgverify.cu", "dk_field.cu", "dk_chain.cu", "dk_stem.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

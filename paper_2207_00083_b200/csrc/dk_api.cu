@@ -343,7 +343,7 @@ dk_status dk_destroy(dk_ctx* c) {
 dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx || option < 0 || option >= DK_OPT_COUNT) return DK_ERR_INVALID_ARG;
   static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0};
-  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 1, 2, 1 << 26, 1 << 20, 1};
+  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 2, 1 << 26, 1 << 20, 1};
   int v = value < lo[option] ? lo[option] : (value > hi[option] ? hi[option] : value);
   if (option == DK_OPT_TC_BK) v = v == 16 ? 16 : 32;
   ctx->opt.v[option] = v;
@@ -479,6 +479,27 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
   s = upload_coefficients(ctx, g, C_host, nullptr, true, false, st, &cv);
   if (s != DK_OK) return s;
   char* ws = static_cast<char*>(ctx->ws);
+  if (g.precision == DK_TF32X3 && ctx->opt.v[DK_OPT_TC_STEM] == 1 && stem_fused_supported(g, tc_smem_optin(ctx))) {
+    // 1-3 input channels: one fp32 kernel encodes the input patch, contracts, decodes and checks; the
+    // encodings, when the caller stores them, come from the streaming encoder (they are tiny here)
+    VerifyScratch vs = verify_scratch(ctx, g);
+    {
+      ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+      s = launch_verify_begin(g, vs, st);
+    }
+    if (s == DK_OK && xbar_save) {
+      ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
+      s = launch_encode(g, x, r, cv.enc, xbar_save, ctx->sm_count, st);
+    }
+    if (s != DK_OK) return s;
+    {
+      ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
+      s = launch_stem_fwd(g, W, x, r, cv, bias, y, vs, fault, ctx->sm_count, st);
+    }
+    if (s != DK_OK) return s;
+    ProfScope ps(ctx, DK_KERNEL_OTHER, 1, st);
+    return launch_verify_finalize(g, cv.nul, vs, verdict, st);
+  }
   const bool stem = stem_shape(g) && tc_stem_supported(ctx, g);
   const Geom g_stem = stem ? tc_stem_gemm_geom(g) : g;
   if (stem || tc_fwd_supported(ctx, g)) {
@@ -649,6 +670,11 @@ static dk_status wgrad_impl(dk_ctx* ctx, const Geom& g, const WsPlan& wp, const 
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
     return tc_wgrad(ctx, g, dtil, dt_lo, xb_hi, xb_lo, xbar_rows, scale, dW, ctx_status_word(ctx), st);
+  }
+  if (ctx->opt.v[DK_OPT_TC_STEM] == 1 && stem_wgrad_fused_supported(g, tc_smem_optin(ctx))) {
+    // 3x3 stem on 3 channels: one fp32 kernel mixes the gradients (Eq. 4) and forms the products
+    ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
+    return launch_stem_wgrad(g, delta, xbar, xbar_rows, cv.dmix, scale, dW, !accumulate, ctx->sm_count, st);
   }
   {
     ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);

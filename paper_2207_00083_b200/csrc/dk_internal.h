@@ -136,6 +136,16 @@ dk_status launch_fused64(const Geom& g, const float* W, const float* x, const fl
                          const float* bias, float* y, float* xsave, const VerifyScratch& vs, const dk_fault* fault,
                          int sm_count, cudaStream_t st);
 
+// Layers with 1-3 input channels (the stems) in one fp32 kernel each way (dk_stem.cu)
+bool stem_fused_supported(const Geom& g, int smem_optin);
+dk_status launch_stem_fwd(const Geom& g, const float* W, const float* x, const float* r, const CoefView& cv,
+                          const float* bias, float* y, const VerifyScratch& vs, const dk_fault* fault, int sm_count,
+                          cudaStream_t st);
+bool stem_wgrad_fused_supported(const Geom& g, int smem_optin);      // 3x3 filters on 3 channels
+dk_status launch_stem_wgrad(const Geom& g, const float* delta, const float* xbar, int xbar_rows, const float* dmix,
+                            float scale, float* dW, bool clear, int sm_count, cudaStream_t st);
+int tc_smem_optin(const dk_ctx* ctx);      // opt-in shared memory per block of the context's device (dk_tc.cu)
+
 // SIMT dense kernels (dk_simt.cu)
 dk_status launch_simt_fwd(const Geom& g, const float* W, const float* xbar, float* ybar,
                           int nsamples, cudaStream_t st);

@@ -391,6 +391,10 @@ dk_status tc_init(dk_ctx* ctx) {
   return DK_OK;
 }
 
+int tc_smem_optin(const dk_ctx* ctx) {
+  return ctx->tc_state ? static_cast<TcState*>(ctx->tc_state)->smem_optin : 0;
+}
+
 void tc_destroy(dk_ctx* ctx) {
   delete static_cast<TcState*>(ctx->tc_state);
   ctx->tc_state = nullptr;
@@ -688,7 +692,7 @@ bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g) {
 }
 
 bool tc_stem_supported(const dk_ctx* ctx, const Geom& g) {
-  if (!ctx->opt.v[DK_OPT_TC_STEM] || g.kind != DK_CONV2D || g.layout != DK_NHWC || g.precision != DK_TF32X3) return false;
+  if (ctx->opt.v[DK_OPT_TC_STEM] == 0 || g.kind != DK_CONV2D || g.layout != DK_NHWC || g.precision != DK_TF32X3) return false;
   if ((g.cin % 4) == 0 || g.kc > 256 || (g.cout % 4) != 0) return false;
   const Geom s = tc_stem_gemm_geom(g);
   return tc_fwd_supported(ctx, s);
