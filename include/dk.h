@@ -226,7 +226,10 @@ DK_API dk_status dk_decode_verify(dk_ctx* ctx, const dk_problem* p, const float*
 /* Encode -> linear -> decode -> verify for one layer in one call (flow steps
  * 3-6 of Section 3.1 without leaving the device).  xbar_save (nullable)
  * receives all K+2 encodings per group, [G*(K+2)][n_in], for later use by
- * dk_linear_bwd_wgrad (Section 6, "Encoded Data Storage").  fault (host
+ * dk_linear_bwd_wgrad (Section 6, "Encoded Data Storage"); for a 1x1
+ * convolution with stride s > 1 on the tensor-core path only the rows and
+ * columns the layer reads (every s-th) are encoded and written, the rest of
+ * xbar_save is left as it is.  fault (host
  * pointer, nullable) injects one wrong accelerator output.  Needs the
  * workspace. */
 DK_API dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W,

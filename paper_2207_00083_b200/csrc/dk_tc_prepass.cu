@@ -59,7 +59,8 @@ template <int ROWS, int COLS, bool LAST_SEPARATE>
 __device__ __forceinline__ void mix_job(const float* __restrict__ in, const float* __restrict__ last,
                                         const float* __restrict__ coef, float* __restrict__ full,
                                         float* __restrict__ hi, float* __restrict__ lo, long long n, int g,
-                                        int chunk, int nchunks, int raw = 0) {
+                                        int chunk, int nchunks, int raw = 0, int pix4 = 0, int width = 0,
+                                        int step = 1) {
   float c[ROWS][COLS];
 #pragma unroll
   for (int i = 0; i < ROWS; ++i)
@@ -70,6 +71,12 @@ __device__ __forceinline__ void mix_job(const float* __restrict__ in, const floa
   const size_t ob = (size_t)g * ROWS * n;
   const long long n4 = n / 4;
   for (long long q = (long long)chunk * blockDim.x + threadIdx.x; q < n4; q += (long long)nchunks * blockDim.x) {
+    if (step > 1) {
+      // a strided 1x1 convolution reads every step-th row and column only: the others are neither encoded
+      // nor written (pix4 = 16-byte vectors per pixel, width = pixels per row)
+      const long long pix = q / pix4;
+      if ((pix % width) % step != 0 || (pix / width) % step != 0) continue;
+    }
     float4 s[COLS];
 #pragma unroll
     for (int k = 0; k < NIN; ++k) s[k] = __ldg(reinterpret_cast<const float4*>(ig + (size_t)k * n) + q);
@@ -104,6 +111,7 @@ struct FwdPrepass {
   float* stats; int nstats; unsigned int* count;   // cleared by block 0
   float4* zero; long long z4; int z_blocks;        // then z_blocks blocks: clear y_bar (split-K calls)
   int raw;                                         // the encodings in `full` serve as leading term (see lo_of_raw)
+  int pix4, width, step;                           // step > 1: only every step-th row and column is encoded
 };
 
 template <int K>
@@ -122,7 +130,8 @@ __global__ void __launch_bounds__(256) fwd_prepass_kernel(const FwdPrepass a) {
       if (threadIdx.x == 0) { a.count[0] = 0u; a.count[1] = 0u; }
     }
     const int g = blockIdx.x / a.per_g, chunk = blockIdx.x - g * a.per_g;
-    mix_job<K + 2, K + 1, true>(a.x, a.r, a.enc, a.full, a.xb_hi, a.xb_lo, a.n_in, g, chunk, a.per_g, a.raw);
+    mix_job<K + 2, K + 1, true>(a.x, a.r, a.enc, a.full, a.xb_hi, a.xb_lo, a.n_in, g, chunk, a.per_g, a.raw, a.pix4, a.width,
+                                a.step);
   } else {
     split_job(reinterpret_cast<const float4*>(a.W), reinterpret_cast<float4*>(a.w_hi),
               reinterpret_cast<float4*>(a.w_lo), a.w4, (int)blockIdx.x - enc_blocks, a.w_blocks);
@@ -175,6 +184,8 @@ dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const fl
   if (raw && full == nullptr) return DK_ERR_INVALID_ARG;
   FwdPrepass a;
   a.raw = raw;
+  const bool strided_1x1 = g.kind == DK_CONV2D && g.kh == 1 && g.kw == 1 && g.pad == 0 && g.stride > 1;
+  a.pix4 = g.cin / 4; a.width = g.w; a.step = strided_1x1 ? g.stride : 1;
   const long long yn = (long long)g.G * g.E * g.n_out;
   a.zero = reinterpret_cast<float4*>(ybar_clear);
   a.z4 = ybar_clear ? (yn + 3) / 4 : 0;           // the y_bar region is padded to 1 KiB

@@ -98,3 +98,12 @@ def flat_out_index(spec, layout: int, co: int, oh: int = 0, ow: int = 0) -> int:
 
 def logical_out_index(spec, co: int, oh: int = 0, ow: int = 0):
     return (co,) if spec.kind == "fc" else (co, oh, ow)
+
+
+def read_positions(spec, a: np.ndarray) -> np.ndarray:
+    """The part of a logical input-shaped array [n, c, h, w] that the layer reads: a strided 1x1 convolution
+    without padding touches every stride-th row and column only (the library leaves the other positions of
+    the stored encodings unwritten); everything else is returned whole."""
+    if a.ndim == 4 and spec.kind == "conv" and spec.kh == 1 and spec.kw == 1 and spec.pad == 0 and spec.stride > 1:
+        return a[:, :, ::spec.stride, ::spec.stride]
+    return a
