@@ -9,6 +9,8 @@ check, and the error of dW (dk_linear_bwd_wgrad against the plain definition).
 prints the table (the copy under profiles/ comes from this command).  The
 bars asserted here are the ones the choice of arithmetic rests on: 1e-3 on y
 and dW wherever a mode is offered for that noise level."""
+import os
+
 import numpy as np
 import pytest
 
@@ -29,7 +31,13 @@ MODES = [(dk.DK_TF32X3, "tf32x3"), (dk.DK_TF32X2_WUNSPLIT, "tf32x2w"), (dk.DK_FP
 
 @pytest.fixture(scope="module")
 def ctx():
+    """The chunk lengths of the tensor-memory accumulation change the arithmetic; DK_TEST_TC_CHUNK / DK_TEST_WG_CHUNK
+    in the environment of this test set the context's options for a sweep (profiles/error_vs_tmem_chunk_*)."""
     c = dk.Context(0)
+    if os.environ.get("DK_TEST_TC_CHUNK"):
+        dk.dk_set_option(c, dk.DK_OPT_TC_CHUNK, int(os.environ["DK_TEST_TC_CHUNK"]))
+    if os.environ.get("DK_TEST_WG_CHUNK"):
+        dk.dk_set_option(c, dk.DK_OPT_WG_CHUNK, int(os.environ["DK_TEST_WG_CHUNK"]))
     yield c
     c.close()
 
