@@ -59,7 +59,7 @@ FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
 # DRAM bytes (read + write) per launch of the GEMM kernel classes, average over the layers' launches, from
 # ncu captures of these kernels (summaries with their commands under profiles/); a workload or class that is
 # absent here has not been captured since the kernels last changed and reports null.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"vgg16_224": {"linear_fwd": 2833418752, "wgrad": 6314548352}}
 
 
 def read_peaks():
