@@ -168,6 +168,11 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  *                     of a TF32 operand) and the pre-pass writes only the second
  *                     term tf32(v - trunc(v)); 0: the pre-pass also writes a
  *                     rounded copy tf32(v) and the second term is tf32(v - tf32(v)).
+ *   DK_OPT_TC_MPACK   1 (default): a stride-1 convolution with at most 64 output
+ *                     channels fills the 128 rows of the forward kernel's tiles with
+ *                     two output rows of the image (rows 64-127 hold the filters of
+ *                     the tap one row up, so one activation box serves both); 0: one
+ *                     output row per tile, half of every product unused.
  *   DK_OPT_TEST_WITHHOLD  test hook, default -1 (off): the producer warp of the
  *                     next tensor-core forward or weight-gradient kernel arms the
  *                     barrier of its n-th pipeline stage but issues no copy for
@@ -177,7 +182,7 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
 enum {
   DK_OPT_TC_CHUNK = 0, DK_OPT_WG_CHUNK = 1, DK_OPT_TC_BK = 2, DK_OPT_TC_PAIR = 3, DK_OPT_WG_PACK = 4,
   DK_OPT_WG_PAIR = 5, DK_OPT_TC_STEM = 6, DK_OPT_FIELD_PATH = 7, DK_OPT_SPIN_LIMIT = 8,
-  DK_OPT_TEST_WITHHOLD = 9, DK_OPT_XBAR_HI = 10, DK_OPT_COUNT = 11
+  DK_OPT_TEST_WITHHOLD = 9, DK_OPT_XBAR_HI = 10, DK_OPT_TC_MPACK = 11, DK_OPT_COUNT = 12
 };
 DK_API dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value);
 DK_API dk_status dk_get_option(dk_ctx* ctx, int32_t option, int32_t* value);

@@ -225,6 +225,11 @@ static WsPlan plan_workspace(const Geom& g) {
     if (rows > xe) xe = rows;
     we = (size_t)g.cout * Kp;
   }
+  if (g.kind == DK_CONV2D && g.cout <= 64 && g.kh >= 2) {
+    // two-output-row tiles of the forward kernel: 128 rows x (kh+1)*kw taps x cin packed weights
+    const size_t packed = (size_t)128 * (g.kh + 1) * g.kw * g.cin;
+    if (packed > we) we = packed;
+  }
   const size_t xb = align_up(xe * sizeof(float), 1024);
   const size_t wb = align_up(we * sizeof(float), 1024);
   w.xbar = off; off += xb;
@@ -304,7 +309,7 @@ dk_status dk_create(dk_ctx** out, int device) {
     return DK_ERR_CUDA;
   }
   c->sm_count = sms;
-  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1};
+  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1, 1};
   for (int i = 0; i < DK_OPT_COUNT; ++i) c->opt.v[i] = kOptDefault[i];
   bool ok = cudaMallocHost(&c->h_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
@@ -342,8 +347,8 @@ dk_status dk_destroy(dk_ctx* c) {
 
 dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx || option < 0 || option >= DK_OPT_COUNT) return DK_ERR_INVALID_ARG;
-  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0};
-  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 2, 1 << 26, 1 << 20, 1};
+  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0, 0};
+  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 2, 1 << 26, 1 << 20, 1, 1};
   int v = value < lo[option] ? lo[option] : (value > hi[option] ? hi[option] : value);
   if (option == DK_OPT_TC_BK) v = v == 16 ? 16 : 32;
   ctx->opt.v[option] = v;
@@ -501,6 +506,8 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     return launch_verify_finalize(g, cv.nul, vs, verdict, st);
   }
   const bool stem = stem_shape(g) && tc_stem_supported(ctx, g);
+  // layers with at most 64 output channels: two output rows per 128-row tile (see dk_tc.cu)
+  if (!stem && ctx->opt.v[DK_OPT_TC_MPACK] && tc_mpack_eligible(g)) g.mpack = 1;
   const Geom g_stem = stem ? tc_stem_gemm_geom(g) : g;
   if (stem || tc_fwd_supported(ctx, g)) {
     // tensor-core path: encode+split pre-pass, then one GEMM whose epilogue
@@ -525,7 +532,7 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
       // one launch: encodings and weights as hi/lo pairs, integrity statistics cleared
       ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
       s = stem ? tc_stem_fwd_prepass(g, x, r, cv.enc, xbar_save, xb_hi, xb_lo, W, w_hi, w_lo, vs, ctx->sm_count, st)
-               : tc_fwd_prepass(g, x, r, cv.enc, full, raw ? nullptr : xb_hi, xb_lo, W, w_hi, w_lo, vs,
+               : tc_fwd_prepass(gg, x, r, cv.enc, full, raw ? nullptr : xb_hi, xb_lo, W, w_hi, w_lo, vs,
                                 prepass_clears ? ybar : nullptr, ctx->sm_count, st, raw);
       if (raw) xb_hi = full;
     }

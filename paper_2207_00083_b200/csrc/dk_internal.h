@@ -17,6 +17,7 @@ struct Geom {
   long long n_in, n_out;    // elements per input / output sample
   int kc;                   // contraction length cin*kh*kw
   int precision;
+  int mpack;                // forward tensor-core kernel: two output rows of the image per 128-row tile (cout <= 64)
   int nprod;                // TF32 products per step of the forward tensor-core kernels: 3, or 2 (W as one term)
   float tol;
   // element strides of one sample: activation (channel, row, col), weights
@@ -175,6 +176,8 @@ void tc_destroy(dk_ctx* ctx);
 // true when the tensor-core kernel takes this geometry (channels-last,
 // stride 1, cin % 4 == 0, not DK_FP32_SIMT)
 bool tc_fwd_supported(const dk_ctx* ctx, const Geom& g);
+// shapes whose forward tiles can hold two output rows (stride-1 convolution, cout <= 64, power-of-two pixel tile)
+bool tc_mpack_eligible(const Geom& g);
 // hi = tf32(src), lo = tf32(src - hi); n % 4 == 0
 // (hi = nullptr, raw = 1: only lo = tf32(src - trunc(src)) is written, the reader takes src itself as hi)
 dk_status tc_split(const float* src, float* hi, float* lo, long long n, int sm_count, cudaStream_t st, int raw = 0);

@@ -162,6 +162,7 @@ encode_split_kernel(const float* __restrict__ x, const float* __restrict__ r, co
 // ---------------------------------------------------------------------------
 struct Tiling {
   int P, bw, bh, bg, WT, HT, GT, MT, ntiles, KB, CB, nstages, BN;
+  bool mpack;              // two output rows of the image in one 128-row tile (cout <= 64)
   bool pair;               // tiles of 256 output channels on CTA pairs
   size_t smem_bytes;
 };
@@ -187,8 +188,10 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
       }
     }
   if (best < 0) return false;
+  t->mpack = g.mpack != 0 && !pair;
+  if (t->mpack) { t->bw = P; t->bh = 1; t->bg = 1; }      // a row segment of P pixels; the tile holds two such rows
   t->WT = (g.wo + t->bw - 1) / t->bw;
-  t->HT = (g.ho + t->bh - 1) / t->bh;
+  t->HT = t->mpack ? (g.ho + 1) / 2 : (g.ho + t->bh - 1) / t->bh;
   t->GT = (g.G + t->bg - 1) / t->bg;
   t->pair = pair;
   t->MT = pair ? (g.cout + BM2 - 1) / BM2 : (g.cout + BM - 1) / BM;
@@ -196,7 +199,7 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
   if (nt > 0x7fffffffLL) return false;
   t->ntiles = (int)nt;
   t->CB = (g.cin + BK - 1) / BK;
-  t->KB = t->CB * g.kh * g.kw;
+  t->KB = t->CB * (t->mpack ? g.kh + 1 : g.kh) * g.kw;
   t->BN = E * P;
   // a CTA of a pair stages its own 128 rows of W and half of the activation rows
   const size_t stage = 2 * ((size_t)BM * BK * 4 + (size_t)(pair ? t->BN / 2 : t->BN) * BK * 4);
@@ -234,9 +237,10 @@ template <int BK>
 bool encode_fwd_maps(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
                      const float* xb_hi, const float* xb_lo, CUtensorMap* ma_hi, CUtensorMap* ma_lo,
                      CUtensorMap* mb_hi, CUtensorMap* mb_lo) {
-  const int taps = g.kh * g.kw;
+  // (two-row tiles: the pre-pass laid the weights out as 128 rows x (kh+1)*kw taps, see tc_fwd_prepass)
+  const int taps = tl.mpack ? (g.kh + 1) * g.kw : g.kh * g.kw;
   {
-    cuuint64_t dims[3] = {(cuuint64_t)g.cin, (cuuint64_t)taps, (cuuint64_t)g.cout};
+    cuuint64_t dims[3] = {(cuuint64_t)g.cin, (cuuint64_t)taps, (cuuint64_t)(tl.mpack ? BM : g.cout)};
     cuuint64_t str[2] = {(cuuint64_t)g.cin * 4, (cuuint64_t)g.cin * taps * 4};
     cuuint32_t box[3] = {(cuuint32_t)BK, 1, (cuuint32_t)BM};
     if (!encode_map(ts, ma_hi, w_hi, 3, dims, str, box, BK * 4) ||
@@ -319,6 +323,7 @@ void fill_params(const TcState* ts, const Geom& g, const Tiling& tl, TcParams* p
   p->spin_cap = (unsigned)ts->opt->v[DK_OPT_SPIN_LIMIT];
   p->withhold = ts->opt->v[DK_OPT_TEST_WITHHOLD];
   p->nprod = g.nprod == 2 ? 2 : 3;
+  p->hmul = tl.mpack ? 2 : 1;
   ts->opt->v[DK_OPT_TEST_WITHHOLD] = -1;      // the hook serves one launch
   p->ksplit = 1;
   p->kb_per_split = tl.KB;
@@ -398,6 +403,13 @@ int tc_smem_optin(const dk_ctx* ctx) {
 void tc_destroy(dk_ctx* ctx) {
   delete static_cast<TcState*>(ctx->tc_state);
   ctx->tc_state = nullptr;
+}
+
+bool tc_mpack_eligible(const Geom& g) {
+  if (g.kind != DK_CONV2D || g.layout != DK_NHWC || g.precision != DK_TF32X3) return false;
+  if (g.cout > 64 || g.kh < 2 || g.stride != 1 || (g.cin % 4) != 0) return false;
+  const int P = tile_pixels(g.K);
+  return (P & (P - 1)) == 0;      // the row segment of P pixels must be a power of two
 }
 
 bool tc_fwd_supported(const dk_ctx* ctx, const Geom& g) {

@@ -63,6 +63,7 @@ struct TcParams {
   int nstages;
   unsigned spin_cap;           // polls after which a wait gives up
   int withhold;                // test hook: the producer arms its n-th stage but issues no copy (-1 = off)
+  int hmul;                    // 2: the tile's rows 64-127 are the image row below rows 0-63 (cout <= 64), else 1
   int nprod;                   // 3: W_hi.x_hi + W_hi.x_lo + W_lo.x_hi; 2: W as one TF32 term, W_lo neither loaded nor used
   // problem
   int cout, ho, wo, G;
@@ -545,7 +546,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
         const int wt = nt % p.WT; nt /= p.WT;
         const int ht = nt % p.HT;
         const int gt = nt / p.HT;
-        const int x0 = wt * p.bw * p.stride - p.pad, y0 = ht * p.bh * p.stride - p.pad;     // input position of tap (0,0)
+        const int x0 = wt * p.bw * p.stride - p.pad, y0 = ht * p.bh * p.hmul * p.stride - p.pad;     // input position of tap (0,0)
         const int g0 = gt * p.bg, m0 = mt * BM;
         for (int kb = kb_lo; kb < kb_hi; ++kb) {
           int ok = 1;
@@ -636,7 +637,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
       const int wt = nt % p.WT; nt /= p.WT;
       const int ht = nt % p.HT;
       const int gt = nt / p.HT;
-      const int co = mt * BM + quad * 32 + lane;
+      // (two-row tiles: lanes 64-127 hold the same output channels for the image row below)
+      const int co = p.hmul == 2 ? (quad & 1) * 32 + lane : mt * BM + quad * 32 + lane;
+      const int ht_e = p.hmul == 2 ? 2 * ht + (quad >> 1) : ht;
       const bool co_ok = co < p.cout;
 
       // ---- sum the chunks of this tile in registers (round to nearest) ----
@@ -669,7 +672,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
       }
       if (!alive) break;
 
-      tile_epilogue<MODE, K>(p, acc, half, lane, co, co_ok, gt, ht, wt);
+      tile_epilogue<MODE, K>(p, acc, half, lane, co, co_ok, gt, ht_e, wt);
     }
     tail_finalize<MODE, K>(p, (int)threadIdx.x - 128, alive, abort_flag + 1);
   }

@@ -112,7 +112,29 @@ struct FwdPrepass {
   float4* zero; long long z4; int z_blocks;        // then z_blocks blocks: clear y_bar (split-K calls)
   int raw;                                         // the encodings in `full` serve as leading term (see lo_of_raw)
   int pix4, width, step;                           // step > 1: only every step-th row and column is encoded
+  int wpack, cout, cin4, kh, kw;                   // wpack: W is laid out for two-output-row tiles (see wpack_job)
 };
+
+// Weights of a layer with at most 64 output channels for tiles that hold two output rows of the image:
+// 128 rows x (kh+1)*kw taps x cin.  Row co < 64 holds W[co][dy][v] at tap (dy, v) (zero at dy = kh); row
+// 64 + co holds W[co][dy-1][v] (zero at dy = 0): the activation box at vertical offset dy is tap dy of the upper
+// output row and tap dy-1 of the lower one.
+__device__ __forceinline__ void wpack_job(const FwdPrepass& a, int block, int nblocks) {
+  const int taps2 = (a.kh + 1) * a.kw;
+  const long long n4 = (long long)128 * taps2 * a.cin4;
+  for (long long i = (long long)block * blockDim.x + threadIdx.x; i < n4; i += (long long)nblocks * blockDim.x) {
+    const int c4 = (int)(i % a.cin4);
+    const int tap = (int)((i / a.cin4) % taps2), row = (int)(i / ((long long)a.cin4 * taps2));
+    const int dy = tap / a.kw, v = tap - dy * a.kw;
+    const int co = row & 63, u = row < 64 ? dy : dy - 1;
+    float4 w = make_float4(0.f, 0.f, 0.f, 0.f), h, l;
+    if (co < a.cout && u >= 0 && u < a.kh)
+      w = __ldg(reinterpret_cast<const float4*>(a.W) + ((long long)(co * a.kh + u) * a.kw + v) * a.cin4 + c4);
+    split4(w, h, l);
+    reinterpret_cast<float4*>(a.w_hi)[i] = h;
+    reinterpret_cast<float4*>(a.w_lo)[i] = l;
+  }
+}
 
 template <int K>
 __global__ void __launch_bounds__(256) fwd_prepass_kernel(const FwdPrepass a) {
@@ -132,6 +154,8 @@ __global__ void __launch_bounds__(256) fwd_prepass_kernel(const FwdPrepass a) {
     const int g = blockIdx.x / a.per_g, chunk = blockIdx.x - g * a.per_g;
     mix_job<K + 2, K + 1, true>(a.x, a.r, a.enc, a.full, a.xb_hi, a.xb_lo, a.n_in, g, chunk, a.per_g, a.raw, a.pix4, a.width,
                                 a.step);
+  } else if (a.wpack) {
+    wpack_job(a, (int)blockIdx.x - enc_blocks, a.w_blocks);
   } else {
     split_job(reinterpret_cast<const float4*>(a.W), reinterpret_cast<float4*>(a.w_hi),
               reinterpret_cast<float4*>(a.w_lo), a.w4, (int)blockIdx.x - enc_blocks, a.w_blocks);
@@ -195,7 +219,8 @@ dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const fl
   const long long cap = (long long)sm_count * 16;
   a.per_g = job_blocks(g.n_in / 4, (cap + g.G - 1) / g.G);
   a.W = W; a.w_hi = w_hi; a.w_lo = w_lo; a.w4 = wn / 4;
-  a.w_blocks = job_blocks(a.w4, cap);
+  a.wpack = g.mpack; a.cout = g.cout; a.cin4 = g.cin / 4; a.kh = g.kh; a.kw = g.kw;
+  a.w_blocks = job_blocks(g.mpack ? (long long)128 * (g.kh + 1) * g.kw * a.cin4 : a.w4, cap);
   a.stats = vs.sumsq; a.nstats = g.G * (g.E + 1); a.count = vs.count;
   const long long blocks = (long long)a.G * a.per_g + a.w_blocks + a.z_blocks;
   if (blocks > 0x7fffffffLL) return DK_ERR_SHAPE;

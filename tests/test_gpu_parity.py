@@ -61,6 +61,13 @@ def small_cases():
         ("wg_pack_cin48", tiny(cin=48, cout=64, h=10, w=10, K=4, G=2)),
         ("wg_pack_cin96", tiny(cin=96, cout=136, h=9, w=9, K=4, G=2)),
         ("wg_pack_2x2", tiny(cin=16, cout=32, h=8, w=8, kh=2, kw=2, pad=0, K=2, G=2)),
+        # forward tiles that hold two output rows (cout <= 64, stride 1): odd height, ragged width, few
+        # channels, K = 1 / 4 / 8 (64 / 32 / 16 pixels per row segment), 5x5 and unpadded 2x2 filters
+        ("mpack_K1_odd", tiny(cin=8, cout=40, h=7, w=9, K=1, G=2)),
+        ("mpack_K8", tiny(cin=16, cout=64, h=6, w=20, K=8, G=1)),
+        ("mpack_5x5", tiny(cin=8, cout=24, h=9, w=33, kh=5, kw=5, pad=2, K=4, G=2)),
+        ("mpack_2x2_nopad", tiny(cin=8, cout=16, h=8, w=8, kh=2, kw=2, pad=0, K=4, G=1)),
+        ("mpack_cin96", tiny(cin=96, cout=64, h=5, w=40, K=4, G=2)),
         # the fused fp64 kernel of pointwise layers: ragged pixel tiles, ragged channel blocks, a ragged last
         # chunk of the contraction (cin 24), every warp layout (cout 8 .. 300), K = 1 .. 8
         ("f64_K8_ragged", tiny(cin=24, cout=40, h=7, w=7, kh=1, kw=1, pad=0, K=8, G=2, sigma_r=1000.0,
