@@ -596,8 +596,20 @@ bool plan_wgrad(const Options& opt, const Geom& g, int smem_optin, int sm_count,
         best = cost; p.bw = bw; p.bh = bh; p.bg = bg;
       }
     }
+  // Layers with at most 64 output channels (3-wide filters, stride 1): rows 0-63 of the tile hold the
+  // gradients of an even image row, rows 64-127 those of the odd row below it, so one box of encodings at
+  // vertical offset dy serves filter row dy for the even rows and dy-1 for the odd ones: kh+1 items over
+  // half the image rows instead of kh half-used items over all of them.
+  // Taken when its padded pixel count x (kh+1) is below the plain tiling's x kh.
+  p.mpack = (opt.v[DK_OPT_TC_MPACK] && g.kind == DK_CONV2D && g.cout <= 64 && g.cin <= 64 && g.kw == 3 && g.kh >= 2 &&
+             g.stride == 1 && opt.v[DK_OPT_WG_PACK]) ? 1 : 0;
+  if (p.mpack) {
+    const long long two_row = (long long)((g.wo + P - 1) / P) * P * ((g.ho + 1) / 2) * g.G * (g.kh + 1);
+    if (two_row >= best * g.kh) p.mpack = 0;
+  }
+  if (p.mpack) { p.bw = P; p.bh = 1; p.bg = 1; }
   p.WT = (g.wo + p.bw - 1) / p.bw;
-  p.HT = (g.ho + p.bh - 1) / p.bh;
+  p.HT = p.mpack ? (g.ho + 1) / 2 : (g.ho + p.bh - 1) / p.bh;
   p.GT = (g.G + p.bg - 1) / p.bg;
   long long pb = (long long)p.WT * p.HT * p.GT;
   if (pb > 0x3fffffffLL) return false;
@@ -619,8 +631,9 @@ bool plan_wgrad(const Options& opt, const Geom& g, int smem_optin, int sm_count,
     p.cb = 256;
     p.tpn = 1;
   }
+  if (p.mpack) p.tpn = g.kw;
   w->BN = p.cb * p.tpn;
-  p.TG = (p.taps + p.tpn - 1) / p.tpn;
+  p.TG = p.mpack ? g.kh + 1 : (p.taps + p.tpn - 1) / p.tpn;
   const int pair_on = opt.v[DK_OPT_WG_PAIR];
   w->pair = pair_on && g.cout > BM;
   p.MT = w->pair ? (g.cout + BM2 - 1) / BM2 : (g.cout + BM - 1) / BM;

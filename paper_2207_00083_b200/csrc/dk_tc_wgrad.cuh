@@ -46,6 +46,7 @@ struct WgTcParams {
   int nstages, chunk;
   unsigned spin_cap;           // polls after which a wait gives up
   int withhold;                // test hook: the producer arms its n-th stage but issues no copy (-1 = off)
+  int mpack;                   // cout <= 64: rows 64-127 of the tile are the gradients one image row below rows 0-63
   int cout, cin;
   float scale;
   float* dW;                   // [cout][taps][cin]
@@ -160,18 +161,26 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
         if (lane >= 2 * (BM / 32) && lane < NBOX) {
           const int gb = (int)rank * (PAIR ? BNL / 32 : 0) + ((lane - 2 * (BM / 32)) >> 1);
           const int slot = (gb * 32) / p.cb;
-          const int tap = tg * p.tpn + slot;
-          bx_c = tap < p.taps ? nb * p.cb + (gb * 32 - slot * p.cb) : p.cin;
-          const int tt = tap < p.taps ? tap : 0;
-          bx_u = tt / p.kw;
-          bx_v = tt - bx_u * p.kw;
+          if (p.mpack) {
+            // two-row tiles: the item is a vertical offset dy = tg (0..kh), its slots the kw taps of a filter
+            // row; rows 0-63 (even image rows) pair the box with tap row dy, rows 64-127 (the odd row below) with tap row dy-1
+            bx_c = nb * p.cb + (gb * 32 - slot * p.cb);
+            bx_u = tg;
+            bx_v = slot;
+          } else {
+            const int tap = tg * p.tpn + slot;
+            bx_c = tap < p.taps ? nb * p.cb + (gb * 32 - slot * p.cb) : p.cin;
+            const int tt = tap < p.taps ? tap : 0;
+            bx_u = tt / p.kw;
+            bx_v = tt - bx_u * p.kw;
+          }
         }
         for (int pb = pb_lo; alive && pb < pb_hi; ++pb) {
           int r = pb;
           const int wt = r % p.WT; r /= p.WT;
           const int ht = r % p.HT;
           const int gt = r / p.HT;
-          const int x0 = wt * p.bw, y0 = ht * p.bh, g0 = gt * p.bg;
+          const int x0 = wt * p.bw, y0 = p.mpack ? 2 * ht : ht * p.bh, g0 = gt * p.bg;      // (two-row tiles step two image rows)
           for (int j = 0; j < p.K1; ++j) {
             int ok = 1;
             if (lane == 0) {
@@ -190,8 +199,11 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
             };
             if (lane < 2 * (BM / 32)) {
               const int cb = lane >> 1;
-              if ((lane & 1) == 0) load(st + cb * kWgBox, &map_d_hi, m0 + cb * 32, x0, y0);
-              else load(st + A_BYTES + cb * kWgBox, &map_d_lo, m0 + cb * 32, x0, y0);
+              // two-row tiles: channel blocks 2 and 3 are channels 0..63 of the gradients one row below
+              const int ch = (p.mpack && cb >= 2) ? (cb - 2) * 32 : m0 + cb * 32;
+              const int yy = (p.mpack && cb >= 2) ? y0 + 1 : y0;
+              if ((lane & 1) == 0) load(st + cb * kWgBox, &map_d_hi, ch, x0, yy);
+              else load(st + A_BYTES + cb * kWgBox, &map_d_lo, ch, x0, yy);
             } else if (lane < NBOX) {
               const int q = lane - 2 * (BM / 32);
               const int cb = q >> 1;
@@ -290,8 +302,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
         }
       }
       if (!alive) break;
-      const int co = mt * MROWS + (int)rank * BM + quad * 32 + lane;
-      if (co < p.cout && nchunks > 0) {
+      // two-row tiles: lanes 64-127 hold the same output channels, paired with the filter row one up
+      const int co = p.mpack ? (quad & 1) * 32 + lane : mt * MROWS + (int)rank * BM + quad * 32 + lane;
+      const int urow = p.mpack ? tg - (quad >> 1) : 0;      // filter row of this lane's products (two-row tiles)
+      if (co < p.cout && nchunks > 0 && (!p.mpack || (urow >= 0 && urow * p.kw < p.taps))) {
         float* row = p.dW + (size_t)co * p.taps * p.cin;
         // 16-byte vector reductions: cin % 4 == 0 and cb % 4 == 0 keep every group
         // of four inside one tap slot, wholly inside or outside the channel range,
@@ -300,7 +314,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
         for (int c = 0; c < NH; c += 4) {
           const int col = half * NH + c;
           const int slot = col / p.cb;
-          const int tap = tg * p.tpn + slot;
+          const int tap = p.mpack ? urow * p.kw + slot : tg * p.tpn + slot;
           const int ch = nb * p.cb + (col - slot * p.cb);
           if (tap < p.taps && ch < p.cin)
             asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(row + (size_t)tap * p.cin + ch),

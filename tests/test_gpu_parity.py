@@ -68,6 +68,8 @@ def small_cases():
         ("mpack_5x5", tiny(cin=8, cout=24, h=9, w=33, kh=5, kw=5, pad=2, K=4, G=2)),
         ("mpack_2x2_nopad", tiny(cin=8, cout=16, h=8, w=8, kh=2, kw=2, pad=0, K=4, G=1)),
         ("mpack_cin96", tiny(cin=96, cout=64, h=5, w=40, K=4, G=2)),
+        ("mpack_wg_ragged", tiny(cin=24, cout=40, h=7, w=60, K=4, G=3)),
+        ("mpack_wg_3x3_nopad", tiny(cin=64, cout=64, h=10, w=34, pad=0, K=2, G=2)),
         # the fused fp64 kernel of pointwise layers: ragged pixel tiles, ragged channel blocks, a ragged last
         # chunk of the contraction (cin 24), every warp layout (cout 8 .. 300), K = 1 .. 8
         ("f64_K8_ragged", tiny(cin=24, cout=40, h=7, w=7, kh=1, kw=1, pad=0, K=8, G=2, sigma_r=1000.0,
