@@ -56,10 +56,21 @@ FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # SMs x FMA lanes x 2
 # fp64 rate of this part: 148 SMs x 64 fp64 FMA lanes x 2 x 1.965 GHz = 37.2 TFLOP/s; a register-resident loop of
 # mma.sync.m8n8k4.f64 measured 37.0 and one of plain fp64 FMAs 36.6 on this machine
 FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
-# DRAM bytes (read + write) per launch of the GEMM kernel classes, average over the layers' launches, from
-# ncu captures of these kernels (summaries with their commands under profiles/); a workload or class that is
-# absent here has not been captured since the kernels last changed and reports null.
-NCU_TRAFFIC_BYTES = {"vgg16_224": {"linear_fwd": 2833418752, "wgrad": 6314548352}}
+# DRAM bytes (read + write) of all launches of a GEMM kernel class in ONE step of the workload, from ncu captures
+# of these kernels (summaries with their commands under profiles/); the bench line divides by the launches per
+# step.  A workload or class that is absent here has not been captured since the kernels last changed and
+# reports null.
+NCU_TRAFFIC_BYTES_PER_STEP = {}
+
+
+def apply_options(dk, ctx, args):
+    """--option NAME=VALUE pairs -> dk_set_option; returns them as a dict for the output line."""
+    out = {}
+    for item in args.option:
+        name, value = item.split("=", 1)
+        dk.dk_set_option(ctx, getattr(dk, "DK_OPT_" + name.upper()), int(value))
+        out[name.upper()] = int(value)
+    return out
 
 
 def read_peaks():
@@ -294,6 +305,7 @@ def run_layer_table(args):
     peaks = read_peaks()
     tf32_peak = peaks["bf16_tflops"] * TF32_OVER_BF16
     ctx = dk.Context(0)
+    options = apply_options(dk, ctx, args)
     gen = torch.Generator(device=dev)
     gen.manual_seed(220700083)
     flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)
@@ -311,7 +323,7 @@ def run_layer_table(args):
         torch.cuda.empty_cache()
     print(json.dumps({"layer_table": args.workload, "tf32_peak_tflops": tf32_peak, "hbm_gbs": peaks["hbm_gbs"],
                       "fp32_alu_peak_tflops": FP32_ALU_PEAK_TFLOPS, "peak_source": peaks["source"],
-                      "rows": rows}), flush=True)
+                      "options": options, "rows": rows}), flush=True)
 
 
 P_FIELD, L_FIELD = 2 ** 25 - 39, 8     # the prime and the fractional bits the paper uses (Section 5)
@@ -538,7 +550,8 @@ def profile_layers(torch, dk, ctx, layers, peaks, tf32_peak, flush, iters=2):
             prof = dk.dk_profile_read(ctx)
             dk.dk_profile_enable(ctx, False)
             ms = tot / iters
-            kms = prof[kind][0] / max(prof[kind][1], 1)
+            kms = prof[kind][0] / iters        # all GEMM launches of one call (a large layer's call has several)
+            nlaunch = prof[kind][1] / iters
             if call == "fwd_tf32x2w":
                 row[call] = {"call_ms": round(ms, 4), "kernel_ms": round(kms, 4),
                              "issued_tflops_kernel": round(2.0 * s.fwd_flops() / kms / 1e9, 2) if kms > 0 else None,
@@ -547,7 +560,11 @@ def profile_layers(torch, dk, ctx, layers, peaks, tf32_peak, flush, iters=2):
             roof = layer_roofs(s, call, peaks, tf32_peak)
             flops = s.fwd_flops() if call == "fwd" else s.wgrad_flops()
             row[call] = {"bound": roof["bound"], "call_ms": round(ms, 4), "kernel_ms": round(kms, 4),
+                         "kernel_launches": nlaunch,
+                         # with several launches the pre-passes of later ranges run beside the GEMM of earlier
+                         # ones on a second stream: their time is then no part of call - kernel
                          "other_kernels_ms": round(sum(v[0] for k, v in prof.items() if k != kind) / iters, 4),
+                         "exposed_other_ms": round(ms - kms, 4),
                          "floor_ms": round(roof["floor_ms"], 4),
                          "frac_of_roof_call": round(roof["floor_ms"] / ms, 4),
                          "frac_of_roof_kernel": round(roof["floor_ms"] / kms, 4) if kms > 0 else None,
@@ -659,6 +676,7 @@ def run_ours(args):
 
     specs = synth.layers(args.workload)
     ctx = dk.Context(local)
+    options = apply_options(dk, ctx, args)
     gen = torch.Generator(device=dev)
     gen.manual_seed(220700083 + rank)
     layers = [make_layer(torch, dk, synth, ctx, s, dev, gen, rank, pinned=False) for s in specs]
@@ -752,21 +770,27 @@ def run_ours(args):
     call = "fwd" if dom == "linear_fwd" else "wgrad"
     dom_specs = [s for s in specs if call == "fwd" or s.wgrad]
     roofs = [layer_roofs(s, call, peaks, tf32_peak) for s in dom_specs]
-    issued_per_launch = sum(r["issued_flops"] for r in roofs) / len(dom_specs)
+    # a large layer's call is served by several launches (ranges of virtual batches), so the unit of this
+    # object is the average launch: one step's flops and bytes over one step's launches of the class
+    launches_per_step = prof[dom][1] / prof_steps
+    issued_per_launch = sum(r["issued_flops"] for r in roofs) / launches_per_step
     avg_ms = prof[dom][0] / max(prof[dom][1], 1)
     achieved = issued_per_launch / (avg_ms * 1e-3) / 1e12
-    alg_bytes = sum(algorithmic_bytes(s, call) for s in dom_specs) / len(dom_specs)
-    traffic = NCU_TRAFFIC_BYTES.get(args.workload, {}).get(dom)
+    alg_bytes = sum(algorithmic_bytes(s, call) for s in dom_specs) / launches_per_step
+    traffic = NCU_TRAFFIC_BYTES_PER_STEP.get(args.workload, {}).get(dom)
+    if traffic is not None:
+        traffic = traffic / launches_per_step
     roofline = {"bound": "tensor", "achieved": achieved, "peak": tf32_peak, "unit": "TFLOP/s",
                 "frac": achieved / tf32_peak, "frac_of_burst_peak": achieved / tf32_burst,
                 "traffic": traffic, "traffic_unit": "bytes per launch (ncu, dram read + write, average over "
-                "the layers' launches)", "algorithmic_bytes": alg_bytes,
-                "algorithmic_bytes_rule": "per call, fp32: fused forward reads (K+1) inputs per group and W, "
+                "the step's launches of this class)", "algorithmic_bytes": alg_bytes,
+                "launches_per_step": launches_per_step,
+                "algorithmic_bytes_rule": "one step's calls over its launches, fp32: fused forward reads (K+1) inputs per group and W, "
                 "writes K outputs and K+1 stored encodings; wgrad reads K gradients and K+1 encodings, writes dW",
                 "kernel": dom, "launches_timed": prof[dom][1], "avg_launch_ms": avg_ms,
                 "flops_per_launch": issued_per_launch,
                 "flops": "issued flops per launch = 3 x masked flops on the tensor-core kernels (3xTF32 split), "
-                         "1 x on the fp32 kernels, averaged over the layers (each launched once per step)",
+                         "1 x on the fp32 kernels, one step's total over one step's launches of the class",
                 "peak_source": f"{peaks['source']} bf16 {'sustained' if long_step else 'burst'} {bf16} TFLOP/s "
                                f"x nominal TF32:BF16 ratio {TF32_OVER_BF16:.4f} (kernel timed inside a "
                                f"{'long' if long_step else 'short'} step)"}
@@ -786,7 +810,7 @@ def run_ours(args):
                    "G": specs[0].G, "flops": "masked (all K+2 fwd / K+1 wgrad encodings)",
                    "l2": f"flushed between steps ({L2_FLUSH_BYTES >> 20} MiB write, untimed); every large "
                          f"layer's tensors exceed L2 by themselves",
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "parallelism": "replicas only" if world > 1 else "single GPU", "options": options},
         "decoded_useful_tflops": value * (K / (K + 2) * fwd_flops + K / (K + 1) * wg_flops) / step_flops,
         "encode_gbs": elem["encode"]["gbs"], "decode_gbs": elem["decode"]["gbs"],
         "encode_frac_hbm": elem["encode"]["frac_hbm"], "decode_frac_hbm": elem["decode"]["frac_hbm"],
@@ -917,6 +941,9 @@ def main():
     ap.add_argument("--field-table", action="store_true")
     ap.add_argument("--layers", default="")
     ap.add_argument("--iters", type=int, default=5)
+    ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
+                    help="a library option for this run, e.g. TC_CHUNK=4 (dk_set_option with DK_OPT_<NAME>); "
+                         "the line then carries it under config.options")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

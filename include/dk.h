@@ -173,6 +173,35 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  *                     two output rows of the image (rows 64-127 hold the filters of
  *                     the tap one row up, so one activation box serves both); 0: one
  *                     output row per tile, half of every product unused.
+ *                     The weight-gradient kernel does the same with an even and
+ *                     an odd row of the gradients.
+ *   DK_OPT_TC_CHUNK_ADAPT  1 (default): DK_OPT_TC_CHUNK is the most the forward kernels add
+ *                     up in tensor memory; a virtual batch whose coefficients
+ *                     amplify errors in the noise term of the encoded outputs
+ *                     (a = max_k sum_i |Cinv[k][i]| |C[i][K]|, in exact arithmetic
+ *                     the noise cancels: sum_i Cinv[k][i] C[i][K] = 0) takes shorter
+ *                     chunks: 8 k-blocks up to a = 8, 4 up to 16, 2 up to 32, 1
+ *                     beyond.  Measured at noise 100x the inputs, the decoded error is
+ *                     about (2.2e-5 + 0.5e-5 x k-blocks) x a of the output scale, so
+ *                     this keeps it below 1e-3 up to a = 32.  0: every tile uses
+ *                     DK_OPT_TC_CHUNK.
+ *   DK_OPT_SLABS      default 1: one pre-pass launch, then one GEMM launch.  n > 1:
+ *                     the tensor-core forward and weight-gradient calls may be cut
+ *                     into up to n ranges of virtual batches (at most 8): the
+ *                     HBM-bound pre-pass (Eq. 1 / Eq. 4 mixing, second TF32 terms)
+ *                     of a later range runs on a stream owned by the context while
+ *                     the GEMM of an earlier range runs on the caller's stream; the
+ *                     call leaves both joined (it is still one unit of work on the
+ *                     caller's stream, and can be captured).  The library picks
+ *                     the count per layer from the sizes.  Outputs, stored
+ *                     encodings and verdicts do not depend on it; dW does within
+ *                     the error of its arithmetic (the contraction is sliced
+ *                     differently).  Off by default because it measured slower on
+ *                     every large layer: the GEMM kernels lose more to the
+ *                     pre-pass's traffic through L2 than the overlap hides.
+ *   DK_OPT_SLABS_FORCE  default 0: the library picks the count; n >= 1: exactly
+ *                     min(n, DK_OPT_SLABS, tiles along the virtual batches) launches,
+ *                     whatever the sizes (for tests and measurements).
  *   DK_OPT_TEST_WITHHOLD  test hook, default -1 (off): the producer warp of the
  *                     next tensor-core forward or weight-gradient kernel arms the
  *                     barrier of its n-th pipeline stage but issues no copy for
@@ -182,7 +211,8 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
 enum {
   DK_OPT_TC_CHUNK = 0, DK_OPT_WG_CHUNK = 1, DK_OPT_TC_BK = 2, DK_OPT_TC_PAIR = 3, DK_OPT_WG_PACK = 4,
   DK_OPT_WG_PAIR = 5, DK_OPT_TC_STEM = 6, DK_OPT_FIELD_PATH = 7, DK_OPT_SPIN_LIMIT = 8,
-  DK_OPT_TEST_WITHHOLD = 9, DK_OPT_XBAR_HI = 10, DK_OPT_TC_MPACK = 11, DK_OPT_COUNT = 12
+  DK_OPT_TEST_WITHHOLD = 9, DK_OPT_XBAR_HI = 10, DK_OPT_TC_MPACK = 11, DK_OPT_SLABS = 12, DK_OPT_SLABS_FORCE = 13,
+  DK_OPT_TC_CHUNK_ADAPT = 14, DK_OPT_COUNT = 15
 };
 DK_API dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value);
 DK_API dk_status dk_get_option(dk_ctx* ctx, int32_t option, int32_t* value);

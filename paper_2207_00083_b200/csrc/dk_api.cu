@@ -105,7 +105,8 @@ dk_status upload_coefficients(dk_ctx* ctx, const Geom& g, const float* C_host,
   const int K = g.K, K1 = K + 1, E = K + 2, G = g.G;
   const size_t n_enc = (size_t)G * E * K1, n_dec = (size_t)G * K * K1, n_nul = (size_t)G * E,
                n_mix = (size_t)G * K1 * K;
-  const size_t total = n_enc + 2 * n_dec + n_nul + n_mix;
+  const size_t n_chk = ((size_t)G + 3) / 4;      // one byte per group
+  const size_t total = n_enc + 2 * n_dec + n_nul + n_mix + n_chk;
   if (total * sizeof(float) > kCoefSlotBytes) return DK_ERR_SHAPE;
   if (!C_host) return DK_ERR_INVALID_ARG;
   if (want_mix && !gamma_host) return DK_ERR_INVALID_ARG;
@@ -122,6 +123,10 @@ dk_status upload_coefficients(dk_ctx* ctx, const Geom& g, const float* C_host,
   float* h_mix = h_nul + n_nul;
   memcpy(h_enc, C_host, n_enc * sizeof(float));
   memset(h_dec, 0, (2 * n_dec + n_nul + n_mix) * sizeof(float));
+  unsigned char* h_chunk = reinterpret_cast<unsigned char*>(h_mix + n_mix);
+  memset(h_chunk, 8, n_chk * 4);
+  view->chunk_cap = 8;
+  view->chunk_tab = nullptr;
 
   if (want_dec || want_mix) {
     double sq[(DK_MAX_K + 1) * (DK_MAX_K + 1)], inv[(DK_MAX_K + 1) * (DK_MAX_K + 1)];
@@ -137,6 +142,23 @@ dk_status upload_coefficients(dk_ctx* ctx, const Geom& g, const float* C_host,
           h_dec[((size_t)gi * K + k) * K1 + i] = hi;
           h_decl[((size_t)gi * K + k) * K1 + i] = (float)(v - (double)hi);
         }
+      // How strongly decoding amplifies an error that is relative to the noise term of the encoded outputs:
+      // a = max_k sum_i |inv[k][i]| |C[i][K]| (in exact arithmetic sum_i inv[k][i] C[i][K] = 0: the noise
+      // cancels).  The forward kernels' accumulator in tensor memory truncates when it adds, a bias that grows
+      // with the k-blocks added there; measured at noise 100x the inputs, the decoded error is about
+      // (2.2e-5 + 0.5e-5 x k-blocks) x a of the output scale.  The chunk lengths below keep that under 1e-3
+      // up to a = 32 (beyond, one k-block per chunk is the best this arithmetic does).
+      {
+        double amp = 0.0;
+        for (int k = 0; k < K; ++k) {
+          double a = 0.0;
+          for (int i = 0; i < K1; ++i) a += fabs(inv[k * K1 + i]) * fabs((double)Cg[i * K1 + K]);
+          amp = a > amp ? a : amp;
+        }
+        const int cap = amp <= 8.0 ? 8 : (amp <= 16.0 ? 4 : (amp <= 32.0 ? 2 : 1));
+        if (cap < view->chunk_cap) view->chunk_cap = cap;
+        h_chunk[gi] = (unsigned char)cap;
+      }
       // null vector: n[0..K] = -C[K+1] . C_sq^{-1}, n[K+1] = 1
       for (int i = 0; i < K1; ++i) {
         double acc = 0.0;
@@ -165,6 +187,10 @@ dk_status upload_coefficients(dk_ctx* ctx, const Geom& g, const float* C_host,
   view->decl = view->dec + n_dec;
   view->nul = view->decl + n_dec;
   view->dmix = view->nul + n_nul;
+  if ((want_dec || want_mix) && ctx->opt.v[DK_OPT_TC_CHUNK_ADAPT])
+    view->chunk_tab = reinterpret_cast<const unsigned char*>(view->dmix + n_mix);
+  else
+    view->chunk_cap = 64;
   return DK_OK;
 }
 
@@ -309,7 +335,7 @@ dk_status dk_create(dk_ctx** out, int device) {
     return DK_ERR_CUDA;
   }
   c->sm_count = sms;
-  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1, 1};
+  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1, 1, 1, 0, 1};
   for (int i = 0; i < DK_OPT_COUNT; ++i) c->opt.v[i] = kOptDefault[i];
   bool ok = cudaMallocHost(&c->h_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
@@ -318,6 +344,10 @@ dk_status dk_create(dk_ctx** out, int device) {
             cudaMalloc(&c->d_cand, kCandCap * sizeof(Candidate)) == cudaSuccess;
   for (int i = 0; ok && i < kCoefSlots; ++i)
     ok = cudaEventCreateWithFlags(&c->slot_ev[i], cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess &&
+       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; ok && i < kMaxSlabs; ++i)
+    ok = cudaEventCreateWithFlags(&c->ev_slab[i], cudaEventDisableTiming) == cudaSuccess;
   c->prof = new (std::nothrow) ProfState();
   ok = ok && c->prof != nullptr;
   if (ok) ok = tc_init(c) == DK_OK;
@@ -333,6 +363,10 @@ dk_status dk_destroy(dk_ctx* c) {
   tc_destroy(c);
   for (int i = 0; i < kCoefSlots; ++i)
     if (c->slot_ev[i]) cudaEventDestroy(c->slot_ev[i]);
+  for (int i = 0; i < kMaxSlabs; ++i)
+    if (c->ev_slab[i]) cudaEventDestroy(c->ev_slab[i]);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->side) cudaStreamDestroy(c->side);
   if (c->prof) {
     for (cudaEvent_t e : c->prof->ev) cudaEventDestroy(e);
     delete c->prof;
@@ -347,8 +381,8 @@ dk_status dk_destroy(dk_ctx* c) {
 
 dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx || option < 0 || option >= DK_OPT_COUNT) return DK_ERR_INVALID_ARG;
-  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0, 0};
-  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 2, 1 << 26, 1 << 20, 1, 1};
+  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0, 0, 1, 0, 0};
+  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 2, 1 << 26, 1 << 20, 1, 1, kMaxSlabs, kMaxSlabs, 1};
   int v = value < lo[option] ? lo[option] : (value > hi[option] ? hi[option] : value);
   if (option == DK_OPT_TC_BK) v = v == 16 ? 16 : 32;
   ctx->opt.v[option] = v;
@@ -459,6 +493,45 @@ dk_status dk_decode_verify(dk_ctx* ctx, const dk_problem* p, const float* ybar,
   return launch_verify_finalize(g, cv.nul, vs, verdict, st);
 }
 
+// Launches a call's groups are cut into: the pre-pass of a later range runs beside the GEMM of an earlier one,
+// so n launches leave 1/n of the pre-pass exposed, and each launch but the last ends with CTAs idle for about
+// half the time of one of its work items.  prep_bytes at a nominal 5.5 TB/s against gemm_flops (as issued) at a
+// nominal 600 TFLOP/s: only the ratio matters.
+static int plan_slabs(const dk_ctx* ctx, int GT, long long rounds, double prep_bytes, double gemm_flops,
+                      double tail_floor = 5e-6) {
+  int cap = ctx->opt.v[DK_OPT_SLABS];
+  if (cap > kMaxSlabs) cap = kMaxSlabs;
+  if (cap > GT) cap = GT;
+  const int force = ctx->opt.v[DK_OPT_SLABS_FORCE];
+  if (force > 0) return force < cap ? force : (cap < 1 ? 1 : cap);
+  if (cap < 2 || rounds < 1) return 1;
+  const double tp = prep_bytes / 5.5e12;
+  double tail = 0.5 * (gemm_flops / 6.0e14) / (double)rounds;
+  if (tail < tail_floor) tail = tail_floor;
+  int best = 1;
+  double best_cost = tp;
+  for (int n = 2; n <= cap; ++n) {
+    const double cost = tp / n + (n - 1) * tail;
+    if (cost < best_cost * 0.98) { best_cost = cost; best = n; }
+  }
+  return best;
+}
+
+// The context's second stream joins the caller's stream for the duration of one call: it starts behind
+// everything already enqueued there, and the caller's stream waits for its last piece of work before the
+// call returns, whatever happens in between.
+struct SideStream {
+  dk_ctx* ctx;
+  cudaStream_t main;
+  bool forked;
+  SideStream(dk_ctx* c, cudaStream_t st) : ctx(c), main(st), forked(false) {
+    forked = cudaEventRecord(c->ev_fork, st) == cudaSuccess && cudaStreamWaitEvent(c->side, c->ev_fork, 0) == cudaSuccess;
+  }
+  ~SideStream() {
+    if (forked && cudaEventRecord(ctx->ev_fork, ctx->side) == cudaSuccess) cudaStreamWaitEvent(main, ctx->ev_fork, 0);
+  }
+};
+
 dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, const float* x,
                            const float* r, const float* C_host, const float* bias, float* y,
                            float* xbar_save, dk_verdict* verdict, const dk_fault* fault,
@@ -528,6 +601,40 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     const int raw = stem ? 0 : ctx->opt.v[DK_OPT_XBAR_HI];
     float* full = xbar_save;
     if (raw && !full) full = reinterpret_cast<float*>(ws + wp.xbar);
+    // Large layers: the groups are cut into ranges; the pre-passes run in order on the context's second stream,
+    // the GEMM of a range starts on the caller's stream as soon as its pre-pass has finished, and the kernel
+    // of the last range takes the final decisions of the check.
+    int nslab = 1, GT = 0, bg = 1;
+    if (!stem && ksplit == 1) {
+      long long rounds = 0;
+      if (tc_fwd_group_tiles(ctx, gg, &GT, &bg, &rounds)) {
+        const double prep = ((double)(g.K + 1) + (raw ? 2.0 : 3.0) * g.E) * g.G * (double)g.n_in * 4.0;
+        nslab = plan_slabs(ctx, GT, rounds, prep, 6.0 * g.G * g.E * (double)g.n_out * g.kc);
+      }
+    }
+    if (nslab > 1) {
+      SideStream fork(ctx, st);
+      if (!fork.forked) return DK_ERR_CUDA;
+      int gt_lo[kMaxSlabs + 1];
+      for (int i = 0; i <= nslab; ++i) gt_lo[i] = (int)((long long)GT * i / nslab);
+      for (int i = 0; i < nslab && s == DK_OK; ++i) {
+        const int g_lo = gt_lo[i] * bg, g_hi = gt_lo[i + 1] * bg < g.G ? gt_lo[i + 1] * bg : g.G;
+        {
+          ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, ctx->side);
+          s = tc_fwd_prepass(gg, x, r, cv.enc, full, raw ? nullptr : xb_hi, xb_lo, W, w_hi, w_lo, vs, nullptr,
+                             ctx->sm_count, ctx->side, raw, g_lo, g_hi - g_lo, i > 0);
+        }
+        if (s == DK_OK && cudaEventRecord(ctx->ev_slab[i], ctx->side) != cudaSuccess) s = DK_ERR_CUDA;
+      }
+      if (raw) xb_hi = full;
+      for (int i = 0; i < nslab && s == DK_OK; ++i) {
+        if (cudaStreamWaitEvent(st, ctx->ev_slab[i], 0) != cudaSuccess) { s = DK_ERR_CUDA; break; }
+        ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
+        s = tc_masked_fwd(ctx, gg, w_hi, w_lo, xb_hi, xb_lo, cv, bias, y, vs, reinterpret_cast<int*>(vs.count + 1),
+                          fault, i == nslab - 1 ? verdict : nullptr, st, gt_lo[i], gt_lo[i + 1] - gt_lo[i]);
+      }
+      return s;
+    }
     {
       // one launch: encodings and weights as hi/lo pairs, integrity statistics cleared
       ProfScope ps(ctx, DK_KERNEL_ENCODE, 1, st);
@@ -543,7 +650,7 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
       {
         ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
         s = tc_linear_fwd(ctx, gg, w_hi, w_lo, xb_hi, xb_lo, ybar, ksplit, prepass_clears,
-                          reinterpret_cast<int*>(vs.count + 1), st);
+                          reinterpret_cast<int*>(vs.count + 1), st, cv.chunk_cap);
       }
       if (s != DK_OK) return s;
       if (fault) {
@@ -666,10 +773,47 @@ static dk_status wgrad_impl(dk_ctx* ctx, const Geom& g, const WsPlan& wp, const 
     float* dt_lo = reinterpret_cast<float*>(ws + wp.ybar);
     float* xb_hi = reinterpret_cast<float*>(ws + wp.xb_hi);
     float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
+    const int raw = ctx->opt.v[DK_OPT_XBAR_HI];
+    int nslab = 1, GT = 0, bg = 1;
+    {
+      long long rounds = 0;
+      if (tc_wgrad_group_tiles(ctx, g, &GT, &bg, &rounds)) {
+        const double prep = (g.K + 2.0 * (g.K + 1)) * g.G * (double)g.n_out * 4.0 +
+                            (raw ? 2.0 : 3.0) * (g.K + 1) * g.G * (double)g.n_in * 4.0;
+        // (every launch slices its own part of the contraction to fill the device, so what a further launch
+        // costs is its fixed part: pipeline fill and the reductions into dW, about 15 us)
+        nslab = plan_slabs(ctx, GT, 1LL << 30, prep, 6.0 * g.G * (g.K + 1) * (double)g.n_out * g.kc, 15e-6);
+      }
+    }
+    if (nslab > 1) {
+      // ranges of groups: the pre-passes in order on the second stream, each range's products on the caller's
+      // stream once its pre-pass has finished (they add into dW, which the first pre-pass clears)
+      SideStream fork(ctx, st);
+      if (!fork.forked) return DK_ERR_CUDA;
+      int gt_lo[kMaxSlabs + 1];
+      for (int i = 0; i <= nslab; ++i) gt_lo[i] = (int)((long long)GT * i / nslab);
+      for (int i = 0; i < nslab && s == DK_OK; ++i) {
+        const int g_lo = gt_lo[i] * bg, g_hi = gt_lo[i + 1] * bg < g.G ? gt_lo[i + 1] * bg : g.G;
+        {
+          ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, ctx->side);
+          s = tc_wgrad_prepass(g, delta, cv.dmix, dtil, dt_lo, xbar, xbar_elems, raw ? nullptr : xb_hi, xb_lo,
+                               accumulate ? nullptr : dW, ctx->sm_count, ctx->side, raw, xbar_rows, g_lo, g_hi - g_lo,
+                               i > 0);
+        }
+        if (s == DK_OK && cudaEventRecord(ctx->ev_slab[i], ctx->side) != cudaSuccess) s = DK_ERR_CUDA;
+      }
+      if (raw) xb_hi = const_cast<float*>(xbar);
+      for (int i = 0; i < nslab && s == DK_OK; ++i) {
+        if (cudaStreamWaitEvent(st, ctx->ev_slab[i], 0) != cudaSuccess) { s = DK_ERR_CUDA; break; }
+        ProfScope ps(ctx, DK_KERNEL_WGRAD, 1, st);
+        s = tc_wgrad(ctx, g, dtil, dt_lo, xb_hi, xb_lo, xbar_rows, scale, dW, ctx_status_word(ctx), st, gt_lo[i],
+                     gt_lo[i + 1] - gt_lo[i]);
+      }
+      return s;
+    }
     {
       // one launch: mixed deltas and stored encodings as hi/lo pairs, dW cleared
       ProfScope ps(ctx, DK_KERNEL_MIX_DELTA, 1, st);
-      const int raw = ctx->opt.v[DK_OPT_XBAR_HI];
       s = tc_wgrad_prepass(g, delta, cv.dmix, dtil, dt_lo, xbar, xbar_elems, raw ? nullptr : xb_hi, xb_lo,
                            accumulate ? nullptr : dW, ctx->sm_count, st, raw, xbar_rows);
       if (raw) xb_hi = const_cast<float*>(xbar);      // the stored encodings are the leading term

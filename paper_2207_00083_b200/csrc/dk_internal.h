@@ -41,9 +41,13 @@ struct CoefView {
   const float* decl;
   const float* nul;
   const float* dmix;
+  int chunk_cap;         // k-blocks (of 32 contraction elements) the forward kernels may add up in tensor memory
+                         // between promotions with these coefficients: the worst group's value, and
+  const unsigned char* chunk_tab;   // one value per group (device; null when the tables were not derived)
 };
 
 constexpr int kCoefSlots = 8;
+constexpr int kMaxSlabs = 8;       // most launches one call's groups are cut into
 constexpr size_t kCoefSlotBytes = 512 * 1024;
 
 // Scratch of the integrity check.  The decision for an element needs the rms
@@ -90,6 +94,10 @@ struct dk_ctx {
   void* tc_state;             // tensor-core path state
   dk::ProfState* prof;        // launch counters and event records
   dk::Options opt;
+  // second stream on which the pre-passes of a call's later group ranges run beside the GEMM of the earlier ones
+  cudaStream_t side;
+  cudaEvent_t ev_fork;
+  cudaEvent_t ev_slab[dk::kMaxSlabs];
 };
 
 namespace dk {
@@ -189,7 +197,8 @@ dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const f
 int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g);
 dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
                         const float* xb_hi, const float* xb_lo, float* ybar, int ksplit, bool ybar_cleared,
-                        int* status_word, cudaStream_t st);
+                        int* status_word, cudaStream_t st, int chunk_cap = 0);
+// (chunk_cap > 0: cap on the k-blocks of 32 added up in tensor memory, see CoefView::chunk_cap)
 // weight gradient on tensor cores (channels-last, stride 1, cin % 4 == 0, cout % 4 == 0)
 bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g);
 // Eq. 4 delta mixing written as a TF32 hi/lo pair, [G*(K+1)][n_out] each
@@ -199,28 +208,39 @@ dk_status tc_mix_split(const Geom& g, const float* delta, const float* dmix, flo
 // caller has cleared (tc_wgrad_prepass does)
 dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* dt_lo,
                    const float* xb_hi, const float* xb_lo, int xbar_rows, float scale, float* dW,
-                   int* status_word, cudaStream_t st);
+                   int* status_word, cudaStream_t st, int gt_lo = 0, int gt_cnt = -1);
+// (gt_cnt >= 0: only the pixel blocks of group tiles [gt_lo, gt_lo + gt_cnt); tc_wgrad_group_tiles gives the
+// number of group tiles, the groups per tile and the rounds of work items a whole launch deals to a CTA)
+bool tc_wgrad_group_tiles(const dk_ctx* ctx, const Geom& g, int* GT, int* bg, long long* rounds);
 // One launch for everything a masked forward call prepares (dk_tc_prepass.cu):
 // Eq. 1 encodings as hi/lo pairs (and in full when `full` is given), W as a
 // hi/lo pair, cleared integrity statistics, and (ybar_clear != nullptr) the
 // y_bar buffer of a split-K call cleared.
 dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const float* enc, float* full,
                          float* xb_hi, float* xb_lo, const float* W, float* w_hi, float* w_lo,
-                         const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st, int raw = 0);
+                         const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st, int raw = 0,
+                         int g_lo = 0, int g_cnt = -1, bool beside = false);
+// (g_lo, g_cnt: only the encodings of groups [g_lo, g_lo + g_cnt); the launch with g_lo = 0 does the rest.
+// beside: the launch is to run next to a GEMM kernel on another stream and takes a small grid of small blocks.)
 // (raw != 0: xb_hi is not written; the reader takes the fp32 encodings in `full` as leading term and
 // xb_lo holds tf32(v - trunc(v)))
 // One launch for what a weight-gradient call prepares: Eq. 4 delta mixing and
 // the stored encodings as hi/lo pairs, dW cleared (dW = nullptr: left as it is).
 dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix, float* dt_hi, float* dt_lo,
                            const float* xbar, long long xbar_elems, float* xb_hi, float* xb_lo, float* dW,
-                           int sm_count, cudaStream_t st, int raw = 0, int xbar_rows = 0);
+                           int sm_count, cudaStream_t st, int raw = 0, int xbar_rows = 0, int g_lo = 0,
+                           int g_cnt = -1, bool beside = false);
+// (g_lo, g_cnt: only groups [g_lo, g_lo + g_cnt); the launch with g_lo = 0 clears dW)
 // (raw != 0: only xb_lo is written, and only for the K+1 encodings of each group that Eq. 4 uses)
 // same contraction with decode + integrity statistics in the epilogue; when
 // `verdict` is given the kernel's last CTA also writes it (no finalize launch)
 dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
                         const float* xb_hi, const float* xb_lo, const CoefView& cv, const float* bias,
                         float* y, const VerifyScratch& vs, int* status_word, const dk_fault* fault,
-                        dk_verdict* verdict, cudaStream_t st);
+                        dk_verdict* verdict, cudaStream_t st, int gt_lo = 0, int gt_cnt = -1);
+// (gt_cnt >= 0: only group tiles [gt_lo, gt_lo + gt_cnt) of the tiling; a call served by several such launches
+// gives `verdict` to the last one.  tc_fwd_group_tiles: group tiles, groups per tile, rounds of tiles per CTA.)
+bool tc_fwd_group_tiles(const dk_ctx* ctx, const Geom& g, int* GT, int* bg, long long* rounds);
 
 // Forward pass of layers with cin % 4 != 0 (3-channel stems) on the tensor-core kernels: the
 // pre-pass lays the kc inputs under the filter out as rows of Kp = kc rounded

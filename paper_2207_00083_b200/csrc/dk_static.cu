@@ -141,6 +141,8 @@ extern "C" dk_status dk_decode_verify_static(int device, const dk_problem* p, co
       cv.decl = d_tab + n_dec;
       cv.nul = d_tab + 2 * n_dec;
       cv.dmix = nullptr;
+      cv.chunk_cap = 8;
+      cv.chunk_tab = nullptr;
       dk::VerifyScratch vs;
       vs.sumsq = d_stat;
       vs.maxrho = reinterpret_cast<int*>(d_stat + (size_t)G * E);

@@ -204,7 +204,8 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
   // a CTA of a pair stages its own 128 rows of W and half of the activation rows
   const size_t stage = 2 * ((size_t)BM * BK * 4 + (size_t)(pair ? t->BN / 2 : t->BN) * BK * 4);
   const size_t ctrl = 1024 + 256;   // alignment slack + barriers
-  int ns = (int)(((size_t)smem_optin - ctrl) / stage);
+  const size_t fixed = 1024 + 64;   // the kernels' static shared memory (table of chunk lengths)
+  int ns = (int)(((size_t)smem_optin - ctrl - fixed) / stage);
   if (ns > kMaxStages) ns = kMaxStages;
   if (ns < 2) return false;
   t->nstages = ns;
@@ -317,9 +318,11 @@ void fill_params(const TcState* ts, const Geom& g, const Tiling& tl, TcParams* p
   p->log2_bw = 0; while ((1 << p->log2_bw) < tl.bw) ++p->log2_bw;
   p->log2_S = 0; while ((1 << p->log2_S) < tl.bw * tl.bh) ++p->log2_S;
   p->WT = tl.WT; p->HT = tl.HT; p->GT = tl.GT; p->MT = tl.MT;
+  p->gt0 = 0;
   p->ntiles = tl.ntiles; p->KB = tl.KB; p->CB = tl.CB;
   // 32-wide k-blocks accumulated in TMEM between promotions (the error grows ~linearly with it)
   p->chunk = ts->opt->v[DK_OPT_TC_CHUNK] * (32 / fwd_bk(ts));
+  p->chunk_tab = nullptr; p->chunk_mul = 32 / fwd_bk(ts);
   p->spin_cap = (unsigned)ts->opt->v[DK_OPT_SPIN_LIMIT];
   p->withhold = ts->opt->v[DK_OPT_TEST_WITHHOLD];
   p->nprod = g.nprod == 2 ? 2 : 3;
@@ -483,9 +486,19 @@ int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g) {
   return best;
 }
 
+bool tc_fwd_group_tiles(const dk_ctx* ctx, const Geom& g, int* GT, int* bg, long long* rounds) {
+  TcState* ts = static_cast<TcState*>(ctx->tc_state);
+  Tiling tl;
+  if (!ts || !plan_fwd(ts, g, &tl)) return false;
+  const int units = tl.pair ? ctx->sm_count / 2 : ctx->sm_count;
+  *GT = tl.GT; *bg = tl.bg;
+  *rounds = (tl.ntiles + units - 1) / units;
+  return true;
+}
+
 dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
                         const float* xb_lo, float* ybar, int ksplit, bool ybar_cleared, int* status_word,
-                        cudaStream_t st) {
+                        cudaStream_t st, int chunk_cap) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!plan_fwd(ts, g, &tl)) return DK_ERR_UNSUPPORTED;
@@ -498,6 +511,7 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
       DK_CUDA_CHECK(cudaMemsetAsync(ybar, 0, (size_t)g.G * g.E * g.n_out * sizeof(float), st));
   }
   prm.out = ybar;
+  if (chunk_cap > 0 && prm.chunk > chunk_cap * (32 / fwd_bk(ts))) prm.chunk = chunk_cap * (32 / fwd_bk(ts));
   prm.status = status_word;
   return launch_bk<MODE_YBAR>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
 }
@@ -505,14 +519,25 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
 dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
                         const float* xb_lo, const CoefView& cv, const float* bias, float* y,
                         const VerifyScratch& vs, int* status_word, const dk_fault* fault, dk_verdict* verdict,
-                        cudaStream_t st) {
+                        cudaStream_t st, int gt_lo, int gt_cnt) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!plan_fwd(ts, g, &tl)) return DK_ERR_UNSUPPORTED;
+  if (gt_cnt >= 0) {
+    // this launch covers group tiles [gt_lo, gt_lo + gt_cnt) only
+    if (gt_lo < 0 || gt_cnt < 1 || gt_lo + gt_cnt > tl.GT) return DK_ERR_INVALID_ARG;
+    tl.ntiles = tl.WT * tl.HT * gt_cnt * tl.MT;
+    tl.GT = gt_cnt;
+  }
   TcParams prm;
   fill_params(ts, g, tl, &prm);
+  if (gt_cnt >= 0) prm.gt0 = gt_lo;
   prm.out = y;
   prm.dec = cv.dec; prm.decl = cv.decl; prm.nul = cv.nul; prm.bias = bias;
+  // ill-conditioned coefficient sets take shorter chunks (see upload_coefficients): per virtual batch where the
+  // kernels' table holds them all, else the worst one's for the whole call
+  if (cv.chunk_tab != nullptr && g.G <= kChunkTabMax) prm.chunk_tab = cv.chunk_tab;
+  else if (cv.chunk_cap > 0 && prm.chunk > cv.chunk_cap * (32 / fwd_bk(ts))) prm.chunk = cv.chunk_cap * (32 / fwd_bk(ts));
   prm.vs = vs;
   prm.status = status_word;
   prm.verdict = verdict;
@@ -582,7 +607,8 @@ struct WgPlan {
   size_t smem_bytes;
 };
 
-bool plan_wgrad(const Options& opt, const Geom& g, int smem_optin, int sm_count, WgPlan* w) {
+bool plan_wgrad(const Options& opt, const Geom& g, int smem_optin, int sm_count, WgPlan* w, int gt_lo = 0,
+                int gt_cnt = -1) {
   WgTcParams& p = w->prm;
   const int P = kWgPix;
   long long best = -1;
@@ -611,9 +637,15 @@ bool plan_wgrad(const Options& opt, const Geom& g, int smem_optin, int sm_count,
   p.WT = (g.wo + p.bw - 1) / p.bw;
   p.HT = p.mpack ? (g.ho + 1) / 2 : (g.ho + p.bh - 1) / p.bh;
   p.GT = (g.G + p.bg - 1) / p.bg;
-  long long pb = (long long)p.WT * p.HT * p.GT;
-  if (pb > 0x3fffffffLL) return false;
-  p.PB = (int)pb;
+  if ((long long)p.WT * p.HT * p.GT > 0x3fffffffLL) return false;
+  p.pb0 = 0;
+  if (gt_cnt >= 0) {
+    // this launch covers group tiles [gt_lo, gt_lo + gt_cnt) only
+    if (gt_lo < 0 || gt_cnt < 1 || gt_lo + gt_cnt > p.GT) return false;
+    p.pb0 = gt_lo * p.WT * p.HT;
+    p.GT = gt_cnt;
+  }
+  p.PB = p.WT * p.HT * p.GT;
   p.K1 = g.K + 1;
   // N tile = tpn tap slots of cb channels.  Few input channels would make a
   // narrow tile (N = 64 or 128 re-reads the 128 rows of dtil from shared memory
@@ -744,12 +776,22 @@ dk_status tc_mix_split(const Geom& g, const float* delta, const float* dmix, flo
   return DK_OK;
 }
 
-dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* dt_lo, const float* xb_hi,
-                   const float* xb_lo, int xbar_rows, float scale, float* dW, int* status_word,
-                   cudaStream_t st) {
+bool tc_wgrad_group_tiles(const dk_ctx* ctx, const Geom& g, int* GT, int* bg, long long* rounds) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   WgPlan w;
-  if (!plan_wgrad(ctx->opt, g, ts->smem_optin, ctx->sm_count, &w)) return DK_ERR_UNSUPPORTED;
+  if (!ts || !plan_wgrad(ctx->opt, g, ts->smem_optin, ctx->sm_count, &w)) return false;
+  const int units = w.pair ? ctx->sm_count / 2 : ctx->sm_count;
+  *GT = w.prm.GT; *bg = w.prm.bg;
+  *rounds = (w.prm.nitems + units - 1) / units;
+  return true;
+}
+
+dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* dt_lo, const float* xb_hi,
+                   const float* xb_lo, int xbar_rows, float scale, float* dW, int* status_word,
+                   cudaStream_t st, int gt_lo, int gt_cnt) {
+  TcState* ts = static_cast<TcState*>(ctx->tc_state);
+  WgPlan w;
+  if (!plan_wgrad(ctx->opt, g, ts->smem_optin, ctx->sm_count, &w, gt_lo, gt_cnt)) return DK_ERR_UNSUPPORTED;
   w.prm.withhold = ctx->opt.v[DK_OPT_TEST_WITHHOLD];
   ctx->opt.v[DK_OPT_TEST_WITHHOLD] = -1;      // the hook serves one launch
   w.prm.scale = scale;

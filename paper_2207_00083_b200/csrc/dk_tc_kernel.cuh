@@ -55,9 +55,14 @@ struct TcParams {
   int bw, bh, bg;              // box shape of the P pixels (bw and bh are powers of two)
   int log2_bw, log2_S;         // log2 of bw and of S = bw*bh
   int WT, HT, GT, MT;          // tiles along width, height, groups, cout
+  int gt0;                     // first group tile of this launch (a call may be served by several launches, each
+                               // covering GT group tiles from gt0 on)
   int ntiles;
   int KB, CB;                  // k-blocks in total and per filter tap
-  int chunk;                   // k-blocks accumulated in TMEM before promotion
+  int chunk;                   // most k-blocks accumulated in TMEM before promotion
+  const unsigned char* chunk_tab;   // nullable, G <= kChunkTabMax entries: per virtual batch, the k-blocks (of 32
+                               // contraction elements) its coefficients allow; copied to shared memory at start
+  int chunk_mul;               // k-blocks per 32 contraction elements
   int ksplit, kb_per_split;    // contraction slices per tile (slices add into `out` with atomics)
   int kw, pad, stride;
   int nstages;
@@ -459,6 +464,24 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
 // `alive` = false: this warp's wait expired; the status is raised before the
 // count so that whoever decides sees it.
 // ---------------------------------------------------------------------------
+// k-blocks a tile accumulates in tensor memory between promotions: the accumulator truncates when it adds, and
+// the decoder multiplies that error by the amplification of the tile's coefficient sets, so ill-conditioned
+// virtual batches take shorter chunks (table from the host, see upload_coefficients).  `tab` = the table in shared
+// memory; t = tile index.
+constexpr int kChunkTabMax = 1024;
+__device__ __forceinline__ void load_chunk_tab(const TcParams& p, unsigned char* tab) {
+  if (p.chunk_tab == nullptr) return;
+  for (int i = threadIdx.x; i < p.G && i < kChunkTabMax; i += blockDim.x) tab[i] = __ldg(p.chunk_tab + i);
+}
+__device__ __forceinline__ int tile_chunk(const TcParams& p, const unsigned char* tab, int t) {
+  if (p.chunk_tab == nullptr) return p.chunk;
+  const int gt = p.gt0 + (t / p.MT) / (p.WT * p.HT);
+  const int g0 = gt * p.bg, g1 = min(p.G, g0 + p.bg);
+  int c = p.chunk;
+  for (int g = g0; g < g1; ++g) c = min(c, (int)tab[g] * p.chunk_mul);
+  return max(c, 1);
+}
+
 template <int MODE, int K>
 __device__ __forceinline__ void tail_finalize(const TcParams& p, int tid, bool alive, volatile int* last_flag) {
   if (MODE != MODE_DECODE || p.verdict == nullptr) return;
@@ -492,6 +515,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
   constexpr int STAGE_BYTES = 2 * (A_BYTES + B_BYTES);
   static_assert(BN % 16 == 0 && BN <= 256 && PH % 8 == 0, "illegal tile");
   extern __shared__ unsigned char smem_raw[];
+  __shared__ unsigned char s_chunk[kChunkTabMax];      // chunk lengths per virtual batch (see tile_chunk)
+  load_chunk_tab(p, s_chunk);
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                          ~static_cast<uintptr_t>(1023));
   unsigned char* ctrl = smem + (size_t)p.nstages * STAGE_BYTES;
@@ -545,7 +570,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
         int nt = t / p.MT;
         const int wt = nt % p.WT; nt /= p.WT;
         const int ht = nt % p.HT;
-        const int gt = nt / p.HT;
+        const int gt = p.gt0 + nt / p.HT;
         const int x0 = wt * p.bw * p.stride - p.pad, y0 = ht * p.bh * p.hmul * p.stride - p.pad;     // input position of tap (0,0)
         const int g0 = gt * p.bg, m0 = mt * BM;
         for (int kb = kb_lo; kb < kb_hi; ++kb) {
@@ -590,13 +615,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
       for (int w = blockIdx.x; alive && w < nwork; w += gridDim.x) {
         const int ks = w % p.ksplit;
         const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
-        const int nchunks = (kb_hi - kb_lo + p.chunk - 1) / p.chunk;
+        const int chunk = tile_chunk(p, s_chunk, w / p.ksplit);
+        const int nchunks = (kb_hi - kb_lo + chunk - 1) / chunk;
         for (int ci = 0; alive && ci < nchunks; ++ci, ++acc_it) {
           const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
           if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag, p.spin_cap)) { alive = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * 256u;
-          const int kb_beg = kb_lo + ci * p.chunk, kb_end = min(kb_hi, kb_beg + p.chunk);
+          const int kb_beg = kb_lo + ci * chunk, kb_end = min(kb_hi, kb_beg + chunk);
           for (int kb = kb_beg; kb < kb_end; ++kb) {
             if (!mbar_wait(full_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
             tc_fence_after();
@@ -631,12 +657,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
     for (int w = blockIdx.x; alive && w < nwork; w += gridDim.x) {
       const int t = w / p.ksplit, ks = w - t * p.ksplit;
       const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
-      const int nchunks = (kb_hi - kb_lo + p.chunk - 1) / p.chunk;
+      const int chunk = tile_chunk(p, s_chunk, t);
+      const int nchunks = (kb_hi - kb_lo + chunk - 1) / chunk;
       const int mt = t % p.MT;
       int nt = t / p.MT;
       const int wt = nt % p.WT; nt /= p.WT;
       const int ht = nt % p.HT;
-      const int gt = nt / p.HT;
+      const int gt = p.gt0 + nt / p.HT;
       // (two-row tiles: lanes 64-127 hold the same output channels for the image row below)
       const int co = p.hmul == 2 ? (quad & 1) * 32 + lane : mt * BM + quad * 32 + lane;
       const int ht_e = p.hmul == 2 ? 2 * ht + (quad >> 1) : ht;
@@ -648,18 +675,19 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
         if (!mbar_wait(tfull_bar + buf, aphase, abort_flag, p.spin_cap)) { alive = false; break; }
         tc_fence_after();
         const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * PH);
+        constexpr int EB = 2;      // encodings per round trip to tensor memory
 #pragma unroll
-        for (int e0 = 0; e0 < E; e0 += 2) {
-          float tmp[2][PH];
+        for (int e0 = 0; e0 < E; e0 += EB) {
+          float tmp[EB][PH];
 #pragma unroll
-          for (int de = 0; de < 2; ++de)
+          for (int de = 0; de < EB; ++de)
             if (e0 + de < E) {
 #pragma unroll
               for (int c = 0; c < PH; c += 8) tc_ld8(tbase + (uint32_t)((e0 + de) * P + c), &tmp[de][c]);
             }
           tc_wait_ld();
 #pragma unroll
-          for (int de = 0; de < 2; ++de)
+          for (int de = 0; de < EB; ++de)
             if (e0 + de < E) {
 #pragma unroll
               for (int j = 0; j < PH; ++j)

@@ -98,6 +98,8 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
   static_assert(E % 2 == 0, "the pair kernel splits the encodings in two halves");
   static_assert(BN % 16 == 0 && BN <= 256 && PH % 8 == 0, "illegal tile");
   extern __shared__ unsigned char smem_raw[];
+  __shared__ unsigned char s_chunk[kChunkTabMax];      // chunk lengths per virtual batch (see tile_chunk)
+  load_chunk_tab(p, s_chunk);
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                          ~static_cast<uintptr_t>(1023));
   unsigned char* ctrl = smem + (size_t)p.nstages * STAGE_BYTES;
@@ -147,7 +149,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
       int nt = t / p.MT;
       const int wt = nt % p.WT; nt /= p.WT;
       const int ht = nt % p.HT;
-      const int gt = nt / p.HT;
+      const int gt = p.gt0 + nt / p.HT;
       const int x0 = wt * p.bw * p.stride - p.pad, y0 = ht * p.bh * p.stride - p.pad, g0 = gt * p.bg;
       const int m0 = mt * BM2 + (int)rank * BM;
       for (int kb = kb_lo; kb < kb_hi; ++kb) {
@@ -191,13 +193,14 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
       for (int w = pair; alive && w < nwork; w += npairs) {
         const int ks = w % p.ksplit;
         const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
-        const int nchunks = (kb_hi - kb_lo + p.chunk - 1) / p.chunk;
+        const int chunk = tile_chunk(p, s_chunk, w / p.ksplit);
+        const int nchunks = (kb_hi - kb_lo + chunk - 1) / chunk;
         for (int ci = 0; alive && ci < nchunks; ++ci, ++acc_it) {
           const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
           if (!mbar_wait(tempty_bar + buf, aphase ^ 1u, abort_flag, p.spin_cap)) { alive = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * 256u;
-          const int kb_beg = kb_lo + ci * p.chunk, kb_end = min(kb_hi, kb_beg + p.chunk);
+          const int kb_beg = kb_lo + ci * chunk, kb_end = min(kb_hi, kb_beg + chunk);
           for (int kb = kb_beg; kb < kb_end; ++kb) {
             if (!mbar_wait(full_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
             tc_fence_after();
@@ -232,12 +235,13 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     for (int w = pair; alive && w < nwork; w += npairs) {
       const int t = w / p.ksplit, ks = w - t * p.ksplit;
       const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
-      const int nchunks = (kb_hi - kb_lo + p.chunk - 1) / p.chunk;
+      const int chunk = tile_chunk(p, s_chunk, t);
+      const int nchunks = (kb_hi - kb_lo + chunk - 1) / chunk;
       const int mt = t % p.MT;
       int nt = t / p.MT;
       const int wt = nt % p.WT; nt /= p.WT;
       const int ht = nt % p.HT;
-      const int gt = nt / p.HT;
+      const int gt = p.gt0 + nt / p.HT;
       const int co = mt * BM2 + (int)rank * BM + quad * 32 + lane;
       const bool co_ok = co < p.cout;
 
@@ -246,21 +250,24 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         if (!mbar_wait(tfull_bar + buf, aphase, abort_flag, p.spin_cap)) { alive = false; break; }
         tc_fence_after();
         const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * PH);
+        constexpr int EB = 2;      // encodings per round trip to tensor memory
 #pragma unroll
-        for (int e0 = 0; e0 < E; e0 += 2) {
-          float tmp[2][PH];
+        for (int e0 = 0; e0 < E; e0 += EB) {
+          float tmp[EB][PH];
 #pragma unroll
-          for (int de = 0; de < 2; ++de) {
+          for (int de = 0; de < EB; ++de)
+            if (e0 + de < E) {
 #pragma unroll
-            for (int c = 0; c < PH; c += 8) tc_ld8(tbase + (uint32_t)((e0 + de) * P + c), &tmp[de][c]);
-          }
+              for (int c = 0; c < PH; c += 8) tc_ld8(tbase + (uint32_t)((e0 + de) * P + c), &tmp[de][c]);
+            }
           tc_wait_ld();
 #pragma unroll
-          for (int de = 0; de < 2; ++de) {
+          for (int de = 0; de < EB; ++de)
+            if (e0 + de < E) {
 #pragma unroll
-            for (int j = 0; j < PH; ++j)
-              acc[e0 + de][j] = (ci == 0) ? tmp[de][j] : acc[e0 + de][j] + tmp[de][j];
-          }
+              for (int j = 0; j < PH; ++j)
+                acc[e0 + de][j] = (ci == 0) ? tmp[de][j] : acc[e0 + de][j] + tmp[de][j];
+            }
         }
         tc_fence_before();
         __syncwarp();

@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(256) fwd_prepass_kernel(const FwdPrepass a) {
     return;
   }
   if ((int)blockIdx.x < enc_blocks) {
-    if (blockIdx.x == 0) {
+    if (blockIdx.x == 0 && a.count != nullptr) {
       for (int i = threadIdx.x; i < a.nstats; i += blockDim.x) a.stats[i] = 0.f;
       if (threadIdx.x == 0) { a.count[0] = 0u; a.count[1] = 0u; }
     }
@@ -202,7 +202,11 @@ int job_blocks(long long n4, long long cap) {
 
 dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const float* enc, float* full,
                          float* xb_hi, float* xb_lo, const float* W, float* w_hi, float* w_lo,
-                         const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st, int raw) {
+                         const VerifyScratch& vs, float* ybar_clear, int sm_count, cudaStream_t st, int raw,
+                         int g_lo, int g_cnt, bool beside) {
+  // groups [g_lo, g_lo + g_cnt) only (g_cnt < 0: all); the launch for g_lo = 0 also splits W and clears
+  const bool first = g_lo == 0;
+  if (g_cnt < 0) g_cnt = g.G - g_lo;
   const long long wn = (long long)g.cout * g.kc;
   if (g.n_in % 4 || wn % 4) return DK_ERR_SHAPE;
   if (raw && full == nullptr) return DK_ERR_INVALID_ARG;
@@ -211,21 +215,29 @@ dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const fl
   const bool strided_1x1 = g.kind == DK_CONV2D && g.kh == 1 && g.kw == 1 && g.pad == 0 && g.stride > 1;
   a.pix4 = g.cin / 4; a.width = g.w; a.step = strided_1x1 ? g.stride : 1;
   const long long yn = (long long)g.G * g.E * g.n_out;
+  if (!first) ybar_clear = nullptr;
   a.zero = reinterpret_cast<float4*>(ybar_clear);
   a.z4 = ybar_clear ? (yn + 3) / 4 : 0;           // the y_bar region is padded to 1 KiB
   a.z_blocks = ybar_clear ? job_blocks(a.z4, (long long)sm_count * 4) : 0;
-  a.x = x; a.r = r; a.enc = enc; a.full = full; a.xb_hi = xb_hi; a.xb_lo = xb_lo;
-  a.n_in = g.n_in; a.G = g.G;
-  const long long cap = (long long)sm_count * 16;
-  a.per_g = job_blocks(g.n_in / 4, (cap + g.G - 1) / g.G);
+  const size_t eoff = (size_t)g_lo * g.E * g.n_in;
+  a.x = x + (size_t)g_lo * g.K * g.n_in; a.r = r + (size_t)g_lo * g.n_in;
+  a.enc = enc + (size_t)g_lo * g.E * (g.K + 1);
+  a.full = full ? full + eoff : nullptr; a.xb_hi = xb_hi ? xb_hi + eoff : nullptr; a.xb_lo = xb_lo + eoff;
+  a.n_in = g.n_in; a.G = g_cnt;
+  // beside a GEMM kernel (one persistent CTA of 32K registers per SM) only a few small blocks fit on an SM, and a
+  // larger grid would keep the GEMM's CTAs off the SMs until this kernel has ended: blocks of 128 threads, two
+  // per SM up to K = 4 (at most 80 registers a thread), one beyond (at most 165)
+  const int threads = beside ? 128 : 256;
+  const long long cap = beside ? (long long)sm_count * (g.K <= 4 ? 2 : 1) : (long long)sm_count * 16;
+  a.per_g = job_blocks(g.n_in / 4, (cap + g_cnt - 1) / g_cnt);
   a.W = W; a.w_hi = w_hi; a.w_lo = w_lo; a.w4 = wn / 4;
   a.wpack = g.mpack; a.cout = g.cout; a.cin4 = g.cin / 4; a.kh = g.kh; a.kw = g.kw;
-  a.w_blocks = job_blocks(g.mpack ? (long long)128 * (g.kh + 1) * g.kw * a.cin4 : a.w4, cap);
-  a.stats = vs.sumsq; a.nstats = g.G * (g.E + 1); a.count = vs.count;
+  a.w_blocks = first ? job_blocks(g.mpack ? (long long)128 * (g.kh + 1) * g.kw * a.cin4 : a.w4, cap) : 0;
+  a.stats = vs.sumsq; a.nstats = first ? g.G * (g.E + 1) : 0; a.count = first ? vs.count : nullptr;
   const long long blocks = (long long)a.G * a.per_g + a.w_blocks + a.z_blocks;
   if (blocks > 0x7fffffffLL) return DK_ERR_SHAPE;
 #define DK_PRE_CASE(KK) \
-  case KK: fwd_prepass_kernel<KK><<<(unsigned)blocks, 256, 0, st>>>(a); break;
+  case KK: fwd_prepass_kernel<KK><<<(unsigned)blocks, threads, 0, st>>>(a); break;
   switch (g.K) {
     DK_PRE_CASE(1) DK_PRE_CASE(2) DK_PRE_CASE(3) DK_PRE_CASE(4)
     DK_PRE_CASE(5) DK_PRE_CASE(6) DK_PRE_CASE(7) DK_PRE_CASE(8)
@@ -238,15 +250,32 @@ dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const fl
 
 dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix, float* dt_hi, float* dt_lo,
                            const float* xbar, long long xbar_elems, float* xb_hi, float* xb_lo, float* dW,
-                           int sm_count, cudaStream_t st, int raw, int xbar_rows) {
+                           int sm_count, cudaStream_t st, int raw, int xbar_rows, int g_lo, int g_cnt, bool beside) {
   const long long dwn = (long long)g.cout * g.kc;
   if (g.n_out % 4 || xbar_elems % 4 || dwn % 4 || g.n_in % 4) return DK_ERR_SHAPE;
+  // groups [g_lo, g_lo + g_cnt) only (g_cnt < 0: all); the launch for g_lo = 0 also clears dW
+  if (g_cnt < 0) g_cnt = g.G - g_lo;
+  if (g_lo > 0 || g_cnt < g.G) {
+    const int rows = xbar_rows > 0 ? xbar_rows : g.K + 1;
+    const long long xoff = (long long)g_lo * rows * g.n_in;
+    long long xe = (long long)g_cnt * rows * g.n_in;
+    if (xoff + xe > xbar_elems) xe = xbar_elems - xoff;
+    const long long doff = (long long)g_lo * (g.K + 1) * g.n_out;
+    delta += (long long)g_lo * g.K * g.n_out; dmix += (long long)g_lo * (g.K + 1) * g.K;
+    dt_hi += doff; dt_lo += doff;
+    xbar += xoff; if (xb_hi) xb_hi += xoff;
+    xb_lo += xoff;
+    xbar_elems = xe;
+    if (g_lo > 0) dW = nullptr;
+  }
   WgPrepass a;
   a.raw = raw; a.row4 = g.n_in / 4; a.period = xbar_rows > 0 ? xbar_rows : 1; a.used = xbar_rows > 0 ? g.K + 1 : 1;
   a.delta = delta; a.dmix = dmix; a.dt_hi = dt_hi; a.dt_lo = dt_lo;
-  a.n_out = g.n_out; a.G = g.G;
-  const long long cap = (long long)sm_count * 16;
-  a.per_g = job_blocks(g.n_out / 4, (cap + g.G - 1) / g.G);
+  a.n_out = g.n_out; a.G = g_cnt;
+  // (beside a GEMM kernel: few small blocks, see tc_fwd_prepass; the cap is shared by the two jobs)
+  const int threads = beside ? 128 : 256;
+  const long long cap = beside ? (long long)sm_count * (g.K <= 4 ? 2 : 1) / 2 + 1 : (long long)sm_count * 16;
+  a.per_g = job_blocks(g.n_out / 4, (cap + g_cnt - 1) / g_cnt);
   a.xbar = xbar; a.xb_hi = xb_hi; a.xb_lo = xb_lo; a.x4 = xbar_elems / 4;
   a.x_blocks = job_blocks(a.x4, cap);
   a.dW = reinterpret_cast<float4*>(dW); a.dw4 = dW ? dwn / 4 : 0;
@@ -254,7 +283,7 @@ dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix,
   const long long blocks = (long long)a.G * a.per_g + a.x_blocks + a.z_blocks;
   if (blocks > 0x7fffffffLL) return DK_ERR_SHAPE;
 #define DK_PRE_CASE(KK) \
-  case KK: wgrad_prepass_kernel<KK><<<(unsigned)blocks, 256, 0, st>>>(a); break;
+  case KK: wgrad_prepass_kernel<KK><<<(unsigned)blocks, threads, 0, st>>>(a); break;
   switch (g.K) {
     DK_PRE_CASE(1) DK_PRE_CASE(2) DK_PRE_CASE(3) DK_PRE_CASE(4)
     DK_PRE_CASE(5) DK_PRE_CASE(6) DK_PRE_CASE(7) DK_PRE_CASE(8)

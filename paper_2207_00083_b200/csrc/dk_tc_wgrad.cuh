@@ -36,7 +36,8 @@ constexpr int kWgBox = kWgPix * 128;       // bytes of one [32 pixels][32 channe
 struct WgTcParams {
   int bw, bh, bg;              // box shape of the 32 pixels: columns, rows, groups
   int WT, HT, GT;              // pixel blocks along width, height, groups
-  int PB;                      // WT*HT*GT
+  int PB;                      // pixel blocks of this launch
+  int pb0;                     // its first pixel block (a call may be served by several launches over ranges of groups)
   int K1;                      // encodings used (K+1)
   int MT, NB, taps;            // cout tiles, channel blocks, filter taps
   int cb, tpn, TG;             // channels per tap slot, tap slots per N tile (BN = cb*tpn), tap groups
@@ -176,7 +177,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
           }
         }
         for (int pb = pb_lo; alive && pb < pb_hi; ++pb) {
-          int r = pb;
+          int r = p.pb0 + pb;
           const int wt = r % p.WT; r /= p.WT;
           const int ht = r % p.HT;
           const int gt = r / p.HT;
@@ -284,7 +285,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
         if (!mbar_wait(tfull_bar + buf, aphase, abort_flag, p.spin_cap)) { alive = false; break; }
         tc_fence_after();
         const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * NH);
-        constexpr int TS = NH > 96 ? 16 : 32;      // columns per round trip (fewer when the sums fill the registers)
+        // columns per round trip to tensor memory: as many as the registers hold beside the NH running sums (a
+        // chunk is promoted in NH / TS round trips, and with short chunks their latency is what the tensor
+        // pipe ends up waiting for)
+        constexpr int TS = NH > 96 ? 16 : NH;      // (128 sums leave room for 16)
 #pragma unroll
         for (int c0 = 0; c0 < NH; c0 += TS) {
           float tmp[TS];
