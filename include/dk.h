@@ -158,8 +158,12 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  *                     has at most 64 elements, else the tensor-core kernels through
  *                     patch rows; 2 always the latter; 0 the generic fp32 kernels.
  *   DK_OPT_FIELD_PATH contraction kernels of the finite-field calls: 0 (default)
- *                     tensor cores (tcgen05 where the shape allows, else mma.sync),
- *                     1 the 64-bit integer-ALU kernels, 2 mma.sync only.
+ *                     tensor cores (tcgen05 with operands fetched by TMA from digit
+ *                     planes where the shape allows: channels-last, stride 1,
+ *                     cin % 64 == 0; else tcgen05 with operands split in registers;
+ *                     else mma.sync), 1 the 64-bit integer-ALU kernels, 2 mma.sync
+ *                     only, 3 as 0 without the TMA-fed kernels (1-3 are
+ *                     cross-checks of the default).
  *   DK_OPT_SPIN_LIMIT polls after which a device-side wait gives up and the call
  *                     reports DK_ERR_TIMEOUT (default 2^22, 2^10..2^26).
  *   DK_OPT_XBAR_HI    how the tensor-core kernels get the leading TF32 term of an

@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "dk_internal.h"
+#include "dk_tc_kernel.cuh"
 
 namespace dk {
 namespace {
@@ -330,6 +331,7 @@ struct DecodeParams {
   long long ch_div;  // channel of position e = (e / ch_div) % cout
   int cout;
   double inv_scale;  // 2^-l
+  int lbits;         // l
   Modulus md;
 };
 
@@ -400,9 +402,11 @@ __global__ void __launch_bounds__(256) field_decode_verify_kernel(DecodeParams p
           float yv[VEC];
 #pragma unroll
           for (int v = 0; v < VEC; ++v) {
-            const double t = (double)cq[v] * p.inv_scale;
-            const double f = floor(t);
-            yv[v] = (float)(((t - f < 0.5) ? f : f + 1.0) * p.inv_scale);
+            // Round(c * 2^-l) = floor(c * 2^-l + 1/2) = (c + 2^(l-1)) >> l in integers (arithmetic shift = floor);
+            // |c| < 2^29 keeps the sum in range and the quotient, below 2^24 for l >= 6, exact in fp32 for any l
+            // once scaled by the power of two (a quotient of more than 24 bits rounds as the product would)
+            const int q = p.lbits > 0 ? (cq[v] + (1 << (p.lbits - 1))) >> p.lbits : cq[v];
+            yv[v] = __int2float_rn(q) * (float)p.inv_scale;      // (2^-l is a power of two: one rounding, as in fp64)
           }
           if (VEC == 4) *reinterpret_cast<float4*>(p.y + o) = make_float4(yv[0], yv[1], yv[2], yv[3 % VEC]);
           else p.y[o] = yv[0];
@@ -1117,6 +1121,407 @@ __global__ void __launch_bounds__(tcf::kThreads, 1) field_fwd_tc_kernel(FwdParam
   }
 }
 
+// ---------------------------------------------------------------------------
+// The forward contraction with operands fetched by TMA.  Both operands are digit planes in global memory
+// (W_q as [digit][cout][k], written by field_w_planes_kernel; x_bar as [digit][sample][h][w][cin], written by
+// field_x_planes_kernel), so a pipeline stage is two bulk tensor copies: 128 rows of W and, for filter tap
+// (u,v), the tile's box of 64 output pixels shifted by (u-pad, v-pad), all four digits of each; positions
+// outside the image are zero-filled by the TMA unit.  One producer thread, one MMA thread, eight warps that
+// read and fold the class sums.  KT = contraction elements per k-tile = bytes per shared-memory row (one
+// swizzle span): 128 when cin % 128 == 0 (two stages), else 64 (cin % 64 == 0, four stages).  Stride 1 only.
+// The products, the merged N = 256 instruction and the folds are those of field_fwd_tc_kernel above.
+// ---------------------------------------------------------------------------
+namespace ftm {
+constexpr int TM = 128, TN = 64;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;      // producer warp, MMA warp, epilogue warps
+constexpr int kFoldK = 8192;                       // contraction elements between folds: 4 pairs * 255^2 * 8192 < 2^31
+
+struct Params {
+  int bw, bh, bs;              // the 64 columns of a tile: a box of bw x bh output pixels of bs samples (powers of two)
+  int WT, HT;                  // tiles along width and height (sample tile = blockIdx.x / (WT*HT))
+  int cblocks;                 // cin / KT
+  int kw, pad;
+  int ktiles, tiles_per_split; // k-tiles in all and per contraction slice (blockIdx.z)
+  int cout, ho, wo, nsamples;
+  long long n_out, ys_c, ys_h, ys_w;
+  u32* y;
+  u64* split_acc;              // nullable: slices add their residues here
+  Modulus md;
+  u32 pow32;
+  int* status;
+  unsigned spin_cap;
+  int withhold;                // test hook: the producer arms this k-tile's stage, copies nothing and stops (-1 = off)
+};
+}  // namespace ftm
+
+// Activations as four digit planes, [digit][sample][h][w][c] bytes (the element order of the source).  The
+// source holds `rows` samples per group of which the first `used` are copied (rows = used: all of them):
+// n = elements written per plane = groups * used * row_elems; row_elems % 16 == 0.
+__global__ void __launch_bounds__(256) field_x_planes_kernel(const u32* __restrict__ x, long long n, uint8_t* __restrict__ planes,
+                                                            long long row_elems, int rows, int used) {
+  const long long chunks = n / 16;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < chunks; i += stride) {
+    long long src = i * 16;
+    if (rows != used) {
+      const long long r = src / row_elems;                 // destination row = group * used + j
+      src += (r / used) * (long long)(rows - used) * row_elems;
+    }
+    u32 pl[4][4];
+#pragma unroll
+    for (int gq = 0; gq < 4; ++gq)
+      digit_planes(__ldg(reinterpret_cast<const uint4*>(x + src) + gq), pl[gq]);
+#pragma unroll
+    for (int dg = 0; dg < 4; ++dg)
+      *reinterpret_cast<uint4*>(planes + (long long)dg * n + i * 16) = make_uint4(pl[0][dg], pl[1][dg], pl[2][dg], pl[3][dg]);
+  }
+}
+
+template <int KT>
+__global__ void __launch_bounds__(ftm::kThreads, 1)
+field_fwd_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+                     const ftm::Params p) {
+  using namespace ftm;
+  constexpr int A_PLANE = TM * KT, B_PLANE = TN * KT, STAGE = 4 * (A_PLANE + B_PLANE);
+  constexpr int NST = KT == 128 ? 2 : 4;
+  constexpr int kFoldTiles = kFoldK / KT;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t full_bar[NST];       // a stage's two copies have landed (transaction bytes)
+  __shared__ uint64_t empty_bar[NST];      // the products that read a stage have completed (one commit)
+  __shared__ uint64_t tfull_bar;           // every product up to a fold point has completed (one commit)
+  __shared__ uint64_t tempty_bar;          // the class sums have been read (one arrival per epilogue warp)
+  __shared__ uint32_t tmem_slot[2];        // [0] TMEM base address, [1] abort flag
+  uint8_t* smem = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int m0 = blockIdx.y * TM;
+  const int wt = blockIdx.x % p.WT, ht = (blockIdx.x / p.WT) % p.HT, stl = blockIdx.x / (p.WT * p.HT);
+  const int x0 = wt * p.bw, y0 = ht * p.bh, s0 = stl * p.bs;
+  const int kt0 = blockIdx.z * p.tiles_per_split;
+  const int ntiles = min(p.tiles_per_split, p.ktiles - kt0);
+  const int nfolds = (ntiles + kFoldTiles - 1) / kFoldTiles;
+
+  if (t == 0) {
+    for (int s = 0; s < NST; ++s) { tc::mbar_init(full_bar + s, 1); tc::mbar_init(empty_bar + s, 1); }
+    tc::mbar_init(&tfull_bar, 1);
+    tc::mbar_init(&tempty_bar, kEpiWarps);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc::smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = tmem_slot[0];
+
+  if (warp == 0) {
+    // ---------------- TMA producer: one thread ----------------
+    if (lane == 0) {
+      for (int kt = 0; kt < ntiles; ++kt) {
+        const int stage = kt % NST;
+        if (kt >= NST && !tc::mbar_wait(empty_bar + stage, (uint32_t)((kt / NST - 1) & 1), abort_flag, p.spin_cap)) break;
+        tc::mbar_expect_tx(full_bar + stage, (uint32_t)STAGE);
+        if (kt == p.withhold) break;      // test hook: armed, nothing copied
+        const int ktg = kt0 + kt;
+        const int tap = ktg / p.cblocks, c0 = (ktg - tap * p.cblocks) * KT;
+        const int u = tap / p.kw, v = tap - u * p.kw;
+        uint8_t* st = smem + (size_t)stage * STAGE;
+        tc::tma_load_3d(st, &map_w, full_bar + stage, ktg * KT, m0, 0);
+        tc::tma_load_5d(st + 4 * A_PLANE, &map_x, full_bar + stage, c0, x0 + v - p.pad, y0 + u - p.pad, s0, 0);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: one thread ----------------
+    if (lane == 0) {
+      // S32 accumulator, unsigned 8-bit A and B, both K-major, M = 128; W's digit a against all four digit planes
+      // of x_bar (adjacent in shared memory) is one instruction with N = 256 whose columns are classes a .. a+3
+      auto idesc_n = [](int n) {
+        return (2u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+      };
+      bool fresh = true;               // no product since the last fold
+      int fold = 0;
+      for (int kt = 0; kt < ntiles; ++kt) {
+        const int stage = kt % NST;
+        if (fresh && fold > 0) {
+          // the class sums of the previous fold must have been read before they are overwritten
+          if (!tc::mbar_wait(&tempty_bar, (uint32_t)((fold - 1) & 1), abort_flag, p.spin_cap)) break;
+          tc::tc_fence_after();
+        }
+        if (!tc::mbar_wait(full_bar + stage, (uint32_t)((kt / NST) & 1), abort_flag, p.spin_cap)) break;
+        tc::tc_fence_after();
+        const uint32_t sa = tc::smem_u32(smem + (size_t)stage * STAGE), sb = sa + 4 * A_PLANE;
+        const uint64_t bdesc = tc::make_desc<KT>(sb);
+#pragma unroll
+        for (int ks = 0; ks < KT / 32; ++ks) {
+          const uint64_t adv = (uint64_t)(ks * 2);       // 32 bytes per k-step, in 16-byte units
+#pragma unroll
+          for (int da = 0; da < 4; ++da) {
+            const uint64_t adesc = tc::make_desc<KT>(sa + da * A_PLANE) + adv;
+            const uint32_t d = tmem_base + (uint32_t)(da * TN);
+            if (fresh && ks == 0 && da > 0) {
+              // classes da .. da+2 have a product already, class da+3 has none
+              tcf::mma_i8(d, adesc, bdesc + adv, idesc_n(3 * TN), 1u);
+              tcf::mma_i8(d + 3 * TN, adesc, tc::make_desc<KT>(sb + 3 * B_PLANE) + adv, idesc_n(TN), 0u);
+            } else {
+              tcf::mma_i8(d, adesc, bdesc + adv, idesc_n(4 * TN), (fresh && ks == 0) ? 0u : 1u);
+            }
+          }
+        }
+        fresh = false;
+        tc::tc_commit(empty_bar + stage);
+        if (kt + 1 == ntiles || ((kt + 1) % kFoldTiles) == 0) {
+          tc::tc_commit(&tfull_bar);      // (a commit covers all earlier products of this thread)
+          fresh = true;
+          ++fold;
+        }
+      }
+    }
+  } else {
+    // ---------------- epilogue: eight warps read the class sums at every fold point and fold them ----------------
+    // this thread: TMEM lane (output channel) 32*q + lane, columns 32*h .. 32*h+31
+    const int q = warp & 3, h = (warp - 2) >> 2;
+    const int m = m0 + q * 32 + lane;
+    bool alive = true;
+    for (int fold = 0; alive && fold < nfolds; ++fold) {
+      if (!tc::mbar_wait(&tfull_bar, (uint32_t)(fold & 1), abort_flag, p.spin_cap)) { alive = false; break; }
+      tc::tc_fence_after();
+#pragma unroll 1
+      for (int cg = 0; cg < 4; ++cg) {
+        int cls[7][8];
+#pragma unroll
+        for (int c = 0; c < 7; ++c)
+          tcf::ld8(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * TN + h * 32 + cg * 8), cls[c]);
+        tc::tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int col = h * 32 + cg * 8 + j;
+          const int dx = col % p.bw, dy = (col / p.bw) % p.bh, ds = col / (p.bw * p.bh);
+          const int ow = x0 + dx, oh = y0 + dy, smp = s0 + ds;
+          if (ow >= p.wo || oh >= p.ho || smp >= p.nsamples || m >= p.cout) continue;
+          const long long off = (long long)smp * p.n_out + (long long)oh * p.ys_h + (long long)ow * p.ys_w +
+                                (long long)m * p.ys_c;
+          const int cc[7] = {cls[0][j], cls[1][j], cls[2][j], cls[3][j], cls[4][j], cls[5][j], cls[6][j]};
+          if (p.split_acc != nullptr) atomicAdd(p.split_acc + off, (u64)fold_classes(0u, cc, p.md, p.pow32));
+          else p.y[off] = fold_classes(fold > 0 ? p.y[off] : 0u, cc, p.md, p.pow32);
+        }
+      }
+      tc::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&tempty_bar);
+    }
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // a bounded wait expired: report, and give copies and products still in flight time to retire
+    if (t == 0 && p.status != nullptr) atomicExch(p.status, (int)DK_ERR_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(16384);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc::tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------
+// The weight-gradient contraction on tcgen05 (Eq. 4-6 in F_p):
+//   dW[co][tap][ci] = sum_{sample, pixel} dtil[sample][pixel][co] * xbar[sample][pixel + tap - pad][ci]   (mod p)
+// M = 128 output channels, N = 64 input channels of one filter tap, the contraction runs over output pixels:
+// the contiguous dimension of neither operand, so both digit-plane tiles are MN-major ([pixel][channel] rows of
+// 128 and 64 bytes, one swizzle span each), fetched by TMA as boxes of 64 pixels (the box of x_bar shifted by the
+// tap; zero fill outside the image).  As in the forward kernels a digit of dtil against all four digit planes
+// of x_bar is one N = 256 instruction, and seven class sums live in tensor memory; they are folded every 8192
+// contraction elements and at the end, and the residues are added to the uint64 accumulators of dW.
+// Grid: (cout tile x channel block x tap, contraction slice).  Stride 1, channels-last, cin and cout % 16 == 0.
+// ---------------------------------------------------------------------------
+namespace fwg {
+constexpr int TM = 128, TN = 64, KP = 64, NST = 4;
+constexpr int A_PLANE = KP * TM, B_PLANE = KP * TN, STAGE = 4 * (A_PLANE + B_PLANE);      // 48 KB
+constexpr size_t kSmem = (size_t)NST * STAGE + 1024;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kFoldStages = 8192 / KP;
+
+struct Params {
+  int bw, bh, bs;              // the 64 pixels of a k-block: bw x bh output pixels of bs samples (powers of two)
+  int WT, HT;                  // pixel blocks along width and height (sample block = pb / (WT*HT))
+  long long PB;                // pixel blocks in all
+  int pb_per_split;
+  int MT, cblocks, kw, pad;
+  int cout, cin;
+  long long ws_o, ws_c, ws_u, ws_v;
+  u64* acc;
+  Modulus md;
+  u32 pow32;
+  int* status;
+  unsigned spin_cap;
+  int withhold;
+};
+
+// MN-major operand: rows of ROW bytes (one swizzle span) along the contraction, 8-row groups ROW*8 bytes apart,
+// further spans of ROW channels `span_bytes` apart
+template <int ROW>
+__device__ __forceinline__ uint64_t desc_mn(uint32_t smem_addr, uint32_t span_bytes) {
+  constexpr uint64_t layout = ROW == 128 ? 2ull : 4ull;
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+  d |= (uint64_t)((span_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((ROW * 8) >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= layout << 61;
+  return d;
+}
+}  // namespace fwg
+
+__global__ void __launch_bounds__(fwg::kThreads, 1)
+field_wgrad_tma_kernel(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_x,
+                       const fwg::Params p) {
+  using namespace fwg;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t full_bar[NST], empty_bar[NST], tfull_bar, tempty_bar;
+  __shared__ uint32_t tmem_slot[2];        // [0] TMEM base address, [1] abort flag
+  uint8_t* smem = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int item = blockIdx.x;
+  const int mt = item % p.MT, cb = (item / p.MT) % p.cblocks, tap = item / (p.MT * p.cblocks);
+  const int m0 = mt * TM, c0 = cb * TN;
+  const int u = tap / p.kw, v = tap - u * p.kw;
+  const long long pb0 = (long long)blockIdx.y * p.pb_per_split;
+  const int nst = (int)min((long long)p.pb_per_split, p.PB - pb0);
+  const int nfolds = (nst + kFoldStages - 1) / kFoldStages;
+
+  if (t == 0) {
+    for (int s = 0; s < NST; ++s) { tc::mbar_init(full_bar + s, 1); tc::mbar_init(empty_bar + s, 1); }
+    tc::mbar_init(&tfull_bar, 1);
+    tc::mbar_init(&tempty_bar, kEpiWarps);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc::smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = tmem_slot[0];
+
+  if (warp == 0) {
+    // ---------------- TMA producer: one thread ----------------
+    if (lane == 0) {
+      for (int k = 0; k < nst; ++k) {
+        const int stage = k % NST;
+        if (k >= NST && !tc::mbar_wait(empty_bar + stage, (uint32_t)((k / NST - 1) & 1), abort_flag, p.spin_cap)) break;
+        tc::mbar_expect_tx(full_bar + stage, (uint32_t)STAGE);
+        if (k == p.withhold) break;      // test hook: armed, nothing copied
+        const long long pb = pb0 + k;
+        const int wt = (int)(pb % p.WT), ht = (int)((pb / p.WT) % p.HT), sb = (int)(pb / ((long long)p.WT * p.HT));
+        const int x0 = wt * p.bw, y0 = ht * p.bh, s0 = sb * p.bs;
+        uint8_t* st = smem + (size_t)stage * STAGE;
+        tc::tma_load_5d(st, &map_d, full_bar + stage, m0, x0, y0, s0, 0);
+        tc::tma_load_5d(st + 4 * A_PLANE, &map_x, full_bar + stage, c0, x0 + v - p.pad, y0 + u - p.pad, s0, 0);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: one thread ----------------
+    if (lane == 0) {
+      // S32 accumulator, unsigned 8-bit A and B, both MN-major, M = 128
+      auto idesc_n = [](int n) {
+        return (2u << 4) | (0u << 7) | (0u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
+               ((uint32_t)(TM >> 4) << 24);
+      };
+      bool fresh = true;
+      int fold = 0;
+      for (int k = 0; k < nst; ++k) {
+        const int stage = k % NST;
+        if (fresh && fold > 0) {
+          if (!tc::mbar_wait(&tempty_bar, (uint32_t)((fold - 1) & 1), abort_flag, p.spin_cap)) break;
+          tc::tc_fence_after();
+        }
+        if (!tc::mbar_wait(full_bar + stage, (uint32_t)((k / NST) & 1), abort_flag, p.spin_cap)) break;
+        tc::tc_fence_after();
+        const uint32_t sa = tc::smem_u32(smem + (size_t)stage * STAGE), sb = sa + 4 * A_PLANE;
+#pragma unroll
+        for (int ks = 0; ks < KP / 32; ++ks) {
+          const uint64_t bdesc = desc_mn<TN>(sb + ks * 32 * TN, B_PLANE);
+#pragma unroll
+          for (int da = 0; da < 4; ++da) {
+            const uint64_t adesc = desc_mn<TM>(sa + da * A_PLANE + ks * 32 * TM, A_PLANE);
+            const uint32_t d = tmem_base + (uint32_t)(da * TN);
+            if (fresh && ks == 0 && da > 0) {
+              // classes da .. da+2 have a product already, class da+3 has none
+              tcf::mma_i8(d, adesc, bdesc, idesc_n(3 * TN), 1u);
+              tcf::mma_i8(d + 3 * TN, adesc, desc_mn<TN>(sb + 3 * B_PLANE + ks * 32 * TN, B_PLANE), idesc_n(TN), 0u);
+            } else {
+              tcf::mma_i8(d, adesc, bdesc, idesc_n(4 * TN), (fresh && ks == 0) ? 0u : 1u);
+            }
+          }
+        }
+        fresh = false;
+        tc::tc_commit(empty_bar + stage);
+        if (k + 1 == nst || ((k + 1) % kFoldStages) == 0) {
+          tc::tc_commit(&tfull_bar);
+          fresh = true;
+          ++fold;
+        }
+      }
+    }
+  } else {
+    // ---------------- epilogue: fold the class sums, add the residues to dW's accumulators ----------------
+    const int q = warp & 3, h = (warp - 2) >> 2;
+    const int co = m0 + q * 32 + lane;
+    bool alive = true;
+    for (int fold = 0; alive && fold < nfolds; ++fold) {
+      if (!tc::mbar_wait(&tfull_bar, (uint32_t)(fold & 1), abort_flag, p.spin_cap)) { alive = false; break; }
+      tc::tc_fence_after();
+#pragma unroll 1
+      for (int cg = 0; cg < 4; ++cg) {
+        int cls[7][8];
+#pragma unroll
+        for (int c = 0; c < 7; ++c)
+          tcf::ld8(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * TN + h * 32 + cg * 8), cls[c]);
+        tc::tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int ci = c0 + h * 32 + cg * 8 + j;
+          if (co >= p.cout || ci >= p.cin) continue;
+          const int cc[7] = {cls[0][j], cls[1][j], cls[2][j], cls[3][j], cls[4][j], cls[5][j], cls[6][j]};
+          atomicAdd(p.acc + (long long)co * p.ws_o + (long long)ci * p.ws_c + (long long)u * p.ws_u + (long long)v * p.ws_v,
+                    (u64)fold_classes(0u, cc, p.md, p.pow32));
+        }
+      }
+      tc::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&tempty_bar);
+    }
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (t == 0 && p.status != nullptr) atomicExch(p.status, (int)DK_ERR_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(16384);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc::tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // How many products of two residues may be added to one residue in a uint64.
 long long terms_per_reduction(u32 p) {
   const u64 pm = (u64)p - 1;
@@ -1153,12 +1558,89 @@ int field_fwd_slices(long long ctas, int ntiles, int sms) {
   return best;
 }
 
+// The TMA-fed forward kernel: digit planes of W_q and x_bar written first, then one CTA per (pixel tile,
+// 128 output channels, contraction slice).  DK_ERR_UNSUPPORTED: the driver refused a tensor map.
+dk_status launch_field_fwd_tma(const dk_ctx* ctx, const Geom& g, const FwdParams& fp, const MmaConsts& mc,
+                               const u32* W, const u32* xbar, int nsamples, uint8_t* wplanes, int kcp,
+                               uint8_t* xplanes, u64* split_acc, size_t split_bytes, int sm_count, int* status,
+                               unsigned spin_cap, int withhold, cudaStream_t st) {
+  const int KT = (g.cin % 128) == 0 ? 128 : 64;
+  ftm::Params q;
+  // the box of 64 output pixels that covers the fewest positions outside the output
+  long long best = -1;
+  q.bw = q.bh = q.bs = 1;
+  for (int bw = 1; bw <= 64; bw *= 2)
+    for (int bh = 1; bw * bh <= 64; bh *= 2) {
+      const int bs = 64 / (bw * bh);
+      const long long cost = (long long)((g.wo + bw - 1) / bw) * bw * ((g.ho + bh - 1) / bh) * bh *
+                             ((nsamples + bs - 1) / bs) * bs;
+      if (best < 0 || cost < best || (cost == best && bw > q.bw)) { best = cost; q.bw = bw; q.bh = bh; q.bs = bs; }
+    }
+  q.WT = (g.wo + q.bw - 1) / q.bw;
+  q.HT = (g.ho + q.bh - 1) / q.bh;
+  const long long tiles = (long long)q.WT * q.HT * ((nsamples + q.bs - 1) / q.bs);
+  const int mtiles = (g.cout + ftm::TM - 1) / ftm::TM;
+  if (tiles > 2147483647LL || mtiles > 65535) return DK_ERR_SHAPE;
+  q.cblocks = g.cin / KT;
+  q.kw = g.kw; q.pad = g.pad;
+  q.ktiles = g.kh * g.kw * q.cblocks;
+  q.cout = g.cout; q.ho = g.ho; q.wo = g.wo; q.nsamples = nsamples;
+  q.n_out = g.n_out; q.ys_c = g.ys_c; q.ys_h = g.ys_h; q.ys_w = g.ys_w;
+  q.y = fp.y; q.md = fp.md; q.pow32 = mc.pow32;
+  q.status = status; q.spin_cap = spin_cap; q.withhold = withhold;
+  const long long n_y = (long long)nsamples * g.n_out;
+  int ns = field_fwd_slices(tiles * mtiles, q.ktiles, sm_count);
+  if (split_acc == nullptr || split_bytes < (size_t)n_y * sizeof(u64)) ns = 1;
+  q.tiles_per_split = (q.ktiles + ns - 1) / ns;
+  ns = (q.ktiles + q.tiles_per_split - 1) / q.tiles_per_split;
+  q.split_acc = ns > 1 ? split_acc : nullptr;
+
+  CUtensorMap map_w, map_x;
+  {
+    const unsigned long long dims[3] = {(unsigned long long)kcp, (unsigned long long)g.cout, 4ull};
+    const unsigned long long str[2] = {(unsigned long long)kcp, (unsigned long long)kcp * g.cout};
+    const unsigned int box[3] = {(unsigned)KT, (unsigned)ftm::TM, 4u};
+    if (!tc_encode_map_bytes(ctx, &map_w, wplanes, 3, dims, str, box, KT)) return DK_ERR_UNSUPPORTED;
+  }
+  {
+    const unsigned long long n_x = (unsigned long long)nsamples * g.n_in;
+    const unsigned long long dims[5] = {(unsigned long long)g.cin, (unsigned long long)g.w, (unsigned long long)g.h,
+                                        (unsigned long long)nsamples, 4ull};
+    const unsigned long long str[4] = {(unsigned long long)g.cin, (unsigned long long)g.cin * g.w,
+                                       (unsigned long long)g.n_in, n_x};
+    const unsigned int box[5] = {(unsigned)KT, (unsigned)q.bw, (unsigned)q.bh, (unsigned)q.bs, 4u};
+    if (!tc_encode_map_bytes(ctx, &map_x, xplanes, 5, dims, str, box, KT)) return DK_ERR_UNSUPPORTED;
+  }
+  const long long chunks = (long long)g.cout * (kcp / 16);
+  field_w_planes_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(W, g.cout, g.kc, kcp, wplanes);
+  DK_CUDA_CHECK(cudaGetLastError());
+  const long long nx = (long long)nsamples * g.n_in;
+  field_x_planes_kernel<<<ew_blocks(nx / 16, sm_count), 256, 0, st>>>(xbar, nx, xplanes, g.n_in, 1, 1);
+  DK_CUDA_CHECK(cudaGetLastError());
+  if (ns > 1) DK_CUDA_CHECK(cudaMemsetAsync(split_acc, 0, (size_t)n_y * sizeof(u64), st));
+  const dim3 grid((unsigned)tiles, (unsigned)mtiles, (unsigned)ns);
+  constexpr size_t kSmem = (size_t)2 * 4 * (ftm::TM + ftm::TN) * 128 + 1024;      // two stages of 128-byte rows = four of 64
+  static const bool attr_ok =
+      cudaFuncSetAttribute(field_fwd_tma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem) == cudaSuccess &&
+      cudaFuncSetAttribute(field_fwd_tma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem) == cudaSuccess;
+  if (!attr_ok) return DK_ERR_CUDA;
+  if (KT == 128) field_fwd_tma_kernel<128><<<grid, ftm::kThreads, kSmem, st>>>(map_w, map_x, q);
+  else field_fwd_tma_kernel<64><<<grid, ftm::kThreads, kSmem, st>>>(map_w, map_x, q);
+  DK_CUDA_CHECK(cudaGetLastError());
+  if (ns > 1) {
+    field_reduce_kernel<<<ew_blocks(n_y, sm_count), 256, 0, st>>>(split_acc, n_y, fp.md, fp.y);
+    DK_CUDA_CHECK(cudaGetLastError());
+  }
+  return DK_OK;
+}
+
 // `wplanes` (nullable): device scratch of at least 4 * cout * round_up(kc, 128) bytes for the digit planes of W;
 // without it the contraction runs on the mma.sync kernel.  `split_acc` (nullable, split_bytes): uint64 scratch
 // in which slices of the contraction meet when a layer has too few output tiles to fill the device.
 dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* ybar, int nsamples, Modulus md,
                            uint8_t* wplanes, size_t wplanes_bytes, u64* split_acc, size_t split_bytes, int sm_count,
-                           int* status, int path, unsigned spin_cap, int withhold, cudaStream_t st) {
+                           int* status, int path, unsigned spin_cap, int withhold, cudaStream_t st,
+                           const dk_ctx* ctx = nullptr, uint8_t* xplanes = nullptr, size_t xplanes_bytes = 0) {
   FwdParams p;
   p.W = W; p.x = xbar; p.y = ybar;
   p.cin = g.cin; p.cout = g.cout; p.h = g.h; p.w = g.w; p.kw = g.kw; p.stride = g.stride;
@@ -1186,6 +1668,14 @@ dk_status launch_field_fwd(const Geom& g, const u32* W, const u32* xbar, u32* yb
     const bool vec4 = g.xs_c == 1 && g.ws_c == 1 && (g.cin % 4) == 0 && aligned16(W) && aligned16(xbar);
     const int kcp = (g.kc + tcf::TK - 1) / tcf::TK * tcf::TK;
     if (vec4 && path != 2 && wplanes != nullptr && wplanes_bytes >= (size_t)4 * g.cout * kcp) {
+      // operands by TMA (path 0 only; option value 3 keeps the kernel that splits x_bar in registers)
+      const long long n_x = (long long)nsamples * g.n_in;
+      if (path == 0 && ctx != nullptr && xplanes != nullptr && xplanes_bytes >= (size_t)4 * n_x &&
+          g.layout == DK_NHWC && g.stride == 1 && (g.cin % 64) == 0 && (n_x % 16) == 0) {
+        dk_status ts = launch_field_fwd_tma(ctx, g, p, mc, W, xbar, nsamples, wplanes, kcp, xplanes, split_acc,
+                                            split_bytes, sm_count, status, spin_cap, withhold, st);
+        if (ts != DK_ERR_UNSUPPORTED) return ts;
+      }
       static const bool tc_attr_ok =
           cudaFuncSetAttribute(field_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)tcf::kSmem) == cudaSuccess;
@@ -1539,7 +2029,7 @@ int ew_blocks(long long n, int sm_count) {
 int* field_status_word(dk_ctx* ctx) { return reinterpret_cast<int*>(ctx->d_vstats + kVerifyStatFloats) + 2; }
 
 struct FieldWs {
-  size_t wq, wpl, wpl_bytes, xq, xbar, ybar, bq, dtil, acc64, total;
+  size_t wq, wpl, wpl_bytes, xq, xbar, ybar, bq, dtil, acc64, xpl, xpl_bytes, total;
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -1555,6 +2045,11 @@ FieldWs plan_field_ws(const Geom& g) {
   w.ybar = off; off += align_up((size_t)g.G * g.E * g.n_out * sizeof(u32), 1024);
   w.bq = off; off += align_up((size_t)g.cout * sizeof(u32), 1024);
   w.dtil = off; off += align_up((size_t)g.G * (g.K + 1) * g.n_out * sizeof(u32), 1024);
+  // digit planes of the encodings (forward) or of the mixed gradients and the encodings (weight gradient)
+  w.xpl_bytes = (size_t)4 * g.G * (g.E * g.n_in + (g.K + 1) * g.n_out);
+  w.xpl = off; off += align_up(w.xpl_bytes, 1024);
+  // last: uint64 accumulators of the weight gradient; the forward kernels' contraction slices meet in whatever
+  // follows this offset
   w.acc64 = off; off += align_up((size_t)g.cout * g.kc * sizeof(u64), 1024);
   w.total = off;
   return w;
@@ -1613,6 +2108,7 @@ dk_status decode_verify_launch(dk_ctx* ctx, const Geom& g, int l, const u32* yba
   dp.ch_div = (g.layout == DK_NCHW) ? (long long)g.ho * g.wo : 1;
   dp.cout = g.cout;
   dp.inv_scale = ldexp(1.0, -l);
+  dp.lbits = l;
   dp.md = md;
   const bool vec4 = (g.n_out % 4) == 0 && aligned16(ybar) && aligned16(yq) && aligned16(y);
   ProfScope ps(ctx, DK_KERNEL_DECODE_VERIFY, 1, st);
@@ -1704,7 +2200,9 @@ dk_status dk_field_linear_fwd(dk_ctx* ctx, const dk_problem* p, uint32_t prime, 
                           have_ws ? wp.wpl_bytes : 0,
                           have_ws ? reinterpret_cast<u64*>(static_cast<char*>(ctx->ws) + wp.acc64) : nullptr,
                           have_ws ? wp.total - wp.acc64 : 0, ctx->sm_count, field_status_word(ctx), ctx->opt.v[DK_OPT_FIELD_PATH], (unsigned)ctx->opt.v[DK_OPT_SPIN_LIMIT],
-                          take_withhold(ctx), st);
+                          take_withhold(ctx), st, ctx,
+                          have_ws ? reinterpret_cast<uint8_t*>(static_cast<char*>(ctx->ws) + wp.xpl) : nullptr,
+                          have_ws ? wp.xpl_bytes : 0);
 }
 
 dk_status dk_field_decode_verify(dk_ctx* ctx, const dk_problem* p, uint32_t prime, int32_t l,
@@ -1776,7 +2274,7 @@ dk_status dk_field_masked_linear(dk_ctx* ctx, const dk_problem* p, uint32_t prim
     s = launch_field_fwd(g, Wq, xbar, ybar, g.G * g.E, md, reinterpret_cast<uint8_t*>(ws + wp.wpl), wp.wpl_bytes,
                          reinterpret_cast<u64*>(ws + wp.acc64), wp.total - wp.acc64, ctx->sm_count,
                          field_status_word(ctx), ctx->opt.v[DK_OPT_FIELD_PATH], (unsigned)ctx->opt.v[DK_OPT_SPIN_LIMIT],
-                          take_withhold(ctx), st);
+                          take_withhold(ctx), st, ctx, reinterpret_cast<uint8_t*>(ws + wp.xpl), wp.xpl_bytes);
   }
   if (s != DK_OK) return s;
   if (fault) {
@@ -1819,6 +2317,79 @@ dk_status dk_field_linear_bwd_wgrad(dk_ctx* ctx, const dk_problem* p, uint32_t p
   const long long n_dw = (long long)g.cout * g.kc;
   const long long tiles = (long long)((g.cout + BM - 1) / BM) * ((g.kc + BN - 1) / BN);
   if ((g.cout + BM - 1) / BM > 65535) return DK_ERR_SHAPE;
+  const long long n_d = (long long)g.G * (g.K + 1) * g.n_out, n_xu = (long long)g.G * (g.K + 1) * g.n_in;
+  if (ctx->opt.v[DK_OPT_FIELD_PATH] == 0 && g.layout == DK_NHWC && g.stride == 1 && (g.cin % 16) == 0 &&
+      (g.cout % 16) == 0 && wp.xpl_bytes >= (size_t)4 * (n_d + n_xu) && aligned16(xbar)) {
+    // tcgen05 kernel on digit planes of the mixed gradients and of the K+1 encodings Eq. 4 uses
+    uint8_t* dpl = reinterpret_cast<uint8_t*>(ws + wp.xpl);
+    uint8_t* xpl = dpl + 4 * n_d;
+    fwg::Params q;
+    const int S = g.G * (g.K + 1);
+    long long best = -1;
+    q.bw = q.bh = q.bs = 1;
+    for (int bw = 1; bw <= fwg::KP; bw *= 2)
+      for (int bh = 1; bw * bh <= fwg::KP; bh *= 2) {
+        const int bs = fwg::KP / (bw * bh);
+        const long long cost = (long long)((g.wo + bw - 1) / bw) * bw * ((g.ho + bh - 1) / bh) * bh *
+                               ((S + bs - 1) / bs) * bs;
+        if (best < 0 || cost < best || (cost == best && bw > q.bw)) { best = cost; q.bw = bw; q.bh = bh; q.bs = bs; }
+      }
+    q.WT = (g.wo + q.bw - 1) / q.bw;
+    q.HT = (g.ho + q.bh - 1) / q.bh;
+    q.PB = (long long)q.WT * q.HT * ((S + q.bs - 1) / q.bs);
+    q.MT = (g.cout + fwg::TM - 1) / fwg::TM;
+    q.cblocks = (g.cin + fwg::TN - 1) / fwg::TN;
+    q.kw = g.kw; q.pad = g.pad; q.cout = g.cout; q.cin = g.cin;
+    q.ws_o = g.ws_o; q.ws_c = g.ws_c; q.ws_u = g.ws_u; q.ws_v = g.ws_v;
+    q.acc = acc; q.md = md; q.pow32 = (u32)((1ull << 32) % md.p);
+    q.status = field_status_word(ctx); q.spin_cap = (unsigned)ctx->opt.v[DK_OPT_SPIN_LIMIT];
+    q.withhold = take_withhold(ctx);
+    const long long items = (long long)q.MT * q.cblocks * g.kh * g.kw;
+    // contraction slices: about two rounds of CTAs on the device, at least 8 k-blocks each
+    long long splits = (2LL * ctx->sm_count + items - 1) / items;
+    if (splits > (q.PB + 7) / 8) splits = (q.PB + 7) / 8;
+    if (splits > 65535) splits = 65535;
+    if (splits < 1) splits = 1;
+    q.pb_per_split = (int)((q.PB + splits - 1) / splits);
+    splits = (q.PB + q.pb_per_split - 1) / q.pb_per_split;
+    CUtensorMap map_d, map_x;
+    bool maps_ok;
+    {
+      const unsigned long long dims[5] = {(unsigned long long)g.cout, (unsigned long long)g.wo, (unsigned long long)g.ho,
+                                          (unsigned long long)S, 4ull};
+      const unsigned long long str[4] = {(unsigned long long)g.cout, (unsigned long long)g.cout * g.wo,
+                                         (unsigned long long)g.n_out, (unsigned long long)n_d};
+      const unsigned int box[5] = {(unsigned)fwg::TM, (unsigned)q.bw, (unsigned)q.bh, (unsigned)q.bs, 4u};
+      maps_ok = tc_encode_map_bytes(ctx, &map_d, dpl, 5, dims, str, box, 128);
+    }
+    if (maps_ok) {
+      const unsigned long long dims[5] = {(unsigned long long)g.cin, (unsigned long long)g.w, (unsigned long long)g.h,
+                                          (unsigned long long)S, 4ull};
+      const unsigned long long str[4] = {(unsigned long long)g.cin, (unsigned long long)g.cin * g.w,
+                                         (unsigned long long)g.n_in, (unsigned long long)n_xu};
+      const unsigned int box[5] = {(unsigned)fwg::TN, (unsigned)q.bw, (unsigned)q.bh, (unsigned)q.bs, 4u};
+      maps_ok = tc_encode_map_bytes(ctx, &map_x, xpl, 5, dims, str, box, 64);
+    }
+    static const bool tma_attr_ok = cudaFuncSetAttribute(field_wgrad_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                         (int)fwg::kSmem) == cudaSuccess;
+    if (maps_ok && tma_attr_ok && items <= 2147483647LL) {
+      {
+        ProfScope ps(ctx, DK_KERNEL_WGRAD, 3, st);
+        field_x_planes_kernel<<<ew_blocks(n_d / 16, ctx->sm_count), 256, 0, st>>>(dtil, n_d, dpl, g.n_out, 1, 1);
+        DK_CUDA_CHECK(cudaGetLastError());
+        field_x_planes_kernel<<<ew_blocks(n_xu / 16, ctx->sm_count), 256, 0, st>>>(xbar, n_xu, xpl, g.n_in, xbar_rows,
+                                                                                  g.K + 1);
+        DK_CUDA_CHECK(cudaGetLastError());
+        DK_CUDA_CHECK(cudaMemsetAsync(acc, 0, (size_t)n_dw * sizeof(u64), st));
+        field_wgrad_tma_kernel<<<dim3((unsigned)items, (unsigned)splits), fwg::kThreads, fwg::kSmem, st>>>(map_d, map_x, q);
+        DK_CUDA_CHECK(cudaGetLastError());
+      }
+      ProfScope ps2(ctx, DK_KERNEL_OTHER, 1, st);
+      field_reduce_kernel<<<ew_blocks(n_dw, ctx->sm_count), 256, 0, st>>>(acc, n_dw, md, dWq);
+      DK_CUDA_CHECK(cudaGetLastError());
+      return DK_OK;
+    }
+  }
   if (ctx->opt.v[DK_OPT_FIELD_PATH] == 1) {
     WgParams wg;
     wg.d = dtil; wg.x = xbar; wg.acc = acc;

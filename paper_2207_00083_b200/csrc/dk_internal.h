@@ -7,6 +7,8 @@
 
 #include "dk.h"
 
+struct CUtensorMap_st;      // the driver's tensor-map type (cuda.h)
+
 namespace dk {
 
 // Geometry of one layer, derived once from dk_problem.
@@ -180,6 +182,10 @@ struct ProfScope {
 
 // tensor-core path (dk_tc.cu)
 dk_status tc_init(dk_ctx* ctx);
+// tiled tensor map over bytes, 64- or 128-byte swizzle, zero fill outside (false: the driver refused it)
+bool tc_encode_map_bytes(const dk_ctx* ctx, ::CUtensorMap_st* m, const void* base, int rank,
+                         const unsigned long long* dims, const unsigned long long* strides_bytes,
+                         const unsigned int* box, int swz_bytes);
 void tc_destroy(dk_ctx* ctx);
 // true when the tensor-core kernel takes this geometry (channels-last,
 // stride 1, cin % 4 == 0, not DK_FP32_SIMT)

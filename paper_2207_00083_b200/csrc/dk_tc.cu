@@ -399,6 +399,22 @@ dk_status tc_init(dk_ctx* ctx) {
   return DK_OK;
 }
 
+// Tiled tensor map over bytes (the digit planes of the finite-field kernels): swz_bytes = 64 or 128.
+bool tc_encode_map_bytes(const dk_ctx* ctx, CUtensorMap* m, const void* base, int rank, const unsigned long long* dims,
+                         const unsigned long long* strides_bytes, const unsigned int* box, int swz_bytes) {
+  const TcState* ts = static_cast<const TcState*>(ctx->tc_state);
+  if (!ts || rank < 1 || rank > 5) return false;
+  cuuint64_t d[5], st[4];
+  cuuint32_t b[5], es[5] = {1, 1, 1, 1, 1};
+  for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; }
+  for (int i = 0; i + 1 < rank; ++i) st[i] = strides_bytes[i];
+  CUresult r = ts->encode(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          swz_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 int tc_smem_optin(const dk_ctx* ctx) {
   return ctx->tc_state ? static_cast<TcState*>(ctx->tc_state)->smem_optin : 0;
 }

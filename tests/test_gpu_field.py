@@ -40,6 +40,12 @@ CASES = [
     ("vgg_cifar_conv3_1_G2", synth.layer("vgg16_cifar", "conv3_1").with_groups(2), dk.DK_NHWC),
     ("vgg_cifar_conv5_1_G2", synth.layer("vgg16_cifar", "conv5_1").with_groups(2), dk.DK_NHWC),
     ("mbv2_project_960_320_G1", synth.layer("mobilenetv2_pw", "project_960_320").with_groups(1), dk.DK_NHWC),
+    # operands fetched by TMA from digit planes (channels-last, stride 1, cin % 64 == 0): 64- and 128-byte rows,
+    # ragged pixel boxes, ragged output channels, no padding, a 5x5 filter
+    ("conv_tma_cin64", tiny(cin=64, cout=72, h=9, w=7, K=2, G=2), dk.DK_NHWC),
+    ("conv_tma_cin128_5x5", tiny(cin=128, cout=130, h=6, w=10, kh=5, kw=5, pad=2, K=3, G=1), dk.DK_NHWC),
+    ("conv_tma_cin192_nopad", tiny(cin=192, cout=16, h=8, w=8, pad=0, K=1, G=3), dk.DK_NHWC),
+    ("fc_tma_cin640", tiny("fc", cin=640, cout=200, K=4, G=5), dk.DK_NHWC),
 ]
 
 
@@ -312,15 +318,15 @@ def test_full_size_layer_sampled_against_the_oracle(ctx, layer):
 
 
 CROSS_CHECK = [c for c in CASES if c[0] in ("conv_tiny_K2", "fc_K8_long", "conv_3x3s2_K5", "conv_ragged_K3_nchw",
-                                            "vgg_cifar_conv3_1_G2", "fc_long_tc")]
+                                            "vgg_cifar_conv3_1_G2", "fc_long_tc", "conv_tma_cin64")]
 
 
-@pytest.mark.parametrize("path", [1, 2], ids=["integer_alu", "mma_sync"])
+@pytest.mark.parametrize("path", [1, 2, 3], ids=["integer_alu", "mma_sync", "tcgen05_register_split"])
 @pytest.mark.parametrize("name,spec,layout", CROSS_CHECK, ids=[c[0] for c in CROSS_CHECK])
 def test_cross_check_kernels_give_the_same_residues(name, spec, layout, path):
-    """Option DK_OPT_FIELD_PATH = 1 selects the 64-bit integer-ALU contraction kernels, 2 keeps the forward
-    contraction on the mma.sync kernel instead of the tcgen05 one: the encoded outputs and the weight
-    gradient are the same residues as the oracle's under each."""
+    """Option DK_OPT_FIELD_PATH = 1 selects the 64-bit integer-ALU contraction kernels, 2 keeps the
+    contractions on the mma.sync kernels instead of the tcgen05 ones, 3 keeps them off the TMA-fed tcgen05
+    kernels: the encoded outputs and the weight gradient are the same residues as the oracle's under each."""
     c = dk.Context(0)
     try:
         dk.dk_set_option(c, dk.DK_OPT_FIELD_PATH, path)
@@ -353,7 +359,8 @@ def test_cross_check_kernels_give_the_same_residues(name, spec, layout, path):
 # (p-1)^2 = 1 (mod p), so a contraction of n such products is n mod p.
 # ---------------------------------------------------------------------------
 ADV_PRIMES = [2 ** 25 - 39, 2 ** 30 - 35]
-ADV_LENGTHS = [8188, 8191, 8192, 8193, 8196, 16380, 16385, 16388, 24580]     # multiples of 4 take the tcgen05 kernel
+# multiples of 4 take a tcgen05 kernel, multiples of 64 the TMA-fed one (64-byte rows; 128-byte rows for multiples of 128)
+ADV_LENGTHS = [8188, 8191, 8192, 8193, 8196, 16380, 16385, 16388, 24580, 8128, 8256, 16320, 16384, 16448, 24640]
 
 
 @pytest.mark.parametrize("prime", ADV_PRIMES)
