@@ -445,13 +445,14 @@ def measure_field(torch, dk, synth, ctx, dev, peaks, flush, workload, want, iter
     mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
     peak = SMS * IMMA_OPS_PER_CLK_SM * mhz * 1e6 / INT8_OPS_PER_FIELD_MAC / 1e12
     peak_tc5 = SMS * UTCIMMA_OPS_PER_CLK_SM * mhz * 1e6 / INT8_OPS_PER_FIELD_MAC / 1e12
-    cin_of = {s.name: s.cin for s in synth.layers(workload)}
+    spec_of = {s.name: s for s in synth.layers(workload)}
     for row in rows:
         for name in ("fwd", "wgrad"):
             if name in row:
-                # the forward contraction of layers with contiguous channels runs on tcgen05.mma.kind::i8,
-                # everything else on mma.sync
-                tc5 = name == "fwd" and cin_of[row["layer"]] % 4 == 0
+                # the library's dispatch (channels-last): the forward contraction runs on tcgen05.mma.kind::i8 when
+                # cin % 4 == 0, the weight gradient when stride 1 and cin, cout % 16 == 0; the rest on mma.sync
+                sp = spec_of[row["layer"]]
+                tc5 = (sp.cin % 4 == 0) if name == "fwd" else (sp.stride == 1 and sp.cin % 16 == 0 and sp.cout % 16 == 0)
                 row[name]["path"] = "tcgen05 kind::i8" if tc5 else "mma.sync u8"
                 row[name]["peak_tmacs"] = round(peak_tc5 if tc5 else peak, 2)
                 row[name]["frac_of_peak_kernel"] = round(row[name]["tmacs_kernel"] / (peak_tc5 if tc5 else peak), 4)
