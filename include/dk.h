@@ -184,11 +184,16 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  *                     amplify errors in the noise term of the encoded outputs
  *                     (a = max_k sum_i |Cinv[k][i]| |C[i][K]|, in exact arithmetic
  *                     the noise cancels: sum_i Cinv[k][i] C[i][K] = 0) takes shorter
- *                     chunks: 8 k-blocks up to a = 8, 4 up to 16, 2 up to 32, 1
+ *                     chunks: 8 k-blocks up to a = 12, 4 up to 20, 2 up to 30, 1
  *                     beyond.  Measured at noise 100x the inputs, the decoded error is
  *                     about (2.2e-5 + 0.5e-5 x k-blocks) x a of the output scale, so
- *                     this keeps it below 1e-3 up to a = 32.  0: every tile uses
+ *                     this keeps it below 1e-3 up to a = 30.  0: every tile uses
  *                     DK_OPT_TC_CHUNK.
+ *   DK_OPT_WG_PACE    1 (default): the persistent CTAs of the tensor-core weight-gradient
+ *                     kernel start each round of work items together (a bounded wait
+ *                     on a device counter, a hint only), so that the items that read
+ *                     the same operands stay close in time and share them in L2;
+ *                     0: every CTA runs ahead as it can.
  *   DK_OPT_SLABS      default 1: one pre-pass launch, then one GEMM launch.  n > 1:
  *                     the tensor-core forward and weight-gradient calls may be cut
  *                     into up to n ranges of virtual batches (at most 8): the
@@ -216,7 +221,7 @@ enum {
   DK_OPT_TC_CHUNK = 0, DK_OPT_WG_CHUNK = 1, DK_OPT_TC_BK = 2, DK_OPT_TC_PAIR = 3, DK_OPT_WG_PACK = 4,
   DK_OPT_WG_PAIR = 5, DK_OPT_TC_STEM = 6, DK_OPT_FIELD_PATH = 7, DK_OPT_SPIN_LIMIT = 8,
   DK_OPT_TEST_WITHHOLD = 9, DK_OPT_XBAR_HI = 10, DK_OPT_TC_MPACK = 11, DK_OPT_SLABS = 12, DK_OPT_SLABS_FORCE = 13,
-  DK_OPT_TC_CHUNK_ADAPT = 14, DK_OPT_COUNT = 15
+  DK_OPT_TC_CHUNK_ADAPT = 14, DK_OPT_WG_PACE = 15, DK_OPT_COUNT = 16
 };
 DK_API dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value);
 DK_API dk_status dk_get_option(dk_ctx* ctx, int32_t option, int32_t* value);

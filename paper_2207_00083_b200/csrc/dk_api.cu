@@ -146,8 +146,10 @@ dk_status upload_coefficients(dk_ctx* ctx, const Geom& g, const float* C_host,
       // a = max_k sum_i |inv[k][i]| |C[i][K]| (in exact arithmetic sum_i inv[k][i] C[i][K] = 0: the noise
       // cancels).  The forward kernels' accumulator in tensor memory truncates when it adds, a bias that grows
       // with the k-blocks added there; measured at noise 100x the inputs, the decoded error is about
-      // (2.2e-5 + 0.5e-5 x k-blocks) x a of the output scale.  The chunk lengths below keep that under 1e-3
-      // up to a = 32 (beyond, one k-block per chunk is the best this arithmetic does).
+      // (2.2e-5 + 0.5e-5 x k-blocks) x a of the output scale for a short contraction (288 elements; less for
+      // long ones).  The chunk lengths below keep that under 1e-3 up to a = 30 (beyond, one k-block per chunk
+      // is the best this arithmetic does): 7.4e-4 at a = 12 with 8 k-blocks, 8.4e-4 at 20 with 4, 9.6e-4 at 30
+      // with 2.
       {
         double amp = 0.0;
         for (int k = 0; k < K; ++k) {
@@ -155,7 +157,7 @@ dk_status upload_coefficients(dk_ctx* ctx, const Geom& g, const float* C_host,
           for (int i = 0; i < K1; ++i) a += fabs(inv[k * K1 + i]) * fabs((double)Cg[i * K1 + K]);
           amp = a > amp ? a : amp;
         }
-        const int cap = amp <= 8.0 ? 8 : (amp <= 16.0 ? 4 : (amp <= 32.0 ? 2 : 1));
+        const int cap = amp <= 12.0 ? 8 : (amp <= 20.0 ? 4 : (amp <= 30.0 ? 2 : 1));
         if (cap < view->chunk_cap) view->chunk_cap = cap;
         h_chunk[gi] = (unsigned char)cap;
       }
@@ -335,7 +337,7 @@ dk_status dk_create(dk_ctx** out, int device) {
     return DK_ERR_CUDA;
   }
   c->sm_count = sms;
-  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1, 1, 1, 0, 1};
+  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1, 1, 1, 0, 1, 1};
   for (int i = 0; i < DK_OPT_COUNT; ++i) c->opt.v[i] = kOptDefault[i];
   bool ok = cudaMallocHost(&c->h_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
@@ -381,8 +383,8 @@ dk_status dk_destroy(dk_ctx* c) {
 
 dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx || option < 0 || option >= DK_OPT_COUNT) return DK_ERR_INVALID_ARG;
-  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0, 0, 1, 0, 0};
-  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 3, 1 << 26, 1 << 20, 1, 1, kMaxSlabs, kMaxSlabs, 1};
+  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0, 0, 1, 0, 0, 0};
+  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 3, 1 << 26, 1 << 20, 1, 1, kMaxSlabs, kMaxSlabs, 1, 1};
   int v = value < lo[option] ? lo[option] : (value > hi[option] ? hi[option] : value);
   if (option == DK_OPT_TC_BK) v = v == 16 ? 16 : 32;
   ctx->opt.v[option] = v;

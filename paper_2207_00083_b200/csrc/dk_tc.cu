@@ -552,8 +552,9 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   prm.dec = cv.dec; prm.decl = cv.decl; prm.nul = cv.nul; prm.bias = bias;
   // ill-conditioned coefficient sets take shorter chunks (see upload_coefficients): per virtual batch where the
   // kernels' table holds them all, else the worst one's for the whole call
-  if (cv.chunk_tab != nullptr && g.G <= kChunkTabMax) prm.chunk_tab = cv.chunk_tab;
-  else if (cv.chunk_cap > 0 && prm.chunk > cv.chunk_cap * (32 / fwd_bk(ts))) prm.chunk = cv.chunk_cap * (32 / fwd_bk(ts));
+  if (cv.chunk_tab != nullptr && g.G <= kChunkTabMax) {
+    if (cv.chunk_cap * (32 / fwd_bk(ts)) < prm.chunk) prm.chunk_tab = cv.chunk_tab;      // (else no group needs less)
+  } else if (cv.chunk_cap > 0 && prm.chunk > cv.chunk_cap * (32 / fwd_bk(ts))) prm.chunk = cv.chunk_cap * (32 / fwd_bk(ts));
   prm.vs = vs;
   prm.status = status_word;
   prm.verdict = verdict;
@@ -813,6 +814,16 @@ dk_status tc_wgrad(dk_ctx* ctx, const Geom& g, const float* dt_hi, const float* 
   w.prm.scale = scale;
   w.prm.dW = dW;
   w.prm.status = status_word;
+  // the pace counter (the word after the status word) only when CTAs take several rounds of items
+  {
+    const int units = w.pair ? ctx->sm_count / 2 : ctx->sm_count;
+    w.prm.pace = nullptr;
+    // (long items only: with short ones the wait costs more than the shared reads save; fc6 measured 17 % slower)
+    if (ctx->opt.v[DK_OPT_WG_PACE] && w.prm.nitems > units && (long long)w.prm.pb_per_split * w.prm.K1 >= 128) {
+      w.prm.pace = reinterpret_cast<unsigned int*>(status_word) + 2;
+      DK_CUDA_CHECK(cudaMemsetAsync(w.prm.pace, 0, sizeof(unsigned int), st));
+    }
+  }
   CUtensorMap md_hi, md_lo, mx_hi, mx_lo;
   {
     cuuint64_t dims[5] = {(cuuint64_t)g.cout, (cuuint64_t)g.wo, (cuuint64_t)g.ho, (cuuint64_t)(g.K + 1),

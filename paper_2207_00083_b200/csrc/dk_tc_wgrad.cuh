@@ -52,6 +52,7 @@ struct WgTcParams {
   float scale;
   float* dW;                   // [cout][taps][cin]
   int* status;
+  unsigned int* pace;          // nullable: counter (zero at launch) with which the CTAs start their rounds of work items together
 };
 
 // Shared-memory descriptor of an MN-major 32-bit operand: [k][32 floats] boxes
@@ -152,7 +153,19 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
       bool alive = true;
       constexpr int NBOX = 2 * (BM / 32) + 2 * (BNL / 32);
       static_assert(NBOX <= 32, "one box per lane");
-      for (int item = first_item; alive && item < p.nitems; item += item_step) {
+      int round = 0;
+      for (int item = first_item; alive && item < p.nitems; item += item_step, ++round) {
+        // Pace.  The items that run at the same time are the filter taps (and channel blocks) of the same few
+        // slices of the contraction: they read the same gradients and, shifted, the same encodings, once from
+        // DRAM and then from L2 -- as long as they stay close in time.  CTAs that drift apart over several rounds
+        // of items lose that (measured: DRAM traffic of three passes over the operands where one would do), so a
+        // CTA starts round r only when all have issued the loads of round r-1, or after a bounded wait: this is
+        // a hint, never a condition for progress.
+        if (p.pace != nullptr && round > 0 && lane == 0 && rank == 0) {
+          const unsigned int target = (unsigned int)round * (unsigned int)item_step;
+          for (int spin = 0; spin < 4096 && *reinterpret_cast<volatile unsigned int*>(p.pace) < target; ++spin)
+            __nanosleep(128);
+        }
         int mt, nb, tg, pb_lo, pb_hi;
         item_range(item, mt, nb, tg, pb_lo, pb_hi);
         const int m0 = mt * MROWS + (int)rank * BM;
@@ -217,6 +230,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
           }
         }
+        if (p.pace != nullptr && alive && lane == 0 && rank == 0) atomicAdd(p.pace, 1u);
       }
     } else if (warp == 1 && lane == 0 && rank == 0) {
       // ---------------- MMA issuer (of a pair: the leader only) ----------------
