@@ -230,11 +230,14 @@ def shape_w(s):
 
 def uses_tensor_cores(s):
     """Mirror of the library's dispatch rule (channels-last, default arithmetic; stride <= 4 and
-    cin % 4 == 0, or a stem: cin % 4 != 0 with a contraction of at most 256 elements)."""
+    cin % 4 == 0, or a stem whose contraction has 65..256 elements: cin % 4 != 0 laid out as patch rows;
+    stems of 1-3 channels with at most 64 elements run in the fused fp32 kernel)."""
     if getattr(s, "precision", "default") != "default":
         return False
     if s.cin % 4 == 0:
         return s.stride <= 4
+    if s.cin <= 3 and s.kc <= 64:
+        return False
     return s.kind == "conv" and s.kc <= 256 and s.cout % 4 == 0
 
 
