@@ -139,11 +139,11 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  * measured best.  They exist for measurements (what a tiling choice costs), for
  * cross-checks in the tests (another kernel for the same result) and for the
  * failure-handling test.  A value outside an option's range is clamped.
- *   DK_OPT_TC_CHUNK   32-wide k-blocks accumulated in tensor memory between two
- *                     promotions to fp32 registers in the forward kernels
- *                     (default 8, 1..64).  CHANGES THE ARITHMETIC: the tensor
- *                     pipe truncates when it adds, so the error of y_bar grows
- *                     with the chunk length.
+ *   DK_OPT_TC_CHUNK   the most 32-wide k-blocks accumulated in tensor memory between
+ *                     two promotions to fp32 registers in the forward kernels
+ *                     (default 8, 1..64; see DK_OPT_TC_CHUNK_ADAPT).  CHANGES THE
+ *                     ARITHMETIC: the tensor pipe truncates when it adds, so the
+ *                     error of y_bar grows with the chunk length.
  *   DK_OPT_WG_CHUNK   the same for the weight-gradient kernel (default 2, 1..64);
  *                     changes the arithmetic likewise.
  *   DK_OPT_TC_BK      k-block of the forward kernel: 32 (default) or 16 floats.

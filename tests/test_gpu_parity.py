@@ -390,3 +390,42 @@ def test_nan_from_the_accelerator_is_flagged(ctx, drawn):
     dk.dk_decode_verify(ctx, p, H.dev(ybar), d["C"], None, y, v)
     got = dk.read_verdict(v)
     assert (got["ok"], got["n_flagged"], got["first_index"]) == (0, 1, 5)
+
+
+# ---------------------------------------------------------------------------
+# ill-conditioned coefficient sets: the chunk length in tensor memory follows the amplification
+# ---------------------------------------------------------------------------
+def _noise_amplification(Cg: np.ndarray) -> float:
+    """max_k sum_i |Cinv[k][i]| |C[i][K]| over the decoded rows k < K of one (K+2) x (K+1) coefficient block:
+    how strongly decoding amplifies an error that is relative to the noise term of the encoded outputs."""
+    K = Cg.shape[1] - 1
+    sq = Cg[:K + 1].astype(np.float64)
+    inv = np.linalg.inv(sq)
+    return float(max(np.sum(np.abs(inv[k]) * np.abs(sq[:, K])) for k in range(K)))
+
+
+def test_ill_conditioned_group_stays_within_the_bar(ctx):
+    """A coefficient set that the input recipe accepts can amplify noise-relative errors twenty-fold.  With
+    a fixed chunk of 8 k-blocks in tensor memory its decoded outputs miss the 1e-3 bar (the accumulator
+    there truncates); the library shortens the chunks of such virtual batches and holds it."""
+    spec = tiny(cin=32, cout=128, h=24, w=24, K=3, G=14)
+    d = synth.draw_layer(spec)
+    amps = [_noise_amplification(d["C"][g]) for g in range(spec.G)]
+    assert max(amps) > 20.0, amps          # the case this test is about (seeded: group 12)
+    p = dk.problem_from_spec(spec, tol=H.TAU)
+    ctx.ensure_workspace(p)
+    W = H.weights_to_dev(d["W"], lay(spec))
+    x, r = H.acts_to_dev(d["x"], lay(spec)), H.acts_to_dev(d["r"], lay(spec))
+    y = H.empty_acts(spec.G * spec.K, spec, "out", lay(spec))
+    v = dk.new_verdict()
+    plain = O.linear_plain(d["W"], d["x"], spec.stride, spec.pad)
+    errs = {}
+    for adapt in (1, 0):
+        dk.dk_set_option(ctx, dk.DK_OPT_TC_CHUNK_ADAPT, adapt)
+        dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y, None, v)
+        got_v = dk.read_verdict(v)
+        assert (got_v["ok"], got_v["n_flagged"], got_v["status"]) == (1, 0, 0)
+        errs[adapt] = H.max_rel(H.acts_from_dev(y, lay(spec)), plain)
+    dk.dk_set_option(ctx, dk.DK_OPT_TC_CHUNK_ADAPT, 1)
+    assert errs[1] < TOL_DECODED
+    assert errs[0] > errs[1]               # (1.35e-3 against 5.4e-4 when this was written)
