@@ -317,6 +317,8 @@ def run_layer_table(args):
     for s in synth.layers(args.workload):
         if want and s.name not in want:
             continue
+        if args.groups > 0:
+            s = s.with_groups(args.groups)      # a smaller batch of the same layer (for profiler captures)
         L = make_layer(torch, dk, synth, ctx, s, dev, gen, 0, pinned=False)
         ctx.ensure_workspace(L["p"])
         row = profile_layers(torch, dk, ctx, [L], peaks, tf32_peak, flush, iters=args.iters)[0]
@@ -945,6 +947,8 @@ def main():
     ap.add_argument("--field-table", action="store_true")
     ap.add_argument("--layers", default="")
     ap.add_argument("--iters", type=int, default=5)
+    ap.add_argument("--groups", type=int, default=0,
+                    help="--layer-table only: this many virtual batches per layer instead of the workload's")
     ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
                     help="a library option for this run, e.g. TC_CHUNK=4 (dk_set_option with DK_OPT_<NAME>); "
                          "the line then carries it under config.options")

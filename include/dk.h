@@ -189,6 +189,15 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  *                     about (2.2e-5 + 0.5e-5 x k-blocks) x a of the output scale, so
  *                     this keeps it below 1e-3 up to a = 30.  0: every tile uses
  *                     DK_OPT_TC_CHUNK.
+ *   DK_OPT_TC_LO_INKERNEL  default 0: the pre-pass writes the second TF32 term of the
+ *                     encoded activations.  1: where the kernel supports it (the
+ *                     single-CTA forward kernel), that term is derived inside the
+ *                     GEMM kernel instead (two warps compute tf32(v - trunc(v)) from
+ *                     the fp32 values a stage's copy brought, in shared memory): a
+ *                     third less traffic into the SMs and no second array in HBM,
+ *                     same results bit for bit, but measured 15-20 % slower kernels
+ *                     (the derivation lengthens every stage of a two-stage pipeline),
+ *                     which outweighs the shorter pre-pass.  Needs DK_OPT_XBAR_HI = 1.
  *   DK_OPT_WG_PACE    1 (default): the persistent CTAs of the tensor-core weight-gradient
  *                     kernel start each round of work items together (a bounded wait
  *                     on a device counter, a hint only), so that the items that read
@@ -221,7 +230,8 @@ enum {
   DK_OPT_TC_CHUNK = 0, DK_OPT_WG_CHUNK = 1, DK_OPT_TC_BK = 2, DK_OPT_TC_PAIR = 3, DK_OPT_WG_PACK = 4,
   DK_OPT_WG_PAIR = 5, DK_OPT_TC_STEM = 6, DK_OPT_FIELD_PATH = 7, DK_OPT_SPIN_LIMIT = 8,
   DK_OPT_TEST_WITHHOLD = 9, DK_OPT_XBAR_HI = 10, DK_OPT_TC_MPACK = 11, DK_OPT_SLABS = 12, DK_OPT_SLABS_FORCE = 13,
-  DK_OPT_TC_CHUNK_ADAPT = 14, DK_OPT_WG_PACE = 15, DK_OPT_COUNT = 16
+  DK_OPT_TC_CHUNK_ADAPT = 14, DK_OPT_WG_PACE = 15, DK_OPT_TC_LO_INKERNEL = 16,
+  DK_OPT_COUNT = 17
 };
 DK_API dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value);
 DK_API dk_status dk_get_option(dk_ctx* ctx, int32_t option, int32_t* value);

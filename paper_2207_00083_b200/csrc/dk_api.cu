@@ -337,7 +337,7 @@ dk_status dk_create(dk_ctx** out, int device) {
     return DK_ERR_CUDA;
   }
   c->sm_count = sms;
-  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1, 1, 1, 0, 1, 1};
+  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1, 1, 1, 0, 1, 1, 0};
   for (int i = 0; i < DK_OPT_COUNT; ++i) c->opt.v[i] = kOptDefault[i];
   bool ok = cudaMallocHost(&c->h_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
@@ -383,8 +383,8 @@ dk_status dk_destroy(dk_ctx* c) {
 
 dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx || option < 0 || option >= DK_OPT_COUNT) return DK_ERR_INVALID_ARG;
-  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0, 0, 1, 0, 0, 0};
-  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 3, 1 << 26, 1 << 20, 1, 1, kMaxSlabs, kMaxSlabs, 1, 1};
+  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0, 0, 1, 0, 0, 0, 0};
+  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 3, 1 << 26, 1 << 20, 1, 1, kMaxSlabs, kMaxSlabs, 1, 1, 1};
   int v = value < lo[option] ? lo[option] : (value > hi[option] ? hi[option] : value);
   if (option == DK_OPT_TC_BK) v = v == 16 ? 16 : 32;
   ctx->opt.v[option] = v;
@@ -449,18 +449,20 @@ dk_status dk_linear_fwd(dk_ctx* ctx, const dk_problem* p, const float* W, const 
     float* w_lo = reinterpret_cast<float*>(ws + wp.w_lo);
     float* xb_hi = reinterpret_cast<float*>(ws + wp.xb_hi);
     float* xb_lo = reinterpret_cast<float*>(ws + wp.xb_lo);
+    const bool lo_in = tc_fwd_lo_inkernel(ctx, g);
     {
       ProfScope ps(ctx, DK_KERNEL_OTHER, 2, st);
       const int raw = ctx->opt.v[DK_OPT_XBAR_HI];
       s = tc_split(W, w_hi, w_lo, (long long)g.cout * g.kc, ctx->sm_count, st);
-      if (s == DK_OK)
+      // (a kernel that derives the second term itself needs no pass over the encodings at all)
+      if (s == DK_OK && !lo_in)
         s = tc_split(xbar, raw ? nullptr : xb_hi, xb_lo, (long long)g.G * g.E * g.n_in, ctx->sm_count, st, raw);
       if (raw) xb_hi = const_cast<float*>(xbar);      // the kernel reads the caller's encodings as leading term
     }
     if (s != DK_OK) return s;
     ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
     return tc_linear_fwd(ctx, g, w_hi, w_lo, xb_hi, xb_lo, ybar, tc_fwd_ksplit(ctx, g), false, ctx_status_word(ctx),
-                         st);
+                         st, 0, lo_in);
   }
   ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
   return launch_simt_fwd(g, W, xbar, ybar, g.G * g.E, st);
@@ -603,6 +605,9 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     const int raw = stem ? 0 : ctx->opt.v[DK_OPT_XBAR_HI];
     float* full = xbar_save;
     if (raw && !full) full = reinterpret_cast<float*>(ws + wp.xbar);
+    // the second term: written by the pre-pass, or derived inside the GEMM kernel (then the array is unused)
+    const bool lo_in = raw && tc_fwd_lo_inkernel(ctx, gg);
+    if (lo_in) xb_lo = nullptr;
     // Large layers: the groups are cut into ranges; the pre-passes run in order on the context's second stream,
     // the GEMM of a range starts on the caller's stream as soon as its pre-pass has finished, and the kernel
     // of the last range takes the final decisions of the check.
@@ -633,7 +638,7 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
         if (cudaStreamWaitEvent(st, ctx->ev_slab[i], 0) != cudaSuccess) { s = DK_ERR_CUDA; break; }
         ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
         s = tc_masked_fwd(ctx, gg, w_hi, w_lo, xb_hi, xb_lo, cv, bias, y, vs, reinterpret_cast<int*>(vs.count + 1),
-                          fault, i == nslab - 1 ? verdict : nullptr, st, gt_lo[i], gt_lo[i + 1] - gt_lo[i]);
+                          fault, i == nslab - 1 ? verdict : nullptr, st, gt_lo[i], gt_lo[i + 1] - gt_lo[i], lo_in);
       }
       return s;
     }
@@ -652,7 +657,7 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
       {
         ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
         s = tc_linear_fwd(ctx, gg, w_hi, w_lo, xb_hi, xb_lo, ybar, ksplit, prepass_clears,
-                          reinterpret_cast<int*>(vs.count + 1), st, cv.chunk_cap);
+                          reinterpret_cast<int*>(vs.count + 1), st, cv.chunk_cap, lo_in);
       }
       if (s != DK_OK) return s;
       if (fault) {
@@ -672,7 +677,7 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
     {
       ProfScope ps(ctx, DK_KERNEL_LINEAR_FWD, 1, st);
       s = tc_masked_fwd(ctx, gg, w_hi, w_lo, xb_hi, xb_lo, cv, bias, y, vs,
-                        reinterpret_cast<int*>(vs.count + 1), fault, verdict, st);
+                        reinterpret_cast<int*>(vs.count + 1), fault, verdict, st, 0, -1, lo_in);
     }
     return s;      // the kernel's last CTA has written the verdict
   }

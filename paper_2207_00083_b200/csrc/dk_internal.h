@@ -203,7 +203,10 @@ dk_status tc_encode_split(const Geom& g, const float* x, const float* r, const f
 int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g);
 dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
                         const float* xb_hi, const float* xb_lo, float* ybar, int ksplit, bool ybar_cleared,
-                        int* status_word, cudaStream_t st, int chunk_cap = 0);
+                        int* status_word, cudaStream_t st, int chunk_cap = 0, bool lo_inkernel = false);
+// (lo_inkernel: xb_lo is neither read nor needed, the kernel derives the second term from the fp32 values in xb_hi;
+// ask tc_fwd_lo_inkernel whether the kernel that serves the geometry can)
+bool tc_fwd_lo_inkernel(const dk_ctx* ctx, const Geom& g);
 // (chunk_cap > 0: cap on the k-blocks of 32 added up in tensor memory, see CoefView::chunk_cap)
 // weight gradient on tensor cores (channels-last, stride 1, cin % 4 == 0, cout % 4 == 0)
 bool tc_wgrad_supported(const dk_ctx* ctx, const Geom& g);
@@ -243,7 +246,8 @@ dk_status tc_wgrad_prepass(const Geom& g, const float* delta, const float* dmix,
 dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo,
                         const float* xb_hi, const float* xb_lo, const CoefView& cv, const float* bias,
                         float* y, const VerifyScratch& vs, int* status_word, const dk_fault* fault,
-                        dk_verdict* verdict, cudaStream_t st, int gt_lo = 0, int gt_cnt = -1);
+                        dk_verdict* verdict, cudaStream_t st, int gt_lo = 0, int gt_cnt = -1,
+                        bool lo_inkernel = false);
 // (gt_cnt >= 0: only group tiles [gt_lo, gt_lo + gt_cnt) of the tiling; a call served by several such launches
 // gives `verdict` to the last one.  tc_fwd_group_tiles: group tiles, groups per tile, rounds of tiles per CTA.)
 bool tc_fwd_group_tiles(const dk_ctx* ctx, const Geom& g, int* GT, int* bg, long long* rounds);

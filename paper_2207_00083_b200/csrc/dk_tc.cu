@@ -252,7 +252,9 @@ bool encode_fwd_maps(const TcState* ts, const Geom& g, const Tiling& tl, const f
     cuuint64_t dims[5] = {(cuuint64_t)g.cin, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.E, (cuuint64_t)g.G};
     cuuint64_t str[4] = {(cuuint64_t)g.cin * 4, (cuuint64_t)g.cin * g.w * 4, (cuuint64_t)g.n_in * 4,
                          (cuuint64_t)g.n_in * g.E * 4};
-    cuuint32_t box[5] = {(cuuint32_t)BK, (cuuint32_t)(tl.bw * g.stride), (cuuint32_t)(tl.bh * g.stride), 1,
+    // (tiles of one virtual batch fetch all their encodings, or a CTA pair's half of them, as one box)
+    const cuuint32_t ebox = tl.bg == 1 ? (cuuint32_t)(tl.pair ? g.E / 2 : g.E) : 1u;
+    cuuint32_t box[5] = {(cuuint32_t)BK, (cuuint32_t)(tl.bw * g.stride), (cuuint32_t)(tl.bh * g.stride), ebox,
                          (cuuint32_t)tl.bg};
     if (!encode_map(ts, mb_hi, xb_hi, 5, dims, str, box, BK * 4, g.stride) ||
         !encode_map(ts, mb_lo, xb_lo, 5, dims, str, box, BK * 4, g.stride))
@@ -265,6 +267,7 @@ template <int BK, int MODE, int K>
 dk_status launch_one(const TcState* ts, const Geom& g, const Tiling& tl, const float* w_hi, const float* w_lo,
                      const float* xb_hi, const float* xb_lo, TcParams& prm, int sm_count, cudaStream_t st) {
   CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo;
+  if (xb_lo == nullptr) xb_lo = xb_hi;      // (the kernel derives the second term: that map is not used)
   if (!encode_fwd_maps<BK>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, &ma_hi, &ma_lo, &mb_hi, &mb_lo)) return DK_ERR_CUDA;
   auto kern = tc_fwd_kernel<BK, MODE, K>;
   static KernelCache kc = {};
@@ -326,6 +329,8 @@ void fill_params(const TcState* ts, const Geom& g, const Tiling& tl, TcParams* p
   p->spin_cap = (unsigned)ts->opt->v[DK_OPT_SPIN_LIMIT];
   p->withhold = ts->opt->v[DK_OPT_TEST_WITHHOLD];
   p->nprod = g.nprod == 2 ? 2 : 3;
+  p->lo_inkernel = 0;
+  p->b_onebox = tl.bg == 1 ? 1 : 0;
   p->hmul = tl.mpack ? 2 : 1;
   ts->opt->v[DK_OPT_TEST_WITHHOLD] = -1;      // the hook serves one launch
   p->ksplit = 1;
@@ -502,6 +507,15 @@ int tc_fwd_ksplit(const dk_ctx* ctx, const Geom& g) {
   return best;
 }
 
+// Whether the forward kernel that serves g derives the activations' second TF32 term itself (then nobody writes
+// or reads that array): option DK_OPT_TC_LO_INKERNEL, and a kernel that has the converter warps.
+bool tc_fwd_lo_inkernel(const dk_ctx* ctx, const Geom& g) {
+  TcState* ts = static_cast<TcState*>(ctx->tc_state);
+  Tiling tl;
+  if (!ts || !ctx->opt.v[DK_OPT_TC_LO_INKERNEL] || !ctx->opt.v[DK_OPT_XBAR_HI] || !plan_fwd(ts, g, &tl)) return false;
+  return !tl.pair;
+}
+
 bool tc_fwd_group_tiles(const dk_ctx* ctx, const Geom& g, int* GT, int* bg, long long* rounds) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
@@ -514,7 +528,7 @@ bool tc_fwd_group_tiles(const dk_ctx* ctx, const Geom& g, int* GT, int* bg, long
 
 dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
                         const float* xb_lo, float* ybar, int ksplit, bool ybar_cleared, int* status_word,
-                        cudaStream_t st, int chunk_cap) {
+                        cudaStream_t st, int chunk_cap, bool lo_inkernel) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!plan_fwd(ts, g, &tl)) return DK_ERR_UNSUPPORTED;
@@ -528,6 +542,8 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   }
   prm.out = ybar;
   if (chunk_cap > 0 && prm.chunk > chunk_cap * (32 / fwd_bk(ts))) prm.chunk = chunk_cap * (32 / fwd_bk(ts));
+  prm.lo_inkernel = (lo_inkernel && !tl.pair) ? 1 : 0;
+  if (lo_inkernel && tl.pair) return DK_ERR_INVALID_ARG;      // (the caller asked tc_fwd_lo_inkernel first)
   prm.status = status_word;
   return launch_bk<MODE_YBAR>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
 }
@@ -535,10 +551,11 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
 dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
                         const float* xb_lo, const CoefView& cv, const float* bias, float* y,
                         const VerifyScratch& vs, int* status_word, const dk_fault* fault, dk_verdict* verdict,
-                        cudaStream_t st, int gt_lo, int gt_cnt) {
+                        cudaStream_t st, int gt_lo, int gt_cnt, bool lo_inkernel) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!plan_fwd(ts, g, &tl)) return DK_ERR_UNSUPPORTED;
+  if (lo_inkernel && tl.pair) return DK_ERR_INVALID_ARG;      // (the caller asked tc_fwd_lo_inkernel first)
   if (gt_cnt >= 0) {
     // this launch covers group tiles [gt_lo, gt_lo + gt_cnt) only
     if (gt_lo < 0 || gt_cnt < 1 || gt_lo + gt_cnt > tl.GT) return DK_ERR_INVALID_ARG;
@@ -548,6 +565,7 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   TcParams prm;
   fill_params(ts, g, tl, &prm);
   if (gt_cnt >= 0) prm.gt0 = gt_lo;
+  prm.lo_inkernel = lo_inkernel ? 1 : 0;
   prm.out = y;
   prm.dec = cv.dec; prm.decl = cv.decl; prm.nul = cv.nul; prm.bias = bias;
   // ill-conditioned coefficient sets take shorter chunks (see upload_coefficients): per virtual batch where the

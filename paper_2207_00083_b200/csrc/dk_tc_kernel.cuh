@@ -70,6 +70,10 @@ struct TcParams {
   int withhold;                // test hook: the producer arms its n-th stage but issues no copy (-1 = off)
   int hmul;                    // 2: the tile's rows 64-127 are the image row below rows 0-63 (cout <= 64), else 1
   int nprod;                   // 3: W_hi.x_hi + W_hi.x_lo + W_lo.x_hi; 2: W as one TF32 term, W_lo neither loaded nor used
+  int b_onebox;                // 1 (tiles of one virtual batch, bg = 1): the encodings of a stage arrive as ONE box over the
+                               // encoding dimension per TF32 term instead of one box per encoding
+  int lo_inkernel;             // 1: the activations' second TF32 term is not loaded: two warps derive it in shared
+                               // memory from the fp32 values the first copy brought (tf32(v - trunc(v)))
   // problem
   int cout, ho, wo, G;
   long long n_out;
@@ -524,14 +528,17 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
   uint64_t* empty_bar = full_bar + kMaxStages;
   uint64_t* tfull_bar = empty_bar + kMaxStages;
   uint64_t* tempty_bar = tfull_bar + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  uint64_t* ready_bar = tempty_bar + 2;        // a stage's second term has been derived (one arrival per converter warp)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ready_bar + kMaxStages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nwork = p.ntiles * p.ksplit;     // work item = (tile, contraction slice)
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.nstages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
+    for (int s = 0; s < p.nstages; ++s) {
+      mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); mbar_init(ready_bar + s, 2);
+    }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + b, 1); mbar_init(tempty_bar + b, kEpiWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -577,7 +584,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
           int ok = 1;
           if (lane == 0) {
             ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
-            if (ok) mbar_expect_tx(full_bar + stage, (uint32_t)(STAGE_BYTES - (p.nprod == 2 ? A_BYTES : 0)));
+            if (ok) mbar_expect_tx(full_bar + stage, (uint32_t)(STAGE_BYTES - (p.nprod == 2 ? A_BYTES : 0) -
+                                                                (p.lo_inkernel ? B_BYTES : 0)));
           }
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) { alive = false; break; }
@@ -590,11 +598,17 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
             tma_load_3d(st, &map_a_hi, full_bar + stage, c0, tap, m0);
           } else if (lane == 1) {
             if (p.nprod == 3) tma_load_3d(st + A_BYTES, &map_a_lo, full_bar + stage, c0, tap, m0);
+          } else if (p.b_onebox) {
+            // (same bytes at the same places as the E boxes below: with one group per tile the encoding is the
+            // slowest dimension of the stage either way; fewer copies measured 4-7 % faster)
+            if (lane == 2) tma_load_5d(st + 2 * A_BYTES, &map_b_hi, full_bar + stage, c0, x0 + v, y0 + u, 0, g0);
+            else if (lane == 3 && !p.lo_inkernel)
+              tma_load_5d(st + 2 * A_BYTES + B_BYTES, &map_b_lo, full_bar + stage, c0, x0 + v, y0 + u, 0, g0);
           } else if (lane < 2 + 2 * E) {
             const int e = (lane - 2) >> 1;
             if ((lane & 1) == 0)
               tma_load_5d(st + 2 * A_BYTES + e * SUB, &map_b_hi, full_bar + stage, c0, x0 + v, y0 + u, e, g0);
-            else
+            else if (!p.lo_inkernel)
               tma_load_5d(st + 2 * A_BYTES + B_BYTES + e * SUB, &map_b_lo, full_bar + stage, c0, x0 + v, y0 + u,
                           e, g0);
           }
@@ -631,18 +645,60 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
             const uint64_t b_hi = make_desc<SWZ>(st + 2 * A_BYTES);
             const uint64_t b_lo = make_desc<SWZ>(st + 2 * A_BYTES + B_BYTES);
             const bool first = kb == kb_beg;
+            // the products that need only what the copies brought go first; the one with the activations' second
+            // term follows, after the converter warps have derived it (when they do)
 #pragma unroll
             for (int kk = 0; kk < BK / 8; ++kk) {
               const uint64_t adv = (uint64_t)(kk * 2);     // 32 bytes per k-step, in 16-byte units
               tc_mma_tf32(d_tmem, a_hi + adv, b_hi + adv, idesc, (first && kk == 0) ? 0u : 1u);
-              tc_mma_tf32(d_tmem, a_hi + adv, b_lo + adv, idesc, 1u);
               if (p.nprod == 3) tc_mma_tf32(d_tmem, a_lo + adv, b_hi + adv, idesc, 1u);
+            }
+            if (p.lo_inkernel) {
+              if (!mbar_wait(ready_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
+              tc_fence_after();
+            }
+#pragma unroll
+            for (int kk = 0; kk < BK / 8; ++kk) {
+              const uint64_t adv = (uint64_t)(kk * 2);
+              tc_mma_tf32(d_tmem, a_hi + adv, b_lo + adv, idesc, 1u);
             }
             tc_commit(empty_bar + stage);
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
           }
           if (alive) tc_commit(tfull_bar + buf);
         }
+      }
+    }
+  } else if (p.lo_inkernel) {
+    // ---------------- converters: warps 2 and 3 ----------------
+    // second TF32 term of the stage's activations, element by element in place of the copy that used to bring
+    // it (the swizzled position of an element is the same in both halves of the stage)
+    const int ctid = (int)threadIdx.x - 64;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool alive = true;
+    for (int w = blockIdx.x; alive && w < nwork; w += gridDim.x) {
+      const int ks = w % p.ksplit;
+      const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
+      for (int kb = kb_lo; kb < kb_hi; ++kb) {
+        if (!mbar_wait(full_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
+        const float4* src = reinterpret_cast<const float4*>(smem + (size_t)stage * STAGE_BYTES + 2 * A_BYTES);
+        float4* dst = reinterpret_cast<float4*>(smem + (size_t)stage * STAGE_BYTES + 2 * A_BYTES + B_BYTES);
+#pragma unroll 4
+        for (int i = ctid; i < B_BYTES / 16; i += 64) {
+          const float4 v = src[i];
+          float4 l;
+          l.x = to_tf32(v.x - __uint_as_float(__float_as_uint(v.x) & 0xffffe000u));
+          l.y = to_tf32(v.y - __uint_as_float(__float_as_uint(v.y) & 0xffffe000u));
+          l.z = to_tf32(v.z - __uint_as_float(__float_as_uint(v.z) & 0xffffe000u));
+          l.w = to_tf32(v.w - __uint_as_float(__float_as_uint(v.w) & 0xffffe000u));
+          dst[i] = l;
+        }
+        // make the stores visible to the tensor core's (asynchronous-proxy) reads, then hand the stage over
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(ready_bar + stage);
+        if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
       }
     }
   }

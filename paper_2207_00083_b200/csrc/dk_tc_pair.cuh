@@ -169,6 +169,11 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
           tma_pair_load_3d(st, &map_a_hi, bar, c0, tap, m0);
         } else if (lane == 1) {
           if (p.nprod == 3) tma_pair_load_3d(st + A_BYTES, &map_a_lo, bar, c0, tap, m0);
+        } else if (p.b_onebox) {
+          // one box over this CTA's half of the encodings per TF32 term (see tc_fwd_kernel)
+          if (lane == 2) tma_pair_load_5d(st + 2 * A_BYTES, &map_b_hi, bar, c0, x0 + v, y0 + u, (int)rank * EH, g0);
+          else if (lane == 3)
+            tma_pair_load_5d(st + 2 * A_BYTES + B_BYTES, &map_b_lo, bar, c0, x0 + v, y0 + u, (int)rank * EH, g0);
         } else if (lane < 2 + 2 * EH) {
           const int i = (lane - 2) >> 1;
           const int e = (int)rank * EH + i;

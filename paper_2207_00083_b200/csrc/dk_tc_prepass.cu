@@ -94,7 +94,7 @@ __device__ __forceinline__ void mix_job(const float* __restrict__ in, const floa
       const size_t off = ob + (size_t)i * n;
       if (full != nullptr) reinterpret_cast<float4*>(full + off)[q] = o;
       if (raw) {
-        reinterpret_cast<float4*>(lo + off)[q] = lo4_of_raw(o);
+        if (lo != nullptr) reinterpret_cast<float4*>(lo + off)[q] = lo4_of_raw(o);
       } else {
         split4(o, h, l);
         reinterpret_cast<float4*>(hi + off)[q] = h;
@@ -222,7 +222,9 @@ dk_status tc_fwd_prepass(const Geom& g, const float* x, const float* r, const fl
   const size_t eoff = (size_t)g_lo * g.E * g.n_in;
   a.x = x + (size_t)g_lo * g.K * g.n_in; a.r = r + (size_t)g_lo * g.n_in;
   a.enc = enc + (size_t)g_lo * g.E * (g.K + 1);
-  a.full = full ? full + eoff : nullptr; a.xb_hi = xb_hi ? xb_hi + eoff : nullptr; a.xb_lo = xb_lo + eoff;
+  a.full = full ? full + eoff : nullptr; a.xb_hi = xb_hi ? xb_hi + eoff : nullptr;
+  a.xb_lo = xb_lo ? xb_lo + eoff : nullptr;      // (null with raw: the GEMM kernel derives the second term itself)
+  if (xb_lo == nullptr && !raw) return DK_ERR_INVALID_ARG;
   a.n_in = g.n_in; a.G = g_cnt;
   // beside a GEMM kernel (one persistent CTA of 32K registers per SM) only a few small blocks fit on an SM, and a
   // larger grid would keep the GEMM's CTAs off the SMs until this kernel has ended: blocks of 128 threads, two

@@ -429,3 +429,41 @@ def test_ill_conditioned_group_stays_within_the_bar(ctx):
     dk.dk_set_option(ctx, dk.DK_OPT_TC_CHUNK_ADAPT, 1)
     assert errs[1] < TOL_DECODED
     assert errs[0] > errs[1]               # (1.35e-3 against 5.4e-4 when this was written)
+
+
+@pytest.mark.parametrize("name", ["vgg_cifar_conv3_1_G2", "conv_tiny_K2", "single_K3_cout160", "mpack_K8", "fc784"])
+def test_second_term_derived_in_the_kernel_gives_the_same_bits(ctx, drawn, name):
+    """DK_OPT_TC_LO_INKERNEL = 1: the single-CTA forward kernel derives tf32(v - trunc(v)) of the encodings in
+    shared memory instead of fetching the array the pre-pass would have written.  Same formula on the same
+    values, so the stored encodings are identical and outputs agree with the default's to the order of their
+    atomic additions, through the fused call and through dk_linear_fwd."""
+    spec = SPECS[IDS.index(name)]
+    d = drawn(spec)
+    K, E = spec.K, spec.K + 2
+    p = dk.problem_from_spec(spec, tol=H.TAU)
+    ctx.ensure_workspace(p)
+    W = H.weights_to_dev(d["W"], lay(spec))
+    x, r = H.acts_to_dev(d["x"], lay(spec)), H.acts_to_dev(d["r"], lay(spec))
+    v = dk.new_verdict()
+    got = {}
+    try:
+        for mode in (0, 1):
+            dk.dk_set_option(ctx, dk.DK_OPT_TC_LO_INKERNEL, mode)
+            y = H.empty_acts(spec.G * K, spec, "out", lay(spec))
+            xsave = H.empty_acts(spec.G * E, spec, "in", lay(spec))
+            dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y, xsave, v)
+            vd = dk.read_verdict(v)
+            ybar = H.empty_acts(spec.G * E, spec, "out", lay(spec))
+            dk.dk_linear_fwd(ctx, p, W, xsave, ybar)
+            torch.cuda.synchronize()
+            assert dk.dk_device_status(ctx) == 0
+            got[mode] = (y, xsave, ybar, vd)
+    finally:
+        dk.dk_set_option(ctx, dk.DK_OPT_TC_LO_INKERNEL, 0)
+    assert (got[1][3]["ok"], got[1][3]["n_flagged"], got[1][3]["status"]) == (1, 0, 0)
+    assert torch.equal(got[0][1], got[1][1])
+    # (small problems run as contraction slices that meet by atomic additions: equal up to that order)
+    for a, b in ((got[0][0], got[1][0]), (got[0][2], got[1][2])):
+        assert float((a - b).abs().max()) <= 1e-4 * float(a.abs().max())
+    plain = O.linear_plain(d["W"], d["x"], spec.stride, spec.pad)
+    assert H.max_rel(H.acts_from_dev(got[1][0], lay(spec)), plain) < TOL_DECODED
