@@ -190,14 +190,15 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  *                     this keeps it below 1e-3 up to a = 30.  0: every tile uses
  *                     DK_OPT_TC_CHUNK.
  *   DK_OPT_TC_LO_INKERNEL  default 0: the pre-pass writes the second TF32 term of the
- *                     encoded activations.  1: where the kernel supports it (the
- *                     single-CTA forward kernel), that term is derived inside the
- *                     GEMM kernel instead (two warps compute tf32(v - trunc(v)) from
- *                     the fp32 values a stage's copy brought, in shared memory): a
- *                     third less traffic into the SMs and no second array in HBM,
- *                     same results bit for bit, but measured 15-20 % slower kernels
- *                     (the derivation lengthens every stage of a two-stage pipeline),
- *                     which outweighs the shorter pre-pass.  Needs DK_OPT_XBAR_HI = 1.
+ *                     encoded activations.  1: that term is derived inside the forward
+ *                     GEMM kernels instead (two warps per CTA compute
+ *                     tf32(v - trunc(v)) from the fp32 values a stage's copy brought, in
+ *                     shared memory): a third less traffic into the SMs and no second
+ *                     array in HBM, same results bit for bit, but measured 15-20 %
+ *                     slower kernels (the derivation lengthens the way of every stage
+ *                     through a pipeline of two to four stages), which outweighs the
+ *                     shorter pre-pass.  2: only in the CTA-pair kernel.  Needs
+ *                     DK_OPT_XBAR_HI = 1.
  *   DK_OPT_WG_PACE    1 (default): the persistent CTAs of the tensor-core weight-gradient
  *                     kernel start each round of work items together (a bounded wait
  *                     on a device counter, a hint only), so that the items that read

@@ -203,7 +203,7 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
   t->BN = E * P;
   // a CTA of a pair stages its own 128 rows of W and half of the activation rows
   const size_t stage = 2 * ((size_t)BM * BK * 4 + (size_t)(pair ? t->BN / 2 : t->BN) * BK * 4);
-  const size_t ctrl = 1024 + 256;   // alignment slack + barriers
+  const size_t ctrl = 1024 + 512;   // alignment slack + barriers
   const size_t fixed = 1024 + 64;   // the kernels' static shared memory (table of chunk lengths)
   int ns = (int)(((size_t)smem_optin - ctrl - fixed) / stage);
   if (ns > kMaxStages) ns = kMaxStages;
@@ -513,7 +513,8 @@ bool tc_fwd_lo_inkernel(const dk_ctx* ctx, const Geom& g) {
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!ts || !ctx->opt.v[DK_OPT_TC_LO_INKERNEL] || !ctx->opt.v[DK_OPT_XBAR_HI] || !plan_fwd(ts, g, &tl)) return false;
-  return !tl.pair;
+  // option value 1: every forward kernel; 2: CTA pairs only (four stages hide the derivation, two do not)
+  return ctx->opt.v[DK_OPT_TC_LO_INKERNEL] == 1 || tl.pair;
 }
 
 bool tc_fwd_group_tiles(const dk_ctx* ctx, const Geom& g, int* GT, int* bg, long long* rounds) {
@@ -542,8 +543,7 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   }
   prm.out = ybar;
   if (chunk_cap > 0 && prm.chunk > chunk_cap * (32 / fwd_bk(ts))) prm.chunk = chunk_cap * (32 / fwd_bk(ts));
-  prm.lo_inkernel = (lo_inkernel && !tl.pair) ? 1 : 0;
-  if (lo_inkernel && tl.pair) return DK_ERR_INVALID_ARG;      // (the caller asked tc_fwd_lo_inkernel first)
+  prm.lo_inkernel = lo_inkernel ? 1 : 0;
   prm.status = status_word;
   return launch_bk<MODE_YBAR>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
 }
@@ -555,7 +555,6 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   TcState* ts = static_cast<TcState*>(ctx->tc_state);
   Tiling tl;
   if (!plan_fwd(ts, g, &tl)) return DK_ERR_UNSUPPORTED;
-  if (lo_inkernel && tl.pair) return DK_ERR_INVALID_ARG;      // (the caller asked tc_fwd_lo_inkernel first)
   if (gt_cnt >= 0) {
     // this launch covers group tiles [gt_lo, gt_lo + gt_cnt) only
     if (gt_lo < 0 || gt_cnt < 1 || gt_lo + gt_cnt > tl.GT) return DK_ERR_INVALID_ARG;

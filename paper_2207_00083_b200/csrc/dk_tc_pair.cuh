@@ -44,6 +44,24 @@ __device__ __forceinline__ uint32_t mapa_shared(uint32_t local, uint32_t rank) {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// bounded wait on a local barrier that the peer CTA's threads arrive on too (their writes to their own
+// shared memory, which the pair's tensor-core instruction reads, must be visible: cluster scope)
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned cap) {
+  for (unsigned i = 0; i < cap; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
 // TMA loads of a CTA pair: the data lands in the issuing CTA's shared memory,
 // the bytes are counted on the barrier at cluster address `bar` (the leader's).
 __device__ __forceinline__ void tma_pair_load_3d(void* dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
@@ -107,7 +125,11 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
   uint64_t* empty_bar = full_bar + kMaxStages;
   uint64_t* tfull_bar = empty_bar + kMaxStages;
   uint64_t* tempty_bar = tfull_bar + 2;                       // used in the leader only
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  // with the second TF32 term derived in the kernel: a CTA's own activation box has landed (transaction bytes),
+  // and, in the leader, both CTAs' converter warps have derived the second term of a stage (4 arrivals)
+  uint64_t* bfull_bar = tempty_bar + 2;
+  uint64_t* ready_bar = bfull_bar + kMaxStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ready_bar + kMaxStages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -116,7 +138,9 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
   const int nwork = p.ntiles * p.ksplit;     // work item = (pair tile, contraction slice)
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.nstages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
+    for (int s = 0; s < p.nstages; ++s) {
+      mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); mbar_init(bfull_bar + s, 1); mbar_init(ready_bar + s, 4);
+    }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + b, 1); mbar_init(tempty_bar + b, 2 * kEpiWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -156,7 +180,10 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         int ok = 1;
         if (lane == 0) {
           ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
-          if (ok && rank == 0) mbar_expect_tx(full_bar + stage, (uint32_t)(2 * (STAGE_BYTES - (p.nprod == 2 ? A_BYTES : 0))));
+          if (ok && rank == 0)
+            mbar_expect_tx(full_bar + stage, (uint32_t)(2 * (STAGE_BYTES - (p.nprod == 2 ? A_BYTES : 0) -
+                                                             (p.lo_inkernel ? 2 * B_BYTES : 0))));
+          if (ok && p.lo_inkernel) mbar_expect_tx(bfull_bar + stage, (uint32_t)B_BYTES);
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) { alive = false; break; }
@@ -171,15 +198,23 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
           if (p.nprod == 3) tma_pair_load_3d(st + A_BYTES, &map_a_lo, bar, c0, tap, m0);
         } else if (p.b_onebox) {
           // one box over this CTA's half of the encodings per TF32 term (see tc_fwd_kernel)
-          if (lane == 2) tma_pair_load_5d(st + 2 * A_BYTES, &map_b_hi, bar, c0, x0 + v, y0 + u, (int)rank * EH, g0);
-          else if (lane == 3)
+          if (lane == 2) {
+            // (second term derived here: the box is counted on this CTA's own barrier, for its converter warps)
+            const uint32_t bbar = p.lo_inkernel ? mapa_shared(smem_u32(bfull_bar + stage), rank) : bar;
+            tma_pair_load_5d(st + 2 * A_BYTES, &map_b_hi, bbar, c0, x0 + v, y0 + u, (int)rank * EH, g0);
+          } else if (lane == 3 && !p.lo_inkernel) {
             tma_pair_load_5d(st + 2 * A_BYTES + B_BYTES, &map_b_lo, bar, c0, x0 + v, y0 + u, (int)rank * EH, g0);
+          }
         } else if (lane < 2 + 2 * EH) {
           const int i = (lane - 2) >> 1;
           const int e = (int)rank * EH + i;
+          // (second term derived here: the boxes are counted on this CTA's own barrier, and none is fetched for
+          // the second term; the transaction bytes each barrier expects are set accordingly above)
           if ((lane & 1) == 0)
-            tma_pair_load_5d(st + 2 * A_BYTES + i * SUB, &map_b_hi, bar, c0, x0 + v, y0 + u, e, g0);
-          else
+            tma_pair_load_5d(st + 2 * A_BYTES + i * SUB, &map_b_hi,
+                             p.lo_inkernel ? mapa_shared(smem_u32(bfull_bar + stage), rank) : bar, c0, x0 + v, y0 + u, e,
+                             g0);
+          else if (!p.lo_inkernel)
             tma_pair_load_5d(st + 2 * A_BYTES + B_BYTES + i * SUB, &map_b_lo, bar, c0, x0 + v, y0 + u, e, g0);
         }
         __syncwarp();
@@ -208,6 +243,8 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
           const int kb_beg = kb_lo + ci * chunk, kb_end = min(kb_hi, kb_beg + chunk);
           for (int kb = kb_beg; kb < kb_end; ++kb) {
             if (!mbar_wait(full_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
+            // (both CTAs' activation boxes have landed and their second terms are derived)
+            if (p.lo_inkernel && !mbar_wait_cluster(ready_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
             tc_fence_after();
             const uint32_t st = smem_u32(smem + (size_t)stage * STAGE_BYTES);
             const uint64_t a_hi = make_desc<SWZ>(st), a_lo = make_desc<SWZ>(st + A_BYTES);
@@ -226,6 +263,37 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
           }
           if (alive) tc_pair_commit(tfull_bar + buf);
         }
+      }
+    }
+  } else if (p.lo_inkernel && warp >= 2) {
+    // ---------------- converters: warps 2 and 3 of both CTAs ----------------
+    // second TF32 term of this CTA's half of the stage's activations (see tc_fwd_kernel); done is reported to
+    // the leader, whose MMA thread issues for both CTAs
+    const int ctid = (int)threadIdx.x - 64;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool alive = true;
+    for (int w = pair; alive && w < nwork; w += npairs) {
+      const int ks = w % p.ksplit;
+      const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
+      for (int kb = kb_lo; kb < kb_hi; ++kb) {
+        if (!mbar_wait(bfull_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
+        const float4* src = reinterpret_cast<const float4*>(smem + (size_t)stage * STAGE_BYTES + 2 * A_BYTES);
+        float4* dst = reinterpret_cast<float4*>(smem + (size_t)stage * STAGE_BYTES + 2 * A_BYTES + B_BYTES);
+#pragma unroll 4
+        for (int i = ctid; i < B_BYTES / 16; i += 64) {
+          const float4 v = src[i];
+          float4 l;
+          l.x = to_tf32(v.x - __uint_as_float(__float_as_uint(v.x) & 0xffffe000u));
+          l.y = to_tf32(v.y - __uint_as_float(__float_as_uint(v.y) & 0xffffe000u));
+          l.z = to_tf32(v.z - __uint_as_float(__float_as_uint(v.z) & 0xffffe000u));
+          l.w = to_tf32(v.w - __uint_as_float(__float_as_uint(v.w) & 0xffffe000u));
+          dst[i] = l;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(ready_bar + stage), 0u));
+        if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
       }
     }
   }
