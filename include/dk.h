@@ -199,6 +199,11 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  *                     through a pipeline of two to four stages), which outweighs the
  *                     shorter pre-pass.  2: only in the CTA-pair kernel.  Needs
  *                     DK_OPT_XBAR_HI = 1.
+ *   DK_OPT_TC_SPLIT_RING  1 (default): the single-CTA forward kernel keeps the W tiles and
+ *                     the activations of its k-blocks in two rings of shared-memory
+ *                     slots filled by two producer warps, the activations' ring one
+ *                     slot deeper (two and three slots for K = 4, where three whole
+ *                     stages do not fit); 0: one ring of whole stages.
  *   DK_OPT_WG_PACE    1 (default): the persistent CTAs of the tensor-core weight-gradient
  *                     kernel start each round of work items together (a bounded wait
  *                     on a device counter, a hint only), so that the items that read
@@ -232,7 +237,7 @@ enum {
   DK_OPT_WG_PAIR = 5, DK_OPT_TC_STEM = 6, DK_OPT_FIELD_PATH = 7, DK_OPT_SPIN_LIMIT = 8,
   DK_OPT_TEST_WITHHOLD = 9, DK_OPT_XBAR_HI = 10, DK_OPT_TC_MPACK = 11, DK_OPT_SLABS = 12, DK_OPT_SLABS_FORCE = 13,
   DK_OPT_TC_CHUNK_ADAPT = 14, DK_OPT_WG_PACE = 15, DK_OPT_TC_LO_INKERNEL = 16,
-  DK_OPT_COUNT = 17
+  DK_OPT_TC_SPLIT_RING = 17, DK_OPT_COUNT = 18
 };
 DK_API dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value);
 DK_API dk_status dk_get_option(dk_ctx* ctx, int32_t option, int32_t* value);

@@ -162,6 +162,8 @@ encode_split_kernel(const float* __restrict__ x, const float* __restrict__ r, co
 // ---------------------------------------------------------------------------
 struct Tiling {
   int P, bw, bh, bg, WT, HT, GT, MT, ntiles, KB, CB, nstages, BN;
+  int nstages_b;           // single-CTA kernel: slots of a separate ring for the activations (0: one ring)
+  size_t smem_one_ring;    // dynamic shared memory of the one-ring layout (the kernel derives the second term itself)
   bool mpack;              // two output rows of the image in one 128-row tile (cout <= 64)
   bool pair;               // tiles of 256 output channels on CTA pairs
   size_t smem_bytes;
@@ -210,6 +212,20 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
   if (ns < 2) return false;
   t->nstages = ns;
   t->smem_bytes = (size_t)ns * stage + ctrl;
+  t->smem_one_ring = t->smem_bytes;
+  t->nstages_b = 0;
+  if (!pair) {
+    // Two rings: the W tiles keep `ns` slots, the activations (the larger part of a k-block) get one more when it
+    // fits: their copies then run a k-block further ahead.  Measured with a three-slot ring for everything
+    // (possible in the two-product mode only): 27-30 % faster kernels than with two slots; the one- and
+    // two-slot hand-over is what the single-CTA kernel loses against its tensor and copy floors.
+    const size_t a2 = 2 * (size_t)BM * BK * 4, b2 = 2 * (size_t)t->BN * BK * 4;
+    int nb = ns + 1;
+    if (nb <= kMaxStages && (size_t)ns * a2 + (size_t)nb * b2 + ctrl + fixed <= (size_t)smem_optin) {
+      t->nstages_b = nb;
+      t->smem_bytes = (size_t)ns * a2 + (size_t)nb * b2 + ctrl;
+    }
+  }
   return true;
 }
 
@@ -330,6 +346,7 @@ void fill_params(const TcState* ts, const Geom& g, const Tiling& tl, TcParams* p
   p->withhold = ts->opt->v[DK_OPT_TEST_WITHHOLD];
   p->nprod = g.nprod == 2 ? 2 : 3;
   p->lo_inkernel = 0;
+  p->nstages_b = ts->opt->v[DK_OPT_TC_SPLIT_RING] ? tl.nstages_b : 0;
   p->b_onebox = tl.bg == 1 ? 1 : 0;
   p->hmul = tl.mpack ? 2 : 1;
   ts->opt->v[DK_OPT_TEST_WITHHOLD] = -1;      // the hook serves one launch
@@ -544,6 +561,7 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   prm.out = ybar;
   if (chunk_cap > 0 && prm.chunk > chunk_cap * (32 / fwd_bk(ts))) prm.chunk = chunk_cap * (32 / fwd_bk(ts));
   prm.lo_inkernel = lo_inkernel ? 1 : 0;
+  if (lo_inkernel) prm.nstages_b = 0;      // (the converter warps work on the one-ring layout)
   prm.status = status_word;
   return launch_bk<MODE_YBAR>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
 }
@@ -565,6 +583,7 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   fill_params(ts, g, tl, &prm);
   if (gt_cnt >= 0) prm.gt0 = gt_lo;
   prm.lo_inkernel = lo_inkernel ? 1 : 0;
+  if (lo_inkernel) prm.nstages_b = 0;      // (the converter warps work on the one-ring layout)
   prm.out = y;
   prm.dec = cv.dec; prm.decl = cv.decl; prm.nul = cv.nul; prm.bias = bias;
   // ill-conditioned coefficient sets take shorter chunks (see upload_coefficients): per virtual batch where the

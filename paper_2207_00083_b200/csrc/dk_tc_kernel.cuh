@@ -66,6 +66,9 @@ struct TcParams {
   int ksplit, kb_per_split;    // contraction slices per tile (slices add into `out` with atomics)
   int kw, pad, stride;
   int nstages;
+  int nstages_b;               // single-CTA forward kernel: 0 = one ring of stages (W tiles and activations together);
+                               // n > 0 = two rings, `nstages` slots for the W tiles and n slots for the activations,
+                               // filled by two producer warps (the activations run one k-block further ahead)
   unsigned spin_cap;           // polls after which a wait gives up
   int withhold;                // test hook: the producer arms its n-th stage but issues no copy (-1 = off)
   int hmul;                    // 2: the tile's rows 64-127 are the image row below rows 0-63 (cout <= 64), else 1
@@ -523,13 +526,21 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
   load_chunk_tab(p, s_chunk);
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                          ~static_cast<uintptr_t>(1023));
-  unsigned char* ctrl = smem + (size_t)p.nstages * STAGE_BYTES;
+  // One ring: stage s = [W_hi][W_lo][x_hi][x_lo] at s * STAGE_BYTES.  Two rings: the W tiles' slots first, then the
+  // activations' slots.
+  const bool split = p.nstages_b > 0;
+  unsigned char* const b_base = split ? smem + (size_t)p.nstages * 2 * A_BYTES : smem + 2 * A_BYTES;
+  const size_t a_pitch = split ? (size_t)2 * A_BYTES : (size_t)STAGE_BYTES;
+  const size_t b_pitch = split ? (size_t)2 * B_BYTES : (size_t)STAGE_BYTES;
+  unsigned char* ctrl = split ? b_base + (size_t)p.nstages_b * 2 * B_BYTES : smem + (size_t)p.nstages * STAGE_BYTES;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(ctrl);
   uint64_t* empty_bar = full_bar + kMaxStages;
   uint64_t* tfull_bar = empty_bar + kMaxStages;
   uint64_t* tempty_bar = tfull_bar + 2;
   uint64_t* ready_bar = tempty_bar + 2;        // a stage's second term has been derived (one arrival per converter warp)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ready_bar + kMaxStages);
+  uint64_t* bfull_bar = ready_bar + kMaxStages;      // the activations' ring, when there are two
+  uint64_t* bempty_bar = bfull_bar + kMaxStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bempty_bar + kMaxStages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -539,6 +550,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
     for (int s = 0; s < p.nstages; ++s) {
       mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); mbar_init(ready_bar + s, 2);
     }
+    for (int s = 0; s < p.nstages_b; ++s) { mbar_init(bfull_bar + s, 1); mbar_init(bempty_bar + s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + b, 1); mbar_init(tempty_bar + b, kEpiWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -561,12 +573,18 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
   static_assert(40 * 128 + 232 * 256 <= 168 * kThreadsTc, "setmaxnreg budget exceeds the CTA's register pool");
   if (warp < 4) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
-  if (warp == 0) {
-    // ---------------- TMA producer ----------------
-    // The whole warp runs the loop: lane 0 waits for the stage and arms its
-    // barrier, then lanes 0..2E+1 issue one bulk tensor copy each, so that the
-    // 2E+2 copies of a stage are issued side by side instead of one after another.
+  if (warp == 0 || (warp == 2 && split)) {
+    // ---------------- TMA producer(s) ----------------
+    // The whole warp runs the loop: lane 0 waits for the slot and arms its barrier, then one lane per copy
+    // issues it, so that the copies of a k-block go out side by side.  One ring: warp 0 fetches everything.
+    // Two rings: warp 0 fetches the W tiles into theirs, warp 2 the activations into theirs.
     {
+      const bool do_a = warp == 0, do_b = !split || warp == 2;
+      uint64_t* const fbar = (split && warp == 2) ? bfull_bar : full_bar;
+      uint64_t* const ebar = (split && warp == 2) ? bempty_bar : empty_bar;
+      const int nst = (split && warp == 2) ? p.nstages_b : p.nstages;
+      const uint32_t tx = (do_a ? (uint32_t)(p.nprod == 2 ? A_BYTES : 2 * A_BYTES) : 0u) +
+                          (do_b ? (uint32_t)(p.lo_inkernel ? B_BYTES : 2 * B_BYTES) : 0u);
       int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool alive = true;
@@ -583,37 +601,37 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
         for (int kb = kb_lo; kb < kb_hi; ++kb) {
           int ok = 1;
           if (lane == 0) {
-            ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
-            if (ok) mbar_expect_tx(full_bar + stage, (uint32_t)(STAGE_BYTES - (p.nprod == 2 ? A_BYTES : 0) -
-                                                                (p.lo_inkernel ? B_BYTES : 0)));
+            ok = mbar_wait(ebar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
+            if (ok) mbar_expect_tx(fbar + stage, tx);
           }
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) { alive = false; break; }
-          if (issued++ == p.withhold) { alive = false; break; }      // test hook: armed, nothing copied
+          if (do_a && issued++ == p.withhold) { alive = false; break; }      // test hook: armed, nothing copied
           const int tap = kb / p.CB, c0 = (kb - tap * p.CB) * BK;
           const int u = tap / p.kw, v = tap - u * p.kw;
-          unsigned char* st = smem + (size_t)stage * STAGE_BYTES;
+          unsigned char* sta = smem + (size_t)stage * a_pitch;
+          unsigned char* stb = b_base + (size_t)stage * b_pitch;
           constexpr int SUB = P * BK * 4;
           if (lane == 0) {
-            tma_load_3d(st, &map_a_hi, full_bar + stage, c0, tap, m0);
+            if (do_a) tma_load_3d(sta, &map_a_hi, fbar + stage, c0, tap, m0);
           } else if (lane == 1) {
-            if (p.nprod == 3) tma_load_3d(st + A_BYTES, &map_a_lo, full_bar + stage, c0, tap, m0);
+            if (do_a && p.nprod == 3) tma_load_3d(sta + A_BYTES, &map_a_lo, fbar + stage, c0, tap, m0);
+          } else if (!do_b) {
           } else if (p.b_onebox) {
             // (same bytes at the same places as the E boxes below: with one group per tile the encoding is the
             // slowest dimension of the stage either way; fewer copies measured 4-7 % faster)
-            if (lane == 2) tma_load_5d(st + 2 * A_BYTES, &map_b_hi, full_bar + stage, c0, x0 + v, y0 + u, 0, g0);
+            if (lane == 2) tma_load_5d(stb, &map_b_hi, fbar + stage, c0, x0 + v, y0 + u, 0, g0);
             else if (lane == 3 && !p.lo_inkernel)
-              tma_load_5d(st + 2 * A_BYTES + B_BYTES, &map_b_lo, full_bar + stage, c0, x0 + v, y0 + u, 0, g0);
+              tma_load_5d(stb + B_BYTES, &map_b_lo, fbar + stage, c0, x0 + v, y0 + u, 0, g0);
           } else if (lane < 2 + 2 * E) {
             const int e = (lane - 2) >> 1;
             if ((lane & 1) == 0)
-              tma_load_5d(st + 2 * A_BYTES + e * SUB, &map_b_hi, full_bar + stage, c0, x0 + v, y0 + u, e, g0);
+              tma_load_5d(stb + e * SUB, &map_b_hi, fbar + stage, c0, x0 + v, y0 + u, e, g0);
             else if (!p.lo_inkernel)
-              tma_load_5d(st + 2 * A_BYTES + B_BYTES + e * SUB, &map_b_lo, full_bar + stage, c0, x0 + v, y0 + u,
-                          e, g0);
+              tma_load_5d(stb + B_BYTES + e * SUB, &map_b_lo, fbar + stage, c0, x0 + v, y0 + u, e, g0);
           }
           __syncwarp();
-          if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+          if (++stage == nst) { stage = 0; phase ^= 1u; }
         }
       }
     }
@@ -622,8 +640,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
     if (lane == 0) {
       constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) |
                                  ((uint32_t)(BM >> 4) << 24);
-      int stage = 0;
-      uint32_t phase = 0;
+      int stage = 0, stage_b = 0;
+      uint32_t phase = 0, phase_b = 0;
       uint32_t acc_it = 0;     // chunks issued so far (all tiles)
       bool alive = true;
       for (int w = blockIdx.x; alive && w < nwork; w += gridDim.x) {
@@ -639,11 +657,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
           const int kb_beg = kb_lo + ci * chunk, kb_end = min(kb_hi, kb_beg + chunk);
           for (int kb = kb_beg; kb < kb_end; ++kb) {
             if (!mbar_wait(full_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
+            if (split && !mbar_wait(bfull_bar + stage_b, phase_b, abort_flag, p.spin_cap)) { alive = false; break; }
             tc_fence_after();
-            const uint32_t st = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-            const uint64_t a_hi = make_desc<SWZ>(st), a_lo = make_desc<SWZ>(st + A_BYTES);
-            const uint64_t b_hi = make_desc<SWZ>(st + 2 * A_BYTES);
-            const uint64_t b_lo = make_desc<SWZ>(st + 2 * A_BYTES + B_BYTES);
+            const uint32_t sta = smem_u32(smem + (size_t)stage * a_pitch);
+            const uint32_t stb = smem_u32(b_base + (size_t)(split ? stage_b : stage) * b_pitch);
+            const uint64_t a_hi = make_desc<SWZ>(sta), a_lo = make_desc<SWZ>(sta + A_BYTES);
+            const uint64_t b_hi = make_desc<SWZ>(stb);
+            const uint64_t b_lo = make_desc<SWZ>(stb + B_BYTES);
             const bool first = kb == kb_beg;
             // the products that need only what the copies brought go first; the one with the activations' second
             // term follows, after the converter warps have derived it (when they do)
@@ -664,6 +684,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
             }
             tc_commit(empty_bar + stage);
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+            if (split) {
+              tc_commit(bempty_bar + stage_b);
+              if (++stage_b == p.nstages_b) { stage_b = 0; phase_b ^= 1u; }
+            }
           }
           if (alive) tc_commit(tfull_bar + buf);
         }
@@ -682,8 +706,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
       const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
       for (int kb = kb_lo; kb < kb_hi; ++kb) {
         if (!mbar_wait(full_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
-        const float4* src = reinterpret_cast<const float4*>(smem + (size_t)stage * STAGE_BYTES + 2 * A_BYTES);
-        float4* dst = reinterpret_cast<float4*>(smem + (size_t)stage * STAGE_BYTES + 2 * A_BYTES + B_BYTES);
+        const float4* src = reinterpret_cast<const float4*>(b_base + (size_t)stage * b_pitch);
+        float4* dst = reinterpret_cast<float4*>(b_base + (size_t)stage * b_pitch + B_BYTES);
 #pragma unroll 4
         for (int i = ctid; i < B_BYTES / 16; i += 64) {
           const float4 v = src[i];
