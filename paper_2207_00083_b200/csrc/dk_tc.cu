@@ -754,12 +754,26 @@ bool plan_wgrad(const Options& opt, const Geom& g, int smem_optin, int sm_count,
   p.withhold = -1;
   p.cout = g.cout; p.cin = g.cin;
   const size_t stage = 2 * ((size_t)(BM / 32) * kWgBox + (size_t)((w->pair ? w->BN / 2 : w->BN) / 32) * kWgBox);
-  const size_t ctrl = 1024 + 256;
+  const size_t ctrl = 1024 + 512;
   int ns = (int)(((size_t)smem_optin - ctrl) / stage);
   if (ns > kMaxStages) ns = kMaxStages;
   if (ns < 2) return false;
   p.nstages = ns;
+  p.nstages_b = 0;
   w->smem_bytes = (size_t)ns * stage + ctrl;
+  if (!w->pair && opt.v[DK_OPT_TC_SPLIT_RING]) {
+    // two rings (see the forward kernel's plan): one more slot for the encodings when that fits, else one more
+    // for the gradients
+    const size_t a2 = 2 * (size_t)(BM / 32) * kWgBox, b2 = 2 * (size_t)(w->BN / 32) * kWgBox;
+    if ((size_t)ns * a2 + (size_t)(ns + 1) * b2 + ctrl <= (size_t)smem_optin && ns + 1 <= kMaxStages) {
+      p.nstages_b = ns + 1;
+      w->smem_bytes = (size_t)ns * a2 + (size_t)(ns + 1) * b2 + ctrl;
+    } else if ((size_t)(ns + 1) * a2 + (size_t)ns * b2 + ctrl <= (size_t)smem_optin && ns + 1 <= kMaxStages) {
+      p.nstages = ns + 1;
+      p.nstages_b = ns;
+      w->smem_bytes = (size_t)(ns + 1) * a2 + (size_t)ns * b2 + ctrl;
+    }
+  }
   return true;
 }
 

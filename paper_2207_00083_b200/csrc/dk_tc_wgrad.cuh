@@ -45,6 +45,8 @@ struct WgTcParams {
   int nitems;                  // MT*NB*taps*nsplit
   int kw, pad, stride;
   int nstages, chunk;
+  int nstages_b;               // single-CTA kernel: 0 = one ring of stages; n > 0 = two rings, `nstages` slots for the
+                               // gradients and n for the encodings, filled by two producer warps
   unsigned spin_cap;           // polls after which a wait gives up
   int withhold;                // test hook: the producer arms its n-th stage but issues no copy (-1 = off)
   int mpack;                   // cout <= 64: rows 64-127 of the tile are the gradients one image row below rows 0-63
@@ -85,12 +87,20 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                          ~static_cast<uintptr_t>(1023));
-  unsigned char* ctrl = smem + (size_t)p.nstages * STAGE_BYTES;
+  // One ring: stage s = [d_hi][d_lo][x_hi][x_lo] at s * STAGE_BYTES.  Two rings (single CTA only): the gradients'
+  // slots first, then the encodings' slots.
+  const bool split = !PAIR && p.nstages_b > 0;
+  unsigned char* const b_base = split ? smem + (size_t)p.nstages * 2 * A_BYTES : smem + 2 * A_BYTES;
+  const size_t a_pitch = split ? (size_t)2 * A_BYTES : (size_t)STAGE_BYTES;
+  const size_t b_pitch = split ? (size_t)2 * B_BYTES : (size_t)STAGE_BYTES;
+  unsigned char* ctrl = split ? b_base + (size_t)p.nstages_b * 2 * B_BYTES : smem + (size_t)p.nstages * STAGE_BYTES;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(ctrl);
   uint64_t* empty_bar = full_bar + kMaxStages;
   uint64_t* tfull_bar = empty_bar + kMaxStages;
   uint64_t* tempty_bar = tfull_bar + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  uint64_t* bfull_bar = tempty_bar + 2;              // the encodings' ring, when there are two
+  uint64_t* bempty_bar = bfull_bar + kMaxStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bempty_bar + kMaxStages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -100,6 +110,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.nstages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
+    for (int s = 0; s < (split ? p.nstages_b : 0); ++s) { mbar_init(bfull_bar + s, 1); mbar_init(bempty_bar + s, 1); }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar + b, 1);
       mbar_init(tempty_bar + b, PAIR ? 2 * kEpiWarps : kEpiWarps);     // a pair's chunks are released on the leader
@@ -144,10 +155,16 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
   static_assert(40 * 128 + 232 * 256 <= 168 * kThreadsTc, "setmaxnreg budget exceeds the CTA's register pool");
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
-    if (warp == 0) {
-      // ---------------- TMA producer ----------------
+    if (warp == 0 || (warp == 2 && split)) {
+      // ---------------- TMA producer(s) ----------------
+      // (two rings: warp 0 fetches the gradients into theirs, warp 2 the encodings into theirs)
       // whole warp: lane 0 arms the stage, then each lane issues its share of
       // the 2*(BM+BN)/32 box copies so that they go out side by side
+      const bool do_a = warp == 0, do_b = !split || warp == 2;
+      uint64_t* const fbar = (split && warp == 2) ? bfull_bar : full_bar;
+      uint64_t* const ebar = (split && warp == 2) ? bempty_bar : empty_bar;
+      const int nst = (split && warp == 2) ? p.nstages_b : p.nstages;
+      const uint32_t tx = (uint32_t)(PAIR ? 2 : 1) * ((do_a ? 2u * A_BYTES : 0u) + (do_b ? 2u * B_BYTES : 0u));
       int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool alive = true;
@@ -161,7 +178,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
         // of items lose that (measured: DRAM traffic of three passes over the operands where one would do), so a
         // CTA starts round r only when all have issued the loads of round r-1, or after a bounded wait: this is
         // a hint, never a condition for progress.
-        if (p.pace != nullptr && round > 0 && lane == 0 && rank == 0) {
+        if (p.pace != nullptr && round > 0 && lane == 0 && rank == 0 && do_a) {
           const unsigned int target = (unsigned int)round * (unsigned int)item_step;
           for (int spin = 0; spin < 4096 && *reinterpret_cast<volatile unsigned int*>(p.pace) < target; ++spin)
             __nanosleep(128);
@@ -198,39 +215,40 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
           for (int j = 0; j < p.K1; ++j) {
             int ok = 1;
             if (lane == 0) {
-              ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
+              ok = mbar_wait(ebar + stage, phase ^ 1u, abort_flag, p.spin_cap) ? 1 : 0;
               // the bytes of both CTAs of a pair are counted on the leader's barrier
-              if (ok && rank == 0) mbar_expect_tx(full_bar + stage, (uint32_t)((PAIR ? 2 : 1) * STAGE_BYTES));
+              if (ok && rank == 0) mbar_expect_tx(fbar + stage, tx);
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) { alive = false; break; }
-            if (issued++ == p.withhold) { alive = false; break; }      // test hook: armed, nothing copied
-            unsigned char* st = smem + (size_t)stage * STAGE_BYTES;
+            if (do_a && issued++ == p.withhold) { alive = false; break; }      // test hook: armed, nothing copied
+            unsigned char* sta = smem + (size_t)stage * a_pitch;
+            unsigned char* stb = b_base + (size_t)stage * b_pitch;
             const uint32_t pbar = PAIR ? mapa_shared(smem_u32(full_bar + stage), 0u) : 0u;
             auto load = [&](void* dst, const CUtensorMap* map, int c0, int c1, int c2) {
               if constexpr (PAIR) tma_pair_load_5d(dst, map, pbar, c0, c1, c2, j, g0);
-              else tma_load_5d(dst, map, full_bar + stage, c0, c1, c2, j, g0);
+              else tma_load_5d(dst, map, fbar + stage, c0, c1, c2, j, g0);
             };
             if (lane < 2 * (BM / 32)) {
               const int cb = lane >> 1;
               // two-row tiles: channel blocks 2 and 3 are channels 0..63 of the gradients one row below
               const int ch = (p.mpack && cb >= 2) ? (cb - 2) * 32 : m0 + cb * 32;
               const int yy = (p.mpack && cb >= 2) ? y0 + 1 : y0;
-              if ((lane & 1) == 0) load(st + cb * kWgBox, &map_d_hi, ch, x0, yy);
-              else load(st + A_BYTES + cb * kWgBox, &map_d_lo, ch, x0, yy);
-            } else if (lane < NBOX) {
+              if (!do_a) {
+              } else if ((lane & 1) == 0) load(sta + cb * kWgBox, &map_d_hi, ch, x0, yy);
+              else load(sta + A_BYTES + cb * kWgBox, &map_d_lo, ch, x0, yy);
+            } else if (lane < NBOX && do_b) {
               const int q = lane - 2 * (BM / 32);
               const int cb = q >> 1;
-              unsigned char* bh = st + 2 * A_BYTES;
               const int xi = x0 * p.stride + bx_v - p.pad, yi = y0 * p.stride + bx_u - p.pad;   // input position
-              if ((q & 1) == 0) load(bh + cb * kWgBox, &map_x_hi, bx_c, xi, yi);
-              else load(bh + B_BYTES + cb * kWgBox, &map_x_lo, bx_c, xi, yi);
+              if ((q & 1) == 0) load(stb + cb * kWgBox, &map_x_hi, bx_c, xi, yi);
+              else load(stb + B_BYTES + cb * kWgBox, &map_x_lo, bx_c, xi, yi);
             }
             __syncwarp();
-            if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+            if (++stage == nst) { stage = 0; phase ^= 1u; }
           }
         }
-        if (p.pace != nullptr && alive && lane == 0 && rank == 0) atomicAdd(p.pace, 1u);
+        if (p.pace != nullptr && alive && lane == 0 && rank == 0 && do_a) atomicAdd(p.pace, 1u);
       }
     } else if (warp == 1 && lane == 0 && rank == 0) {
       // ---------------- MMA issuer (of a pair: the leader only) ----------------
@@ -244,8 +262,8 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
         if constexpr (PAIR) tc_pair_commit(bar);
         else tc_commit(bar);
       };
-      int stage = 0;
-      uint32_t phase = 0;
+      int stage = 0, stage_b = 0;
+      uint32_t phase = 0, phase_b = 0;
       uint32_t acc_it = 0;
       bool alive = true;
       for (int item = first_item; alive && item < p.nitems; item += item_step) {
@@ -261,11 +279,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
           const int kb_end = min(KB, (ci + 1) * p.chunk);
           for (int kb = ci * p.chunk; kb < kb_end; ++kb) {
             if (!mbar_wait(full_bar + stage, phase, abort_flag, p.spin_cap)) { alive = false; break; }
+            if (split && !mbar_wait(bfull_bar + stage_b, phase_b, abort_flag, p.spin_cap)) { alive = false; break; }
             tc_fence_after();
-            const uint32_t st = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-            const uint64_t a_hi = make_desc_mn(st, kWgBox), a_lo = make_desc_mn(st + A_BYTES, kWgBox);
-            const uint64_t b_hi = make_desc_mn(st + 2 * A_BYTES, kWgBox);
-            const uint64_t b_lo = make_desc_mn(st + 2 * A_BYTES + B_BYTES, kWgBox);
+            const uint32_t sta = smem_u32(smem + (size_t)stage * a_pitch);
+            const uint32_t stb = smem_u32(b_base + (size_t)(split ? stage_b : stage) * b_pitch);
+            const uint64_t a_hi = make_desc_mn(sta, kWgBox), a_lo = make_desc_mn(sta + A_BYTES, kWgBox);
+            const uint64_t b_hi = make_desc_mn(stb, kWgBox);
+            const uint64_t b_lo = make_desc_mn(stb + B_BYTES, kWgBox);
             const bool first = kb == ci * p.chunk;
 #pragma unroll
             for (int kk = 0; kk < kWgPix / 8; ++kk) {
@@ -276,6 +296,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap map_d_hi, const __grid_const
             }
             commit(empty_bar + stage);
             if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+            if (split) {
+              commit(bempty_bar + stage_b);
+              if (++stage_b == p.nstages_b) { stage_b = 0; phase_b ^= 1u; }
+            }
           }
           if (alive) commit(tfull_bar + buf);
         }
