@@ -34,7 +34,8 @@
  *    K_p private inputs followed by the first M - 1 noise vectors in x, the
  *    M-th noise vector in r, and pass C[g] = [A^T; redundant row] with
  *    A = [A1; A2].  Rows K_p..K-1 of each group's y then hold <W, r_m>
- *    (to be dropped), and dk_linear_bwd_wgrad takes zero deltas for those rows.
+ *    (to be dropped; with option DK_OPT_NOISE_ROWS = M - 1 they are not even
+ *    computed or stored), and dk_linear_bwd_wgrad takes zero deltas for those rows.
  *    K_p + M - 1 <= DK_MAX_K.
  *  - An integrity violation is a RESULT (dk_verdict.ok = 0), not an error:
  *    the call still returns DK_OK.
@@ -204,6 +205,13 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  *                     slots filled by two producer warps, the activations' ring one
  *                     slot deeper (two and three slots for K = 4, where three whole
  *                     stages do not fit); 0: one ring of whole stages.
+ *   DK_OPT_NOISE_ROWS default 0.  n > 0: the last n of the K inputs of every virtual batch
+ *                     are noise vectors (the relabelling of Section 4.5's colluding-
+ *                     accelerator scheme onto these calls, see above): dk_masked_linear
+ *                     and dk_decode_verify neither compute nor store the decoded rows
+ *                     of those inputs (rows K-n .. K-1 of each group of y are left as
+ *                     they were); encoding, the products and the integrity check are
+ *                     unchanged.  At most K-1.
  *   DK_OPT_WG_PACE    1 (default): the persistent CTAs of the tensor-core weight-gradient
  *                     kernel start each round of work items together (a bounded wait
  *                     on a device counter, a hint only), so that the items that read
@@ -237,7 +245,7 @@ enum {
   DK_OPT_WG_PAIR = 5, DK_OPT_TC_STEM = 6, DK_OPT_FIELD_PATH = 7, DK_OPT_SPIN_LIMIT = 8,
   DK_OPT_TEST_WITHHOLD = 9, DK_OPT_XBAR_HI = 10, DK_OPT_TC_MPACK = 11, DK_OPT_SLABS = 12, DK_OPT_SLABS_FORCE = 13,
   DK_OPT_TC_CHUNK_ADAPT = 14, DK_OPT_WG_PACE = 15, DK_OPT_TC_LO_INKERNEL = 16,
-  DK_OPT_TC_SPLIT_RING = 17, DK_OPT_COUNT = 18
+  DK_OPT_TC_SPLIT_RING = 17, DK_OPT_NOISE_ROWS = 18, DK_OPT_COUNT = 19
 };
 DK_API dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value);
 DK_API dk_status dk_get_option(dk_ctx* ctx, int32_t option, int32_t* value);

@@ -28,6 +28,7 @@ dk_status make_geom(const dk_problem* p, Geom* g) {
   g->E = p->K + 2;
   g->precision = (p->precision == DK_PREC_DEFAULT || p->precision == DK_TF32X2_WUNSPLIT) ? DK_TF32X3 : p->precision;
   g->nprod = p->precision == DK_TF32X2_WUNSPLIT ? 2 : 3;
+  g->kstore = p->K;
   g->tol = p->tol > 0.f ? p->tol : 1e-4f;
   if (p->kind == DK_FC) {
     g->h = g->w = g->kh = g->kw = g->stride = 1;
@@ -337,7 +338,7 @@ dk_status dk_create(dk_ctx** out, int device) {
     return DK_ERR_CUDA;
   }
   c->sm_count = sms;
-  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1, 1, 1, 0, 1, 1, 0, 1};
+  static const int kOptDefault[DK_OPT_COUNT] = {8, 2, 32, 1, 1, 1, 1, 0, 1 << 22, -1, 1, 1, 1, 0, 1, 1, 0, 1, 0};
   for (int i = 0; i < DK_OPT_COUNT; ++i) c->opt.v[i] = kOptDefault[i];
   bool ok = cudaMallocHost(&c->h_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
             cudaMalloc(&c->d_stage, kCoefSlots * kCoefSlotBytes) == cudaSuccess &&
@@ -381,10 +382,18 @@ dk_status dk_destroy(dk_ctx* c) {
   return DK_OK;
 }
 
+// Section 4.5 relabelling: the last DK_OPT_NOISE_ROWS inputs of every group are noise vectors, whose decoded
+// outputs are neither computed nor stored (at least one row stays).
+static void apply_noise_rows(const dk_ctx* ctx, Geom* g) {
+  int n = ctx->opt.v[DK_OPT_NOISE_ROWS];
+  if (n > g->K - 1) n = g->K - 1;
+  g->kstore = g->K - (n > 0 ? n : 0);
+}
+
 dk_status dk_set_option(dk_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx || option < 0 || option >= DK_OPT_COUNT) return DK_ERR_INVALID_ARG;
-  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0, 0, 1, 0, 0, 0, 0, 0};
-  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 3, 1 << 26, 1 << 20, 1, 1, kMaxSlabs, kMaxSlabs, 1, 1, 2, 1};
+  static const int lo[DK_OPT_COUNT] = {1, 1, 16, 0, 0, 0, 0, 0, 1 << 10, -1, 0, 0, 1, 0, 0, 0, 0, 0, 0};
+  static const int hi[DK_OPT_COUNT] = {64, 64, 32, 1, 1, 1, 2, 3, 1 << 26, 1 << 20, 1, 1, kMaxSlabs, kMaxSlabs, 1, 1, 2, 1, DK_MAX_K - 1};
   int v = value < lo[option] ? lo[option] : (value > hi[option] ? hi[option] : value);
   if (option == DK_OPT_TC_BK) v = v == 16 ? 16 : 32;
   ctx->opt.v[option] = v;
@@ -476,6 +485,7 @@ dk_status dk_decode_verify(dk_ctx* ctx, const dk_problem* p, const float* ybar,
   Geom g;
   dk_status s = make_geom(p, &g);
   if (s != DK_OK) return s;
+  apply_noise_rows(ctx, &g);
   DeviceGuard dg(ctx->device);
   if (!dg.ok) return DK_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -547,6 +557,7 @@ dk_status dk_masked_linear(dk_ctx* ctx, const dk_problem* p, const float* W, con
   Geom g;
   dk_status s = make_geom(p, &g);
   if (s != DK_OK) return s;
+  apply_noise_rows(ctx, &g);
   if (fault) {
     if (fault->group < 0 || fault->group >= g.G || fault->enc < 0 || fault->enc >= g.E ||
         fault->out_index < 0 || fault->out_index >= g.n_out)

@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(kThreads)
 decode_verify_kernel(const float* __restrict__ ybar, const float* __restrict__ dec,
                      const float* __restrict__ decl, const float* __restrict__ nul,
                      const float* __restrict__ bias, float* __restrict__ y, VerifyScratch vs,
-                     long long n, float tau, int cout, long long cdiv) {
+                     long long n, float tau, int cout, long long cdiv, int kstore) {
   constexpr int K1 = K + 1, E = K + 2;
   const int g = blockIdx.y;
   // One fp32 coefficient per term: the fp32 sum's own rounding is as large as
@@ -169,6 +169,7 @@ decode_verify_kernel(const float* __restrict__ ybar, const float* __restrict__ d
     }
 #pragma unroll
     for (int k = 0; k < K; ++k) {
+      if (k >= kstore) continue;      // (a noise vector in the place of a private input: its output is not wanted)
       f4 o;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
@@ -239,10 +240,10 @@ dk_status launch_dv(const Geom& g, const float* ybar, const CoefView& cv, const 
   long long cdiv = (g.layout == DK_NCHW && g.kind == DK_CONV2D) ? (long long)g.ho * g.wo : 1;
   if (g.n_out % 4 == 0)
     decode_verify_kernel<K, true><<<grid, kThreads, 0, st>>>(
-        ybar, cv.dec, cv.decl, cv.nul, bias, y, vs, g.n_out, g.tol, g.cout, cdiv);
+        ybar, cv.dec, cv.decl, cv.nul, bias, y, vs, g.n_out, g.tol, g.cout, cdiv, g.kstore);
   else
     decode_verify_kernel<K, false><<<grid, kThreads, 0, st>>>(
-        ybar, cv.dec, cv.decl, cv.nul, bias, y, vs, g.n_out, g.tol, g.cout, cdiv);
+        ybar, cv.dec, cv.decl, cv.nul, bias, y, vs, g.n_out, g.tol, g.cout, cdiv, g.kstore);
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
 }

@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(kThreads64)
 decode_verify64_kernel(const double* __restrict__ ybar, const float* __restrict__ dec,
                        const float* __restrict__ decl, const float* __restrict__ nul,
                        const float* __restrict__ bias, float* __restrict__ y, VerifyScratch vs,
-                       long long n, float tau, int cout, long long cdiv) {
+                       long long n, float tau, int cout, long long cdiv, int kstore) {
   constexpr int K1 = K + 1, E = K + 2;
   __shared__ float s_red[kThreads64 / 32][E + 1];
   const int g = blockIdx.y;
@@ -69,6 +69,7 @@ decode_verify64_kernel(const double* __restrict__ ybar, const float* __restrict_
     const double b = bias != nullptr ? (double)__ldg(bias + (e / cdiv) % cout) : 0.0;
 #pragma unroll
     for (int k = 0; k < K; ++k) {
+      if (k >= kstore) continue;      // (a noise vector in the place of a private input)
       double acc = 0.0;
 #pragma unroll
       for (int i = 0; i < K1; ++i) {
@@ -163,7 +164,7 @@ dk_status launch_decode_verify64(const Geom& g, const double* ybar, const CoefVi
   dim3 grid = grid_for(g.n_out, g.G, sm_count);
   const long long cdiv = (g.layout == DK_NCHW && g.kind == DK_CONV2D) ? (long long)g.ho * g.wo : 1;
   DK_K_SWITCH(g.K, (decode_verify64_kernel<KK><<<grid, kThreads64, 0, st>>>(
-                       ybar, cv.dec, cv.decl, cv.nul, bias, y, vs, g.n_out, g.tol, g.cout, cdiv)));
+                       ybar, cv.dec, cv.decl, cv.nul, bias, y, vs, g.n_out, g.tol, g.cout, cdiv, g.kstore)));
   DK_CUDA_CHECK(cudaGetLastError());
   return DK_OK;
 }

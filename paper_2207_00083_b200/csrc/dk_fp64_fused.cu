@@ -45,6 +45,7 @@ struct F64Params {
   int f_group, f_enc;
   long long f_index;          // pixel * cout + channel
   float f_delta;
+  int kstore;                 // decoded rows k >= kstore of a group are neither computed nor stored
 };
 
 __device__ __forceinline__ void dmma(double (&c)[2], double a, double b) {
@@ -172,6 +173,7 @@ __global__ void __launch_bounds__(kThreads, 3) fused64_kernel(const F64Params p)
       if (ok) {
 #pragma unroll
         for (int k = 0; k < K; ++k) {
+          if (k >= p.kstore) continue;
           double yv = 0.0;
 #pragma unroll
           for (int i = 0; i < K1; ++i) yv = fma(cdec[k * K1 + i], v[i], yv);
@@ -252,6 +254,7 @@ dk_status launch_fused64(const Geom& g, const float* W, const float* x, const fl
   p.mtiles = (g.cout + rows - 1) / rows;
   p.ntiles = (long long)p.tiles_per_g * g.G * p.mtiles;
   p.f_group = -1; p.f_enc = 0; p.f_index = -1; p.f_delta = 0.f;
+  p.kstore = g.kstore;
   if (fault) { p.f_group = fault->group; p.f_enc = fault->enc; p.f_index = fault->out_index; p.f_delta = fault->delta; }
   const int E = g.E, K1 = g.K + 1;
   const size_t smem = ((size_t)E * P * S + (size_t)rows * S + (size_t)E * K1 + (size_t)g.K * K1 + E) * sizeof(double);

@@ -21,6 +21,8 @@ struct Geom {
   int precision;
   int mpack;                // forward tensor-core kernel: two output rows of the image per 128-row tile (cout <= 64)
   int nprod;                // TF32 products per step of the forward tensor-core kernels: 3, or 2 (W as one term)
+  int kstore;               // decoded rows k < kstore of each group are computed and stored (K, or K minus the noise
+                            // vectors that stand in the place of private inputs, Section 4.5)
   float tol;
   // element strides of one sample: activation (channel, row, col), weights
   // (cout, cin, u, v), output (channel, row, col)

@@ -34,6 +34,7 @@ struct StemFwdParams {
   int f_group, f_enc;
   long long f_index;
   float f_delta;
+  int kstore;                  // decoded rows k >= kstore of a group are neither computed nor stored
 };
 
 template <int K>
@@ -148,6 +149,7 @@ __global__ void __launch_bounds__(kThreads, 2) stem_fwd_kernel(const StemFwdPara
       if (pix_ok) {
 #pragma unroll
         for (int k = 0; k < K; ++k) {
+          if (k >= p.kstore) continue;
           float yv[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) yv[j] = cdec[k * K1] * acc[0][j];
@@ -386,6 +388,7 @@ dk_status launch_stem_fwd(const Geom& g, const float* W, const float* x, const f
   p.tiles_w = (g.wo + kTileW - 1) / kTileW;
   p.ntiles = (long long)g.G * g.ho * p.tiles_w;
   p.f_group = -1; p.f_enc = 0; p.f_index = -1; p.f_delta = 0.f;
+  p.kstore = g.kstore;
   if (fault) { p.f_group = fault->group; p.f_enc = fault->enc; p.f_index = fault->out_index; p.f_delta = fault->delta; }
   const size_t smem = stem_fwd_smem(g);
   const long long cap = 2LL * sm_count;

@@ -354,6 +354,7 @@ void fill_params(const TcState* ts, const Geom& g, const Tiling& tl, TcParams* p
   p->kb_per_split = tl.KB;
   p->kw = g.kw; p->pad = g.pad; p->stride = g.stride; p->nstages = tl.nstages;
   p->cout = g.cout; p->ho = g.ho; p->wo = g.wo; p->G = g.G;
+  p->kstore = g.kstore;
   p->n_out = g.n_out;
   p->out = nullptr; p->dec = p->decl = p->nul = p->bias = nullptr;
   p->vs.sumsq = nullptr; p->vs.maxrho = nullptr; p->vs.count = nullptr; p->vs.cand = nullptr;

@@ -79,6 +79,7 @@ struct TcParams {
                                // memory from the fp32 values the first copy brought (tf32(v - trunc(v)))
   // problem
   int cout, ho, wo, G;
+  int kstore;                  // decoded rows k >= kstore of a group (noise vectors, Section 4.5) are neither computed nor stored
   long long n_out;
   // outputs / epilogue inputs
   float* out;                  // MODE_YBAR: ybar [G*E][ho][wo][cout]; MODE_DECODE: y [G*K][ho][wo][cout]
@@ -300,6 +301,7 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
       // would contribute.
 #pragma unroll
       for (int k = 0; k < K; ++k) {
+        if (k >= p.kstore) continue;
         float ck[K1];
 #pragma unroll
         for (int i = 0; i < K1; ++i) ck[i] = __ldg(p.dec + ((size_t)g * K + k) * K1 + i);
@@ -379,6 +381,7 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
       const float bias_co = (p.bias != nullptr && co_ok) ? __ldg(p.bias + co) : 0.f;
 #pragma unroll
       for (int k = 0; k < K; ++k) {
+        if (k >= p.kstore) continue;
         int cg = -1;
         float ch[K1], cl[K1];
 #pragma unroll

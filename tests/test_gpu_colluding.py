@@ -114,3 +114,48 @@ def test_weight_gradient_of_the_private_inputs(ctx, name, spec, K, M):
                                  spec.kh, spec.kw, spec.stride, spec.pad)
         total = part if total is None else total + part
     assert H.max_rel(got, total) < TOL_DECODED
+
+
+# also through the kernels that are not the tensor-core epilogue: fp32 SIMT (channels-first would do too), the
+# fp64 regime's fused pointwise kernel and its general path
+SKIP_CASES = CASES + [
+    ("pw_K2_M2_fp64_fused", spec_for("conv", 2, 2, cin=32, cout=48, h=6, w=6, kh=1, kw=1, pad=0, precision="fp64"), 2, 2),
+    ("conv_K2_M2_fp64", spec_for("conv", 2, 2, cin=8, cout=12, h=6, w=6, precision="fp64"), 2, 2),
+]
+
+
+@pytest.mark.parametrize("name,spec,K,M", SKIP_CASES, ids=[c[0] for c in SKIP_CASES])
+def test_outputs_of_the_noise_rows_are_not_stored_when_told_so(ctx, name, spec, K, M):
+    """DK_OPT_NOISE_ROWS = M - 1: the rows of y that would hold <W, r_m> stay as they were, the private rows
+    and the verdict are those of the default call (fused call, and dk_decode_verify on the same y_bar)."""
+    d = synth.draw_colluding(spec, K, M)
+    KL, E = spec.K, spec.K + 2
+    p = dk.problem_from_spec(spec, tol=H.TAU)
+    ctx.ensure_workspace(p)
+    W = H.weights_to_dev(d["W"], lay(spec))
+    x, r = H.acts_to_dev(d["x"], lay(spec)), H.acts_to_dev(d["r"], lay(spec))
+    v = dk.new_verdict()
+    y_all = H.empty_acts(spec.G * KL, spec, "out", lay(spec))
+    dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y_all, None, v)
+    want_v = dk.read_verdict(v)
+    xbar = H.acts_to_dev(O.encode(d["x"], d["r"], d["C"]).astype(np.float32), lay(spec))
+    ybar = H.empty_acts(spec.G * E, spec, "out", lay(spec))
+    dk.dk_linear_fwd(ctx, p, W, xbar, ybar)
+    try:
+        dk.dk_set_option(ctx, dk.DK_OPT_NOISE_ROWS, M - 1)
+        sentinel = -12345.0
+        for call in ("fused", "decode"):
+            y = H.empty_acts(spec.G * KL, spec, "out", lay(spec))
+            y.fill_(sentinel)
+            if call == "fused":
+                dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y, None, v)
+            else:
+                dk.dk_decode_verify(ctx, p, ybar, d["C"], None, y, v)
+            got_v = dk.read_verdict(v)
+            assert (got_v["ok"], got_v["n_flagged"], got_v["status"]) == (want_v["ok"], want_v["n_flagged"], 0)
+            yv, ya = y.reshape(spec.G, KL, -1), y_all.reshape(spec.G, KL, -1)
+            assert bool((yv[:, K:] == sentinel).all()), call
+            # (small problems meet by atomic additions in y_bar: equal up to that order)
+            assert float((yv[:, :K] - ya[:, :K]).abs().max()) <= 1e-4 * float(ya.abs().max()), call
+    finally:
+        dk.dk_set_option(ctx, dk.DK_OPT_NOISE_ROWS, 0)
