@@ -174,7 +174,8 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
   const int E = g.E;
   const int P = tile_pixels(g.K);
   // Box shape bw x bh x bg with bw*bh*bg = P (bw, bh powers of two): the one
-  // that covers the fewest out-of-range positions; ties go to wider rows.
+  // that covers the fewest out-of-range positions, weighted by what its
+  // epilogue and copies cost; ties go to wider rows.
   t->P = P;
   t->bw = t->bh = t->bg = 1;
   long long best = -1;
@@ -183,8 +184,12 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
       if (P % (bw * bh)) continue;
       const int bg = P / (bw * bh);
       if (bg > 256) continue;
-      const long long cost = (long long)((g.wo + bw - 1) / bw) * bw * ((g.ho + bh - 1) / bh) * bh *
-                             ((g.G + bg - 1) / bg) * bg;
+      long long cost = (long long)((g.wo + bw - 1) / bw) * bw * ((g.ho + bh - 1) / bh) * bh *
+                       ((g.G + bg - 1) / bg) * bg * 64;
+      // (measured on 28x28 and 14x14 images: a tile whose epilogue threads each span several groups runs ~30 %
+      // longer than one with 12 % of its positions out of range; per-encoding boxes cost a few per cent)
+      if (bw * bh < P / 2) cost += cost * 5 / 16;
+      else if (bg > 1) cost += cost / 32;
       if (best < 0 || cost < best || (cost == best && (bw > t->bw || (bw == t->bw && bh > t->bh)))) {
         best = cost; t->bw = bw; t->bh = bh; t->bg = bg;
       }

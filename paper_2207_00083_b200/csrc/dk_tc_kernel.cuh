@@ -225,18 +225,25 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
   // warps are few, so their speed depends on independent instructions from
   // different pixels being in flight together.  Offsets fit 32 bits (n_out
   // is checked on the host).
-  const bool one_group = p.bg == 1;
+  // The same walk serves a tile of several groups whose groups hold at least
+  // PH pixels each (S and PH are powers of two): this thread's PH pixels then
+  // lie in one group, `g1`.  A group past the last one leaves every pixel
+  // invalid; its coefficients are read from the last group and not used.
+  const bool one_group = S >= PH;
+  const int g1raw = gt * p.bg + ((half * PH) >> p.log2_S);
+  const bool g1_ok = g1raw < p.G;
+  const int g1 = g1_ok ? g1raw : p.G - 1;
   const int oh0 = ht * p.bh, ow0 = wt * p.bw;
   auto pixel = [&](int j, int& off) -> bool {      // one_group only
-    const int pix = half * PH + j;
+    const int pix = (half * PH + j) & (S - 1);
     const int oh = oh0 + (pix >> p.log2_bw), ow = ow0 + (pix & (p.bw - 1));
     off = (oh * p.wo + ow) * p.cout;
-    return oh < p.ho && ow < p.wo;
+    return oh < p.ho && ow < p.wo && g1_ok;
   };
 
   if (MODE == MODE_YBAR) {
     if (one_group) {
-      float* base = p.out + ((size_t)gt * E) * p.n_out + co;
+      float* base = p.out + ((size_t)g1 * E) * p.n_out + co;
 #pragma unroll
       for (int j = 0; j < PH; ++j) {
         int off;
@@ -280,7 +287,7 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
       }
     }
     if (one_group) {
-      const int g = gt;
+      const int g = g1;
       const float bias_co = (p.bias != nullptr && co_ok) ? __ldg(p.bias + co) : 0.f;
       // Offsets and validity of this thread's pixels, once; sums of pixels outside
       // the tensor (or of a channel past cout) are cleared so that the passes

@@ -56,6 +56,11 @@ def small_cases():
         ("pair_s2_cout256", tiny(cin=64, cout=256, h=14, w=14, stride=2, K=4, G=2)),
         # odd K keeps the single-CTA kernel even with many output channels
         ("single_K3_cout160", tiny(cin=16, cout=160, h=7, w=9, K=3, G=2)),
+        # forward tiles of two virtual batches, half a tile each (4x4 pixel boxes): an odd number of virtual
+        # batches leaves the last tile's second half empty; CTA pair and single CTA
+        ("two_groups_pair_oddG", tiny(cin=32, cout=256, h=4, w=4, K=4, G=5)),
+        ("two_groups_single_oddG", tiny(cin=16, cout=96, h=4, w=4, K=3, G=3)),
+        ("two_groups_12x12", tiny(cin=32, cout=136, h=12, w=12, K=4, G=3)),
         # weight-gradient N tiles: 3 taps x 64 with a partly filled slot (cin 48),
         # 2 taps x 128 (cin 96, odd tap count), 4 taps of a 2x2 filter
         ("wg_pack_cin48", tiny(cin=48, cout=64, h=10, w=10, K=4, G=2)),
