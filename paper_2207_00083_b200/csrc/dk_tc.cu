@@ -169,6 +169,10 @@ struct Tiling {
   size_t smem_bytes;
 };
 
+// Tiles whose activations arrive as one box over the encodings per TF32 term: those of one virtual batch, and
+// those of two batches of P/2 pixels (the box then spans both, see TcParams::gbox)
+bool onebox_tiles(const Tiling& t) { return t.bg == 1 || (t.bg == 2 && t.bw * t.bh * 2 == t.P); }
+
 template <int BK>
 bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
   const int E = g.E;
@@ -274,7 +278,7 @@ bool encode_fwd_maps(const TcState* ts, const Geom& g, const Tiling& tl, const f
     cuuint64_t str[4] = {(cuuint64_t)g.cin * 4, (cuuint64_t)g.cin * g.w * 4, (cuuint64_t)g.n_in * 4,
                          (cuuint64_t)g.n_in * g.E * 4};
     // (tiles of one virtual batch fetch all their encodings, or a CTA pair's half of them, as one box)
-    const cuuint32_t ebox = tl.bg == 1 ? (cuuint32_t)(tl.pair ? g.E / 2 : g.E) : 1u;
+    const cuuint32_t ebox = onebox_tiles(tl) ? (cuuint32_t)(tl.pair ? g.E / 2 : g.E) : 1u;
     cuuint32_t box[5] = {(cuuint32_t)BK, (cuuint32_t)(tl.bw * g.stride), (cuuint32_t)(tl.bh * g.stride), ebox,
                          (cuuint32_t)tl.bg};
     if (!encode_map(ts, mb_hi, xb_hi, 5, dims, str, box, BK * 4, g.stride) ||
@@ -352,7 +356,8 @@ void fill_params(const TcState* ts, const Geom& g, const Tiling& tl, TcParams* p
   p->nprod = g.nprod == 2 ? 2 : 3;
   p->lo_inkernel = 0;
   p->nstages_b = ts->opt->v[DK_OPT_TC_SPLIT_RING] ? tl.nstages_b : 0;
-  p->b_onebox = tl.bg == 1 ? 1 : 0;
+  p->b_onebox = onebox_tiles(tl) ? 1 : 0;
+  p->gbox = p->b_onebox && tl.bg == 2 ? 1 : 0;
   p->hmul = tl.mpack ? 2 : 1;
   ts->opt->v[DK_OPT_TEST_WITHHOLD] = -1;      // the hook serves one launch
   p->ksplit = 1;

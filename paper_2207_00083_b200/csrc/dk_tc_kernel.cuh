@@ -75,6 +75,9 @@ struct TcParams {
   int nprod;                   // 3: W_hi.x_hi + W_hi.x_lo + W_lo.x_hi; 2: W as one TF32 term, W_lo neither loaded nor used
   int b_onebox;                // 1 (tiles of one virtual batch, bg = 1): the encodings of a stage arrive as ONE box over the
                                // encoding dimension per TF32 term instead of one box per encoding
+  int gbox;                    // 1 (with b_onebox; tiles of two virtual batches of P/2 pixels): that box spans both
+                               // batches, so the tile's columns run batch-major (batch, encoding, pixel) within
+                               // each CTA's share instead of (encoding, batch, pixel)
   int lo_inkernel;             // 1: the activations' second TF32 term is not loaded: two warps derive it in shared
                                // memory from the fp32 values the first copy brought (tf32(v - trunc(v)))
   // problem
@@ -196,6 +199,14 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
   d |= (uint64_t)1 << 46;                             // descriptor version of this architecture
   d |= layout << 61;
   return d;
+}
+
+// First accumulator column of encoding e for the `half`-th P/2 pixels of a tile.  `share` = encodings whose
+// activations one CTA stages (all of them; half of them in a CTA pair).
+template <int P>
+__device__ __forceinline__ uint32_t tile_column(int gbox, int share, int e, int half) {
+  const int r = e / share, el = e - r * share;
+  return (uint32_t)(gbox ? (r * share * 2 + half * share + el) * (P / 2) : e * P + half * (P / 2));
 }
 
 // ---------------------------------------------------------------------------
@@ -764,7 +775,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
         const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
         if (!mbar_wait(tfull_bar + buf, aphase, abort_flag, p.spin_cap)) { alive = false; break; }
         tc_fence_after();
-        const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * PH);
+        const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16);
         constexpr int EB = 2;      // encodings per round trip to tensor memory
 #pragma unroll
         for (int e0 = 0; e0 < E; e0 += EB) {
@@ -772,8 +783,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
 #pragma unroll
           for (int de = 0; de < EB; ++de)
             if (e0 + de < E) {
+              const uint32_t col = tile_column<P>(p.gbox, E, e0 + de, half);
 #pragma unroll
-              for (int c = 0; c < PH; c += 8) tc_ld8(tbase + (uint32_t)((e0 + de) * P + c), &tmp[de][c]);
+              for (int c = 0; c < PH; c += 8) tc_ld8(tbase + col + (uint32_t)c, &tmp[de][c]);
             }
           tc_wait_ld();
 #pragma unroll

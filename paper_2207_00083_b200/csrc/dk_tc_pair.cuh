@@ -322,7 +322,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         const uint32_t buf = acc_it & 1u, aphase = (acc_it >> 1) & 1u;
         if (!mbar_wait(tfull_bar + buf, aphase, abort_flag, p.spin_cap)) { alive = false; break; }
         tc_fence_after();
-        const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * PH);
+        const uint32_t tbase = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16);
         constexpr int EB = 2;      // encodings per round trip to tensor memory
 #pragma unroll
         for (int e0 = 0; e0 < E; e0 += EB) {
@@ -330,8 +330,9 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
 #pragma unroll
           for (int de = 0; de < EB; ++de)
             if (e0 + de < E) {
+              const uint32_t col = tile_column<P>(p.gbox, EH, e0 + de, half);
 #pragma unroll
-              for (int c = 0; c < PH; c += 8) tc_ld8(tbase + (uint32_t)((e0 + de) * P + c), &tmp[de][c]);
+              for (int c = 0; c < PH; c += 8) tc_ld8(tbase + col + (uint32_t)c, &tmp[de][c]);
             }
           tc_wait_ld();
 #pragma unroll
