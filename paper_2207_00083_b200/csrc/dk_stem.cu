@@ -239,9 +239,12 @@ __global__ void __launch_bounds__(kThreads, 1) stem_wgrad_kernel(const StemWgPar
   constexpr int K1 = K + 1, CIN = 3;
   extern __shared__ float4 smem4[];
   float* Ds = reinterpret_cast<float*>(smem4);                 // [K1][32][64] mixed gradients of the row segment
-  float* Xs = Ds + (size_t)K1 * kTileW * 64;                   // [K1][3][PW][3] stored encodings under it
-  const int patch = kWgKH * p.PW * CIN;
-  float* cmix = Xs + (size_t)K1 * patch;                       // [K1][K]
+  // stored encodings under it, two buffers: [K1][3][PW][4] (a pixel's 3 channels in a 16-byte slot, so that the
+  // three taps of a filter row are three aligned 16-byte reads); the next tile's patch arrives by asynchronous
+  // copies while this tile is contracted
+  float* Xs0 = Ds + (size_t)K1 * kTileW * 64;
+  const int xbuf = K1 * kWgKH * p.PW * 4;                      // floats of one buffer
+  float* cmix = Xs0 + 2 * (size_t)xbuf;                        // [K1][K]
   const int tid = threadIdx.x, cog = tid & 15, stream = tid >> 4;
   const int cb = blockIdx.y * 64;
   const long long n_in = (long long)p.h * p.w * CIN, n_out = (long long)p.ho * p.wo * p.cout;
@@ -253,10 +256,9 @@ __global__ void __launch_bounds__(kThreads, 1) stem_wgrad_kernel(const StemWgPar
   // the gradients of a tile are fetched into registers while the previous tile is being contracted
   float4 dn[2][K];
   auto fetch = [&](long long t) {
-    const int tw = (int)(t % p.tiles_w);
-    const long long rest = t / p.tiles_w;
-    const int oy = (int)(rest % p.ho);
-    const int g = (int)(rest / p.ho);
+    const int ti = (int)(t < p.ntiles ? t : 0);
+    const int tw = ti % p.tiles_w, rest = ti / p.tiles_w;
+    const int oy = rest % p.ho, g = rest / p.ho;
 #pragma unroll
     for (int h2 = 0; h2 < 2; ++h2) {
       const int u4 = tid + h2 * kThreads;
@@ -270,14 +272,40 @@ __global__ void __launch_bounds__(kThreads, 1) stem_wgrad_kernel(const StemWgPar
                        : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   };
+  // asynchronous 4-byte copies of tile t's patch of the stored encodings 0..K into buffer `b` (zeros outside the image)
+  auto stage_patch = [&](long long t, int b) {
+    if (t < p.ntiles) {
+      const int ti = (int)t;                                   // (the host checked that the tile count fits 31 bits)
+      const int tw = ti % p.tiles_w, rest = ti / p.tiles_w;
+      const int oy = rest % p.ho, g = rest / p.ho;
+      const int iy0 = oy * p.stride - p.pad, ix0 = tw * kTileW * p.stride - p.pad;
+      float* xb = Xs0 + (size_t)b * xbuf;
+      // a patch row of one encoding is PW * 3 consecutive values of the image: one warp per row, no division by
+      // run-time values per element
+      const int roww = p.PW * CIN;
+      for (int row = tid >> 5; row < K1 * kWgKH; row += kThreads / 32) {
+        const int j = row / kWgKH, u = row - j * kWgKH;
+        const int iy = iy0 + u;
+        const bool row_in = iy >= 0 && iy < p.h;
+        const float* srow = p.xbar + ((size_t)g * p.xbar_rows + j) * n_in + ((long long)iy * p.w + ix0) * CIN;
+        float* drow = xb + (size_t)row * p.PW * 4;
+        for (int e = tid & 31; e < roww; e += 32) {
+          const int px = e / CIN, c = e - px * CIN;
+          const int ix = ix0 + px;
+          const bool in = row_in && ix >= 0 && ix < p.w;
+          const uint32_t dst = (uint32_t)__cvta_generic_to_shared(drow + px * 4 + c);
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(dst), "l"(in ? srow + e : p.xbar), "r"(in ? 4 : 0));
+        }
+      }
+    }
+    asm volatile("cp.async.commit_group;\n" ::);
+  };
   fetch(blockIdx.x);
+  stage_patch(blockIdx.x, 0);
+  int cur = 0;
 
-  for (long long t = blockIdx.x; t < p.ntiles; t += gridDim.x) {
-    const int tw = (int)(t % p.tiles_w);
-    const long long rest = t / p.tiles_w;
-    const int oy = (int)(rest % p.ho);
-    const int g = (int)(rest / p.ho);
-    const int ox0 = tw * kTileW;
+  for (long long t = blockIdx.x; t < p.ntiles; t += gridDim.x, cur ^= 1) {
+    const int g = (int)t / p.tiles_w / p.ho;
     __syncthreads();
     if (g != loaded_g) {
       for (int i = tid; i < K1 * K; i += kThreads) cmix[i] = __ldg(p.dmix + (size_t)g * K1 * K + i);
@@ -303,37 +331,34 @@ __global__ void __launch_bounds__(kThreads, 1) stem_wgrad_kernel(const StemWgPar
         *reinterpret_cast<float4*>(Ds + ((size_t)j * kTileW + px) * 64 + c4) = o;
       }
     }
-    // the stored encodings 0..K of the group under the segment
-    {
-      const int iy0 = oy * p.stride - p.pad, ix0 = ox0 * p.stride - p.pad;
-      for (int i = tid; i < K1 * patch; i += kThreads) {
-        const int j = i / patch, r = i - j * patch;
-        const int c = r % CIN, px = (r / CIN) % p.PW, u = r / (CIN * p.PW);
-        const int iy = iy0 + u, ix = ix0 + px;
-        const bool in = iy >= 0 && iy < p.h && ix >= 0 && ix < p.w;
-        Xs[i] = in ? __ldg(p.xbar + ((size_t)g * p.xbar_rows + j) * n_in + ((size_t)iy * p.w + ix) * CIN + c) : 0.f;
-      }
-    }
-    fetch(t + gridDim.x);            // in flight during the products below
+    stage_patch(t + gridDim.x, cur ^ 1);   // (that buffer's last readers passed the barrier above)
+    fetch(t + gridDim.x);                  // in flight during the products below
+    asm volatile("cp.async.wait_group 1;\n" ::: "memory");      // this tile's patch has landed (the next one may be in flight)
     __syncthreads();
+    const float* Xs = Xs0 + (size_t)cur * xbuf;
 #pragma unroll 1
     for (int pp = 0; pp < kTileW / 16; ++pp) {
       const int px = stream + 16 * pp;
-#pragma unroll 1
+      // (unrolled: the loads of the next encoding are issued under the products of this one)
+#pragma unroll
       for (int j = 0; j < K1; ++j) {
         const float4 d = *reinterpret_cast<const float4*>(Ds + ((size_t)j * kTileW + px) * 64 + cog * 4);
-        const float* xp = Xs + (size_t)j * patch + (size_t)px * p.stride * CIN;
+        const float4* xp = reinterpret_cast<const float4*>(Xs) + (size_t)j * kWgKH * p.PW + (size_t)px * p.stride;
 #pragma unroll
-        for (int u = 0; u < kWgKH; ++u)
+        for (int u = 0; u < kWgKH; ++u) {
+          const float4 x0 = xp[u * p.PW], x1 = xp[u * p.PW + 1], x2 = xp[u * p.PW + 2];
+          const float xv[kWgKWC] = {x0.x, x0.y, x0.z, x1.x, x1.y, x1.z, x2.x, x2.y, x2.z};
 #pragma unroll
           for (int vc = 0; vc < kWgKWC; ++vc) {
-            const float xv = xp[(size_t)u * p.PW * CIN + vc];
             float* a = acc[u * kWgKWC + vc];
-            a[0] = fmaf(xv, d.x, a[0]); a[1] = fmaf(xv, d.y, a[1]); a[2] = fmaf(xv, d.z, a[2]); a[3] = fmaf(xv, d.w, a[3]);
+            a[0] = fmaf(xv[vc], d.x, a[0]); a[1] = fmaf(xv[vc], d.y, a[1]);
+            a[2] = fmaf(xv[vc], d.z, a[2]); a[3] = fmaf(xv[vc], d.w, a[3]);
           }
+        }
       }
     }
   }
+  asm volatile("cp.async.wait_group 0;\n" ::: "memory");
   // the two streams of a warp meet by shuffle, the eight warps in shared memory, the CTAs in dW
   __syncthreads();
 #pragma unroll
@@ -364,7 +389,7 @@ size_t stem_wgrad_smem(const Geom& g) {
   size_t ds = (size_t)K1 * kTileW * 64;
   const size_t red = (size_t)(kThreads / 32) * 64 * kWgKC;
   if (ds < red) ds = red;
-  return (ds + (size_t)K1 * kWgKH * PW * 3 + (size_t)K1 * g.K + 4) * sizeof(float);
+  return (ds + 2 * (size_t)K1 * kWgKH * PW * 4 + (size_t)K1 * g.K + 4) * sizeof(float);
 }
 
 }  // namespace
@@ -417,6 +442,7 @@ namespace dk {
 bool stem_wgrad_fused_supported(const Geom& g, int smem_optin) {
   if (g.kind != DK_CONV2D || g.layout != DK_NHWC || g.precision != DK_TF32X3) return false;
   if (g.cin != 3 || g.kh != kWgKH || g.kw != 3 || (g.cout % 4) != 0) return false;
+  if ((long long)g.G * g.ho * ((g.wo + kTileW - 1) / kTileW) >= (1LL << 31)) return false;   // tile indices in 32 bits
   return stem_wgrad_smem(g) <= (size_t)smem_optin - 1024;
 }
 
