@@ -55,11 +55,11 @@ __global__ void __launch_bounds__(kThreads, 2) stem_fwd_kernel(const StemFwdPara
   int loaded_g = -1;
   bool w_loaded = false;
 
+  const int roww = p.PW * p.cin;     // a patch row is that many consecutive values of the image
   for (long long t = blockIdx.x; t < p.ntiles; t += gridDim.x) {
-    const int tw = (int)(t % p.tiles_w);
-    const long long rest = t / p.tiles_w;
-    const int oy = (int)(rest % p.ho);
-    const int g = (int)(rest / p.ho);
+    const int ti = (int)t;           // (the host checked that the tile count fits 31 bits)
+    const int tw = ti % p.tiles_w, rest = ti / p.tiles_w;
+    const int oy = rest % p.ho, g = rest / p.ho;
     const int ox0 = tw * kTileW;
     __syncthreads();                 // the previous tile's reads of Xs, Ws and the tables are done
     if (g != loaded_g) {
@@ -74,13 +74,15 @@ __global__ void __launch_bounds__(kThreads, 2) stem_fwd_kernel(const StemFwdPara
       const float* xg = p.x + (size_t)g * K * n_in;
       const float* rg = p.r + (size_t)g * n_in;
       const int iy0 = oy * p.stride - p.pad, ix0 = ox0 * p.stride - p.pad;
+      // (element e of a patch row lies in the image when e_lo <= e < e_hi: no division per element)
+      const int e_lo = max(0, -ix0) * p.cin, e_hi = min(p.PW, p.w - ix0) * p.cin;
       for (int i = tid; i < patch; i += kThreads) {
-        const int c = i % p.cin;
-        const int px = (i / p.cin) % p.PW, u = i / (p.cin * p.PW);
-        const int iy = iy0 + u, ix = ix0 + px;
+        int u = 0, e = i;
+        while (e >= roww) { e -= roww; ++u; }
+        const int iy = iy0 + u;
         float s[K1];
-        const bool in = iy >= 0 && iy < p.h && ix >= 0 && ix < p.w;
-        const long long off = ((long long)iy * p.w + ix) * p.cin + c;
+        const bool in = iy >= 0 && iy < p.h && e >= e_lo && e < e_hi;
+        const long long off = ((long long)iy * p.w + ix0) * p.cin + e;
 #pragma unroll
         for (int k = 0; k < K; ++k) s[k] = in ? __ldg(xg + (size_t)k * n_in + off) : 0.f;
         s[K] = in ? __ldg(rg + off) : 0.f;
@@ -113,21 +115,29 @@ __global__ void __launch_bounds__(kThreads, 2) stem_fwd_kernel(const StemFwdPara
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[e][j] = 0.f;
       {
-        int k = 0;
+        // one filter element: the K+2 encodings of this thread's pixel against its 8 channels
+        auto element = [&](const float* xrow, int vc, int k) {
+          float xe[EP];
+#pragma unroll
+          for (int q = 0; q < EP / 4; ++q)
+            *reinterpret_cast<float4*>(xe + 4 * q) = *reinterpret_cast<const float4*>(xrow + (size_t)vc * EP + 4 * q);
+          const float4 w0 = *reinterpret_cast<const float4*>(Ws + k * 64 + cog * 4);
+          const float4 w1 = *reinterpret_cast<const float4*>(Ws + k * 64 + 32 + cog * 4);
+          const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+          for (int e = 0; e < E; ++e)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[e][j] = fmaf(xe[e], wv[j], acc[e][j]);
+        };
+        const int rowk = p.kw * p.cin;
         for (int u = 0; u < p.kh; ++u) {
           const float* xrow = Xs + ((size_t)u * p.PW + (size_t)pl * p.stride) * p.cin * EP;
-          for (int vc = 0; vc < p.kw * p.cin; ++vc, ++k) {
-            float xe[EP];
+          if (rowk == 9) {             // 3 taps x 3 channels, the usual stem: straight-line code
 #pragma unroll
-            for (int q = 0; q < EP / 4; ++q)
-              *reinterpret_cast<float4*>(xe + 4 * q) = *reinterpret_cast<const float4*>(xrow + (size_t)vc * EP + 4 * q);
-            const float4 w0 = *reinterpret_cast<const float4*>(Ws + k * 64 + cog * 4);
-            const float4 w1 = *reinterpret_cast<const float4*>(Ws + k * 64 + 32 + cog * 4);
-            const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-#pragma unroll
-            for (int e = 0; e < E; ++e)
-#pragma unroll
-              for (int j = 0; j < 8; ++j) acc[e][j] = fmaf(xe[e], wv[j], acc[e][j]);
+            for (int vc = 0; vc < 9; ++vc) element(xrow, vc, u * 9 + vc);
+          } else {
+#pragma unroll 3
+            for (int vc = 0; vc < rowk; ++vc) element(xrow, vc, u * rowk + vc);
           }
         }
       }
@@ -146,6 +156,10 @@ __global__ void __launch_bounds__(kThreads, 2) stem_fwd_kernel(const StemFwdPara
       float sq[E], maxrho = 0.f;
 #pragma unroll
       for (int e = 0; e < E; ++e) sq[e] = 0.f;
+      const bool whole = co0 + 8 <= p.cout && (p.cout & 3) == 0;      // this thread's 8 channels as two 16-byte stores
+      float bj[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) bj[j] = (p.bias && co0 + j < p.cout) ? __ldg(p.bias + co0 + j) : 0.f;
       if (pix_ok) {
 #pragma unroll
         for (int k = 0; k < K; ++k) {
@@ -160,16 +174,13 @@ __global__ void __launch_bounds__(kThreads, 2) stem_fwd_kernel(const StemFwdPara
             for (int j = 0; j < 8; ++j) yv[j] = fmaf(c, acc[i][j], yv[j]);
           }
           float* dst = p.y + ((size_t)g * K + k) * n_out + obase + co0;
-          if (co0 + 8 <= p.cout && (p.cout & 3) == 0) {
-            float bj[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) bj[j] = p.bias ? __ldg(p.bias + co0 + j) : 0.f;
+          if (whole) {
             *reinterpret_cast<float4*>(dst) = make_float4(yv[0] + bj[0], yv[1] + bj[1], yv[2] + bj[2], yv[3] + bj[3]);
             *reinterpret_cast<float4*>(dst + 4) = make_float4(yv[4] + bj[4], yv[5] + bj[5], yv[6] + bj[6], yv[7] + bj[7]);
           } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-              if (co0 + j < p.cout) dst[j] = yv[j] + (p.bias ? __ldg(p.bias + co0 + j) : 0.f);
+              if (co0 + j < p.cout) dst[j] = yv[j] + bj[j];
           }
         }
 #pragma unroll
@@ -398,6 +409,7 @@ bool stem_fused_supported(const Geom& g, int smem_optin) {
   if (g.kind != DK_CONV2D || g.layout != DK_NHWC || g.precision != DK_TF32X3) return false;
   // (longer contractions, e.g. a 7x7 stem, measured faster on the tensor-core kernels through patch rows)
   if ((g.cin % 4) == 0 || g.cin > 4 || g.kc > 64) return false;
+  if ((long long)g.G * g.ho * ((g.wo + kTileW - 1) / kTileW) >= (1LL << 31)) return false;   // tile indices in 32 bits
   return stem_fwd_smem(g) <= (size_t)smem_optin / 2 - 1024;      // two CTAs per SM
 }
 
