@@ -184,10 +184,13 @@ bool plan_tiling(const Geom& g, int smem_optin, Tiling* t, bool pair = false) {
   t->bw = t->bh = t->bg = 1;
   long long best = -1;
   for (int bw = 1; bw <= P; bw *= 2)
-    for (int bh = 1; bw * bh <= P; bh *= 2) {
+    for (int bh = 1; bw * bh <= P; ++bh) {
       if (P % (bw * bh)) continue;
       const int bg = P / (bw * bh);
       if (bg > 256) continue;
+      // (a height that is no power of two, e.g. 16 x 3 of the 48 pixels at K = 2, only for boxes of one virtual
+      // batch: the epilogue's walk over several batches splits pixel indices with shifts and masks)
+      if ((bh & (bh - 1)) != 0 && bg != 1) continue;
       long long cost = (long long)((g.wo + bw - 1) / bw) * bw * ((g.ho + bh - 1) / bh) * bh *
                        ((g.G + bg - 1) / bg) * bg * 64;
       // (measured on 28x28 and 14x14 images: a tile whose epilogue threads each span several groups runs ~30 %

@@ -52,7 +52,7 @@ __host__ __device__ constexpr int tile_pixels(int K) {
 
 struct TcParams {
   // tiling
-  int bw, bh, bg;              // box shape of the P pixels (bw and bh are powers of two)
+  int bw, bh, bg;              // box shape of the P pixels (bw a power of two; bh too unless bg = 1)
   int log2_bw, log2_S;         // log2 of bw and of S = bw*bh
   int WT, HT, GT, MT;          // tiles along width, height, groups, cout
   int gt0;                     // first group tile of this launch (a call may be served by several launches, each
@@ -224,7 +224,8 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
   // position of this thread's j-th pixel; false when it lies outside the tensor
   auto locate = [&](int j, int& g, int& oh, int& ow) -> bool {
     const int pix = half * PH + j;
-    const int gl = pix >> p.log2_S, rem = pix & (S - 1);      // S and bw are powers of two
+    // (S and bw are powers of two; a box of one group may have any height)
+    const int gl = p.bg == 1 ? 0 : pix >> p.log2_S, rem = p.bg == 1 ? pix : pix & (S - 1);
     g = gt * p.bg + gl;
     oh = ht * p.bh + (rem >> p.log2_bw);
     ow = wt * p.bw + (rem & (p.bw - 1));
@@ -246,7 +247,7 @@ __device__ __forceinline__ void tile_epilogue(const TcParams& p, float (&acc)[K 
   const int g1 = g1_ok ? g1raw : p.G - 1;
   const int oh0 = ht * p.bh, ow0 = wt * p.bw;
   auto pixel = [&](int j, int& off) -> bool {      // one_group only
-    const int pix = (half * PH + j) & (S - 1);
+    const int pix = p.bg == 1 ? half * PH + j : (half * PH + j) & (S - 1);
     const int oh = oh0 + (pix >> p.log2_bw), ow = ow0 + (pix & (p.bw - 1));
     off = (oh * p.wo + ow) * p.cout;
     return oh < p.ho && ow < p.wo && g1_ok;
