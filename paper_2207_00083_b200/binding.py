@@ -23,7 +23,7 @@ DK_NHWC, DK_NCHW = 0, 1
 DK_PREC_DEFAULT, DK_TF32X3, DK_FP32_SIMT, DK_FP64_SIMT, DK_TF32X2_WUNSPLIT = 0, 1, 2, 3, 4
 (DK_OPT_TC_CHUNK, DK_OPT_WG_CHUNK, DK_OPT_TC_BK, DK_OPT_TC_PAIR, DK_OPT_WG_PACK, DK_OPT_WG_PAIR, DK_OPT_TC_STEM,
  DK_OPT_FIELD_PATH, DK_OPT_SPIN_LIMIT, DK_OPT_TEST_WITHHOLD, DK_OPT_XBAR_HI, DK_OPT_TC_MPACK,
- DK_OPT_SLABS, DK_OPT_SLABS_FORCE, DK_OPT_TC_CHUNK_ADAPT, DK_OPT_WG_PACE, DK_OPT_TC_LO_INKERNEL, DK_OPT_TC_SPLIT_RING, DK_OPT_NOISE_ROWS) = range(19)
+ DK_OPT_SLABS, DK_OPT_SLABS_FORCE, DK_OPT_TC_CHUNK_ADAPT, DK_OPT_WG_PACE, DK_OPT_TC_LO_INKERNEL, DK_OPT_TC_SPLIT_RING, DK_OPT_NOISE_ROWS, DK_OPT_TC_PACE) = range(20)
 DK_ERR_TIMEOUT = 6
 STATUS_NAMES = ["DK_OK", "DK_ERR_INVALID_ARG", "DK_ERR_SHAPE", "DK_ERR_SINGULAR", "DK_ERR_WORKSPACE",
                 "DK_ERR_CUDA", "DK_ERR_TIMEOUT", "DK_ERR_UNSUPPORTED"]

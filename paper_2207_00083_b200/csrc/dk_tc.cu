@@ -358,6 +358,7 @@ void fill_params(const TcState* ts, const Geom& g, const Tiling& tl, TcParams* p
   p->withhold = ts->opt->v[DK_OPT_TEST_WITHHOLD];
   p->nprod = g.nprod == 2 ? 2 : 3;
   p->lo_inkernel = 0;
+  p->pace = nullptr; p->pace_every = 1;
   p->nstages_b = ts->opt->v[DK_OPT_TC_SPLIT_RING] ? tl.nstages_b : 0;
   p->b_onebox = onebox_tiles(tl) ? 1 : 0;
   p->gbox = p->b_onebox && tl.bg == 2 ? 1 : 0;
@@ -617,6 +618,16 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
     prm.f_oh = (int)(pix / g.wo);
     prm.f_ow = (int)(pix - (long long)prm.f_oh * g.wo);
     prm.f_delta = fault->delta;
+  }
+  {
+    // pace (see tc_fwd_kernel): only when every CTA (pair) walks several meetings' worth of whole tiles
+    const int every = ctx->opt.v[DK_OPT_TC_PACE];
+    const int units = tl.pair ? ctx->sm_count / 2 : ctx->sm_count;
+    if (every > 0 && prm.ksplit == 1 && tl.ntiles / units >= 2 * every) {
+      prm.pace = reinterpret_cast<unsigned int*>(status_word) + 3;
+      prm.pace_every = every;
+      DK_CUDA_CHECK(cudaMemsetAsync(prm.pace, 0, sizeof(unsigned int), st));
+    }
   }
   return launch_bk<MODE_DECODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
 }

@@ -78,6 +78,8 @@ struct TcParams {
   int gbox;                    // 1 (with b_onebox; tiles of two virtual batches of P/2 pixels): that box spans both
                                // batches, so the tile's columns run batch-major (batch, encoding, pixel) within
                                // each CTA's share instead of (encoding, batch, pixel)
+  unsigned int* pace;          // nullable: counter (zero at launch) that keeps the CTAs' walks over the tiles together
+  int pace_every;              // tiles between two meetings on that counter
   int lo_inkernel;             // 1: the activations' second TF32 term is not loaded: two warps derive it in shared
                                // memory from the fp32 values the first copy brought (tf32(v - trunc(v)))
   // problem
@@ -610,7 +612,20 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
       int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool alive = true;
-      for (int w = blockIdx.x; alive && w < nwork; w += gridDim.x) {
+      int round = 0;
+      for (int w = blockIdx.x; alive && w < nwork; w += gridDim.x, ++round) {
+        // Pace.  The CTAs walk the tiles side by side (tile = CTA + round * grid), so the tiles in flight are
+        // neighbours in the image and share their halo rows through L2 -- while the CTAs stay together.  Over
+        // hundreds of rounds they drift apart and the halo is fetched from DRAM again (measured on a 224 x 224
+        // layer: 1.02 x the operands' bytes with 42 rounds, 1.55 x with 339).  So every pace_every rounds a CTA
+        // goes on only when all have issued the loads of the round before, or after a bounded wait: a hint,
+        // never a condition for progress.  (A CTA that waits here has a tile left, so every CTA had one in the
+        // round before and has counted.)
+        if (p.pace != nullptr && do_a && lane == 0 && round > 0 && round % p.pace_every == 0) {
+          const unsigned int target = (unsigned int)(round / p.pace_every) * gridDim.x;
+          for (int spin = 0; spin < 4096 && *reinterpret_cast<volatile unsigned int*>(p.pace) < target; ++spin)
+            __nanosleep(64);
+        }
         const int t = w / p.ksplit, ks = w - t * p.ksplit;
         const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
         const int mt = t % p.MT;
@@ -655,6 +670,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constan
           __syncwarp();
           if (++stage == nst) { stage = 0; phase ^= 1u; }
         }
+        // (the last round before a meeting: this CTA's loads of it are out)
+        if (p.pace != nullptr && alive && do_a && lane == 0 && (round + 1) % p.pace_every == 0) atomicAdd(p.pace, 1u);
       }
     }
   } else if (warp == 1) {

@@ -166,7 +166,14 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     int stage = 0, issued = 0;
     uint32_t phase = 0;
     bool alive = true;
-    for (int w = pair; alive && w < nwork; w += npairs) {
+    int round = 0;
+    for (int w = pair; alive && w < nwork; w += npairs, ++round) {
+      // pace (see tc_fwd_kernel): the leaders meet every pace_every rounds; the peer's copies follow within the ring
+      if (p.pace != nullptr && rank == 0 && lane == 0 && round > 0 && round % p.pace_every == 0) {
+        const unsigned int target = (unsigned int)(round / p.pace_every) * (unsigned int)npairs;
+        for (int spin = 0; spin < 4096 && *reinterpret_cast<volatile unsigned int*>(p.pace) < target; ++spin)
+          __nanosleep(64);
+      }
       const int t = w / p.ksplit, ks = w - t * p.ksplit;
       const int kb_lo = ks * p.kb_per_split, kb_hi = min(p.KB, kb_lo + p.kb_per_split);
       const int mt = t % p.MT;
@@ -220,6 +227,7 @@ tc_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         __syncwarp();
         if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
       }
+      if (p.pace != nullptr && alive && rank == 0 && lane == 0 && (round + 1) % p.pace_every == 0) atomicAdd(p.pace, 1u);
     }
   } else if (warp == 1 && rank == 0) {
     // ---------------- MMA issuer (leader only) ----------------
