@@ -60,7 +60,7 @@ FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
 # of these kernels (summaries with their commands under profiles/); the bench line divides by the launches per
 # step.  A workload or class that is absent here has not been captured since the kernels last changed and
 # reports null.
-NCU_TRAFFIC_BYTES_PER_STEP = {"vgg16_224": {"linear_fwd": 49712526336, "wgrad": 73664149504}}
+NCU_TRAFFIC_BYTES_PER_STEP = {"vgg16_224": {"linear_fwd": 45109597952, "wgrad": 69636159232}}
 
 
 def apply_options(dk, ctx, args):
