@@ -142,3 +142,33 @@ def test_library_picks_the_number_of_ranges_when_allowed(ctx):
             assert (got["ok"], got["status"]) == (1, 0)
             n = launches(ctx, "linear_fwd")
             assert (n >= 2) if (several and allowed > 1) else (n == 1)
+
+
+@pytest.mark.parametrize("name,cout", [("single_cta", 128), ("cta_pairs", 256)])
+def test_paced_forward_gives_the_same_bits(ctx, name, cout):
+    """DK_OPT_TC_PACE only decides when a CTA starts its next tiles: outputs, stored encodings and the verdict of a
+    call whose CTAs walk many rounds of tiles are the same with the meetings off, at every tile and at the default."""
+    spec = spec_of(cin=32, cout=cout, h=56, w=56, K=4, G=24)      # 2352 tiles (x 1 M tile): 16 or 32 rounds
+    d = synth.draw_layer(spec, with_delta=False)
+    lay = dk.DK_NHWC
+    p = dk.problem_from_spec(spec, tol=H.TAU)
+    ctx.ensure_workspace(p)
+    W, x, r = H.weights_to_dev(d["W"], lay), H.acts_to_dev(d["x"], lay), H.acts_to_dev(d["r"], lay)
+    v = dk.new_verdict()
+    out = {}
+    for every in (0, 1, 8):
+        dk.dk_set_option(ctx, dk.DK_OPT_TC_PACE, every)
+        y = H.empty_acts(spec.G * spec.K, spec, "out", lay)
+        xsave = H.empty_acts(spec.G * (spec.K + 2), spec, "in", lay)
+        y.fill_(float("nan")); xsave.fill_(float("nan"))
+        dk.dk_masked_linear(ctx, p, W, x, r, d["C"], None, y, xsave, v)
+        torch.cuda.synchronize()
+        got = dk.read_verdict(v)
+        assert (got["ok"], got["n_flagged"], got["status"]) == (1, 0, 0)
+        assert dk.dk_device_status(ctx) == 0
+        out[every] = (y, xsave)
+    for every in (1, 8):
+        assert torch.equal(out[0][0], out[every][0])
+        assert torch.equal(out[0][1], out[every][1])
+    plain = O.linear_plain(d["W"], d["x"][:4], spec.stride, spec.pad)
+    assert H.max_rel(H.acts_from_dev(out[8][0], lay)[:4], plain) < TOL_DECODED
