@@ -207,8 +207,9 @@ DK_API dk_status dk_destroy(dk_ctx* ctx);
  *                     stages do not fit); 0: one ring of whole stages.
  *   DK_OPT_NOISE_ROWS default 0.  n > 0: the last n of the K inputs of every virtual batch
  *                     are noise vectors (the relabelling of Section 4.5's colluding-
- *                     accelerator scheme onto these calls, see above): dk_masked_linear
- *                     and dk_decode_verify neither compute nor store the decoded rows
+ *                     accelerator scheme onto these calls, see above): dk_masked_linear,
+ *                     dk_decode_verify, dk_field_masked_linear and
+ *                     dk_field_decode_verify neither compute nor store the decoded rows
  *                     of those inputs (rows K-n .. K-1 of each group of y are left as
  *                     they were); encoding, the products and the integrity check are
  *                     unchanged.  At most K-1.

@@ -332,6 +332,7 @@ struct DecodeParams {
   int cout;
   double inv_scale;  // 2^-l
   int lbits;         // l
+  int kstore;        // decoded rows k >= kstore of a group (noise vectors, Section 4.5) are neither computed nor stored
   Modulus md;
 };
 
@@ -373,6 +374,7 @@ __global__ void __launch_bounds__(256) field_decode_verify_kernel(DecodeParams p
         }
 #pragma unroll
       for (int k = 0; k < K; ++k) {
+        if (k >= p.kstore) continue;
         u64 acc[VEC];
 #pragma unroll
         for (int v = 0; v < VEC; ++v) acc[v] = 0;
@@ -2109,6 +2111,11 @@ dk_status decode_verify_launch(dk_ctx* ctx, const Geom& g, int l, const u32* yba
   dp.cout = g.cout;
   dp.inv_scale = ldexp(1.0, -l);
   dp.lbits = l;
+  {      // Section 4.5 relabelling, as in the floating-point calls: at least one row stays
+    int n = ctx->opt.v[DK_OPT_NOISE_ROWS];
+    if (n > g.K - 1) n = g.K - 1;
+    dp.kstore = g.K - (n > 0 ? n : 0);
+  }
   dp.md = md;
   const bool vec4 = (g.n_out % 4) == 0 && aligned16(ybar) && aligned16(yq) && aligned16(y);
   ProfScope ps(ctx, DK_KERNEL_DECODE_VERIFY, 1, st);

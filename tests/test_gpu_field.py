@@ -405,3 +405,36 @@ def test_wgrad_on_maximal_residues(ctx, prime, pixels):
     d64 = np.full((1, spec.cout, 1, pixels), prime - 1, dtype=np.int64)
     x64 = np.full((1, spec.cin, 1, pixels), prime - 1, dtype=np.int64)
     assert F.field_wgrad_plain_at(d64, x64, 3, 5, 0, 0, prime, 1, 0) == want
+
+
+@pytest.mark.parametrize("name,spec,layout", [c for c in CASES if c[1].K >= 2][:4],
+                         ids=[c[0] for c in CASES if c[1].K >= 2][:4])
+def test_noise_rows_are_not_decoded_when_told_so(ctx, name, spec, layout):
+    """DK_OPT_NOISE_ROWS = n in the finite field (Section 4.5's relabelling): the last n decoded rows of every
+    virtual batch keep what the buffers held, the other rows and the verdict are those of the default call."""
+    d = synth.draw_field_layer(spec, P)
+    p = dk.problem_from_spec(spec, layout=layout)
+    ctx.ensure_workspace(p, field=True)
+    K, n = spec.K, spec.K - 1
+    C = u32(d["Cq"])
+    W_dev, x_dev = H.weights_to_dev(d["W"], layout), H.acts_to_dev(d["x"], layout)
+    rq_dev = res_acts_to_dev(d["rq"], layout)
+    v = dk.new_verdict()
+    y_all = H.empty_acts(spec.batch, spec, "out", layout)
+    yq_all = torch.empty(y_all.shape, dtype=torch.int32, device="cuda")
+    dk.dk_field_masked_linear(ctx, p, P, L, W_dev, x_dev, rq_dev, C, None, y_all, yq_all, None, v)
+    want_v = dk.read_verdict(v)
+    try:
+        dk.dk_set_option(ctx, dk.DK_OPT_NOISE_ROWS, n)
+        y = torch.full_like(y_all, -12345.0)
+        yq = torch.full_like(yq_all, -12345)
+        dk.dk_field_masked_linear(ctx, p, P, L, W_dev, x_dev, rq_dev, C, None, y, yq, None, v)
+        got_v = dk.read_verdict(v)
+        assert (got_v["ok"], got_v["n_flagged"], got_v["first_index"]) == \
+               (want_v["ok"], want_v["n_flagged"], want_v["first_index"])
+        for got, ref, sentinel in ((y, y_all, -12345.0), (yq, yq_all, -12345)):
+            a, b = got.reshape(spec.G, K, -1), ref.reshape(spec.G, K, -1)
+            assert bool((a[:, K - n:] == sentinel).all())
+            assert torch.equal(a[:, :K - n], b[:, :K - n])
+    finally:
+        dk.dk_set_option(ctx, dk.DK_OPT_NOISE_ROWS, 0)
