@@ -81,7 +81,6 @@ int resident_pairs(Kern kern, KernelCache& kc, int dev, size_t smem, int sm_coun
 }
 
 constexpr int kSwz128Atom32 = 1128;
-constexpr int kBK = 32;          // k-block: 32 fp32 = one 128-byte swizzle span per row
 
 // k-block of the forward kernel: 32 fp32 (128-byte rows, fewer and larger
 // stages) or 16 (64-byte rows, twice as many stages in the same shared memory)

@@ -537,7 +537,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
               const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
               const TcParams p) {
-  constexpr int E = K + 2, K1 = K + 1;
+  constexpr int E = K + 2;
   constexpr int P = tile_pixels(K), PH = P / 2;
   constexpr int BN = E * P;
   constexpr int SWZ = BK * 4;
