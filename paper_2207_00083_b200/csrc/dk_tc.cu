@@ -558,6 +558,19 @@ bool tc_fwd_group_tiles(const dk_ctx* ctx, const Geom& g, int* GT, int* bg, long
   return true;
 }
 
+// Pace of the forward kernels (see tc_fwd_kernel): only when every CTA (pair) walks several meetings' worth of whole
+// tiles.  The counter is the word three after the status word, cleared on the stream before the launch.
+static dk_status arm_pace(const dk_ctx* ctx, const Tiling& tl, TcParams* prm, int* status_word, cudaStream_t st) {
+  const int every = ctx->opt.v[DK_OPT_TC_PACE];
+  const int units = tl.pair ? ctx->sm_count / 2 : ctx->sm_count;
+  if (every > 0 && status_word != nullptr && prm->ksplit == 1 && tl.ntiles / units >= 2 * every) {
+    prm->pace = reinterpret_cast<unsigned int*>(status_word) + 3;
+    prm->pace_every = every;
+    DK_CUDA_CHECK(cudaMemsetAsync(prm->pace, 0, sizeof(unsigned int), st));
+  }
+  return DK_OK;
+}
+
 dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const float* w_lo, const float* xb_hi,
                         const float* xb_lo, float* ybar, int ksplit, bool ybar_cleared, int* status_word,
                         cudaStream_t st, int chunk_cap, bool lo_inkernel) {
@@ -577,6 +590,7 @@ dk_status tc_linear_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
   prm.lo_inkernel = lo_inkernel ? 1 : 0;
   if (lo_inkernel) prm.nstages_b = 0;      // (the converter warps work on the one-ring layout)
   prm.status = status_word;
+  if (dk_status e = arm_pace(ctx, tl, &prm, status_word, st)) return e;
   return launch_bk<MODE_YBAR>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
 }
 
@@ -618,16 +632,7 @@ dk_status tc_masked_fwd(dk_ctx* ctx, const Geom& g, const float* w_hi, const flo
     prm.f_ow = (int)(pix - (long long)prm.f_oh * g.wo);
     prm.f_delta = fault->delta;
   }
-  {
-    // pace (see tc_fwd_kernel): only when every CTA (pair) walks several meetings' worth of whole tiles
-    const int every = ctx->opt.v[DK_OPT_TC_PACE];
-    const int units = tl.pair ? ctx->sm_count / 2 : ctx->sm_count;
-    if (every > 0 && prm.ksplit == 1 && tl.ntiles / units >= 2 * every) {
-      prm.pace = reinterpret_cast<unsigned int*>(status_word) + 3;
-      prm.pace_every = every;
-      DK_CUDA_CHECK(cudaMemsetAsync(prm.pace, 0, sizeof(unsigned int), st));
-    }
-  }
+  if (dk_status e = arm_pace(ctx, tl, &prm, status_word, st)) return e;
   return launch_bk<MODE_DECODE>(ts, g, tl, w_hi, w_lo, xb_hi, xb_lo, prm, ctx->sm_count, st);
 }
 
